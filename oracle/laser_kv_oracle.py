@@ -1,0 +1,276 @@
+"""fp64 CPU oracle for LASER-KV's prefill-time token selection (TEST INFRASTRUCTURE ONLY).
+
+This module is the slow, plain statement of what the CUDA path must compute. It is used by
+the tests, by the smoke check and by the benchmark's CPU-baseline leg, and by nothing else:
+the product path never imports it, and it imports nothing from the product path. It shares
+no code, table or helper with the CUDA kernels.
+
+Everything is numpy in float64 on the exact values of the bf16 input bits (decoded here by
+this module's own routine). A library matmul serves as the inner-product step; there is no
+blocking, fusion or reordering beyond what the paper's definitions state.
+
+What each function follows:
+
+* ``budget``            - Appendix B, Eq. 1 (effective budget from block size and context length).
+* ``partition``         - Section 3.1 (protection divisor n: anchors B/n, local window B/n,
+                          recall budget B - 2B/n) and Algorithm 1 lines 4 and 7 (alpha split).
+* ``window_scores``     - Section 3.3 "Precision" and Algorithm 1 line 3, per layer and per
+                          KV head: attention probabilities of the window queries over the
+                          block's keys, summed over the queries of the KV head's GQA group.
+* ``simhash_buckets``   - Section 3.3 "Recall" and Algorithm 1's hash functions h_r, taken as
+                          K-bit SimHash (sign of Gaussian hyperplane projections) per table.
+* ``collision_counts``  - Algorithm 1 line 6: number of (query, table) pairs whose bucket equals
+                          the key's bucket (S_lsh is this count divided by R * number of queries).
+* ``topk_lower_index``  - the TopK of Algorithm 1 lines 4 and 7, ties to the lower index.
+* ``select_indices``    - Algorithm 1 lines 3-8 on the candidate set left by Section 3.1.
+* ``select_block`` / ``AppendOnlyCache`` - Section 3 (only selected tokens are kept) and the
+                          introduction's append-only accumulative memory.
+
+Readings taken where the paper is silent (rounding of B/n and alpha*B_long, per-block anchors,
+softmax over the block's own keys, bit = [projection >= 0], tie rule) are listed in the design
+notes of the repository and restated at each function.
+
+Parity status: budget/partition, softmax scores, SimHash bits, collision counts, top-k and
+append are each pinned by closed forms, hand cases, invariants or brute force in the CPU test
+suite. The numeric scores and chosen index sets on realistic data have no printed example in
+the paper ("parity unpinned by a worked example"); they are pinned only through those
+properties.
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass, field
+
+import numpy as np
+
+__all__ = [
+    "bf16_bits_to_f64", "budget", "partition", "window_scores", "simhash_projections",
+    "simhash_buckets", "collision_counts", "topk_lower_index", "select_indices",
+    "select_block", "AppendOnlyCache", "BlockResult",
+]
+
+
+# ----------------------------------------------------------------------------------------------
+# input decoding
+# ----------------------------------------------------------------------------------------------
+def bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:
+    """Exact value of bfloat16 bit patterns (uint16) as float64.
+
+    A bfloat16 is the upper half of an IEEE binary32, so widening is exact.
+    """
+    b = np.ascontiguousarray(bits, dtype=np.uint16)
+    f32 = (b.astype(np.uint32) << np.uint32(16)).view(np.float32)
+    return f32.astype(np.float64)
+
+
+# ----------------------------------------------------------------------------------------------
+# budget arithmetic
+# ----------------------------------------------------------------------------------------------
+def budget(context_len: int, block_size: int, ratio: float = 0.25) -> int:
+    """Eq. 1 (Appendix B): B = floor(2 r S_block L / (S_block + L)), in IEEE double."""
+    if context_len <= 0 or block_size <= 0 or not (ratio > 0.0):
+        raise ValueError("context_len, block_size and ratio must be positive")
+    num = 2.0 * float(ratio) * float(block_size) * float(context_len)
+    return int(math.floor(num / (float(block_size) + float(context_len))))
+
+
+def partition(B: int, n: int, alpha: float = 0.75):
+    """Section 3.1 + Algorithm 1 lines 4/7.
+
+    Returns (anchors, local, B_long, k_exact, k_lsh) with
+      anchors = local = floor(B / n)      (the syntactic set 2B/n, each half rounded down)
+      B_long  = B - 2*floor(B/n)          (recall budget; absorbs the rounding remainder so the
+                                           keep count is exactly B)
+      k_exact = floor(alpha * B_long)     (IEEE double product, then floor)
+      k_lsh   = B_long - k_exact
+    n = 2 gives B_long = 0 (only anchors and the local window are kept).
+    """
+    if B < 0 or n < 2 or not (0.0 <= alpha <= 1.0):
+        raise ValueError("need B >= 0, n >= 2, 0 <= alpha <= 1")
+    a = B // n
+    b_long = B - 2 * a
+    k_e = int(math.floor(float(alpha) * float(b_long)))
+    k_e = max(0, min(k_e, b_long))
+    return a, a, b_long, k_e, b_long - k_e
+
+
+# ----------------------------------------------------------------------------------------------
+# step 1: observation-window attention scores (Section 3.3 "Precision", Algorithm 1 line 3)
+# ----------------------------------------------------------------------------------------------
+def window_scores(q_bits: np.ndarray, k_bits: np.ndarray, scale: float | None = None) -> np.ndarray:
+    """S_exact[j] = sum over the group's window queries of softmax_j(<q, k_j> * scale).
+
+    q_bits: uint16 [n_queries, d]  - every window query of every query head in the KV head's
+                                     GQA group (G*W rows).
+    k_bits: uint16 [S, d]          - the block's keys for this KV head.
+    The softmax is over all S keys of the block (no causal mask, no pooling); scale defaults
+    to 1/sqrt(d). Returns float64 [S]; each query contributes a row that sums to 1.
+    """
+    q = bf16_bits_to_f64(q_bits)
+    k = bf16_bits_to_f64(k_bits)
+    d = k.shape[1]
+    if scale is None:
+        scale = 1.0 / math.sqrt(d)
+    s = (q @ k.T) * float(scale)                      # [n_queries, S] logits
+    s = s - s.max(axis=1, keepdims=True)
+    p = np.exp(s)
+    p = p / p.sum(axis=1, keepdims=True)              # attention probabilities per query
+    return p.sum(axis=0)
+
+
+# ----------------------------------------------------------------------------------------------
+# step 2: SimHash signatures and collision counts (Section 3.3 "Recall", Algorithm 1 line 6)
+# ----------------------------------------------------------------------------------------------
+def simhash_projections(x_bits: np.ndarray, p_bits: np.ndarray) -> np.ndarray:
+    """<p_m, x> for every vector x and every hyperplane p_m, float64 [N, L*K]."""
+    return bf16_bits_to_f64(x_bits) @ bf16_bits_to_f64(p_bits).T
+
+
+def simhash_buckets(x_bits: np.ndarray, p_bits: np.ndarray, n_bits: int, n_tables: int):
+    """K-bit SimHash bucket of every vector in every table.
+
+    Hyperplane m = r*K + b is bit b of table r; bit = 1 iff the projection is >= 0; the bucket
+    id is sum_b bit_b * 2**b. Returns (buckets int64 [N, L], min_abs float64 [N, L]) where
+    min_abs is the smallest |projection| among the table's K bits (used by comparisons that
+    exempt signs decided by a projection smaller than 1e-6 in magnitude).
+    """
+    proj = simhash_projections(x_bits, p_bits)
+    n = proj.shape[0]
+    if proj.shape[1] != n_bits * n_tables:
+        raise ValueError("hyperplane count must be n_bits * n_tables")
+    proj = proj.reshape(n, n_tables, n_bits)
+    bits = (proj >= 0.0).astype(np.int64)
+    weights = (1 << np.arange(n_bits, dtype=np.int64))
+    return (bits * weights).sum(axis=2), np.abs(proj).min(axis=2)
+
+
+def collision_counts(q_buckets: np.ndarray, k_buckets: np.ndarray) -> np.ndarray:
+    """count[j] = sum over queries and tables of 1[h_r(q) = h_r(k_j)]  (Algorithm 1 line 6,
+    before the division by R and by the number of queries).
+
+    q_buckets int [n_queries, L], k_buckets int [S, L] -> int64 [S]. Written as the plain loop
+    over queries (each step compares one query's L buckets with every key's).
+    """
+    q_buckets = np.asarray(q_buckets)
+    k_buckets = np.asarray(k_buckets)
+    counts = np.zeros(k_buckets.shape[0], dtype=np.int64)
+    for qi in range(q_buckets.shape[0]):
+        counts += (k_buckets == q_buckets[qi][None, :]).sum(axis=1)
+    return counts
+
+
+# ----------------------------------------------------------------------------------------------
+# step 3: two-stage top-k (Algorithm 1 lines 4-8)
+# ----------------------------------------------------------------------------------------------
+def topk_lower_index(candidates: np.ndarray, score: np.ndarray, k: int) -> np.ndarray:
+    """The k candidates with the largest score; among equal scores the lower index wins.
+
+    candidates: ascending int array of indices into ``score``. Returns the picks in ascending
+    index order. Implemented as a full stable sort by descending score.
+    """
+    candidates = np.asarray(candidates, dtype=np.int64)
+    if k <= 0 or candidates.size == 0:
+        return np.zeros(0, dtype=np.int64)
+    k = min(k, candidates.size)
+    vals = np.asarray(score)[candidates]
+    order = np.argsort(-vals, kind="stable")          # stable: ties keep ascending index order
+    return np.sort(candidates[order[:k]])
+
+
+def select_indices(s_exact: np.ndarray, counts: np.ndarray, S: int, anchors: int,
+                   k_exact: int, k_lsh: int):
+    """Algorithm 1 on the candidate set C = [anchors, S - anchors).
+
+    Returns (K_exact, K_lsh, idx): the exact-stage picks, the LSH-stage picks from the residual
+    C \\ K_exact, and the kept indices of the block in ascending order: anchors [0, a), the
+    picks, and the local window [S - a, S).
+    """
+    cand = np.arange(anchors, S - anchors, dtype=np.int64)
+    k_ex = topk_lower_index(cand, s_exact, k_exact)
+    residual = np.setdiff1d(cand, k_ex, assume_unique=True)
+    k_ls = topk_lower_index(residual, counts, k_lsh)
+    idx = np.concatenate([np.arange(0, anchors, dtype=np.int64), k_ex, k_ls,
+                          np.arange(S - anchors, S, dtype=np.int64)])
+    return k_ex, k_ls, np.sort(idx)
+
+
+# ----------------------------------------------------------------------------------------------
+# the whole per-block path for one (layer, sequence)
+# ----------------------------------------------------------------------------------------------
+@dataclass
+class BlockResult:
+    s_exact: np.ndarray          # float64 [H_kv, S]
+    counts: np.ndarray           # int64   [H_kv, S]
+    key_buckets: np.ndarray      # int64   [H_kv, S, L]
+    key_min_abs: np.ndarray      # float64 [H_kv, S, L]
+    query_buckets: np.ndarray    # int64   [H_kv, G*W, L]
+    query_min_abs: np.ndarray    # float64 [H_kv, G*W, L]
+    k_exact: list                # per KV head: ascending picks of the exact stage
+    k_lsh: list                  # per KV head: ascending picks of the LSH stage
+    idx: np.ndarray              # int64   [H_kv, B] kept block-local indices, ascending
+
+
+def select_block(k_bits: np.ndarray, q_bits: np.ndarray, p_bits: np.ndarray, *, n_bits: int,
+                 n_tables: int, B: int, n: int, alpha: float = 0.75,
+                 scale: float | None = None) -> BlockResult:
+    """Steps 1-3 for one block of one (layer, sequence).
+
+    k_bits uint16 [H_kv, S, d]; q_bits uint16 [H_q, W, d] (query head h*G+g belongs to KV head
+    h); p_bits uint16 [L*K, d]. Each KV head selects independently.
+    """
+    h_kv, S, d = k_bits.shape
+    h_q, W, _ = q_bits.shape
+    if h_q % h_kv:
+        raise ValueError("n_q_heads must be a multiple of n_kv_heads")
+    G = h_q // h_kv
+    a, _, _b_long, k_e, k_l = partition(B, n, alpha)
+    if 2 * a > S or B > S:
+        raise ValueError("budget does not fit the block")
+    out = BlockResult(np.zeros((h_kv, S)), np.zeros((h_kv, S), np.int64),
+                      np.zeros((h_kv, S, n_tables), np.int64), np.zeros((h_kv, S, n_tables)),
+                      np.zeros((h_kv, G * W, n_tables), np.int64),
+                      np.zeros((h_kv, G * W, n_tables)), [], [], np.zeros((h_kv, B), np.int64))
+    for h in range(h_kv):
+        qg = q_bits[h * G:(h + 1) * G].reshape(G * W, d)
+        out.s_exact[h] = window_scores(qg, k_bits[h], scale)
+        out.key_buckets[h], out.key_min_abs[h] = simhash_buckets(k_bits[h], p_bits, n_bits, n_tables)
+        out.query_buckets[h], out.query_min_abs[h] = simhash_buckets(qg, p_bits, n_bits, n_tables)
+        out.counts[h] = collision_counts(out.query_buckets[h], out.key_buckets[h])
+        k_ex, k_ls, idx = select_indices(out.s_exact[h], out.counts[h], S, a, k_e, k_l)
+        out.k_exact.append(k_ex)
+        out.k_lsh.append(k_ls)
+        out.idx[h] = idx
+    return out
+
+
+@dataclass
+class AppendOnlyCache:
+    """Accumulative cache of one (layer, sequence): entries are only ever appended.
+
+    K, V hold raw bf16 bit patterns [H_kv, capacity, d]; pos holds absolute token positions
+    [H_kv, capacity]; length is the same for every KV head (B per block).
+    """
+    n_kv_heads: int
+    head_dim: int
+    capacity: int
+    K: np.ndarray = field(init=False)
+    V: np.ndarray = field(init=False)
+    pos: np.ndarray = field(init=False)
+    length: int = 0
+
+    def __post_init__(self):
+        self.K = np.zeros((self.n_kv_heads, self.capacity, self.head_dim), np.uint16)
+        self.V = np.zeros((self.n_kv_heads, self.capacity, self.head_dim), np.uint16)
+        self.pos = np.full((self.n_kv_heads, self.capacity), -1, np.int32)
+
+    def append(self, k_bits: np.ndarray, v_bits: np.ndarray, idx: np.ndarray, block_start: int):
+        """Copy rows idx[h] of the block into [length, length + B) and advance length by B."""
+        B = idx.shape[1]
+        if self.length + B > self.capacity:
+            raise ValueError("cache capacity exceeded")
+        for h in range(self.n_kv_heads):
+            sl = slice(self.length, self.length + B)
+            self.K[h, sl] = k_bits[h, idx[h]]
+            self.V[h, sl] = v_bits[h, idx[h]]
+            self.pos[h, sl] = (block_start + idx[h]).astype(np.int32)
+        self.length += B
