@@ -1,0 +1,203 @@
+/*
+ * laser_kv.h - C ABI of the B200 (sm_100a) implementation of LASER-KV's prefill-time token
+ * selection: for every block of a long context, score the block's keys against the
+ * observation-window queries, hash keys and queries with SimHash and count collisions, run the
+ * paper's two-stage Exact-LSH top-k per KV head with the keep count fixed by the protection
+ * divisor n, and append the selected K/V rows to an append-only per-layer cache.
+ *
+ * Conventions for every entry point
+ *   - Returns a laser_kv_status_t (0 = success) unless stated otherwise; never throws or aborts.
+ *   - "dev" pointers are CUDA device pointers on the handle's device; "host" pointers are
+ *     ordinary host memory. All tensors are bfloat16 bit patterns (uint16) unless stated.
+ *   - The caller owns every device buffer (inputs, hyperplanes, cache, workspace). The library
+ *     owns only the host-side handle. No entry point in this header's main section allocates
+ *     device memory.
+ *   - Device pointers must be 16-byte aligned, strides multiples of 8 elements
+ *     (LASER_KV_ERR_ALIGNMENT otherwise).
+ *   - Kernel launches are asynchronous on the caller's stream; nothing is copied back to the
+ *     host unless the entry point says so.
+ *   - There is no CPU fallback: without a CUDA device laser_kv_init fails with LASER_KV_ERR_CUDA.
+ */
+#ifndef LASER_KV_H_
+#define LASER_KV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct laser_kv_ctx* laser_kv_handle_t;
+
+typedef enum {
+  LASER_KV_OK = 0,
+  LASER_KV_ERR_INVALID_ARG = 1,   /* null pointer, out-of-range value, inconsistent config    */
+  LASER_KV_ERR_UNSUPPORTED = 2,   /* valid by the paper but outside what the kernels handle   */
+  LASER_KV_ERR_CAPACITY = 3,      /* cache or workspace too small; nothing was written        */
+  LASER_KV_ERR_ALIGNMENT = 4,     /* pointer or stride alignment                              */
+  LASER_KV_ERR_CUDA = 5,          /* a CUDA runtime/driver call failed (see last_error)       */
+  LASER_KV_ERR_TIMEOUT = 6,       /* a bounded device-side wait gave up (status word)         */
+  LASER_KV_ERR_STATE = 7          /* call sequence error (e.g. debug view before any call)    */
+} laser_kv_status_t;
+
+/* One configuration per handle. Zero-initialise, then fill. */
+typedef struct {
+  int32_t n_layers;            /* independent per-layer caches                                   */
+  int32_t batch;               /* independent sequences processed together by each call          */
+  int32_t n_q_heads;           /* H_q                                                            */
+  int32_t n_kv_heads;          /* H_kv; H_q % H_kv == 0; G = H_q / H_kv (GQA group)              */
+  int32_t head_dim;            /* d; must be 128                                                 */
+  int32_t block_size;          /* S: tokens per block (Section 3.2); multiple of 8               */
+  int32_t window;              /* W: observation-window queries per query head                   */
+  int32_t max_blocks;          /* cache capacity per (layer, sequence, KV head) = max_blocks * B */
+  int32_t max_blocks_per_call; /* upper bound on n_blocks of one select call (sizes workspace)   */
+  int32_t lsh_bits;            /* K: sign bits per SimHash table, 1..12                          */
+  int32_t lsh_tables;          /* L: number of tables (the paper's R hash rounds)                */
+  int32_t protection_divisor;  /* n >= 2 (Section 3.1)                                           */
+  int32_t budget_per_block;    /* B; 0 => Eq. 1 from ratio, block_size and context_len           */
+  int32_t debug;               /* nonzero: also keep per-key bucket ids for laser_kv_debug_view  */
+  int64_t context_len;         /* L of Eq. 1 (only read when budget_per_block == 0)              */
+  double  ratio;               /* r of Eq. 1; 0 => 0.25                                          */
+  double  alpha;               /* exact share of the recall budget; negative => 0.75             */
+  float   softmax_scale;       /* 0 => 1/sqrt(head_dim)                                          */
+  int32_t device;              /* CUDA device ordinal                                            */
+} laser_kv_config_t;
+
+/* Views returned by laser_kv_cache_view: entries [0, len) of every (sequence, KV head) are
+ * final and never change again (append-only memory, Sections 1 and 3). Strides in elements. */
+typedef struct {
+  void*    K;                  /* dev bf16 [batch][H_kv][cap][d]                                 */
+  void*    V;                  /* dev bf16 [batch][H_kv][cap][d]                                 */
+  int32_t* pos;                /* dev int32 [batch][H_kv][cap]: absolute token positions         */
+  int64_t  len;                /* entries valid per (sequence, KV head); the same for all        */
+  int64_t  cap;                /* capacity per (sequence, KV head)                               */
+  int64_t  kv_strides[3];      /* batch, head, entry strides of K and V (last dim contiguous)    */
+  int64_t  pos_strides[2];     /* batch, head strides of pos                                     */
+} laser_kv_view_t;
+
+/* Intermediate results of the most recent select call (pointers into the workspace, valid
+ * until the next select call). nb = that call's n_blocks; GW = G*W. */
+typedef struct {
+  const float*    s_exact;       /* dev fp32  [batch][H_kv][nb][S]   summed window attention     */
+  const uint32_t* counts;        /* dev u32   [batch][H_kv][nb][S]   collision counts            */
+  const float*    lse2;          /* dev fp32  [batch][H_kv][nb][GW]  log2-sum-exp2 per query     */
+  const uint16_t* query_buckets; /* dev u16   [batch][H_kv][GW][L]                               */
+  const uint16_t* key_buckets;   /* dev u16   [batch][H_kv][nb][S][L]; NULL unless config.debug  */
+  const uint16_t* hist;          /* dev u16   [batch][H_kv][L][2^K]  query-bucket histogram      */
+  const int32_t*  idx;           /* dev int32 [batch][H_kv][nb][B]   kept block-local indices    */
+  int32_t n_blocks, batch, n_kv_heads, block_size, budget, gw, lsh_tables, lsh_bits;
+  int32_t n_sign_fixups;         /* host: near-zero projections recomputed exactly (last poll)   */
+} laser_kv_debug_t;
+
+/* Appendix B, Eq. 1: B = floor(2 r S_block L / (S_block + L)) evaluated in IEEE double.
+ * Returns B, or -1 for non-positive arguments. Host only. */
+int32_t laser_kv_budget(int64_t context_len, int32_t block_size, double ratio);
+
+/* Section 3.1 and Algorithm 1 lines 4/7: anchors = local = floor(B/n); recall budget
+ * B_long = B - 2*floor(B/n); k_exact = floor(alpha * B_long) (double); k_lsh = B_long - k_exact.
+ * Any output pointer may be NULL. n < 2, B < 0 or alpha outside [0,1] => INVALID_ARG. Host only. */
+laser_kv_status_t laser_kv_partition(int32_t B, int32_t n, double alpha, int32_t* anchors,
+                                     int32_t* local, int32_t* k_exact, int32_t* k_lsh);
+
+/* Bytes the caller must provide for the cache and the workspace of a configuration.
+ * Host only; validates the configuration. */
+laser_kv_status_t laser_kv_query_sizes(const laser_kv_config_t* cfg, size_t* cache_bytes,
+                                       size_t* workspace_bytes);
+
+/* Creates a handle. hyperplanes: dev bf16 [L*K][d], row r*K + b = bit b of table r (Section 3.3,
+ * the hash functions h_r taken as K-bit SimHash); read by every later call, owned by the caller.
+ * cache_mem / workspace: dev buffers of at least the sizes laser_kv_query_sizes reports, 256-byte
+ * aligned, owned by the caller and used until laser_kv_destroy. The cache need not be cleared. */
+laser_kv_status_t laser_kv_init(const laser_kv_config_t* cfg, const void* hyperplanes,
+                                void* cache_mem, size_t cache_bytes, void* workspace,
+                                size_t workspace_bytes, laser_kv_handle_t* out);
+
+/* The hot path (Algorithm 1 on each block, then append): processes n_blocks consecutive blocks
+ * of one layer for all `batch` sequences.
+ *   K_blk, V_blk : dev bf16 [batch][H_kv][n_blocks*S][d] addressed through kv_strides =
+ *                  {batch, head, token} strides in elements (last dim contiguous); block i of
+ *                  this call occupies tokens [i*S, (i+1)*S).
+ *   Q_win        : dev bf16 [batch][H_q][W][d] through q_strides = {batch, head, query}; the
+ *                  same window scores every block of the call; query head h*G+g belongs to KV
+ *                  head h.
+ * Per block and KV head it keeps exactly B tokens: the first and last floor(B/n) of the block,
+ * the k_exact candidates with the largest summed attention probability, and the k_lsh remaining
+ * candidates with the most SimHash collisions (ties: lower index). Rows are appended in
+ * ascending position at [len, len + n_blocks*B); len advances on the host. The blocks' absolute
+ * positions continue from the blocks already appended to this layer.
+ * Errors: CAPACITY if the cache cannot take n_blocks more blocks or n_blocks exceeds
+ * max_blocks_per_call (nothing is launched). */
+laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, const void* K_blk,
+                                        const void* V_blk, const void* Q_win,
+                                        const int64_t kv_strides[3], const int64_t q_strides[3],
+                                        int32_t n_blocks, void* stream);
+
+/* Same path driven from HOST memory: copies the (contiguous) host tensors K_host, V_host
+ * [batch][H_kv][n_blocks*S][d] and Q_host [batch][H_q][W][d] into the caller's device staging
+ * buffers K_stage, V_stage, Q_stage (same shapes), runs laser_kv_select_block on them, and
+ * copies the appended positions (int32 [batch][H_kv][n_blocks*B]) to pos_out_host. All copies
+ * are asynchronous on `stream` (pin the host buffers for overlap); the call does not
+ * synchronise. pos_out_host may be NULL. */
+laser_kv_status_t laser_kv_select_block_host(laser_kv_handle_t h, int32_t layer,
+                                             const void* K_host, const void* V_host,
+                                             const void* Q_host, void* K_stage, void* V_stage,
+                                             void* Q_stage, int32_t n_blocks,
+                                             int32_t* pos_out_host, void* stream);
+
+/* Current view of one layer's cache. Host only (no synchronisation: pending kernels on the
+ * caller's stream may still be writing entries counted in len). */
+laser_kv_status_t laser_kv_cache_view(laser_kv_handle_t h, int32_t layer, laser_kv_view_t* out);
+
+/* Pointers to the last call's intermediates; STATE before the first select call. */
+laser_kv_status_t laser_kv_debug_view(laser_kv_handle_t h, laser_kv_debug_t* out);
+
+/* Synchronises `stream`, reads the device status word and returns OK or the first error a
+ * kernel recorded (TIMEOUT for a bounded wait that gave up, CAPACITY if the exact-sign
+ * recompute list overflowed). Clears the word. */
+laser_kv_status_t laser_kv_poll_status(laser_kv_handle_t h, void* stream);
+
+/* Forgets the contents of one layer's cache (layer = -1: all layers). Host only. */
+laser_kv_status_t laser_kv_reset(laser_kv_handle_t h, int32_t layer);
+
+void laser_kv_destroy(laser_kv_handle_t h);
+
+const char* laser_kv_status_string(laser_kv_status_t s);
+
+/* Text of the most recent error on this handle ("" if none). NULL handle: the most recent
+ * error of a call that had no handle (init, query_sizes, step entry points). */
+const char* laser_kv_last_error(laser_kv_handle_t h);
+
+/* Number of this library's kernels launched by the calling process so far (all handles). */
+int64_t laser_kv_launch_count(void);
+
+/* ---- step-level entry points (same kernels as the hot path, caller-fed inputs) ------------- */
+
+/* Algorithm 1 lines 4-8 on given scores: for each of n_segments independent segments of S
+ * tokens, pick k_exact of the candidates [anchors, S - anchors) by s_exact (fp32, larger first),
+ * then k_lsh of the remaining candidates by counts (u32, larger first), ties to the lower index,
+ * and write the kept indices [0, anchors) + picks + [S - anchors, S) in ascending order.
+ *   s_exact dev fp32 [n_segments][S]; counts dev u32 [n_segments][S];
+ *   idx_out dev int32 [n_segments][2*anchors + k_exact + k_lsh].
+ * Needs 2*anchors + k_exact + k_lsh <= S. */
+laser_kv_status_t laser_kv_two_stage_topk(const float* s_exact, const uint32_t* counts,
+                                          int32_t n_segments, int32_t S, int32_t anchors,
+                                          int32_t k_exact, int32_t k_lsh, int32_t* idx_out,
+                                          void* stream);
+
+/* Append step (Sections 1 and 3): for each of n_segments segments copies rows idx[seg][i] of the
+ * segment's K and V (dev bf16, row length d = 128, consecutive rows `src_row_stride` elements
+ * apart, segment s starting at src + s*src_seg_stride) to dst rows [dst_offset + i] of the
+ * segment's cache (segments dst_seg_stride elements apart, rows d apart) and writes
+ * pos_base + idx[seg][i] to pos_out[s*pos_seg_stride + dst_offset + i]. */
+laser_kv_status_t laser_kv_gather_append(const void* K_src, const void* V_src,
+                                         int64_t src_seg_stride, int64_t src_row_stride,
+                                         const int32_t* idx, int32_t n_segments, int32_t n_keep,
+                                         void* K_dst, void* V_dst, int64_t dst_seg_stride,
+                                         int32_t* pos_out, int64_t pos_seg_stride,
+                                         int64_t dst_offset, int32_t pos_base, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LASER_KV_H_ */

@@ -1,0 +1,669 @@
+// Host runtime and C ABI of the LASER-KV selection library: configuration checks, budget
+// arithmetic (Appendix B Eq. 1, Section 3.1), workspace carving, TMA descriptors and the launch
+// sequence of one select call. Every step of the path runs in the CUDA kernels included below;
+// there is no CPU path.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+#include <string>
+#include <vector>
+
+#include "../../include/laser_kv.h"
+#include "aux_kernels.cuh"
+#include "stream_gemm.cuh"
+
+namespace {
+
+using namespace lkv;
+
+constexpr int kHeadDim = 128;
+constexpr size_t kAlign = 256;
+constexpr int kMaxSmem = 227 * 1024;
+
+std::atomic<long long> g_launches{0};
+thread_local std::string g_last_error;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct Derived {
+  int B, anchors, k_exact, k_lsh, G, GW;
+  int tiles_in_block, tiles_per_cta, n_split;
+  int TC, n_chunks;
+  double alpha, ratio;
+  float scale;
+  int fix_cap;
+  long long cap;       // cache entries per (sequence, KV head)
+  int nseg_max;
+};
+
+struct Carve {
+  size_t ctrl, hist, qbuckets, lse_part, lse2, s_exact, counts, idx, fix_items, key_buckets, total;
+};
+
+size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+}  // namespace
+
+struct laser_kv_ctx {
+  laser_kv_config_t cfg;
+  Derived d;
+  Carve carve;
+  uint8_t* ws = nullptr;
+  uint16_t* cacheK = nullptr;
+  uint16_t* cacheV = nullptr;
+  int32_t* cachePos = nullptr;
+  const uint16_t* P = nullptr;
+  CUtensorMap mapP;
+  EncodeTiledFn encode = nullptr;
+  std::vector<long long> blocks_done;   // per layer
+  std::string last_error;
+  bool have_call = false;
+  int last_nb = 0;
+  int last_fixups = 0;
+};
+
+namespace {
+
+laser_kv_status_t fail(laser_kv_ctx* h, laser_kv_status_t s, const char* fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof buf, fmt, ap);
+  va_end(ap);
+  if (h) h->last_error = buf;
+  g_last_error = buf;
+  return s;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Largest supported tables-per-chunk for the projection pass: K*TC a multiple of 16 and at
+// most 256 columns, L divisible by TC, histogram slice + operands within shared memory.
+int pick_tc(int K, int L) {
+  const int cands[3] = {32, 16, 8};
+  for (int tc : cands) {
+    if (L % tc) continue;
+    const int n = K * tc;
+    if (n > 256 || (n % 16)) continue;
+    const uint32_t smem = stream_smem_bytes(kProj, n, tc * (2 << K), 0);
+    if (smem > (uint32_t)kMaxSmem) continue;
+    return tc;
+  }
+  return 0;
+}
+
+laser_kv_status_t derive(const laser_kv_config_t* c, Derived* d) {
+  if (!c) return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "config is NULL");
+  if (c->n_layers < 1 || c->batch < 1 || c->n_q_heads < 1 || c->n_kv_heads < 1 ||
+      c->block_size < 1 || c->window < 1 || c->max_blocks < 1 || c->max_blocks_per_call < 1 ||
+      c->lsh_bits < 1 || c->lsh_tables < 1)
+    return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "config: counts must be positive");
+  if (c->n_q_heads % c->n_kv_heads)
+    return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "config: n_q_heads must be a multiple of n_kv_heads");
+  if (c->protection_divisor < 2)
+    return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "config: protection_divisor must be >= 2");
+  if (c->head_dim != kHeadDim)
+    return fail(nullptr, LASER_KV_ERR_UNSUPPORTED, "config: head_dim must be 128");
+  if (c->block_size % 8 || c->block_size > 16384)
+    return fail(nullptr, LASER_KV_ERR_UNSUPPORTED, "config: block_size must be a multiple of 8, at most 16384");
+  d->alpha = c->alpha < 0 ? 0.75 : c->alpha;
+  if (d->alpha > 1.0) return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "config: alpha must be in [0,1]");
+  d->ratio = c->ratio == 0 ? 0.25 : c->ratio;
+  if (d->ratio < 0) return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "config: ratio must be positive");
+  d->B = c->budget_per_block;
+  if (d->B == 0) {
+    if (c->context_len <= 0)
+      return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "config: budget_per_block == 0 needs context_len");
+    d->B = laser_kv_budget(c->context_len, c->block_size, d->ratio);
+  }
+  if (d->B < 0 || d->B > c->block_size)
+    return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "config: budget %d does not fit a block of %d", d->B, c->block_size);
+  int loc;
+  laser_kv_partition(d->B, c->protection_divisor, d->alpha, &d->anchors, &loc, &d->k_exact, &d->k_lsh);
+  d->G = c->n_q_heads / c->n_kv_heads;
+  d->GW = d->G * c->window;
+  if (d->GW % 16 || d->GW > 256 || c->window > 256 || d->G > 256)
+    return fail(nullptr, LASER_KV_ERR_UNSUPPORTED,
+                "config: G*W = %d must be a multiple of 16 and at most 256", d->GW);
+  if (!(c->lsh_bits == 4 || c->lsh_bits == 6 || c->lsh_bits == 8 || c->lsh_bits == 10 || c->lsh_bits == 12))
+    return fail(nullptr, LASER_KV_ERR_UNSUPPORTED, "config: lsh_bits must be one of 4, 6, 8, 10, 12");
+  d->TC = pick_tc(c->lsh_bits, c->lsh_tables);
+  if (!d->TC)
+    return fail(nullptr, LASER_KV_ERR_UNSUPPORTED, "config: lsh_tables must be a multiple of 8 (bits %d)", c->lsh_bits);
+  if ((long long)d->GW * c->lsh_tables > 0x7fffffffLL)
+    return fail(nullptr, LASER_KV_ERR_UNSUPPORTED, "config: G*W*lsh_tables too large");
+  d->n_chunks = c->lsh_tables / d->TC;
+  d->tiles_in_block = (c->block_size + kTileKeys - 1) / kTileKeys;
+  d->tiles_per_cta = d->tiles_in_block < 16 ? d->tiles_in_block : 16;
+  d->n_split = (d->tiles_in_block + d->tiles_per_cta - 1) / d->tiles_per_cta;
+  d->scale = c->softmax_scale == 0.f ? 1.0f / std::sqrt((float)c->head_dim) : c->softmax_scale;
+  d->cap = (long long)c->max_blocks * d->B;
+  const long long nseg = (long long)c->batch * c->n_kv_heads * c->max_blocks_per_call;
+  if (nseg > (1 << 22)) return fail(nullptr, LASER_KV_ERR_UNSUPPORTED, "config: too many segments per call");
+  d->nseg_max = (int)nseg;
+  long long fc = nseg * c->block_size * (long long)c->lsh_tables / 256;
+  if (fc < 4096) fc = 4096;
+  if (fc > (1 << 26)) fc = 1 << 26;
+  d->fix_cap = (int)fc;
+  return LASER_KV_OK;
+}
+
+void carve_ws(const laser_kv_config_t* c, const Derived& d, Carve* v) {
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+  const size_t nseg = d.nseg_max, S = c->block_size;
+  const size_t bh = (size_t)c->batch * c->n_kv_heads;
+  v->ctrl = take(256);
+  v->hist = take(bh * c->lsh_tables * ((size_t)2 << c->lsh_bits));
+  v->qbuckets = take(bh * d.GW * c->lsh_tables * 2);
+  v->lse_part = take(nseg * d.n_split * d.GW * sizeof(float2));
+  v->lse2 = take(nseg * d.GW * 4);
+  v->s_exact = take(nseg * S * 4);
+  v->counts = take(nseg * S * 4);
+  v->idx = take(nseg * (size_t)(d.B > 0 ? d.B : 1) * 4);
+  v->fix_items = take((size_t)d.fix_cap * sizeof(int4));
+  v->key_buckets = take(c->debug ? nseg * S * c->lsh_tables * 2 : 0);
+  v->total = off;
+}
+
+size_t cache_bytes_of(const laser_kv_config_t* c, const Derived& d) {
+  const size_t per = (size_t)c->n_layers * c->batch * c->n_kv_heads * (size_t)d.cap;
+  return align_up(per * kHeadDim * 2) * 2 + align_up(per * 4);
+}
+
+bool encode_map(laser_kv_ctx* h, CUtensorMap* m, const void* ptr, int rank, const uint64_t* dims,
+                const uint64_t* strides_bytes, const uint32_t* box) {
+  cuuint64_t gd[4];
+  cuuint64_t gs[3];
+  cuuint32_t bx[4], es[4];
+  for (int i = 0; i < rank; ++i) { gd[i] = dims[i]; bx[i] = box[i]; es[i] = 1; }
+  for (int i = 0; i + 1 < rank; ++i) gs[i] = strides_bytes[i];
+  const CUresult r = h->encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank,
+                               const_cast<void*>(ptr), gd, gs, bx, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    fail(h, LASER_KV_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+    return false;
+  }
+  return true;
+}
+
+template <int MODE, int KB, int TCv>
+cudaError_t launch_stream(const CUtensorMap& mk, const CUtensorMap& ms, const StreamArgs& a, int grid,
+                          uint32_t smem, cudaStream_t st) {
+  static bool attr_done = false;   // per instantiation; the attribute is per device function
+  cudaError_t e = cudaSuccess;
+  if (!attr_done) {
+    e = cudaFuncSetAttribute(stream_kernel<MODE, KB, TCv>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+    if (e != cudaSuccess) return e;
+    attr_done = true;
+  }
+  stream_kernel<MODE, KB, TCv><<<grid, kStreamThreads, smem, st>>>(mk, ms, a);
+  g_launches.fetch_add(1);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_proj(int K, int TCv, const CUtensorMap& mk, const CUtensorMap& ms, const StreamArgs& a,
+                        int grid, uint32_t smem, cudaStream_t st) {
+#define LKV_CASE(KB, T) if (K == KB && TCv == T) return launch_stream<kProj, KB, T>(mk, ms, a, grid, smem, st)
+  LKV_CASE(4, 8);  LKV_CASE(4, 16);  LKV_CASE(4, 32);
+  LKV_CASE(6, 8);  LKV_CASE(6, 16);  LKV_CASE(6, 32);
+  LKV_CASE(8, 8);  LKV_CASE(8, 16);  LKV_CASE(8, 32);
+  LKV_CASE(10, 8); LKV_CASE(10, 16);
+  LKV_CASE(12, 8); LKV_CASE(12, 16);
+#undef LKV_CASE
+  return cudaErrorInvalidValue;
+}
+
+laser_kv_status_t launch_select(const float* s_exact, const uint32_t* counts, int n_seg, int S, int anchors,
+                                int k_exact, int k_lsh, int32_t* idx, cudaStream_t st) {
+  static bool attr_done = false;
+  const size_t smem = (size_t)S * 9;
+  if (!attr_done) {
+    if (cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem - 2048) != cudaSuccess)
+      return fail(nullptr, LASER_KV_ERR_CUDA, "cudaFuncSetAttribute(select_kernel) failed");
+    attr_done = true;
+  }
+  SelectArgs a{s_exact, counts, idx, S, anchors, k_exact, k_lsh};
+  select_kernel<<<n_seg, kSelThreads, smem, st>>>(a);
+  g_launches.fetch_add(1);
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(nullptr, LASER_KV_ERR_CUDA, "select_kernel launch: %s", cudaGetErrorString(e));
+  return LASER_KV_OK;
+}
+
+laser_kv_status_t launch_append(const AppendArgs& a, int n_seg, cudaStream_t st) {
+  if (a.B <= 0 || n_seg <= 0) return LASER_KV_OK;
+  dim3 grid((a.B + kAppendRowsPerCta - 1) / kAppendRowsPerCta, n_seg);
+  append_kernel<<<grid, 256, 0, st>>>(a);
+  g_launches.fetch_add(1);
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(nullptr, LASER_KV_ERR_CUDA, "append_kernel launch: %s", cudaGetErrorString(e));
+  return LASER_KV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int32_t laser_kv_budget(int64_t context_len, int32_t block_size, double ratio) {
+  if (context_len <= 0 || block_size <= 0 || !(ratio > 0.0)) return -1;
+  const double num = 2.0 * ratio * (double)block_size * (double)context_len;
+  const double q = std::floor(num / ((double)block_size + (double)context_len));
+  return q > 2147483647.0 ? -1 : (int32_t)q;
+}
+
+laser_kv_status_t laser_kv_partition(int32_t B, int32_t n, double alpha, int32_t* anchors, int32_t* local,
+                                     int32_t* k_exact, int32_t* k_lsh) {
+  if (B < 0 || n < 2 || !(alpha >= 0.0 && alpha <= 1.0))
+    return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "partition: need B >= 0, n >= 2, 0 <= alpha <= 1");
+  const int32_t a = B / n;
+  const int32_t b_long = B - 2 * a;
+  int32_t ke = (int32_t)std::floor(alpha * (double)b_long);
+  if (ke < 0) ke = 0;
+  if (ke > b_long) ke = b_long;
+  if (anchors) *anchors = a;
+  if (local) *local = a;
+  if (k_exact) *k_exact = ke;
+  if (k_lsh) *k_lsh = b_long - ke;
+  return LASER_KV_OK;
+}
+
+laser_kv_status_t laser_kv_query_sizes(const laser_kv_config_t* cfg, size_t* cache_bytes, size_t* workspace_bytes) {
+  Derived d;
+  const laser_kv_status_t s = derive(cfg, &d);
+  if (s != LASER_KV_OK) return s;
+  Carve v;
+  carve_ws(cfg, d, &v);
+  if (cache_bytes) *cache_bytes = cache_bytes_of(cfg, d);
+  if (workspace_bytes) *workspace_bytes = v.total;
+  return LASER_KV_OK;
+}
+
+laser_kv_status_t laser_kv_init(const laser_kv_config_t* cfg, const void* hyperplanes, void* cache_mem,
+                                size_t cache_bytes, void* workspace, size_t workspace_bytes,
+                                laser_kv_handle_t* out) {
+  if (!out) return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "init: out is NULL");
+  *out = nullptr;
+  Derived d;
+  laser_kv_status_t s = derive(cfg, &d);
+  if (s != LASER_KV_OK) return s;
+  if (!hyperplanes || !cache_mem || !workspace)
+    return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "init: NULL device buffer");
+  if ((reinterpret_cast<uintptr_t>(cache_mem) | reinterpret_cast<uintptr_t>(workspace)) & (kAlign - 1))
+    return fail(nullptr, LASER_KV_ERR_ALIGNMENT, "init: cache and workspace must be 256-byte aligned");
+  if (!aligned16(hyperplanes)) return fail(nullptr, LASER_KV_ERR_ALIGNMENT, "init: hyperplanes must be 16-byte aligned");
+  Carve v;
+  carve_ws(cfg, d, &v);
+  if (cache_bytes < cache_bytes_of(cfg, d) || workspace_bytes < v.total)
+    return fail(nullptr, LASER_KV_ERR_CAPACITY, "init: cache needs %zu bytes, workspace %zu bytes",
+                cache_bytes_of(cfg, d), v.total);
+  int ndev = 0;
+  cudaError_t e = cudaGetDeviceCount(&ndev);
+  if (e != cudaSuccess || ndev <= cfg->device)
+    return fail(nullptr, LASER_KV_ERR_CUDA, "init: no usable CUDA device %d (%s); this library has no CPU path",
+                cfg->device, cudaGetErrorString(e));
+  if ((e = cudaSetDevice(cfg->device)) != cudaSuccess)
+    return fail(nullptr, LASER_KV_ERR_CUDA, "init: cudaSetDevice: %s", cudaGetErrorString(e));
+  cudaDeviceProp prop;
+  if ((e = cudaGetDeviceProperties(&prop, cfg->device)) != cudaSuccess)
+    return fail(nullptr, LASER_KV_ERR_CUDA, "init: cudaGetDeviceProperties: %s", cudaGetErrorString(e));
+  if (prop.major != 10)
+    return fail(nullptr, LASER_KV_ERR_UNSUPPORTED, "init: device is sm_%d%d; the kernels are built for sm_100a only",
+                prop.major, prop.minor);
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+  if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn)
+    return fail(nullptr, LASER_KV_ERR_CUDA, "init: cuTensorMapEncodeTiled not available from the driver");
+
+  laser_kv_ctx* h = new laser_kv_ctx();
+  h->cfg = *cfg;
+  h->d = d;
+  h->carve = v;
+  h->ws = static_cast<uint8_t*>(workspace);
+  h->encode = reinterpret_cast<EncodeTiledFn>(fn);
+  const size_t per = (size_t)cfg->n_layers * cfg->batch * cfg->n_kv_heads * (size_t)d.cap;
+  uint8_t* cm = static_cast<uint8_t*>(cache_mem);
+  h->cacheK = reinterpret_cast<uint16_t*>(cm);
+  h->cacheV = reinterpret_cast<uint16_t*>(cm + align_up(per * kHeadDim * 2));
+  h->cachePos = reinterpret_cast<int32_t*>(cm + 2 * align_up(per * kHeadDim * 2));
+  h->P = static_cast<const uint16_t*>(hyperplanes);
+  h->blocks_done.assign(cfg->n_layers, 0);
+  {
+    const uint64_t dims[2] = {(uint64_t)kHeadDim, (uint64_t)cfg->lsh_tables * cfg->lsh_bits};
+    const uint64_t strides[1] = {(uint64_t)kHeadDim * 2};
+    const uint32_t box[2] = {(uint32_t)kAtomCols, (uint32_t)(d.TC * cfg->lsh_bits)};
+    if (!encode_map(h, &h->mapP, h->P, 2, dims, strides, box)) {
+      const std::string msg = h->last_error;
+      delete h;
+      return fail(nullptr, LASER_KV_ERR_CUDA, "%s", msg.c_str());
+    }
+  }
+  if ((e = cudaMemset(h->ws + v.ctrl, 0, 256)) != cudaSuccess) {
+    delete h;
+    return fail(nullptr, LASER_KV_ERR_CUDA, "init: cudaMemset: %s", cudaGetErrorString(e));
+  }
+  *out = h;
+  return LASER_KV_OK;
+}
+
+laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, const void* K_blk, const void* V_blk,
+                                        const void* Q_win, const int64_t kv_strides[3], const int64_t q_strides[3],
+                                        int32_t n_blocks, void* stream) {
+  if (!h) return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "select_block: NULL handle");
+  const laser_kv_config_t& c = h->cfg;
+  const Derived& d = h->d;
+  if (layer < 0 || layer >= c.n_layers) return fail(h, LASER_KV_ERR_INVALID_ARG, "select_block: layer %d out of range", layer);
+  if (!K_blk || !V_blk || !Q_win || !kv_strides || !q_strides)
+    return fail(h, LASER_KV_ERR_INVALID_ARG, "select_block: NULL argument");
+  if (n_blocks < 1) return fail(h, LASER_KV_ERR_INVALID_ARG, "select_block: n_blocks must be >= 1");
+  if (n_blocks > c.max_blocks_per_call)
+    return fail(h, LASER_KV_ERR_CAPACITY, "select_block: n_blocks %d exceeds max_blocks_per_call %d", n_blocks, c.max_blocks_per_call);
+  if (h->blocks_done[layer] + n_blocks > c.max_blocks)
+    return fail(h, LASER_KV_ERR_CAPACITY, "select_block: layer %d cache holds %lld of %d blocks; cannot append %d",
+                layer, h->blocks_done[layer], c.max_blocks, n_blocks);
+  if (!aligned16(K_blk) || !aligned16(V_blk) || !aligned16(Q_win))
+    return fail(h, LASER_KV_ERR_ALIGNMENT, "select_block: device pointers must be 16-byte aligned");
+  for (int i = 0; i < 3; ++i)
+    if (kv_strides[i] < 0 || q_strides[i] < 0 || (kv_strides[i] % 8) || (q_strides[i] % 8))
+      return fail(h, LASER_KV_ERR_ALIGNMENT, "select_block: strides must be non-negative multiples of 8 elements");
+  if (kv_strides[2] < kHeadDim || q_strides[2] < kHeadDim)
+    return fail(h, LASER_KV_ERR_INVALID_ARG, "select_block: row stride smaller than head_dim");
+  if ((long long)(h->blocks_done[layer] + n_blocks) * c.block_size > 0x7fffffffLL)
+    return fail(h, LASER_KV_ERR_UNSUPPORTED, "select_block: absolute positions exceed int32");
+
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int S = c.block_size, nb = n_blocks, B = d.B;
+  const int nseg = c.batch * c.n_kv_heads * nb;
+  uint8_t* ws = h->ws;
+  int* ctrl = reinterpret_cast<int*>(ws + h->carve.ctrl);
+  uint16_t* hist = reinterpret_cast<uint16_t*>(ws + h->carve.hist);
+  uint16_t* qb = reinterpret_cast<uint16_t*>(ws + h->carve.qbuckets);
+  float2* lse_part = reinterpret_cast<float2*>(ws + h->carve.lse_part);
+  float* lse2 = reinterpret_cast<float*>(ws + h->carve.lse2);
+  float* s_exact = reinterpret_cast<float*>(ws + h->carve.s_exact);
+  uint32_t* counts = reinterpret_cast<uint32_t*>(ws + h->carve.counts);
+  int32_t* idx = reinterpret_cast<int32_t*>(ws + h->carve.idx);
+  int4* fix_items = reinterpret_cast<int4*>(ws + h->carve.fix_items);
+  uint16_t* key_buckets = c.debug ? reinterpret_cast<uint16_t*>(ws + h->carve.key_buckets) : nullptr;
+
+  // TMA descriptors for this call's K and Q_win
+  CUtensorMap mapK, mapQ;
+  {
+    const uint64_t dims[4] = {(uint64_t)kHeadDim, (uint64_t)nb * S, (uint64_t)c.n_kv_heads, (uint64_t)c.batch};
+    // a dimension of extent 1 never advances; give it a dense stride if the caller passed 0
+    const uint64_t s_tok = (uint64_t)kv_strides[2];
+    const uint64_t s_head = kv_strides[1] > 0 ? (uint64_t)kv_strides[1] : s_tok * (uint64_t)nb * S;
+    const uint64_t s_batch = kv_strides[0] > 0 ? (uint64_t)kv_strides[0] : s_head * (uint64_t)c.n_kv_heads;
+    if ((c.n_kv_heads > 1 && kv_strides[1] == 0) || (c.batch > 1 && kv_strides[0] == 0))
+      return fail(h, LASER_KV_ERR_INVALID_ARG, "select_block: zero stride on a dimension of extent > 1");
+    const uint64_t strides[3] = {s_tok * 2, s_head * 2, s_batch * 2};
+    const uint32_t box[4] = {(uint32_t)kAtomCols, (uint32_t)kTileKeys, 1, 1};
+    if (!encode_map(h, &mapK, K_blk, 4, dims, strides, box)) return LASER_KV_ERR_CUDA;
+  }
+  {
+    const uint64_t dims[4] = {(uint64_t)kHeadDim, (uint64_t)c.window, (uint64_t)c.n_q_heads, (uint64_t)c.batch};
+    const uint64_t s_w = (uint64_t)q_strides[2];
+    const uint64_t s_head = q_strides[1] > 0 ? (uint64_t)q_strides[1] : s_w * (uint64_t)c.window;
+    const uint64_t s_batch = q_strides[0] > 0 ? (uint64_t)q_strides[0] : s_head * (uint64_t)c.n_q_heads;
+    if ((c.n_q_heads > 1 && q_strides[1] == 0) || (c.batch > 1 && q_strides[0] == 0))
+      return fail(h, LASER_KV_ERR_INVALID_ARG, "select_block: zero stride on a dimension of extent > 1");
+    const uint64_t strides[3] = {s_w * 2, s_head * 2, s_batch * 2};
+    const uint32_t box[4] = {(uint32_t)kAtomCols, (uint32_t)c.window, (uint32_t)d.G, 1};
+    if (!encode_map(h, &mapQ, Q_win, 4, dims, strides, box)) return LASER_KV_ERR_CUDA;
+  }
+
+  cudaError_t e;
+#define LKV_CUDA(call, what)                                                                   \
+  if ((e = (call)) != cudaSuccess) return fail(h, LASER_KV_ERR_CUDA, "select_block: %s: %s", what, cudaGetErrorString(e))
+
+  // fix-up counter (ctrl[1]) and changed counter (ctrl[2]) restart; the status word (ctrl[0]) is kept
+  LKV_CUDA(cudaMemsetAsync(ctrl + 1, 0, 8, st), "memset ctrl");
+  LKV_CUDA(cudaMemsetAsync(counts, 0, (size_t)nseg * S * 4, st), "memset counts");
+
+  // 1. query signatures and bucket histogram
+  {
+    QprepArgs qa{static_cast<const uint16_t*>(Q_win), q_strides[0], q_strides[1], q_strides[2], h->P, hist, qb,
+                 c.n_kv_heads, d.G, c.window, d.GW, c.lsh_bits, c.lsh_tables};
+    const size_t smem = (size_t)c.lsh_bits * 128 * 8 + ((size_t)4 << c.lsh_bits);
+    dim3 grid(c.lsh_tables, c.n_kv_heads, c.batch);
+    qprep_kernel<<<grid, 256, smem, st>>>(qa);
+    g_launches.fetch_add(1);
+    LKV_CUDA(cudaGetLastError(), "qprep_kernel");
+  }
+
+  StreamArgs sa;
+  memset(&sa, 0, sizeof sa);
+  sa.S = S; sa.nb = nb; sa.t0 = 0; sa.tn = nb; sa.H_kv = c.n_kv_heads; sa.batch = c.batch;
+  sa.G = d.G; sa.W = c.window; sa.GW = d.GW;
+  sa.tiles_per_cta = d.tiles_per_cta; sa.n_split = d.n_split;
+  sa.n_chunks = d.n_chunks; sa.tables_per_chunk = d.TC; sa.lsh_bits = c.lsh_bits; sa.lsh_tables = c.lsh_tables;
+  sa.scale_log2e = d.scale * 1.4426950408889634f;
+  sa.lse_part = lse_part; sa.lse2 = lse2; sa.s_exact = s_exact; sa.counts = counts; sa.hist = hist;
+  sa.key_buckets = key_buckets; sa.fix_items = fix_items; sa.fix_count = ctrl + 1; sa.fix_cap = d.fix_cap;
+  sa.status = ctrl;
+
+  const int base_ctas = c.batch * c.n_kv_heads * nb * d.n_split;
+  // 2. per-query log-sum-exp over each block's keys
+  {
+    StreamArgs a1 = sa;
+    a1.stat_rows = d.GW;
+    a1.stat_rows_alloc = ((d.GW + 127) / 128) * 128;
+    const uint32_t smem = stream_smem_bytes(kLse, a1.stat_rows_alloc, 0, d.GW);
+    LKV_CUDA((launch_stream<kLse, 0, 0>(mapK, mapQ, a1, base_ctas, smem, st)), "lse pass");
+  }
+  // 3. summed attention probabilities per key
+  {
+    StreamArgs a2 = sa;
+    a2.stat_rows = d.GW;
+    a2.stat_rows_alloc = d.GW;
+    const uint32_t smem = stream_smem_bytes(kScore, a2.stat_rows_alloc, 0, d.GW);
+    LKV_CUDA((launch_stream<kScore, 0, 0>(mapK, mapQ, a2, base_ctas, smem, st)), "score pass");
+  }
+  // 4. key signatures and collision counts
+  {
+    StreamArgs a3 = sa;
+    a3.stat_rows = d.TC * c.lsh_bits;
+    a3.stat_rows_alloc = a3.stat_rows;
+    const uint32_t smem = stream_smem_bytes(kProj, a3.stat_rows_alloc, d.TC * (2 << c.lsh_bits), 0);
+    LKV_CUDA(launch_proj(c.lsh_bits, d.TC, mapK, h->mapP, a3, base_ctas * d.n_chunks, smem, st), "projection pass");
+  }
+  // 5. exact signs where the tensor-core projection was too close to zero
+  {
+    SignfixArgs fa{static_cast<const uint16_t*>(K_blk), kv_strides[0], kv_strides[1], kv_strides[2], h->P, hist,
+                   counts, key_buckets, fix_items, ctrl + 1, d.fix_cap, c.n_kv_heads, nb, S, c.lsh_bits,
+                   c.lsh_tables, ctrl + 2};
+    signfix_kernel<<<296, 256, 0, st>>>(fa);
+    g_launches.fetch_add(1);
+    LKV_CUDA(cudaGetLastError(), "signfix_kernel");
+  }
+  // 6. two-stage top-k
+  {
+    const laser_kv_status_t s = launch_select(s_exact, counts, nseg, S, d.anchors, d.k_exact, d.k_lsh, idx, st);
+    if (s != LASER_KV_OK) { h->last_error = g_last_error; return s; }
+  }
+  // 7. gather + append
+  {
+    const long long done = h->blocks_done[layer];
+    const size_t layer_off = (size_t)layer * c.batch * c.n_kv_heads * (size_t)d.cap;
+    AppendArgs aa{static_cast<const uint16_t*>(K_blk), static_cast<const uint16_t*>(V_blk),
+                  kv_strides[0], kv_strides[1], kv_strides[2], c.n_kv_heads, nb, S, B, idx,
+                  h->cacheK + layer_off * kHeadDim, h->cacheV + layer_off * kHeadDim, h->cachePos + layer_off,
+                  d.cap * kHeadDim, d.cap, done * B, (int)(done * S)};
+    const laser_kv_status_t s = launch_append(aa, nseg, st);
+    if (s != LASER_KV_OK) { h->last_error = g_last_error; return s; }
+  }
+#undef LKV_CUDA
+  h->blocks_done[layer] += nb;
+  h->have_call = true;
+  h->last_nb = nb;
+  return LASER_KV_OK;
+}
+
+laser_kv_status_t laser_kv_select_block_host(laser_kv_handle_t h, int32_t layer, const void* K_host, const void* V_host,
+                                             const void* Q_host, void* K_stage, void* V_stage, void* Q_stage,
+                                             int32_t n_blocks, int32_t* pos_out_host, void* stream) {
+  if (!h) return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "select_block_host: NULL handle");
+  if (!K_host || !V_host || !Q_host || !K_stage || !V_stage || !Q_stage)
+    return fail(h, LASER_KV_ERR_INVALID_ARG, "select_block_host: NULL argument");
+  if (layer < 0 || layer >= h->cfg.n_layers) return fail(h, LASER_KV_ERR_INVALID_ARG, "select_block_host: layer out of range");
+  if (n_blocks < 1 || n_blocks > h->cfg.max_blocks_per_call)
+    return fail(h, LASER_KV_ERR_CAPACITY, "select_block_host: n_blocks out of range");
+  const laser_kv_config_t& c = h->cfg;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t T = (size_t)n_blocks * c.block_size;
+  const size_t kv_bytes = (size_t)c.batch * c.n_kv_heads * T * kHeadDim * 2;
+  const size_t q_bytes = (size_t)c.batch * c.n_q_heads * c.window * kHeadDim * 2;
+  cudaError_t e;
+  if ((e = cudaMemcpyAsync(K_stage, K_host, kv_bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
+      (e = cudaMemcpyAsync(V_stage, V_host, kv_bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
+      (e = cudaMemcpyAsync(Q_stage, Q_host, q_bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess)
+    return fail(h, LASER_KV_ERR_CUDA, "select_block_host: H2D copy: %s", cudaGetErrorString(e));
+  const int64_t kvs[3] = {(int64_t)c.n_kv_heads * (int64_t)T * kHeadDim, (int64_t)T * kHeadDim, kHeadDim};
+  const int64_t qs[3] = {(int64_t)c.n_q_heads * c.window * kHeadDim, (int64_t)c.window * kHeadDim, kHeadDim};
+  const long long before = h->blocks_done[layer];
+  const laser_kv_status_t s = laser_kv_select_block(h, layer, K_stage, V_stage, Q_stage, kvs, qs, n_blocks, stream);
+  if (s != LASER_KV_OK) return s;
+  if (pos_out_host) {
+    const Derived& d = h->d;
+    const size_t layer_off = (size_t)layer * c.batch * c.n_kv_heads * (size_t)d.cap;
+    const int32_t* src = h->cachePos + layer_off + before * d.B;
+    e = cudaMemcpy2DAsync(pos_out_host, (size_t)n_blocks * d.B * 4, src, (size_t)d.cap * 4, (size_t)n_blocks * d.B * 4,
+                          (size_t)c.batch * c.n_kv_heads, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return fail(h, LASER_KV_ERR_CUDA, "select_block_host: D2H copy: %s", cudaGetErrorString(e));
+  }
+  return LASER_KV_OK;
+}
+
+laser_kv_status_t laser_kv_cache_view(laser_kv_handle_t h, int32_t layer, laser_kv_view_t* out) {
+  if (!h || !out) return fail(h, LASER_KV_ERR_INVALID_ARG, "cache_view: NULL argument");
+  if (layer < 0 || layer >= h->cfg.n_layers) return fail(h, LASER_KV_ERR_INVALID_ARG, "cache_view: layer out of range");
+  const laser_kv_config_t& c = h->cfg;
+  const Derived& d = h->d;
+  const size_t layer_off = (size_t)layer * c.batch * c.n_kv_heads * (size_t)d.cap;
+  out->K = h->cacheK + layer_off * kHeadDim;
+  out->V = h->cacheV + layer_off * kHeadDim;
+  out->pos = h->cachePos + layer_off;
+  out->len = h->blocks_done[layer] * d.B;
+  out->cap = d.cap;
+  out->kv_strides[0] = (int64_t)c.n_kv_heads * d.cap * kHeadDim;
+  out->kv_strides[1] = d.cap * kHeadDim;
+  out->kv_strides[2] = kHeadDim;
+  out->pos_strides[0] = (int64_t)c.n_kv_heads * d.cap;
+  out->pos_strides[1] = d.cap;
+  return LASER_KV_OK;
+}
+
+laser_kv_status_t laser_kv_debug_view(laser_kv_handle_t h, laser_kv_debug_t* out) {
+  if (!h || !out) return fail(h, LASER_KV_ERR_INVALID_ARG, "debug_view: NULL argument");
+  if (!h->have_call) return fail(h, LASER_KV_ERR_STATE, "debug_view: no select call yet");
+  const laser_kv_config_t& c = h->cfg;
+  uint8_t* ws = h->ws;
+  out->s_exact = reinterpret_cast<const float*>(ws + h->carve.s_exact);
+  out->counts = reinterpret_cast<const uint32_t*>(ws + h->carve.counts);
+  out->lse2 = reinterpret_cast<const float*>(ws + h->carve.lse2);
+  out->query_buckets = reinterpret_cast<const uint16_t*>(ws + h->carve.qbuckets);
+  out->key_buckets = c.debug ? reinterpret_cast<const uint16_t*>(ws + h->carve.key_buckets) : nullptr;
+  out->hist = reinterpret_cast<const uint16_t*>(ws + h->carve.hist);
+  out->idx = reinterpret_cast<const int32_t*>(ws + h->carve.idx);
+  out->n_blocks = h->last_nb;
+  out->batch = c.batch;
+  out->n_kv_heads = c.n_kv_heads;
+  out->block_size = c.block_size;
+  out->budget = h->d.B;
+  out->gw = h->d.GW;
+  out->lsh_tables = c.lsh_tables;
+  out->lsh_bits = c.lsh_bits;
+  out->n_sign_fixups = h->last_fixups;
+  return LASER_KV_OK;
+}
+
+laser_kv_status_t laser_kv_poll_status(laser_kv_handle_t h, void* stream) {
+  if (!h) return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "poll_status: NULL handle");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int host[4] = {0, 0, 0, 0};
+  cudaError_t e = cudaMemcpyAsync(host, h->ws + h->carve.ctrl, sizeof host, cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) return fail(h, LASER_KV_ERR_CUDA, "poll_status: %s", cudaGetErrorString(e));
+  h->last_fixups = host[1];
+  if (host[0] != 0) {
+    cudaMemsetAsync(h->ws + h->carve.ctrl, 0, 4, st);
+    cudaStreamSynchronize(st);
+    if (host[0] == LASER_KV_ERR_TIMEOUT) return fail(h, LASER_KV_ERR_TIMEOUT, "a bounded device-side wait gave up");
+    if (host[0] == LASER_KV_ERR_CAPACITY)
+      return fail(h, LASER_KV_ERR_CAPACITY, "exact-sign recompute list overflowed (%d items, capacity %d)", host[1], h->d.fix_cap);
+    return fail(h, (laser_kv_status_t)host[0], "device status word %d", host[0]);
+  }
+  return LASER_KV_OK;
+}
+
+laser_kv_status_t laser_kv_reset(laser_kv_handle_t h, int32_t layer) {
+  if (!h) return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "reset: NULL handle");
+  if (layer < -1 || layer >= h->cfg.n_layers) return fail(h, LASER_KV_ERR_INVALID_ARG, "reset: layer out of range");
+  if (layer == -1) std::fill(h->blocks_done.begin(), h->blocks_done.end(), 0);
+  else h->blocks_done[layer] = 0;
+  return LASER_KV_OK;
+}
+
+void laser_kv_destroy(laser_kv_handle_t h) { delete h; }
+
+const char* laser_kv_status_string(laser_kv_status_t s) {
+  switch (s) {
+    case LASER_KV_OK: return "ok";
+    case LASER_KV_ERR_INVALID_ARG: return "invalid argument";
+    case LASER_KV_ERR_UNSUPPORTED: return "unsupported configuration";
+    case LASER_KV_ERR_CAPACITY: return "capacity exceeded";
+    case LASER_KV_ERR_ALIGNMENT: return "misaligned pointer or stride";
+    case LASER_KV_ERR_CUDA: return "CUDA error";
+    case LASER_KV_ERR_TIMEOUT: return "device-side wait timed out";
+    case LASER_KV_ERR_STATE: return "call sequence error";
+  }
+  return "unknown status";
+}
+
+const char* laser_kv_last_error(laser_kv_handle_t h) { return h ? h->last_error.c_str() : g_last_error.c_str(); }
+
+int64_t laser_kv_launch_count(void) { return g_launches.load(); }
+
+laser_kv_status_t laser_kv_two_stage_topk(const float* s_exact, const uint32_t* counts, int32_t n_segments, int32_t S,
+                                          int32_t anchors, int32_t k_exact, int32_t k_lsh, int32_t* idx_out,
+                                          void* stream) {
+  if (!s_exact || !counts || !idx_out) return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "two_stage_topk: NULL argument");
+  if (n_segments < 1 || S < 1 || anchors < 0 || k_exact < 0 || k_lsh < 0)
+    return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "two_stage_topk: negative or zero size");
+  if (2LL * anchors + k_exact + k_lsh > S)
+    return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "two_stage_topk: keep count exceeds the segment");
+  if (S > 16384) return fail(nullptr, LASER_KV_ERR_UNSUPPORTED, "two_stage_topk: S > 16384");
+  if (2 * anchors + k_exact + k_lsh == 0) return LASER_KV_OK;
+  return launch_select(s_exact, counts, n_segments, S, anchors, k_exact, k_lsh, idx_out, static_cast<cudaStream_t>(stream));
+}
+
+laser_kv_status_t laser_kv_gather_append(const void* K_src, const void* V_src, int64_t src_seg_stride,
+                                         int64_t src_row_stride, const int32_t* idx, int32_t n_segments,
+                                         int32_t n_keep, void* K_dst, void* V_dst, int64_t dst_seg_stride,
+                                         int32_t* pos_out, int64_t pos_seg_stride, int64_t dst_offset, int32_t pos_base,
+                                         void* stream) {
+  if (!K_src || !V_src || !idx || !K_dst || !V_dst || !pos_out)
+    return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "gather_append: NULL argument");
+  if (n_segments < 1 || n_keep < 0 || dst_offset < 0) return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "gather_append: bad size");
+  if (!aligned16(K_src) || !aligned16(V_src) || !aligned16(K_dst) || !aligned16(V_dst) || (src_seg_stride % 8) ||
+      (src_row_stride % 8) || (dst_seg_stride % 8))
+    return fail(nullptr, LASER_KV_ERR_ALIGNMENT, "gather_append: pointers 16-byte aligned, strides multiples of 8");
+  AppendArgs aa{static_cast<const uint16_t*>(K_src), static_cast<const uint16_t*>(V_src), src_seg_stride, 0,
+                src_row_stride, 1, 1, 0, n_keep, idx, static_cast<uint16_t*>(K_dst), static_cast<uint16_t*>(V_dst),
+                pos_out, dst_seg_stride, pos_seg_stride, dst_offset, pos_base};
+  return launch_append(aa, n_segments, static_cast<cudaStream_t>(stream));
+}
+
+}  // extern "C"

@@ -1,0 +1,321 @@
+// The non-GEMM kernels of the selection path:
+//   qprep_kernel   - SimHash bucket codes of the window queries and the per-table histogram of
+//                    those codes (Section 3.3 "Recall"; Algorithm 1 line 6 counts collisions
+//                    against exactly these query buckets).
+//   signfix_kernel - exact recomputation of key sign bits whose tensor-core projection was too
+//                    close to zero to trust, with the matching correction of the counts.
+//   select_kernel  - Algorithm 1 lines 4-8: two-stage top-k per (sequence, KV head, block) by
+//                    shared-memory radix selection, ties to the lower index, ascending output.
+//   append_kernel  - gather of the kept K/V rows into the append-only cache (16-byte vectors).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace lkv {
+
+__device__ __forceinline__ double bf16_to_f64(uint16_t b) {
+  return static_cast<double>(__uint_as_float(static_cast<uint32_t>(b) << 16));
+}
+
+// ------------------------------------------------------------------------------------------------
+// Query side: one CTA per (table r, KV head h, sequence b); thread q handles window query q of the
+// head's group. Projections are accumulated in fp64 (products of two bf16 are exact in fp64), so
+// query sign bits need no guard. Bucket code: hyperplane r*K + b0 sits at bit K-1-b0.
+// ------------------------------------------------------------------------------------------------
+struct QprepArgs {
+  const uint16_t* Q;      // [batch][H_q][W][d] via strides
+  long long qs_b, qs_h, qs_w;
+  const uint16_t* P;      // [L*K][128]
+  uint16_t* hist;         // [batch][H_kv][L][2^K]
+  uint16_t* qbuckets;     // [batch][H_kv][GW][L]
+  int H_kv, G, W, GW, K, L;
+};
+
+__global__ void __launch_bounds__(256) qprep_kernel(const QprepArgs a) {
+  extern __shared__ uint8_t smem_q[];
+  double* planes = reinterpret_cast<double*>(smem_q);                       // [K][128]
+  uint32_t* bins = reinterpret_cast<uint32_t*>(smem_q + (size_t)a.K * 128 * 8);  // [2^K]
+  const int r = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  const int nbins = 1 << a.K;
+  for (int i = threadIdx.x; i < a.K * 128; i += blockDim.x)
+    planes[i] = bf16_to_f64(a.P[(size_t)r * a.K * 128 + i]);
+  for (int i = threadIdx.x; i < nbins; i += blockDim.x) bins[i] = 0;
+  __syncthreads();
+  for (int q = threadIdx.x; q < a.GW; q += blockDim.x) {
+    const int g = q / a.W, w = q % a.W;
+    const uint16_t* row = a.Q + b * a.qs_b + (long long)(h * a.G + g) * a.qs_h + w * a.qs_w;
+    uint32_t code = 0;
+    for (int bit = 0; bit < a.K; ++bit) {
+      const double* p = planes + bit * 128;
+      double acc = 0.0;
+      for (int c = 0; c < 128; c += 8) {
+        const uint4 v = *reinterpret_cast<const uint4*>(row + c);
+        const uint32_t ww[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          acc = fma(bf16_to_f64((uint16_t)(ww[e] & 0xFFFF)), p[c + 2 * e], acc);
+          acc = fma(bf16_to_f64((uint16_t)(ww[e] >> 16)), p[c + 2 * e + 1], acc);
+        }
+      }
+      code = (code << 1) | (acc >= 0.0 ? 1u : 0u);
+    }
+    atomicAdd(&bins[code], 1u);
+    a.qbuckets[((size_t)(b * a.H_kv + h) * a.GW + q) * a.L + r] = (uint16_t)code;
+  }
+  __syncthreads();
+  uint16_t* out = a.hist + ((size_t)(b * a.H_kv + h) * a.L + r) * nbins;
+  for (int i = threadIdx.x; i < nbins; i += blockDim.x) out[i] = (uint16_t)bins[i];
+}
+
+// ------------------------------------------------------------------------------------------------
+// Exact recomputation of flagged key signs. One warp per item; fp64 accumulation of the exact
+// bf16 products. If the exact bucket code differs from the provisional one the key's count is
+// corrected by hist[new] - hist[old].
+// ------------------------------------------------------------------------------------------------
+struct SignfixArgs {
+  const uint16_t* Kp;     // keys via strides
+  long long ks_b, ks_h, ks_t;
+  const uint16_t* P;
+  const uint16_t* hist;
+  uint32_t* counts;
+  uint16_t* key_buckets;  // or nullptr
+  const int4* items;
+  const int* n_items;
+  int cap;
+  int H_kv, nb, S, K, L;
+  int* n_changed;
+};
+
+__global__ void __launch_bounds__(256) signfix_kernel(const SignfixArgs a) {
+  const int lane = threadIdx.x & 31;
+  const int wid = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int nwarps = (gridDim.x * blockDim.x) >> 5;
+  const int n = min(*a.n_items, a.cap);
+  for (int it = wid; it < n; it += nwarps) {
+    const int4 item = a.items[it];
+    const int seg = item.x, key = item.y, r = item.z, old_code = item.w;
+    const int t = seg % a.nb;
+    const int h = (seg / a.nb) % a.H_kv;
+    const int b = seg / (a.nb * a.H_kv);
+    const uint16_t* krow = a.Kp + b * a.ks_b + h * a.ks_h + ((long long)t * a.S + key) * a.ks_t;
+    const uint2 kv = *reinterpret_cast<const uint2*>(krow + lane * 4);
+    const double k0 = bf16_to_f64((uint16_t)(kv.x & 0xFFFF)), k1 = bf16_to_f64((uint16_t)(kv.x >> 16));
+    const double k2 = bf16_to_f64((uint16_t)(kv.y & 0xFFFF)), k3 = bf16_to_f64((uint16_t)(kv.y >> 16));
+    uint32_t code = 0;
+    for (int bit = 0; bit < a.K; ++bit) {
+      const uint2 pv = *reinterpret_cast<const uint2*>(a.P + ((size_t)r * a.K + bit) * 128 + lane * 4);
+      double acc = k0 * bf16_to_f64((uint16_t)(pv.x & 0xFFFF));
+      acc = fma(k1, bf16_to_f64((uint16_t)(pv.x >> 16)), acc);
+      acc = fma(k2, bf16_to_f64((uint16_t)(pv.y & 0xFFFF)), acc);
+      acc = fma(k3, bf16_to_f64((uint16_t)(pv.y >> 16)), acc);
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+      code = (code << 1) | (acc >= 0.0 ? 1u : 0u);
+    }
+    if (lane == 0 && (int)code != old_code) {
+      const uint16_t* hr = a.hist + ((size_t)(b * a.H_kv + h) * a.L + r) * ((size_t)1 << a.K);
+      const uint32_t delta = (uint32_t)hr[code] - (uint32_t)hr[old_code];
+      atomicAdd(a.counts + (size_t)seg * a.S + key, delta);
+      if (a.key_buckets) a.key_buckets[((size_t)seg * a.S + key) * a.L + r] = (uint16_t)code;
+      atomicAdd(a.n_changed, 1);
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Two-stage top-k. One CTA of 1024 threads per segment; scores and counts live in shared memory.
+// ------------------------------------------------------------------------------------------------
+constexpr int kSelThreads = 1024;
+
+__device__ __forceinline__ uint32_t orderable_f32(float f) {
+  const uint32_t u = __float_as_uint(f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// Exclusive scan of one int per thread over the whole CTA; `total` receives the sum.
+__device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums, int& total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int incl = v;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const int n = __shfl_up_sync(0xffffffffu, incl, off);
+    if (lane >= off) incl += n;
+  }
+  if (lane == 31) warp_sums[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    int s = warp_sums[lane];
+    int si = s;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const int n = __shfl_up_sync(0xffffffffu, si, off);
+      if (lane >= off) si += n;
+    }
+    warp_sums[lane] = si - s;          // exclusive warp offsets
+    if (lane == 31) warp_sums[32] = si;
+  }
+  __syncthreads();
+  const int res = warp_sums[warp] + incl - v;
+  total = warp_sums[32];
+  __syncthreads();
+  return res;
+}
+
+// Among the participating elements j in [lo, hi) (flag[j] == 0) finds the k-th largest value T
+// (k >= 1, k <= number of participants) and how many elements equal to T belong to the top k.
+__device__ void radix_select_kth(const uint32_t* vals, const uint8_t* flag, int lo, int hi, int k,
+                                 int* hist, int* misc, uint32_t& T, int& need) {
+  uint32_t prefix = 0, mask = 0;
+  int remaining = k;
+  for (int shift = 24; shift >= 0; shift -= 8) {
+    for (int i = threadIdx.x; i < 256; i += kSelThreads) hist[i] = 0;
+    __syncthreads();
+    for (int j = lo + threadIdx.x; j < hi; j += kSelThreads) {
+      if (!flag[j]) {
+        const uint32_t u = vals[j];
+        if ((u & mask) == prefix) atomicAdd(&hist[(u >> shift) & 255], 1);
+      }
+    }
+    __syncthreads();
+    if (threadIdx.x < 32) {
+      const int lane = threadIdx.x;
+      int c[8], tot = 0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { c[i] = hist[255 - 8 * lane - i]; tot += c[i]; }
+      int incl = tot;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const int n = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += n;
+      }
+      const int excl = incl - tot;       // elements with a larger digit than this lane's range
+      if (excl < remaining && remaining <= incl) {
+        int run = excl;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          if (run < remaining && remaining <= run + c[i]) { misc[0] = 255 - 8 * lane - i; misc[1] = remaining - run; }
+          run += c[i];
+        }
+      }
+    }
+    __syncthreads();
+    prefix |= (uint32_t)misc[0] << shift;
+    mask |= 0xFFu << shift;
+    remaining = misc[1];
+    __syncthreads();
+  }
+  T = prefix;
+  need = remaining;
+}
+
+// Marks (flag = 1) the k largest participating elements of [lo, hi); equal values: lower index.
+__device__ void mark_topk(const uint32_t* vals, uint8_t* flag, int lo, int hi, int k, int* hist,
+                          int* misc, int* warp_sums) {
+  if (k <= 0) return;                    // uniform across the CTA
+  uint32_t T;
+  int need;
+  radix_select_kth(vals, flag, lo, hi, k, hist, misc, T, need);
+  const int n = hi - lo;
+  const int per = (n + kSelThreads - 1) / kSelThreads;
+  const int j0 = lo + threadIdx.x * per;
+  const int j1 = min(hi, j0 + per);
+  int eq = 0;
+  for (int j = j0; j < j1; ++j) eq += (!flag[j] && vals[j] == T) ? 1 : 0;
+  int total;
+  int rank = block_exclusive_scan(eq, warp_sums, total);
+  for (int j = j0; j < j1; ++j) {
+    if (flag[j]) continue;
+    const uint32_t u = vals[j];
+    if (u > T) flag[j] = 1;
+    else if (u == T) { if (rank < need) flag[j] = 1; ++rank; }
+  }
+  __syncthreads();
+}
+
+struct SelectArgs {
+  const float* s_exact;     // [n_seg][S]
+  const uint32_t* counts;   // [n_seg][S]
+  int32_t* idx;             // [n_seg][B]
+  int S, anchors, k_exact, k_lsh;
+};
+
+__global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectArgs a) {
+  extern __shared__ uint8_t smem_sel[];
+  uint32_t* ukey = reinterpret_cast<uint32_t*>(smem_sel);
+  uint32_t* ucnt = ukey + a.S;
+  uint8_t* flag = reinterpret_cast<uint8_t*>(ucnt + a.S);
+  __shared__ int hist[256];
+  __shared__ int misc[2];
+  __shared__ int warp_sums[33];
+  const int seg = blockIdx.x;
+  const int S = a.S, lo = a.anchors, hi = a.S - a.anchors;
+  const int B = 2 * a.anchors + a.k_exact + a.k_lsh;
+  for (int j = threadIdx.x; j < S; j += kSelThreads) {
+    ukey[j] = orderable_f32(a.s_exact[(size_t)seg * S + j]);
+    ucnt[j] = a.counts[(size_t)seg * S + j];
+    flag[j] = (j < lo || j >= hi) ? 1 : 0;
+  }
+  __syncthreads();
+  mark_topk(ukey, flag, lo, hi, a.k_exact, hist, misc, warp_sums);   // K_exact
+  mark_topk(ucnt, flag, lo, hi, a.k_lsh, hist, misc, warp_sums);     // K_lsh from the residual
+  // ordered compaction of all kept indices
+  const int per = (S + kSelThreads - 1) / kSelThreads;
+  const int j0 = threadIdx.x * per, j1 = min(S, j0 + per);
+  int cnt = 0;
+  for (int j = j0; j < j1; ++j) cnt += flag[j];
+  int total;
+  int out = block_exclusive_scan(cnt, warp_sums, total);
+  for (int j = j0; j < j1; ++j)
+    if (flag[j]) { if (out < B) a.idx[(size_t)seg * B + out] = j; ++out; }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Gather + append. 16 threads move one 256-byte row of K and of V as 16-byte vectors.
+// ------------------------------------------------------------------------------------------------
+struct AppendArgs {
+  const uint16_t* K;
+  const uint16_t* V;
+  long long ks_b, ks_h, ks_t;   // source strides (elements): batch, head, token
+  int H_kv, nb, S, B;
+  const int32_t* idx;           // [batch][H_kv][nb][B]
+  uint16_t* Kc;
+  uint16_t* Vc;
+  int32_t* pos;
+  long long c_seg_stride;       // elements between (batch, head) cache slabs
+  long long pos_seg_stride;
+  long long dst_off0;           // first destination entry of block t = 0
+  int pos_base0;                // absolute position of token 0 of block t = 0
+};
+
+constexpr int kAppendRowsPerCta = 64;
+
+__device__ __forceinline__ uint4 ld_nc_v4(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+
+__global__ void __launch_bounds__(256) append_kernel(const AppendArgs a) {
+  const int seg = blockIdx.y;                      // (b*H_kv + h)*nb + t
+  const int t = seg % a.nb;
+  const int bh = seg / a.nb;
+  const int h = bh % a.H_kv, b = bh / a.H_kv;
+  const int part = threadIdx.x & 15;
+  const int i_end = min(a.B, (int)(blockIdx.x + 1) * kAppendRowsPerCta);
+  const long long src_base = b * a.ks_b + h * a.ks_h + (long long)t * a.S * a.ks_t;
+  const long long dst_base = bh * a.c_seg_stride + (a.dst_off0 + (long long)t * a.B) * 128;
+  for (int i = blockIdx.x * kAppendRowsPerCta + (threadIdx.x >> 4); i < i_end; i += 16) {
+    const int src = a.idx[(size_t)seg * a.B + i];
+    const long long so = src_base + (long long)src * a.ks_t + part * 8;
+    const long long dof = dst_base + (long long)i * 128 + part * 8;
+    const uint4 kv = ld_nc_v4(a.K + so);
+    const uint4 vv = ld_nc_v4(a.V + so);
+    *reinterpret_cast<uint4*>(a.Kc + dof) = kv;
+    *reinterpret_cast<uint4*>(a.Vc + dof) = vv;
+    if (part == 0) a.pos[bh * a.pos_seg_stride + a.dst_off0 + (long long)t * a.B + i] = a.pos_base0 + t * a.S + src;
+  }
+}
+
+}  // namespace lkv

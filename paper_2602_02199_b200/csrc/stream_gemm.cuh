@@ -1,0 +1,398 @@
+// Key-streaming tensor-core kernels for the two dense contractions of the selection path:
+//   * the window-score contraction Q_win . K^T  (Section 3.3 "Precision", Algorithm 1 line 3)
+//   * the hyperplane projection K . P^T         (Section 3.3 "Recall", hash functions h_r)
+// One warp-specialised skeleton serves three passes. A CTA keeps one small operand stationary
+// in shared memory (the group's window queries, or a chunk of hyperplanes with the matching
+// slice of the query-bucket histogram) and streams 128-key tiles of one (sequence, KV head,
+// block) through a TMA -> tcgen05.mma -> TMEM -> register pipeline:
+//
+//   kLse   : D[query][key]; every thread owns one query row and keeps an online
+//            (max, sum-exp2) pair over the CTA's keys -> per-split partials of log-sum-exp.
+//   kScore : D[key][query]; every thread owns one key and sums exp2(s - lse_q) over the
+//            group's queries -> S_exact[key].
+//   kProj  : D[key][hyperplane]; every thread owns one key, packs sign bits into K-bit bucket
+//            ids, looks the buckets up in the query-bucket histogram (count of window queries
+//            per bucket) and adds the collisions to count[key]. Signs decided by a projection
+//            that is tiny relative to the key's other projections are queued for an exact
+//            recomputation.
+//
+// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner,
+// warps 2..5 = epilogue (TMEM lane quarter = warp_id % 4).
+#pragma once
+#include "ptx.cuh"
+
+namespace lkv {
+
+constexpr int kTileKeys = 128;                 // keys per streamed tile (UMMA M or N)
+constexpr int kAtomCols = 64;                  // bf16 elements per 128-byte swizzle row
+constexpr int kTileAtomBytes = kTileKeys * 128;  // one 64-column half of a key tile
+constexpr int kTileBytes = 2 * kTileAtomBytes;   // 128 keys x 128 dims bf16
+constexpr int kStages = 4;
+constexpr int kStreamThreads = 192;
+constexpr int kTmemCols = 512;
+constexpr int kAccStride = 256;                // TMEM columns per accumulator buffer
+constexpr int kMaxStatRows = 256;
+
+enum StreamMode { kLse = 0, kScore = 1, kProj = 2 };
+
+enum : int { kStatusOk = 0, kStatusCapacity = 3, kStatusTimeout = 6 };
+
+struct StreamArgs {
+  // problem geometry
+  int S;               // keys per block
+  int nb;              // blocks in this call
+  int t0, tn;          // block range [t0, t0 + tn) handled by this launch
+  int H_kv, batch;
+  int G, W, GW;        // GQA group size, window, G*W
+  int tiles_per_cta;   // key tiles per CTA
+  int n_split;         // CTAs along the keys of one block
+  int stat_rows;       // rows of the stationary operand (GW, or tables_per_chunk * lsh_bits)
+  int stat_rows_alloc; // rows reserved per 64-column half in shared memory (multiple of 8)
+  int n_chunks, tables_per_chunk, lsh_bits, lsh_tables;
+  float scale_log2e;   // softmax scale * log2(e)
+  // buffers (device)
+  float2* lse_part;        // [seg][n_split][GW]  (max, sum) in the log2 domain
+  float* lse2;             // [seg][GW]
+  float* s_exact;          // [seg][S]
+  uint32_t* counts;        // [seg][S]
+  const uint16_t* hist;    // [batch][H_kv][L][2^K]
+  uint16_t* key_buckets;   // [seg][S][L] or nullptr
+  int4* fix_items;         // (seg, key, table, provisional bucket)
+  int* fix_count;
+  int fix_cap;
+  int* status;
+};
+
+__device__ __forceinline__ void record_status(int* status, int code) {
+  atomicCAS(status, kStatusOk, code);
+}
+
+struct StreamSmem {
+  uint32_t stat, stages, hist, lse, bars, tmem_slot;  // shared-space byte addresses
+};
+
+// Shared memory carve-up, identical on host (sizes) and device (addresses).
+__host__ __device__ inline uint32_t stream_smem_bytes(int mode, int stat_rows_alloc,
+                                                      int hist_bytes, int GW) {
+  uint32_t b = 2u * stat_rows_alloc * 128u + kStages * kTileBytes;
+  if (mode == kProj) b += (hist_bytes + 127u) & ~127u;
+  if (mode == kScore) b += ((GW * 4u) + 127u) & ~127u;
+  b += 256;          // barriers + TMEM slot
+  return b + 1024;   // slack for 1024-byte alignment of the base
+}
+
+template <int MODE, int KBITS, int TC>
+__global__ void __launch_bounds__(kStreamThreads, 1)
+stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, head, batch)
+              const __grid_constant__ CUtensorMap map_stat,   // Q: (d, W, H_q, batch) | P: (d, L*K)
+              const StreamArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+
+  // ---- which work item -------------------------------------------------------------------
+  int bid = blockIdx.x;
+  int chunk = 0;
+  if (MODE == kProj) { chunk = bid % a.n_chunks; bid /= a.n_chunks; }
+  const int split = bid % a.n_split; bid /= a.n_split;
+  const int tl = bid % a.tn; bid /= a.tn;
+  const int h = bid % a.H_kv;
+  const int b = bid / a.H_kv;
+  const int t = a.t0 + tl;
+  const int seg = (b * a.H_kv + h) * a.nb + t;
+  const int tiles_in_block = (a.S + kTileKeys - 1) / kTileKeys;
+  const int tile0 = split * a.tiles_per_cta;
+  const int ntiles = min(a.tiles_per_cta, tiles_in_block - tile0);
+
+  // ---- shared memory ---------------------------------------------------------------------
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t stat_atom_bytes = a.stat_rows_alloc * 128u;
+  StreamSmem sm;
+  sm.stat = base;
+  sm.stages = sm.stat + 2u * stat_atom_bytes;
+  uint32_t cur = sm.stages + kStages * kTileBytes;
+  const uint32_t hist_bytes = (MODE == kProj) ? (uint32_t)TC * (2u << KBITS) : 0u;
+  sm.hist = cur;
+  if (MODE == kProj) cur += (hist_bytes + 127u) & ~127u;
+  sm.lse = cur;
+  if (MODE == kScore) cur += ((a.GW * 4u) + 127u) & ~127u;
+  sm.bars = cur;
+  sm.tmem_slot = cur + 128;
+  const uint32_t bar_full = sm.bars;                 // kStages barriers
+  const uint32_t bar_empty = sm.bars + 8 * kStages;  // kStages barriers
+  const uint32_t bar_tfull = sm.bars + 16 * kStages; // 2 barriers
+  const uint32_t bar_tempty = bar_tfull + 16;        // 2 barriers
+  const uint32_t bar_stat = bar_tempty + 16;         // 1 barrier
+  uint8_t* const gen_base = smem_raw + (base - smem_u32(smem_raw));
+  const uint16_t* hist_s = reinterpret_cast<const uint16_t*>(gen_base + (sm.hist - base));
+  float* lse_s = reinterpret_cast<float*>(gen_base + (sm.lse - base));
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_base + (sm.tmem_slot - base));
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+    for (int s = 0; s < 2; ++s) { mbar_init(bar_tfull + 8 * s, 1); mbar_init(bar_tempty + 8 * s, 128); }
+    mbar_init(bar_stat, 1);
+    fence_mbar_init();
+  }
+  if (warp == 1) { tmem_alloc(sm.tmem_slot, kTmemCols); tmem_relinquish(); }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int nmb = (MODE == kLse) ? (a.GW + 127) / 128 : 1;   // query row blocks of 128
+
+  if (warp == 0) {
+    // ================= TMA producer =================
+    if (lane == 0) {
+      bool ok = true;
+      tma_prefetch_desc(&map_keys);
+      tma_prefetch_desc(&map_stat);
+      // stationary operand (+ histogram slice)
+      const uint32_t stat_bytes = 2u * a.stat_rows * 128u;
+      mbar_expect_tx(bar_stat, stat_bytes + hist_bytes);
+      if (MODE == kProj) {
+        const int row0 = chunk * a.stat_rows;
+        tma_load_2d(sm.stat, &map_stat, bar_stat, 0, row0);
+        tma_load_2d(sm.stat + stat_atom_bytes, &map_stat, bar_stat, kAtomCols, row0);
+        const uint16_t* hsrc = a.hist + ((size_t)(b * a.H_kv + h) * a.lsh_tables +
+                                         (size_t)chunk * TC) * ((size_t)1 << KBITS);
+        bulk_load(sm.hist, hsrc, hist_bytes, bar_stat);
+      } else {
+        tma_load_4d(sm.stat, &map_stat, bar_stat, 0, 0, h * a.G, b);
+        tma_load_4d(sm.stat + stat_atom_bytes, &map_stat, bar_stat, kAtomCols, 0, h * a.G, b);
+      }
+      int issued = 0;
+      for (int i = 0; i < ntiles && ok; ++i) {
+        const int s = i % kStages;
+        const int round = i / kStages;
+        if (round > 0) ok = mbar_wait(bar_empty + 8 * s, (round - 1) & 1);
+        if (!ok) break;
+        const uint32_t dst = sm.stages + s * kTileBytes;
+        const int token = t * a.S + (tile0 + i) * kTileKeys;
+        mbar_expect_tx(bar_full + 8 * s, kTileBytes);
+        tma_load_4d(dst, &map_keys, bar_full + 8 * s, 0, token, h, b);
+        tma_load_4d(dst + kTileAtomBytes, &map_keys, bar_full + 8 * s, kAtomCols, token, h, b);
+        issued = i + 1;
+      }
+      if (!ok) {
+        record_status(a.status, kStatusTimeout);
+        // let copies already in flight land before the CTA may exit
+        for (int i = max(0, issued - kStages); i < issued; ++i)
+          mbar_wait(bar_full + 8 * (i % kStages), (i / kStages) & 1);
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ================= MMA issuer =================
+    if (lane == 0) {
+      bool ok = mbar_wait(bar_stat, 0);
+      const uint32_t idesc = (MODE == kLse) ? umma_idesc_bf16(128, kTileKeys)
+                                            : umma_idesc_bf16(128, a.stat_rows);
+      for (int i = 0; i < ntiles && ok; ++i) {
+        const int s = i % kStages;
+        const int acc = i & 1;
+        if (i >= 2) ok = mbar_wait(bar_tempty + 8 * acc, ((i >> 1) - 1) & 1);
+        if (ok) ok = mbar_wait(bar_full + 8 * s, (i / kStages) & 1);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t tile = sm.stages + s * kTileBytes;
+        for (int mb = 0; mb < nmb; ++mb) {
+          const uint32_t d = tmem_base + acc * kAccStride + mb * 128;
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            const uint32_t koff = (k & 3) * 32;
+            const uint32_t tile_k = tile + (k >> 2) * kTileAtomBytes + koff;
+            const uint32_t stat_k = sm.stat + (k >> 2) * stat_atom_bytes + koff;
+            if (MODE == kLse) {
+              umma_bf16(d, umma_sdesc_sw128(stat_k + mb * (128 * 128)), umma_sdesc_sw128(tile_k),
+                        idesc, k > 0);
+            } else {
+              umma_bf16(d, umma_sdesc_sw128(tile_k), umma_sdesc_sw128(stat_k), idesc, k > 0);
+            }
+          }
+        }
+        umma_commit(bar_empty + 8 * s);     // stage reusable once these MMAs have read it
+        umma_commit(bar_tfull + 8 * acc);   // accumulator ready for the epilogue
+      }
+      if (!ok) record_status(a.status, kStatusTimeout);
+    }
+    __syncwarp();
+  } else {
+    // ================= epilogue warps =================
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;                   // TMEM lane owned by this thread
+    const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
+    const int etid = threadIdx.x - 64;                     // 0..127
+    bool ok = true;
+
+    if (MODE == kLse) {
+      float m[2] = {-INFINITY, -INFINITY};
+      float l[2] = {0.f, 0.f};
+      for (int i = 0; i < ntiles && ok; ++i) {
+        const int acc = i & 1;
+        ok = mbar_wait(bar_tfull + 8 * acc, (i >> 1) & 1);
+        if (!ok) break;
+        tc_fence_after();
+        const int nvalid = min(kTileKeys, a.S - (tile0 + i) * kTileKeys);
+#pragma unroll
+        for (int mb = 0; mb < 2; ++mb) {
+          if (mb < nmb) {
+            for (int c = 0; c < 4; ++c) {
+              if (c * 32 >= nvalid) break;
+              uint32_t v[32];
+              tmem_ld_x32(t_lane + acc * kAccStride + mb * 128 + c * 32, v);
+              tmem_wait_ld();
+              const int lim = nvalid - c * 32;             // >= 1
+              float tv[32];
+              float cmax = -INFINITY;
+#pragma unroll
+              for (int k = 0; k < 32; ++k) {
+                tv[k] = (k < lim) ? __uint_as_float(v[k]) * a.scale_log2e : -INFINITY;
+                cmax = fmaxf(cmax, tv[k]);
+              }
+              const float m_new = fmaxf(m[mb], cmax);
+              float add = 0.f;
+#pragma unroll
+              for (int k = 0; k < 32; ++k) add += ex2_approx(tv[k] - m_new);
+              l[mb] = l[mb] * ex2_approx(m[mb] - m_new) + add;
+              m[mb] = m_new;
+            }
+          }
+        }
+        tc_fence_before();
+        mbar_arrive(bar_tempty + 8 * acc);
+      }
+      if (ok) {
+#pragma unroll
+        for (int mb = 0; mb < 2; ++mb) {
+          const int q = mb * 128 + row;
+          if (mb < nmb && q < a.GW)
+            a.lse_part[((size_t)seg * a.n_split + split) * a.GW + q] = make_float2(m[mb], l[mb]);
+        }
+      }
+    } else if (MODE == kScore) {
+      // combine the splits' (max, sum) partials into log2-sum-exp2 per query
+      for (int q = etid; q < a.GW; q += 128) {
+        const float2* p = a.lse_part + (size_t)seg * a.n_split * a.GW + q;
+        float mx = -INFINITY;
+        for (int s2 = 0; s2 < a.n_split; ++s2) mx = fmaxf(mx, p[(size_t)s2 * a.GW].x);
+        float sum = 0.f;
+        for (int s2 = 0; s2 < a.n_split; ++s2) {
+          const float2 e = p[(size_t)s2 * a.GW];
+          sum += e.y * exp2f(e.x - mx);
+        }
+        const float r = mx + log2f(sum);
+        lse_s[q] = r;
+        if (split == 0) a.lse2[(size_t)seg * a.GW + q] = r;
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      for (int i = 0; i < ntiles && ok; ++i) {
+        const int acc = i & 1;
+        ok = mbar_wait(bar_tfull + 8 * acc, (i >> 1) & 1);
+        if (!ok) break;
+        tc_fence_after();
+        float sum = 0.f;
+        for (int c0 = 0; c0 < a.GW; c0 += 32) {
+          uint32_t v[32];
+          if (c0 + 32 <= a.GW) {
+            tmem_ld_x32(t_lane + acc * kAccStride + c0, v);
+            tmem_wait_ld();
+#pragma unroll
+            for (int k = 0; k < 32; k += 4) {
+              const float4 ls = *reinterpret_cast<const float4*>(lse_s + c0 + k);
+              sum += ex2_approx(fmaf(__uint_as_float(v[k + 0]), a.scale_log2e, -ls.x));
+              sum += ex2_approx(fmaf(__uint_as_float(v[k + 1]), a.scale_log2e, -ls.y));
+              sum += ex2_approx(fmaf(__uint_as_float(v[k + 2]), a.scale_log2e, -ls.z));
+              sum += ex2_approx(fmaf(__uint_as_float(v[k + 3]), a.scale_log2e, -ls.w));
+            }
+          } else {  // GW % 32 == 16
+            tmem_ld_x16(t_lane + acc * kAccStride + c0, v);
+            tmem_wait_ld();
+#pragma unroll
+            for (int k = 0; k < 16; ++k)
+              sum += ex2_approx(fmaf(__uint_as_float(v[k]), a.scale_log2e, -lse_s[c0 + k]));
+          }
+        }
+        tc_fence_before();
+        mbar_arrive(bar_tempty + 8 * acc);
+        const int key = (tile0 + i) * kTileKeys + row;
+        if (key < a.S) a.s_exact[(size_t)seg * a.S + key] = sum;
+      }
+    } else {
+      // ---- kProj: sign bits -> bucket codes -> histogram lookups ----
+      // Bucket code of a table: bit b of the table (hyperplane r*K + b) sits at position
+      // K-1-b, i.e. the first hyperplane is the most significant bit; bit = [projection >= 0].
+      ok = mbar_wait(bar_stat, 0);   // histogram slice landed (async-proxy writes visible after the wait)
+      constexpr int NCOLS = KBITS * TC;
+      constexpr uint32_t bucket_mask = (1u << KBITS) - 1u;
+      for (int i = 0; i < ntiles && ok; ++i) {
+        const int acc = i & 1;
+        ok = mbar_wait(bar_tfull + 8 * acc, (i >> 1) & 1);
+        if (!ok) break;
+        tc_fence_after();
+        const int key = (tile0 + i) * kTileKeys + row;
+        const bool valid = key < a.S;
+        const uint32_t t_acc = t_lane + acc * kAccStride;
+        uint32_t partial = 0;
+        uint32_t neg = 0;
+        float amin = INFINITY;
+        float tau = 0.f;
+#pragma unroll
+        for (int c0 = 0; c0 < NCOLS; c0 += 32) {
+          uint32_t v[32];
+          constexpr int kFull = 32;
+          const bool full = (c0 + kFull <= NCOLS);
+          if (full) tmem_ld_x32(t_acc + c0, v); else tmem_ld_x16(t_acc + c0, v);
+          tmem_wait_ld();
+          if (c0 == 0) {
+            // scale of this key's projections, from the first 16 hyperplanes of the chunk
+            float amax = 0.f;
+#pragma unroll
+            for (int k = 0; k < 16; ++k) amax = fmaxf(amax, fabsf(__uint_as_float(v[k])));
+            tau = amax * (1.0f / 32768.0f);
+          }
+#pragma unroll
+          for (int k = 0; k < 32; ++k) {
+            if (c0 + k < NCOLS) {
+              const uint32_t x = v[k];
+              neg = __funnelshift_l(x, neg, 1);            // (neg << 1) | sign(x)
+              amin = fminf(amin, fabsf(__uint_as_float(x)));
+              if ((c0 + k) % KBITS == KBITS - 1) {
+                const int rl = (c0 + k) / KBITS;           // table within the chunk
+                const uint32_t code = (~neg) & bucket_mask;
+                partial += hist_s[((uint32_t)rl << KBITS) + code];
+                if (valid) {
+                  const int r = chunk * TC + rl;
+                  if (a.key_buckets)
+                    a.key_buckets[((size_t)seg * a.S + key) * a.lsh_tables + r] = (uint16_t)code;
+                  if (!(amin >= tau)) {
+                    const int slot = atomicAdd(a.fix_count, 1);
+                    if (slot < a.fix_cap) a.fix_items[slot] = make_int4(seg, key, r, (int)code);
+                    else record_status(a.status, kStatusCapacity);
+                  }
+                }
+                neg = 0;
+                amin = INFINITY;
+              }
+            }
+          }
+        }
+        tc_fence_before();
+        mbar_arrive(bar_tempty + 8 * acc);
+        if (valid) atomicAdd(a.counts + (size_t)seg * a.S + key, partial);
+      }
+    }
+    if (!ok) record_status(a.status, kStatusTimeout);
+  }
+
+  // ---- teardown ----------------------------------------------------------------------------
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+}  // namespace lkv

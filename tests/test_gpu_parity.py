@@ -1,0 +1,182 @@
+"""CUDA path vs the fp64 oracle, element by element, through the C ABI."""
+import numpy as np
+import pytest
+
+from oracle import laser_kv_oracle as O
+from paper_2602_02199_b200 import synth
+
+from parity_util import check_run, run_workload_layer, to_np
+
+pytestmark = pytest.mark.gpu
+
+
+def test_tiny_config_all_blocks_all_heads():
+    w = synth.workload("tiny")
+    run = run_workload_layer(w, 0)
+    stats = check_run(w, run)
+    assert len(stats) == 8 * 4
+
+
+@pytest.mark.parametrize("S,B,n,alpha", [
+    (1000, 300, 4, 0.75),      # ragged: last key tile has 104 keys
+    (136, 40, 4, 0.5),         # one full tile + 8 keys
+    (512, 128, 2, 0.75),       # n = 2: empty recall budget
+    (512, 129, 2, 0.75),       # n = 2 with an odd budget: one LSH pick
+    (640, 200, 4, 1.0),        # LSH stage disabled: pure attention top-k
+    (640, 200, 4, 0.0),        # exact stage disabled: pure LSH top-k
+    (384, 384, 4, 0.75),       # keep everything
+    (256, 0, 4, 0.75),         # keep nothing
+])
+def test_shrunken_and_degenerate_shapes(S, B, n, alpha):
+    w = synth.workload("tiny").with_(name=f"s{S}", block_size=S, context_len=3 * S, protection_divisor=n,
+                                     alpha=alpha)
+    run = run_workload_layer(w, 0, budget=B, alpha=alpha)
+    check_run(w, run, alpha=alpha)
+
+
+def test_gqa7_k10_shape_with_rope_and_batch():
+    # Qwen-like group of 7 (G*W = 224), 10-bit tables, two sequences
+    w = synth.workload("qwen7b_128k").with_(name="qwen_small", batch=2, block_size=520, context_len=4 * 520,
+                                            lsh_bits=10, lsh_tables=16, needles="uniform:4", n_layers=1)
+    run = run_workload_layer(w, 0)
+    check_run(w, run)
+
+
+def test_outlier_tokens_and_n_sweep():
+    for n in (2, 4, 8):
+        w = synth.workload("llama8b_64k").with_(name=f"out{n}", block_size=768, context_len=2 * 768,
+                                                protection_divisor=n, n_layers=1)
+        run = run_workload_layer(w, 0)
+        check_run(w, run)
+
+
+def test_token_major_layout_gives_identical_results():
+    w = synth.workload("tiny").with_(block_size=256, context_len=1024)
+    r1 = run_workload_layer(w, 0)
+    r2 = run_workload_layer(w, 0, layout="bshd")
+    d1, d2 = r1["engine"].laser_kv_debug_view(), r2["engine"].laser_kv_debug_view()
+    assert (to_np(d1.idx) == to_np(d2.idx)).all()
+    assert (to_np(d1.counts) == to_np(d2.counts)).all()
+    assert (to_np(d1.s_exact) == to_np(d2.s_exact)).all()
+    check_run(w, r2)
+
+
+def test_append_only_across_calls_and_capacity():
+    import torch
+    from paper_2602_02199_b200 import binding as Bn
+    w = synth.workload("tiny").with_(block_size=256, context_len=1024, n_layers=2)
+    B = Bn.laser_kv_budget(w.context_len, w.block_size)
+    dev = torch.device("cuda", 0)
+    P = torch.from_numpy(synth.hyperplanes(w).view(np.int16)).to(dev)
+    cfg = Bn.make_config(n_layers=2, batch=1, n_q_heads=32, n_kv_heads=8, block_size=256, window=32, max_blocks=4,
+                         max_blocks_per_call=4, lsh_bits=8, lsh_tables=16, protection_divisor=4,
+                         budget_per_block=B)
+    one = Bn.LaserKV(cfg, P)
+    inc = Bn.LaserKV(cfg, P)
+    K, V = synth.kv_blocks(w, 1, 0, 0, 4)
+    Q = synth.q_window(w, 1, 0)
+    tK = torch.from_numpy(K.view(np.int16)).to(dev)[None]
+    tV = torch.from_numpy(V.view(np.int16)).to(dev)[None]
+    tQ = torch.from_numpy(Q.view(np.int16)).to(dev)[None]
+    one.laser_kv_select_block(1, tK, tV, tQ, 4)
+    one.laser_kv_poll_status()
+    Kc1, Vc1, p1, n1 = one.laser_kv_cache_view(1)
+    assert n1 == 4 * B and one.laser_kv_cache_view(0)[3] == 0
+    prev = None
+    for t in range(4):
+        sl = slice(t * 256, (t + 1) * 256)
+        inc.laser_kv_select_block(1, tK[:, :, sl], tV[:, :, sl], tQ, 1)
+        inc.laser_kv_poll_status()
+        Kc, Vc, p, n = inc.laser_kv_cache_view(1)
+        assert n == (t + 1) * B
+        snap = (to_np(Kc[:, :, :n]).copy(), to_np(Vc[:, :, :n]).copy(), to_np(p[:, :, :n]).copy())
+        if prev is not None:       # earlier entries never change
+            m = prev[2].shape[2]
+            assert (snap[0][:, :, :m] == prev[0]).all() and (snap[1][:, :, :m] == prev[1]).all()
+            assert (snap[2][:, :, :m] == prev[2]).all()
+        prev = snap
+    assert (prev[0] == to_np(Kc1[:, :, :n1])).all() and (prev[1] == to_np(Vc1[:, :, :n1])).all()
+    assert (prev[2] == to_np(p1[:, :, :n1])).all()
+    with pytest.raises(Bn.LaserKVError) as e:
+        inc.laser_kv_select_block(1, tK[:, :, :256], tV[:, :, :256], tQ, 1)
+    assert e.value.status == Bn.ERR_CAPACITY
+    assert inc.laser_kv_cache_view(1)[3] == 4 * B
+    inc.laser_kv_reset(1)
+    assert inc.laser_kv_cache_view(1)[3] == 0
+
+
+def test_same_inputs_twice_give_identical_bytes():
+    w = synth.workload("tiny").with_(block_size=512, context_len=1024)
+    r1 = run_workload_layer(w, 0)
+    r2 = run_workload_layer(w, 0)
+    for a, b in zip(r1["engine"].laser_kv_cache_view(0)[:3], r2["engine"].laser_kv_cache_view(0)[:3]):
+        n = r1["n_blocks"] * r1["B"]
+        assert (to_np(a[:, :, :n]) == to_np(b[:, :, :n])).all()
+
+
+def test_two_stage_topk_entry_point_against_oracle():
+    import torch
+    from paper_2602_02199_b200 import binding as Bn
+    rng = np.random.default_rng(5)
+    for S, a, ke, kl in ((1024, 100, 150, 60), (8192, 963, 1446, 483), (200, 0, 200, 0), (200, 0, 0, 200),
+                         (333 * 8, 17, 1, 1), (4096, 455, 0, 0), (16384, 2000, 3000, 1000)):
+        n_seg = 5
+        # quantised scores and small integer counts: many exact ties in both stages
+        s = (rng.integers(0, 50, (n_seg, S)) / 64.0).astype(np.float32)
+        s[0] = rng.random(S).astype(np.float32)
+        s[1, :] = 0.25
+        c = rng.integers(0, 7, (n_seg, S)).astype(np.int32)
+        c[2, :] = 3
+        idx = Bn.laser_kv_two_stage_topk(torch.from_numpy(s).cuda(), torch.from_numpy(c).cuda(), a, ke, kl)
+        torch.cuda.synchronize()
+        idx = to_np(idx)
+        for g in range(n_seg):
+            want = O.select_indices(s[g].astype(np.float64), c[g].astype(np.int64), S, a, ke, kl)[2]
+            assert (idx[g] == want).all(), (S, a, ke, kl, g)
+
+
+def test_gather_append_entry_point_bit_exact():
+    import torch
+    from paper_2602_02199_b200 import binding as Bn
+    rng = np.random.default_rng(6)
+    n_seg, rows, cap, keep = 3, 500, 700, 123
+    K = rng.integers(0, 65536, (n_seg, rows, 128)).astype(np.uint16)
+    V = rng.integers(0, 65536, (n_seg, rows, 128)).astype(np.uint16)
+    idx = np.stack([np.sort(rng.choice(rows, keep, replace=False)) for _ in range(n_seg)]).astype(np.int32)
+    Kd = torch.zeros((n_seg, cap, 128), dtype=torch.int16, device="cuda")
+    Vd = torch.zeros_like(Kd)
+    pos = torch.full((n_seg, cap), -1, dtype=torch.int32, device="cuda")
+    Bn.laser_kv_gather_append(torch.from_numpy(K.view(np.int16)).cuda(), torch.from_numpy(V.view(np.int16)).cuda(),
+                              torch.from_numpy(idx).cuda(), Kd, Vd, pos, 200, 5000)
+    torch.cuda.synchronize()
+    Kd, Vd, pos = to_np(Kd).view(np.uint16), to_np(Vd).view(np.uint16), to_np(pos)
+    for g in range(n_seg):
+        assert (Kd[g, 200:200 + keep] == K[g, idx[g]]).all() and (Vd[g, 200:200 + keep] == V[g, idx[g]]).all()
+        assert (pos[g, 200:200 + keep] == 5000 + idx[g]).all()
+        assert (Kd[g, :200] == 0).all() and (Kd[g, 200 + keep:] == 0).all() and (pos[g, :200] == -1).all()
+
+
+def test_headline_config_full_size_sampled_segments():
+    # 128k context, 16 blocks of 8192 in one call (the launch shape the benchmark times); the
+    # oracle checks sampled (head, block) segments in full and the cache of every segment.
+    w = synth.workload("llama8b_128k")
+    run = run_workload_layer(w, 3, debug=1)
+    segs = [(0, 0, 0), (0, 3, 1), (0, 5, 7), (0, 7, 15), (0, 2, 11)]   # blocks holding needles included
+    check_run(w, run, segments=segs)
+
+
+@pytest.mark.parametrize("name,n_blocks,segs", [
+    ("llama8b_32k", 8, [(0, 1, 0), (0, 6, 5)]),
+    ("qwen7b_128k", 6, [(0, 0, 0), (2, 3, 4), (3, 1, 5)]),
+])
+def test_other_configs_sampled_segments(name, n_blocks, segs):
+    w = synth.workload(name)
+    run = run_workload_layer(w, 1, n_blocks=n_blocks)
+    check_run(w, run, segments=segs)
+
+
+def test_64k_config_n_sweep_sampled_segments():
+    for n, seg in ((2, (0, 0, 1)), (4, (0, 4, 0)), (8, (0, 7, 2))):
+        w = synth.workload("llama8b_64k").with_(protection_divisor=n)
+        run = run_workload_layer(w, 2, n_blocks=3)
+        check_run(w, run, segments=[seg])
