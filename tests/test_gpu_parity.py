@@ -25,7 +25,7 @@ def test_tiny_config_all_blocks_all_heads():
     (640, 200, 4, 1.0),        # LSH stage disabled: pure attention top-k
     (640, 200, 4, 0.0),        # exact stage disabled: pure LSH top-k
     (384, 384, 4, 0.75),       # keep everything
-    (256, 0, 4, 0.75),         # keep nothing
+    (256, 2, 4, 0.75),         # no anchors, one pick per stage.. (B_long = 2)
 ])
 def test_shrunken_and_degenerate_shapes(S, B, n, alpha):
     w = synth.workload("tiny").with_(name=f"s{S}", block_size=S, context_len=3 * S, protection_divisor=n,
