@@ -1,0 +1,373 @@
+#!/usr/bin/env python
+"""Benchmark of the LASER-KV prefill-time selection hot path on B200.
+
+A step is one pass of the whole path (query signatures, log-sum-exp pass, score pass,
+projection + collision pass, exact-sign fix-up, two-stage top-k, gather + append) over one layer
+of one 128k-token context: 16 blocks of 8192 tokens in one select call, Llama-3-8B shape
+(32 query heads, 8 KV heads, head_dim 128, window 64, SimHash 10 bits x 64 tables, n = 4).
+Metric: KV tokens scored+compacted per second per layer.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+Prints ONE JSON line. With N > 1 (under torchrun) every rank runs the same job on its own GPU
+with its own seeded inputs (the path has no exchange step: weak scaling, no collective on the
+data path); the time is the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from paper_2602_02199_b200 import synth  # noqa: E402
+
+METRIC = "kv_tokens_scored_and_compacted_per_s_per_layer"
+UNIT = "tokens/s"
+
+# DRAM bytes (read + write) of one launch of the dominant kernel from an ncu capture, keyed by
+# workload; see profiles/. None = not captured for this workload.
+NCU_TRAFFIC_BYTES = {}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm=float(p["hbm_gbs"]), tf=float(p["bf16_tflops"]),
+                    tf_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
+    return dict(hbm=6650.0, tf=1590.0, tf_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        rows = [l for (t, l) in self.lines if t0 - 0.05 <= t <= t1 + 0.15] or [l for (_, l) in self.lines]
+        for l in rows:
+            f = [x.strip() for x in l.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def algorithmic_work(w: synth.Workload, B: int):
+    """Per step (one layer, all blocks, all sequences): bytes the method must move and flops of
+    each contraction counted once."""
+    d, S, nb = w.head_dim, w.block_size, w.n_blocks
+    hk, hq, W = w.n_kv_heads, w.n_q_heads, w.window
+    planes = w.lsh_bits * w.lsh_tables
+    tokens = w.batch * nb * S
+    k_bytes = tokens * hk * d * 2
+    sel = w.batch * nb * hk * B * d * 2
+    bytes_alg = k_bytes + w.batch * hq * W * d * 2 + planes * d * 2 + 3 * sel + w.batch * nb * hk * B * 4
+    fl_score = 2.0 * w.batch * nb * hq * W * S * d
+    fl_proj = 2.0 * w.batch * nb * hk * S * planes * d
+    fl_q = 2.0 * w.batch * hq * W * planes * d
+    return dict(tokens=tokens, bytes=bytes_alg, flops=fl_score + fl_proj + fl_q, fl_score=fl_score, fl_proj=fl_proj,
+                gather_bytes=4 * sel)
+
+
+# ----------------------------------------------------------------------------------------------
+# reference arm: the CPU oracle, as it stands, on a bounded sample of the same workload
+# ----------------------------------------------------------------------------------------------
+def oracle_sample_step(w, k_blk, q, P, heads, B):
+    from oracle import laser_kv_oracle as O
+    hk = len(heads)
+    G = w.group
+    kb = k_blk[heads]
+    qb = np.concatenate([q[h * G:(h + 1) * G] for h in heads])
+    return O.select_block(kb, qb, P, n_bits=w.lsh_bits, n_tables=w.lsh_tables, B=B, n=w.protection_divisor,
+                          alpha=w.alpha)
+
+
+def time_oracle(w, steps, warmup, target_s=1.5):
+    """Times the oracle on `heads_per_step` KV heads of one block per step; returns tokens/s where a
+    block counts as S tokens only when all H_kv heads were processed."""
+    from oracle import laser_kv_oracle as O
+    B = O.budget(w.context_len, w.block_size, w.ratio)
+    k_blk, v_blk = synth.kv_block(w, 0, 0, 1)
+    q, P = synth.q_window(w, 0, 0), synth.hyperplanes(w)
+    t0 = time.perf_counter()
+    oracle_sample_step(w, k_blk, q, P, [0], B)
+    one = time.perf_counter() - t0
+    heads_per_step = int(max(1, min(w.n_kv_heads, round(target_s / max(one, 1e-3)))))
+    heads = list(range(heads_per_step))
+    for _ in range(warmup):
+        oracle_sample_step(w, k_blk, q, P, heads, B)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        r = oracle_sample_step(w, k_blk, q, P, heads, B)
+        cache = O.AppendOnlyCache(len(heads), w.head_dim, B)
+        cache.append(k_blk[heads], v_blk[heads], r.idx, w.block_size)
+    dt = (time.perf_counter() - t0) / steps
+    tokens_per_step = w.block_size * heads_per_step / w.n_kv_heads
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    sample = (f"{heads_per_step} of {w.n_kv_heads} KV heads of one {w.block_size}-token block per step "
+              f"(block 1 of {w.n_blocks}, layer 0); a block counts as {w.block_size} tokens when all heads are done")
+    return tokens_per_step / dt, dt, cores, sample
+
+
+def run_reference(args, w, rank, world):
+    if rank != 0:
+        return
+    steps = max(1, min(args.steps, 40))
+    value, dt, cores, sample = time_oracle(w, steps, min(args.warmup, 3))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": min(args.warmup, 3), "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "context_len": w.context_len, "block_size": w.block_size,
+                   "note": "CPU oracle (numpy fp64) timed on the host cores; bounded sample per step"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------------------------
+# our arm
+# ----------------------------------------------------------------------------------------------
+def run_ours(args, w, rank, world, local_rank):
+    import torch
+    import torch.distributed as dist
+    from paper_2602_02199_b200 import binding as Bn
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    S, nb, d = w.block_size, w.n_blocks, w.head_dim
+    B = Bn.laser_kv_budget(w.context_len, S, w.ratio)
+    n_sets = args.input_sets          # distinct layers cycled through so inputs exceed L2
+    host = []
+    for i in range(n_sets):
+        layer = rank * n_sets + i
+        Ks, Vs, Qs = [], [], []
+        for b in range(w.batch):
+            k, v = synth.kv_blocks(w, layer, b, 0, nb)
+            Ks.append(k); Vs.append(v); Qs.append(synth.q_window(w, layer, b))
+        hk = torch.from_numpy(np.stack(Ks).view(np.int16)).pin_memory()
+        hv = torch.from_numpy(np.stack(Vs).view(np.int16)).pin_memory()
+        hq = torch.from_numpy(np.stack(Qs).view(np.int16)).pin_memory()
+        host.append((hk, hv, hq))
+    devs = [(a.to(dev), b.to(dev), c.to(dev)) for (a, b, c) in host]
+    P = torch.from_numpy(synth.hyperplanes(w).view(np.int16)).to(dev)
+    cfg = Bn.make_config(n_layers=n_sets, batch=w.batch, n_q_heads=w.n_q_heads, n_kv_heads=w.n_kv_heads,
+                         block_size=S, window=w.window, max_blocks=nb, max_blocks_per_call=nb, lsh_bits=w.lsh_bits,
+                         lsh_tables=w.lsh_tables, protection_divisor=w.protection_divisor, budget_per_block=B,
+                         alpha=w.alpha, device=local_rank)
+    eng = Bn.LaserKV(cfg, P)
+    work = algorithmic_work(w, B)
+
+    def step(i):
+        s = i % n_sets
+        eng.laser_kv_reset(s)
+        eng.laser_kv_select_block(s, devs[s][0], devs[s][1], devs[s][2], nb)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(i)
+    eng.laser_kv_poll_status()
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    eng.laser_kv_profile_enable(True)
+    launches0 = Bn.laser_kv_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t_wall0 = time.time()
+    e0.record()
+    for i in range(args.steps):
+        step(i)
+    e1.record()
+    barrier()
+    t_wall1 = time.time()
+    ms = e0.elapsed_time(e1)
+    launches = Bn.laser_kv_launch_count() - launches0
+    prof = eng.laser_kv_profile_read()
+    eng.laser_kv_profile_enable(False)
+    eng.laser_kv_poll_status()
+    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
+
+    # ---- end to end: pinned host inputs -> device, select, appended positions -> host ----
+    stage = tuple(torch.empty_like(t) for t in devs[0])
+    pos_host = torch.empty((w.batch, w.n_kv_heads, nb * B), dtype=torch.int32).pin_memory()
+    e2e_steps = max(1, min(args.steps, args.e2e_steps))
+
+    def e2e_step(i):
+        s = i % n_sets
+        eng.laser_kv_reset(s)
+        eng.laser_kv_select_block_host(s, host[s][0], host[s][1], host[s][2], stage[0], stage[1], stage[2], nb,
+                                       pos_host)
+
+    e2e_step(0)
+    barrier()
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    f0.record()
+    for i in range(e2e_steps):
+        e2e_step(i)
+    f1.record()
+    barrier()
+    e2e_ms = f0.elapsed_time(f1)
+    eng.laser_kv_poll_status()
+    assert int(pos_host[0, 0, 0]) == 0 and int(pos_host[0, 0, -1]) == w.context_len - 1
+
+    t = torch.tensor([ms, e2e_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms, e2e_ms = float(t[0]), float(t[1])
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = load_peaks()
+    ms_per_step = ms / args.steps
+    value = world * work["tokens"] * args.steps / (ms * 1e-3)
+    e2e_value = world * work["tokens"] * e2e_steps / (e2e_ms * 1e-3)
+    h2d = sum(int(x.numel()) * 2 for x in host[0])
+    d2h = int(pos_host.numel()) * 4
+
+    # dominant kernel and its roofline
+    kern = {k: v for k, v in prof.items() if v[1] > 0}
+    total_kernel_ms = sum(v[0] for v in kern.values())
+    dom = max(kern, key=lambda k: kern[k][0])
+    dom_ms = kern[dom][0] / kern[dom][1]
+    fl = {"stream_kernel<proj>": work["fl_proj"], "stream_kernel<score>": work["fl_score"],
+          "stream_kernel<lse>": work["fl_score"]}
+    if dom in fl:
+        achieved = fl[dom] / (dom_ms * 1e-3) / 1e12
+        roof = {"kernel": dom, "bound": "tensor", "achieved": achieved, "peak": peaks["tf"], "unit": "TFLOP/s",
+                "frac": achieved / peaks["tf"], "traffic": NCU_TRAFFIC_BYTES.get(w.name),
+                "peak_source": f"bf16_tflops (burst), {peaks['source']}",
+                "flops_per_launch": fl[dom], "ms_per_launch": dom_ms}
+    else:
+        gb = work["gather_bytes"] if dom == "append_kernel" else work["bytes"]
+        achieved = gb / (dom_ms * 1e-3) / 1e9
+        roof = {"kernel": dom, "bound": "hbm", "achieved": achieved, "peak": peaks["hbm"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm"], "traffic": NCU_TRAFFIC_BYTES.get(w.name),
+                "peak_source": f"hbm_gbs, {peaks['source']}", "bytes_per_launch": gb, "ms_per_launch": dom_ms}
+    t_hbm = work["bytes"] / (peaks["hbm"] * 1e9)
+    t_tensor = work["flops"] / (peaks["tf"] * 1e12)
+    path = {
+        "hbm_frac": t_hbm / (ms_per_step * 1e-3), "tensor_frac": t_tensor / (ms_per_step * 1e-3),
+        "binding_frac": max(t_hbm, t_tensor) / (ms_per_step * 1e-3),
+        "bytes_alg_per_step": work["bytes"], "flops_alg_per_step": work["flops"],
+        "kernels_ms_per_step": {k: v[0] / v[1] for k, v in kern.items()},
+        "kernel_share": {k: v[0] / total_kernel_ms for k, v in kern.items()},
+    }
+
+    cpu_value, cpu_dt, cores, sample = time_oracle(w, steps=max(1, args.cpu_steps), warmup=1)
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "context_len": w.context_len, "block_size": S, "blocks_per_call": nb,
+                   "batch": w.batch, "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads, "window": w.window,
+                   "lsh_bits": w.lsh_bits, "lsh_tables": w.lsh_tables, "protection_divisor": w.protection_divisor,
+                   "budget_per_block": B, "alpha": w.alpha,
+                   "l2": f"inputs larger than L2: {n_sets} layers of K+V ({2 * host[0][0].numel() * 2 >> 20} MiB each) cycled",
+                   "parallelism": "replicas" if world > 1 else "single"},
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps},
+        "gpu_launches": int(launches),
+        "roofline": roof,
+        "path_roofline": path,
+        "cpu_baseline": {"value": cpu_value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama8b_128k", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--input-sets", type=int, default=2)
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--cpu-steps", type=int, default=6)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    w = synth.workload(args.workload)
+    if args.impl == "reference":
+        run_reference(args, w, rank, world)
+    else:
+        run_ours(args, w, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

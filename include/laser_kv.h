@@ -52,8 +52,8 @@ typedef struct {
   int32_t window;              /* W: observation-window queries per query head                   */
   int32_t max_blocks;          /* cache capacity per (layer, sequence, KV head) = max_blocks * B */
   int32_t max_blocks_per_call; /* upper bound on n_blocks of one select call (sizes workspace)   */
-  int32_t lsh_bits;            /* K: sign bits per SimHash table, 1..12                          */
-  int32_t lsh_tables;          /* L: number of tables (the paper's R hash rounds)                */
+  int32_t lsh_bits;            /* K: sign bits per SimHash table: 4, 6, 8, 10 or 12               */
+  int32_t lsh_tables;          /* L: tables (the paper's R hash rounds); a multiple of 8          */
   int32_t protection_divisor;  /* n >= 2 (Section 3.1)                                           */
   int32_t budget_per_block;    /* B; 0 => Eq. 1 from ratio, block_size and context_len           */
   int32_t debug;               /* nonzero: also keep per-key bucket ids for laser_kv_debug_view  */
@@ -77,7 +77,9 @@ typedef struct {
 } laser_kv_view_t;
 
 /* Intermediate results of the most recent select call (pointers into the workspace, valid
- * until the next select call). nb = that call's n_blocks; GW = G*W. */
+ * until the next select call). nb = that call's n_blocks; GW = G*W. A bucket code packs a table's
+ * K sign bits with the table's first hyperplane as the most significant bit:
+ * code = sum_b [<p_{r*K+b}, x> >= 0] << (K-1-b). hist is indexed by that code. */
 typedef struct {
   const float*    s_exact;       /* dev fp32  [batch][H_kv][nb][S]   summed window attention     */
   const uint32_t* counts;        /* dev u32   [batch][H_kv][nb][S]   collision counts            */
@@ -170,6 +172,16 @@ const char* laser_kv_last_error(laser_kv_handle_t h);
 
 /* Number of this library's kernels launched by the calling process so far (all handles). */
 int64_t laser_kv_launch_count(void);
+
+/* Optional per-kernel timing. When enabled, every select call records CUDA events on the caller's
+ * stream between its kernels (no synchronisation, no device memory). laser_kv_profile_read waits
+ * for the recorded events, adds the elapsed times to per-kernel totals and reports them:
+ * names[i] is a static string, total_ms[i] the accumulated device time and launches[i] the number
+ * of launches of kernel i since profiling was enabled; *n_kernels is set to the number of entries
+ * (at most 16; pass arrays of 16). Enabling resets the totals. */
+laser_kv_status_t laser_kv_profile_enable(laser_kv_handle_t h, int32_t on);
+laser_kv_status_t laser_kv_profile_read(laser_kv_handle_t h, int32_t* n_kernels, const char** names,
+                                        float* total_ms, int32_t* launches);
 
 /* ---- step-level entry points (same kernels as the hot path, caller-fed inputs) ------------- */
 

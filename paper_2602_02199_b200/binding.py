@@ -15,7 +15,8 @@ EXPORTS = [
     "laser_kv_select_block", "laser_kv_select_block_host", "laser_kv_cache_view",
     "laser_kv_debug_view", "laser_kv_poll_status", "laser_kv_reset", "laser_kv_destroy",
     "laser_kv_status_string", "laser_kv_last_error", "laser_kv_launch_count",
-    "laser_kv_two_stage_topk", "laser_kv_gather_append",
+    "laser_kv_two_stage_topk", "laser_kv_gather_append", "laser_kv_profile_enable",
+    "laser_kv_profile_read",
 ]
 
 
@@ -106,6 +107,10 @@ def load(build_if_missing: bool = True) -> C.CDLL:
     lib.laser_kv_two_stage_topk.argtypes = [vp, vp, i32, i32, i32, i32, i32, vp, vp]
     lib.laser_kv_gather_append.restype = i32
     lib.laser_kv_gather_append.argtypes = [vp, vp, i64, i64, vp, i32, i32, vp, vp, i64, vp, i64, i64, i32, vp]
+    lib.laser_kv_profile_enable.restype = i32
+    lib.laser_kv_profile_enable.argtypes = [vp, i32]
+    lib.laser_kv_profile_read.restype = i32
+    lib.laser_kv_profile_read.argtypes = [vp, p(i32), p(C.c_char_p), p(C.c_float), p(i32)]
     _lib = lib
     return lib
 
@@ -267,6 +272,18 @@ class LaserKV:
 
     def laser_kv_poll_status(self, stream=None):
         _check(self.lib.laser_kv_poll_status(self.handle, _stream_ptr(stream)), self.handle)
+
+    def laser_kv_profile_enable(self, on=True):
+        _check(self.lib.laser_kv_profile_enable(self.handle, 1 if on else 0), self.handle)
+
+    def laser_kv_profile_read(self):
+        """-> {kernel name: (total device ms, launches)} since profiling was enabled."""
+        n = C.c_int32()
+        names = (C.c_char_p * 16)()
+        ms = (C.c_float * 16)()
+        cnt = (C.c_int32 * 16)()
+        _check(self.lib.laser_kv_profile_read(self.handle, C.byref(n), names, ms, cnt), self.handle)
+        return {names[i].decode(): (float(ms[i]), int(cnt[i])) for i in range(n.value)}
 
     def laser_kv_reset(self, layer=-1):
         _check(self.lib.laser_kv_reset(self.handle, layer), self.handle)

@@ -26,6 +26,10 @@ constexpr int kHeadDim = 128;
 constexpr size_t kAlign = 256;
 constexpr int kMaxSmem = 227 * 1024;
 
+constexpr int kProfKernels = 8;
+const char* const kProfNames[kProfKernels] = {"memset", "qprep_kernel", "stream_kernel<lse>", "stream_kernel<score>",
+                                              "stream_kernel<proj>", "signfix_kernel", "select_kernel", "append_kernel"};
+
 std::atomic<long long> g_launches{0};
 thread_local std::string g_last_error;
 
@@ -69,6 +73,12 @@ struct laser_kv_ctx {
   bool have_call = false;
   int last_nb = 0;
   int last_fixups = 0;
+  // optional per-kernel timing (events only; no device memory)
+  bool profiling = false;
+  std::vector<cudaEvent_t> ev_pool;
+  std::vector<std::vector<cudaEvent_t>> ev_pending;
+  float prof_ms[kProfKernels] = {0};
+  int prof_launches[kProfKernels] = {0};
 };
 
 namespace {
@@ -428,10 +438,21 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
 #define LKV_CUDA(call, what)                                                                   \
   if ((e = (call)) != cudaSuccess) return fail(h, LASER_KV_ERR_CUDA, "select_block: %s: %s", what, cudaGetErrorString(e))
 
+  std::vector<cudaEvent_t> marks;
+  auto mark = [&]() {
+    if (!h->profiling) return;
+    cudaEvent_t ev;
+    if (!h->ev_pool.empty()) { ev = h->ev_pool.back(); h->ev_pool.pop_back(); }
+    else if (cudaEventCreate(&ev) != cudaSuccess) return;
+    cudaEventRecord(ev, st);
+    marks.push_back(ev);
+  };
+  mark();
   // fix-up counter (ctrl[1]) and changed counter (ctrl[2]) restart; the status word (ctrl[0]) is kept
   LKV_CUDA(cudaMemsetAsync(ctrl + 1, 0, 8, st), "memset ctrl");
   LKV_CUDA(cudaMemsetAsync(counts, 0, (size_t)nseg * S * 4, st), "memset counts");
 
+  mark();
   // 1. query signatures and bucket histogram
   {
     QprepArgs qa{static_cast<const uint16_t*>(Q_win), q_strides[0], q_strides[1], q_strides[2], h->P, hist, qb,
@@ -455,6 +476,7 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
   sa.status = ctrl;
 
   const int base_ctas = c.batch * c.n_kv_heads * nb * d.n_split;
+  mark();
   // 2. per-query log-sum-exp over each block's keys
   {
     StreamArgs a1 = sa;
@@ -463,6 +485,7 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
     const uint32_t smem = stream_smem_bytes(kLse, a1.stat_rows_alloc, 0, d.GW);
     LKV_CUDA((launch_stream<kLse, 0, 0>(mapK, mapQ, a1, base_ctas, smem, st)), "lse pass");
   }
+  mark();
   // 3. summed attention probabilities per key
   {
     StreamArgs a2 = sa;
@@ -471,6 +494,7 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
     const uint32_t smem = stream_smem_bytes(kScore, a2.stat_rows_alloc, 0, d.GW);
     LKV_CUDA((launch_stream<kScore, 0, 0>(mapK, mapQ, a2, base_ctas, smem, st)), "score pass");
   }
+  mark();
   // 4. key signatures and collision counts
   {
     StreamArgs a3 = sa;
@@ -479,6 +503,7 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
     const uint32_t smem = stream_smem_bytes(kProj, a3.stat_rows_alloc, d.TC * (2 << c.lsh_bits), 0);
     LKV_CUDA(launch_proj(c.lsh_bits, d.TC, mapK, h->mapP, a3, base_ctas * d.n_chunks, smem, st), "projection pass");
   }
+  mark();
   // 5. exact signs where the tensor-core projection was too close to zero
   {
     SignfixArgs fa{static_cast<const uint16_t*>(K_blk), kv_strides[0], kv_strides[1], kv_strides[2], h->P, hist,
@@ -488,11 +513,13 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
     g_launches.fetch_add(1);
     LKV_CUDA(cudaGetLastError(), "signfix_kernel");
   }
+  mark();
   // 6. two-stage top-k
   {
     const laser_kv_status_t s = launch_select(s_exact, counts, nseg, S, d.anchors, d.k_exact, d.k_lsh, idx, st);
     if (s != LASER_KV_OK) { h->last_error = g_last_error; return s; }
   }
+  mark();
   // 7. gather + append
   {
     const long long done = h->blocks_done[layer];
@@ -505,6 +532,9 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
     if (s != LASER_KV_OK) { h->last_error = g_last_error; return s; }
   }
 #undef LKV_CUDA
+  mark();
+  if (h->profiling && marks.size() == kProfKernels + 1) h->ev_pending.push_back(marks);
+  else for (cudaEvent_t ev : marks) h->ev_pool.push_back(ev);
   h->blocks_done[layer] += nb;
   h->have_call = true;
   h->last_nb = nb;
@@ -616,7 +646,40 @@ laser_kv_status_t laser_kv_reset(laser_kv_handle_t h, int32_t layer) {
   return LASER_KV_OK;
 }
 
-void laser_kv_destroy(laser_kv_handle_t h) { delete h; }
+void laser_kv_destroy(laser_kv_handle_t h) {
+  if (!h) return;
+  for (auto& set : h->ev_pending) for (cudaEvent_t ev : set) cudaEventDestroy(ev);
+  for (cudaEvent_t ev : h->ev_pool) cudaEventDestroy(ev);
+  delete h;
+}
+
+laser_kv_status_t laser_kv_profile_enable(laser_kv_handle_t h, int32_t on) {
+  if (!h) return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "profile_enable: NULL handle");
+  for (auto& set : h->ev_pending) for (cudaEvent_t ev : set) h->ev_pool.push_back(ev);
+  h->ev_pending.clear();
+  for (int i = 0; i < kProfKernels; ++i) { h->prof_ms[i] = 0.f; h->prof_launches[i] = 0; }
+  h->profiling = on != 0;
+  return LASER_KV_OK;
+}
+
+laser_kv_status_t laser_kv_profile_read(laser_kv_handle_t h, int32_t* n_kernels, const char** names, float* total_ms,
+                                        int32_t* launches) {
+  if (!h || !n_kernels || !names || !total_ms || !launches)
+    return fail(h, LASER_KV_ERR_INVALID_ARG, "profile_read: NULL argument");
+  for (auto& set : h->ev_pending) {
+    cudaError_t e = cudaEventSynchronize(set.back());
+    if (e != cudaSuccess) return fail(h, LASER_KV_ERR_CUDA, "profile_read: %s", cudaGetErrorString(e));
+    for (int i = 0; i < kProfKernels; ++i) {
+      float ms = 0.f;
+      if (cudaEventElapsedTime(&ms, set[i], set[i + 1]) == cudaSuccess) { h->prof_ms[i] += ms; h->prof_launches[i] += 1; }
+    }
+    for (cudaEvent_t ev : set) h->ev_pool.push_back(ev);
+  }
+  h->ev_pending.clear();
+  *n_kernels = kProfKernels;
+  for (int i = 0; i < kProfKernels; ++i) { names[i] = kProfNames[i]; total_ms[i] = h->prof_ms[i]; launches[i] = h->prof_launches[i]; }
+  return LASER_KV_OK;
+}
 
 const char* laser_kv_status_string(laser_kv_status_t s) {
   switch (s) {
