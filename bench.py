@@ -255,9 +255,10 @@ def run_ours(args, w, rank, world, local_rank):
     clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
 
     # ---- end to end: pinned host inputs -> device, select, appended positions -> host ----
-    stage = tuple(torch.empty_like(t) for t in devs[0])
-    pos_host = torch.empty((w.batch, w.n_kv_heads, nb * B), dtype=torch.int32).pin_memory()
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
+    e2e_ms = float("nan")
+    pos_host = torch.empty((w.batch, w.n_kv_heads, nb * B), dtype=torch.int32).pin_memory()
+    stage = None if args.skip_e2e else tuple(torch.empty_like(t) for t in devs[0])
 
     def e2e_step(i):
         s = i % n_sets
@@ -265,17 +266,18 @@ def run_ours(args, w, rank, world, local_rank):
         eng.laser_kv_select_block_host(s, host[s][0], host[s][1], host[s][2], stage[0], stage[1], stage[2], nb,
                                        pos_host)
 
-    e2e_step(0)
-    barrier()
-    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    f0.record()
-    for i in range(e2e_steps):
-        e2e_step(i)
-    f1.record()
-    barrier()
-    e2e_ms = f0.elapsed_time(f1)
-    eng.laser_kv_poll_status()
-    assert int(pos_host[0, 0, 0]) == 0 and int(pos_host[0, 0, -1]) == w.context_len - 1
+    if not args.skip_e2e:
+        e2e_step(0)
+        barrier()
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record()
+        for i in range(e2e_steps):
+            e2e_step(i)
+        f1.record()
+        barrier()
+        e2e_ms = f0.elapsed_time(f1)
+        eng.laser_kv_poll_status()
+        assert int(pos_host[0, 0, 0]) == 0 and int(pos_host[0, 0, -1]) == w.context_len - 1
 
     t = torch.tensor([ms, e2e_ms], dtype=torch.float64, device=dev)
     if world > 1:
@@ -322,7 +324,10 @@ def run_ours(args, w, rank, world, local_rank):
         "kernel_share": {k: v[0] / total_kernel_ms for k, v in kern.items()},
     }
 
-    cpu_value, cpu_dt, cores, sample = time_oracle(w, steps=max(1, args.cpu_steps), warmup=1)
+    if args.skip_cpu:
+        cpu_value, cores, sample = None, 0, "skipped (--skip-cpu)"
+    else:
+        cpu_value, _, cores, sample = time_oracle(w, steps=max(1, args.cpu_steps), warmup=1)
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -350,13 +355,15 @@ def run_ours(args, w, rank, world, local_rank):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama8b_128k", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--input-sets", type=int, default=2)
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--cpu-steps", type=int, default=6)
+    ap.add_argument("--skip-cpu", action="store_true", help="omit the oracle timing (profiling runs)")
+    ap.add_argument("--skip-e2e", action="store_true", help="omit the host-buffer timing (profiling runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     rank = int(os.environ.get("RANK", "0"))

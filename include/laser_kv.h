@@ -197,6 +197,26 @@ laser_kv_status_t laser_kv_two_stage_topk(const float* s_exact, const uint32_t* 
                                           int32_t k_exact, int32_t k_lsh, int32_t* idx_out,
                                           void* stream);
 
+/* Step 1 of the path alone (Section 3.3 "Precision", Algorithm 1 line 3, per layer and KV head):
+ * S_exact[b][h][t][j] = sum over the window queries (g, w) of KV head h's group of
+ * softmax_j(<q_{g,w}, k_j> * scale), the softmax taken over the S keys of block t.
+ *   K_blk, Q_win, kv_strides, q_strides, n_blocks : as for laser_kv_select_block.
+ *   softmax_scale : 0 => 1/sqrt(128).
+ *   scratch       : dev, 256-byte aligned, at least laser_kv_window_scores_scratch_bytes(...) bytes,
+ *                   owned by the caller; holds the per-query log-sum-exp partials between the two
+ *                   kernels. Its first int is a status word (0, or LASER_KV_ERR_TIMEOUT if a bounded
+ *                   device-side wait gave up).
+ *   s_exact_out   : dev fp32 [batch][H_kv][n_blocks][S].
+ * head_dim is 128; G*W must be a multiple of 16 and at most 256. */
+size_t laser_kv_window_scores_scratch_bytes(int32_t batch, int32_t n_q_heads, int32_t n_kv_heads,
+                                            int32_t block_size, int32_t window, int32_t n_blocks);
+laser_kv_status_t laser_kv_window_scores(const void* K_blk, const void* Q_win,
+                                         const int64_t kv_strides[3], const int64_t q_strides[3],
+                                         int32_t batch, int32_t n_q_heads, int32_t n_kv_heads,
+                                         int32_t block_size, int32_t window, int32_t n_blocks,
+                                         float softmax_scale, void* scratch, size_t scratch_bytes,
+                                         float* s_exact_out, void* stream);
+
 /* Append step (Sections 1 and 3): for each of n_segments segments copies rows idx[seg][i] of the
  * segment's K and V (dev bf16, row length d = 128, consecutive rows `src_row_stride` elements
  * apart, segment s starting at src + s*src_seg_stride) to dst rows [dst_offset + i] of the

@@ -16,7 +16,7 @@ EXPORTS = [
     "laser_kv_debug_view", "laser_kv_poll_status", "laser_kv_reset", "laser_kv_destroy",
     "laser_kv_status_string", "laser_kv_last_error", "laser_kv_launch_count",
     "laser_kv_two_stage_topk", "laser_kv_gather_append", "laser_kv_profile_enable",
-    "laser_kv_profile_read",
+    "laser_kv_profile_read", "laser_kv_window_scores", "laser_kv_window_scores_scratch_bytes",
 ]
 
 
@@ -111,6 +111,11 @@ def load(build_if_missing: bool = True) -> C.CDLL:
     lib.laser_kv_profile_enable.argtypes = [vp, i32]
     lib.laser_kv_profile_read.restype = i32
     lib.laser_kv_profile_read.argtypes = [vp, p(i32), p(C.c_char_p), p(C.c_float), p(i32)]
+    lib.laser_kv_window_scores_scratch_bytes.restype = sz
+    lib.laser_kv_window_scores_scratch_bytes.argtypes = [i32] * 6
+    lib.laser_kv_window_scores.restype = i32
+    lib.laser_kv_window_scores.argtypes = [vp, vp, p(i64), p(i64), i32, i32, i32, i32, i32, i32, C.c_float, vp, sz,
+                                           vp, vp]
     _lib = lib
     return lib
 
@@ -307,3 +312,26 @@ def laser_kv_gather_append(K_src, V_src, idx, K_dst, V_dst, pos_out, dst_offset,
     _check(load().laser_kv_gather_append(_ptr(K_src), _ptr(V_src), K_src.stride(0), K_src.stride(1), _ptr(idx),
                                          n_seg, n_keep, _ptr(K_dst), _ptr(V_dst), K_dst.stride(0), _ptr(pos_out),
                                          pos_out.stride(0), dst_offset, pos_base, _stream_ptr(stream)))
+
+
+def laser_kv_window_scores_scratch_bytes(batch, n_q_heads, n_kv_heads, block_size, window, n_blocks) -> int:
+    return int(load().laser_kv_window_scores_scratch_bytes(batch, n_q_heads, n_kv_heads, block_size, window, n_blocks))
+
+
+def laser_kv_window_scores(K_blk, Q_win, block_size, n_blocks, softmax_scale=0.0, scratch=None, stream=None):
+    """K_blk [batch][H_kv][n_blocks*S][128], Q_win [batch][H_q][W][128] (2-byte device tensors) ->
+    S_exact fp32 [batch][H_kv][n_blocks][S]. `scratch` (uint8 device tensor) is allocated by torch
+    when not given."""
+    import torch
+    batch, h_kv = K_blk.shape[0], K_blk.shape[1]
+    h_q, window = Q_win.shape[1], Q_win.shape[2]
+    need = laser_kv_window_scores_scratch_bytes(batch, h_q, h_kv, block_size, window, n_blocks)
+    if scratch is None:
+        scratch = torch.empty(max(need, 256), dtype=torch.uint8, device=K_blk.device)
+    out = torch.empty((batch, h_kv, n_blocks, block_size), dtype=torch.float32, device=K_blk.device)
+    ks = (C.c_int64 * 3)(*K_blk.stride()[:3])
+    qs = (C.c_int64 * 3)(*Q_win.stride()[:3])
+    _check(load().laser_kv_window_scores(_ptr(K_blk), _ptr(Q_win), ks, qs, batch, h_q, h_kv, block_size, window,
+                                         n_blocks, softmax_scale, _ptr(scratch), scratch.numel(), _ptr(out),
+                                         _stream_ptr(stream)))
+    return out

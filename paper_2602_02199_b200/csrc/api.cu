@@ -712,6 +712,144 @@ laser_kv_status_t laser_kv_two_stage_topk(const float* s_exact, const uint32_t* 
   return launch_select(s_exact, counts, n_segments, S, anchors, k_exact, k_lsh, idx_out, static_cast<cudaStream_t>(stream));
 }
 
+// ---- window scores on caller-fed inputs ----------------------------------------------------------
+namespace {
+
+struct ScoreGeom {
+  int batch, H_q, H_kv, S, W, nb, G, GW, tiles_in_block, tiles_per_cta, n_split, nseg;
+  float scale;
+  size_t off_part, off_lse2, total;   // scratch layout: [0,256) status word, partials, lse2
+};
+
+laser_kv_status_t score_geometry(int32_t batch, int32_t n_q_heads, int32_t n_kv_heads, int32_t block_size,
+                                 int32_t window, int32_t n_blocks, float softmax_scale, ScoreGeom* g) {
+  if (batch < 1 || n_q_heads < 1 || n_kv_heads < 1 || block_size < 1 || window < 1 || n_blocks < 1)
+    return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "window_scores: sizes must be positive");
+  if (n_q_heads % n_kv_heads) return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "window_scores: n_q_heads %% n_kv_heads != 0");
+  g->batch = batch; g->H_q = n_q_heads; g->H_kv = n_kv_heads; g->S = block_size; g->W = window; g->nb = n_blocks;
+  g->G = n_q_heads / n_kv_heads;
+  g->GW = g->G * window;
+  if (g->GW % 16 || g->GW > 256 || window > 256 || block_size % 8)
+    return fail(nullptr, LASER_KV_ERR_UNSUPPORTED, "window_scores: G*W must be a multiple of 16, at most 256; block_size a multiple of 8");
+  const long long nseg = (long long)batch * n_kv_heads * n_blocks;
+  if (nseg > (1 << 22) || (long long)n_blocks * block_size > 0x7fffffffLL)
+    return fail(nullptr, LASER_KV_ERR_UNSUPPORTED, "window_scores: too many segments");
+  g->nseg = (int)nseg;
+  g->tiles_in_block = (block_size + kTileKeys - 1) / kTileKeys;
+  g->tiles_per_cta = g->tiles_in_block < 16 ? g->tiles_in_block : 16;
+  g->n_split = (g->tiles_in_block + g->tiles_per_cta - 1) / g->tiles_per_cta;
+  g->scale = softmax_scale == 0.f ? 1.0f / std::sqrt((float)kHeadDim) : softmax_scale;
+  g->off_part = 256;
+  g->off_lse2 = align_up(g->off_part + (size_t)g->nseg * g->n_split * g->GW * sizeof(float2));
+  g->total = align_up(g->off_lse2 + (size_t)g->nseg * g->GW * 4);
+  return LASER_KV_OK;
+}
+
+EncodeTiledFn driver_encode_fn() {
+  static EncodeTiledFn cached = nullptr;
+  if (cached) return cached;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess)
+    return nullptr;
+  cached = reinterpret_cast<EncodeTiledFn>(fn);
+  return cached;
+}
+
+// Log-sum-exp pass then score pass, with the partials in `scratch` (device, g.total bytes).
+laser_kv_status_t run_window_scores(const ScoreGeom& g, const void* K_blk, const void* Q_win, const int64_t kv_strides[3],
+                                    const int64_t q_strides[3], uint8_t* scratch, float* s_exact_out, cudaStream_t st) {
+  if (!K_blk || !Q_win || !kv_strides || !q_strides || !s_exact_out)
+    return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "window_scores: NULL argument");
+  if (!aligned16(K_blk) || !aligned16(Q_win) || !aligned16(s_exact_out))
+    return fail(nullptr, LASER_KV_ERR_ALIGNMENT, "window_scores: device pointers must be 16-byte aligned");
+  for (int i = 0; i < 3; ++i)
+    if (kv_strides[i] < 0 || q_strides[i] < 0 || (kv_strides[i] % 8) || (q_strides[i] % 8))
+      return fail(nullptr, LASER_KV_ERR_ALIGNMENT, "window_scores: strides must be non-negative multiples of 8 elements");
+  if (kv_strides[2] < kHeadDim || q_strides[2] < kHeadDim || (g.H_kv > 1 && !kv_strides[1]) || (g.batch > 1 && !kv_strides[0]) ||
+      (g.H_q > 1 && !q_strides[1]) || (g.batch > 1 && !q_strides[0]))
+    return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "window_scores: bad strides");
+  EncodeTiledFn enc = driver_encode_fn();
+  if (!enc) return fail(nullptr, LASER_KV_ERR_CUDA, "window_scores: cuTensorMapEncodeTiled not available (no CUDA driver?)");
+  CUtensorMap mapK, mapQ;
+  const cuuint32_t ones[4] = {1, 1, 1, 1};
+  {
+    const cuuint64_t s_tok = (cuuint64_t)kv_strides[2];
+    const cuuint64_t s_head = kv_strides[1] > 0 ? (cuuint64_t)kv_strides[1] : s_tok * (cuuint64_t)g.nb * g.S;
+    const cuuint64_t s_batch = kv_strides[0] > 0 ? (cuuint64_t)kv_strides[0] : s_head * (cuuint64_t)g.H_kv;
+    const cuuint64_t dims[4] = {(cuuint64_t)kHeadDim, (cuuint64_t)g.nb * g.S, (cuuint64_t)g.H_kv, (cuuint64_t)g.batch};
+    const cuuint64_t strides[3] = {s_tok * 2, s_head * 2, s_batch * 2};
+    const cuuint32_t box[4] = {(cuuint32_t)kAtomCols, (cuuint32_t)kTileKeys, 1, 1};
+    const CUresult r = enc(&mapK, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(K_blk), dims, strides, box, ones,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(nullptr, LASER_KV_ERR_CUDA, "window_scores: tensor map of K failed (CUresult %d)", (int)r);
+  }
+  {
+    const cuuint64_t s_w = (cuuint64_t)q_strides[2];
+    const cuuint64_t s_head = q_strides[1] > 0 ? (cuuint64_t)q_strides[1] : s_w * (cuuint64_t)g.W;
+    const cuuint64_t s_batch = q_strides[0] > 0 ? (cuuint64_t)q_strides[0] : s_head * (cuuint64_t)g.H_q;
+    const cuuint64_t dims[4] = {(cuuint64_t)kHeadDim, (cuuint64_t)g.W, (cuuint64_t)g.H_q, (cuuint64_t)g.batch};
+    const cuuint64_t strides[3] = {s_w * 2, s_head * 2, s_batch * 2};
+    const cuuint32_t box[4] = {(cuuint32_t)kAtomCols, (cuuint32_t)g.W, (cuuint32_t)g.G, 1};
+    const CUresult r = enc(&mapQ, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(Q_win), dims, strides, box, ones,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(nullptr, LASER_KV_ERR_CUDA, "window_scores: tensor map of Q failed (CUresult %d)", (int)r);
+  }
+  cudaError_t e;
+  // the status word must start at zero; the partials are fully overwritten before they are read
+  if ((e = cudaMemsetAsync(scratch, 0, 256, st)) != cudaSuccess)
+    return fail(nullptr, LASER_KV_ERR_CUDA, "window_scores: memset: %s", cudaGetErrorString(e));
+  StreamArgs sa;
+  memset(&sa, 0, sizeof sa);
+  sa.S = g.S; sa.nb = g.nb; sa.t0 = 0; sa.tn = g.nb; sa.H_kv = g.H_kv; sa.batch = g.batch;
+  sa.G = g.G; sa.W = g.W; sa.GW = g.GW; sa.tiles_per_cta = g.tiles_per_cta; sa.n_split = g.n_split;
+  sa.scale_log2e = g.scale * 1.4426950408889634f;
+  sa.lse_part = reinterpret_cast<float2*>(scratch + g.off_part);
+  sa.lse2 = reinterpret_cast<float*>(scratch + g.off_lse2);
+  sa.s_exact = s_exact_out;
+  sa.status = reinterpret_cast<int*>(scratch);
+  const int ctas = g.nseg * g.n_split;
+  StreamArgs a1 = sa;
+  a1.stat_rows = g.GW;
+  a1.stat_rows_alloc = ((g.GW + 127) / 128) * 128;
+  if ((e = launch_stream<kLse, 0, 0>(mapK, mapQ, a1, ctas, stream_smem_bytes(kLse, a1.stat_rows_alloc, 0, g.GW), st)) != cudaSuccess)
+    return fail(nullptr, LASER_KV_ERR_CUDA, "window_scores: lse pass: %s", cudaGetErrorString(e));
+  StreamArgs a2 = sa;
+  a2.stat_rows = g.GW;
+  a2.stat_rows_alloc = g.GW;
+  if ((e = launch_stream<kScore, 0, 0>(mapK, mapQ, a2, ctas, stream_smem_bytes(kScore, a2.stat_rows_alloc, 0, g.GW), st)) != cudaSuccess)
+    return fail(nullptr, LASER_KV_ERR_CUDA, "window_scores: score pass: %s", cudaGetErrorString(e));
+  return LASER_KV_OK;
+}
+
+}  // namespace
+
+size_t laser_kv_window_scores_scratch_bytes(int32_t batch, int32_t n_q_heads, int32_t n_kv_heads, int32_t block_size,
+                                            int32_t window, int32_t n_blocks) {
+  ScoreGeom g;
+  if (score_geometry(batch, n_q_heads, n_kv_heads, block_size, window, n_blocks, 0.f, &g) != LASER_KV_OK) return 0;
+  return g.total;
+}
+
+laser_kv_status_t laser_kv_window_scores(const void* K_blk, const void* Q_win, const int64_t kv_strides[3],
+                                         const int64_t q_strides[3], int32_t batch, int32_t n_q_heads, int32_t n_kv_heads,
+                                         int32_t block_size, int32_t window, int32_t n_blocks, float softmax_scale,
+                                         void* scratch, size_t scratch_bytes, float* s_exact_out, void* stream) {
+  ScoreGeom g;
+  const laser_kv_status_t s = score_geometry(batch, n_q_heads, n_kv_heads, block_size, window, n_blocks, softmax_scale, &g);
+  if (s != LASER_KV_OK) return s;
+  if (!scratch) return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "window_scores: scratch is NULL");
+  if (reinterpret_cast<uintptr_t>(scratch) & (kAlign - 1))
+    return fail(nullptr, LASER_KV_ERR_ALIGNMENT, "window_scores: scratch must be 256-byte aligned");
+  if (scratch_bytes < g.total)
+    return fail(nullptr, LASER_KV_ERR_CAPACITY, "window_scores: scratch needs %zu bytes, got %zu", g.total, scratch_bytes);
+  return run_window_scores(g, K_blk, Q_win, kv_strides, q_strides, static_cast<uint8_t*>(scratch), s_exact_out,
+                           static_cast<cudaStream_t>(stream));
+}
+
 laser_kv_status_t laser_kv_gather_append(const void* K_src, const void* V_src, int64_t src_seg_stride,
                                          int64_t src_row_stride, const int32_t* idx, int32_t n_segments,
                                          int32_t n_keep, void* K_dst, void* V_dst, int64_t dst_seg_stride,

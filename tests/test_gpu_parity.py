@@ -135,6 +135,32 @@ def test_two_stage_topk_entry_point_against_oracle():
             assert (idx[g] == want).all(), (S, a, ke, kl, g)
 
 
+def test_window_scores_entry_point_against_oracle():
+    import torch
+    from paper_2602_02199_b200 import binding as Bn
+    from parity_util import SCORE_ATOL, SCORE_RTOL
+    for name, S, nb in (("tiny", 1024, 2), ("qwen7b_128k", 1000, 3), ("llama8b_128k", 4096, 2)):
+        w = synth.workload(name).with_(block_size=S, context_len=8 * S, batch=1)
+        K, _ = synth.kv_blocks(w, 0, 0, 2, nb)
+        Q = synth.q_window(w, 0, 0)
+        tK = torch.from_numpy(K.view(np.int16)).cuda()[None]
+        tQ = torch.from_numpy(Q.view(np.int16)).cuda()[None]
+        for scale in (0.0, 0.05):
+            out = to_np(Bn.laser_kv_window_scores(tK, tQ, S, nb, softmax_scale=scale))
+            torch.cuda.synchronize()
+            G = w.group
+            for h in (0, w.n_kv_heads - 1):
+                for t in range(nb):
+                    want = O.window_scores(Q[h * G:(h + 1) * G].reshape(-1, 128), K[h, t * S:(t + 1) * S],
+                                           None if scale == 0.0 else scale)
+                    err = np.abs(out[0, h, t] - want)
+                    assert (err <= SCORE_RTOL * np.abs(want) + SCORE_ATOL).all(), (name, h, t, err.max())
+    assert Bn.laser_kv_window_scores_scratch_bytes(1, 32, 8, 8192, 64, 16) > 0
+    with pytest.raises(Bn.LaserKVError) as e:
+        Bn.laser_kv_window_scores(tK, tQ, S, nb, scratch=torch.empty(256, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == Bn.ERR_CAPACITY
+
+
 def test_gather_append_entry_point_bit_exact():
     import torch
     from paper_2602_02199_b200 import binding as Bn
