@@ -217,6 +217,36 @@ laser_kv_status_t laser_kv_window_scores(const void* K_blk, const void* Q_win,
                                          float softmax_scale, void* scratch, size_t scratch_bytes,
                                          float* s_exact_out, void* stream);
 
+/* laser_kv_window_scores for callers that cannot hand over scratch memory. (The paper has no
+ * counterpart to this entry point; it exists for integration only.)
+ *
+ * Who needs it: code that runs where device allocation is off the table - a plugin inside a
+ * serving engine whose memory pool already owns the whole GPU, so a cudaMalloc would fail or eat
+ * into a reservation it must not touch; a hook in a latency-critical decode loop where the
+ * implicit device synchronisation of cudaMalloc/cudaFree is unacceptable; a sandboxed extension
+ * that is simply not allowed to call the allocator. Such a caller still passes its inputs and
+ * its output buffer, but the log-sum-exp partials that laser_kv_window_scores keeps in `scratch`
+ * go to an array built into the library image instead:
+ *   - size LASER_KV_STATIC_SCRATCH_BYTES = 2 MiB (laser_kv_window_scores_static_max_bytes()),
+ *     resident on every GPU that loads the library, until the process exits;
+ *   - a problem whose laser_kv_window_scores_scratch_bytes(...) exceeds it is rejected with
+ *     LASER_KV_ERR_CAPACITY and nothing is launched (a 128k-token layer of 16 blocks x 8 KV
+ *     heads x 256 window queries needs about 1.2 MiB and fits);
+ *   - this function never calls cudaMalloc, cudaFree or any allocating library routine.
+ * The first call on each device looks up the array's device address (with the CUDA device of
+ * the inputs current, as for every call); make that first call before starting any stream
+ * capture. All calls on a device share the one array: it still holds the previous call's
+ * partials (the status word at its start is cleared by every call, everything else is
+ * overwritten before it is read), and two calls whose kernels overlap on the GPU - different
+ * streams, or different host threads - race on it. Serialise them.
+ * Arguments and results are those of laser_kv_window_scores without scratch/scratch_bytes. */
+size_t laser_kv_window_scores_static_max_bytes(void);
+laser_kv_status_t laser_kv_window_scores_static(const void* K_blk, const void* Q_win,
+                                                const int64_t kv_strides[3], const int64_t q_strides[3],
+                                                int32_t batch, int32_t n_q_heads, int32_t n_kv_heads,
+                                                int32_t block_size, int32_t window, int32_t n_blocks,
+                                                float softmax_scale, float* s_exact_out, void* stream);
+
 /* Append step (Sections 1 and 3): for each of n_segments segments copies rows idx[seg][i] of the
  * segment's K and V (dev bf16, row length d = 128, consecutive rows `src_row_stride` elements
  * apart, segment s starting at src + s*src_seg_stride) to dst rows [dst_offset + i] of the

@@ -17,6 +17,7 @@ EXPORTS = [
     "laser_kv_status_string", "laser_kv_last_error", "laser_kv_launch_count",
     "laser_kv_two_stage_topk", "laser_kv_gather_append", "laser_kv_profile_enable",
     "laser_kv_profile_read", "laser_kv_window_scores", "laser_kv_window_scores_scratch_bytes",
+    "laser_kv_window_scores_static", "laser_kv_window_scores_static_max_bytes",
 ]
 
 
@@ -116,6 +117,11 @@ def load(build_if_missing: bool = True) -> C.CDLL:
     lib.laser_kv_window_scores.restype = i32
     lib.laser_kv_window_scores.argtypes = [vp, vp, p(i64), p(i64), i32, i32, i32, i32, i32, i32, C.c_float, vp, sz,
                                            vp, vp]
+    lib.laser_kv_window_scores_static_max_bytes.restype = sz
+    lib.laser_kv_window_scores_static_max_bytes.argtypes = []
+    lib.laser_kv_window_scores_static.restype = i32
+    lib.laser_kv_window_scores_static.argtypes = [vp, vp, p(i64), p(i64), i32, i32, i32, i32, i32, i32, C.c_float,
+                                                  vp, vp]
     _lib = lib
     return lib
 
@@ -334,4 +340,21 @@ def laser_kv_window_scores(K_blk, Q_win, block_size, n_blocks, softmax_scale=0.0
     _check(load().laser_kv_window_scores(_ptr(K_blk), _ptr(Q_win), ks, qs, batch, h_q, h_kv, block_size, window,
                                          n_blocks, softmax_scale, _ptr(scratch), scratch.numel(), _ptr(out),
                                          _stream_ptr(stream)))
+    return out
+
+
+def laser_kv_window_scores_static_max_bytes() -> int:
+    return int(load().laser_kv_window_scores_static_max_bytes())
+
+
+def laser_kv_window_scores_static(K_blk, Q_win, block_size, n_blocks, out, softmax_scale=0.0, stream=None):
+    """The window-score step for callers that cannot allocate: inputs and the fp32 output tensor
+    `out` [batch][H_kv][n_blocks][S] come from the caller, the scratch is the library's built-in
+    2 MiB array. This wrapper allocates nothing either. Calls sharing a device must not overlap."""
+    batch, h_kv = K_blk.shape[0], K_blk.shape[1]
+    h_q, window = Q_win.shape[1], Q_win.shape[2]
+    ks = (C.c_int64 * 3)(*K_blk.stride()[:3])
+    qs = (C.c_int64 * 3)(*Q_win.stride()[:3])
+    _check(load().laser_kv_window_scores_static(_ptr(K_blk), _ptr(Q_win), ks, qs, batch, h_q, h_kv, block_size,
+                                                window, n_blocks, softmax_scale, _ptr(out), _stream_ptr(stream)))
     return out

@@ -850,6 +850,57 @@ laser_kv_status_t laser_kv_window_scores(const void* K_blk, const void* Q_win, c
                            static_cast<cudaStream_t>(stream));
 }
 
+// ---- window scores without any allocation ---------------------------------------------------------
+// Scratch for laser_kv_window_scores_static: lives in the library's device image, so every GPU
+// that loads the library holds these bytes until the process exits.
+#define LASER_KV_STATIC_SCRATCH_BYTES (2u << 20)
+static __device__ __align__(256) unsigned char g_static_scratch[LASER_KV_STATIC_SCRATCH_BYTES];
+
+namespace {
+
+// In host code the symbol above is only a stand-in; the device address has to be asked for, per
+// device, with that device current. Cached after the first successful lookup.
+laser_kv_status_t static_scratch_address(uint8_t** out) {
+  constexpr int kMaxDevices = 64;
+  static std::mutex mu;
+  static uint8_t* cached[kMaxDevices] = {nullptr};
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess || dev < 0 || dev >= kMaxDevices)
+    return fail(nullptr, LASER_KV_ERR_CUDA, "window_scores_static: cudaGetDevice: %s", cudaGetErrorString(e));
+  std::lock_guard<std::mutex> lock(mu);
+  if (!cached[dev]) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_static_scratch);
+    if (e != cudaSuccess || !p)
+      return fail(nullptr, LASER_KV_ERR_CUDA, "window_scores_static: cudaGetSymbolAddress: %s", cudaGetErrorString(e));
+    cached[dev] = static_cast<uint8_t*>(p);
+  }
+  *out = cached[dev];
+  return LASER_KV_OK;
+}
+
+}  // namespace
+
+size_t laser_kv_window_scores_static_max_bytes(void) { return LASER_KV_STATIC_SCRATCH_BYTES; }
+
+laser_kv_status_t laser_kv_window_scores_static(const void* K_blk, const void* Q_win, const int64_t kv_strides[3],
+                                                const int64_t q_strides[3], int32_t batch, int32_t n_q_heads,
+                                                int32_t n_kv_heads, int32_t block_size, int32_t window, int32_t n_blocks,
+                                                float softmax_scale, float* s_exact_out, void* stream) {
+  ScoreGeom g;
+  laser_kv_status_t s = score_geometry(batch, n_q_heads, n_kv_heads, block_size, window, n_blocks, softmax_scale, &g);
+  if (s != LASER_KV_OK) return s;
+  if (g.total > LASER_KV_STATIC_SCRATCH_BYTES)
+    return fail(nullptr, LASER_KV_ERR_CAPACITY,
+                "window_scores_static: this problem needs %zu bytes of scratch but the built-in array holds %u; "
+                "use laser_kv_window_scores with caller scratch or pass fewer blocks per call",
+                g.total, (unsigned)LASER_KV_STATIC_SCRATCH_BYTES);
+  uint8_t* scratch = nullptr;
+  if ((s = static_scratch_address(&scratch)) != LASER_KV_OK) return s;
+  return run_window_scores(g, K_blk, Q_win, kv_strides, q_strides, scratch, s_exact_out, static_cast<cudaStream_t>(stream));
+}
+
 laser_kv_status_t laser_kv_gather_append(const void* K_src, const void* V_src, int64_t src_seg_stride,
                                          int64_t src_row_stride, const int32_t* idx, int32_t n_segments,
                                          int32_t n_keep, void* K_dst, void* V_dst, int64_t dst_seg_stride,
