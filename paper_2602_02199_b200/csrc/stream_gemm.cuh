@@ -16,8 +16,9 @@
 //            that is tiny relative to the key's other projections are queued for an exact
 //            recomputation.
 //
-// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner,
-// warps 2..5 = epilogue (TMEM lane quarter = warp_id % 4).
+// Warp roles (320 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner,
+// warps 2..9 = two epilogue groups of four warps (TMEM lane quarter = warp_id % 4) that split
+// the accumulator columns of every tile.
 #pragma once
 #include "ptx.cuh"
 
@@ -28,7 +29,9 @@ constexpr int kAtomCols = 64;                  // bf16 elements per 128-byte swi
 constexpr int kTileAtomBytes = kTileKeys * 128;  // one 64-column half of a key tile
 constexpr int kTileBytes = 2 * kTileAtomBytes;   // 128 keys x 128 dims bf16
 constexpr int kStages = 4;
-constexpr int kStreamThreads = 192;
+constexpr int kStreamThreads = 320;
+constexpr int kEpilogueThreads = 256;
+constexpr int kXwgBytes = 2048;                // exchange area between the two epilogue groups
 constexpr int kTmemCols = 512;
 constexpr int kAccStride = 256;                // TMEM columns per accumulator buffer
 constexpr int kMaxStatRows = 256;
@@ -36,6 +39,36 @@ constexpr int kMaxStatRows = 256;
 enum StreamMode { kLse = 0, kScore = 1, kProj = 2 };
 
 enum : int { kStatusOk = 0, kStatusCapacity = 3, kStatusTimeout = 6 };
+
+template <int N> struct IntTag { static constexpr int value = N; };
+
+// Walks the 32-bit columns [c_begin, c_end) of the calling thread's TMEM lane (c_begin a multiple
+// of 32, length a multiple of 16 and at most 128) in chunks of 32 (a last chunk of 16), loading
+// chunk i+1 while f(values, first column, IntTag<count>) works on chunk i.
+template <class F>
+__device__ __forceinline__ void walk_columns(uint32_t taddr, int c_begin, int c_end, F&& f) {
+  const int n = c_end - c_begin;
+  if (n <= 0) return;
+  uint32_t va[32], vb[32];
+  if (n >= 32) { tmem_ld_x32(taddr + c_begin, va); tmem_wait_ld_dep32(va); }
+  else { tmem_ld_x16(taddr + c_begin, va); tmem_wait_ld_dep16(va); }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int off = i * 32;
+    if (off < n) {
+      uint32_t* cur = (i & 1) ? vb : va;
+      uint32_t* nxt = (i & 1) ? va : vb;
+      const int rest = n - off - 32;       // columns after this chunk
+      if (rest >= 32) tmem_ld_x32(taddr + c_begin + off + 32, nxt);
+      else if (rest > 0) tmem_ld_x16(taddr + c_begin + off + 32, nxt);
+      if (n - off >= 32) f(cur, c_begin + off, IntTag<32>{});
+      else f(cur, c_begin + off, IntTag<16>{});
+      if (rest >= 32) tmem_wait_ld_dep32(nxt);
+      else if (rest > 0) tmem_wait_ld_dep16(nxt);
+    }
+  }
+}
+
 
 struct StreamArgs {
   // problem geometry
@@ -67,8 +100,67 @@ __device__ __forceinline__ void record_status(int* status, int code) {
   atomicCAS(status, kStatusOk, code);
 }
 
+// Tables [T_BEGIN, T_END) of the chunk for the calling thread's key: packs the sign bits of each
+// table's K projections into a bucket code, looks the code up in the histogram slice and
+// returns the summed collisions. A table whose smallest |projection| is below 2^-15 of the
+// largest |projection| among the key's first 16 hyperplanes of the chunk is queued for an exact
+// recomputation of its signs.
+template <int KBITS, int T_BEGIN, int T_END>
+__device__ __forceinline__ uint32_t proj_tables(uint32_t t_acc, const uint16_t* hist_s, const StreamArgs& a,
+                                                int seg, int key, int table0, bool valid) {
+  constexpr int CB = T_BEGIN * KBITS, CE = T_END * KBITS;
+  constexpr int L0 = CB / 32 * 32;
+  constexpr int NCHUNK = (CE - L0 + 31) / 32;
+  constexpr uint32_t bucket_mask = (1u << KBITS) - 1u;
+  uint32_t v[2][32];
+  uint32_t v16[16];
+  tmem_ld_x32(t_acc + L0, v[0]);
+  tmem_ld_x16(t_acc, v16);
+  tmem_wait_ld_dep32(v[0]);
+  tmem_wait_ld_dep16(v16);
+  float amax = 0.f;
+#pragma unroll
+  for (int k = 0; k < 16; ++k) amax = fmaxf(amax, fabsf(__uint_as_float(v16[k])));
+  const float tau = amax * (1.0f / 32768.0f);
+  uint32_t partial = 0, neg = 0;
+  float amin = INFINITY;
+#pragma unroll
+  for (int c = 0; c < NCHUNK; ++c) {
+    if (c + 1 < NCHUNK) tmem_ld_x32(t_acc + L0 + 32 * (c + 1), v[(c + 1) & 1]);
+#pragma unroll
+    for (int k = 0; k < 32; k += 2) {
+      const int col = L0 + 32 * c + k;
+      // K is even and CB is a multiple of K, so a pair of columns never straddles two tables
+      if (col >= CB && col < CE) {
+        const uint32_t x0 = v[c & 1][k], x1 = v[c & 1][k + 1];
+        neg = __funnelshift_l(x0, neg, 1);                 // (neg << 1) | sign(x0)
+        neg = __funnelshift_l(x1, neg, 1);
+        amin = fminf(amin, fminf(fabsf(__uint_as_float(x0)), fabsf(__uint_as_float(x1))));
+        if ((col + 1) % KBITS == KBITS - 1) {
+          const int rl = (col + 1) / KBITS;                // table within the chunk
+          const uint32_t code = (~neg) & bucket_mask;
+          partial += hist_s[((uint32_t)rl << KBITS) + code];
+          if (valid) {
+            const int r = table0 + rl;
+            if (a.key_buckets) a.key_buckets[((size_t)seg * a.S + key) * a.lsh_tables + r] = (uint16_t)code;
+            if (!(amin >= tau)) {
+              const int slot = atomicAdd(a.fix_count, 1);
+              if (slot < a.fix_cap) a.fix_items[slot] = make_int4(seg, key, r, (int)code);
+              else record_status(a.status, kStatusCapacity);
+            }
+          }
+          neg = 0;
+          amin = INFINITY;
+        }
+      }
+    }
+    if (c + 1 < NCHUNK) tmem_wait_ld_dep32(v[(c + 1) & 1]);
+  }
+  return partial;
+}
+
 struct StreamSmem {
-  uint32_t stat, stages, hist, lse, bars, tmem_slot;  // shared-space byte addresses
+  uint32_t stat, stages, hist, lse, xwg, bars, tmem_slot;  // shared-space byte addresses
 };
 
 // Shared memory carve-up, identical on host (sizes) and device (addresses).
@@ -77,6 +169,7 @@ __host__ __device__ inline uint32_t stream_smem_bytes(int mode, int stat_rows_al
   uint32_t b = 2u * stat_rows_alloc * 128u + kStages * kTileBytes;
   if (mode == kProj) b += (hist_bytes + 127u) & ~127u;
   if (mode == kScore) b += ((GW * 4u) + 127u) & ~127u;
+  b += kXwgBytes;
   b += 256;          // barriers + TMEM slot
   return b + 1024;   // slack for 1024-byte alignment of the base
 }
@@ -116,6 +209,8 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
   if (MODE == kProj) cur += (hist_bytes + 127u) & ~127u;
   sm.lse = cur;
   if (MODE == kScore) cur += ((a.GW * 4u) + 127u) & ~127u;
+  sm.xwg = cur;
+  cur += kXwgBytes;
   sm.bars = cur;
   sm.tmem_slot = cur + 128;
   const uint32_t bar_full = sm.bars;                 // kStages barriers
@@ -126,11 +221,12 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
   uint8_t* const gen_base = smem_raw + (base - smem_u32(smem_raw));
   const uint16_t* hist_s = reinterpret_cast<const uint16_t*>(gen_base + (sm.hist - base));
   float* lse_s = reinterpret_cast<float*>(gen_base + (sm.lse - base));
+  uint8_t* xwg_s = gen_base + (sm.xwg - base);
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_base + (sm.tmem_slot - base));
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
-    for (int s = 0; s < 2; ++s) { mbar_init(bar_tfull + 8 * s, 1); mbar_init(bar_tempty + 8 * s, 128); }
+    for (int s = 0; s < 2; ++s) { mbar_init(bar_tfull + 8 * s, 1); mbar_init(bar_tempty + 8 * s, kEpilogueThreads); }
     mbar_init(bar_stat, 1);
     fence_mbar_init();
   }
@@ -219,61 +315,79 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
     }
     __syncwarp();
   } else {
-    // ================= epilogue warps =================
+    // ================= epilogue warps: two groups of four =================
+    // Both groups cover all 128 TMEM lanes (lane quarter = warp_id % 4); they split the
+    // accumulator columns of every tile between them.
     const int quarter = warp & 3;
     const int row = quarter * 32 + lane;                   // TMEM lane owned by this thread
     const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
-    const int etid = threadIdx.x - 64;                     // 0..127
+    const int etid = threadIdx.x - 64;                     // 0..255
+    const int wg = etid >> 7;                              // epilogue group 0 / 1
     bool ok = true;
 
-    if (MODE == kLse) {
-      float m[2] = {-INFINITY, -INFINITY};
-      float l[2] = {0.f, 0.f};
+    if constexpr (MODE == kLse) {
+      // group g owns query block g (G*W > 128) or half of the key columns (G*W <= 128)
+      const int mb = (nmb == 2) ? wg : 0;
+      const int c_begin = (nmb == 2) ? 0 : wg * 64;
+      const int c_end = (nmb == 2) ? kTileKeys : wg * 64 + 64;
+      float m = -INFINITY, l = 0.f;
+      const float c2 = a.scale_log2e;
       for (int i = 0; i < ntiles && ok; ++i) {
         const int acc = i & 1;
         ok = mbar_wait(bar_tfull + 8 * acc, (i >> 1) & 1);
         if (!ok) break;
         tc_fence_after();
         const int nvalid = min(kTileKeys, a.S - (tile0 + i) * kTileKeys);
+        const int ce = min(c_end, (nvalid + 15) & ~15);
+        walk_columns(t_lane + acc * kAccStride + mb * 128, c_begin, ce, [&](const uint32_t* v, int col0, auto cnt_tag) {
+          constexpr int CNT = decltype(cnt_tag)::value;
+          const int lim = nvalid - col0;                   // valid columns in this chunk (>= 1)
+          float cmax = -INFINITY;
+          if (lim >= CNT) {
 #pragma unroll
-        for (int mb = 0; mb < 2; ++mb) {
-          if (mb < nmb) {
-            for (int c = 0; c < 4; ++c) {
-              if (c * 32 >= nvalid) break;
-              uint32_t v[32];
-              tmem_ld_x32(t_lane + acc * kAccStride + mb * 128 + c * 32, v);
-              tmem_wait_ld();
-              const int lim = nvalid - c * 32;             // >= 1
-              float tv[32];
-              float cmax = -INFINITY;
+            for (int k = 0; k < CNT; ++k) cmax = fmaxf(cmax, __uint_as_float(v[k]));
+            const float m_new = fmaxf(m, cmax * c2);
+            float add0 = 0.f, add1 = 0.f;
 #pragma unroll
-              for (int k = 0; k < 32; ++k) {
-                tv[k] = (k < lim) ? __uint_as_float(v[k]) * a.scale_log2e : -INFINITY;
-                cmax = fmaxf(cmax, tv[k]);
-              }
-              const float m_new = fmaxf(m[mb], cmax);
-              float add = 0.f;
-#pragma unroll
-              for (int k = 0; k < 32; ++k) add += ex2_approx(tv[k] - m_new);
-              l[mb] = l[mb] * ex2_approx(m[mb] - m_new) + add;
-              m[mb] = m_new;
+            for (int k = 0; k < CNT; ++k) {
+              const float x = fmaf(__uint_as_float(v[k]), c2, -m_new);
+              const float e = ((k * 5) % 16 < 5) ? ex2_poly(x) : ex2_approx(x);
+              if (k & 1) add1 += e; else add0 += e;
             }
+            l = l * ex2_approx(m - m_new) + (add0 + add1);
+            m = m_new;
+          } else {
+#pragma unroll
+            for (int k = 0; k < CNT; ++k) if (k < lim) cmax = fmaxf(cmax, __uint_as_float(v[k]));
+            const float m_new = fmaxf(m, cmax * c2);
+            float add = 0.f;
+#pragma unroll
+            for (int k = 0; k < CNT; ++k)
+              if (k < lim) add += ex2_approx(fmaf(__uint_as_float(v[k]), c2, -m_new));
+            l = l * ex2_approx(m - m_new) + add;
+            m = m_new;
           }
-        }
+        });
         tc_fence_before();
         mbar_arrive(bar_tempty + 8 * acc);
       }
-      if (ok) {
-#pragma unroll
-        for (int mb = 0; mb < 2; ++mb) {
-          const int q = mb * 128 + row;
-          if (mb < nmb && q < a.GW)
-            a.lse_part[((size_t)seg * a.n_split + split) * a.GW + q] = make_float2(m[mb], l[mb]);
+      if (nmb == 2) {
+        const int q = mb * 128 + row;
+        if (ok && q < a.GW) a.lse_part[((size_t)seg * a.n_split + split) * a.GW + q] = make_float2(m, l);
+      } else {
+        float2* xch = reinterpret_cast<float2*>(xwg_s);
+        if (wg == 1) xch[row] = make_float2(m, l);
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        if (wg == 0 && ok && row < a.GW) {
+          const float2 o = xch[row];
+          const float mx = fmaxf(m, o.x);
+          const float lt = (mx == -INFINITY) ? 0.f : l * ex2_approx(m - mx) + o.y * ex2_approx(o.x - mx);
+          a.lse_part[((size_t)seg * a.n_split + split) * a.GW + row] = make_float2(mx, lt);
         }
       }
-    } else if (MODE == kScore) {
+    } else if constexpr (MODE == kScore) {
       // combine the splits' (max, sum) partials into log2-sum-exp2 per query
-      for (int q = etid; q < a.GW; q += 128) {
+      for (int q = etid; q < a.GW; q += 256) {
         const float2* p = a.lse_part + (size_t)seg * a.n_split * a.GW + q;
         float mx = -INFINITY;
         for (int s2 = 0; s2 < a.n_split; ++s2) mx = fmaxf(mx, p[(size_t)s2 * a.GW].x);
@@ -286,46 +400,49 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
         lse_s[q] = r;
         if (split == 0) a.lse2[(size_t)seg * a.GW + q] = r;
       }
-      asm volatile("bar.sync 1, 128;" ::: "memory");
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      // group 0 sums queries [0, cs), group 1 queries [cs, G*W); both ranges start 32-aligned
+      const int cs = ((a.GW / 32 + 1) / 2) * 32;
+      const int c_begin = wg ? cs : 0;
+      const int c_end = wg ? a.GW : cs;
+      const float c2 = a.scale_log2e;
+      float* part = reinterpret_cast<float*>(xwg_s);       // [2 accumulators][128 keys]
       for (int i = 0; i < ntiles && ok; ++i) {
         const int acc = i & 1;
         ok = mbar_wait(bar_tfull + 8 * acc, (i >> 1) & 1);
         if (!ok) break;
         tc_fence_after();
-        float sum = 0.f;
-        for (int c0 = 0; c0 < a.GW; c0 += 32) {
-          uint32_t v[32];
-          if (c0 + 32 <= a.GW) {
-            tmem_ld_x32(t_lane + acc * kAccStride + c0, v);
-            tmem_wait_ld();
+        float s0 = 0.f, s1 = 0.f;
+        walk_columns(t_lane + acc * kAccStride, c_begin, c_end, [&](const uint32_t* v, int col0, auto cnt_tag) {
+          constexpr int CNT = decltype(cnt_tag)::value;
 #pragma unroll
-            for (int k = 0; k < 32; k += 4) {
-              const float4 ls = *reinterpret_cast<const float4*>(lse_s + c0 + k);
-              sum += ex2_approx(fmaf(__uint_as_float(v[k + 0]), a.scale_log2e, -ls.x));
-              sum += ex2_approx(fmaf(__uint_as_float(v[k + 1]), a.scale_log2e, -ls.y));
-              sum += ex2_approx(fmaf(__uint_as_float(v[k + 2]), a.scale_log2e, -ls.z));
-              sum += ex2_approx(fmaf(__uint_as_float(v[k + 3]), a.scale_log2e, -ls.w));
+          for (int k = 0; k < CNT; k += 4) {
+            const float4 ls = *reinterpret_cast<const float4*>(lse_s + col0 + k);
+            const float lsv[4] = {ls.x, ls.y, ls.z, ls.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const float x = fmaf(__uint_as_float(v[k + e]), c2, -lsv[e]);
+              const float ex = (((k + e) * 5) % 16 < 5) ? ex2_poly(x) : ex2_approx(x);
+              if (e & 1) s1 += ex; else s0 += ex;
             }
-          } else {  // GW % 32 == 16
-            tmem_ld_x16(t_lane + acc * kAccStride + c0, v);
-            tmem_wait_ld();
-#pragma unroll
-            for (int k = 0; k < 16; ++k)
-              sum += ex2_approx(fmaf(__uint_as_float(v[k]), a.scale_log2e, -lse_s[c0 + k]));
           }
-        }
+        });
         tc_fence_before();
         mbar_arrive(bar_tempty + 8 * acc);
-        const int key = (tile0 + i) * kTileKeys + row;
-        if (key < a.S) a.s_exact[(size_t)seg * a.S + key] = sum;
+        const float sum = s0 + s1;
+        if (wg == 1) part[acc * 128 + row] = sum;
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        if (wg == 0) {
+          const int key = (tile0 + i) * kTileKeys + row;
+          if (key < a.S) a.s_exact[(size_t)seg * a.S + key] = sum + part[acc * 128 + row];
+        }
       }
     } else {
       // ---- kProj: sign bits -> bucket codes -> histogram lookups ----
       // Bucket code of a table: bit b of the table (hyperplane r*K + b) sits at position
       // K-1-b, i.e. the first hyperplane is the most significant bit; bit = [projection >= 0].
+      // Group 0 handles the chunk's first TC/2 tables, group 1 the rest.
       ok = mbar_wait(bar_stat, 0);   // histogram slice landed (async-proxy writes visible after the wait)
-      constexpr int NCOLS = KBITS * TC;
-      constexpr uint32_t bucket_mask = (1u << KBITS) - 1u;
       for (int i = 0; i < ntiles && ok; ++i) {
         const int acc = i & 1;
         ok = mbar_wait(bar_tfull + 8 * acc, (i >> 1) & 1);
@@ -334,50 +451,9 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
         const int key = (tile0 + i) * kTileKeys + row;
         const bool valid = key < a.S;
         const uint32_t t_acc = t_lane + acc * kAccStride;
-        uint32_t partial = 0;
-        uint32_t neg = 0;
-        float amin = INFINITY;
-        float tau = 0.f;
-#pragma unroll
-        for (int c0 = 0; c0 < NCOLS; c0 += 32) {
-          uint32_t v[32];
-          constexpr int kFull = 32;
-          const bool full = (c0 + kFull <= NCOLS);
-          if (full) tmem_ld_x32(t_acc + c0, v); else tmem_ld_x16(t_acc + c0, v);
-          tmem_wait_ld();
-          if (c0 == 0) {
-            // scale of this key's projections, from the first 16 hyperplanes of the chunk
-            float amax = 0.f;
-#pragma unroll
-            for (int k = 0; k < 16; ++k) amax = fmaxf(amax, fabsf(__uint_as_float(v[k])));
-            tau = amax * (1.0f / 32768.0f);
-          }
-#pragma unroll
-          for (int k = 0; k < 32; ++k) {
-            if (c0 + k < NCOLS) {
-              const uint32_t x = v[k];
-              neg = __funnelshift_l(x, neg, 1);            // (neg << 1) | sign(x)
-              amin = fminf(amin, fabsf(__uint_as_float(x)));
-              if ((c0 + k) % KBITS == KBITS - 1) {
-                const int rl = (c0 + k) / KBITS;           // table within the chunk
-                const uint32_t code = (~neg) & bucket_mask;
-                partial += hist_s[((uint32_t)rl << KBITS) + code];
-                if (valid) {
-                  const int r = chunk * TC + rl;
-                  if (a.key_buckets)
-                    a.key_buckets[((size_t)seg * a.S + key) * a.lsh_tables + r] = (uint16_t)code;
-                  if (!(amin >= tau)) {
-                    const int slot = atomicAdd(a.fix_count, 1);
-                    if (slot < a.fix_cap) a.fix_items[slot] = make_int4(seg, key, r, (int)code);
-                    else record_status(a.status, kStatusCapacity);
-                  }
-                }
-                neg = 0;
-                amin = INFINITY;
-              }
-            }
-          }
-        }
+        uint32_t partial;
+        if (wg == 0) partial = proj_tables<KBITS, 0, TC / 2>(t_acc, hist_s, a, seg, key, chunk * TC, valid);
+        else partial = proj_tables<KBITS, TC / 2, TC>(t_acc, hist_s, a, seg, key, chunk * TC, valid);
         tc_fence_before();
         mbar_arrive(bar_tempty + 8 * acc);
         if (valid) atomicAdd(a.counts + (size_t)seg * a.S + key, partial);
