@@ -457,9 +457,15 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
   {
     QprepArgs qa{static_cast<const uint16_t*>(Q_win), q_strides[0], q_strides[1], q_strides[2], h->P, hist, qb,
                  c.n_kv_heads, d.G, c.window, d.GW, c.lsh_bits, c.lsh_tables};
-    const size_t smem = (size_t)c.lsh_bits * 128 * 8 + ((size_t)4 << c.lsh_bits);
+    const size_t smem = qprep_smem_bytes(c.lsh_bits);
     dim3 grid(c.lsh_tables, c.n_kv_heads, c.batch);
-    qprep_kernel<<<grid, 256, smem, st>>>(qa);
+    switch (c.lsh_bits) {
+      case 4: qprep_kernel<4><<<grid, kQprepThreads, smem, st>>>(qa); break;
+      case 6: qprep_kernel<6><<<grid, kQprepThreads, smem, st>>>(qa); break;
+      case 8: qprep_kernel<8><<<grid, kQprepThreads, smem, st>>>(qa); break;
+      case 10: qprep_kernel<10><<<grid, kQprepThreads, smem, st>>>(qa); break;
+      default: qprep_kernel<12><<<grid, kQprepThreads, smem, st>>>(qa); break;
+    }
     g_launches.fetch_add(1);
     LKV_CUDA(cudaGetLastError(), "qprep_kernel");
   }
@@ -509,7 +515,7 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
     SignfixArgs fa{static_cast<const uint16_t*>(K_blk), kv_strides[0], kv_strides[1], kv_strides[2], h->P, hist,
                    counts, key_buckets, fix_items, ctrl + 1, d.fix_cap, c.n_kv_heads, nb, S, c.lsh_bits,
                    c.lsh_tables, ctrl + 2};
-    signfix_kernel<<<296, 256, 0, st>>>(fa);
+    signfix_kernel<<<kSignfixCtas, 256, 0, st>>>(fa);
     g_launches.fetch_add(1);
     LKV_CUDA(cudaGetLastError(), "signfix_kernel");
   }

@@ -18,9 +18,11 @@ __device__ __forceinline__ double bf16_to_f64(uint16_t b) {
 }
 
 // ------------------------------------------------------------------------------------------------
-// Query side: one CTA per (table r, KV head h, sequence b); thread q handles window query q of the
-// head's group. Projections are accumulated in fp64 (products of two bf16 are exact in fp64), so
-// query sign bits need no guard. Bucket code: hyperplane r*K + b0 sits at bit K-1-b0.
+// Query side: one CTA per (table r, KV head h, sequence b); a thread handles window queries q and
+// q + 128 of the head's group. Projections are accumulated in fp64 (products of two bf16 are exact
+// in fp64), so query sign bits need no guard. Every query element is widened to fp64 once and
+// feeds the K accumulators of the table; the plane values come from shared memory as 16-byte
+// broadcasts shared by both queries. Bucket code: hyperplane r*K + b0 sits at bit K-1-b0.
 // ------------------------------------------------------------------------------------------------
 struct QprepArgs {
   const uint16_t* Q;      // [batch][H_q][W][d] via strides
@@ -31,46 +33,78 @@ struct QprepArgs {
   int H_kv, G, W, GW, K, L;
 };
 
-__global__ void __launch_bounds__(256) qprep_kernel(const QprepArgs a) {
-  extern __shared__ uint8_t smem_q[];
-  double* planes = reinterpret_cast<double*>(smem_q);                       // [K][128]
-  uint32_t* bins = reinterpret_cast<uint32_t*>(smem_q + (size_t)a.K * 128 * 8);  // [2^K]
+constexpr int kQprepThreads = 128;
+
+__host__ __device__ inline size_t qprep_smem_bytes(int K) { return (size_t)K * 128 * 8 + ((size_t)4 << K); }
+
+template <int K>
+__global__ void __launch_bounds__(kQprepThreads) qprep_kernel(const QprepArgs a) {
+  extern __shared__ __align__(16) uint8_t smem_q[];
+  double* planes = reinterpret_cast<double*>(smem_q);                          // [K][128]
+  uint32_t* bins = reinterpret_cast<uint32_t*>(smem_q + (size_t)K * 128 * 8);   // [2^K]
   const int r = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
-  const int nbins = 1 << a.K;
-  for (int i = threadIdx.x; i < a.K * 128; i += blockDim.x)
-    planes[i] = bf16_to_f64(a.P[(size_t)r * a.K * 128 + i]);
-  for (int i = threadIdx.x; i < nbins; i += blockDim.x) bins[i] = 0;
+  constexpr int nbins = 1 << K;
+  for (int i = threadIdx.x; i < K * 128; i += kQprepThreads)
+    planes[i] = bf16_to_f64(a.P[(size_t)r * K * 128 + i]);
+  for (int i = threadIdx.x; i < nbins; i += kQprepThreads) bins[i] = 0;
   __syncthreads();
-  for (int q = threadIdx.x; q < a.GW; q += blockDim.x) {
-    const int g = q / a.W, w = q % a.W;
-    const uint16_t* row = a.Q + b * a.qs_b + (long long)(h * a.G + g) * a.qs_h + w * a.qs_w;
-    uint32_t code = 0;
-    for (int bit = 0; bit < a.K; ++bit) {
-      const double* p = planes + bit * 128;
-      double acc = 0.0;
-      for (int c = 0; c < 128; c += 8) {
-        const uint4 v = *reinterpret_cast<const uint4*>(row + c);
-        const uint32_t ww[4] = {v.x, v.y, v.z, v.w};
+  for (int q0 = threadIdx.x; q0 < a.GW; q0 += 2 * kQprepThreads) {
+    const int q1 = q0 + kQprepThreads;
+    const bool two = q1 < a.GW;
+    const uint16_t* row0 = a.Q + b * a.qs_b + (long long)(h * a.G + q0 / a.W) * a.qs_h + (q0 % a.W) * a.qs_w;
+    const uint16_t* row1 = two ? a.Q + b * a.qs_b + (long long)(h * a.G + q1 / a.W) * a.qs_h + (q1 % a.W) * a.qs_w : row0;
+    double acc0[K], acc1[K];
+#pragma unroll
+    for (int bit = 0; bit < K; ++bit) { acc0[bit] = 0.0; acc1[bit] = 0.0; }
+    for (int c = 0; c < 128; c += 8) {
+      const uint4 v0 = *reinterpret_cast<const uint4*>(row0 + c);
+      const uint4 v1 = *reinterpret_cast<const uint4*>(row1 + c);
+      const uint32_t w0[4] = {v0.x, v0.y, v0.z, v0.w};
+      const uint32_t w1[4] = {v1.x, v1.y, v1.z, v1.w};
+      double x0[8], x1[8];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        x0[2 * e] = bf16_to_f64((uint16_t)(w0[e] & 0xFFFF));
+        x0[2 * e + 1] = bf16_to_f64((uint16_t)(w0[e] >> 16));
+        x1[2 * e] = bf16_to_f64((uint16_t)(w1[e] & 0xFFFF));
+        x1[2 * e + 1] = bf16_to_f64((uint16_t)(w1[e] >> 16));
+      }
+#pragma unroll
+      for (int bit = 0; bit < K; ++bit) {
+        const double2* p = reinterpret_cast<const double2*>(planes + bit * 128 + c);
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-          acc = fma(bf16_to_f64((uint16_t)(ww[e] & 0xFFFF)), p[c + 2 * e], acc);
-          acc = fma(bf16_to_f64((uint16_t)(ww[e] >> 16)), p[c + 2 * e + 1], acc);
+          const double2 pp = p[e];
+          acc0[bit] = fma(x0[2 * e], pp.x, acc0[bit]);
+          acc0[bit] = fma(x0[2 * e + 1], pp.y, acc0[bit]);
+          acc1[bit] = fma(x1[2 * e], pp.x, acc1[bit]);
+          acc1[bit] = fma(x1[2 * e + 1], pp.y, acc1[bit]);
         }
       }
-      code = (code << 1) | (acc >= 0.0 ? 1u : 0u);
     }
-    atomicAdd(&bins[code], 1u);
-    a.qbuckets[((size_t)(b * a.H_kv + h) * a.GW + q) * a.L + r] = (uint16_t)code;
+    uint32_t code0 = 0, code1 = 0;
+#pragma unroll
+    for (int bit = 0; bit < K; ++bit) {
+      code0 = (code0 << 1) | (acc0[bit] >= 0.0 ? 1u : 0u);
+      code1 = (code1 << 1) | (acc1[bit] >= 0.0 ? 1u : 0u);
+    }
+    atomicAdd(&bins[code0], 1u);
+    a.qbuckets[((size_t)(b * a.H_kv + h) * a.GW + q0) * a.L + r] = (uint16_t)code0;
+    if (two) {
+      atomicAdd(&bins[code1], 1u);
+      a.qbuckets[((size_t)(b * a.H_kv + h) * a.GW + q1) * a.L + r] = (uint16_t)code1;
+    }
   }
   __syncthreads();
   uint16_t* out = a.hist + ((size_t)(b * a.H_kv + h) * a.L + r) * nbins;
-  for (int i = threadIdx.x; i < nbins; i += blockDim.x) out[i] = (uint16_t)bins[i];
+  for (int i = threadIdx.x; i < nbins; i += kQprepThreads) out[i] = (uint16_t)bins[i];
 }
 
 // ------------------------------------------------------------------------------------------------
-// Exact recomputation of flagged key signs. One warp per item; fp64 accumulation of the exact
-// bf16 products. If the exact bucket code differs from the provisional one the key's count is
-// corrected by hist[new] - hist[old].
+// Exact recomputation of flagged key signs. One warp per item; every lane holds four key elements
+// and forms its share of all K dot products at once (independent fp64 accumulators, exact bf16
+// products), then the K partial sums are reduced across the warp. If the exact bucket code
+// differs from the provisional one the key's count is corrected by hist[new] - hist[old].
 // ------------------------------------------------------------------------------------------------
 struct SignfixArgs {
   const uint16_t* Kp;     // keys via strides
@@ -86,6 +120,9 @@ struct SignfixArgs {
   int* n_changed;
 };
 
+constexpr int kMaxLshBits = 12;
+constexpr int kSignfixCtas = 1184;   // 8 CTAs of 8 warps per SM: a few items per warp at most
+
 __global__ void __launch_bounds__(256) signfix_kernel(const SignfixArgs a) {
   const int lane = threadIdx.x & 31;
   const int wid = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -99,19 +136,30 @@ __global__ void __launch_bounds__(256) signfix_kernel(const SignfixArgs a) {
     const int b = seg / (a.nb * a.H_kv);
     const uint16_t* krow = a.Kp + b * a.ks_b + h * a.ks_h + ((long long)t * a.S + key) * a.ks_t;
     const uint2 kv = *reinterpret_cast<const uint2*>(krow + lane * 4);
+    uint2 pv[kMaxLshBits];
+#pragma unroll
+    for (int bit = 0; bit < kMaxLshBits; ++bit)
+      pv[bit] = (bit < a.K) ? *reinterpret_cast<const uint2*>(a.P + ((size_t)r * a.K + bit) * 128 + lane * 4)
+                            : make_uint2(0u, 0u);
     const double k0 = bf16_to_f64((uint16_t)(kv.x & 0xFFFF)), k1 = bf16_to_f64((uint16_t)(kv.x >> 16));
     const double k2 = bf16_to_f64((uint16_t)(kv.y & 0xFFFF)), k3 = bf16_to_f64((uint16_t)(kv.y >> 16));
-    uint32_t code = 0;
-    for (int bit = 0; bit < a.K; ++bit) {
-      const uint2 pv = *reinterpret_cast<const uint2*>(a.P + ((size_t)r * a.K + bit) * 128 + lane * 4);
-      double acc = k0 * bf16_to_f64((uint16_t)(pv.x & 0xFFFF));
-      acc = fma(k1, bf16_to_f64((uint16_t)(pv.x >> 16)), acc);
-      acc = fma(k2, bf16_to_f64((uint16_t)(pv.y & 0xFFFF)), acc);
-      acc = fma(k3, bf16_to_f64((uint16_t)(pv.y >> 16)), acc);
+    double acc[kMaxLshBits];
 #pragma unroll
-      for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
-      code = (code << 1) | (acc >= 0.0 ? 1u : 0u);
+    for (int bit = 0; bit < kMaxLshBits; ++bit) {
+      double s = k0 * bf16_to_f64((uint16_t)(pv[bit].x & 0xFFFF));
+      s = fma(k1, bf16_to_f64((uint16_t)(pv[bit].x >> 16)), s);
+      s = fma(k2, bf16_to_f64((uint16_t)(pv[bit].y & 0xFFFF)), s);
+      acc[bit] = fma(k3, bf16_to_f64((uint16_t)(pv[bit].y >> 16)), s);
     }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+#pragma unroll
+      for (int bit = 0; bit < kMaxLshBits; ++bit) acc[bit] += __shfl_xor_sync(0xffffffffu, acc[bit], off);
+    }
+    uint32_t code = 0;
+#pragma unroll
+    for (int bit = 0; bit < kMaxLshBits; ++bit)
+      if (bit < a.K) code = (code << 1) | (acc[bit] >= 0.0 ? 1u : 0u);
     if (lane == 0 && (int)code != old_code) {
       const uint16_t* hr = a.hist + ((size_t)(b * a.H_kv + h) * a.L + r) * ((size_t)1 << a.K);
       const uint32_t delta = (uint32_t)hr[code] - (uint32_t)hr[old_code];

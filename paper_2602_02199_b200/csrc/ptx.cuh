@@ -245,6 +245,22 @@ __device__ __forceinline__ void tmem_wait_ld_dep16(uint32_t* r) {
                : "memory");
 }
 
+// Orders every later use of r[0..N) after the preceding volatile asm statements (in particular a
+// tcgen05.wait::ld) without emitting an instruction: the registers are named as read-write
+// operands of an empty volatile asm. N must be a multiple of 2.
+template <int N>
+__device__ __forceinline__ void reg_fence(uint32_t* r) {
+  static_assert(N % 2 == 0, "even register count");
+  if constexpr (N >= 8) {
+    asm volatile("" : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7])
+                 :: "memory");
+    reg_fence<N - 8>(r + 8);
+  } else if constexpr (N >= 2) {
+    asm volatile("" : "+r"(r[0]), "+r"(r[1]) :: "memory");
+    reg_fence<N - 2>(r + 2);
+  }
+}
+
 // 2^x on the FMA pipe (no MUFU): round-to-nearest split x = n + f, f in [-0.5, 0.5], degree-4
 // minimax polynomial for 2^f (max relative error 2.7e-6), exponent patched in with one integer
 // multiply-add. Valid for x >= -126 after the clamp; larger negatives return 2^-126.
@@ -258,6 +274,23 @@ __device__ __forceinline__ float ex2_poly(float x) {
   p = fmaf(p, f, 0.6931217908859253f);
   p = fmaf(p, f, 0.9999992847442627f);
   return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+}
+
+// Three-input minimum / maximum of magnitudes, one instruction each.
+__device__ __forceinline__ float min3_abs(float a, float b, float c) {
+  float d;
+  asm("min.abs.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+__device__ __forceinline__ float max3_abs(float a, float b, float c) {
+  float d;
+  asm("max.abs.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
 }
 
 __device__ __forceinline__ float ex2_approx(float x) {

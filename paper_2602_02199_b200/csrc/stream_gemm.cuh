@@ -100,61 +100,81 @@ __device__ __forceinline__ void record_status(int* status, int code) {
   atomicCAS(status, kStatusOk, code);
 }
 
+// Loads the 32-bit columns [CB, CE) of the calling thread's TMEM lane into r[0 .. CE-CB) as a
+// sequence of power-of-two loads, each starting at a multiple of its own width.
+template <int CB, int CE>
+__device__ __forceinline__ void tmem_ld_range(uint32_t taddr, uint32_t* r) {
+  if constexpr (CB < CE) {
+    constexpr int W = (CB % 32 == 0 && CB + 32 <= CE) ? 32
+                    : (CB % 16 == 0 && CB + 16 <= CE) ? 16
+                    : (CB % 8 == 0 && CB + 8 <= CE)   ? 8
+                    : (CB % 4 == 0 && CB + 4 <= CE)   ? 4
+                    : (CB % 2 == 0 && CB + 2 <= CE)   ? 2 : 1;
+    tmem_ld_cols<W>(taddr + CB, r);
+    tmem_ld_range<CB + W, CE>(taddr, r + W);
+  }
+}
+
 // Tables [T_BEGIN, T_END) of the chunk for the calling thread's key: packs the sign bits of each
 // table's K projections into a bucket code, looks the code up in the histogram slice and
 // returns the summed collisions. A table whose smallest |projection| is below 2^-15 of the
 // largest |projection| among the key's first 16 hyperplanes of the chunk is queued for an exact
-// recomputation of its signs.
+// recomputation of its signs. All of the thread's columns are read into registers first and the
+// accumulator buffer is handed back to the MMA warp (arrive on `bar_release`) before the
+// arithmetic starts; the per-table work is branch-free so that the tables interleave.
 template <int KBITS, int T_BEGIN, int T_END>
-__device__ __forceinline__ uint32_t proj_tables(uint32_t t_acc, const uint16_t* hist_s, const StreamArgs& a,
-                                                int seg, int key, int table0, bool valid) {
+__device__ __forceinline__ uint32_t proj_tables(uint32_t t_acc, uint32_t bar_release, const uint16_t* hist_s,
+                                                const StreamArgs& a, int seg, int key, int table0, bool valid) {
+  constexpr int NT = T_END - T_BEGIN;
   constexpr int CB = T_BEGIN * KBITS, CE = T_END * KBITS;
-  constexpr int L0 = CB / 32 * 32;
-  constexpr int NCHUNK = (CE - L0 + 31) / 32;
   constexpr uint32_t bucket_mask = (1u << KBITS) - 1u;
-  uint32_t v[2][32];
+  uint32_t v[CE - CB];
   uint32_t v16[16];
-  tmem_ld_x32(t_acc + L0, v[0]);
+  tmem_ld_range<CB, CE>(t_acc, v);
   tmem_ld_x16(t_acc, v16);
-  tmem_wait_ld_dep32(v[0]);
-  tmem_wait_ld_dep16(v16);
+  tmem_wait_ld();
+  reg_fence<CE - CB>(v);
+  reg_fence<16>(v16);
+  tc_fence_before();
+  mbar_arrive(bar_release);
   float amax = 0.f;
 #pragma unroll
-  for (int k = 0; k < 16; ++k) amax = fmaxf(amax, fabsf(__uint_as_float(v16[k])));
+  for (int k = 0; k < 16; k += 2) amax = max3_abs(__uint_as_float(v16[k]), __uint_as_float(v16[k + 1]), amax);
   const float tau = amax * (1.0f / 32768.0f);
-  uint32_t partial = 0, neg = 0;
-  float amin = INFINITY;
+  uint32_t code[NT];
+  float amin[NT];
 #pragma unroll
-  for (int c = 0; c < NCHUNK; ++c) {
-    if (c + 1 < NCHUNK) tmem_ld_x32(t_acc + L0 + 32 * (c + 1), v[(c + 1) & 1]);
+  for (int t = 0; t < NT; ++t) {
+    uint32_t neg = 0;
+    float mn = INFINITY;
 #pragma unroll
-    for (int k = 0; k < 32; k += 2) {
-      const int col = L0 + 32 * c + k;
-      // K is even and CB is a multiple of K, so a pair of columns never straddles two tables
-      if (col >= CB && col < CE) {
-        const uint32_t x0 = v[c & 1][k], x1 = v[c & 1][k + 1];
-        neg = __funnelshift_l(x0, neg, 1);                 // (neg << 1) | sign(x0)
-        neg = __funnelshift_l(x1, neg, 1);
-        amin = fminf(amin, fminf(fabsf(__uint_as_float(x0)), fabsf(__uint_as_float(x1))));
-        if ((col + 1) % KBITS == KBITS - 1) {
-          const int rl = (col + 1) / KBITS;                // table within the chunk
-          const uint32_t code = (~neg) & bucket_mask;
-          partial += hist_s[((uint32_t)rl << KBITS) + code];
-          if (valid) {
-            const int r = table0 + rl;
-            if (a.key_buckets) a.key_buckets[((size_t)seg * a.S + key) * a.lsh_tables + r] = (uint16_t)code;
-            if (!(amin >= tau)) {
-              const int slot = atomicAdd(a.fix_count, 1);
-              if (slot < a.fix_cap) a.fix_items[slot] = make_int4(seg, key, r, (int)code);
-              else record_status(a.status, kStatusCapacity);
-            }
-          }
-          neg = 0;
-          amin = INFINITY;
-        }
+    for (int k = 0; k < KBITS; k += 2) {
+      const uint32_t x0 = v[t * KBITS + k], x1 = v[t * KBITS + k + 1];
+      neg = __funnelshift_l(x0, neg, 1);                   // (neg << 1) | sign(x0)
+      neg = __funnelshift_l(x1, neg, 1);
+      mn = min3_abs(__uint_as_float(x0), __uint_as_float(x1), mn);
+    }
+    code[t] = (~neg) & bucket_mask;
+    amin[t] = mn;
+  }
+  uint32_t partial = 0;
+  float lowest = INFINITY;
+#pragma unroll
+  for (int t = 0; t < NT; ++t) {
+    partial += hist_s[((uint32_t)(T_BEGIN + t) << KBITS) + code[t]];
+    lowest = fminf(lowest, amin[t]);
+  }
+  if (valid && (a.key_buckets != nullptr || !(lowest >= tau))) {
+#pragma unroll
+    for (int t = 0; t < NT; ++t) {
+      const int r = table0 + T_BEGIN + t;
+      if (a.key_buckets) a.key_buckets[((size_t)seg * a.S + key) * a.lsh_tables + r] = (uint16_t)code[t];
+      if (!(amin[t] >= tau)) {
+        const int slot = atomicAdd(a.fix_count, 1);
+        if (slot < a.fix_cap) a.fix_items[slot] = make_int4(seg, key, r, (int)code[t]);
+        else record_status(a.status, kStatusCapacity);
       }
     }
-    if (c + 1 < NCHUNK) tmem_wait_ld_dep32(v[(c + 1) & 1]);
   }
   return partial;
 }
@@ -451,11 +471,10 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
         const int key = (tile0 + i) * kTileKeys + row;
         const bool valid = key < a.S;
         const uint32_t t_acc = t_lane + acc * kAccStride;
+        const uint32_t bar_rel = bar_tempty + 8 * acc;
         uint32_t partial;
-        if (wg == 0) partial = proj_tables<KBITS, 0, TC / 2>(t_acc, hist_s, a, seg, key, chunk * TC, valid);
-        else partial = proj_tables<KBITS, TC / 2, TC>(t_acc, hist_s, a, seg, key, chunk * TC, valid);
-        tc_fence_before();
-        mbar_arrive(bar_tempty + 8 * acc);
+        if (wg == 0) partial = proj_tables<KBITS, 0, TC / 2>(t_acc, bar_rel, hist_s, a, seg, key, chunk * TC, valid);
+        else partial = proj_tables<KBITS, TC / 2, TC>(t_acc, bar_rel, hist_s, a, seg, key, chunk * TC, valid);
         if (valid) atomicAdd(a.counts + (size_t)seg * a.S + key, partial);
       }
     }
