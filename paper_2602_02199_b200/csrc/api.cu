@@ -40,7 +40,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 
 struct Derived {
   int B, anchors, k_exact, k_lsh, G, GW;
-  int tiles_in_block, tiles_per_cta, n_split;
+  int tiles_in_block;
   int TC, n_chunks;
   double alpha, ratio;
   float scale;
@@ -68,6 +68,7 @@ struct laser_kv_ctx {
   const uint16_t* P = nullptr;
   CUtensorMap mapP;
   EncodeTiledFn encode = nullptr;
+  int num_sms = 1;
   std::vector<long long> blocks_done;   // per layer
   std::string last_error;
   bool have_call = false;
@@ -96,6 +97,23 @@ laser_kv_status_t fail(laser_kv_ctx* h, laser_kv_status_t s, const char* fmt, ..
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// Persistent grid of a streaming launch: one CTA per SM, never more CTAs than tiles.
+int stream_grid(long long n_tiles, int num_sms) {
+  long long g = num_sms < kMaxStreamCtas ? num_sms : kMaxStreamCtas;
+  if (g < 1) g = 1;
+  return (int)(n_tiles < g ? n_tiles : g);
+}
+
+// Log-sum-exp partial slots per segment when `grid` CTAs split the tiles of `nseg` equally long
+// segments into equal contiguous slices: a segment meets at most ceil(grid / nseg) + 1 slices.
+int lse_slots(int grid, int nseg) { return (grid + nseg - 1) / nseg + 1; }
+
+// Bytes that hold the partials of any launch over at most `nseg_max` segments, whatever the grid:
+// nseg * lse_slots(grid, nseg) <= grid + 2 * nseg.
+size_t lse_part_bytes_bound(size_t nseg_max, int GW) {
+  return ((size_t)kMaxStreamCtas + 2 * nseg_max) * (size_t)GW * sizeof(float2);
+}
+
 // Largest supported tables-per-chunk for the projection pass: K*TC a multiple of 16 and at
 // most 256 columns, L divisible by TC, histogram slice + operands within shared memory.
 int pick_tc(int K, int L) {
@@ -104,7 +122,7 @@ int pick_tc(int K, int L) {
     if (L % tc) continue;
     const int n = K * tc;
     if (n > 256 || (n % 16)) continue;
-    const uint32_t smem = stream_smem_bytes(kProj, n, tc * (2 << K), 0);
+    const uint32_t smem = stream_smem_bytes(kProj, n, tc * (2 << K));
     if (smem > (uint32_t)kMaxSmem) continue;
     return tc;
   }
@@ -153,8 +171,8 @@ laser_kv_status_t derive(const laser_kv_config_t* c, Derived* d) {
     return fail(nullptr, LASER_KV_ERR_UNSUPPORTED, "config: G*W*lsh_tables too large");
   d->n_chunks = c->lsh_tables / d->TC;
   d->tiles_in_block = (c->block_size + kTileKeys - 1) / kTileKeys;
-  d->tiles_per_cta = d->tiles_in_block < 16 ? d->tiles_in_block : 16;
-  d->n_split = (d->tiles_in_block + d->tiles_per_cta - 1) / d->tiles_per_cta;
+  if (c->softmax_scale < 0.f || c->softmax_scale != c->softmax_scale)
+    return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "config: softmax_scale must be positive (0 selects 1/sqrt(head_dim))");
   d->scale = c->softmax_scale == 0.f ? 1.0f / std::sqrt((float)c->head_dim) : c->softmax_scale;
   d->cap = (long long)c->max_blocks * d->B;
   const long long nseg = (long long)c->batch * c->n_kv_heads * c->max_blocks_per_call;
@@ -175,7 +193,7 @@ void carve_ws(const laser_kv_config_t* c, const Derived& d, Carve* v) {
   v->ctrl = take(256);
   v->hist = take(bh * c->lsh_tables * ((size_t)2 << c->lsh_bits));
   v->qbuckets = take(bh * d.GW * c->lsh_tables * 2);
-  v->lse_part = take(nseg * d.n_split * d.GW * sizeof(float2));
+  v->lse_part = take(lse_part_bytes_bound(nseg, d.GW));
   v->lse2 = take(nseg * d.GW * 4);
   v->s_exact = take(nseg * S * 4);
   v->counts = take(nseg * S * 4);
@@ -343,6 +361,7 @@ laser_kv_status_t laser_kv_init(const laser_kv_config_t* cfg, const void* hyperp
   h->carve = v;
   h->ws = static_cast<uint8_t*>(workspace);
   h->encode = reinterpret_cast<EncodeTiledFn>(fn);
+  h->num_sms = prop.multiProcessorCount;
   const size_t per = (size_t)cfg->n_layers * cfg->batch * cfg->n_kv_heads * (size_t)d.cap;
   uint8_t* cm = static_cast<uint8_t*>(cache_mem);
   h->cacheK = reinterpret_cast<uint16_t*>(cm);
@@ -472,23 +491,25 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
 
   StreamArgs sa;
   memset(&sa, 0, sizeof sa);
-  sa.S = S; sa.nb = nb; sa.t0 = 0; sa.tn = nb; sa.H_kv = c.n_kv_heads; sa.batch = c.batch;
+  sa.S = S; sa.nb = nb; sa.H_kv = c.n_kv_heads; sa.batch = c.batch;
   sa.G = d.G; sa.W = c.window; sa.GW = d.GW;
-  sa.tiles_per_cta = d.tiles_per_cta; sa.n_split = d.n_split;
+  sa.tiles_in_block = d.tiles_in_block; sa.nseg = nseg;
+  const long long seg_tiles = (long long)nseg * d.tiles_in_block;
+  const int base_ctas = stream_grid(seg_tiles, h->num_sms);
+  sa.n_tiles = seg_tiles; sa.lse_ctas = base_ctas; sa.n_slot = lse_slots(base_ctas, nseg);
   sa.n_chunks = d.n_chunks; sa.tables_per_chunk = d.TC; sa.lsh_bits = c.lsh_bits; sa.lsh_tables = c.lsh_tables;
   sa.scale_log2e = d.scale * 1.4426950408889634f;
   sa.lse_part = lse_part; sa.lse2 = lse2; sa.s_exact = s_exact; sa.counts = counts; sa.hist = hist;
   sa.key_buckets = key_buckets; sa.fix_items = fix_items; sa.fix_count = ctrl + 1; sa.fix_cap = d.fix_cap;
   sa.status = ctrl;
 
-  const int base_ctas = c.batch * c.n_kv_heads * nb * d.n_split;
   mark();
   // 2. per-query log-sum-exp over each block's keys
   {
     StreamArgs a1 = sa;
     a1.stat_rows = d.GW;
     a1.stat_rows_alloc = ((d.GW + 127) / 128) * 128;
-    const uint32_t smem = stream_smem_bytes(kLse, a1.stat_rows_alloc, 0, d.GW);
+    const uint32_t smem = stream_smem_bytes(kLse, a1.stat_rows_alloc, 0);
     LKV_CUDA((launch_stream<kLse, 0, 0>(mapK, mapQ, a1, base_ctas, smem, st)), "lse pass");
   }
   mark();
@@ -497,7 +518,7 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
     StreamArgs a2 = sa;
     a2.stat_rows = d.GW;
     a2.stat_rows_alloc = d.GW;
-    const uint32_t smem = stream_smem_bytes(kScore, a2.stat_rows_alloc, 0, d.GW);
+    const uint32_t smem = stream_smem_bytes(kScore, a2.stat_rows_alloc, 0);
     LKV_CUDA((launch_stream<kScore, 0, 0>(mapK, mapQ, a2, base_ctas, smem, st)), "score pass");
   }
   mark();
@@ -506,8 +527,10 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
     StreamArgs a3 = sa;
     a3.stat_rows = d.TC * c.lsh_bits;
     a3.stat_rows_alloc = a3.stat_rows;
-    const uint32_t smem = stream_smem_bytes(kProj, a3.stat_rows_alloc, d.TC * (2 << c.lsh_bits), 0);
-    LKV_CUDA(launch_proj(c.lsh_bits, d.TC, mapK, h->mapP, a3, base_ctas * d.n_chunks, smem, st), "projection pass");
+    a3.n_tiles = seg_tiles * d.n_chunks;
+    const uint32_t smem = stream_smem_bytes(kProj, a3.stat_rows_alloc, d.TC * (2 << c.lsh_bits));
+    LKV_CUDA(launch_proj(c.lsh_bits, d.TC, mapK, h->mapP, a3, stream_grid(a3.n_tiles, h->num_sms), smem, st),
+             "projection pass");
   }
   mark();
   // 5. exact signs where the tensor-core projection was too close to zero
@@ -722,7 +745,7 @@ laser_kv_status_t laser_kv_two_stage_topk(const float* s_exact, const uint32_t* 
 namespace {
 
 struct ScoreGeom {
-  int batch, H_q, H_kv, S, W, nb, G, GW, tiles_in_block, tiles_per_cta, n_split, nseg;
+  int batch, H_q, H_kv, S, W, nb, G, GW, tiles_in_block, nseg;
   float scale;
   size_t off_part, off_lse2, total;   // scratch layout: [0,256) status word, partials, lse2
 };
@@ -742,11 +765,11 @@ laser_kv_status_t score_geometry(int32_t batch, int32_t n_q_heads, int32_t n_kv_
     return fail(nullptr, LASER_KV_ERR_UNSUPPORTED, "window_scores: too many segments");
   g->nseg = (int)nseg;
   g->tiles_in_block = (block_size + kTileKeys - 1) / kTileKeys;
-  g->tiles_per_cta = g->tiles_in_block < 16 ? g->tiles_in_block : 16;
-  g->n_split = (g->tiles_in_block + g->tiles_per_cta - 1) / g->tiles_per_cta;
+  if (softmax_scale < 0.f || softmax_scale != softmax_scale)
+    return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "window_scores: softmax_scale must be positive (0 selects 1/sqrt(128))");
   g->scale = softmax_scale == 0.f ? 1.0f / std::sqrt((float)kHeadDim) : softmax_scale;
   g->off_part = 256;
-  g->off_lse2 = align_up(g->off_part + (size_t)g->nseg * g->n_split * g->GW * sizeof(float2));
+  g->off_lse2 = align_up(g->off_part + lse_part_bytes_bound((size_t)g->nseg, g->GW));
   g->total = align_up(g->off_lse2 + (size_t)g->nseg * g->GW * 4);
   return LASER_KV_OK;
 }
@@ -810,23 +833,29 @@ laser_kv_status_t run_window_scores(const ScoreGeom& g, const void* K_blk, const
     return fail(nullptr, LASER_KV_ERR_CUDA, "window_scores: memset: %s", cudaGetErrorString(e));
   StreamArgs sa;
   memset(&sa, 0, sizeof sa);
-  sa.S = g.S; sa.nb = g.nb; sa.t0 = 0; sa.tn = g.nb; sa.H_kv = g.H_kv; sa.batch = g.batch;
-  sa.G = g.G; sa.W = g.W; sa.GW = g.GW; sa.tiles_per_cta = g.tiles_per_cta; sa.n_split = g.n_split;
+  int dev = 0, num_sms = 0;
+  if ((e = cudaGetDevice(&dev)) != cudaSuccess ||
+      (e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess)
+    return fail(nullptr, LASER_KV_ERR_CUDA, "window_scores: device query: %s", cudaGetErrorString(e));
+  sa.S = g.S; sa.nb = g.nb; sa.H_kv = g.H_kv; sa.batch = g.batch;
+  sa.G = g.G; sa.W = g.W; sa.GW = g.GW; sa.tiles_in_block = g.tiles_in_block; sa.nseg = g.nseg;
+  sa.n_tiles = (long long)g.nseg * g.tiles_in_block;
+  const int ctas = stream_grid(sa.n_tiles, num_sms);
+  sa.lse_ctas = ctas; sa.n_slot = lse_slots(ctas, g.nseg);
   sa.scale_log2e = g.scale * 1.4426950408889634f;
   sa.lse_part = reinterpret_cast<float2*>(scratch + g.off_part);
   sa.lse2 = reinterpret_cast<float*>(scratch + g.off_lse2);
   sa.s_exact = s_exact_out;
   sa.status = reinterpret_cast<int*>(scratch);
-  const int ctas = g.nseg * g.n_split;
   StreamArgs a1 = sa;
   a1.stat_rows = g.GW;
   a1.stat_rows_alloc = ((g.GW + 127) / 128) * 128;
-  if ((e = launch_stream<kLse, 0, 0>(mapK, mapQ, a1, ctas, stream_smem_bytes(kLse, a1.stat_rows_alloc, 0, g.GW), st)) != cudaSuccess)
+  if ((e = launch_stream<kLse, 0, 0>(mapK, mapQ, a1, ctas, stream_smem_bytes(kLse, a1.stat_rows_alloc, 0), st)) != cudaSuccess)
     return fail(nullptr, LASER_KV_ERR_CUDA, "window_scores: lse pass: %s", cudaGetErrorString(e));
   StreamArgs a2 = sa;
   a2.stat_rows = g.GW;
   a2.stat_rows_alloc = g.GW;
-  if ((e = launch_stream<kScore, 0, 0>(mapK, mapQ, a2, ctas, stream_smem_bytes(kScore, a2.stat_rows_alloc, 0, g.GW), st)) != cudaSuccess)
+  if ((e = launch_stream<kScore, 0, 0>(mapK, mapQ, a2, ctas, stream_smem_bytes(kScore, a2.stat_rows_alloc, 0), st)) != cudaSuccess)
     return fail(nullptr, LASER_KV_ERR_CUDA, "window_scores: score pass: %s", cudaGetErrorString(e));
   return LASER_KV_OK;
 }

@@ -1,24 +1,30 @@
 // Key-streaming tensor-core kernels for the two dense contractions of the selection path:
 //   * the window-score contraction Q_win . K^T  (Section 3.3 "Precision", Algorithm 1 line 3)
 //   * the hyperplane projection K . P^T         (Section 3.3 "Recall", hash functions h_r)
-// One warp-specialised skeleton serves three passes. A CTA keeps one small operand stationary
-// in shared memory (the group's window queries, or a chunk of hyperplanes with the matching
-// slice of the query-bucket histogram) and streams 128-key tiles of one (sequence, KV head,
-// block) through a TMA -> tcgen05.mma -> TMEM -> register pipeline:
+// One persistent, warp-specialised skeleton serves three passes. The 128-key tiles of a launch
+// form one sequence (hyperplane chunk, sequence, KV head, block, tile); every CTA owns a
+// contiguous, equally long slice of it. A CTA keeps one small operand stationary in shared
+// memory (the window queries of the current KV head, or a chunk of hyperplanes with the matching
+// slice of the query-bucket histogram), reloads it only when its slice crosses into another
+// head or chunk, and streams key tiles through a TMA -> tcgen05.mma -> TMEM -> register pipeline:
 //
-//   kLse   : D[query][key]; every thread owns one query row and keeps an online
-//            (max, sum-exp2) pair over the CTA's keys -> per-split partials of log-sum-exp.
-//   kScore : D[key][query]; every thread owns one key and sums exp2(s - lse_q) over the
-//            group's queries -> S_exact[key].
-//   kProj  : D[key][hyperplane]; every thread owns one key, packs sign bits into K-bit bucket
-//            ids, looks the buckets up in the query-bucket histogram (count of window queries
-//            per bucket) and adds the collisions to count[key]. Signs decided by a projection
-//            that is tiny relative to the key's other projections are queued for an exact
-//            recomputation.
+//   kLse   : D[query][key]; a thread owns one query row and a range of key columns and keeps an
+//            online (max, sum-exp2) pair; at the end of each block's run of tiles the column
+//            groups are merged and one partial per (block segment, CTA) goes to global memory.
+//   kScore : D[key][query]; a thread owns one key and a range of query columns and sums
+//            exp2(s - lse_q); the four column groups are added in a fixed order -> S_exact[key].
+//   kProj  : D[key][hyperplane]; a thread owns one key and a range of tables, packs sign bits
+//            into K-bit bucket ids, looks the buckets up in the query-bucket histogram (count of
+//            window queries per bucket) and adds the collisions to count[key]. Signs decided by
+//            a projection that is tiny relative to the key's other projections are queued for
+//            an exact recomputation.
 //
-// Warp roles (320 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner,
-// warps 2..9 = two epilogue groups of four warps (TMEM lane quarter = warp_id % 4) that split
-// the accumulator columns of every tile.
+// Warp roles (576 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner,
+// warps 2..17 = four epilogue groups of four warps (TMEM lane quarter = warp_id % 4) that split
+// the accumulator columns of every tile. An epilogue thread copies its columns to registers,
+// hands the accumulator buffer back to the MMA warp and only then does its arithmetic.
+// All cross-warp hand-offs are mbarriers with bounded waits; there is no CTA-wide barrier
+// inside the tile loop.
 #pragma once
 #include "ptx.cuh"
 
@@ -29,62 +35,38 @@ constexpr int kAtomCols = 64;                  // bf16 elements per 128-byte swi
 constexpr int kTileAtomBytes = kTileKeys * 128;  // one 64-column half of a key tile
 constexpr int kTileBytes = 2 * kTileAtomBytes;   // 128 keys x 128 dims bf16
 constexpr int kStages = 4;
-constexpr int kStreamThreads = 320;
-constexpr int kEpilogueThreads = 256;
-constexpr int kXwgBytes = 2048;                // exchange area between the two epilogue groups
+constexpr int kEpiGroups = 4;
+constexpr int kEpilogueThreads = kEpiGroups * 128;
+constexpr int kStreamThreads = 64 + kEpilogueThreads;
+constexpr int kEpiCols = 64;                   // accumulator columns an epilogue thread holds at most
+constexpr int kXchBytes = 8192;                // exchange area between epilogue warps
 constexpr int kTmemCols = 512;
 constexpr int kAccStride = 256;                // TMEM columns per accumulator buffer
 constexpr int kMaxStatRows = 256;
+constexpr int kMaxStreamCtas = 256;            // upper bound of the persistent grid (slot arithmetic)
+constexpr int kPolyPairsOf32 = 12;             // of every 32 column pairs, this many take 2^x on the FMA pipe
 
 enum StreamMode { kLse = 0, kScore = 1, kProj = 2 };
 
 enum : int { kStatusOk = 0, kStatusCapacity = 3, kStatusTimeout = 6 };
 
-template <int N> struct IntTag { static constexpr int value = N; };
-
-// Walks the 32-bit columns [c_begin, c_end) of the calling thread's TMEM lane (c_begin a multiple
-// of 32, length a multiple of 16 and at most 128) in chunks of 32 (a last chunk of 16), loading
-// chunk i+1 while f(values, first column, IntTag<count>) works on chunk i.
-template <class F>
-__device__ __forceinline__ void walk_columns(uint32_t taddr, int c_begin, int c_end, F&& f) {
-  const int n = c_end - c_begin;
-  if (n <= 0) return;
-  uint32_t va[32], vb[32];
-  if (n >= 32) { tmem_ld_x32(taddr + c_begin, va); tmem_wait_ld_dep32(va); }
-  else { tmem_ld_x16(taddr + c_begin, va); tmem_wait_ld_dep16(va); }
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int off = i * 32;
-    if (off < n) {
-      uint32_t* cur = (i & 1) ? vb : va;
-      uint32_t* nxt = (i & 1) ? va : vb;
-      const int rest = n - off - 32;       // columns after this chunk
-      if (rest >= 32) tmem_ld_x32(taddr + c_begin + off + 32, nxt);
-      else if (rest > 0) tmem_ld_x16(taddr + c_begin + off + 32, nxt);
-      if (n - off >= 32) f(cur, c_begin + off, IntTag<32>{});
-      else f(cur, c_begin + off, IntTag<16>{});
-      if (rest >= 32) tmem_wait_ld_dep32(nxt);
-      else if (rest > 0) tmem_wait_ld_dep16(nxt);
-    }
-  }
-}
-
-
 struct StreamArgs {
   // problem geometry
   int S;               // keys per block
   int nb;              // blocks in this call
-  int t0, tn;          // block range [t0, t0 + tn) handled by this launch
   int H_kv, batch;
   int G, W, GW;        // GQA group size, window, G*W
-  int tiles_per_cta;   // key tiles per CTA
-  int n_split;         // CTAs along the keys of one block
+  int tiles_in_block;  // ceil(S / 128)
+  int nseg;            // batch * H_kv * nb
+  long long n_tiles;   // tiles of this launch: nseg * tiles_in_block (* n_chunks for kProj)
+  int lse_ctas;        // grid of the kLse launch over the same segments (slot arithmetic)
+  int n_slot;          // log-sum-exp partial slots per segment
   int stat_rows;       // rows of the stationary operand (GW, or tables_per_chunk * lsh_bits)
   int stat_rows_alloc; // rows reserved per 64-column half in shared memory (multiple of 8)
   int n_chunks, tables_per_chunk, lsh_bits, lsh_tables;
-  float scale_log2e;   // softmax scale * log2(e)
+  float scale_log2e;   // softmax scale * log2(e), positive
   // buffers (device)
-  float2* lse_part;        // [seg][n_split][GW]  (max, sum) in the log2 domain
+  float2* lse_part;        // [seg][n_slot][GW]  (max, sum) in the log2 domain
   float* lse2;             // [seg][GW]
   float* s_exact;          // [seg][S]
   uint32_t* counts;        // [seg][S]
@@ -100,6 +82,35 @@ __device__ __forceinline__ void record_status(int* status, int code) {
   atomicCAS(status, kStatusOk, code);
 }
 
+// The CTA whose slice [c*T/G, (c+1)*T/G) of a T-tile sequence split over G CTAs holds tile x.
+__host__ __device__ inline int cta_of_tile(long long x, long long T, int G) {
+  return (int)(((x + 1) * G - 1) / T);
+}
+
+// Position in the tile sequence.
+struct TileCursor {
+  int chunk, seg, tib;
+};
+__device__ __forceinline__ TileCursor cursor_at(long long x, const StreamArgs& a) {
+  const long long per_chunk = (long long)a.nseg * a.tiles_in_block;
+  TileCursor c;
+  c.chunk = (int)(x / per_chunk);
+  const long long r = x - (long long)c.chunk * per_chunk;
+  c.seg = (int)(r / a.tiles_in_block);
+  c.tib = (int)(r - (long long)c.seg * a.tiles_in_block);
+  return c;
+}
+__device__ __forceinline__ void cursor_advance(TileCursor& c, const StreamArgs& a) {
+  if (++c.tib == a.tiles_in_block) {
+    c.tib = 0;
+    if (++c.seg == a.nseg) { c.seg = 0; ++c.chunk; }
+  }
+}
+// Tiles with the same group id share the stationary operand.
+__device__ __forceinline__ int cursor_group(const TileCursor& c, const StreamArgs& a) {
+  return c.chunk * (a.batch * a.H_kv) + c.seg / a.nb;
+}
+
 // Loads the 32-bit columns [CB, CE) of the calling thread's TMEM lane into r[0 .. CE-CB) as a
 // sequence of power-of-two loads, each starting at a multiple of its own width.
 template <int CB, int CE>
@@ -113,6 +124,54 @@ __device__ __forceinline__ void tmem_ld_range(uint32_t taddr, uint32_t* r) {
     tmem_ld_cols<W>(taddr + CB, r);
     tmem_ld_range<CB + W, CE>(taddr, r + W);
   }
+}
+
+// Reads `ncols` (a multiple of 16, at most 64) columns starting at taddr into v[0..64); the rest
+// of v is set to -infinity, which every consumer turns into a zero contribution.
+__device__ __forceinline__ void load_epi_cols(uint32_t taddr, int ncols, uint32_t* v) {
+#pragma unroll
+  for (int j = 0; j < kEpiCols / 16; ++j) {
+    if (16 * j < ncols) {
+      tmem_ld_x16(taddr + 16 * j, v + 16 * j);
+    } else {
+#pragma unroll
+      for (int k = 0; k < 16; ++k) v[16 * j + k] = 0xff800000u;
+    }
+  }
+  tmem_wait_ld();
+  reg_fence<kEpiCols>(v);
+}
+
+// sum over k < N of 2^(v[k] * c2 + addend[k]); addend is per column (kScore: -lse of the query,
+// read from shared memory) or one value for all columns (kLse: -running max). Pairs of columns
+// go through packed fp32 arithmetic; a fixed subset of the pairs evaluates 2^x with the
+// polynomial on the FMA pipe, the others use the special-function unit.
+template <int N, bool PER_COLUMN>
+__device__ __forceinline__ float sum_exp2(const uint32_t* v, float c2, const float* addend_s, float addend_all) {
+  const float2 c22 = make_float2(c2, c2);
+  float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
+#pragma unroll
+  for (int k = 0; k < N; k += 4) {
+    float2 ad0, ad1;
+    if constexpr (PER_COLUMN) {
+      const float4 ls = *reinterpret_cast<const float4*>(addend_s + k);
+      ad0 = make_float2(ls.x, ls.y);
+      ad1 = make_float2(ls.z, ls.w);
+    } else {
+      ad0 = make_float2(addend_all, addend_all);
+      ad1 = ad0;
+    }
+    const float2 x0 = fma2(make_float2(__uint_as_float(v[k]), __uint_as_float(v[k + 1])), c22, ad0);
+    const float2 x1 = fma2(make_float2(__uint_as_float(v[k + 2]), __uint_as_float(v[k + 3])), c22, ad1);
+    const int p0 = k / 2, p1 = k / 2 + 1;     // pair indices, compile-time after unrolling
+    const float2 e0 = ((p0 * kPolyPairsOf32) % 32 < kPolyPairsOf32) ? ex2_poly2(x0)
+                                                                     : make_float2(ex2_approx(x0.x), ex2_approx(x0.y));
+    const float2 e1 = ((p1 * kPolyPairsOf32) % 32 < kPolyPairsOf32) ? ex2_poly2(x1)
+                                                                     : make_float2(ex2_approx(x1.x), ex2_approx(x1.y));
+    acc0 = add2(acc0, e0);
+    acc1 = add2(acc1, e1);
+  }
+  return (acc0.x + acc0.y) + (acc1.x + acc1.y);
 }
 
 // Tables [T_BEGIN, T_END) of the chunk for the calling thread's key: packs the sign bits of each
@@ -179,17 +238,11 @@ __device__ __forceinline__ uint32_t proj_tables(uint32_t t_acc, uint32_t bar_rel
   return partial;
 }
 
-struct StreamSmem {
-  uint32_t stat, stages, hist, lse, xwg, bars, tmem_slot;  // shared-space byte addresses
-};
-
 // Shared memory carve-up, identical on host (sizes) and device (addresses).
-__host__ __device__ inline uint32_t stream_smem_bytes(int mode, int stat_rows_alloc,
-                                                      int hist_bytes, int GW) {
+__host__ __device__ inline uint32_t stream_smem_bytes(int mode, int stat_rows_alloc, int hist_bytes) {
   uint32_t b = 2u * stat_rows_alloc * 128u + kStages * kTileBytes;
   if (mode == kProj) b += (hist_bytes + 127u) & ~127u;
-  if (mode == kScore) b += ((GW * 4u) + 127u) & ~127u;
-  b += kXwgBytes;
+  b += kXchBytes;    // exchange area: per-warp log-sum-exp values, cross-group partials
   b += 256;          // barriers + TMEM slot
   return b + 1024;   // slack for 1024-byte alignment of the base
 }
@@ -203,123 +256,139 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
 
-  // ---- which work item -------------------------------------------------------------------
-  int bid = blockIdx.x;
-  int chunk = 0;
-  if (MODE == kProj) { chunk = bid % a.n_chunks; bid /= a.n_chunks; }
-  const int split = bid % a.n_split; bid /= a.n_split;
-  const int tl = bid % a.tn; bid /= a.tn;
-  const int h = bid % a.H_kv;
-  const int b = bid / a.H_kv;
-  const int t = a.t0 + tl;
-  const int seg = (b * a.H_kv + h) * a.nb + t;
-  const int tiles_in_block = (a.S + kTileKeys - 1) / kTileKeys;
-  const int tile0 = split * a.tiles_per_cta;
-  const int ntiles = min(a.tiles_per_cta, tiles_in_block - tile0);
+  // ---- this CTA's slice of the tile sequence ------------------------------------------------
+  const long long x_begin = (long long)blockIdx.x * a.n_tiles / gridDim.x;
+  const long long x_end = (long long)(blockIdx.x + 1) * a.n_tiles / gridDim.x;
 
   // ---- shared memory ---------------------------------------------------------------------
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t stat_atom_bytes = a.stat_rows_alloc * 128u;
-  StreamSmem sm;
-  sm.stat = base;
-  sm.stages = sm.stat + 2u * stat_atom_bytes;
-  uint32_t cur = sm.stages + kStages * kTileBytes;
+  const uint32_t sm_stat = base;
+  const uint32_t sm_stages = sm_stat + 2u * stat_atom_bytes;
+  uint32_t cur = sm_stages + kStages * kTileBytes;
   const uint32_t hist_bytes = (MODE == kProj) ? (uint32_t)TC * (2u << KBITS) : 0u;
-  sm.hist = cur;
+  const uint32_t sm_hist = cur;
   if (MODE == kProj) cur += (hist_bytes + 127u) & ~127u;
-  sm.lse = cur;
-  if (MODE == kScore) cur += ((a.GW * 4u) + 127u) & ~127u;
-  sm.xwg = cur;
-  cur += kXwgBytes;
-  sm.bars = cur;
-  sm.tmem_slot = cur + 128;
-  const uint32_t bar_full = sm.bars;                 // kStages barriers
-  const uint32_t bar_empty = sm.bars + 8 * kStages;  // kStages barriers
-  const uint32_t bar_tfull = sm.bars + 16 * kStages; // 2 barriers
-  const uint32_t bar_tempty = bar_tfull + 16;        // 2 barriers
-  const uint32_t bar_stat = bar_tempty + 16;         // 1 barrier
+  const uint32_t sm_xch = cur;
+  cur += kXchBytes;
+  const uint32_t sm_bars = cur;
+  const uint32_t sm_tmem_slot = cur + 192;
+  const uint32_t bar_full = sm_bars;                   // kStages barriers: tile landed
+  const uint32_t bar_empty = sm_bars + 8 * kStages;    // kStages barriers: tile consumed by the MMAs
+  const uint32_t bar_tfull = sm_bars + 16 * kStages;   // 2: accumulator complete
+  const uint32_t bar_tempty = bar_tfull + 16;          // 2: accumulator copied out by all epilogue threads
+  const uint32_t bar_stat = bar_tempty + 16;           // stationary operand landed
+  const uint32_t bar_stat_free = bar_stat + 8;         // stationary operand no longer in use
+  const uint32_t bar_xa = bar_stat_free + 8;           // 2: mode-specific hand-off, "data written"
+  const uint32_t bar_xb = bar_xa + 16;                 // 2: mode-specific hand-off, "data consumed"
   uint8_t* const gen_base = smem_raw + (base - smem_u32(smem_raw));
-  const uint16_t* hist_s = reinterpret_cast<const uint16_t*>(gen_base + (sm.hist - base));
-  float* lse_s = reinterpret_cast<float*>(gen_base + (sm.lse - base));
-  uint8_t* xwg_s = gen_base + (sm.xwg - base);
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_base + (sm.tmem_slot - base));
+  const uint16_t* hist_s = reinterpret_cast<const uint16_t*>(gen_base + (sm_hist - base));
+  uint8_t* const xch_s = gen_base + (sm_xch - base);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_base + (sm_tmem_slot - base));
+
+  const int nmb = (MODE == kLse) ? (a.GW + 127) / 128 : 1;   // query row blocks of 128
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
     for (int s = 0; s < 2; ++s) { mbar_init(bar_tfull + 8 * s, 1); mbar_init(bar_tempty + 8 * s, kEpilogueThreads); }
     mbar_init(bar_stat, 1);
+    mbar_init(bar_stat_free, kEpilogueThreads);
+    if (MODE == kLse) {
+      mbar_init(bar_xa, kEpilogueThreads - nmb * 128);   // column groups 1.. wrote their (max, sum)
+      mbar_init(bar_xb, nmb * 128);                      // column group 0 merged them
+    } else {
+      for (int s = 0; s < 2; ++s) { mbar_init(bar_xa + 8 * s, kEpilogueThreads - 128); mbar_init(bar_xb + 8 * s, 128); }
+    }
     fence_mbar_init();
   }
-  if (warp == 1) { tmem_alloc(sm.tmem_slot, kTmemCols); tmem_relinquish(); }
+  if (warp == 1) { tmem_alloc(sm_tmem_slot, kTmemCols); tmem_relinquish(); }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  const int nmb = (MODE == kLse) ? (a.GW + 127) / 128 : 1;   // query row blocks of 128
-
   if (warp == 0) {
     // ================= TMA producer =================
-    if (lane == 0) {
+    if (lane == 0 && x_begin < x_end) {
       bool ok = true;
       tma_prefetch_desc(&map_keys);
       tma_prefetch_desc(&map_stat);
-      // stationary operand (+ histogram slice)
-      const uint32_t stat_bytes = 2u * a.stat_rows * 128u;
-      mbar_expect_tx(bar_stat, stat_bytes + hist_bytes);
-      if (MODE == kProj) {
-        const int row0 = chunk * a.stat_rows;
-        tma_load_2d(sm.stat, &map_stat, bar_stat, 0, row0);
-        tma_load_2d(sm.stat + stat_atom_bytes, &map_stat, bar_stat, kAtomCols, row0);
-        const uint16_t* hsrc = a.hist + ((size_t)(b * a.H_kv + h) * a.lsh_tables +
-                                         (size_t)chunk * TC) * ((size_t)1 << KBITS);
-        bulk_load(sm.hist, hsrc, hist_bytes, bar_stat);
-      } else {
-        tma_load_4d(sm.stat, &map_stat, bar_stat, 0, 0, h * a.G, b);
-        tma_load_4d(sm.stat + stat_atom_bytes, &map_stat, bar_stat, kAtomCols, 0, h * a.G, b);
-      }
-      int issued = 0;
-      for (int i = 0; i < ntiles && ok; ++i) {
-        const int s = i % kStages;
-        const int round = i / kStages;
-        if (round > 0) ok = mbar_wait(bar_empty + 8 * s, (round - 1) & 1);
+      TileCursor c = cursor_at(x_begin, a);
+      int gid_cur = -1, gen = 0;
+      long long it = 0;
+      for (long long x = x_begin; x < x_end; ++x, ++it, cursor_advance(c, a)) {
+        const int bh = c.seg / a.nb;
+        const int t = c.seg - bh * a.nb;
+        const int h = bh % a.H_kv, b = bh / a.H_kv;
+        const int gid = cursor_group(c, a);
+        if (gid != gid_cur) {
+          // stationary operand (+ histogram slice) of the new head / chunk
+          if (gen > 0) ok = mbar_wait(bar_stat_free, (uint32_t)(gen - 1) & 1);
+          if (!ok) break;
+          const uint32_t stat_bytes = 2u * a.stat_rows * 128u;
+          mbar_expect_tx(bar_stat, stat_bytes + hist_bytes);
+          if (MODE == kProj) {
+            const int row0 = c.chunk * a.stat_rows;
+            tma_load_2d(sm_stat, &map_stat, bar_stat, 0, row0);
+            tma_load_2d(sm_stat + stat_atom_bytes, &map_stat, bar_stat, kAtomCols, row0);
+            const uint16_t* hsrc = a.hist + ((size_t)bh * a.lsh_tables + (size_t)c.chunk * TC) * ((size_t)1 << KBITS);
+            bulk_load(sm_hist, hsrc, hist_bytes, bar_stat);
+          } else {
+            tma_load_4d(sm_stat, &map_stat, bar_stat, 0, 0, h * a.G, b);
+            tma_load_4d(sm_stat + stat_atom_bytes, &map_stat, bar_stat, kAtomCols, 0, h * a.G, b);
+          }
+          gid_cur = gid;
+          ++gen;
+        }
+        const int s = (int)(it % kStages);
+        if (it >= kStages) ok = mbar_wait(bar_empty + 8 * s, (uint32_t)((it / kStages) - 1) & 1);
         if (!ok) break;
-        const uint32_t dst = sm.stages + s * kTileBytes;
-        const int token = t * a.S + (tile0 + i) * kTileKeys;
+        const uint32_t dst = sm_stages + s * kTileBytes;
+        const int token = t * a.S + c.tib * kTileKeys;
         mbar_expect_tx(bar_full + 8 * s, kTileBytes);
         tma_load_4d(dst, &map_keys, bar_full + 8 * s, 0, token, h, b);
         tma_load_4d(dst + kTileAtomBytes, &map_keys, bar_full + 8 * s, kAtomCols, token, h, b);
-        issued = i + 1;
       }
       if (!ok) {
         record_status(a.status, kStatusTimeout);
         // let copies already in flight land before the CTA may exit
-        for (int i = max(0, issued - kStages); i < issued; ++i)
-          mbar_wait(bar_full + 8 * (i % kStages), (i / kStages) & 1);
+        for (long long i = (it > kStages ? it - kStages : 0); i < it; ++i)
+          mbar_wait(bar_full + 8 * (int)(i % kStages), (uint32_t)(i / kStages) & 1);
+        if (gen > 0) mbar_wait(bar_stat, (uint32_t)(gen - 1) & 1);
       }
     }
     __syncwarp();
   } else if (warp == 1) {
     // ================= MMA issuer =================
-    if (lane == 0) {
-      bool ok = mbar_wait(bar_stat, 0);
+    if (lane == 0 && x_begin < x_end) {
+      bool ok = true;
       const uint32_t idesc = (MODE == kLse) ? umma_idesc_bf16(128, kTileKeys)
                                             : umma_idesc_bf16(128, a.stat_rows);
-      for (int i = 0; i < ntiles && ok; ++i) {
-        const int s = i % kStages;
-        const int acc = i & 1;
-        if (i >= 2) ok = mbar_wait(bar_tempty + 8 * acc, ((i >> 1) - 1) & 1);
-        if (ok) ok = mbar_wait(bar_full + 8 * s, (i / kStages) & 1);
+      TileCursor c = cursor_at(x_begin, a);
+      int gid_cur = -1, gen = 0;
+      long long it = 0;
+      for (long long x = x_begin; x < x_end; ++x, ++it, cursor_advance(c, a)) {
+        const int gid = cursor_group(c, a);
+        if (gid != gid_cur) {
+          ok = mbar_wait(bar_stat, (uint32_t)gen & 1);
+          if (!ok) break;
+          gid_cur = gid;
+          ++gen;
+        }
+        const int s = (int)(it % kStages);
+        const int acc = (int)(it & 1);
+        if (it >= 2) ok = mbar_wait(bar_tempty + 8 * acc, (uint32_t)((it >> 1) - 1) & 1);
+        if (ok) ok = mbar_wait(bar_full + 8 * s, (uint32_t)(it / kStages) & 1);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t tile = sm.stages + s * kTileBytes;
+        const uint32_t tile = sm_stages + s * kTileBytes;
         for (int mb = 0; mb < nmb; ++mb) {
           const uint32_t d = tmem_base + acc * kAccStride + mb * 128;
 #pragma unroll
           for (int k = 0; k < 8; ++k) {
             const uint32_t koff = (k & 3) * 32;
             const uint32_t tile_k = tile + (k >> 2) * kTileAtomBytes + koff;
-            const uint32_t stat_k = sm.stat + (k >> 2) * stat_atom_bytes + koff;
+            const uint32_t stat_k = sm_stat + (k >> 2) * stat_atom_bytes + koff;
             if (MODE == kLse) {
               umma_bf16(d, umma_sdesc_sw128(stat_k + mb * (128 * 128)), umma_sdesc_sw128(tile_k),
                         idesc, k > 0);
@@ -334,148 +403,190 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
       if (!ok) record_status(a.status, kStatusTimeout);
     }
     __syncwarp();
-  } else {
-    // ================= epilogue warps: two groups of four =================
-    // Both groups cover all 128 TMEM lanes (lane quarter = warp_id % 4); they split the
+  } else if (x_begin < x_end) {
+    // ================= epilogue warps: four groups of four =================
+    // Every group covers all 128 TMEM lanes (lane quarter = warp_id % 4); the groups split the
     // accumulator columns of every tile between them.
     const int quarter = warp & 3;
     const int row = quarter * 32 + lane;                   // TMEM lane owned by this thread
     const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
-    const int etid = threadIdx.x - 64;                     // 0..255
-    const int wg = etid >> 7;                              // epilogue group 0 / 1
+    const int ewarp = warp - 2;                            // 0..15
+    const int wg = ewarp >> 2;                             // epilogue group 0..3
+    const float c2 = a.scale_log2e;
     bool ok = true;
+    TileCursor c = cursor_at(x_begin, a);
+    long long it = 0;
 
     if constexpr (MODE == kLse) {
-      // group g owns query block g (G*W > 128) or half of the key columns (G*W <= 128)
-      const int mb = (nmb == 2) ? wg : 0;
-      const int c_begin = (nmb == 2) ? 0 : wg * 64;
-      const int c_end = (nmb == 2) ? kTileKeys : wg * 64 + 64;
+      // group -> (query row block, key column range)
+      const int ncg = kEpiGroups / nmb;                    // column groups: 4 (G*W <= 128) or 2
+      const int mb = wg % nmb, cg = wg / nmb;
+      const int cw = kTileKeys / ncg;                      // 32 or 64 key columns per thread
+      const int c0 = cg * cw;
+      const int q = mb * 128 + row;                        // this thread's query
+      float2* xch = reinterpret_cast<float2*>(xch_s);      // [ncg - 1][nmb * 128]
       float m = -INFINITY, l = 0.f;
-      const float c2 = a.scale_log2e;
-      for (int i = 0; i < ntiles && ok; ++i) {
-        const int acc = i & 1;
-        ok = mbar_wait(bar_tfull + 8 * acc, (i >> 1) & 1);
+      int flushes = 0;
+      for (long long x = x_begin; x < x_end; ++x, ++it) {
+        const int acc = (int)(it & 1);
+        ok = mbar_wait(bar_tfull + 8 * acc, (uint32_t)(it >> 1) & 1);
         if (!ok) break;
         tc_fence_after();
-        const int nvalid = min(kTileKeys, a.S - (tile0 + i) * kTileKeys);
-        const int ce = min(c_end, (nvalid + 15) & ~15);
-        walk_columns(t_lane + acc * kAccStride + mb * 128, c_begin, ce, [&](const uint32_t* v, int col0, auto cnt_tag) {
-          constexpr int CNT = decltype(cnt_tag)::value;
-          const int lim = nvalid - col0;                   // valid columns in this chunk (>= 1)
-          float cmax = -INFINITY;
-          if (lim >= CNT) {
-#pragma unroll
-            for (int k = 0; k < CNT; ++k) cmax = fmaxf(cmax, __uint_as_float(v[k]));
-            const float m_new = fmaxf(m, cmax * c2);
-            float add0 = 0.f, add1 = 0.f;
-#pragma unroll
-            for (int k = 0; k < CNT; ++k) {
-              const float x = fmaf(__uint_as_float(v[k]), c2, -m_new);
-              const float e = ((k * 5) % 16 < 5) ? ex2_poly(x) : ex2_approx(x);
-              if (k & 1) add1 += e; else add0 += e;
-            }
-            l = l * ex2_approx(m - m_new) + (add0 + add1);
-            m = m_new;
-          } else {
-#pragma unroll
-            for (int k = 0; k < CNT; ++k) if (k < lim) cmax = fmaxf(cmax, __uint_as_float(v[k]));
-            const float m_new = fmaxf(m, cmax * c2);
-            float add = 0.f;
-#pragma unroll
-            for (int k = 0; k < CNT; ++k)
-              if (k < lim) add += ex2_approx(fmaf(__uint_as_float(v[k]), c2, -m_new));
-            l = l * ex2_approx(m - m_new) + add;
-            m = m_new;
-          }
-        });
+        uint32_t v[kEpiCols];
+        load_epi_cols(t_lane + acc * kAccStride + mb * 128 + c0, cw, v);
         tc_fence_before();
         mbar_arrive(bar_tempty + 8 * acc);
-      }
-      if (nmb == 2) {
-        const int q = mb * 128 + row;
-        if (ok && q < a.GW) a.lse_part[((size_t)seg * a.n_split + split) * a.GW + q] = make_float2(m, l);
-      } else {
-        float2* xch = reinterpret_cast<float2*>(xwg_s);
-        if (wg == 1) xch[row] = make_float2(m, l);
-        asm volatile("bar.sync 1, 256;" ::: "memory");
-        if (wg == 0 && ok && row < a.GW) {
-          const float2 o = xch[row];
-          const float mx = fmaxf(m, o.x);
-          const float lt = (mx == -INFINITY) ? 0.f : l * ex2_approx(m - mx) + o.y * ex2_approx(o.x - mx);
-          a.lse_part[((size_t)seg * a.n_split + split) * a.GW + row] = make_float2(mx, lt);
+        const int nvalid = a.S - c.tib * kTileKeys;          // >= 1; columns at or beyond it hold no key
+        if (nvalid < c0 + cw) {
+#pragma unroll
+          for (int k = 0; k < kEpiCols; ++k) if (c0 + k >= nvalid) v[k] = 0xff800000u;
         }
+        float cmax = -INFINITY;
+#pragma unroll
+        for (int k = 0; k < kEpiCols; k += 2) cmax = max3(__uint_as_float(v[k]), __uint_as_float(v[k + 1]), cmax);
+        const float m_new = fmaxf(m, cmax * c2);
+        const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
+        const float add = (cw == 64) ? sum_exp2<64, false>(v, c2, nullptr, -m_use)
+                                     : sum_exp2<32, false>(v, c2, nullptr, -m_use);
+        l = l * ex2_approx(m - m_use) + add;
+        m = m_new;
+        // end of this segment's run of tiles inside the slice: merge the column groups, write
+        // one partial, start over
+        TileCursor nx = c;
+        cursor_advance(nx, a);
+        const bool last = (x + 1 == x_end);
+        if (last || nx.seg != c.seg) {
+          if (cg > 0) {
+            if (flushes > 0) ok = mbar_wait(bar_xb, (uint32_t)(flushes - 1) & 1);
+            if (!ok) break;
+            xch[(cg - 1) * (nmb * 128) + q] = make_float2(m, l);
+            mbar_arrive(bar_xa);
+          } else {
+            ok = mbar_wait(bar_xa, (uint32_t)flushes & 1);
+            if (!ok) break;
+            float mx = m;
+            for (int g2 = 1; g2 < ncg; ++g2) mx = fmaxf(mx, xch[(g2 - 1) * (nmb * 128) + q].x);
+            float lt = (mx == -INFINITY) ? 0.f : l * ex2_approx(m - mx);
+            for (int g2 = 1; g2 < ncg; ++g2) {
+              const float2 o = xch[(g2 - 1) * (nmb * 128) + q];
+              if (o.x != -INFINITY) lt += o.y * ex2_approx(o.x - mx);
+            }
+            mbar_arrive(bar_xb);
+            if (q < a.GW) {
+              const int slot = (int)blockIdx.x - cta_of_tile((long long)c.seg * a.tiles_in_block, a.n_tiles, gridDim.x);
+              a.lse_part[((size_t)c.seg * a.n_slot + slot) * a.GW + q] = make_float2(mx, lt);
+            }
+          }
+          ++flushes;
+          m = -INFINITY;
+          l = 0.f;
+        }
+        if (!last && cursor_group(nx, a) != cursor_group(c, a)) mbar_arrive(bar_stat_free);
+        c = nx;
       }
     } else if constexpr (MODE == kScore) {
-      // combine the splits' (max, sum) partials into log2-sum-exp2 per query
-      for (int q = etid; q < a.GW; q += 256) {
-        const float2* p = a.lse_part + (size_t)seg * a.n_split * a.GW + q;
-        float mx = -INFINITY;
-        for (int s2 = 0; s2 < a.n_split; ++s2) mx = fmaxf(mx, p[(size_t)s2 * a.GW].x);
-        float sum = 0.f;
-        for (int s2 = 0; s2 < a.n_split; ++s2) {
-          const float2 e = p[(size_t)s2 * a.GW];
-          sum += e.y * exp2f(e.x - mx);
+      // group g sums the query columns [c0, c1); widths are multiples of 16, at most 64
+      const int cw = ((a.GW + kEpiGroups - 1) / kEpiGroups + 15) & ~15;
+      const int c0 = wg * cw;
+      const int c1 = min(a.GW, c0 + cw);
+      const int ncols = max(0, c1 - c0);
+      float* lw = reinterpret_cast<float*>(xch_s) + ewarp * kEpiCols;        // this warp's -lse values
+      float* part = reinterpret_cast<float*>(xch_s + 16 * kEpiCols * 4);     // [2 acc][3 groups][128 keys]
+      int seg_cur = -1;
+      for (long long x = x_begin; x < x_end; ++x, ++it) {
+        if (c.seg != seg_cur) {
+          // log2-sum-exp2 of this warp's queries from the partials of the CTAs that covered the segment
+          const long long first = (long long)c.seg * a.tiles_in_block;
+          const int cf = cta_of_tile(first, a.n_tiles, a.lse_ctas);
+          const int n_used = cta_of_tile(first + a.tiles_in_block - 1, a.n_tiles, a.lse_ctas) - cf + 1;
+          __syncwarp();
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+            const int qq = c0 + lane + 32 * half;
+            float neg_lse = 0.f;
+            if (qq < c1) {
+              const float2* p = a.lse_part + (size_t)c.seg * a.n_slot * a.GW + qq;
+              float mx = -INFINITY;
+              for (int s2 = 0; s2 < n_used; ++s2) mx = fmaxf(mx, p[(size_t)s2 * a.GW].x);
+              float sum = 0.f;
+              for (int s2 = 0; s2 < n_used; ++s2) {
+                const float2 e = p[(size_t)s2 * a.GW];
+                if (e.x != -INFINITY) sum += e.y * exp2f(e.x - mx);
+              }
+              const float r = mx + log2f(sum);
+              neg_lse = -r;
+              if (c.tib == 0 && quarter == 0) a.lse2[(size_t)c.seg * a.GW + qq] = r;
+            }
+            lw[lane + 32 * half] = neg_lse;
+          }
+          __syncwarp();
+          seg_cur = c.seg;
         }
-        const float r = mx + log2f(sum);
-        lse_s[q] = r;
-        if (split == 0) a.lse2[(size_t)seg * a.GW + q] = r;
-      }
-      asm volatile("bar.sync 1, 256;" ::: "memory");
-      // group 0 sums queries [0, cs), group 1 queries [cs, G*W); both ranges start 32-aligned
-      const int cs = ((a.GW / 32 + 1) / 2) * 32;
-      const int c_begin = wg ? cs : 0;
-      const int c_end = wg ? a.GW : cs;
-      const float c2 = a.scale_log2e;
-      float* part = reinterpret_cast<float*>(xwg_s);       // [2 accumulators][128 keys]
-      for (int i = 0; i < ntiles && ok; ++i) {
-        const int acc = i & 1;
-        ok = mbar_wait(bar_tfull + 8 * acc, (i >> 1) & 1);
+        const int acc = (int)(it & 1);
+        ok = mbar_wait(bar_tfull + 8 * acc, (uint32_t)(it >> 1) & 1);
         if (!ok) break;
         tc_fence_after();
-        float s0 = 0.f, s1 = 0.f;
-        walk_columns(t_lane + acc * kAccStride, c_begin, c_end, [&](const uint32_t* v, int col0, auto cnt_tag) {
-          constexpr int CNT = decltype(cnt_tag)::value;
-#pragma unroll
-          for (int k = 0; k < CNT; k += 4) {
-            const float4 ls = *reinterpret_cast<const float4*>(lse_s + col0 + k);
-            const float lsv[4] = {ls.x, ls.y, ls.z, ls.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const float x = fmaf(__uint_as_float(v[k + e]), c2, -lsv[e]);
-              const float ex = (((k + e) * 5) % 16 < 5) ? ex2_poly(x) : ex2_approx(x);
-              if (e & 1) s1 += ex; else s0 += ex;
-            }
-          }
-        });
+        uint32_t v[kEpiCols];
+        load_epi_cols(t_lane + acc * kAccStride + c0, ncols, v);
         tc_fence_before();
         mbar_arrive(bar_tempty + 8 * acc);
-        const float sum = s0 + s1;
-        if (wg == 1) part[acc * 128 + row] = sum;
-        asm volatile("bar.sync 1, 256;" ::: "memory");
-        if (wg == 0) {
-          const int key = (tile0 + i) * kTileKeys + row;
-          if (key < a.S) a.s_exact[(size_t)seg * a.S + key] = sum + part[acc * 128 + row];
+        float sum = 0.f;
+        if (ncols > 32) sum = sum_exp2<64, true>(v, c2, lw, 0.f);
+        else if (ncols > 0) sum = sum_exp2<32, true>(v, c2, lw, 0.f);
+        // groups 1..3 hand their sums to group 0, which adds them in a fixed order
+        if (wg > 0) {
+          if (it >= 2) ok = mbar_wait(bar_xb + 8 * acc, (uint32_t)((it >> 1) - 1) & 1);
+          if (!ok) break;
+          part[(acc * 3 + (wg - 1)) * 128 + row] = sum;
+          mbar_arrive(bar_xa + 8 * acc);
+        } else {
+          ok = mbar_wait(bar_xa + 8 * acc, (uint32_t)(it >> 1) & 1);
+          if (!ok) break;
+          const float tot = ((sum + part[(acc * 3 + 0) * 128 + row]) + part[(acc * 3 + 1) * 128 + row]) +
+                            part[(acc * 3 + 2) * 128 + row];
+          mbar_arrive(bar_xb + 8 * acc);
+          const int key = c.tib * kTileKeys + row;
+          if (key < a.S) a.s_exact[(size_t)c.seg * a.S + key] = tot;
         }
+        TileCursor nx = c;
+        cursor_advance(nx, a);
+        if (x + 1 < x_end && cursor_group(nx, a) != cursor_group(c, a)) mbar_arrive(bar_stat_free);
+        c = nx;
       }
     } else {
       // ---- kProj: sign bits -> bucket codes -> histogram lookups ----
       // Bucket code of a table: bit b of the table (hyperplane r*K + b) sits at position
       // K-1-b, i.e. the first hyperplane is the most significant bit; bit = [projection >= 0].
-      // Group 0 handles the chunk's first TC/2 tables, group 1 the rest.
-      ok = mbar_wait(bar_stat, 0);   // histogram slice landed (async-proxy writes visible after the wait)
-      for (int i = 0; i < ntiles && ok; ++i) {
-        const int acc = i & 1;
-        ok = mbar_wait(bar_tfull + 8 * acc, (i >> 1) & 1);
+      // Group g handles tables [g*TC/4, (g+1)*TC/4) of the chunk.
+      constexpr int TQ = TC / kEpiGroups;
+      int gid_cur = -1, gen = 0;
+      for (long long x = x_begin; x < x_end; ++x, ++it) {
+        const int gid = cursor_group(c, a);
+        if (gid != gid_cur) {
+          ok = mbar_wait(bar_stat, (uint32_t)gen & 1);   // histogram slice landed (async-proxy writes visible after the wait)
+          if (!ok) break;
+          gid_cur = gid;
+          ++gen;
+        }
+        const int acc = (int)(it & 1);
+        ok = mbar_wait(bar_tfull + 8 * acc, (uint32_t)(it >> 1) & 1);
         if (!ok) break;
         tc_fence_after();
-        const int key = (tile0 + i) * kTileKeys + row;
+        const int key = c.tib * kTileKeys + row;
         const bool valid = key < a.S;
         const uint32_t t_acc = t_lane + acc * kAccStride;
         const uint32_t bar_rel = bar_tempty + 8 * acc;
+        const int table0 = c.chunk * TC;
         uint32_t partial;
-        if (wg == 0) partial = proj_tables<KBITS, 0, TC / 2>(t_acc, bar_rel, hist_s, a, seg, key, chunk * TC, valid);
-        else partial = proj_tables<KBITS, TC / 2, TC>(t_acc, bar_rel, hist_s, a, seg, key, chunk * TC, valid);
-        if (valid) atomicAdd(a.counts + (size_t)seg * a.S + key, partial);
+        if (wg == 0) partial = proj_tables<KBITS, 0, TQ>(t_acc, bar_rel, hist_s, a, c.seg, key, table0, valid);
+        else if (wg == 1) partial = proj_tables<KBITS, TQ, 2 * TQ>(t_acc, bar_rel, hist_s, a, c.seg, key, table0, valid);
+        else if (wg == 2) partial = proj_tables<KBITS, 2 * TQ, 3 * TQ>(t_acc, bar_rel, hist_s, a, c.seg, key, table0, valid);
+        else partial = proj_tables<KBITS, 3 * TQ, 4 * TQ>(t_acc, bar_rel, hist_s, a, c.seg, key, table0, valid);
+        if (valid) atomicAdd(a.counts + (size_t)c.seg * a.S + key, partial);
+        TileCursor nx = c;
+        cursor_advance(nx, a);
+        if (x + 1 < x_end && cursor_group(nx, a) != gid) mbar_arrive(bar_stat_free);
+        c = nx;
       }
     }
     if (!ok) record_status(a.status, kStatusTimeout);
