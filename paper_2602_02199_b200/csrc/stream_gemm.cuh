@@ -87,9 +87,10 @@ __host__ __device__ inline int cta_of_tile(long long x, long long T, int G) {
   return (int)(((x + 1) * G - 1) / T);
 }
 
-// Position in the tile sequence.
+// Position in the tile sequence: hyperplane chunk, (sequence, KV head) pair, block, tile in block.
 struct TileCursor {
-  int chunk, seg, tib;
+  int chunk, bh, t, tib;
+  int seg;             // bh * nb + t
 };
 __device__ __forceinline__ TileCursor cursor_at(long long x, const StreamArgs& a) {
   const long long per_chunk = (long long)a.nseg * a.tiles_in_block;
@@ -98,17 +99,26 @@ __device__ __forceinline__ TileCursor cursor_at(long long x, const StreamArgs& a
   const long long r = x - (long long)c.chunk * per_chunk;
   c.seg = (int)(r / a.tiles_in_block);
   c.tib = (int)(r - (long long)c.seg * a.tiles_in_block);
+  c.bh = c.seg / a.nb;
+  c.t = c.seg - c.bh * a.nb;
   return c;
 }
 __device__ __forceinline__ void cursor_advance(TileCursor& c, const StreamArgs& a) {
   if (++c.tib == a.tiles_in_block) {
     c.tib = 0;
-    if (++c.seg == a.nseg) { c.seg = 0; ++c.chunk; }
+    ++c.seg;
+    if (++c.t == a.nb) {
+      c.t = 0;
+      if (++c.bh == a.batch * a.H_kv) { c.bh = 0; c.seg = 0; ++c.chunk; }
+    }
   }
 }
-// Tiles with the same group id share the stationary operand.
-__device__ __forceinline__ int cursor_group(const TileCursor& c, const StreamArgs& a) {
-  return c.chunk * (a.batch * a.H_kv) + c.seg / a.nb;
+// The tile after c belongs to another segment / needs another stationary operand.
+__device__ __forceinline__ bool cursor_last_of_segment(const TileCursor& c, const StreamArgs& a) {
+  return c.tib == a.tiles_in_block - 1;
+}
+__device__ __forceinline__ bool cursor_last_of_group(const TileCursor& c, const StreamArgs& a) {
+  return c.tib == a.tiles_in_block - 1 && c.t == a.nb - 1;
 }
 
 // Loads the 32-bit columns [CB, CE) of the calling thread's TMEM lane into r[0 .. CE-CB) as a
@@ -126,20 +136,13 @@ __device__ __forceinline__ void tmem_ld_range(uint32_t taddr, uint32_t* r) {
   }
 }
 
-// Reads `ncols` (a multiple of 16, at most 64) columns starting at taddr into v[0..64); the rest
-// of v is set to -infinity, which every consumer turns into a zero contribution.
-__device__ __forceinline__ void load_epi_cols(uint32_t taddr, int ncols, uint32_t* v) {
+// Reads NC (a multiple of 16) columns starting at taddr into v.
+template <int NC>
+__device__ __forceinline__ void load_epi_cols(uint32_t taddr, uint32_t* v) {
 #pragma unroll
-  for (int j = 0; j < kEpiCols / 16; ++j) {
-    if (16 * j < ncols) {
-      tmem_ld_x16(taddr + 16 * j, v + 16 * j);
-    } else {
-#pragma unroll
-      for (int k = 0; k < 16; ++k) v[16 * j + k] = 0xff800000u;
-    }
-  }
+  for (int j = 0; j < NC / 16; ++j) tmem_ld_x16(taddr + 16 * j, v + 16 * j);
   tmem_wait_ld();
-  reg_fence<kEpiCols>(v);
+  reg_fence<NC>(v);
 }
 
 // sum over k < N of 2^(v[k] * c2 + addend[k]); addend is per column (kScore: -lse of the query,
@@ -238,6 +241,198 @@ __device__ __forceinline__ uint32_t proj_tables(uint32_t t_acc, uint32_t bar_rel
   return partial;
 }
 
+// What an epilogue thread knows about its place in the CTA.
+struct EpiCtx {
+  int quarter, lane, row;      // TMEM lane quarter of the warp, lane in the warp, TMEM lane of the thread
+  int ewarp, wg;               // epilogue warp 0..15, epilogue group 0..3
+  uint32_t t_lane;             // TMEM address of the thread's lane, column 0
+  long long x_begin, x_end;    // the CTA's slice of the tile sequence
+  uint32_t bar_tfull, bar_tempty, bar_stat, bar_stat_free, bar_xa, bar_xb;
+  uint8_t* xch_s;              // exchange area
+  const uint16_t* hist_s;      // histogram slice (kProj)
+};
+
+// kLse: CW key columns per thread (64 when G*W > 128: two query row blocks x two column groups;
+// 32 otherwise: one row block x four column groups).
+template <int CW>
+__device__ __forceinline__ bool lse_epilogue(const StreamArgs& a, const EpiCtx& e, int nmb) {
+  constexpr int ncg = kTileKeys / CW;                  // column groups
+  const int mb = e.wg % nmb, cg = e.wg / nmb;
+  const int c0 = cg * CW;
+  const int q = mb * 128 + e.row;                      // this thread's query
+  const int nq = nmb * 128;
+  float2* xch = reinterpret_cast<float2*>(e.xch_s);    // [ncg - 1][nq]
+  const float c2 = a.scale_log2e;
+  const uint32_t t_col = e.t_lane + mb * 128 + c0;
+  float m = -INFINITY, l = 0.f;
+  int flushes = 0;
+  TileCursor c = cursor_at(e.x_begin, a);
+  long long it = 0;
+  for (long long x = e.x_begin; x < e.x_end; ++x, ++it) {
+    const int acc = (int)(it & 1);
+    if (!mbar_wait(e.bar_tfull + 8 * acc, (uint32_t)(it >> 1) & 1)) return false;
+    tc_fence_after();
+    uint32_t v[CW];
+    load_epi_cols<CW>(t_col + acc * kAccStride, v);
+    tc_fence_before();
+    mbar_arrive(e.bar_tempty + 8 * acc);
+    const int nvalid = a.S - c.tib * kTileKeys;        // >= 1; columns at or beyond it hold no key
+    if (nvalid < c0 + CW) {
+      asm volatile("" ::: "memory");                   // keeps this rare path a real branch
+#pragma unroll
+      for (int k = 0; k < CW; ++k) if (c0 + k >= nvalid) v[k] = 0xff800000u;
+    }
+    float cmax = -INFINITY;
+#pragma unroll
+    for (int k = 0; k < CW; k += 2) cmax = max3(__uint_as_float(v[k]), __uint_as_float(v[k + 1]), cmax);
+    const float m_new = fmaxf(m, cmax * c2);
+    const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
+    const float add = sum_exp2<CW, false>(v, c2, nullptr, -m_use);
+    l = l * ex2_approx(m - m_use) + add;
+    m = m_new;
+    const bool last = (x + 1 == e.x_end);
+    if (last || cursor_last_of_segment(c, a)) {
+      // end of this segment's run of tiles inside the slice: merge the column groups, write one
+      // partial, start over
+      if (cg > 0) {
+        if (flushes > 0 && !mbar_wait(e.bar_xb, (uint32_t)(flushes - 1) & 1)) return false;
+        xch[(cg - 1) * nq + q] = make_float2(m, l);
+        mbar_arrive(e.bar_xa);
+      } else {
+        if (!mbar_wait(e.bar_xa, (uint32_t)flushes & 1)) return false;
+        float mx = m;
+#pragma unroll
+        for (int g2 = 1; g2 < ncg; ++g2) mx = fmaxf(mx, xch[(g2 - 1) * nq + q].x);
+        float lt = (mx == -INFINITY) ? 0.f : l * ex2_approx(m - mx);
+#pragma unroll
+        for (int g2 = 1; g2 < ncg; ++g2) {
+          const float2 o = xch[(g2 - 1) * nq + q];
+          if (o.x != -INFINITY) lt += o.y * ex2_approx(o.x - mx);
+        }
+        mbar_arrive(e.bar_xb);
+        if (q < a.GW) {
+          const int slot = (int)blockIdx.x - cta_of_tile((long long)c.seg * a.tiles_in_block, a.n_tiles, gridDim.x);
+          a.lse_part[((size_t)c.seg * a.n_slot + slot) * a.GW + q] = make_float2(mx, lt);
+        }
+      }
+      ++flushes;
+      m = -INFINITY;
+      l = 0.f;
+    }
+    if (!last && cursor_last_of_group(c, a)) mbar_arrive(e.bar_stat_free);
+    cursor_advance(c, a);
+  }
+  return true;
+}
+
+// kScore: NC query columns [c0, c0 + NC) per thread; the groups' sums meet in group 0.
+template <int NC>
+__device__ __forceinline__ bool score_epilogue(const StreamArgs& a, const EpiCtx& e, int c0) {
+  float* lw = reinterpret_cast<float*>(e.xch_s) + e.ewarp * kEpiCols;       // this warp's -lse values
+  float* part = reinterpret_cast<float*>(e.xch_s + 16 * kEpiCols * 4);      // [2 acc][3 groups][128 keys]
+  const float c2 = a.scale_log2e;
+  bool new_seg = true;
+  TileCursor c = cursor_at(e.x_begin, a);
+  long long it = 0;
+  for (long long x = e.x_begin; x < e.x_end; ++x, ++it) {
+    if (new_seg && NC > 0) {
+      // log2-sum-exp2 of this warp's queries from the partials of the CTAs that covered the segment
+      const long long first = (long long)c.seg * a.tiles_in_block;
+      const int cf = cta_of_tile(first, a.n_tiles, a.lse_ctas);
+      const int n_used = cta_of_tile(first + a.tiles_in_block - 1, a.n_tiles, a.lse_ctas) - cf + 1;
+      __syncwarp();
+#pragma unroll
+      for (int half = 0; half < (NC + 31) / 32; ++half) {
+        const int j = e.lane + 32 * half;
+        if (j < NC) {
+          const int qq = c0 + j;
+          const float2* p = a.lse_part + (size_t)c.seg * a.n_slot * a.GW + qq;
+          float mx = -INFINITY;
+          for (int s2 = 0; s2 < n_used; ++s2) mx = fmaxf(mx, p[(size_t)s2 * a.GW].x);
+          float sum = 0.f;
+          for (int s2 = 0; s2 < n_used; ++s2) {
+            const float2 pe = p[(size_t)s2 * a.GW];
+            if (pe.x != -INFINITY) sum += pe.y * exp2f(pe.x - mx);
+          }
+          const float r = mx + log2f(sum);
+          if (c.tib == 0 && e.quarter == 0) a.lse2[(size_t)c.seg * a.GW + qq] = r;
+          lw[j] = -r;
+        }
+      }
+      __syncwarp();
+    }
+    const int acc = (int)(it & 1);
+    if (!mbar_wait(e.bar_tfull + 8 * acc, (uint32_t)(it >> 1) & 1)) return false;
+    tc_fence_after();
+    float sum = 0.f;
+    if constexpr (NC > 0) {
+      uint32_t v[NC];
+      load_epi_cols<NC>(e.t_lane + acc * kAccStride + c0, v);
+      tc_fence_before();
+      mbar_arrive(e.bar_tempty + 8 * acc);
+      sum = sum_exp2<NC, true>(v, c2, lw, 0.f);
+    } else {
+      tc_fence_before();
+      mbar_arrive(e.bar_tempty + 8 * acc);
+    }
+    // groups 1..3 hand their sums to group 0, which adds them in a fixed order
+    if (e.wg > 0) {
+      if (it >= 2 && !mbar_wait(e.bar_xb + 8 * acc, (uint32_t)((it >> 1) - 1) & 1)) return false;
+      part[(acc * 3 + (e.wg - 1)) * 128 + e.row] = sum;
+      mbar_arrive(e.bar_xa + 8 * acc);
+    } else {
+      if (!mbar_wait(e.bar_xa + 8 * acc, (uint32_t)(it >> 1) & 1)) return false;
+      const float tot = ((sum + part[(acc * 3 + 0) * 128 + e.row]) + part[(acc * 3 + 1) * 128 + e.row]) +
+                        part[(acc * 3 + 2) * 128 + e.row];
+      mbar_arrive(e.bar_xb + 8 * acc);
+      const int key = c.tib * kTileKeys + e.row;
+      if (key < a.S) a.s_exact[(size_t)c.seg * a.S + key] = tot;
+    }
+    new_seg = cursor_last_of_segment(c, a);
+    if (x + 1 < e.x_end && cursor_last_of_group(c, a)) mbar_arrive(e.bar_stat_free);
+    cursor_advance(c, a);
+  }
+  return true;
+}
+
+// kProj: sign bits -> bucket codes -> histogram lookups.
+// Bucket code of a table: bit b of the table (hyperplane r*K + b) sits at position K-1-b, i.e.
+// the first hyperplane is the most significant bit; bit = [projection >= 0].
+// Group g handles tables [g*TC/4, (g+1)*TC/4) of the chunk.
+template <int KBITS, int TC>
+__device__ __forceinline__ bool proj_epilogue(const StreamArgs& a, const EpiCtx& e) {
+  constexpr int TQ = TC / kEpiGroups;
+  bool new_group = true;
+  int gen = 0;
+  TileCursor c = cursor_at(e.x_begin, a);
+  long long it = 0;
+  for (long long x = e.x_begin; x < e.x_end; ++x, ++it) {
+    if (new_group) {
+      // histogram slice landed (async-proxy writes are visible after the wait)
+      if (!mbar_wait(e.bar_stat, (uint32_t)gen & 1)) return false;
+      ++gen;
+    }
+    const int acc = (int)(it & 1);
+    if (!mbar_wait(e.bar_tfull + 8 * acc, (uint32_t)(it >> 1) & 1)) return false;
+    tc_fence_after();
+    const int key = c.tib * kTileKeys + e.row;
+    const bool valid = key < a.S;
+    const uint32_t t_acc = e.t_lane + acc * kAccStride;
+    const uint32_t bar_rel = e.bar_tempty + 8 * acc;
+    const int table0 = c.chunk * TC;
+    uint32_t partial;
+    if (e.wg == 0) partial = proj_tables<KBITS, 0, TQ>(t_acc, bar_rel, e.hist_s, a, c.seg, key, table0, valid);
+    else if (e.wg == 1) partial = proj_tables<KBITS, TQ, 2 * TQ>(t_acc, bar_rel, e.hist_s, a, c.seg, key, table0, valid);
+    else if (e.wg == 2) partial = proj_tables<KBITS, 2 * TQ, 3 * TQ>(t_acc, bar_rel, e.hist_s, a, c.seg, key, table0, valid);
+    else partial = proj_tables<KBITS, 3 * TQ, 4 * TQ>(t_acc, bar_rel, e.hist_s, a, c.seg, key, table0, valid);
+    if (valid) atomicAdd(a.counts + (size_t)c.seg * a.S + key, partial);
+    new_group = cursor_last_of_group(c, a);
+    if (new_group && x + 1 < e.x_end) mbar_arrive(e.bar_stat_free);
+    cursor_advance(c, a);
+  }
+  return true;
+}
+
 // Shared memory carve-up, identical on host (sizes) and device (addresses).
 __host__ __device__ inline uint32_t stream_smem_bytes(int mode, int stat_rows_alloc, int hist_bytes) {
   uint32_t b = 2u * stat_rows_alloc * 128u + kStages * kTileBytes;
@@ -314,40 +509,40 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
       tma_prefetch_desc(&map_keys);
       tma_prefetch_desc(&map_stat);
       TileCursor c = cursor_at(x_begin, a);
-      int gid_cur = -1, gen = 0;
+      bool new_group = true;
+      int gen = 0, h = 0, b = 0;
       long long it = 0;
-      for (long long x = x_begin; x < x_end; ++x, ++it, cursor_advance(c, a)) {
-        const int bh = c.seg / a.nb;
-        const int t = c.seg - bh * a.nb;
-        const int h = bh % a.H_kv, b = bh / a.H_kv;
-        const int gid = cursor_group(c, a);
-        if (gid != gid_cur) {
+      for (long long x = x_begin; x < x_end; ++x, ++it) {
+        if (new_group) {
           // stationary operand (+ histogram slice) of the new head / chunk
           if (gen > 0) ok = mbar_wait(bar_stat_free, (uint32_t)(gen - 1) & 1);
           if (!ok) break;
+          b = c.bh / a.H_kv;
+          h = c.bh - b * a.H_kv;
           const uint32_t stat_bytes = 2u * a.stat_rows * 128u;
           mbar_expect_tx(bar_stat, stat_bytes + hist_bytes);
           if (MODE == kProj) {
             const int row0 = c.chunk * a.stat_rows;
             tma_load_2d(sm_stat, &map_stat, bar_stat, 0, row0);
             tma_load_2d(sm_stat + stat_atom_bytes, &map_stat, bar_stat, kAtomCols, row0);
-            const uint16_t* hsrc = a.hist + ((size_t)bh * a.lsh_tables + (size_t)c.chunk * TC) * ((size_t)1 << KBITS);
+            const uint16_t* hsrc = a.hist + ((size_t)c.bh * a.lsh_tables + (size_t)c.chunk * TC) * ((size_t)1 << KBITS);
             bulk_load(sm_hist, hsrc, hist_bytes, bar_stat);
           } else {
             tma_load_4d(sm_stat, &map_stat, bar_stat, 0, 0, h * a.G, b);
             tma_load_4d(sm_stat + stat_atom_bytes, &map_stat, bar_stat, kAtomCols, 0, h * a.G, b);
           }
-          gid_cur = gid;
           ++gen;
         }
         const int s = (int)(it % kStages);
         if (it >= kStages) ok = mbar_wait(bar_empty + 8 * s, (uint32_t)((it / kStages) - 1) & 1);
         if (!ok) break;
         const uint32_t dst = sm_stages + s * kTileBytes;
-        const int token = t * a.S + c.tib * kTileKeys;
+        const int token = c.t * a.S + c.tib * kTileKeys;
         mbar_expect_tx(bar_full + 8 * s, kTileBytes);
         tma_load_4d(dst, &map_keys, bar_full + 8 * s, 0, token, h, b);
         tma_load_4d(dst + kTileAtomBytes, &map_keys, bar_full + 8 * s, kAtomCols, token, h, b);
+        new_group = cursor_last_of_group(c, a);
+        cursor_advance(c, a);
       }
       if (!ok) {
         record_status(a.status, kStatusTimeout);
@@ -365,14 +560,13 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
       const uint32_t idesc = (MODE == kLse) ? umma_idesc_bf16(128, kTileKeys)
                                             : umma_idesc_bf16(128, a.stat_rows);
       TileCursor c = cursor_at(x_begin, a);
-      int gid_cur = -1, gen = 0;
+      bool new_group = true;
+      int gen = 0;
       long long it = 0;
-      for (long long x = x_begin; x < x_end; ++x, ++it, cursor_advance(c, a)) {
-        const int gid = cursor_group(c, a);
-        if (gid != gid_cur) {
+      for (long long x = x_begin; x < x_end; ++x, ++it) {
+        if (new_group) {
           ok = mbar_wait(bar_stat, (uint32_t)gen & 1);
           if (!ok) break;
-          gid_cur = gid;
           ++gen;
         }
         const int s = (int)(it % kStages);
@@ -399,6 +593,8 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
         }
         umma_commit(bar_empty + 8 * s);     // stage reusable once these MMAs have read it
         umma_commit(bar_tfull + 8 * acc);   // accumulator ready for the epilogue
+        new_group = cursor_last_of_group(c, a);
+        cursor_advance(c, a);
       }
       if (!ok) record_status(a.status, kStatusTimeout);
     }
@@ -407,187 +603,36 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
     // ================= epilogue warps: four groups of four =================
     // Every group covers all 128 TMEM lanes (lane quarter = warp_id % 4); the groups split the
     // accumulator columns of every tile between them.
-    const int quarter = warp & 3;
-    const int row = quarter * 32 + lane;                   // TMEM lane owned by this thread
-    const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
-    const int ewarp = warp - 2;                            // 0..15
-    const int wg = ewarp >> 2;                             // epilogue group 0..3
-    const float c2 = a.scale_log2e;
-    bool ok = true;
-    TileCursor c = cursor_at(x_begin, a);
-    long long it = 0;
-
+    EpiCtx e;
+    e.quarter = warp & 3;
+    e.lane = lane;
+    e.row = e.quarter * 32 + lane;
+    e.t_lane = tmem_base + ((uint32_t)(e.quarter * 32) << 16);
+    e.ewarp = warp - 2;
+    e.wg = e.ewarp >> 2;
+    e.x_begin = x_begin;
+    e.x_end = x_end;
+    e.bar_tfull = bar_tfull; e.bar_tempty = bar_tempty; e.bar_stat = bar_stat; e.bar_stat_free = bar_stat_free;
+    e.bar_xa = bar_xa; e.bar_xb = bar_xb;
+    e.xch_s = xch_s;
+    e.hist_s = hist_s;
+    bool ok;
     if constexpr (MODE == kLse) {
-      // group -> (query row block, key column range)
-      const int ncg = kEpiGroups / nmb;                    // column groups: 4 (G*W <= 128) or 2
-      const int mb = wg % nmb, cg = wg / nmb;
-      const int cw = kTileKeys / ncg;                      // 32 or 64 key columns per thread
-      const int c0 = cg * cw;
-      const int q = mb * 128 + row;                        // this thread's query
-      float2* xch = reinterpret_cast<float2*>(xch_s);      // [ncg - 1][nmb * 128]
-      float m = -INFINITY, l = 0.f;
-      int flushes = 0;
-      for (long long x = x_begin; x < x_end; ++x, ++it) {
-        const int acc = (int)(it & 1);
-        ok = mbar_wait(bar_tfull + 8 * acc, (uint32_t)(it >> 1) & 1);
-        if (!ok) break;
-        tc_fence_after();
-        uint32_t v[kEpiCols];
-        load_epi_cols(t_lane + acc * kAccStride + mb * 128 + c0, cw, v);
-        tc_fence_before();
-        mbar_arrive(bar_tempty + 8 * acc);
-        const int nvalid = a.S - c.tib * kTileKeys;          // >= 1; columns at or beyond it hold no key
-        if (nvalid < c0 + cw) {
-#pragma unroll
-          for (int k = 0; k < kEpiCols; ++k) if (c0 + k >= nvalid) v[k] = 0xff800000u;
-        }
-        float cmax = -INFINITY;
-#pragma unroll
-        for (int k = 0; k < kEpiCols; k += 2) cmax = max3(__uint_as_float(v[k]), __uint_as_float(v[k + 1]), cmax);
-        const float m_new = fmaxf(m, cmax * c2);
-        const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
-        const float add = (cw == 64) ? sum_exp2<64, false>(v, c2, nullptr, -m_use)
-                                     : sum_exp2<32, false>(v, c2, nullptr, -m_use);
-        l = l * ex2_approx(m - m_use) + add;
-        m = m_new;
-        // end of this segment's run of tiles inside the slice: merge the column groups, write
-        // one partial, start over
-        TileCursor nx = c;
-        cursor_advance(nx, a);
-        const bool last = (x + 1 == x_end);
-        if (last || nx.seg != c.seg) {
-          if (cg > 0) {
-            if (flushes > 0) ok = mbar_wait(bar_xb, (uint32_t)(flushes - 1) & 1);
-            if (!ok) break;
-            xch[(cg - 1) * (nmb * 128) + q] = make_float2(m, l);
-            mbar_arrive(bar_xa);
-          } else {
-            ok = mbar_wait(bar_xa, (uint32_t)flushes & 1);
-            if (!ok) break;
-            float mx = m;
-            for (int g2 = 1; g2 < ncg; ++g2) mx = fmaxf(mx, xch[(g2 - 1) * (nmb * 128) + q].x);
-            float lt = (mx == -INFINITY) ? 0.f : l * ex2_approx(m - mx);
-            for (int g2 = 1; g2 < ncg; ++g2) {
-              const float2 o = xch[(g2 - 1) * (nmb * 128) + q];
-              if (o.x != -INFINITY) lt += o.y * ex2_approx(o.x - mx);
-            }
-            mbar_arrive(bar_xb);
-            if (q < a.GW) {
-              const int slot = (int)blockIdx.x - cta_of_tile((long long)c.seg * a.tiles_in_block, a.n_tiles, gridDim.x);
-              a.lse_part[((size_t)c.seg * a.n_slot + slot) * a.GW + q] = make_float2(mx, lt);
-            }
-          }
-          ++flushes;
-          m = -INFINITY;
-          l = 0.f;
-        }
-        if (!last && cursor_group(nx, a) != cursor_group(c, a)) mbar_arrive(bar_stat_free);
-        c = nx;
-      }
+      ok = (nmb == 2) ? lse_epilogue<64>(a, e, nmb) : lse_epilogue<32>(a, e, nmb);
     } else if constexpr (MODE == kScore) {
       // group g sums the query columns [c0, c1); widths are multiples of 16, at most 64
       const int cw = ((a.GW + kEpiGroups - 1) / kEpiGroups + 15) & ~15;
-      const int c0 = wg * cw;
-      const int c1 = min(a.GW, c0 + cw);
-      const int ncols = max(0, c1 - c0);
-      float* lw = reinterpret_cast<float*>(xch_s) + ewarp * kEpiCols;        // this warp's -lse values
-      float* part = reinterpret_cast<float*>(xch_s + 16 * kEpiCols * 4);     // [2 acc][3 groups][128 keys]
-      int seg_cur = -1;
-      for (long long x = x_begin; x < x_end; ++x, ++it) {
-        if (c.seg != seg_cur) {
-          // log2-sum-exp2 of this warp's queries from the partials of the CTAs that covered the segment
-          const long long first = (long long)c.seg * a.tiles_in_block;
-          const int cf = cta_of_tile(first, a.n_tiles, a.lse_ctas);
-          const int n_used = cta_of_tile(first + a.tiles_in_block - 1, a.n_tiles, a.lse_ctas) - cf + 1;
-          __syncwarp();
-#pragma unroll
-          for (int half = 0; half < 2; ++half) {
-            const int qq = c0 + lane + 32 * half;
-            float neg_lse = 0.f;
-            if (qq < c1) {
-              const float2* p = a.lse_part + (size_t)c.seg * a.n_slot * a.GW + qq;
-              float mx = -INFINITY;
-              for (int s2 = 0; s2 < n_used; ++s2) mx = fmaxf(mx, p[(size_t)s2 * a.GW].x);
-              float sum = 0.f;
-              for (int s2 = 0; s2 < n_used; ++s2) {
-                const float2 e = p[(size_t)s2 * a.GW];
-                if (e.x != -INFINITY) sum += e.y * exp2f(e.x - mx);
-              }
-              const float r = mx + log2f(sum);
-              neg_lse = -r;
-              if (c.tib == 0 && quarter == 0) a.lse2[(size_t)c.seg * a.GW + qq] = r;
-            }
-            lw[lane + 32 * half] = neg_lse;
-          }
-          __syncwarp();
-          seg_cur = c.seg;
-        }
-        const int acc = (int)(it & 1);
-        ok = mbar_wait(bar_tfull + 8 * acc, (uint32_t)(it >> 1) & 1);
-        if (!ok) break;
-        tc_fence_after();
-        uint32_t v[kEpiCols];
-        load_epi_cols(t_lane + acc * kAccStride + c0, ncols, v);
-        tc_fence_before();
-        mbar_arrive(bar_tempty + 8 * acc);
-        float sum = 0.f;
-        if (ncols > 32) sum = sum_exp2<64, true>(v, c2, lw, 0.f);
-        else if (ncols > 0) sum = sum_exp2<32, true>(v, c2, lw, 0.f);
-        // groups 1..3 hand their sums to group 0, which adds them in a fixed order
-        if (wg > 0) {
-          if (it >= 2) ok = mbar_wait(bar_xb + 8 * acc, (uint32_t)((it >> 1) - 1) & 1);
-          if (!ok) break;
-          part[(acc * 3 + (wg - 1)) * 128 + row] = sum;
-          mbar_arrive(bar_xa + 8 * acc);
-        } else {
-          ok = mbar_wait(bar_xa + 8 * acc, (uint32_t)(it >> 1) & 1);
-          if (!ok) break;
-          const float tot = ((sum + part[(acc * 3 + 0) * 128 + row]) + part[(acc * 3 + 1) * 128 + row]) +
-                            part[(acc * 3 + 2) * 128 + row];
-          mbar_arrive(bar_xb + 8 * acc);
-          const int key = c.tib * kTileKeys + row;
-          if (key < a.S) a.s_exact[(size_t)c.seg * a.S + key] = tot;
-        }
-        TileCursor nx = c;
-        cursor_advance(nx, a);
-        if (x + 1 < x_end && cursor_group(nx, a) != cursor_group(c, a)) mbar_arrive(bar_stat_free);
-        c = nx;
+      const int c0 = e.wg * cw;
+      const int ncols = max(0, min(a.GW, c0 + cw) - c0);
+      switch (ncols) {
+        case 64: ok = score_epilogue<64>(a, e, c0); break;
+        case 48: ok = score_epilogue<48>(a, e, c0); break;
+        case 32: ok = score_epilogue<32>(a, e, c0); break;
+        case 16: ok = score_epilogue<16>(a, e, c0); break;
+        default: ok = score_epilogue<0>(a, e, c0); break;
       }
     } else {
-      // ---- kProj: sign bits -> bucket codes -> histogram lookups ----
-      // Bucket code of a table: bit b of the table (hyperplane r*K + b) sits at position
-      // K-1-b, i.e. the first hyperplane is the most significant bit; bit = [projection >= 0].
-      // Group g handles tables [g*TC/4, (g+1)*TC/4) of the chunk.
-      constexpr int TQ = TC / kEpiGroups;
-      int gid_cur = -1, gen = 0;
-      for (long long x = x_begin; x < x_end; ++x, ++it) {
-        const int gid = cursor_group(c, a);
-        if (gid != gid_cur) {
-          ok = mbar_wait(bar_stat, (uint32_t)gen & 1);   // histogram slice landed (async-proxy writes visible after the wait)
-          if (!ok) break;
-          gid_cur = gid;
-          ++gen;
-        }
-        const int acc = (int)(it & 1);
-        ok = mbar_wait(bar_tfull + 8 * acc, (uint32_t)(it >> 1) & 1);
-        if (!ok) break;
-        tc_fence_after();
-        const int key = c.tib * kTileKeys + row;
-        const bool valid = key < a.S;
-        const uint32_t t_acc = t_lane + acc * kAccStride;
-        const uint32_t bar_rel = bar_tempty + 8 * acc;
-        const int table0 = c.chunk * TC;
-        uint32_t partial;
-        if (wg == 0) partial = proj_tables<KBITS, 0, TQ>(t_acc, bar_rel, hist_s, a, c.seg, key, table0, valid);
-        else if (wg == 1) partial = proj_tables<KBITS, TQ, 2 * TQ>(t_acc, bar_rel, hist_s, a, c.seg, key, table0, valid);
-        else if (wg == 2) partial = proj_tables<KBITS, 2 * TQ, 3 * TQ>(t_acc, bar_rel, hist_s, a, c.seg, key, table0, valid);
-        else partial = proj_tables<KBITS, 3 * TQ, 4 * TQ>(t_acc, bar_rel, hist_s, a, c.seg, key, table0, valid);
-        if (valid) atomicAdd(a.counts + (size_t)c.seg * a.S + key, partial);
-        TileCursor nx = c;
-        cursor_advance(nx, a);
-        if (x + 1 < x_end && cursor_group(nx, a) != gid) mbar_arrive(bar_stat_free);
-        c = nx;
-      }
+      ok = proj_epilogue<KBITS, TC>(a, e);
     }
     if (!ok) record_status(a.status, kStatusTimeout);
   }
