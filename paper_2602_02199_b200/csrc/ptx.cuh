@@ -225,6 +225,26 @@ __device__ __forceinline__ uint64_t umma_sdesc_sw128(uint32_t saddr) {
          (static_cast<uint64_t>(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
 }
 
+// The same descriptor split in two words: the high word is one constant for every operand of
+// these kernels, the low word is (address >> 4) plus the version bit, so stepping through an
+// operand is a 32-bit add of (byte offset >> 4).
+constexpr uint32_t kSdescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint32_t umma_sdesc_lo(uint32_t saddr) {
+  return ((saddr & 0x3FFFFu) >> 4) | (1u << 16);
+}
+// tcgen05.mma with both shared-memory descriptors given by their low words.
+__device__ __forceinline__ void umma_bf16_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc,
+                                             uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "mov.b64 da, {%1, %5};\n\t"
+      "mov.b64 db, {%2, %5};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}" ::"r"(d_tmem),
+      "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kSdescHi)
+      : "memory");
+}
+
 // tcgen05.wait::ld that also names the loaded registers as in/out operands, so that no use of
 // them can be scheduled before the wait (the loads are asynchronous until then).
 __device__ __forceinline__ void tmem_wait_ld_dep32(uint32_t* r) {

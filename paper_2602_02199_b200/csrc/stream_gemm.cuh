@@ -555,10 +555,14 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
     __syncwarp();
   } else if (warp == 1) {
     // ================= MMA issuer =================
-    if (lane == 0 && x_begin < x_end) {
+    // The whole warp walks the loop (uniform waits and address arithmetic); one elected lane
+    // issues the MMAs and their commits.
+    if (x_begin < x_end) {
       bool ok = true;
       const uint32_t idesc = (MODE == kLse) ? umma_idesc_bf16(128, kTileKeys)
                                             : umma_idesc_bf16(128, a.stat_rows);
+      const uint32_t stat_lo = umma_sdesc_lo(sm_stat);
+      const uint32_t stat_atom_lo = stat_atom_bytes >> 4;
       TileCursor c = cursor_at(x_begin, a);
       bool new_group = true;
       int gen = 0;
@@ -575,28 +579,29 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
         if (ok) ok = mbar_wait(bar_full + 8 * s, (uint32_t)(it / kStages) & 1);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t tile = sm_stages + s * kTileBytes;
-        for (int mb = 0; mb < nmb; ++mb) {
-          const uint32_t d = tmem_base + acc * kAccStride + mb * 128;
+        const uint32_t tile_lo = umma_sdesc_lo(sm_stages + s * kTileBytes);
+        const uint32_t d0 = tmem_base + acc * kAccStride;
+        if (elect_one()) {
 #pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            const uint32_t koff = (k & 3) * 32;
-            const uint32_t tile_k = tile + (k >> 2) * kTileAtomBytes + koff;
-            const uint32_t stat_k = sm_stat + (k >> 2) * stat_atom_bytes + koff;
-            if (MODE == kLse) {
-              umma_bf16(d, umma_sdesc_sw128(stat_k + mb * (128 * 128)), umma_sdesc_sw128(tile_k),
-                        idesc, k > 0);
-            } else {
-              umma_bf16(d, umma_sdesc_sw128(tile_k), umma_sdesc_sw128(stat_k), idesc, k > 0);
+          for (int mb = 0; mb < 2; ++mb) {
+            if (mb < nmb) {
+#pragma unroll
+              for (int k = 0; k < 8; ++k) {
+                const uint32_t tile_k = tile_lo + (k >> 2) * (kTileAtomBytes >> 4) + (k & 3) * 2;
+                const uint32_t stat_k = stat_lo + (k >> 2) * stat_atom_lo + (k & 3) * 2 + mb * ((128 * 128) >> 4);
+                if (MODE == kLse) umma_bf16_lo(d0 + mb * 128, stat_k, tile_k, idesc, k > 0);
+                else umma_bf16_lo(d0, tile_k, stat_k, idesc, k > 0);
+              }
             }
           }
+          umma_commit(bar_empty + 8 * s);     // stage reusable once these MMAs have read it
+          umma_commit(bar_tfull + 8 * acc);   // accumulator ready for the epilogue
         }
-        umma_commit(bar_empty + 8 * s);     // stage reusable once these MMAs have read it
-        umma_commit(bar_tfull + 8 * acc);   // accumulator ready for the epilogue
+        __syncwarp();
         new_group = cursor_last_of_group(c, a);
         cursor_advance(c, a);
       }
-      if (!ok) record_status(a.status, kStatusTimeout);
+      if (!ok && lane == 0) record_status(a.status, kStatusTimeout);
     }
     __syncwarp();
   } else if (x_begin < x_end) {
