@@ -252,6 +252,7 @@ def run_ours(args, w, rank, world, local_rank):
     prof = eng.laser_kv_profile_read()
     eng.laser_kv_profile_enable(False)
     eng.laser_kv_poll_status()
+    sign_fixups = int(eng.laser_kv_debug_view().n_sign_fixups)
     clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
 
     # ---- end to end: pinned host inputs -> device, select, appended positions -> host ----
@@ -322,6 +323,7 @@ def run_ours(args, w, rank, world, local_rank):
         "bytes_alg_per_step": work["bytes"], "flops_alg_per_step": work["flops"],
         "kernels_ms_per_step": {k: v[0] / v[1] for k, v in kern.items()},
         "kernel_share": {k: v[0] / total_kernel_ms for k, v in kern.items()},
+        "exact_sign_items_last_step": sign_fixups,
     }
 
     if args.skip_cpu:

@@ -26,8 +26,8 @@ constexpr int kHeadDim = 128;
 constexpr size_t kAlign = 256;
 constexpr int kMaxSmem = 227 * 1024;
 
-constexpr int kProfKernels = 8;
-const char* const kProfNames[kProfKernels] = {"memset", "qprep_kernel", "stream_kernel<lse>", "stream_kernel<score>",
+constexpr int kProfKernels = 7;
+const char* const kProfNames[kProfKernels] = {"qprep_kernel", "stream_kernel<lse>", "stream_kernel<score>",
                                               "stream_kernel<proj>", "signfix_kernel", "select_kernel", "append_kernel"};
 
 std::atomic<long long> g_launches{0};
@@ -467,15 +467,12 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
     marks.push_back(ev);
   };
   mark();
-  // fix-up counter (ctrl[1]) and changed counter (ctrl[2]) restart; the status word (ctrl[0]) is kept
-  LKV_CUDA(cudaMemsetAsync(ctrl + 1, 0, 8, st), "memset ctrl");
-  LKV_CUDA(cudaMemsetAsync(counts, 0, (size_t)nseg * S * 4, st), "memset counts");
-
-  mark();
-  // 1. query signatures and bucket histogram
+  // 1. query signatures and bucket histogram; also clears the counts and restarts the fix-up
+  //    counter (ctrl[1]) and the changed counter (ctrl[2]); the status word (ctrl[0]) is kept
   {
     QprepArgs qa{static_cast<const uint16_t*>(Q_win), q_strides[0], q_strides[1], q_strides[2], h->P, hist, qb,
-                 c.n_kv_heads, d.G, c.window, d.GW, c.lsh_bits, c.lsh_tables};
+                 c.n_kv_heads, d.G, c.window, d.GW, c.lsh_bits, c.lsh_tables,
+                 reinterpret_cast<uint4*>(counts), (long long)nseg * S / 4, ctrl + 1};
     const size_t smem = qprep_smem_bytes(c.lsh_bits);
     dim3 grid(c.lsh_tables, c.n_kv_heads, c.batch);
     switch (c.lsh_bits) {

@@ -31,6 +31,9 @@ struct QprepArgs {
   uint16_t* hist;         // [batch][H_kv][L][2^K]
   uint16_t* qbuckets;     // [batch][H_kv][GW][L]
   int H_kv, G, W, GW, K, L;
+  uint4* zero_begin;      // the call's collision counts, cleared here (16-byte units)
+  long long zero_n;
+  int* counters;          // fix-up and changed counters, restarted here
 };
 
 constexpr int kQprepThreads = 128;
@@ -44,6 +47,15 @@ __global__ void __launch_bounds__(kQprepThreads) qprep_kernel(const QprepArgs a)
   uint32_t* bins = reinterpret_cast<uint32_t*>(smem_q + (size_t)K * 128 * 8);   // [2^K]
   const int r = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   constexpr int nbins = 1 << K;
+  {
+    // this CTA's share of the count array; the projection pass accumulates into it later
+    const long long cta = ((long long)b * gridDim.y + h) * gridDim.x + r;
+    const long long nctas = (long long)gridDim.x * gridDim.y * gridDim.z;
+    const long long per = (a.zero_n + nctas - 1) / nctas;
+    const long long z0 = cta * per, z1 = min(a.zero_n, z0 + per);
+    for (long long i = z0 + threadIdx.x; i < z1; i += kQprepThreads) a.zero_begin[i] = make_uint4(0u, 0u, 0u, 0u);
+    if (cta == 0 && threadIdx.x < 2) a.counters[threadIdx.x] = 0;
+  }
   for (int i = threadIdx.x; i < K * 128; i += kQprepThreads)
     planes[i] = bf16_to_f64(a.P[(size_t)r * K * 128 + i]);
   for (int i = threadIdx.x; i < nbins; i += kQprepThreads) bins[i] = 0;
@@ -101,10 +113,11 @@ __global__ void __launch_bounds__(kQprepThreads) qprep_kernel(const QprepArgs a)
 }
 
 // ------------------------------------------------------------------------------------------------
-// Exact recomputation of flagged key signs. One warp per item; every lane holds four key elements
-// and forms its share of all K dot products at once (independent fp64 accumulators, exact bf16
-// products), then the K partial sums are reduced across the warp. If the exact bucket code
-// differs from the provisional one the key's count is corrected by hist[new] - hist[old].
+// Exact recomputation of flagged key signs. An item names a key, a table, the provisional bucket
+// code and a mask of the code bits whose projection was too small to trust. One warp per item:
+// for every masked bit the 128-term dot product is formed in fp64 (exact bf16 products, four
+// terms per lane, warp reduction) and the bit is replaced by its exact sign. If the bucket code
+// changes, the key's count is corrected by hist[new] - hist[old].
 // ------------------------------------------------------------------------------------------------
 struct SignfixArgs {
   const uint16_t* Kp;     // keys via strides
@@ -113,15 +126,14 @@ struct SignfixArgs {
   const uint16_t* hist;
   uint32_t* counts;
   uint16_t* key_buckets;  // or nullptr
-  const int4* items;
+  const int4* items;      // (segment, key, table, code | mask << 16)
   const int* n_items;
   int cap;
   int H_kv, nb, S, K, L;
   int* n_changed;
 };
 
-constexpr int kMaxLshBits = 12;
-constexpr int kSignfixCtas = 1184;   // 8 CTAs of 8 warps per SM: a few items per warp at most
+constexpr int kSignfixCtas = 592;   // 4 CTAs of 8 warps per SM: a few items per warp at most
 
 __global__ void __launch_bounds__(256) signfix_kernel(const SignfixArgs a) {
   const int lane = threadIdx.x & 31;
@@ -130,37 +142,31 @@ __global__ void __launch_bounds__(256) signfix_kernel(const SignfixArgs a) {
   const int n = min(*a.n_items, a.cap);
   for (int it = wid; it < n; it += nwarps) {
     const int4 item = a.items[it];
-    const int seg = item.x, key = item.y, r = item.z, old_code = item.w;
+    const int seg = item.x, key = item.y, r = item.z;
+    const uint32_t old_code = (uint32_t)item.w & 0xFFFFu;
+    uint32_t mask = (uint32_t)item.w >> 16;
     const int t = seg % a.nb;
     const int h = (seg / a.nb) % a.H_kv;
     const int b = seg / (a.nb * a.H_kv);
     const uint16_t* krow = a.Kp + b * a.ks_b + h * a.ks_h + ((long long)t * a.S + key) * a.ks_t;
     const uint2 kv = *reinterpret_cast<const uint2*>(krow + lane * 4);
-    uint2 pv[kMaxLshBits];
-#pragma unroll
-    for (int bit = 0; bit < kMaxLshBits; ++bit)
-      pv[bit] = (bit < a.K) ? *reinterpret_cast<const uint2*>(a.P + ((size_t)r * a.K + bit) * 128 + lane * 4)
-                            : make_uint2(0u, 0u);
     const double k0 = bf16_to_f64((uint16_t)(kv.x & 0xFFFF)), k1 = bf16_to_f64((uint16_t)(kv.x >> 16));
     const double k2 = bf16_to_f64((uint16_t)(kv.y & 0xFFFF)), k3 = bf16_to_f64((uint16_t)(kv.y >> 16));
-    double acc[kMaxLshBits];
+    uint32_t code = old_code;
+    while (mask) {
+      const int pos = 31 - __clz(mask);          // code bit; hyperplane r*K + (K-1-pos)
+      mask &= ~(1u << pos);
+      const int bit = a.K - 1 - pos;
+      const uint2 pv = *reinterpret_cast<const uint2*>(a.P + ((size_t)r * a.K + bit) * 128 + lane * 4);
+      double acc = k0 * bf16_to_f64((uint16_t)(pv.x & 0xFFFF));
+      acc = fma(k1, bf16_to_f64((uint16_t)(pv.x >> 16)), acc);
+      acc = fma(k2, bf16_to_f64((uint16_t)(pv.y & 0xFFFF)), acc);
+      acc = fma(k3, bf16_to_f64((uint16_t)(pv.y >> 16)), acc);
 #pragma unroll
-    for (int bit = 0; bit < kMaxLshBits; ++bit) {
-      double s = k0 * bf16_to_f64((uint16_t)(pv[bit].x & 0xFFFF));
-      s = fma(k1, bf16_to_f64((uint16_t)(pv[bit].x >> 16)), s);
-      s = fma(k2, bf16_to_f64((uint16_t)(pv[bit].y & 0xFFFF)), s);
-      acc[bit] = fma(k3, bf16_to_f64((uint16_t)(pv[bit].y >> 16)), s);
+      for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+      code = (code & ~(1u << pos)) | ((acc >= 0.0 ? 1u : 0u) << pos);
     }
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-#pragma unroll
-      for (int bit = 0; bit < kMaxLshBits; ++bit) acc[bit] += __shfl_xor_sync(0xffffffffu, acc[bit], off);
-    }
-    uint32_t code = 0;
-#pragma unroll
-    for (int bit = 0; bit < kMaxLshBits; ++bit)
-      if (bit < a.K) code = (code << 1) | (acc[bit] >= 0.0 ? 1u : 0u);
-    if (lane == 0 && (int)code != old_code) {
+    if (lane == 0 && code != old_code) {
       const uint16_t* hr = a.hist + ((size_t)(b * a.H_kv + h) * a.L + r) * ((size_t)1 << a.K);
       const uint32_t delta = (uint32_t)hr[code] - (uint32_t)hr[old_code];
       atomicAdd(a.counts + (size_t)seg * a.S + key, delta);

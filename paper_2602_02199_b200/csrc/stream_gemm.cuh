@@ -72,7 +72,7 @@ struct StreamArgs {
   uint32_t* counts;        // [seg][S]
   const uint16_t* hist;    // [batch][H_kv][L][2^K]
   uint16_t* key_buckets;   // [seg][S][L] or nullptr
-  int4* fix_items;         // (seg, key, table, provisional bucket)
+  int4* fix_items;         // (seg, key, table, provisional bucket | doubtful bits << 16)
   int* fix_count;
   int fix_cap;
   int* status;
@@ -232,8 +232,12 @@ __device__ __forceinline__ uint32_t proj_tables(uint32_t t_acc, uint32_t bar_rel
       const int r = table0 + T_BEGIN + t;
       if (a.key_buckets) a.key_buckets[((size_t)seg * a.S + key) * a.lsh_tables + r] = (uint16_t)code[t];
       if (!(amin[t] >= tau)) {
+        uint32_t doubt = 0;                                // code bits whose projection is below tau
+#pragma unroll
+        for (int k = 0; k < KBITS; ++k)
+          if (!(fabsf(__uint_as_float(v[t * KBITS + k])) >= tau)) doubt |= 1u << (KBITS - 1 - k);
         const int slot = atomicAdd(a.fix_count, 1);
-        if (slot < a.fix_cap) a.fix_items[slot] = make_int4(seg, key, r, (int)code[t]);
+        if (slot < a.fix_cap) a.fix_items[slot] = make_int4(seg, key, r, (int)(code[t] | (doubt << 16)));
         else record_status(a.status, kStatusCapacity);
       }
     }
