@@ -40,31 +40,57 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-// One attempt: the hardware may park the thread for up to `kSuspendHintNs` before it answers.
-constexpr uint32_t kSuspendHintNs = 20000;
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+// Bounded waits for the phase with the given parity, written as one PTX loop each so that the
+// fast path (phase already complete) is a try_wait and a branch. Both return false when the poll
+// budget ran out; the budgets correspond to a second or more, far beyond any legitimate wait of
+// these kernels.
+//
+// mbar_wait_spin polls back to back: for the one thread whose reaction time is on the critical
+// path (the MMA issuer).
+constexpr uint32_t kMaxSpinPolls = 1u << 26;
+__device__ __forceinline__ bool mbar_wait_spin(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "{\n\t.reg .pred p;\n\t.reg .u32 n;\n\t"
+      "mov.u32 n, 0;\n"
+      "LKV_SPIN_TRY:\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "@p bra LKV_SPIN_DONE;\n\t"
+      "add.u32 n, n, 1;\n\t"
+      "setp.lt.u32 p, n, %3;\n\t"
+      "@p bra LKV_SPIN_TRY;\n\t"
+      "setp.ne.u32 p, n, n;\n"
+      "LKV_SPIN_DONE:\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
-      : "r"(bar), "r"(parity), "r"(kSuspendHintNs)
+      : "r"(bar), "r"(parity), "r"(kMaxSpinPolls)
       : "memory");
   return ok != 0;
 }
 
-// About two seconds at 2 GHz: far beyond any legitimate wait of these kernels.
-constexpr long long kWaitBudgetCycles = 4000000000LL;
-
-// Bounded wait for the phase with the given parity. Returns false when the budget ran out.
+// mbar_wait sleeps a few tens of nanoseconds between polls, so that many waiting warps leave the
+// issue slots to the working ones.
+constexpr uint32_t kBackoffNs = 32;
+constexpr uint32_t kMaxPolls = 1u << 25;
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
-  while (!mbar_try_wait(bar, parity)) {
-    if (clock64() - t0 > kWaitBudgetCycles) return false;
-  }
-  return true;
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .u32 n;\n\t"
+      "mov.u32 n, 0;\n"
+      "LKV_WAIT_TRY:\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "@p bra LKV_WAIT_DONE;\n\t"
+      "nanosleep.u32 %4;\n\t"
+      "add.u32 n, n, 1;\n\t"
+      "setp.lt.u32 p, n, %3;\n\t"
+      "@p bra LKV_WAIT_TRY;\n\t"
+      "setp.ne.u32 p, n, n;\n"
+      "LKV_WAIT_DONE:\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity), "r"(kMaxPolls), "r"(kBackoffNs)
+      : "memory");
+  return ok != 0;
 }
 
 // ---- TMA -------------------------------------------------------------------------------------

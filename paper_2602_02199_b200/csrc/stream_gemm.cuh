@@ -41,7 +41,14 @@ constexpr int kStreamThreads = 64 + kEpilogueThreads;
 constexpr int kEpiCols = 64;                   // accumulator columns an epilogue thread holds at most
 constexpr int kXchBytes = 8192;                // exchange area between epilogue warps
 constexpr int kTmemCols = 512;
-constexpr int kAccStride = 256;                // TMEM columns per accumulator buffer
+constexpr int kAccStride = 256;                // TMEM columns per accumulator buffer (kLse, kScore: two buffers)
+constexpr int kMaxAcc = 4;                     // most accumulator buffers of any mode
+
+// kProj accumulators are TC*K columns wide: as many buffers as fit the 512 TMEM columns, at most 4.
+__host__ __device__ constexpr int proj_acc_stride(int kbits, int tc) { return (kbits * tc + 31) / 32 * 32; }
+__host__ __device__ constexpr int proj_num_acc(int kbits, int tc) {
+  return 512 / proj_acc_stride(kbits, tc) < kMaxAcc ? 512 / proj_acc_stride(kbits, tc) : kMaxAcc;
+}
 constexpr int kMaxStatRows = 256;
 constexpr int kMaxStreamCtas = 256;            // upper bound of the persistent grid (slot arithmetic)
 constexpr int kPolyPairsOf32 = 12;             // of every 32 column pairs, this many take 2^x on the FMA pipe
@@ -256,6 +263,23 @@ struct EpiCtx {
   const uint16_t* hist_s;      // histogram slice (kProj)
 };
 
+// A run: the tiles of one block segment that fall inside the CTA's slice. The epilogue loops walk
+// the slice run by run, so that the per-tile work carries no segment or group bookkeeping.
+struct TileRun {
+  TileCursor c;        // first tile of the run
+  int ntiles;
+  bool ends_group;     // the tile after the run (if any) needs another stationary operand
+};
+__device__ __forceinline__ TileRun run_at(long long x, long long x_end, const StreamArgs& a) {
+  TileRun r;
+  r.c = cursor_at(x, a);
+  const long long left = x_end - x;
+  const int in_block = a.tiles_in_block - r.c.tib;
+  r.ntiles = left < in_block ? (int)left : in_block;
+  r.ends_group = (r.c.tib + r.ntiles == a.tiles_in_block) && (r.c.t == a.nb - 1);
+  return r;
+}
+
 // kLse: CW key columns per thread (64 when G*W > 128: two query row blocks x two column groups;
 // 32 otherwise: one row block x four column groups).
 template <int CW>
@@ -268,63 +292,59 @@ __device__ __forceinline__ bool lse_epilogue(const StreamArgs& a, const EpiCtx& 
   float2* xch = reinterpret_cast<float2*>(e.xch_s);    // [ncg - 1][nq]
   const float c2 = a.scale_log2e;
   const uint32_t t_col = e.t_lane + mb * 128 + c0;
-  float m = -INFINITY, l = 0.f;
   int flushes = 0;
-  TileCursor c = cursor_at(e.x_begin, a);
-  long long it = 0;
-  for (long long x = e.x_begin; x < e.x_end; ++x, ++it) {
-    const int acc = (int)(it & 1);
-    if (!mbar_wait(e.bar_tfull + 8 * acc, (uint32_t)(it >> 1) & 1)) return false;
-    tc_fence_after();
-    uint32_t v[CW];
-    load_epi_cols<CW>(t_col + acc * kAccStride, v);
-    tc_fence_before();
-    mbar_arrive(e.bar_tempty + 8 * acc);
-    const int nvalid = a.S - c.tib * kTileKeys;        // >= 1; columns at or beyond it hold no key
-    if (nvalid < c0 + CW) {
-      asm volatile("" ::: "memory");                   // keeps this rare path a real branch
+  uint32_t it = 0;
+  for (long long x = e.x_begin; x < e.x_end;) {
+    const TileRun r = run_at(x, e.x_end, a);
+    float m = -INFINITY, l = 0.f;
+    int nvalid = a.S - r.c.tib * kTileKeys - c0;       // key columns of this thread's range that hold a key
+    for (int j = 0; j < r.ntiles; ++j, ++it, nvalid -= kTileKeys) {
+      const uint32_t acc = it & 1;
+      if (!mbar_wait(e.bar_tfull + 8 * acc, (it >> 1) & 1)) return false;
+      tc_fence_after();
+      uint32_t v[CW];
+      load_epi_cols<CW>(t_col + acc * kAccStride, v);
+      tc_fence_before();
+      mbar_arrive(e.bar_tempty + 8 * acc);
+      if (nvalid < CW) {
+        asm volatile("" ::: "memory");                 // keeps this rare path a real branch
 #pragma unroll
-      for (int k = 0; k < CW; ++k) if (c0 + k >= nvalid) v[k] = 0xff800000u;
-    }
-    float cmax = -INFINITY;
-#pragma unroll
-    for (int k = 0; k < CW; k += 2) cmax = max3(__uint_as_float(v[k]), __uint_as_float(v[k + 1]), cmax);
-    const float m_new = fmaxf(m, cmax * c2);
-    const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
-    const float add = sum_exp2<CW, false>(v, c2, nullptr, -m_use);
-    l = l * ex2_approx(m - m_use) + add;
-    m = m_new;
-    const bool last = (x + 1 == e.x_end);
-    if (last || cursor_last_of_segment(c, a)) {
-      // end of this segment's run of tiles inside the slice: merge the column groups, write one
-      // partial, start over
-      if (cg > 0) {
-        if (flushes > 0 && !mbar_wait(e.bar_xb, (uint32_t)(flushes - 1) & 1)) return false;
-        xch[(cg - 1) * nq + q] = make_float2(m, l);
-        mbar_arrive(e.bar_xa);
-      } else {
-        if (!mbar_wait(e.bar_xa, (uint32_t)flushes & 1)) return false;
-        float mx = m;
-#pragma unroll
-        for (int g2 = 1; g2 < ncg; ++g2) mx = fmaxf(mx, xch[(g2 - 1) * nq + q].x);
-        float lt = (mx == -INFINITY) ? 0.f : l * ex2_approx(m - mx);
-#pragma unroll
-        for (int g2 = 1; g2 < ncg; ++g2) {
-          const float2 o = xch[(g2 - 1) * nq + q];
-          if (o.x != -INFINITY) lt += o.y * ex2_approx(o.x - mx);
-        }
-        mbar_arrive(e.bar_xb);
-        if (q < a.GW) {
-          const int slot = (int)blockIdx.x - cta_of_tile((long long)c.seg * a.tiles_in_block, a.n_tiles, gridDim.x);
-          a.lse_part[((size_t)c.seg * a.n_slot + slot) * a.GW + q] = make_float2(mx, lt);
-        }
+        for (int k = 0; k < CW; ++k) if (k >= nvalid) v[k] = 0xff800000u;
       }
-      ++flushes;
-      m = -INFINITY;
-      l = 0.f;
+      float cmax = -INFINITY;
+#pragma unroll
+      for (int k = 0; k < CW; k += 2) cmax = max3(__uint_as_float(v[k]), __uint_as_float(v[k + 1]), cmax);
+      const float m_new = fmaxf(m, cmax * c2);
+      const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
+      const float add = sum_exp2<CW, false>(v, c2, nullptr, -m_use);
+      l = l * ex2_approx(m - m_use) + add;
+      m = m_new;
     }
-    if (!last && cursor_last_of_group(c, a)) mbar_arrive(e.bar_stat_free);
-    cursor_advance(c, a);
+    // end of this segment's run of tiles: merge the column groups, write one partial
+    if (cg > 0) {
+      if (flushes > 0 && !mbar_wait(e.bar_xb, (uint32_t)(flushes - 1) & 1)) return false;
+      xch[(cg - 1) * nq + q] = make_float2(m, l);
+      mbar_arrive(e.bar_xa);
+    } else {
+      if (!mbar_wait(e.bar_xa, (uint32_t)flushes & 1)) return false;
+      float mx = m;
+#pragma unroll
+      for (int g2 = 1; g2 < ncg; ++g2) mx = fmaxf(mx, xch[(g2 - 1) * nq + q].x);
+      float lt = (mx == -INFINITY) ? 0.f : l * ex2_approx(m - mx);
+#pragma unroll
+      for (int g2 = 1; g2 < ncg; ++g2) {
+        const float2 o = xch[(g2 - 1) * nq + q];
+        if (o.x != -INFINITY) lt += o.y * ex2_approx(o.x - mx);
+      }
+      mbar_arrive(e.bar_xb);
+      if (q < a.GW) {
+        const int slot = (int)blockIdx.x - cta_of_tile((long long)r.c.seg * a.tiles_in_block, a.n_tiles, gridDim.x);
+        a.lse_part[((size_t)r.c.seg * a.n_slot + slot) * a.GW + q] = make_float2(mx, lt);
+      }
+    }
+    ++flushes;
+    x += r.ntiles;
+    if (r.ends_group && x < e.x_end) mbar_arrive(e.bar_stat_free);
   }
   return true;
 }
@@ -335,13 +355,12 @@ __device__ __forceinline__ bool score_epilogue(const StreamArgs& a, const EpiCtx
   float* lw = reinterpret_cast<float*>(e.xch_s) + e.ewarp * kEpiCols;       // this warp's -lse values
   float* part = reinterpret_cast<float*>(e.xch_s + 16 * kEpiCols * 4);      // [2 acc][3 groups][128 keys]
   const float c2 = a.scale_log2e;
-  bool new_seg = true;
-  TileCursor c = cursor_at(e.x_begin, a);
-  long long it = 0;
-  for (long long x = e.x_begin; x < e.x_end; ++x, ++it) {
-    if (new_seg && NC > 0) {
+  uint32_t it = 0;
+  for (long long x = e.x_begin; x < e.x_end;) {
+    const TileRun r = run_at(x, e.x_end, a);
+    if constexpr (NC > 0) {
       // log2-sum-exp2 of this warp's queries from the partials of the CTAs that covered the segment
-      const long long first = (long long)c.seg * a.tiles_in_block;
+      const long long first = (long long)r.c.seg * a.tiles_in_block;
       const int cf = cta_of_tile(first, a.n_tiles, a.lse_ctas);
       const int n_used = cta_of_tile(first + a.tiles_in_block - 1, a.n_tiles, a.lse_ctas) - cf + 1;
       __syncwarp();
@@ -350,7 +369,7 @@ __device__ __forceinline__ bool score_epilogue(const StreamArgs& a, const EpiCtx
         const int j = e.lane + 32 * half;
         if (j < NC) {
           const int qq = c0 + j;
-          const float2* p = a.lse_part + (size_t)c.seg * a.n_slot * a.GW + qq;
+          const float2* p = a.lse_part + (size_t)r.c.seg * a.n_slot * a.GW + qq;
           float mx = -INFINITY;
           for (int s2 = 0; s2 < n_used; ++s2) mx = fmaxf(mx, p[(size_t)s2 * a.GW].x);
           float sum = 0.f;
@@ -358,43 +377,45 @@ __device__ __forceinline__ bool score_epilogue(const StreamArgs& a, const EpiCtx
             const float2 pe = p[(size_t)s2 * a.GW];
             if (pe.x != -INFINITY) sum += pe.y * exp2f(pe.x - mx);
           }
-          const float r = mx + log2f(sum);
-          if (c.tib == 0 && e.quarter == 0) a.lse2[(size_t)c.seg * a.GW + qq] = r;
-          lw[j] = -r;
+          const float lse = mx + log2f(sum);
+          if (r.c.tib == 0 && e.quarter == 0) a.lse2[(size_t)r.c.seg * a.GW + qq] = lse;
+          lw[j] = -lse;
         }
       }
       __syncwarp();
     }
-    const int acc = (int)(it & 1);
-    if (!mbar_wait(e.bar_tfull + 8 * acc, (uint32_t)(it >> 1) & 1)) return false;
-    tc_fence_after();
-    float sum = 0.f;
-    if constexpr (NC > 0) {
-      uint32_t v[NC];
-      load_epi_cols<NC>(e.t_lane + acc * kAccStride + c0, v);
-      tc_fence_before();
-      mbar_arrive(e.bar_tempty + 8 * acc);
-      sum = sum_exp2<NC, true>(v, c2, lw, 0.f);
-    } else {
-      tc_fence_before();
-      mbar_arrive(e.bar_tempty + 8 * acc);
+    float* out = a.s_exact + (size_t)r.c.seg * a.S;
+    int key = r.c.tib * kTileKeys + e.row;
+    for (int j = 0; j < r.ntiles; ++j, ++it, key += kTileKeys) {
+      const uint32_t acc = it & 1;
+      if (!mbar_wait(e.bar_tfull + 8 * acc, (it >> 1) & 1)) return false;
+      tc_fence_after();
+      float sum = 0.f;
+      if constexpr (NC > 0) {
+        uint32_t v[NC];
+        load_epi_cols<NC>(e.t_lane + acc * kAccStride + c0, v);
+        tc_fence_before();
+        mbar_arrive(e.bar_tempty + 8 * acc);
+        sum = sum_exp2<NC, true>(v, c2, lw, 0.f);
+      } else {
+        tc_fence_before();
+        mbar_arrive(e.bar_tempty + 8 * acc);
+      }
+      // groups 1..3 hand their sums to group 0, which adds them in a fixed order
+      if (e.wg > 0) {
+        if (it >= 2 && !mbar_wait(e.bar_xb + 8 * acc, ((it >> 1) - 1) & 1)) return false;
+        part[(acc * 3 + (e.wg - 1)) * 128 + e.row] = sum;
+        mbar_arrive(e.bar_xa + 8 * acc);
+      } else {
+        if (!mbar_wait(e.bar_xa + 8 * acc, (it >> 1) & 1)) return false;
+        const float tot = ((sum + part[(acc * 3 + 0) * 128 + e.row]) + part[(acc * 3 + 1) * 128 + e.row]) +
+                          part[(acc * 3 + 2) * 128 + e.row];
+        mbar_arrive(e.bar_xb + 8 * acc);
+        if (key < a.S) out[key] = tot;
+      }
     }
-    // groups 1..3 hand their sums to group 0, which adds them in a fixed order
-    if (e.wg > 0) {
-      if (it >= 2 && !mbar_wait(e.bar_xb + 8 * acc, (uint32_t)((it >> 1) - 1) & 1)) return false;
-      part[(acc * 3 + (e.wg - 1)) * 128 + e.row] = sum;
-      mbar_arrive(e.bar_xa + 8 * acc);
-    } else {
-      if (!mbar_wait(e.bar_xa + 8 * acc, (uint32_t)(it >> 1) & 1)) return false;
-      const float tot = ((sum + part[(acc * 3 + 0) * 128 + e.row]) + part[(acc * 3 + 1) * 128 + e.row]) +
-                        part[(acc * 3 + 2) * 128 + e.row];
-      mbar_arrive(e.bar_xb + 8 * acc);
-      const int key = c.tib * kTileKeys + e.row;
-      if (key < a.S) a.s_exact[(size_t)c.seg * a.S + key] = tot;
-    }
-    new_seg = cursor_last_of_segment(c, a);
-    if (x + 1 < e.x_end && cursor_last_of_group(c, a)) mbar_arrive(e.bar_stat_free);
-    cursor_advance(c, a);
+    x += r.ntiles;
+    if (r.ends_group && x < e.x_end) mbar_arrive(e.bar_stat_free);
   }
   return true;
 }
@@ -406,33 +427,35 @@ __device__ __forceinline__ bool score_epilogue(const StreamArgs& a, const EpiCtx
 template <int KBITS, int TC>
 __device__ __forceinline__ bool proj_epilogue(const StreamArgs& a, const EpiCtx& e) {
   constexpr int TQ = TC / kEpiGroups;
+  constexpr uint32_t NACC = proj_num_acc(KBITS, TC), STRIDE = proj_acc_stride(KBITS, TC);
   bool new_group = true;
-  int gen = 0;
-  TileCursor c = cursor_at(e.x_begin, a);
-  long long it = 0;
-  for (long long x = e.x_begin; x < e.x_end; ++x, ++it) {
+  uint32_t gen = 0, acc = 0, acc_phase = 0;
+  for (long long x = e.x_begin; x < e.x_end;) {
+    const TileRun r = run_at(x, e.x_end, a);
     if (new_group) {
       // histogram slice landed (async-proxy writes are visible after the wait)
-      if (!mbar_wait(e.bar_stat, (uint32_t)gen & 1)) return false;
+      if (!mbar_wait(e.bar_stat, gen & 1)) return false;
       ++gen;
     }
-    const int acc = (int)(it & 1);
-    if (!mbar_wait(e.bar_tfull + 8 * acc, (uint32_t)(it >> 1) & 1)) return false;
-    tc_fence_after();
-    const int key = c.tib * kTileKeys + e.row;
-    const bool valid = key < a.S;
-    const uint32_t t_acc = e.t_lane + acc * kAccStride;
-    const uint32_t bar_rel = e.bar_tempty + 8 * acc;
-    const int table0 = c.chunk * TC;
-    uint32_t partial;
-    if (e.wg == 0) partial = proj_tables<KBITS, 0, TQ>(t_acc, bar_rel, e.hist_s, a, c.seg, key, table0, valid);
-    else if (e.wg == 1) partial = proj_tables<KBITS, TQ, 2 * TQ>(t_acc, bar_rel, e.hist_s, a, c.seg, key, table0, valid);
-    else if (e.wg == 2) partial = proj_tables<KBITS, 2 * TQ, 3 * TQ>(t_acc, bar_rel, e.hist_s, a, c.seg, key, table0, valid);
-    else partial = proj_tables<KBITS, 3 * TQ, 4 * TQ>(t_acc, bar_rel, e.hist_s, a, c.seg, key, table0, valid);
-    if (valid) atomicAdd(a.counts + (size_t)c.seg * a.S + key, partial);
-    new_group = cursor_last_of_group(c, a);
-    if (new_group && x + 1 < e.x_end) mbar_arrive(e.bar_stat_free);
-    cursor_advance(c, a);
+    uint32_t* cnt = a.counts + (size_t)r.c.seg * a.S;
+    const int table0 = r.c.chunk * TC;
+    int key = r.c.tib * kTileKeys + e.row;
+    for (int j = 0; j < r.ntiles; ++j, key += kTileKeys) {
+      if (!mbar_wait_spin(e.bar_tfull + 8 * acc, acc_phase)) return false;
+      tc_fence_after();
+      const bool valid = key < a.S;
+      const uint32_t t_acc = e.t_lane + acc * STRIDE, bar_rel = e.bar_tempty + 8 * acc;
+      uint32_t partial;
+      if (e.wg == 0) partial = proj_tables<KBITS, 0, TQ>(t_acc, bar_rel, e.hist_s, a, r.c.seg, key, table0, valid);
+      else if (e.wg == 1) partial = proj_tables<KBITS, TQ, 2 * TQ>(t_acc, bar_rel, e.hist_s, a, r.c.seg, key, table0, valid);
+      else if (e.wg == 2) partial = proj_tables<KBITS, 2 * TQ, 3 * TQ>(t_acc, bar_rel, e.hist_s, a, r.c.seg, key, table0, valid);
+      else partial = proj_tables<KBITS, 3 * TQ, 4 * TQ>(t_acc, bar_rel, e.hist_s, a, r.c.seg, key, table0, valid);
+      if (valid) atomicAdd(cnt + key, partial);
+      if (++acc == NACC) { acc = 0; acc_phase ^= 1; }
+    }
+    x += r.ntiles;
+    new_group = r.ends_group;
+    if (new_group && x < e.x_end) mbar_arrive(e.bar_stat_free);
   }
   return true;
 }
@@ -474,9 +497,9 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
   const uint32_t sm_tmem_slot = cur + 192;
   const uint32_t bar_full = sm_bars;                   // kStages barriers: tile landed
   const uint32_t bar_empty = sm_bars + 8 * kStages;    // kStages barriers: tile consumed by the MMAs
-  const uint32_t bar_tfull = sm_bars + 16 * kStages;   // 2: accumulator complete
-  const uint32_t bar_tempty = bar_tfull + 16;          // 2: accumulator copied out by all epilogue threads
-  const uint32_t bar_stat = bar_tempty + 16;           // stationary operand landed
+  const uint32_t bar_tfull = sm_bars + 16 * kStages;   // kMaxAcc: accumulator complete
+  const uint32_t bar_tempty = bar_tfull + 8 * kMaxAcc; // kMaxAcc: accumulator copied out by all epilogue threads
+  const uint32_t bar_stat = bar_tempty + 8 * kMaxAcc;  // stationary operand landed
   const uint32_t bar_stat_free = bar_stat + 8;         // stationary operand no longer in use
   const uint32_t bar_xa = bar_stat_free + 8;           // 2: mode-specific hand-off, "data written"
   const uint32_t bar_xb = bar_xa + 16;                 // 2: mode-specific hand-off, "data consumed"
@@ -489,7 +512,7 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
-    for (int s = 0; s < 2; ++s) { mbar_init(bar_tfull + 8 * s, 1); mbar_init(bar_tempty + 8 * s, kEpilogueThreads); }
+    for (int s = 0; s < kMaxAcc; ++s) { mbar_init(bar_tfull + 8 * s, 1); mbar_init(bar_tempty + 8 * s, kEpilogueThreads); }
     mbar_init(bar_stat, 1);
     mbar_init(bar_stat_free, kEpilogueThreads);
     if (MODE == kLse) {
@@ -565,6 +588,9 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
       bool ok = true;
       const uint32_t idesc = (MODE == kLse) ? umma_idesc_bf16(128, kTileKeys)
                                             : umma_idesc_bf16(128, a.stat_rows);
+      constexpr uint32_t NACC = (MODE == kProj) ? proj_num_acc(KBITS, TC) : 2;
+      constexpr uint32_t ACC_STRIDE = (MODE == kProj) ? proj_acc_stride(KBITS, TC) : kAccStride;
+      uint32_t acc = 0, acc_phase = 0;
       const uint32_t stat_lo = umma_sdesc_lo(sm_stat);
       const uint32_t stat_atom_lo = stat_atom_bytes >> 4;
       TileCursor c = cursor_at(x_begin, a);
@@ -573,18 +599,17 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
       long long it = 0;
       for (long long x = x_begin; x < x_end; ++x, ++it) {
         if (new_group) {
-          ok = mbar_wait(bar_stat, (uint32_t)gen & 1);
+          ok = mbar_wait_spin(bar_stat, (uint32_t)gen & 1);
           if (!ok) break;
           ++gen;
         }
         const int s = (int)(it % kStages);
-        const int acc = (int)(it & 1);
-        if (it >= 2) ok = mbar_wait(bar_tempty + 8 * acc, (uint32_t)((it >> 1) - 1) & 1);
-        if (ok) ok = mbar_wait(bar_full + 8 * s, (uint32_t)(it / kStages) & 1);
+        if (it >= NACC) ok = mbar_wait_spin(bar_tempty + 8 * acc, acc_phase ^ 1);
+        if (ok) ok = mbar_wait_spin(bar_full + 8 * s, (uint32_t)(it / kStages) & 1);
         if (!ok) break;
         tc_fence_after();
         const uint32_t tile_lo = umma_sdesc_lo(sm_stages + s * kTileBytes);
-        const uint32_t d0 = tmem_base + acc * kAccStride;
+        const uint32_t d0 = tmem_base + acc * ACC_STRIDE;
         if (elect_one()) {
 #pragma unroll
           for (int mb = 0; mb < 2; ++mb) {
@@ -602,6 +627,7 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
           umma_commit(bar_tfull + 8 * acc);   // accumulator ready for the epilogue
         }
         __syncwarp();
+        if (++acc == NACC) { acc = 0; acc_phase ^= 1; }
         new_group = cursor_last_of_group(c, a);
         cursor_advance(c, a);
       }
