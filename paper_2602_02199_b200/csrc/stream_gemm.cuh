@@ -184,25 +184,30 @@ __device__ __forceinline__ float sum_exp2(const uint32_t* v, float c2, const flo
   return (acc0.x + acc0.y) + (acc1.x + acc1.y);
 }
 
-// Tables [T_BEGIN, T_END) of the chunk for the calling thread's key: packs the sign bits of each
-// table's K projections into a bucket code, looks the code up in the histogram slice and
-// returns the summed collisions. A table whose smallest |projection| is below 2^-15 of the
-// largest |projection| among the key's first 16 hyperplanes of the chunk is queued for an exact
-// recomputation of its signs. All of the thread's columns are read into registers first and the
-// accumulator buffer is handed back to the MMA warp (arrive on `bar_release`) before the
-// arithmetic starts; the per-table work is branch-free so that the tables interleave.
-template <int KBITS, int T_BEGIN, int T_END>
+// NT consecutive tables of the chunk, starting at table `t_begin` (a multiple of NT), for the
+// calling thread's key: packs the sign bits of each table's K projections into a bucket code,
+// looks the code up in the histogram slice and returns the summed collisions. A table whose
+// smallest |projection| is below 2^-15 of the largest |projection| among the key's first 16
+// hyperplanes of the chunk is queued for an exact recomputation of its signs. All of the thread's
+// columns are read into registers first and the accumulator buffer is handed back to the MMA warp
+// (arrive on `bar_release`) before the arithmetic starts; the per-table work is branch-free so
+// that the tables interleave. `t_begin` is a run-time value so that the four epilogue groups
+// share one copy of this code.
+template <int KBITS, int NT>
 __device__ __forceinline__ uint32_t proj_tables(uint32_t t_acc, uint32_t bar_release, const uint16_t* hist_s,
-                                                const StreamArgs& a, int seg, int key, int table0, bool valid) {
-  constexpr int NT = T_END - T_BEGIN;
-  constexpr int CB = T_BEGIN * KBITS, CE = T_END * KBITS;
+                                                const StreamArgs& a, int seg, int key, int table0, int t_begin,
+                                                bool valid) {
+  constexpr int NC = NT * KBITS;                               // columns of this thread
+  constexpr int LD = (NC & -NC) < 32 ? (NC & -NC) : 32;        // load width: a power of two that divides NC
   constexpr uint32_t bucket_mask = (1u << KBITS) - 1u;
-  uint32_t v[CE - CB];
+  uint32_t v[NC];
   uint32_t v16[16];
-  tmem_ld_range<CB, CE>(t_acc, v);
+  const uint32_t t_col = t_acc + t_begin * KBITS;
+#pragma unroll
+  for (int j = 0; j < NC / LD; ++j) tmem_ld_cols<LD>(t_col + j * LD, v + j * LD);
   tmem_ld_x16(t_acc, v16);
   tmem_wait_ld();
-  reg_fence<CE - CB>(v);
+  reg_fence<NC>(v);
   reg_fence<16>(v16);
   tc_fence_before();
   mbar_arrive(bar_release);
@@ -226,17 +231,18 @@ __device__ __forceinline__ uint32_t proj_tables(uint32_t t_acc, uint32_t bar_rel
     code[t] = (~neg) & bucket_mask;
     amin[t] = mn;
   }
+  const uint16_t* hist_g = hist_s + ((uint32_t)t_begin << KBITS);
   uint32_t partial = 0;
   float lowest = INFINITY;
 #pragma unroll
   for (int t = 0; t < NT; ++t) {
-    partial += hist_s[((uint32_t)(T_BEGIN + t) << KBITS) + code[t]];
+    partial += hist_g[((uint32_t)t << KBITS) + code[t]];
     lowest = fminf(lowest, amin[t]);
   }
   if (valid && (a.key_buckets != nullptr || !(lowest >= tau))) {
 #pragma unroll
     for (int t = 0; t < NT; ++t) {
-      const int r = table0 + T_BEGIN + t;
+      const int r = table0 + t_begin + t;
       if (a.key_buckets) a.key_buckets[((size_t)seg * a.S + key) * a.lsh_tables + r] = (uint16_t)code[t];
       if (!(amin[t] >= tau)) {
         uint32_t doubt = 0;                                // code bits whose projection is below tau
@@ -444,12 +450,8 @@ __device__ __forceinline__ bool proj_epilogue(const StreamArgs& a, const EpiCtx&
       if (!mbar_wait_spin(e.bar_tfull + 8 * acc, acc_phase)) return false;
       tc_fence_after();
       const bool valid = key < a.S;
-      const uint32_t t_acc = e.t_lane + acc * STRIDE, bar_rel = e.bar_tempty + 8 * acc;
-      uint32_t partial;
-      if (e.wg == 0) partial = proj_tables<KBITS, 0, TQ>(t_acc, bar_rel, e.hist_s, a, r.c.seg, key, table0, valid);
-      else if (e.wg == 1) partial = proj_tables<KBITS, TQ, 2 * TQ>(t_acc, bar_rel, e.hist_s, a, r.c.seg, key, table0, valid);
-      else if (e.wg == 2) partial = proj_tables<KBITS, 2 * TQ, 3 * TQ>(t_acc, bar_rel, e.hist_s, a, r.c.seg, key, table0, valid);
-      else partial = proj_tables<KBITS, 3 * TQ, 4 * TQ>(t_acc, bar_rel, e.hist_s, a, r.c.seg, key, table0, valid);
+      const uint32_t partial = proj_tables<KBITS, TQ>(e.t_lane + acc * STRIDE, e.bar_tempty + 8 * acc, e.hist_s, a,
+                                                      r.c.seg, key, table0, e.wg * TQ, valid);
       if (valid) atomicAdd(cnt + key, partial);
       if (++acc == NACC) { acc = 0; acc_phase ^= 1; }
     }
