@@ -35,9 +35,15 @@ from paper_2602_02199_b200 import synth  # noqa: E402
 METRIC = "kv_tokens_scored_and_compacted_per_s_per_layer"
 UNIT = "tokens/s"
 
-# DRAM bytes (read + write) of one launch of the dominant kernel from an ncu capture, keyed by
-# workload; see profiles/. None = not captured for this workload.
-NCU_TRAFFIC_BYTES = {}
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch, from the ncu capture
+# summarised in profiles/select_call_llama8b_128k.md, keyed by (workload, kernel). A missing key
+# means: not captured for this workload, or the kernel has changed since the capture.
+NCU_TRAFFIC_BYTES = {
+    ("llama8b_128k", "stream_kernel<proj>"): 274773760 + 7303680,
+    ("llama8b_128k", "stream_kernel<lse>"): 269266688 + 3940096,
+    ("llama8b_128k", "stream_kernel<score>"): 270398208 + 7105536,
+    ("llama8b_128k", "append_kernel"): 254747648 + 200837632,
+}
 
 
 def load_peaks():
@@ -306,14 +312,14 @@ def run_ours(args, w, rank, world, local_rank):
     if dom in fl:
         achieved = fl[dom] / (dom_ms * 1e-3) / 1e12
         roof = {"kernel": dom, "bound": "tensor", "achieved": achieved, "peak": peaks["tf"], "unit": "TFLOP/s",
-                "frac": achieved / peaks["tf"], "traffic": NCU_TRAFFIC_BYTES.get(w.name),
+                "frac": achieved / peaks["tf"], "traffic": NCU_TRAFFIC_BYTES.get((w.name, dom)),
                 "peak_source": f"bf16_tflops (burst), {peaks['source']}",
                 "flops_per_launch": fl[dom], "ms_per_launch": dom_ms}
     else:
         gb = work["gather_bytes"] if dom == "append_kernel" else work["bytes"]
         achieved = gb / (dom_ms * 1e-3) / 1e9
         roof = {"kernel": dom, "bound": "hbm", "achieved": achieved, "peak": peaks["hbm"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm"], "traffic": NCU_TRAFFIC_BYTES.get(w.name),
+                "frac": achieved / peaks["hbm"], "traffic": NCU_TRAFFIC_BYTES.get((w.name, dom)),
                 "peak_source": f"hbm_gbs, {peaks['source']}", "bytes_per_launch": gb, "ms_per_launch": dom_ms}
     t_hbm = work["bytes"] / (peaks["hbm"] * 1e9)
     t_tensor = work["flops"] / (peaks["tf"] * 1e12)
