@@ -19,9 +19,11 @@
 //            a projection that is tiny relative to the key's other projections are queued for
 //            an exact recomputation.
 //
-// Warp roles (576 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner,
-// warps 2..17 = four epilogue groups of four warps (TMEM lane quarter = warp_id % 4) that split
-// the accumulator columns of every tile. An epilogue thread copies its columns to registers,
+// Warp roles (608 threads): warp 0 = TMA producer, warps 1 and 2 = MMA issuers (warp 1 also owns
+// the TMEM allocation), warps 3..18 = four epilogue groups of four warps (TMEM lane quarter =
+// warp_id % 4) that split the accumulator columns of every tile. The tensor pipe runs only while
+// an issuing thread feeds it (it queues next to nothing), so the two MMA warps take alternate
+// tiles: the waits, fences and commits of one overlap the MMAs of the other. An epilogue thread copies its columns to registers,
 // hands the accumulator buffer back to the MMA warp and only then does its arithmetic.
 // All cross-warp hand-offs are mbarriers with bounded waits; there is no CTA-wide barrier
 // inside the tile loop.
@@ -37,7 +39,8 @@ constexpr int kTileBytes = 2 * kTileAtomBytes;   // 128 keys x 128 dims bf16
 constexpr int kStages = 4;
 constexpr int kEpiGroups = 4;
 constexpr int kEpilogueThreads = kEpiGroups * 128;
-constexpr int kStreamThreads = 64 + kEpilogueThreads;
+constexpr int kMmaWarps = 2;
+constexpr int kStreamThreads = 32 * (1 + kMmaWarps) + kEpilogueThreads;
 constexpr int kEpiCols = 64;                   // accumulator columns an epilogue thread holds at most
 constexpr int kXchBytes = 8192;                // exchange area between epilogue warps
 constexpr int kTmemCols = 512;
@@ -51,7 +54,7 @@ __host__ __device__ constexpr int proj_num_acc(int kbits, int tc) {
 }
 constexpr int kMaxStatRows = 256;
 constexpr int kMaxStreamCtas = 256;            // upper bound of the persistent grid (slot arithmetic)
-constexpr int kPolyPairsOf32 = 12;             // of every 32 column pairs, this many take 2^x on the FMA pipe
+constexpr int kPolyPairsOf32 = 10;             // of every 32 column pairs, this many take 2^x on the FMA pipe
 
 enum StreamMode { kLse = 0, kScore = 1, kProj = 2 };
 
@@ -582,54 +585,56 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
       }
     }
     __syncwarp();
-  } else if (warp == 1) {
-    // ================= MMA issuer =================
-    // The whole warp walks the loop (uniform waits and address arithmetic); one elected lane
-    // issues the MMAs and their commits.
+  } else if (warp <= kMmaWarps) {
+    // ================= MMA issuers =================
+    // Both warps walk the whole slice (uniform waits and address arithmetic) and issue alternate
+    // tiles; within a warp one elected lane issues the MMAs and their commits.
     if (x_begin < x_end) {
       bool ok = true;
+      const uint32_t mine = (uint32_t)(warp - 1);
       const uint32_t idesc = (MODE == kLse) ? umma_idesc_bf16(128, kTileKeys)
                                             : umma_idesc_bf16(128, a.stat_rows);
       constexpr uint32_t NACC = (MODE == kProj) ? proj_num_acc(KBITS, TC) : 2;
       constexpr uint32_t ACC_STRIDE = (MODE == kProj) ? proj_acc_stride(KBITS, TC) : kAccStride;
-      uint32_t acc = 0, acc_phase = 0;
       const uint32_t stat_lo = umma_sdesc_lo(sm_stat);
       const uint32_t stat_atom_lo = stat_atom_bytes >> 4;
       TileCursor c = cursor_at(x_begin, a);
-      bool new_group = true;
-      int gen = 0;
-      long long it = 0;
+      bool new_group = true, need_stat = false;
+      uint32_t gen = 0, it = 0;
       for (long long x = x_begin; x < x_end; ++x, ++it) {
-        if (new_group) {
-          ok = mbar_wait_spin(bar_stat, (uint32_t)gen & 1);
+        if (new_group) { ++gen; need_stat = true; }   // stationary operand number `gen` serves this tile
+        if (it % kMmaWarps == mine) {
+          if (need_stat) {
+            ok = mbar_wait_spin(bar_stat, (gen - 1) & 1);
+            if (!ok) break;
+            need_stat = false;
+          }
+          const uint32_t s = it % kStages;
+          const uint32_t acc = it % NACC, use = it / NACC;
+          if (use > 0) ok = mbar_wait_spin(bar_tempty + 8 * acc, (use - 1) & 1);
+          if (ok) ok = mbar_wait_spin(bar_full + 8 * s, (it / kStages) & 1);
           if (!ok) break;
-          ++gen;
-        }
-        const int s = (int)(it % kStages);
-        if (it >= NACC) ok = mbar_wait_spin(bar_tempty + 8 * acc, acc_phase ^ 1);
-        if (ok) ok = mbar_wait_spin(bar_full + 8 * s, (uint32_t)(it / kStages) & 1);
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t tile_lo = umma_sdesc_lo(sm_stages + s * kTileBytes);
-        const uint32_t d0 = tmem_base + acc * ACC_STRIDE;
-        if (elect_one()) {
+          tc_fence_after();
+          const uint32_t tile_lo = umma_sdesc_lo(sm_stages + s * kTileBytes);
+          const uint32_t d0 = tmem_base + acc * ACC_STRIDE;
+          if (elect_one()) {
 #pragma unroll
-          for (int mb = 0; mb < 2; ++mb) {
-            if (mb < nmb) {
+            for (int mb = 0; mb < 2; ++mb) {
+              if (mb < nmb) {
 #pragma unroll
-              for (int k = 0; k < 8; ++k) {
-                const uint32_t tile_k = tile_lo + (k >> 2) * (kTileAtomBytes >> 4) + (k & 3) * 2;
-                const uint32_t stat_k = stat_lo + (k >> 2) * stat_atom_lo + (k & 3) * 2 + mb * ((128 * 128) >> 4);
-                if (MODE == kLse) umma_bf16_lo(d0 + mb * 128, stat_k, tile_k, idesc, k > 0);
-                else umma_bf16_lo(d0, tile_k, stat_k, idesc, k > 0);
+                for (int k = 0; k < 8; ++k) {
+                  const uint32_t tile_k = tile_lo + (k >> 2) * (kTileAtomBytes >> 4) + (k & 3) * 2;
+                  const uint32_t stat_k = stat_lo + (k >> 2) * stat_atom_lo + (k & 3) * 2 + mb * ((128 * 128) >> 4);
+                  if (MODE == kLse) umma_bf16_lo(d0 + mb * 128, stat_k, tile_k, idesc, k > 0);
+                  else umma_bf16_lo(d0, tile_k, stat_k, idesc, k > 0);
+                }
               }
             }
+            umma_commit(bar_empty + 8 * s);     // stage reusable once these MMAs have read it
+            umma_commit(bar_tfull + 8 * acc);   // accumulator ready for the epilogue
           }
-          umma_commit(bar_empty + 8 * s);     // stage reusable once these MMAs have read it
-          umma_commit(bar_tfull + 8 * acc);   // accumulator ready for the epilogue
+          __syncwarp();
         }
-        __syncwarp();
-        if (++acc == NACC) { acc = 0; acc_phase ^= 1; }
         new_group = cursor_last_of_group(c, a);
         cursor_advance(c, a);
       }
@@ -645,7 +650,7 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
     e.lane = lane;
     e.row = e.quarter * 32 + lane;
     e.t_lane = tmem_base + ((uint32_t)(e.quarter * 32) << 16);
-    e.ewarp = warp - 2;
+    e.ewarp = warp - 1 - kMmaWarps;
     e.wg = e.ewarp >> 2;
     e.x_begin = x_begin;
     e.x_end = x_end;
