@@ -17,6 +17,7 @@
 #include "../../include/laser_kv.h"
 #include "aux_kernels.cuh"
 #include "stream_gemm.cuh"
+#include "query_proj.cuh"
 
 namespace {
 
@@ -27,7 +28,7 @@ constexpr size_t kAlign = 256;
 constexpr int kMaxSmem = 227 * 1024;
 
 constexpr int kProfKernels = 7;
-const char* const kProfNames[kProfKernels] = {"qprep_kernel", "stream_kernel<lse>", "stream_kernel<score>",
+const char* const kProfNames[kProfKernels] = {"qsig_kernel", "stream_kernel<lse>", "stream_kernel<score>",
                                               "stream_kernel<proj>", "signfix_kernel", "select_kernel", "append_kernel"};
 
 std::atomic<long long> g_launches{0};
@@ -66,7 +67,8 @@ struct laser_kv_ctx {
   uint16_t* cacheV = nullptr;
   int32_t* cachePos = nullptr;
   const uint16_t* P = nullptr;
-  CUtensorMap mapP;
+  CUtensorMap mapP;    // hyperplanes, box = one chunk of the projection pass
+  CUtensorMap mapPq;   // hyperplanes, box = the eight tables of one query-signature CTA
   EncodeTiledFn encode = nullptr;
   int num_sms = 1;
   std::vector<long long> blocks_done;   // per layer
@@ -253,6 +255,32 @@ cudaError_t launch_proj(int K, int TCv, const CUtensorMap& mk, const CUtensorMap
   return cudaErrorInvalidValue;
 }
 
+template <int KB>
+cudaError_t launch_qsig_t(const CUtensorMap& mq, const CUtensorMap& mp, const QsigArgs& a, dim3 grid, uint32_t smem,
+                          cudaStream_t st) {
+  static bool attr_done = false;   // per instantiation; the attribute is per device function
+  if (!attr_done) {
+    const cudaError_t e = cudaFuncSetAttribute(qsig_kernel<KB>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+    if (e != cudaSuccess) return e;
+    attr_done = true;
+  }
+  qsig_kernel<KB><<<grid, kQsigThreads, smem, st>>>(mq, mp, a);
+  g_launches.fetch_add(1);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_qsig(int K, const CUtensorMap& mq, const CUtensorMap& mp, const QsigArgs& a, dim3 grid, uint32_t smem,
+                        cudaStream_t st) {
+  switch (K) {
+    case 4: return launch_qsig_t<4>(mq, mp, a, grid, smem, st);
+    case 6: return launch_qsig_t<6>(mq, mp, a, grid, smem, st);
+    case 8: return launch_qsig_t<8>(mq, mp, a, grid, smem, st);
+    case 10: return launch_qsig_t<10>(mq, mp, a, grid, smem, st);
+    case 12: return launch_qsig_t<12>(mq, mp, a, grid, smem, st);
+  }
+  return cudaErrorInvalidValue;
+}
+
 laser_kv_status_t launch_select(const float* s_exact, const uint32_t* counts, int n_seg, int S, int anchors,
                                 int k_exact, int k_lsh, int32_t* idx, cudaStream_t st) {
   static bool attr_done = false;
@@ -373,7 +401,8 @@ laser_kv_status_t laser_kv_init(const laser_kv_config_t* cfg, const void* hyperp
     const uint64_t dims[2] = {(uint64_t)kHeadDim, (uint64_t)cfg->lsh_tables * cfg->lsh_bits};
     const uint64_t strides[1] = {(uint64_t)kHeadDim * 2};
     const uint32_t box[2] = {(uint32_t)kAtomCols, (uint32_t)(d.TC * cfg->lsh_bits)};
-    if (!encode_map(h, &h->mapP, h->P, 2, dims, strides, box)) {
+    const uint32_t boxq[2] = {(uint32_t)kAtomCols, (uint32_t)(kQsigTables * cfg->lsh_bits)};
+    if (!encode_map(h, &h->mapP, h->P, 2, dims, strides, box) || !encode_map(h, &h->mapPq, h->P, 2, dims, strides, boxq)) {
       const std::string msg = h->last_error;
       delete h;
       return fail(nullptr, LASER_KV_ERR_CUDA, "%s", msg.c_str());
@@ -467,23 +496,15 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
     marks.push_back(ev);
   };
   mark();
-  // 1. query signatures and bucket histogram; also clears the counts and restarts the fix-up
-  //    counter (ctrl[1]) and the changed counter (ctrl[2]); the status word (ctrl[0]) is kept
+  // 1. query signatures and bucket histograms; the kernel also clears the counts and restarts the
+  //    fix-up counter (ctrl[1]) and the changed counter (ctrl[2]); the status word (ctrl[0]) is kept
   {
-    QprepArgs qa{static_cast<const uint16_t*>(Q_win), q_strides[0], q_strides[1], q_strides[2], h->P, hist, qb,
-                 c.n_kv_heads, d.G, c.window, d.GW, c.lsh_bits, c.lsh_tables,
-                 reinterpret_cast<uint4*>(counts), (long long)nseg * S / 4, ctrl + 1};
-    const size_t smem = qprep_smem_bytes(c.lsh_bits);
-    dim3 grid(c.lsh_tables, c.n_kv_heads, c.batch);
-    switch (c.lsh_bits) {
-      case 4: qprep_kernel<4><<<grid, kQprepThreads, smem, st>>>(qa); break;
-      case 6: qprep_kernel<6><<<grid, kQprepThreads, smem, st>>>(qa); break;
-      case 8: qprep_kernel<8><<<grid, kQprepThreads, smem, st>>>(qa); break;
-      case 10: qprep_kernel<10><<<grid, kQprepThreads, smem, st>>>(qa); break;
-      default: qprep_kernel<12><<<grid, kQprepThreads, smem, st>>>(qa); break;
-    }
-    g_launches.fetch_add(1);
-    LKV_CUDA(cudaGetLastError(), "qprep_kernel");
+    const int q_alloc = ((d.GW + 127) / 128) * 128;
+    QsigArgs qa{static_cast<const uint16_t*>(Q_win), q_strides[0], q_strides[1], q_strides[2], h->P, hist, qb,
+                c.n_kv_heads, d.G, c.window, d.GW, q_alloc, c.lsh_tables,
+                reinterpret_cast<uint4*>(counts), (long long)nseg * S / 4, ctrl + 1, ctrl};
+    dim3 grid(c.lsh_tables / kQsigTables, c.n_kv_heads, c.batch);
+    LKV_CUDA(launch_qsig(c.lsh_bits, mapQ, h->mapPq, qa, grid, qsig_smem_bytes(q_alloc, c.lsh_bits), st), "qsig_kernel");
   }
 
   StreamArgs sa;

@@ -1,7 +1,4 @@
 // The non-GEMM kernels of the selection path:
-//   qprep_kernel   - SimHash bucket codes of the window queries and the per-table histogram of
-//                    those codes (Section 3.3 "Recall"; Algorithm 1 line 6 counts collisions
-//                    against exactly these query buckets).
 //   signfix_kernel - exact recomputation of key sign bits whose tensor-core projection was too
 //                    close to zero to trust, with the matching correction of the counts.
 //   select_kernel  - Algorithm 1 lines 4-8: two-stage top-k per (sequence, KV head, block) by
@@ -15,101 +12,6 @@ namespace lkv {
 
 __device__ __forceinline__ double bf16_to_f64(uint16_t b) {
   return static_cast<double>(__uint_as_float(static_cast<uint32_t>(b) << 16));
-}
-
-// ------------------------------------------------------------------------------------------------
-// Query side: one CTA per (table r, KV head h, sequence b); a thread handles window queries q and
-// q + 128 of the head's group. Projections are accumulated in fp64 (products of two bf16 are exact
-// in fp64), so query sign bits need no guard. Every query element is widened to fp64 once and
-// feeds the K accumulators of the table; the plane values come from shared memory as 16-byte
-// broadcasts shared by both queries. Bucket code: hyperplane r*K + b0 sits at bit K-1-b0.
-// ------------------------------------------------------------------------------------------------
-struct QprepArgs {
-  const uint16_t* Q;      // [batch][H_q][W][d] via strides
-  long long qs_b, qs_h, qs_w;
-  const uint16_t* P;      // [L*K][128]
-  uint16_t* hist;         // [batch][H_kv][L][2^K]
-  uint16_t* qbuckets;     // [batch][H_kv][GW][L]
-  int H_kv, G, W, GW, K, L;
-  uint4* zero_begin;      // the call's collision counts, cleared here (16-byte units)
-  long long zero_n;
-  int* counters;          // fix-up and changed counters, restarted here
-};
-
-constexpr int kQprepThreads = 128;
-
-__host__ __device__ inline size_t qprep_smem_bytes(int K) { return (size_t)K * 128 * 8 + ((size_t)4 << K); }
-
-template <int K>
-__global__ void __launch_bounds__(kQprepThreads) qprep_kernel(const QprepArgs a) {
-  extern __shared__ __align__(16) uint8_t smem_q[];
-  double* planes = reinterpret_cast<double*>(smem_q);                          // [K][128]
-  uint32_t* bins = reinterpret_cast<uint32_t*>(smem_q + (size_t)K * 128 * 8);   // [2^K]
-  const int r = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
-  constexpr int nbins = 1 << K;
-  {
-    // this CTA's share of the count array; the projection pass accumulates into it later
-    const long long cta = ((long long)b * gridDim.y + h) * gridDim.x + r;
-    const long long nctas = (long long)gridDim.x * gridDim.y * gridDim.z;
-    const long long per = (a.zero_n + nctas - 1) / nctas;
-    const long long z0 = cta * per, z1 = min(a.zero_n, z0 + per);
-    for (long long i = z0 + threadIdx.x; i < z1; i += kQprepThreads) a.zero_begin[i] = make_uint4(0u, 0u, 0u, 0u);
-    if (cta == 0 && threadIdx.x < 2) a.counters[threadIdx.x] = 0;
-  }
-  for (int i = threadIdx.x; i < K * 128; i += kQprepThreads)
-    planes[i] = bf16_to_f64(a.P[(size_t)r * K * 128 + i]);
-  for (int i = threadIdx.x; i < nbins; i += kQprepThreads) bins[i] = 0;
-  __syncthreads();
-  for (int q0 = threadIdx.x; q0 < a.GW; q0 += 2 * kQprepThreads) {
-    const int q1 = q0 + kQprepThreads;
-    const bool two = q1 < a.GW;
-    const uint16_t* row0 = a.Q + b * a.qs_b + (long long)(h * a.G + q0 / a.W) * a.qs_h + (q0 % a.W) * a.qs_w;
-    const uint16_t* row1 = two ? a.Q + b * a.qs_b + (long long)(h * a.G + q1 / a.W) * a.qs_h + (q1 % a.W) * a.qs_w : row0;
-    double acc0[K], acc1[K];
-#pragma unroll
-    for (int bit = 0; bit < K; ++bit) { acc0[bit] = 0.0; acc1[bit] = 0.0; }
-    for (int c = 0; c < 128; c += 8) {
-      const uint4 v0 = *reinterpret_cast<const uint4*>(row0 + c);
-      const uint4 v1 = *reinterpret_cast<const uint4*>(row1 + c);
-      const uint32_t w0[4] = {v0.x, v0.y, v0.z, v0.w};
-      const uint32_t w1[4] = {v1.x, v1.y, v1.z, v1.w};
-      double x0[8], x1[8];
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        x0[2 * e] = bf16_to_f64((uint16_t)(w0[e] & 0xFFFF));
-        x0[2 * e + 1] = bf16_to_f64((uint16_t)(w0[e] >> 16));
-        x1[2 * e] = bf16_to_f64((uint16_t)(w1[e] & 0xFFFF));
-        x1[2 * e + 1] = bf16_to_f64((uint16_t)(w1[e] >> 16));
-      }
-#pragma unroll
-      for (int bit = 0; bit < K; ++bit) {
-        const double2* p = reinterpret_cast<const double2*>(planes + bit * 128 + c);
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const double2 pp = p[e];
-          acc0[bit] = fma(x0[2 * e], pp.x, acc0[bit]);
-          acc0[bit] = fma(x0[2 * e + 1], pp.y, acc0[bit]);
-          acc1[bit] = fma(x1[2 * e], pp.x, acc1[bit]);
-          acc1[bit] = fma(x1[2 * e + 1], pp.y, acc1[bit]);
-        }
-      }
-    }
-    uint32_t code0 = 0, code1 = 0;
-#pragma unroll
-    for (int bit = 0; bit < K; ++bit) {
-      code0 = (code0 << 1) | (acc0[bit] >= 0.0 ? 1u : 0u);
-      code1 = (code1 << 1) | (acc1[bit] >= 0.0 ? 1u : 0u);
-    }
-    atomicAdd(&bins[code0], 1u);
-    a.qbuckets[((size_t)(b * a.H_kv + h) * a.GW + q0) * a.L + r] = (uint16_t)code0;
-    if (two) {
-      atomicAdd(&bins[code1], 1u);
-      a.qbuckets[((size_t)(b * a.H_kv + h) * a.GW + q1) * a.L + r] = (uint16_t)code1;
-    }
-  }
-  __syncthreads();
-  uint16_t* out = a.hist + ((size_t)(b * a.H_kv + h) * a.L + r) * nbins;
-  for (int i = threadIdx.x; i < nbins; i += kQprepThreads) out[i] = (uint16_t)bins[i];
 }
 
 // ------------------------------------------------------------------------------------------------
