@@ -281,8 +281,10 @@ cudaError_t launch_qsig(int K, const CUtensorMap& mq, const CUtensorMap& mp, con
   return cudaErrorInvalidValue;
 }
 
+// `count_max` bounds every count (0 = no bound known): it lets the count stage skip radix passes
+// over bytes that are zero everywhere.
 laser_kv_status_t launch_select(const float* s_exact, const uint32_t* counts, int n_seg, int S, int anchors,
-                                int k_exact, int k_lsh, int32_t* idx, cudaStream_t st) {
+                                int k_exact, int k_lsh, uint32_t count_max, int32_t* idx, cudaStream_t st) {
   static bool attr_done = false;
   const size_t smem = (size_t)S * 9;
   if (!attr_done) {
@@ -290,7 +292,12 @@ laser_kv_status_t launch_select(const float* s_exact, const uint32_t* counts, in
       return fail(nullptr, LASER_KV_ERR_CUDA, "cudaFuncSetAttribute(select_kernel) failed");
     attr_done = true;
   }
-  SelectArgs a{s_exact, counts, idx, S, anchors, k_exact, k_lsh};
+  int top_shift = 24;
+  if (count_max != 0) {
+    top_shift = 0;
+    while (top_shift < 24 && (count_max >> (top_shift + 8)) != 0) top_shift += 8;
+  }
+  SelectArgs a{s_exact, counts, idx, S, anchors, k_exact, k_lsh, top_shift};
   select_kernel<<<n_seg, kSelThreads, smem, st>>>(a);
   g_launches.fetch_add(1);
   const cudaError_t e = cudaGetLastError();
@@ -563,7 +570,8 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
   mark();
   // 6. two-stage top-k
   {
-    const laser_kv_status_t s = launch_select(s_exact, counts, nseg, S, d.anchors, d.k_exact, d.k_lsh, idx, st);
+    const laser_kv_status_t s = launch_select(s_exact, counts, nseg, S, d.anchors, d.k_exact, d.k_lsh,
+                                                (uint32_t)d.GW * (uint32_t)c.lsh_tables, idx, st);
     if (s != LASER_KV_OK) { h->last_error = g_last_error; return s; }
   }
   mark();
@@ -756,7 +764,7 @@ laser_kv_status_t laser_kv_two_stage_topk(const float* s_exact, const uint32_t* 
     return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "two_stage_topk: keep count exceeds the segment");
   if (S > 16384) return fail(nullptr, LASER_KV_ERR_UNSUPPORTED, "two_stage_topk: S > 16384");
   if (2 * anchors + k_exact + k_lsh == 0) return LASER_KV_OK;
-  return launch_select(s_exact, counts, n_segments, S, anchors, k_exact, k_lsh, idx_out, static_cast<cudaStream_t>(stream));
+  return launch_select(s_exact, counts, n_segments, S, anchors, k_exact, k_lsh, 0u, idx_out, static_cast<cudaStream_t>(stream));
 }
 
 // ---- window scores on caller-fed inputs ----------------------------------------------------------

@@ -16,9 +16,9 @@ __device__ __forceinline__ double bf16_to_f64(uint16_t b) {
 
 // ------------------------------------------------------------------------------------------------
 // Exact recomputation of flagged key signs. An item names a key, a table, the provisional bucket
-// code and a mask of the code bits whose projection was too small to trust. One warp per item:
-// for every masked bit the 128-term dot product is formed in fp64 (exact bf16 products, four
-// terms per lane, warp reduction) and the bit is replaced by its exact sign. If the bucket code
+// code and a mask of the code bits whose projection was too small to trust. Eight lanes per item:
+// for every masked bit the 128-term dot product is formed in fp64 (exact bf16 products, sixteen
+// terms per lane, reduction over the eight lanes) and the bit is replaced by its exact sign. If the bucket code
 // changes, the key's count is corrected by hist[new] - hist[old].
 // ------------------------------------------------------------------------------------------------
 struct SignfixArgs {
@@ -35,14 +35,16 @@ struct SignfixArgs {
   int* n_changed;
 };
 
-constexpr int kSignfixCtas = 592;   // 4 CTAs of 8 warps per SM: a few items per warp at most
+constexpr int kSignfixCtas = 1184;   // 8 CTAs of 256 threads per SM: all resident, about one item per lane group
 
 __global__ void __launch_bounds__(256) signfix_kernel(const SignfixArgs a) {
   const int lane = threadIdx.x & 31;
-  const int wid = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  const int nwarps = (gridDim.x * blockDim.x) >> 5;
+  const int sl = lane & 7;                              // lane within the group of eight that shares an item
+  const uint32_t gmask = 0xFFu << (lane & 24);          // the group's lanes
+  const int gid = (blockIdx.x * blockDim.x + threadIdx.x) >> 3;
+  const int ngroups = (gridDim.x * blockDim.x) >> 3;
   const int n = min(*a.n_items, a.cap);
-  for (int it = wid; it < n; it += nwarps) {
+  for (int it = gid; it < n; it += ngroups) {
     const int4 item = a.items[it];
     const int seg = item.x, key = item.y, r = item.z;
     const uint32_t old_code = (uint32_t)item.w & 0xFFFFu;
@@ -50,25 +52,29 @@ __global__ void __launch_bounds__(256) signfix_kernel(const SignfixArgs a) {
     const int t = seg % a.nb;
     const int h = (seg / a.nb) % a.H_kv;
     const int b = seg / (a.nb * a.H_kv);
-    const uint16_t* krow = a.Kp + b * a.ks_b + h * a.ks_h + ((long long)t * a.S + key) * a.ks_t;
-    const uint2 kv = *reinterpret_cast<const uint2*>(krow + lane * 4);
-    const double k0 = bf16_to_f64((uint16_t)(kv.x & 0xFFFF)), k1 = bf16_to_f64((uint16_t)(kv.x >> 16));
-    const double k2 = bf16_to_f64((uint16_t)(kv.y & 0xFFFF)), k3 = bf16_to_f64((uint16_t)(kv.y >> 16));
+    // sixteen key elements per lane
+    const uint16_t* krow = a.Kp + b * a.ks_b + h * a.ks_h + ((long long)t * a.S + key) * a.ks_t + sl * 16;
+    const uint4 ka = *reinterpret_cast<const uint4*>(krow), kb = *reinterpret_cast<const uint4*>(krow + 8);
+    const uint32_t kw[8] = {ka.x, ka.y, ka.z, ka.w, kb.x, kb.y, kb.z, kb.w};
     uint32_t code = old_code;
     while (mask) {
       const int pos = 31 - __clz(mask);          // code bit; hyperplane r*K + (K-1-pos)
       mask &= ~(1u << pos);
-      const int bit = a.K - 1 - pos;
-      const uint2 pv = *reinterpret_cast<const uint2*>(a.P + ((size_t)r * a.K + bit) * 128 + lane * 4);
-      double acc = k0 * bf16_to_f64((uint16_t)(pv.x & 0xFFFF));
-      acc = fma(k1, bf16_to_f64((uint16_t)(pv.x >> 16)), acc);
-      acc = fma(k2, bf16_to_f64((uint16_t)(pv.y & 0xFFFF)), acc);
-      acc = fma(k3, bf16_to_f64((uint16_t)(pv.y >> 16)), acc);
+      const uint16_t* prow = a.P + ((size_t)r * a.K + (a.K - 1 - pos)) * 128 + sl * 16;
+      const uint4 pa = *reinterpret_cast<const uint4*>(prow), pb = *reinterpret_cast<const uint4*>(prow + 8);
+      const uint32_t pw[8] = {pa.x, pa.y, pa.z, pa.w, pb.x, pb.y, pb.z, pb.w};
+      double acc0 = 0.0, acc1 = 0.0;
 #pragma unroll
-      for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+      for (int e = 0; e < 8; ++e) {
+        acc0 = fma(bf16_to_f64((uint16_t)(kw[e] & 0xFFFF)), bf16_to_f64((uint16_t)(pw[e] & 0xFFFF)), acc0);
+        acc1 = fma(bf16_to_f64((uint16_t)(kw[e] >> 16)), bf16_to_f64((uint16_t)(pw[e] >> 16)), acc1);
+      }
+      double acc = acc0 + acc1;
+#pragma unroll
+      for (int off = 4; off > 0; off >>= 1) acc += __shfl_xor_sync(gmask, acc, off);
       code = (code & ~(1u << pos)) | ((acc >= 0.0 ? 1u : 0u) << pos);
     }
-    if (lane == 0 && code != old_code) {
+    if (sl == 0 && code != old_code) {
       const uint16_t* hr = a.hist + ((size_t)(b * a.H_kv + h) * a.L + r) * ((size_t)1 << a.K);
       const uint32_t delta = (uint32_t)hr[code] - (uint32_t)hr[old_code];
       atomicAdd(a.counts + (size_t)seg * a.S + key, delta);
@@ -119,11 +125,13 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums, int& 
 
 // Among the participating elements j in [lo, hi) (flag[j] == 0) finds the k-th largest value T
 // (k >= 1, k <= number of participants) and how many elements equal to T belong to the top k.
-__device__ void radix_select_kth(const uint32_t* vals, const uint8_t* flag, int lo, int hi, int k,
+// `top_shift` is the position of the highest byte that can differ between values (24 for arbitrary
+// 32-bit keys); the bytes above it must be zero in every value.
+__device__ void radix_select_kth(const uint32_t* vals, const uint8_t* flag, int lo, int hi, int k, int top_shift,
                                  int* hist, int* misc, uint32_t& T, int& need) {
-  uint32_t prefix = 0, mask = 0;
+  uint32_t prefix = 0, mask = ~((top_shift >= 24) ? 0xFFFFFFFFu : ((1u << (top_shift + 8)) - 1u));
   int remaining = k;
-  for (int shift = 24; shift >= 0; shift -= 8) {
+  for (int shift = top_shift; shift >= 0; shift -= 8) {
     for (int i = threadIdx.x; i < 256; i += kSelThreads) hist[i] = 0;
     __syncthreads();
     for (int j = lo + threadIdx.x; j < hi; j += kSelThreads) {
@@ -165,12 +173,12 @@ __device__ void radix_select_kth(const uint32_t* vals, const uint8_t* flag, int 
 }
 
 // Marks (flag = 1) the k largest participating elements of [lo, hi); equal values: lower index.
-__device__ void mark_topk(const uint32_t* vals, uint8_t* flag, int lo, int hi, int k, int* hist,
+__device__ void mark_topk(const uint32_t* vals, uint8_t* flag, int lo, int hi, int k, int top_shift, int* hist,
                           int* misc, int* warp_sums) {
   if (k <= 0) return;                    // uniform across the CTA
   uint32_t T;
   int need;
-  radix_select_kth(vals, flag, lo, hi, k, hist, misc, T, need);
+  radix_select_kth(vals, flag, lo, hi, k, top_shift, hist, misc, T, need);
   const int n = hi - lo;
   const int per = (n + kSelThreads - 1) / kSelThreads;
   const int j0 = lo + threadIdx.x * per;
@@ -193,6 +201,7 @@ struct SelectArgs {
   const uint32_t* counts;   // [n_seg][S]
   int32_t* idx;             // [n_seg][B]
   int S, anchors, k_exact, k_lsh;
+  int count_top_shift;      // highest byte position (0, 8, 16 or 24) in which two counts can differ
 };
 
 __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectArgs a) {
@@ -212,8 +221,8 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectArgs
     flag[j] = (j < lo || j >= hi) ? 1 : 0;
   }
   __syncthreads();
-  mark_topk(ukey, flag, lo, hi, a.k_exact, hist, misc, warp_sums);   // K_exact
-  mark_topk(ucnt, flag, lo, hi, a.k_lsh, hist, misc, warp_sums);     // K_lsh from the residual
+  mark_topk(ukey, flag, lo, hi, a.k_exact, 24, hist, misc, warp_sums);            // K_exact
+  mark_topk(ucnt, flag, lo, hi, a.k_lsh, a.count_top_shift, hist, misc, warp_sums);  // K_lsh from the residual
   // ordered compaction of all kept indices
   const int per = (S + kSelThreads - 1) / kSelThreads;
   const int j0 = threadIdx.x * per, j1 = min(S, j0 + per);
