@@ -42,6 +42,22 @@ def test_gqa7_k10_shape_with_rope_and_batch():
     check_run(w, run)
 
 
+@pytest.mark.parametrize("K,L,hq,hkv,W,S", [
+    (4, 8, 2, 2, 16, 264),       # G*W = 16: three of the four score groups have no columns
+    (6, 24, 4, 2, 24, 392),      # G*W = 48, 6-bit tables, 24 tables in chunks of 8
+    (12, 8, 8, 2, 64, 520),      # G*W = 256, 12-bit tables, one chunk
+    (12, 16, 4, 4, 32, 136),     # 12-bit tables in one chunk of 16: two accumulator buffers of 192 columns
+    (8, 32, 6, 2, 48, 648),      # G*W = 144: two query row blocks, the second one ragged; chunk of 32 tables
+    (10, 8, 16, 2, 16, 1032),    # G = 8, W = 16
+])
+def test_hash_and_group_geometries(K, L, hq, hkv, W, S):
+    w = synth.workload("tiny").with_(name=f"geo{K}_{L}_{hq}_{hkv}_{W}", n_q_heads=hq, n_kv_heads=hkv, window=W,
+                                     lsh_bits=K, lsh_tables=L, block_size=S, context_len=3 * S,
+                                     needles="uniform:3")
+    run = run_workload_layer(w, 0)
+    check_run(w, run)
+
+
 def test_outlier_tokens_and_n_sweep():
     for n in (2, 4, 8):
         w = synth.workload("llama8b_64k").with_(name=f"out{n}", block_size=768, context_len=2 * 768,
