@@ -247,6 +247,41 @@ laser_kv_status_t laser_kv_window_scores_static(const void* K_blk, const void* Q
                                                 int32_t block_size, int32_t window, int32_t n_blocks,
                                                 float softmax_scale, float* s_exact_out, void* stream);
 
+/* Steps 2 and 3 of the path alone (Section 3.3 "Recall", Algorithm 1 line 6, per layer and KV head):
+ * count[b][h][t][j] = number of (window query of KV head h's group, table r) pairs whose K-bit
+ * SimHash bucket h_r(q) equals h_r(k_j), k_j the j-th key of block t; S_lsh = count / (L * G * W).
+ *   K_blk, Q_win, kv_strides, q_strides, n_blocks : as for laser_kv_select_block.
+ *   hyperplanes : dev bf16 [lsh_tables * lsh_bits][128], table-major (row r*K + b = bit b of table r).
+ *   scratch     : dev, 256-byte aligned, at least laser_kv_collision_counts_scratch_bytes(...) bytes,
+ *                 owned by the caller (query histogram, query codes, exact-sign work list). Its first
+ *                 int is a status word (0, LASER_KV_ERR_TIMEOUT, or LASER_KV_ERR_CAPACITY if the
+ *                 exact-sign list overflowed).
+ *   counts_out  : dev u32 [batch][H_kv][n_blocks][S].
+ * head_dim is 128; lsh_bits in {4,6,8,10,12}; lsh_tables a multiple of 8. */
+size_t laser_kv_collision_counts_scratch_bytes(int32_t batch, int32_t n_q_heads, int32_t n_kv_heads,
+                                               int32_t block_size, int32_t window, int32_t n_blocks,
+                                               int32_t lsh_bits, int32_t lsh_tables);
+laser_kv_status_t laser_kv_collision_counts(const void* K_blk, const void* Q_win, const void* hyperplanes,
+                                            const int64_t kv_strides[3], const int64_t q_strides[3],
+                                            int32_t batch, int32_t n_q_heads, int32_t n_kv_heads,
+                                            int32_t block_size, int32_t window, int32_t n_blocks,
+                                            int32_t lsh_bits, int32_t lsh_tables, void* scratch,
+                                            size_t scratch_bytes, uint32_t* counts_out, void* stream);
+
+/* Consensus aggregation (Section 3.3 "Precision" as printed: a candidate's score is the attention
+ * it receives summed over all layers and heads, so that one index set serves every head): adds the
+ * per-head outputs of laser_kv_window_scores and laser_kv_collision_counts over the n_heads heads,
+ *   s_acc[b][t][j] (+)= sum_h s_exact[b][h][t][j],   c_acc[b][t][j] (+)= sum_h counts[b][h][t][j],
+ * overwriting the sums when carry == 0 and adding to them when carry != 0 (further layers).
+ * Heads are added in ascending order, so the fp32 sums are reproducible. Feed the sums to
+ * laser_kv_two_stage_topk (n_segments = batch * n_blocks) and the resulting index lists to
+ * laser_kv_gather_append once per head.
+ *   s_exact dev fp32, counts dev u32 [batch][n_heads][n_blocks][S]; s_acc dev fp32, c_acc dev u32
+ *   [batch][n_blocks][S]; all 16-byte aligned; S a multiple of 4. */
+laser_kv_status_t laser_kv_consensus_accumulate(const float* s_exact, const uint32_t* counts, int32_t batch,
+                                                int32_t n_heads, int32_t n_blocks, int32_t block_size,
+                                                int32_t carry, float* s_acc, uint32_t* c_acc, void* stream);
+
 /* Append step (Sections 1 and 3): for each of n_segments segments copies rows idx[seg][i] of the
  * segment's K and V (dev bf16, row length d = 128, consecutive rows `src_row_stride` elements
  * apart, segment s starting at src + s*src_seg_stride) to dst rows [dst_offset + i] of the

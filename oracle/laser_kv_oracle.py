@@ -243,6 +243,29 @@ def select_block(k_bits: np.ndarray, q_bits: np.ndarray, p_bits: np.ndarray, *, 
     return out
 
 
+def select_block_consensus(k_layers, q_layers, p_bits: np.ndarray, *, n_bits: int, n_tables: int, B: int,
+                           n: int, alpha: float = 0.75, scale: float | None = None):
+    """Consensus form of steps 1-3 for one block of one sequence (Section 3.3 "Precision" as printed:
+    a candidate's exact score is the attention it receives from the query summed over all layers
+    and heads; Algorithm 1 then picks one index set that every head keeps).
+
+    k_layers[l] uint16 [H_kv, S, d] and q_layers[l] uint16 [H_q, W, d] for every layer l. The exact
+    scores and the collision counts of all (layer, KV head) pairs are added up; the two-stage
+    top-k runs once on the sums. Returns (s_sum float64 [S], c_sum int64 [S], k_exact, k_lsh, idx).
+    """
+    s_sum = None
+    c_sum = None
+    for k_bits, q_bits in zip(k_layers, q_layers):
+        r = select_block(k_bits, q_bits, p_bits, n_bits=n_bits, n_tables=n_tables, B=B, n=n, alpha=alpha, scale=scale)
+        for h in range(k_bits.shape[0]):
+            s_sum = r.s_exact[h].copy() if s_sum is None else s_sum + r.s_exact[h]
+            c_sum = r.counts[h].copy() if c_sum is None else c_sum + r.counts[h]
+    S = s_sum.shape[0]
+    a, _, _b_long, k_e, k_l = partition(B, n, alpha)
+    k_ex, k_ls, idx = select_indices(s_sum, c_sum, S, a, k_e, k_l)
+    return s_sum, c_sum, k_ex, k_ls, idx
+
+
 @dataclass
 class AppendOnlyCache:
     """Accumulative cache of one (layer, sequence): entries are only ever appended.

@@ -18,6 +18,7 @@ EXPORTS = [
     "laser_kv_two_stage_topk", "laser_kv_gather_append", "laser_kv_profile_enable",
     "laser_kv_profile_read", "laser_kv_window_scores", "laser_kv_window_scores_scratch_bytes",
     "laser_kv_window_scores_static", "laser_kv_window_scores_static_max_bytes",
+    "laser_kv_collision_counts", "laser_kv_collision_counts_scratch_bytes", "laser_kv_consensus_accumulate",
 ]
 
 
@@ -122,6 +123,13 @@ def load(build_if_missing: bool = True) -> C.CDLL:
     lib.laser_kv_window_scores_static.restype = i32
     lib.laser_kv_window_scores_static.argtypes = [vp, vp, p(i64), p(i64), i32, i32, i32, i32, i32, i32, C.c_float,
                                                   vp, vp]
+    lib.laser_kv_collision_counts_scratch_bytes.restype = sz
+    lib.laser_kv_collision_counts_scratch_bytes.argtypes = [i32] * 8
+    lib.laser_kv_collision_counts.restype = i32
+    lib.laser_kv_collision_counts.argtypes = [vp, vp, vp, p(i64), p(i64), i32, i32, i32, i32, i32, i32, i32, i32, vp, sz,
+                                              vp, vp]
+    lib.laser_kv_consensus_accumulate.restype = i32
+    lib.laser_kv_consensus_accumulate.argtypes = [vp, vp, i32, i32, i32, i32, i32, vp, vp, vp]
     _lib = lib
     return lib
 
@@ -341,6 +349,40 @@ def laser_kv_window_scores(K_blk, Q_win, block_size, n_blocks, softmax_scale=0.0
                                          n_blocks, softmax_scale, _ptr(scratch), scratch.numel(), _ptr(out),
                                          _stream_ptr(stream)))
     return out
+
+
+def laser_kv_collision_counts(K_blk, Q_win, hyperplanes, block_size, n_blocks, lsh_bits, lsh_tables, scratch=None,
+                              stream=None):
+    """K_blk [batch][H_kv][n_blocks*S][128], Q_win [batch][H_q][W][128], hyperplanes [L*K][128] (2-byte
+    device tensors) -> collision counts int32 [batch][H_kv][n_blocks][S]. Returns (counts, scratch); the
+    first int of scratch is the status word. `scratch` is allocated by torch when not given."""
+    import torch
+    batch, h_kv = K_blk.shape[0], K_blk.shape[1]
+    h_q, window = Q_win.shape[1], Q_win.shape[2]
+    need = int(load().laser_kv_collision_counts_scratch_bytes(batch, h_q, h_kv, block_size, window, n_blocks,
+                                                              lsh_bits, lsh_tables))
+    if scratch is None:
+        scratch = torch.empty(max(need, 256), dtype=torch.uint8, device=K_blk.device)
+    out = torch.empty((batch, h_kv, n_blocks, block_size), dtype=torch.int32, device=K_blk.device)
+    ks = (C.c_int64 * 3)(*K_blk.stride()[:3])
+    qs = (C.c_int64 * 3)(*Q_win.stride()[:3])
+    _check(load().laser_kv_collision_counts(_ptr(K_blk), _ptr(Q_win), _ptr(hyperplanes), ks, qs, batch, h_q, h_kv,
+                                            block_size, window, n_blocks, lsh_bits, lsh_tables, _ptr(scratch),
+                                            scratch.numel(), _ptr(out), _stream_ptr(stream)))
+    return out, scratch
+
+
+def laser_kv_consensus_accumulate(s_exact, counts, s_acc=None, c_acc=None, carry=False, stream=None):
+    """Sums [batch][H][n_blocks][S] scores (fp32) and counts (int32) over the heads into
+    [batch][n_blocks][S] accumulators; carry=True adds to the given accumulators."""
+    import torch
+    batch, heads, nb, S = s_exact.shape
+    if s_acc is None:
+        s_acc = torch.empty((batch, nb, S), dtype=torch.float32, device=s_exact.device)
+        c_acc = torch.empty((batch, nb, S), dtype=torch.int32, device=s_exact.device)
+    _check(load().laser_kv_consensus_accumulate(_ptr(s_exact), _ptr(counts), batch, heads, nb, S, 1 if carry else 0,
+                                                _ptr(s_acc), _ptr(c_acc), _stream_ptr(stream)))
+    return s_acc, c_acc
 
 
 def laser_kv_window_scores_static_max_bytes() -> int:

@@ -962,6 +962,177 @@ laser_kv_status_t laser_kv_window_scores_static(const void* K_blk, const void* Q
   return run_window_scores(g, K_blk, Q_win, kv_strides, q_strides, scratch, s_exact_out, static_cast<cudaStream_t>(stream));
 }
 
+// ---- collision counts on caller-fed inputs ---------------------------------------------------------
+namespace {
+
+struct CountGeom {
+  ScoreGeom g;
+  int K, L, TC, n_chunks, fix_cap;
+  size_t off_hist, off_qb, off_fix, total;   // scratch layout after the 256-byte control block
+};
+
+laser_kv_status_t count_geometry(int32_t batch, int32_t n_q_heads, int32_t n_kv_heads, int32_t block_size, int32_t window,
+                                 int32_t n_blocks, int32_t lsh_bits, int32_t lsh_tables, CountGeom* cg) {
+  const laser_kv_status_t s = score_geometry(batch, n_q_heads, n_kv_heads, block_size, window, n_blocks, 0.f, &cg->g);
+  if (s != LASER_KV_OK) return s;
+  if (!(lsh_bits == 4 || lsh_bits == 6 || lsh_bits == 8 || lsh_bits == 10 || lsh_bits == 12) || lsh_tables < 1)
+    return fail(nullptr, LASER_KV_ERR_UNSUPPORTED, "collision_counts: lsh_bits must be one of 4, 6, 8, 10, 12");
+  cg->K = lsh_bits;
+  cg->L = lsh_tables;
+  cg->TC = pick_tc(lsh_bits, lsh_tables);
+  if (!cg->TC) return fail(nullptr, LASER_KV_ERR_UNSUPPORTED, "collision_counts: lsh_tables must be a multiple of 8");
+  if ((long long)cg->g.GW * lsh_tables > 0x7fffffffLL)
+    return fail(nullptr, LASER_KV_ERR_UNSUPPORTED, "collision_counts: G*W*lsh_tables too large");
+  cg->n_chunks = lsh_tables / cg->TC;
+  long long fc = (long long)cg->g.nseg * block_size * lsh_tables / 256;
+  if (fc < 4096) fc = 4096;
+  if (fc > (1 << 26)) fc = 1 << 26;
+  cg->fix_cap = (int)fc;
+  const size_t bh = (size_t)batch * n_kv_heads;
+  size_t off = 256;
+  cg->off_hist = off; off = align_up(off + bh * lsh_tables * ((size_t)2 << lsh_bits));
+  cg->off_qb = off;   off = align_up(off + bh * cg->g.GW * lsh_tables * 2);
+  cg->off_fix = off;  off = align_up(off + (size_t)cg->fix_cap * sizeof(int4));
+  cg->total = off;
+  return LASER_KV_OK;
+}
+
+bool encode_bf16_map(EncodeTiledFn enc, CUtensorMap* m, const void* ptr, int rank, const cuuint64_t* dims,
+                     const cuuint64_t* strides_bytes, const cuuint32_t* box) {
+  const cuuint32_t ones[4] = {1, 1, 1, 1};
+  return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(ptr), dims, strides_bytes, box, ones,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+size_t laser_kv_collision_counts_scratch_bytes(int32_t batch, int32_t n_q_heads, int32_t n_kv_heads, int32_t block_size,
+                                               int32_t window, int32_t n_blocks, int32_t lsh_bits, int32_t lsh_tables) {
+  CountGeom cg;
+  if (count_geometry(batch, n_q_heads, n_kv_heads, block_size, window, n_blocks, lsh_bits, lsh_tables, &cg) != LASER_KV_OK)
+    return 0;
+  return cg.total;
+}
+
+laser_kv_status_t laser_kv_collision_counts(const void* K_blk, const void* Q_win, const void* hyperplanes,
+                                            const int64_t kv_strides[3], const int64_t q_strides[3], int32_t batch,
+                                            int32_t n_q_heads, int32_t n_kv_heads, int32_t block_size, int32_t window,
+                                            int32_t n_blocks, int32_t lsh_bits, int32_t lsh_tables, void* scratch,
+                                            size_t scratch_bytes, uint32_t* counts_out, void* stream) {
+  CountGeom cg;
+  const laser_kv_status_t gs = count_geometry(batch, n_q_heads, n_kv_heads, block_size, window, n_blocks, lsh_bits,
+                                              lsh_tables, &cg);
+  if (gs != LASER_KV_OK) return gs;
+  const ScoreGeom& g = cg.g;
+  if (!K_blk || !Q_win || !hyperplanes || !kv_strides || !q_strides || !scratch || !counts_out)
+    return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "collision_counts: NULL argument");
+  if (!aligned16(K_blk) || !aligned16(Q_win) || !aligned16(hyperplanes) || !aligned16(counts_out) ||
+      (reinterpret_cast<uintptr_t>(scratch) & (kAlign - 1)))
+    return fail(nullptr, LASER_KV_ERR_ALIGNMENT, "collision_counts: pointers must be 16-byte aligned, scratch 256-byte aligned");
+  if (scratch_bytes < cg.total)
+    return fail(nullptr, LASER_KV_ERR_CAPACITY, "collision_counts: scratch needs %zu bytes, got %zu", cg.total, scratch_bytes);
+  for (int i = 0; i < 3; ++i)
+    if (kv_strides[i] < 0 || q_strides[i] < 0 || (kv_strides[i] % 8) || (q_strides[i] % 8))
+      return fail(nullptr, LASER_KV_ERR_ALIGNMENT, "collision_counts: strides must be non-negative multiples of 8 elements");
+  if (kv_strides[2] < kHeadDim || q_strides[2] < kHeadDim || (g.H_kv > 1 && !kv_strides[1]) || (g.batch > 1 && !kv_strides[0]) ||
+      (g.H_q > 1 && !q_strides[1]) || (g.batch > 1 && !q_strides[0]))
+    return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "collision_counts: bad strides");
+  EncodeTiledFn enc = driver_encode_fn();
+  if (!enc) return fail(nullptr, LASER_KV_ERR_CUDA, "collision_counts: cuTensorMapEncodeTiled not available (no CUDA driver?)");
+  CUtensorMap mapK, mapQ, mapP, mapPq;
+  {
+    const cuuint64_t s_tok = (cuuint64_t)kv_strides[2];
+    const cuuint64_t s_head = kv_strides[1] > 0 ? (cuuint64_t)kv_strides[1] : s_tok * (cuuint64_t)g.nb * g.S;
+    const cuuint64_t s_batch = kv_strides[0] > 0 ? (cuuint64_t)kv_strides[0] : s_head * (cuuint64_t)g.H_kv;
+    const cuuint64_t dims[4] = {(cuuint64_t)kHeadDim, (cuuint64_t)g.nb * g.S, (cuuint64_t)g.H_kv, (cuuint64_t)g.batch};
+    const cuuint64_t strides[3] = {s_tok * 2, s_head * 2, s_batch * 2};
+    const cuuint32_t box[4] = {(cuuint32_t)kAtomCols, (cuuint32_t)kTileKeys, 1, 1};
+    const cuuint64_t s_w = (cuuint64_t)q_strides[2];
+    const cuuint64_t q_head = q_strides[1] > 0 ? (cuuint64_t)q_strides[1] : s_w * (cuuint64_t)g.W;
+    const cuuint64_t q_batch = q_strides[0] > 0 ? (cuuint64_t)q_strides[0] : q_head * (cuuint64_t)g.H_q;
+    const cuuint64_t qdims[4] = {(cuuint64_t)kHeadDim, (cuuint64_t)g.W, (cuuint64_t)g.H_q, (cuuint64_t)g.batch};
+    const cuuint64_t qstrides[3] = {s_w * 2, q_head * 2, q_batch * 2};
+    const cuuint32_t qbox[4] = {(cuuint32_t)kAtomCols, (cuuint32_t)g.W, (cuuint32_t)g.G, 1};
+    const cuuint64_t pdims[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)lsh_tables * lsh_bits};
+    const cuuint64_t pstrides[1] = {(cuuint64_t)kHeadDim * 2};
+    const cuuint32_t pbox[2] = {(cuuint32_t)kAtomCols, (cuuint32_t)(cg.TC * lsh_bits)};
+    const cuuint32_t pqbox[2] = {(cuuint32_t)kAtomCols, (cuuint32_t)(kQsigTables * lsh_bits)};
+    if (!encode_bf16_map(enc, &mapK, K_blk, 4, dims, strides, box) || !encode_bf16_map(enc, &mapQ, Q_win, 4, qdims, qstrides, qbox) ||
+        !encode_bf16_map(enc, &mapP, hyperplanes, 2, pdims, pstrides, pbox) ||
+        !encode_bf16_map(enc, &mapPq, hyperplanes, 2, pdims, pstrides, pqbox))
+      return fail(nullptr, LASER_KV_ERR_CUDA, "collision_counts: cuTensorMapEncodeTiled failed");
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  cudaError_t e;
+  int dev = 0, num_sms = 0;
+  if ((e = cudaGetDevice(&dev)) != cudaSuccess ||
+      (e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess)
+    return fail(nullptr, LASER_KV_ERR_CUDA, "collision_counts: device query: %s", cudaGetErrorString(e));
+  uint8_t* sc = static_cast<uint8_t*>(scratch);
+  int* ctrl = reinterpret_cast<int*>(sc);
+  uint16_t* hist = reinterpret_cast<uint16_t*>(sc + cg.off_hist);
+  uint16_t* qb = reinterpret_cast<uint16_t*>(sc + cg.off_qb);
+  int4* fix_items = reinterpret_cast<int4*>(sc + cg.off_fix);
+  // the status word must start at zero; the query-signature kernel restarts the other counters
+  if ((e = cudaMemsetAsync(sc, 0, 256, st)) != cudaSuccess)
+    return fail(nullptr, LASER_KV_ERR_CUDA, "collision_counts: memset: %s", cudaGetErrorString(e));
+  const uint16_t* P = static_cast<const uint16_t*>(hyperplanes);
+  {
+    const int q_alloc = ((g.GW + 127) / 128) * 128;
+    QsigArgs qa{static_cast<const uint16_t*>(Q_win), q_strides[0], q_strides[1], q_strides[2], P, hist, qb,
+                g.H_kv, g.G, g.W, g.GW, q_alloc, lsh_tables,
+                reinterpret_cast<uint4*>(counts_out), (long long)g.nseg * g.S / 4, ctrl + 1, ctrl};
+    dim3 grid(lsh_tables / kQsigTables, g.H_kv, g.batch);
+    if ((e = launch_qsig(lsh_bits, mapQ, mapPq, qa, grid, qsig_smem_bytes(q_alloc, lsh_bits), st)) != cudaSuccess)
+      return fail(nullptr, LASER_KV_ERR_CUDA, "collision_counts: qsig_kernel: %s", cudaGetErrorString(e));
+  }
+  {
+    StreamArgs sa;
+    memset(&sa, 0, sizeof sa);
+    sa.S = g.S; sa.nb = g.nb; sa.H_kv = g.H_kv; sa.batch = g.batch;
+    sa.G = g.G; sa.W = g.W; sa.GW = g.GW; sa.tiles_in_block = g.tiles_in_block; sa.nseg = g.nseg;
+    sa.n_chunks = cg.n_chunks; sa.tables_per_chunk = cg.TC; sa.lsh_bits = lsh_bits; sa.lsh_tables = lsh_tables;
+    sa.n_tiles = (long long)g.nseg * g.tiles_in_block * cg.n_chunks;
+    sa.stat_rows = cg.TC * lsh_bits; sa.stat_rows_alloc = sa.stat_rows;
+    sa.counts = counts_out; sa.hist = hist; sa.fix_items = fix_items; sa.fix_count = ctrl + 1; sa.fix_cap = cg.fix_cap;
+    sa.status = ctrl;
+    const uint32_t smem = stream_smem_bytes(kProj, sa.stat_rows_alloc, cg.TC * (2 << lsh_bits));
+    if ((e = launch_proj(lsh_bits, cg.TC, mapK, mapP, sa, stream_grid(sa.n_tiles, num_sms), smem, st)) != cudaSuccess)
+      return fail(nullptr, LASER_KV_ERR_CUDA, "collision_counts: projection pass: %s", cudaGetErrorString(e));
+  }
+  {
+    SignfixArgs fa{static_cast<const uint16_t*>(K_blk), kv_strides[0], kv_strides[1], kv_strides[2], P, hist, counts_out,
+                   nullptr, fix_items, ctrl + 1, cg.fix_cap, g.H_kv, g.nb, g.S, lsh_bits, lsh_tables, ctrl + 2};
+    signfix_kernel<<<kSignfixCtas, 256, 0, st>>>(fa);
+    g_launches.fetch_add(1);
+    if ((e = cudaGetLastError()) != cudaSuccess)
+      return fail(nullptr, LASER_KV_ERR_CUDA, "collision_counts: signfix_kernel: %s", cudaGetErrorString(e));
+  }
+  return LASER_KV_OK;
+}
+
+laser_kv_status_t laser_kv_consensus_accumulate(const float* s_exact, const uint32_t* counts, int32_t batch,
+                                                int32_t n_heads, int32_t n_blocks, int32_t block_size, int32_t carry,
+                                                float* s_acc, uint32_t* c_acc, void* stream) {
+  if (!s_exact || !counts || !s_acc || !c_acc) return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "consensus_accumulate: NULL argument");
+  if (batch < 1 || n_heads < 1 || n_blocks < 1 || block_size < 1 || (block_size % 4))
+    return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "consensus_accumulate: sizes must be positive, block_size a multiple of 4");
+  if (!aligned16(s_exact) || !aligned16(counts) || !aligned16(s_acc) || !aligned16(c_acc))
+    return fail(nullptr, LASER_KV_ERR_ALIGNMENT, "consensus_accumulate: pointers must be 16-byte aligned");
+  const long long n4 = (long long)n_blocks * block_size / 4;
+  ConsensusArgs a{reinterpret_cast<const float4*>(s_exact), reinterpret_cast<const uint4*>(counts),
+                  reinterpret_cast<float4*>(s_acc), reinterpret_cast<uint4*>(c_acc), n4, batch, n_heads, carry ? 1 : 0};
+  const long long total = (long long)batch * n4;
+  long long blocks = (total + 255) / 256;
+  if (blocks > 148 * 8) blocks = 148 * 8;
+  consensus_kernel<<<(unsigned)blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(a);
+  g_launches.fetch_add(1);
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(nullptr, LASER_KV_ERR_CUDA, "consensus_kernel launch: %s", cudaGetErrorString(e));
+  return LASER_KV_OK;
+}
+
 laser_kv_status_t laser_kv_gather_append(const void* K_src, const void* V_src, int64_t src_seg_stride,
                                          int64_t src_row_stride, const int32_t* idx, int32_t n_segments,
                                          int32_t n_keep, void* K_dst, void* V_dst, int64_t dst_seg_stride,

@@ -283,4 +283,37 @@ __global__ void __launch_bounds__(256) append_kernel(const AppendArgs a) {
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Consensus aggregation: the paper's Algorithm 1 line 3 scores a candidate with the attention it
+// receives from all heads (and layers). For every sequence b and position i of the call's blocks,
+// adds the scores and the collision counts of the H KV heads and either stores the sums or adds
+// them to sums carried over from other layers.
+// ------------------------------------------------------------------------------------------------
+struct ConsensusArgs {
+  const float4* s;        // [batch][H][n4]  (n4 = n_blocks * S / 4)
+  const uint4* c;         // [batch][H][n4]
+  float4* s_acc;          // [batch][n4]
+  uint4* c_acc;           // [batch][n4]
+  long long n4;
+  int batch, H;
+  int carry;              // 0: overwrite the sums, 1: add to them
+};
+
+__global__ void __launch_bounds__(256) consensus_kernel(const ConsensusArgs a) {
+  const long long total = (long long)a.batch * a.n4;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+    const long long b = i / a.n4, j = i - b * a.n4;
+    float4 fs = a.carry ? a.s_acc[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+    uint4 cs = a.carry ? a.c_acc[i] : make_uint4(0u, 0u, 0u, 0u);
+    for (int h = 0; h < a.H; ++h) {              // fixed order: deterministic sums
+      const float4 x = a.s[(b * a.H + h) * a.n4 + j];
+      const uint4 y = a.c[(b * a.H + h) * a.n4 + j];
+      fs.x += x.x; fs.y += x.y; fs.z += x.z; fs.w += x.w;
+      cs.x += y.x; cs.y += y.y; cs.z += y.z; cs.w += y.w;
+    }
+    a.s_acc[i] = fs;
+    a.c_acc[i] = cs;
+  }
+}
+
 }  // namespace lkv

@@ -146,3 +146,50 @@ def test_cache_is_append_only_with_increasing_positions():
         assert (np.diff(cache.pos[h, :cache.length]) > 0).all()
     with pytest.raises(ValueError):
         cache.append(k, v, r.idx, 4 * 128)
+
+
+def _small_layers(n_layers, seed=3, S=96, hkv=2, hq=4, W=8, K=4, L=8):
+    w = synth.workload("tiny").with_(name="cons", n_layers=n_layers, n_q_heads=hq, n_kv_heads=hkv, window=W,
+                                     lsh_bits=K, lsh_tables=L, block_size=S, context_len=2 * S, seed=seed)
+    ks = [synth.kv_block(w, l, 0, 1)[0] for l in range(n_layers)]
+    qs = [synth.q_window(w, l, 0) for l in range(n_layers)]
+    return w, ks, qs, synth.hyperplanes(w)
+
+
+def test_consensus_reduces_to_the_single_head_rule():
+    # one layer with one KV head: the consensus sums are that head's own scores and counts
+    w, ks, qs, P = _small_layers(1, hkv=1, hq=2)
+    r = O.select_block(ks[0], qs[0], P, n_bits=4, n_tables=8, B=40, n=4)
+    s, c, k_ex, k_ls, idx = O.select_block_consensus(ks, qs, P, n_bits=4, n_tables=8, B=40, n=4)
+    assert (s == r.s_exact[0]).all() and (c == r.counts[0]).all()
+    assert idx.tolist() == r.idx[0].tolist() and k_ex.tolist() == r.k_exact[0].tolist()
+
+
+def test_consensus_sums_over_heads_and_layers():
+    w, ks, qs, P = _small_layers(3)
+    s, c, k_ex, k_ls, idx = O.select_block_consensus(ks, qs, P, n_bits=4, n_tables=8, B=40, n=4)
+    # plain definition: add every (layer, head) array, then run the two-stage rule once
+    s_ref = np.zeros(96)
+    c_ref = np.zeros(96, np.int64)
+    for l in range(3):
+        r = O.select_block(ks[l], qs[l], P, n_bits=4, n_tables=8, B=40, n=4)
+        s_ref += r.s_exact.sum(axis=0)
+        c_ref += r.counts.sum(axis=0)
+    assert np.allclose(s, s_ref, rtol=1e-13, atol=0) and (c == c_ref).all()
+    # every softmax row sums to one: the block total is (layers * query heads * window)
+    assert abs(s.sum() - 3 * 4 * 8) < 1e-9
+    a, _, _, k_e, k_l = O.partition(40, 4)
+    assert len(idx) == 40 and len(k_ex) == k_e and len(k_ls) == k_l
+    assert idx.tolist() == O.select_indices(s_ref, c_ref, 96, a, k_e, k_l)[2].tolist()
+    # the order of layers does not matter beyond rounding; counts are exact
+    s2, c2, *_ = O.select_block_consensus(ks[::-1], qs[::-1], P, n_bits=4, n_tables=8, B=40, n=4)
+    assert np.allclose(s2, s, rtol=1e-13, atol=0) and (c2 == c).all()
+
+
+def test_consensus_of_identical_layers_keeps_the_selection():
+    # the same layer repeated: sums scale by the repeat count, the chosen set does not change
+    w, ks, qs, P = _small_layers(1)
+    one = O.select_block_consensus(ks, qs, P, n_bits=4, n_tables=8, B=40, n=4)
+    four = O.select_block_consensus(ks * 4, qs * 4, P, n_bits=4, n_tables=8, B=40, n=4)
+    assert np.allclose(four[0], 4 * one[0], rtol=1e-13, atol=0) and (four[1] == 4 * one[1]).all()
+    assert four[4].tolist() == one[4].tolist()
