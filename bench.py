@@ -360,6 +360,105 @@ def run_ours(args, w, rank, world, local_rank):
         dist.destroy_process_group()
 
 
+def run_consensus(args, w, rank, world, local_rank):
+    """Consensus policy (scores and counts summed over all KV heads, one index set per block): a
+    step scores one layer (window scores + collision counts), folds it into the running sums,
+    selects on the sums and gathers every head with the shared set. Step-level entry points; no
+    per-kernel breakdown."""
+    import torch
+    import torch.distributed as dist
+    from paper_2602_02199_b200 import binding as Bn
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    S, nb, H = w.block_size, w.n_blocks, w.n_kv_heads
+    B = Bn.laser_kv_budget(w.context_len, S, w.ratio)
+    a, _, k_e, k_l = Bn.laser_kv_partition(B, w.protection_divisor, w.alpha)
+    sets = []
+    for i in range(args.input_sets):
+        k, v = synth.kv_blocks(w, rank * args.input_sets + i, 0, 0, nb)
+        q = synth.q_window(w, rank * args.input_sets + i, 0)
+        sets.append(tuple(torch.from_numpy(x.view(np.int16))[None].to(dev) for x in (k, v, q)))
+    P = torch.from_numpy(synth.hyperplanes(w).view(np.int16)).to(dev)
+    Kd = torch.zeros((H, nb * B, w.head_dim), dtype=torch.int16, device=dev)
+    Vd = torch.zeros_like(Kd)
+    pos = torch.zeros((H, nb * B), dtype=torch.int32, device=dev)
+    s_acc = torch.zeros((1, nb, S), dtype=torch.float32, device=dev)
+    c_acc = torch.zeros((1, nb, S), dtype=torch.int32, device=dev)
+    scr_s = torch.empty(Bn.laser_kv_window_scores_scratch_bytes(1, w.n_q_heads, H, S, w.window, nb), dtype=torch.uint8,
+                        device=dev)
+    scr_c = None
+
+    def step(i):
+        nonlocal scr_c
+        tk, tv, tq = sets[i % len(sets)]
+        s = Bn.laser_kv_window_scores(tk, tq, S, nb, scratch=scr_s)
+        c, scr_c = Bn.laser_kv_collision_counts(tk, tq, P, S, nb, w.lsh_bits, w.lsh_tables, scratch=scr_c)
+        Bn.laser_kv_consensus_accumulate(s, c, s_acc, c_acc, carry=False)
+        idx = Bn.laser_kv_two_stage_topk(s_acc.view(nb, S), c_acc.view(nb, S), a, k_e, k_l)
+        for h in range(H):
+            Bn.laser_kv_gather_append(tk[0, h].view(nb, S, 128), tv[0, h].view(nb, S, 128), idx, Kd[h].view(nb, B, 128),
+                                      Vd[h].view(nb, B, 128), pos[h].view(nb, B), 0, 0)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    launches0 = Bn.laser_kv_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t0 = time.time()
+    e0.record()
+    for i in range(args.steps):
+        step(i)
+    e1.record()
+    barrier()
+    t1 = time.time()
+    ms = e0.elapsed_time(e1)
+    launches = Bn.laser_kv_launch_count() - launches0
+    assert int(scr_c[:4].view(torch.int32)[0]) == 0 and int(scr_s[:4].view(torch.int32)[0]) == 0
+    clocks = sampler.stop(t0, t1) if rank == 0 else None
+    t = torch.tensor([ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.destroy_process_group()
+    if rank != 0:
+        return
+    ms = float(t[0])
+    peaks = load_peaks()
+    work = algorithmic_work(w, B)
+    ms_per_step = ms / args.steps
+    t_tensor = work["flops"] / (peaks["tf"] * 1e12)
+    t_hbm = work["bytes"] / (peaks["hbm"] * 1e9)
+    line = {
+        "metric": METRIC, "value": world * work["tokens"] * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "policy": "consensus over the KV heads of a layer, one index set per block",
+                   "context_len": w.context_len, "block_size": S, "blocks_per_call": nb, "budget_per_block": B,
+                   "l2": f"inputs larger than L2: {len(sets)} layers of K+V cycled"},
+        "clocks": clocks, "e2e": None, "gpu_launches": int(launches),
+        "roofline": {"kernel": "whole step", "bound": "tensor", "achieved": work["flops"] / (ms_per_step * 1e-3) / 1e12,
+                     "peak": peaks["tf"], "unit": "TFLOP/s", "frac": t_tensor / (ms_per_step * 1e-3), "traffic": None,
+                     "peak_source": f"bf16_tflops (burst), {peaks['source']}"},
+        "path_roofline": {"hbm_frac": t_hbm / (ms_per_step * 1e-3), "tensor_frac": t_tensor / (ms_per_step * 1e-3)},
+        "cpu_baseline": None,
+    }
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -367,6 +466,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama8b_128k", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--policy", default="per_head", choices=["per_head", "consensus"],
+                    help="per_head: the hot path (every KV head selects for itself); consensus: one index set per block")
     ap.add_argument("--input-sets", type=int, default=2)
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--cpu-steps", type=int, default=6)
@@ -380,6 +481,8 @@ def main():
     w = synth.workload(args.workload)
     if args.impl == "reference":
         run_reference(args, w, rank, world)
+    elif args.policy == "consensus":
+        run_consensus(args, w, rank, world, local_rank)
     else:
         run_ours(args, w, rank, world, local_rank)
 
