@@ -39,10 +39,10 @@ UNIT = "tokens/s"
 # summarised in profiles/select_call_llama8b_128k.md, keyed by (workload, kernel). A missing key
 # means: not captured for this workload, or the kernel has changed since the capture.
 NCU_TRAFFIC_BYTES = {
-    ("llama8b_128k", "stream_kernel<proj>"): 274773760 + 7303680,
-    ("llama8b_128k", "stream_kernel<lse>"): 269266688 + 3940096,
-    ("llama8b_128k", "stream_kernel<score>"): 270398208 + 7105536,
-    ("llama8b_128k", "append_kernel"): 254747648 + 200837632,
+    ("llama8b_128k", "stream_kernel<proj>"): 274789120 + 7261184,
+    ("llama8b_128k", "stream_kernel<lse>"): 269266944 + 3838720,
+    ("llama8b_128k", "stream_kernel<score>"): 270472192 + 7939584,
+    ("llama8b_128k", "append_kernel"): 254743808 + 201296896,
 }
 
 
