@@ -223,6 +223,11 @@ def run_ours(args, w, rank, world, local_rank):
                          alpha=w.alpha, device=local_rank)
     eng = Bn.LaserKV(cfg, P)
     work = algorithmic_work(w, B)
+    _, _, k_exact, k_lsh = Bn.laser_kv_partition(B, w.protection_divisor, w.alpha)
+    if k_lsh == 0:        # exact attention only: the hash passes are not part of the method's work
+        work["flops"] = work["fl_score"]
+    elif k_exact == 0:    # LSH only
+        work["flops"] -= work["fl_score"]
 
     def step(i):
         s = i % n_sets
@@ -468,6 +473,9 @@ def main():
     ap.add_argument("--workload", default="llama8b_128k", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--policy", default="per_head", choices=["per_head", "consensus"],
                     help="per_head: the hot path (every KV head selects for itself); consensus: one index set per block")
+    ap.add_argument("--alpha", type=float, default=None,
+                    help="exact share of the recall budget (1 = exact attention only, 0 = LSH only; default: the workload's 0.75)")
+    ap.add_argument("--divisor", type=int, default=None, help="protection divisor n (default: the workload's)")
     ap.add_argument("--input-sets", type=int, default=2)
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--cpu-steps", type=int, default=6)
@@ -479,6 +487,10 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     w = synth.workload(args.workload)
+    if args.alpha is not None:
+        w = w.with_(alpha=args.alpha)
+    if args.divisor is not None:
+        w = w.with_(protection_divisor=args.divisor)
     if args.impl == "reference":
         run_reference(args, w, rank, world)
     elif args.policy == "consensus":

@@ -56,7 +56,10 @@ typedef struct {
   int32_t lsh_tables;          /* L: tables (the paper's R hash rounds); a multiple of 8          */
   int32_t protection_divisor;  /* n >= 2 (Section 3.1)                                           */
   int32_t budget_per_block;    /* B; 0 => Eq. 1 from ratio, block_size and context_len           */
-  int32_t debug;               /* nonzero: also keep per-key bucket ids for laser_kv_debug_view  */
+  int32_t debug;               /* nonzero: also keep per-key bucket ids for laser_kv_debug_view,
+                                  and compute both stages even when one has no picks to make
+                                  (alpha = 1, alpha = 0, n = 2); zero: a stage without picks is
+                                  skipped and its debug arrays are not refreshed               */
   int64_t context_len;         /* L of Eq. 1 (only read when budget_per_block == 0)              */
   double  ratio;               /* r of Eq. 1; 0 => 0.25                                          */
   double  alpha;               /* exact share of the recall budget; negative => 0.75             */

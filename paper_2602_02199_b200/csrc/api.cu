@@ -503,9 +503,14 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
     marks.push_back(ev);
   };
   mark();
+  // A stage whose share of the recall budget is empty (alpha = 1: no LSH picks; alpha = 0 or n = 2:
+  // no exact picks) is not computed, unless the debug view was asked for, which shows every
+  // intermediate result.
+  const bool need_lsh = d.k_lsh > 0 || c.debug;
+  const bool need_exact = d.k_exact > 0 || c.debug;
   // 1. query signatures and bucket histograms; the kernel also clears the counts and restarts the
   //    fix-up counter (ctrl[1]) and the changed counter (ctrl[2]); the status word (ctrl[0]) is kept
-  {
+  if (need_lsh) {
     const int q_alloc = ((d.GW + 127) / 128) * 128;
     QsigArgs qa{static_cast<const uint16_t*>(Q_win), q_strides[0], q_strides[1], q_strides[2], h->P, hist, qb,
                 c.n_kv_heads, d.G, c.window, d.GW, q_alloc, c.lsh_tables,
@@ -530,7 +535,7 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
 
   mark();
   // 2. per-query log-sum-exp over each block's keys
-  {
+  if (need_exact) {
     StreamArgs a1 = sa;
     a1.stat_rows = d.GW;
     a1.stat_rows_alloc = ((d.GW + 127) / 128) * 128;
@@ -539,7 +544,7 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
   }
   mark();
   // 3. summed attention probabilities per key
-  {
+  if (need_exact) {
     StreamArgs a2 = sa;
     a2.stat_rows = d.GW;
     a2.stat_rows_alloc = d.GW;
@@ -548,7 +553,7 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
   }
   mark();
   // 4. key signatures and collision counts
-  {
+  if (need_lsh) {
     StreamArgs a3 = sa;
     a3.stat_rows = d.TC * c.lsh_bits;
     a3.stat_rows_alloc = a3.stat_rows;
@@ -559,7 +564,7 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
   }
   mark();
   // 5. exact signs where the tensor-core projection was too close to zero
-  {
+  if (need_lsh) {
     SignfixArgs fa{static_cast<const uint16_t*>(K_blk), kv_strides[0], kv_strides[1], kv_strides[2], h->P, hist,
                    counts, key_buckets, fix_items, ctrl + 1, d.fix_cap, c.n_kv_heads, nb, S, c.lsh_bits,
                    c.lsh_tables, ctrl + 2};

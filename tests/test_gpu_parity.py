@@ -130,6 +130,19 @@ def test_same_inputs_twice_give_identical_bytes():
         assert (to_np(a[:, :, :n]) == to_np(b[:, :, :n])).all()
 
 
+@pytest.mark.parametrize("alpha", [1.0, 0.0])
+def test_single_stage_policies_skip_the_unused_stage_and_keep_the_cache(alpha):
+    # alpha = 1 (exact attention only) and alpha = 0 (LSH only): without the debug view the unused
+    # stage is not computed; the cache must equal the one of the run that computed everything
+    w = synth.workload("tiny").with_(block_size=640, context_len=1280, alpha=alpha)
+    full = run_workload_layer(w, 0, alpha=alpha, debug=1)
+    check_run(w, full, alpha=alpha)
+    lean = run_workload_layer(w, 0, alpha=alpha, debug=0)
+    n = full["n_blocks"] * full["B"]
+    for x, y in zip(full["engine"].laser_kv_cache_view(0)[:3], lean["engine"].laser_kv_cache_view(0)[:3]):
+        assert (to_np(x[:, :, :n]) == to_np(y[:, :, :n])).all()
+
+
 def test_two_stage_topk_entry_point_against_oracle():
     import torch
     from paper_2602_02199_b200 import binding as Bn
