@@ -52,7 +52,6 @@ __host__ __device__ constexpr int proj_acc_stride(int kbits, int tc) { return (k
 __host__ __device__ constexpr int proj_num_acc(int kbits, int tc) {
   return 512 / proj_acc_stride(kbits, tc) < kMaxAcc ? 512 / proj_acc_stride(kbits, tc) : kMaxAcc;
 }
-constexpr int kMaxStatRows = 256;
 constexpr int kMaxStreamCtas = 256;            // upper bound of the persistent grid (slot arithmetic)
 constexpr int kPolyPairsOf32 = 10;             // of every 32 column pairs, this many take 2^x on the FMA pipe
 
@@ -129,21 +128,6 @@ __device__ __forceinline__ bool cursor_last_of_segment(const TileCursor& c, cons
 }
 __device__ __forceinline__ bool cursor_last_of_group(const TileCursor& c, const StreamArgs& a) {
   return c.tib == a.tiles_in_block - 1 && c.t == a.nb - 1;
-}
-
-// Loads the 32-bit columns [CB, CE) of the calling thread's TMEM lane into r[0 .. CE-CB) as a
-// sequence of power-of-two loads, each starting at a multiple of its own width.
-template <int CB, int CE>
-__device__ __forceinline__ void tmem_ld_range(uint32_t taddr, uint32_t* r) {
-  if constexpr (CB < CE) {
-    constexpr int W = (CB % 32 == 0 && CB + 32 <= CE) ? 32
-                    : (CB % 16 == 0 && CB + 16 <= CE) ? 16
-                    : (CB % 8 == 0 && CB + 8 <= CE)   ? 8
-                    : (CB % 4 == 0 && CB + 4 <= CE)   ? 4
-                    : (CB % 2 == 0 && CB + 2 <= CE)   ? 2 : 1;
-    tmem_ld_cols<W>(taddr + CB, r);
-    tmem_ld_range<CB + W, CE>(taddr, r + W);
-  }
 }
 
 // Reads NC (a multiple of 16) columns starting at taddr into v.
