@@ -25,6 +25,8 @@ What each function follows:
 * ``select_indices``    - Algorithm 1 lines 3-8 on the candidate set left by Section 3.1.
 * ``select_block`` / ``AppendOnlyCache`` - Section 3 (only selected tokens are kept) and the
                           introduction's append-only accumulative memory.
+* ``decode_attention``  - Section 3 (the kept tokens serve the decoding phase): softmax attention
+                          of one decode query over the cache entries of its KV head.
 
 Readings taken where the paper is silent (rounding of B/n and alpha*B_long, per-block anchors,
 softmax over the block's own keys, bit = [projection >= 0], tie rule) are listed in the design
@@ -297,3 +299,30 @@ class AppendOnlyCache:
             self.V[h, sl] = v_bits[h, idx[h]]
             self.pos[h, sl] = (block_start + idx[h]).astype(np.int32)
         self.length += B
+
+
+# ----------------------------------------------------------------------------------------------
+# decoding over the kept tokens (Section 3: only the selected tokens stay in the cache and are
+# used for the decoding phase)
+# ----------------------------------------------------------------------------------------------
+def decode_attention(q_bits: np.ndarray, k_bits: np.ndarray, v_bits: np.ndarray,
+                     scale: float | None = None) -> np.ndarray:
+    """out[g] = sum_i softmax_i(<q_g, k_i> * scale) * v_i over the cache entries of one KV head.
+
+    q_bits: uint16 [G, d]   - the decode-step queries of the KV head's query heads.
+    k_bits, v_bits: uint16 [len, d] - the head's cache entries (len >= 1).
+    Plain softmax attention, no mask (every cache entry precedes the decode position); scale
+    defaults to 1/sqrt(d). Returns float64 [G, d].
+    """
+    q = bf16_bits_to_f64(q_bits)
+    k = bf16_bits_to_f64(k_bits)
+    v = bf16_bits_to_f64(v_bits)
+    if k.shape[0] < 1:
+        raise ValueError("decode_attention needs at least one cache entry")
+    if scale is None:
+        scale = 1.0 / math.sqrt(k.shape[1])
+    s = (q @ k.T) * float(scale)                      # [G, len]
+    s = s - s.max(axis=1, keepdims=True)
+    p = np.exp(s)
+    p = p / p.sum(axis=1, keepdims=True)
+    return p @ v
