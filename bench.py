@@ -464,6 +464,101 @@ def run_consensus(args, w, rank, world, local_rank):
     print(json.dumps(line), flush=True)
 
 
+def run_decode(args, w, rank, world, local_rank):
+    """Decode-phase attention over the compacted cache: the caches of `input_sets` layers are filled
+    by select calls (untimed); a step is one decode query per head attending over one layer's cache
+    (layers cycled, each cache larger than L2 for the long-context workloads)."""
+    import torch
+    import torch.distributed as dist
+    from paper_2602_02199_b200 import binding as Bn
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    S, nb, H = w.block_size, w.n_blocks, w.n_kv_heads
+    B = Bn.laser_kv_budget(w.context_len, S, w.ratio)
+    n_layers = max(2, args.input_sets)
+    P = torch.from_numpy(synth.hyperplanes(w).view(np.int16)).to(dev)
+    cfg = Bn.make_config(n_layers=n_layers, batch=w.batch, n_q_heads=w.n_q_heads, n_kv_heads=H, block_size=S,
+                         window=w.window, max_blocks=nb, max_blocks_per_call=nb, lsh_bits=w.lsh_bits,
+                         lsh_tables=w.lsh_tables, protection_divisor=w.protection_divisor, budget_per_block=B,
+                         alpha=w.alpha, debug=0, device=local_rank)
+    eng = Bn.LaserKV(cfg, P)
+    qs = []
+    for layer in range(n_layers):
+        ks, vs, qw = [], [], []
+        for b in range(w.batch):
+            k, v = synth.kv_blocks(w, rank * n_layers + layer, b, 0, nb)
+            ks.append(k); vs.append(v); qw.append(synth.q_window(w, rank * n_layers + layer, b))
+        tk, tv, tq = (torch.from_numpy(np.stack(x).view(np.int16)).to(dev) for x in (ks, vs, qw))
+        eng.laser_kv_select_block(layer, tk, tv, tq, nb)
+        eng.laser_kv_poll_status()
+        qs.append(tq[:, :, w.window - 1, :].contiguous())        # the last window query as the decode query
+        del tk, tv
+    out = torch.empty(w.batch, w.n_q_heads, 128, dtype=torch.float32, device=dev)
+    length = nb * B
+
+    def step(i):
+        eng.laser_kv_decode_attention(i % n_layers, qs[i % n_layers], out=out)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    launches0 = Bn.laser_kv_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t0 = time.time()
+    e0.record()
+    for i in range(args.steps):
+        step(i)
+    e1.record()
+    barrier()
+    t1 = time.time()
+    ms = e0.elapsed_time(e1)
+    launches = Bn.laser_kv_launch_count() - launches0
+    eng.laser_kv_poll_status()
+    clocks = sampler.stop(t0, t1) if rank == 0 else None
+    t = torch.tensor([ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.destroy_process_group()
+    if rank != 0:
+        return
+    ms = float(t[0])
+    peaks = load_peaks()
+    ms_per_step = ms / args.steps
+    entries = w.batch * H * length                               # cache entries read per step
+    nbytes = entries * 2 * 128 * 2 + w.batch * w.n_q_heads * 128 * (2 + 4)
+    achieved = nbytes / (ms_per_step * 1e-3) / 1e9
+    line = {
+        "metric": "decode_attention_cache_entries_per_s_per_layer", "value": world * entries * args.steps / (ms * 1e-3),
+        "unit": "cache entries/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": w.name, "policy": "decode attention over the compacted cache of one layer",
+                   "context_len": w.context_len, "cache_len_per_head": length, "batch": w.batch,
+                   "l2": f"{n_layers} layers' caches cycled ({entries * 512 / 1e6:.0f} MB each)"},
+        "clocks": clocks, "e2e": None, "gpu_launches": int(launches),
+        "roofline": {"kernel": "decode_chunk_kernel + decode_combine_kernel", "bound": "hbm", "achieved": achieved,
+                     "peak": peaks["hbm"], "unit": "GB/s", "frac": achieved / peaks["hbm"], "traffic": None,
+                     "peak_source": f"hbm_gbs, {peaks['source']}"},
+        "cpu_baseline": None,
+    }
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -471,8 +566,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama8b_128k", choices=sorted(synth.WORKLOADS))
-    ap.add_argument("--policy", default="per_head", choices=["per_head", "consensus"],
-                    help="per_head: the hot path (every KV head selects for itself); consensus: one index set per block")
+    ap.add_argument("--policy", default="per_head", choices=["per_head", "consensus", "decode"],
+                    help="per_head: the hot path (every KV head selects for itself); consensus: one index set per block; "
+                         "decode: attention of one decode step over the compacted cache")
     ap.add_argument("--alpha", type=float, default=None,
                     help="exact share of the recall budget (1 = exact attention only, 0 = LSH only; default: the workload's 0.75)")
     ap.add_argument("--divisor", type=int, default=None, help="protection divisor n (default: the workload's)")
@@ -495,6 +591,8 @@ def main():
         run_reference(args, w, rank, world)
     elif args.policy == "consensus":
         run_consensus(args, w, rank, world, local_rank)
+    elif args.policy == "decode":
+        run_decode(args, w, rank, world, local_rank)
     else:
         run_ours(args, w, rank, world, local_rank)
 

@@ -297,6 +297,27 @@ laser_kv_status_t laser_kv_gather_append(const void* K_src, const void* V_src,
                                          int32_t* pos_out, int64_t pos_seg_stride,
                                          int64_t dst_offset, int32_t pos_base, void* stream);
 
+/* Decode-phase attention over a layer's compacted cache (Section 3: once a block is processed only
+ * the selected tokens stay in the KV cache and serve the decoding phase; Section 4.1 evaluates the
+ * answers generated from that cache). For every sequence b and query head hq of KV head
+ * h = hq / G it computes, over the len = blocks appended so far * B cache entries of (b, h),
+ *   out[b][hq][:] = sum_i softmax_i(<Q_dec[b][hq], K_cache[b][h][i]> * scale) * V_cache[b][h][i].
+ * bf16 inputs, products and sums in fp32, output fp32.
+ *   Q_dec         : dev bf16, element (b, hq, :) at Q_dec + b*q_strides[0] + hq*q_strides[1], row of
+ *                   128 contiguous elements; 16-byte aligned, strides multiples of 8 elements.
+ *   softmax_scale : 0 selects the handle's configured scale.
+ *   out           : dev fp32 [batch][n_q_heads][128], 16-byte aligned.
+ *   scratch       : dev, 16-byte aligned, at least laser_kv_decode_attention_scratch_bytes(h) bytes
+ *                   (per-chunk partial sums), owned by the caller, reusable after the stream has
+ *                   passed the call.
+ * Asynchronous on `stream`, ordered after earlier select calls on the same stream. Errors:
+ * LASER_KV_ERR_STATE when the layer's cache is empty, LASER_KV_ERR_UNSUPPORTED for more than 8 query
+ * heads per KV head or more than 1 Mi entries per head, LASER_KV_ERR_CAPACITY for a short scratch. */
+size_t laser_kv_decode_attention_scratch_bytes(laser_kv_handle_t h);
+laser_kv_status_t laser_kv_decode_attention(laser_kv_handle_t h, int32_t layer, const void* Q_dec,
+                                            const int64_t q_strides[2], float softmax_scale, float* out,
+                                            void* scratch, size_t scratch_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -19,6 +19,7 @@ EXPORTS = [
     "laser_kv_profile_read", "laser_kv_window_scores", "laser_kv_window_scores_scratch_bytes",
     "laser_kv_window_scores_static", "laser_kv_window_scores_static_max_bytes",
     "laser_kv_collision_counts", "laser_kv_collision_counts_scratch_bytes", "laser_kv_consensus_accumulate",
+    "laser_kv_decode_attention", "laser_kv_decode_attention_scratch_bytes",
 ]
 
 
@@ -130,6 +131,10 @@ def load(build_if_missing: bool = True) -> C.CDLL:
                                               vp, vp]
     lib.laser_kv_consensus_accumulate.restype = i32
     lib.laser_kv_consensus_accumulate.argtypes = [vp, vp, i32, i32, i32, i32, i32, vp, vp, vp]
+    lib.laser_kv_decode_attention_scratch_bytes.restype = sz
+    lib.laser_kv_decode_attention_scratch_bytes.argtypes = [vp]
+    lib.laser_kv_decode_attention.restype = i32
+    lib.laser_kv_decode_attention.argtypes = [vp, i32, vp, p(i64), C.c_float, vp, vp, sz, vp]
     _lib = lib
     return lib
 
@@ -288,6 +293,22 @@ class LaserKV:
                       (d.batch, d.n_kv_heads, L, 1 << d.lsh_bits)),
             idx=view(d.idx, nseg * max(d.budget, 1) * 4, torch.int32, shp + (max(d.budget, 1),)),
             n_sign_fixups=int(d.n_sign_fixups))
+
+    def laser_kv_decode_attention(self, layer, Q_dec, softmax_scale=0.0, out=None, stream=None):
+        """Q_dec: [batch][H_q][d] 2-byte tensor (contiguous last dim) -> fp32 [batch][H_q][d]."""
+        torch = self._torch
+        c = self.cfg
+        assert Q_dec.stride(2) == 1 and Q_dec.element_size() == 2
+        if getattr(self, "_decode_scratch", None) is None:
+            nbytes = int(self.lib.laser_kv_decode_attention_scratch_bytes(self.handle))
+            self._decode_scratch = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+        if out is None:
+            out = torch.empty(c.batch, c.n_q_heads, 128, dtype=torch.float32, device=self.device)
+        qs = (C.c_int64 * 2)(*Q_dec.stride()[:2])
+        _check(self.lib.laser_kv_decode_attention(self.handle, layer, _ptr(Q_dec), qs, softmax_scale, _ptr(out),
+                                                  _ptr(self._decode_scratch), self._decode_scratch.numel(),
+                                                  _stream_ptr(stream)), self.handle)
+        return out
 
     def laser_kv_poll_status(self, stream=None):
         _check(self.lib.laser_kv_poll_status(self.handle, _stream_ptr(stream)), self.handle)

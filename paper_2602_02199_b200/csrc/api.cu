@@ -18,6 +18,7 @@
 #include "aux_kernels.cuh"
 #include "stream_gemm.cuh"
 #include "query_proj.cuh"
+#include "decode_attn.cuh"
 
 namespace {
 
@@ -652,6 +653,67 @@ laser_kv_status_t laser_kv_cache_view(laser_kv_handle_t h, int32_t layer, laser_
   out->kv_strides[2] = kHeadDim;
   out->pos_strides[0] = (int64_t)c.n_kv_heads * d.cap;
   out->pos_strides[1] = d.cap;
+  return LASER_KV_OK;
+}
+
+size_t laser_kv_decode_attention_scratch_bytes(laser_kv_handle_t h) {
+  if (!h) return 0;
+  const laser_kv_config_t& c = h->cfg;
+  const long long n_chunks = ((long long)h->d.cap + kDecChunk - 1) / kDecChunk;
+  return (size_t)c.batch * c.n_q_heads * n_chunks * kDecPartFloats * sizeof(float);
+}
+
+laser_kv_status_t laser_kv_decode_attention(laser_kv_handle_t h, int32_t layer, const void* Q_dec,
+                                            const int64_t q_strides[2], float softmax_scale, float* out,
+                                            void* scratch, size_t scratch_bytes, void* stream) {
+  if (!h) return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "decode_attention: NULL handle");
+  if (!Q_dec || !q_strides || !out || !scratch) return fail(h, LASER_KV_ERR_INVALID_ARG, "decode_attention: NULL argument");
+  const laser_kv_config_t& c = h->cfg;
+  const Derived& d = h->d;
+  if (layer < 0 || layer >= c.n_layers) return fail(h, LASER_KV_ERR_INVALID_ARG, "decode_attention: layer %d out of range", layer);
+  if (!aligned16(Q_dec) || !aligned16(out) || !aligned16(scratch))
+    return fail(h, LASER_KV_ERR_ALIGNMENT, "decode_attention: device pointers must be 16-byte aligned");
+  if (q_strides[0] < 0 || q_strides[1] < 0 || (q_strides[0] % 8) || (q_strides[1] % 8))
+    return fail(h, LASER_KV_ERR_ALIGNMENT, "decode_attention: strides must be non-negative multiples of 8 elements");
+  if (softmax_scale < 0.f || softmax_scale != softmax_scale)
+    return fail(h, LASER_KV_ERR_INVALID_ARG, "decode_attention: softmax_scale must be positive (0 selects the configured scale)");
+  const int G = c.n_q_heads / c.n_kv_heads;
+  if (G > kDecMaxGroup) return fail(h, LASER_KV_ERR_UNSUPPORTED, "decode_attention: more than %d query heads per KV head", kDecMaxGroup);
+  const long long len = h->blocks_done[layer] * d.B;
+  if (len < 1) return fail(h, LASER_KV_ERR_STATE, "decode_attention: layer %d cache is empty", layer);
+  const long long n_chunks = (len + kDecChunk - 1) / kDecChunk;
+  if (n_chunks > kDecMaxChunks) return fail(h, LASER_KV_ERR_UNSUPPORTED, "decode_attention: cache longer than %d entries", kDecMaxChunks * kDecChunk);
+  const size_t need = (size_t)c.batch * c.n_q_heads * n_chunks * kDecPartFloats * sizeof(float);
+  if (scratch_bytes < need) return fail(h, LASER_KV_ERR_CAPACITY, "decode_attention: scratch needs %zu bytes, got %zu", need, scratch_bytes);
+
+  const size_t layer_off = (size_t)layer * c.batch * c.n_kv_heads * (size_t)d.cap * kHeadDim;
+  DecodeArgs a;
+  a.Kc = h->cacheK + layer_off;
+  a.Vc = h->cacheV + layer_off;
+  a.seg_stride = (long long)d.cap * kHeadDim;
+  a.Q = static_cast<const uint16_t*>(Q_dec);
+  a.qs_b = q_strides[0];
+  a.qs_h = q_strides[1];
+  a.part = static_cast<float*>(scratch);
+  a.out = out;
+  a.H_kv = c.n_kv_heads;
+  a.G = G;
+  a.len = (int)len;
+  a.n_chunks = (int)n_chunks;
+  a.scale_log2e = (softmax_scale == 0.f ? d.scale : softmax_scale) * 1.4426950408889634f;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const dim3 grid((unsigned)n_chunks, (unsigned)c.n_kv_heads, (unsigned)c.batch);
+  if (G == 1) decode_chunk_kernel<1><<<grid, kDecThreads, 0, st>>>(a);
+  else if (G == 2) decode_chunk_kernel<2><<<grid, kDecThreads, 0, st>>>(a);
+  else if (G <= 4) decode_chunk_kernel<4><<<grid, kDecThreads, 0, st>>>(a);
+  else decode_chunk_kernel<8><<<grid, kDecThreads, 0, st>>>(a);
+  g_launches.fetch_add(1);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(h, LASER_KV_ERR_CUDA, "decode_chunk_kernel launch: %s", cudaGetErrorString(e));
+  decode_combine_kernel<<<dim3((unsigned)c.n_q_heads, (unsigned)c.batch), 128, 0, st>>>(a);
+  g_launches.fetch_add(1);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(h, LASER_KV_ERR_CUDA, "decode_combine_kernel launch: %s", cudaGetErrorString(e));
   return LASER_KV_OK;
 }
 
