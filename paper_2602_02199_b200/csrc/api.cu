@@ -316,6 +316,34 @@ laser_kv_status_t launch_append(const AppendArgs& a, int n_seg, cudaStream_t st)
   return LASER_KV_OK;
 }
 
+
+// Splits per (sequence, KV head) of a decode call: as many as fill the GPU's resident CTAs once,
+// never more than tiles in the cache.
+struct DecodeGeom { int sets, ctas_per_sm; };
+DecodeGeom decode_geom(int G) { return G <= 4 ? DecodeGeom{1, 2} : DecodeGeom{2, 1}; }
+int decode_splits(const laser_kv_ctx* h, long long len) {
+  const laser_kv_config_t& c = h->cfg;
+  const DecodeGeom g = decode_geom(c.n_q_heads / c.n_kv_heads);
+  long long n = (long long)h->num_sms * g.ctas_per_sm / ((long long)c.batch * c.n_kv_heads);
+  const long long tiles = (len + kDecTile - 1) / kDecTile;
+  if (n > tiles) n = tiles;
+  if (n > kDecMaxSplit) n = kDecMaxSplit;
+  return n < 1 ? 1 : (int)n;
+}
+
+template <int GT, int NSET, int NS>
+cudaError_t launch_decode_split(const DecodeArgs& a, dim3 grid, cudaStream_t st) {
+  constexpr uint32_t smem = dec_smem_bytes(GT, NSET, NS);
+  static bool configured = false;       // per instantiation; the attribute is idempotent
+  if (!configured) {
+    const cudaError_t e = cudaFuncSetAttribute(decode_split_kernel<GT, NSET, NS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  decode_split_kernel<GT, NSET, NS><<<grid, kDecSetThreads * NSET, smem, st>>>(a);
+  return cudaGetLastError();
+}
+
 }  // namespace
 
 extern "C" {
@@ -656,11 +684,11 @@ laser_kv_status_t laser_kv_cache_view(laser_kv_handle_t h, int32_t layer, laser_
   return LASER_KV_OK;
 }
 
+
 size_t laser_kv_decode_attention_scratch_bytes(laser_kv_handle_t h) {
   if (!h) return 0;
   const laser_kv_config_t& c = h->cfg;
-  const long long n_chunks = ((long long)h->d.cap + kDecChunk - 1) / kDecChunk;
-  return (size_t)c.batch * c.n_q_heads * n_chunks * kDecPartFloats * sizeof(float);
+  return (size_t)c.batch * c.n_q_heads * decode_splits(h, h->d.cap) * kDecPartFloats * sizeof(float);
 }
 
 laser_kv_status_t laser_kv_decode_attention(laser_kv_handle_t h, int32_t layer, const void* Q_dec,
@@ -681,9 +709,9 @@ laser_kv_status_t laser_kv_decode_attention(laser_kv_handle_t h, int32_t layer, 
   if (G > kDecMaxGroup) return fail(h, LASER_KV_ERR_UNSUPPORTED, "decode_attention: more than %d query heads per KV head", kDecMaxGroup);
   const long long len = h->blocks_done[layer] * d.B;
   if (len < 1) return fail(h, LASER_KV_ERR_STATE, "decode_attention: layer %d cache is empty", layer);
-  const long long n_chunks = (len + kDecChunk - 1) / kDecChunk;
-  if (n_chunks > kDecMaxChunks) return fail(h, LASER_KV_ERR_UNSUPPORTED, "decode_attention: cache longer than %d entries", kDecMaxChunks * kDecChunk);
-  const size_t need = (size_t)c.batch * c.n_q_heads * n_chunks * kDecPartFloats * sizeof(float);
+  if (len > 0x7fffffffLL) return fail(h, LASER_KV_ERR_UNSUPPORTED, "decode_attention: cache longer than 2^31 entries");
+  const int n_split = decode_splits(h, len);
+  const size_t need = (size_t)c.batch * c.n_q_heads * n_split * kDecPartFloats * sizeof(float);
   if (scratch_bytes < need) return fail(h, LASER_KV_ERR_CAPACITY, "decode_attention: scratch needs %zu bytes, got %zu", need, scratch_bytes);
 
   const size_t layer_off = (size_t)layer * c.batch * c.n_kv_heads * (size_t)d.cap * kHeadDim;
@@ -699,17 +727,18 @@ laser_kv_status_t laser_kv_decode_attention(laser_kv_handle_t h, int32_t layer, 
   a.H_kv = c.n_kv_heads;
   a.G = G;
   a.len = (int)len;
-  a.n_chunks = (int)n_chunks;
+  a.n_split = n_split;
   a.scale_log2e = (softmax_scale == 0.f ? d.scale : softmax_scale) * 1.4426950408889634f;
+  a.status = reinterpret_cast<int*>(h->ws + h->carve.ctrl);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const dim3 grid((unsigned)n_chunks, (unsigned)c.n_kv_heads, (unsigned)c.batch);
-  if (G == 1) decode_chunk_kernel<1><<<grid, kDecThreads, 0, st>>>(a);
-  else if (G == 2) decode_chunk_kernel<2><<<grid, kDecThreads, 0, st>>>(a);
-  else if (G <= 4) decode_chunk_kernel<4><<<grid, kDecThreads, 0, st>>>(a);
-  else decode_chunk_kernel<8><<<grid, kDecThreads, 0, st>>>(a);
+  const dim3 grid((unsigned)n_split, (unsigned)c.n_kv_heads, (unsigned)c.batch);
+  cudaError_t e;
+  if (G == 1) e = launch_decode_split<1, 1, 3>(a, grid, st);
+  else if (G == 2) e = launch_decode_split<2, 1, 3>(a, grid, st);
+  else if (G <= 4) e = launch_decode_split<4, 1, 3>(a, grid, st);
+  else e = launch_decode_split<4, 2, 4>(a, grid, st);
   g_launches.fetch_add(1);
-  cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess) return fail(h, LASER_KV_ERR_CUDA, "decode_chunk_kernel launch: %s", cudaGetErrorString(e));
+  if (e != cudaSuccess) return fail(h, LASER_KV_ERR_CUDA, "decode_split_kernel launch: %s", cudaGetErrorString(e));
   decode_combine_kernel<<<dim3((unsigned)c.n_q_heads, (unsigned)c.batch), 128, 0, st>>>(a);
   g_launches.fetch_add(1);
   e = cudaGetLastError();

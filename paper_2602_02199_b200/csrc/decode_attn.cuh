@@ -2,27 +2,33 @@
 // in the KV cache and are used for the decoding phase): for every sequence and query head,
 //   out = sum_i softmax_i(<q, k_i> * scale) * v_i     over the cache entries i in [0, len)
 // of the query head's KV head. The cache is read once (K and V rows, 256 bytes each): the op is
-// bound by HBM bandwidth, so the kernels are plain CUDA-core code shaped for coalesced 16-byte
-// loads, with all query heads of a GQA group sharing every row that is read.
+// bound by HBM bandwidth, so the arithmetic is plain CUDA-core code fed from shared memory by a
+// ring of bulk copies, and all query heads of a GQA group share every row that is read.
 //
-//   decode_chunk_kernel   - one CTA per (chunk of cache entries, KV head, sequence): scores of the
-//                           chunk for the G query heads of the group, softmax numerators relative
-//                           to the chunk's own maximum, weighted sum of the chunk's V rows ->
-//                           partial (max, sum, G x 128 accumulator) per chunk.
-//   decode_combine_kernel - merges the chunks' partials per query head (fixed order).
+//   decode_split_kernel   - one CTA per (split of the cache entries, KV head, sequence); the number
+//                           of splits fills the GPU exactly once. Tiles of 64 K rows and 64 V rows
+//                           arrive through cp.async.bulk into a ring of stages; per tile: scores
+//                           of the G query heads, softmax numerators relative to a running
+//                           reference maximum (raised only when a score exceeds it by 2^20, so the
+//                           common tile needs one barrier), weighted sum of the V rows.
+//                           -> partial (reference max, sum, G x 128 accumulator) per split.
+//   decode_combine_kernel - merges the splits' partials per query head (fixed order).
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "ptx.cuh"
+#include "stream_gemm.cuh"
+
 namespace lkv {
 
-constexpr int kDecThreads = 256;
-constexpr int kDecWarps = kDecThreads / 32;
-constexpr int kDecChunk = 512;          // cache entries per CTA
-constexpr int kDecMaxGroup = 8;         // query heads per KV head, at most
-constexpr int kDecPartFloats = 128 + 2; // per (chunk, query head): accumulator, max, sum
-constexpr int kDecMaxChunks = 2048;     // 1 Mi cache entries per head
-constexpr int kDecRowsInFlight = 4;     // rows a half-warp requests before it starts computing
+constexpr int kDecTile = 64;            // cache rows per stage (16 KB of K and 16 KB of V)
+constexpr int kDecTileBytes = kDecTile * 256;
+constexpr int kDecSetThreads = 256;     // threads that work on one set of up to four query heads
+constexpr int kDecMaxGroup = 8;         // query heads per KV head, at most (two sets of four)
+constexpr int kDecPartFloats = 128 + 2; // per (split, query head): accumulator, reference max, sum
+constexpr int kDecMaxSplit = 512;
+constexpr float kDecRescaleAt = 20.f;   // log2 units a score may exceed the reference maximum by
 
 struct DecodeArgs {
   const uint16_t* Kc;     // cache keys   [batch][H_kv][cap][128]
@@ -30,10 +36,11 @@ struct DecodeArgs {
   long long seg_stride;   // elements between (sequence, KV head) slabs
   const uint16_t* Q;      // decode queries [batch][H_q][128] via strides
   long long qs_b, qs_h;
-  float* part;            // [batch][H_kv][n_chunks][G][130]
+  float* part;            // [batch][H_kv][n_split][G][130]
   float* out;             // [batch][H_q][128]
-  int H_kv, G, len, n_chunks;
+  int H_kv, G, len, n_split;
   float scale_log2e;
+  int* status;
 };
 
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
@@ -43,58 +50,112 @@ __device__ __forceinline__ void unpack8(const uint4& w, float* x) {
   x[4] = bf16_lo(w.z); x[5] = bf16_hi(w.z); x[6] = bf16_lo(w.w); x[7] = bf16_hi(w.w);
 }
 
-// GT = query heads per KV head rounded up to a power of two (register arrays are sized by it).
-template <int GT>
-__global__ void __launch_bounds__(kDecThreads, GT <= 4 ? 4 : 2) decode_chunk_kernel(const DecodeArgs a) {
-  __shared__ float sc[GT][kDecChunk];                              // scores, then softmax numerators
-  __shared__ float red[kDecWarps / 2][GT][128];                    // output accumulators of warp pairs
-  __shared__ float stat[GT][2];                                    // chunk max and sum per query head
-  const int chunk = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int l16 = lane & 15, half = lane >> 4;                     // 16 lanes share one cache row
-  const int e0 = chunk * kDecChunk;
-  const int n_e = min(kDecChunk, a.len - e0);
-  const uint16_t* Kb = a.Kc + (long long)(b * a.H_kv + h) * a.seg_stride + (long long)e0 * 128 + l16 * 8;
-  const uint16_t* Vb = a.Vc + (long long)(b * a.H_kv + h) * a.seg_stride + (long long)e0 * 128 + l16 * 8;
-  constexpr int kStep = 2 * kDecWarps;                             // rows per pass of the CTA
+// Shared memory of one CTA: NS stages of (K tile, V tile), then the small arrays.
+__host__ __device__ constexpr uint32_t dec_smem_bytes(int gt, int nset, int ns) {
+  return (uint32_t)ns * 2u * kDecTileBytes            // stages
+         + 2u * 2u * (gt * nset) * kDecTile * 4u      // scores and numerators, double-buffered
+         + 2u * (gt * nset) * 4u                      // reference maxima, rescale factors
+         + (uint32_t)nset * 8u * gt * 4u              // per-warp sums of numerators
+         + (uint32_t)ns * 8u + 16u;                   // mbarriers, failure flag
+}
 
-  // this lane's 8 dims of every query of the group
+// GT = query heads per set (1, 2 or 4; register arrays are sized by it), NSET = sets (1 or 2; a
+// set is 8 warps that walk every tile for their own heads), NS = stages of the ring.
+template <int GT, int NSET, int NS>
+__global__ void __launch_bounds__(kDecSetThreads * NSET, NSET == 1 ? 2 : 1) decode_split_kernel(const DecodeArgs a) {
+  extern __shared__ __align__(128) uint8_t dsm[];
+  constexpr int NH = GT * NSET;
+  constexpr int NT = kDecSetThreads * NSET;
+  uint8_t* tiles = dsm;
+  float* sc_s = reinterpret_cast<float*>(dsm + NS * 2 * kDecTileBytes);   // [2][NH][64] scaled scores
+  float* sc_p = sc_s + 2 * NH * kDecTile;                                  // [2][NH][64] numerators
+  float* m_ref = sc_p + 2 * NH * kDecTile;                                 // [NH]
+  float* fac = m_ref + NH;                                                 // [NH]
+  float* lred = fac + NH;                                                  // [NSET*8][GT]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(lred + NSET * 8 * GT);      // [NS]
+  volatile int* failed = reinterpret_cast<volatile int*>(bars + NS);
+
+  const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int set = warp >> 3, wset = warp & 7;
+  const int l16 = lane & 15, half = lane >> 4;                     // 16 lanes share one cache row
+  const int hw = wset * 2 + half;                                  // half-warp within the set
+  const int e_begin = (int)((long long)split * a.len / a.n_split);
+  const int n_rows = (int)((long long)(split + 1) * a.len / a.n_split) - e_begin;
+  const int n_tiles = (n_rows + kDecTile - 1) / kDecTile;
+  const uint16_t* Kb = a.Kc + (long long)(b * a.H_kv + h) * a.seg_stride + (long long)e_begin * 128;
+  const uint16_t* Vb = a.Vc + (long long)(b * a.H_kv + h) * a.seg_stride + (long long)e_begin * 128;
+
+  if (tid == 0) {
+    for (int s = 0; s < NS; ++s) mbar_init(smem_u32(&bars[s]), 1);
+    fence_mbar_init();
+    *failed = 0;
+  }
+  if (tid < NH) m_ref[tid] = -INFINITY;
+  __syncthreads();
+  auto issue = [&](int t) {                                        // one thread: both copies of tile t
+    const int st = t % NS;
+    const uint32_t bytes = (uint32_t)min(kDecTile, n_rows - t * kDecTile) * 256u;
+    const uint32_t bar = smem_u32(&bars[st]);
+    mbar_expect_tx(bar, 2u * bytes);
+    bulk_load(smem_u32(tiles + st * 2 * kDecTileBytes), Kb + (long long)t * kDecTile * 128, bytes, bar);
+    bulk_load(smem_u32(tiles + st * 2 * kDecTileBytes + kDecTileBytes), Vb + (long long)t * kDecTile * 128, bytes, bar);
+  };
+  if (tid == 0)
+    for (int t = 0; t < NS - 1 && t < n_tiles; ++t) issue(t);
+
+  // this lane's 8 dims of every query of the set
   float q[GT][8];
 #pragma unroll
   for (int g = 0; g < GT; ++g) {
-    if (g < a.G) {
-      unpack8(*reinterpret_cast<const uint4*>(a.Q + b * a.qs_b + (long long)(h * a.G + g) * a.qs_h + l16 * 8), q[g]);
+    if (set * GT + g < a.G) {
+      unpack8(*reinterpret_cast<const uint4*>(a.Q + b * a.qs_b + (long long)(h * a.G + set * GT + g) * a.qs_h + l16 * 8), q[g]);
     } else {
 #pragma unroll
       for (int i = 0; i < 8; ++i) q[g][i] = 0.f;
     }
   }
+  float2 acc[GT][4];
+  float lsum[GT];
+#pragma unroll
+  for (int g = 0; g < GT; ++g) {
+    lsum[g] = 0.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) acc[g][i] = make_float2(0.f, 0.f);
+  }
 
-  // ---- scores: a half-warp per row; several rows are requested before the first is used ----------
-  for (int eb = warp * 2 + half; eb < kDecChunk; eb += kStep * kDecRowsInFlight) {
-    uint4 w[kDecRowsInFlight];
+  bool alive = true;
+  for (int t = 0; t < n_tiles; ++t) {
+    const int st = t % NS, buf = t & 1;
+    const int rows_here = min(kDecTile, n_rows - t * kDecTile);
+    const uint8_t* kt = tiles + st * 2 * kDecTileBytes + l16 * 16;
+    const uint8_t* vt = kt + kDecTileBytes;
+    float* s_buf = sc_s + buf * NH * kDecTile;
+    float* p_buf = sc_p + buf * NH * kDecTile;
+    bool flag = false;
+    if (!mbar_wait(smem_u32(&bars[st]), (uint32_t)(t / NS) & 1u)) { *failed = 1; flag = true; }
+
+    // ---- scores: a half-warp per row, four rows per half-warp ----------------------------------
+    uint4 w[4];
 #pragma unroll
-    for (int r = 0; r < kDecRowsInFlight; ++r) {
-      const int e = eb + r * kStep;
-      w[r] = (e < n_e) ? *reinterpret_cast<const uint4*>(Kb + (long long)e * 128) : make_uint4(0u, 0u, 0u, 0u);
-    }
+    for (int r = 0; r < 4; ++r) w[r] = *reinterpret_cast<const uint4*>(kt + (hw + 16 * r) * 256);
 #pragma unroll
-    for (int r = 0; r < kDecRowsInFlight; ++r) {
-      const int e = eb + r * kStep;
+    for (int r = 0; r < 4; ++r) {
+      const int row = hw + 16 * r;
       float k[8];
       unpack8(w[r], k);
       float s[GT];
 #pragma unroll
       for (int g = 0; g < GT; ++g) {
-        float2 t = make_float2(0.f, 0.f);
+        float2 x = make_float2(0.f, 0.f);
 #pragma unroll
         for (int i = 0; i < 8; i += 2)
-          t = __ffma2_rn(make_float2(k[i], k[i + 1]), make_float2(q[g][i], q[g][i + 1]), t);
-        s[g] = t.x + t.y;
+          x = __ffma2_rn(make_float2(k[i], k[i + 1]), make_float2(q[g][i], q[g][i + 1]), x);
+        s[g] = x.x + x.y;
       }
       // sum over the row's 16 lanes; while more than one head is left, each step also halves the
       // heads a lane keeps, so that the lane ends up with the full sum of one head
-      int mine = 0;                                 // the head this lane will hold
+      int mine = 0;
       int left = GT;
 #pragma unroll
       for (int off = 8; off > 0; off >>= 1) {
@@ -115,114 +176,136 @@ __global__ void __launch_bounds__(kDecThreads, GT <= 4 ? 4 : 2) decode_chunk_ker
         }
       }
       // lanes that hold the same head hold the same sum; the lowest of them stores it
-      constexpr int kDup = GT >= 16 ? 1 : 16 / GT;  // lanes per head after the reduction
-      if ((l16 & (kDup - 1)) == 0 && mine < a.G) sc[mine][e] = (e < n_e) ? s[0] * a.scale_log2e : -INFINITY;
+      constexpr int kDup = 16 / GT;
+      const int head = set * GT + mine;
+      if ((l16 & (kDup - 1)) == 0 && head < a.G) {
+        const float sv = row < rows_here ? s[0] * a.scale_log2e : -INFINITY;   // stale rows of a short tile
+        const float m = m_ref[head];
+        s_buf[head * kDecTile + row] = sv;
+        p_buf[head * kDecTile + row] = exp2f(sv - m);
+        flag |= sv > m + kDecRescaleAt;
+      }
     }
-  }
-  __syncthreads();
-
-  // ---- softmax numerators relative to the chunk's maximum: warp g takes query head g ---------------
-  for (int g = warp; g < a.G; g += kDecWarps) {
-    float m = -INFINITY;
-    for (int e = lane; e < kDecChunk; e += 32) m = fmaxf(m, sc[g][e]);
+    const int any = __syncthreads_or(flag);
+    // every thread is past the V rows of tile t-1: its stage takes tile t+NS-1
+    if (tid == 0 && t + NS - 1 < n_tiles) issue(t + NS - 1);
+    if (any) {
+      if (*failed) { alive = false; break; }                       // uniform: read after the barrier
+      // raise the reference maxima to the tile's maxima: warp g redoes head g's numerators
+      if (warp < a.G) {
+        const float s0 = s_buf[warp * kDecTile + lane], s1 = s_buf[warp * kDecTile + lane + 32];
+        float tm = fmaxf(s0, s1);
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
-    float l = 0.f;
-    for (int e = lane; e < kDecChunk; e += 32) {
-      const float p = exp2f(sc[g][e] - m);          // n_e >= 1, so m is finite
-      sc[g][e] = p;
-      l += p;
-    }
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) l += __shfl_xor_sync(0xffffffffu, l, off);
-    if (lane == 0) { stat[g][0] = m; stat[g][1] = l; }
-  }
-  __syncthreads();
-
-  // ---- weighted sum of the chunk's V rows: the lane keeps 8 dims for each head of the group --------
-  float2 acc[GT][4];
-#pragma unroll
-  for (int g = 0; g < GT; ++g)
-#pragma unroll
-    for (int i = 0; i < 4; ++i) acc[g][i] = make_float2(0.f, 0.f);
-  for (int eb = warp * 2 + half; eb < kDecChunk; eb += kStep * kDecRowsInFlight) {
-    uint4 w[kDecRowsInFlight];
-#pragma unroll
-    for (int r = 0; r < kDecRowsInFlight; ++r) {
-      const int e = eb + r * kStep;
-      w[r] = (e < n_e) ? *reinterpret_cast<const uint4*>(Vb + (long long)e * 128) : make_uint4(0u, 0u, 0u, 0u);
-    }
-#pragma unroll
-    for (int r = 0; r < kDecRowsInFlight; ++r) {
-      const int e = eb + r * kStep;                 // e < kDecChunk always; rows past n_e have p = 0
-      float v[8];
-      unpack8(w[r], v);
+        for (int off = 16; off > 0; off >>= 1) tm = fmaxf(tm, __shfl_xor_sync(0xffffffffu, tm, off));
+        const float m_old = m_ref[warp];
+        const float m_new = fmaxf(m_old, tm);                      // finite: the tile has a valid row
+        p_buf[warp * kDecTile + lane] = exp2f(s0 - m_new);
+        p_buf[warp * kDecTile + lane + 32] = exp2f(s1 - m_new);
+        __syncwarp();
+        if (lane == 0) { fac[warp] = exp2f(m_old - m_new); m_ref[warp] = m_new; }
+      }
+      __syncthreads();
 #pragma unroll
       for (int g = 0; g < GT; ++g) {
-        if (g < a.G) {
-          const float p = sc[g][e];
-          const float2 pp = make_float2(p, p);
+        if (set * GT + g < a.G) {
+          const float f = fac[set * GT + g];
+          lsum[g] *= f;
 #pragma unroll
-          for (int i = 0; i < 4; ++i) acc[g][i] = __ffma2_rn(pp, make_float2(v[2 * i], v[2 * i + 1]), acc[g][i]);
+          for (int i = 0; i < 4; ++i) { acc[g][i].x *= f; acc[g][i].y *= f; }
+        }
+      }
+    }
+
+    // ---- weighted sum of the tile's V rows: the lane keeps 8 dims for each head of the set ------
+#pragma unroll
+    for (int r = 0; r < 4; ++r) w[r] = *reinterpret_cast<const uint4*>(vt + (hw + 16 * r) * 256);
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      const int row = hw + 16 * r;
+      if (row < rows_here) {                                       // stale rows may hold anything
+        float v[8];
+        unpack8(w[r], v);
+#pragma unroll
+        for (int g = 0; g < GT; ++g) {
+          if (set * GT + g < a.G) {
+            const float p = p_buf[(set * GT + g) * kDecTile + row];
+            const float2 pp = make_float2(p, p);
+            lsum[g] += p;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) acc[g][i] = __ffma2_rn(pp, make_float2(v[2 * i], v[2 * i + 1]), acc[g][i]);
+          }
         }
       }
     }
   }
+  if (!alive) {                                                    // a copy never arrived: report, write nothing
+    if (tid == 0) record_status(a.status, kStatusTimeout);
+    return;
+  }
+  __syncthreads();                                                 // every tile is consumed: the stages are free
+
   // the two half-warps of a warp hold different rows of the same dims
 #pragma unroll
-  for (int g = 0; g < GT; ++g)
+  for (int g = 0; g < GT; ++g) {
+    lsum[g] += __shfl_xor_sync(0xffffffffu, lsum[g], 16);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       acc[g][i].x += __shfl_xor_sync(0xffffffffu, acc[g][i].x, 16);
       acc[g][i].y += __shfl_xor_sync(0xffffffffu, acc[g][i].y, 16);
     }
-  // across warps in two rounds (odd warps write, even warps add; then the four sums are added)
-  if ((warp & 1) && half == 0) {
+  }
+  float* red = reinterpret_cast<float*>(tiles);                    // [NSET*8 warps][GT][128]
+  if (half == 0) {
 #pragma unroll
-    for (int g = 0; g < GT; ++g)
+    for (int g = 0; g < GT; ++g) {
+      float4* dst = reinterpret_cast<float4*>(red + (warp * GT + g) * 128 + l16 * 8);
+      dst[0] = make_float4(acc[g][0].x, acc[g][0].y, acc[g][1].x, acc[g][1].y);
+      dst[1] = make_float4(acc[g][2].x, acc[g][2].y, acc[g][3].x, acc[g][3].y);
+    }
+    if (l16 == 0) {
 #pragma unroll
-      for (int i = 0; i < 4; ++i)
-        *reinterpret_cast<float2*>(&red[warp >> 1][g][l16 * 8 + 2 * i]) = acc[g][i];
+      for (int g = 0; g < GT; ++g) lred[warp * GT + g] = lsum[g];
+    }
   }
   __syncthreads();
-  if (!(warp & 1) && half == 0) {
+  float* part = a.part + (((long long)(b * a.H_kv + h) * a.n_split + split) * a.G) * kDecPartFloats;
+  for (int i = tid; i < a.G * 128; i += NT) {
+    const int head = i >> 7, d = i & 127;
+    const float* src = red + ((head / GT) * 8 * GT + head % GT) * 128 + d;   // warp 0 of the head's set
+    float sum = 0.f;
 #pragma unroll
-    for (int g = 0; g < GT; ++g)
+    for (int wi = 0; wi < 8; ++wi) sum += src[wi * GT * 128];
+    part[head * kDecPartFloats + d] = sum;
+  }
+  if (tid < a.G) {
+    const float* src = lred + (tid / GT) * 8 * GT + tid % GT;
+    float l = 0.f;
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        float2* slot = reinterpret_cast<float2*>(&red[warp >> 1][g][l16 * 8 + 2 * i]);
-        const float2 o = *slot;
-        *slot = make_float2(acc[g][i].x + o.x, acc[g][i].y + o.y);
-      }
+    for (int wi = 0; wi < 8; ++wi) l += src[wi * GT];
+    part[tid * kDecPartFloats + 128] = m_ref[tid];
+    part[tid * kDecPartFloats + 129] = l;
   }
-  __syncthreads();
-  float* part = a.part + (((long long)(b * a.H_kv + h) * a.n_chunks + chunk) * a.G) * kDecPartFloats;
-  for (int i = threadIdx.x; i < a.G * 128; i += kDecThreads) {
-    const int g = i >> 7, d = i & 127;
-    part[g * kDecPartFloats + d] = (red[0][g][d] + red[1][g][d]) + (red[2][g][d] + red[3][g][d]);
-  }
-  if (threadIdx.x < a.G * 2) part[(threadIdx.x >> 1) * kDecPartFloats + 128 + (threadIdx.x & 1)] = stat[threadIdx.x >> 1][threadIdx.x & 1];
 }
 
-// One CTA of 128 threads per (query head, sequence): thread d merges dim d over the chunks.
+// One CTA of 128 threads per (query head, sequence): thread d merges dim d over the splits.
 __global__ void __launch_bounds__(128) decode_combine_kernel(const DecodeArgs a) {
-  __shared__ float wgt[kDecMaxChunks];
+  __shared__ float wgt[kDecMaxSplit];
   __shared__ float red_m[4], red_l[4];
   const int hq = blockIdx.x, b = blockIdx.y;
   const int h = hq / a.G, g = hq % a.G;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const float* part = a.part + (((long long)(b * a.H_kv + h) * a.n_chunks) * a.G + g) * kDecPartFloats;
-  const long long cstride = (long long)a.G * kDecPartFloats;
+  const float* part = a.part + (((long long)(b * a.H_kv + h) * a.n_split) * a.G + g) * kDecPartFloats;
+  const int cstride = a.G * kDecPartFloats;
 
   float m = -INFINITY;
-  for (int c = threadIdx.x; c < a.n_chunks; c += 128) m = fmaxf(m, part[c * cstride + 128]);
+  for (int c = threadIdx.x; c < a.n_split; c += 128) m = fmaxf(m, part[c * cstride + 128]);
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
   if (lane == 0) red_m[warp] = m;
   __syncthreads();
   m = fmaxf(fmaxf(red_m[0], red_m[1]), fmaxf(red_m[2], red_m[3]));
   float l = 0.f;
-  for (int c = threadIdx.x; c < a.n_chunks; c += 128) {
+  for (int c = threadIdx.x; c < a.n_split; c += 128) {
     const float wc = exp2f(part[c * cstride + 128] - m);
     wgt[c] = wc;
     l += wc * part[c * cstride + 129];
@@ -234,16 +317,18 @@ __global__ void __launch_bounds__(128) decode_combine_kernel(const DecodeArgs a)
   l = (red_l[0] + red_l[1]) + (red_l[2] + red_l[3]);
 
   const int d = threadIdx.x;
-  float o0 = 0.f, o1 = 0.f, o2 = 0.f, o3 = 0.f;
-  int c = 0;
-  for (; c + 4 <= a.n_chunks; c += 4) {
-    o0 = fmaf(wgt[c], part[c * cstride + d], o0);
-    o1 = fmaf(wgt[c + 1], part[(c + 1) * cstride + d], o1);
-    o2 = fmaf(wgt[c + 2], part[(c + 2) * cstride + d], o2);
-    o3 = fmaf(wgt[c + 3], part[(c + 3) * cstride + d], o3);
+  float o[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) o[j] = 0.f;
+  for (int c0 = 0; c0 < a.n_split; c0 += 8) {
+    float x[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) x[j] = c0 + j < a.n_split ? part[(c0 + j) * cstride + d] : 0.f;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) o[j] = fmaf(c0 + j < a.n_split ? wgt[c0 + j] : 0.f, x[j], o[j]);
   }
-  for (; c < a.n_chunks; ++c) o0 = fmaf(wgt[c], part[c * cstride + d], o0);
-  a.out[((long long)b * a.H_kv * a.G + hq) * 128 + d] = ((o0 + o1) + (o2 + o3)) / l;
+  a.out[((long long)b * a.H_kv * a.G + hq) * 128 + d] =
+      (((o[0] + o[1]) + (o[2] + o[3])) + ((o[4] + o[5]) + (o[6] + o[7]))) / l;
 }
 
 }  // namespace lkv

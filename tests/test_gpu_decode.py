@@ -28,16 +28,20 @@ def _oracle_cache(w, run, b):
     return cache
 
 
-@pytest.mark.parametrize("name,S,nb,batch,strided", [
-    ("tiny", 520, 3, 1, True),            # G = 4, ragged last chunk (390 entries)
-    ("llama8b_32k", 1032, 2, 2, False),   # G = 4, several chunks
-    ("qwen7b_128k", 776, 3, 2, True),     # G = 7: the padded group of 8
+@pytest.mark.parametrize("name,S,nb,batch,budget,strided,scale", [
+    ("tiny", 520, 3, 1, None, True, None),             # G = 4, one ragged tile per split
+    ("llama8b_32k", 1032, 2, 2, None, False, None),    # G = 4, two sequences
+    ("qwen7b_128k", 776, 3, 2, None, True, None),      # G = 7: two sets of heads
+    # budget = block size keeps every token, so the kept set has no near-ties to depend on
+    ("tiny", 1016, 9, 1, 1016, False, None),           # several tiles per split: the ring wraps, ragged tail
+    ("qwen7b_128k", 1016, 12, 1, 1016, True, None),    # the same for two sets of heads
+    ("tiny", 1016, 9, 1, 1016, False, 6.0),            # logits hundreds apart: the reference maximum is raised late
 ])
-def test_decode_attention_against_oracle(name, S, nb, batch, strided):
+def test_decode_attention_against_oracle(name, S, nb, batch, budget, strided, scale):
     import torch
     w = synth.workload(name).with_(block_size=S, context_len=nb * S, batch=batch, n_layers=1, lsh_tables=16,
                                    needles="uniform:4")
-    run = run_workload_layer(w, 0, n_blocks=nb, debug=1)
+    run = run_workload_layer(w, 0, n_blocks=nb, debug=0, budget=budget)
     eng = run["engine"]
     rng = np.random.default_rng(1234)
     if strided:
@@ -47,7 +51,7 @@ def test_decode_attention_against_oracle(name, S, nb, batch, strided):
     else:
         q_bits = synth.f32_to_bf16_bits((rng.standard_normal((batch, w.n_q_heads, 128)) * 1.5).astype(np.float32))
         tq = torch.from_numpy(q_bits.view(np.int16)).cuda()
-    out = eng.laser_kv_decode_attention(0, tq)
+    out = eng.laser_kv_decode_attention(0, tq, softmax_scale=0.0 if scale is None else scale)
     eng.laser_kv_poll_status()
     got = to_np(out)
     _, _, pos, length = eng.laser_kv_cache_view(0)
@@ -59,7 +63,7 @@ def test_decode_attention_against_oracle(name, S, nb, batch, strided):
         assert cache.length == length
         assert (pos[b, :, :length] == cache.pos[:, :length]).all()       # same tokens kept, same order
         for h in range(w.n_kv_heads):
-            want = O.decode_attention(q_bits[b, h * G:(h + 1) * G], cache.K[h, :length], cache.V[h, :length])
+            want = O.decode_attention(q_bits[b, h * G:(h + 1) * G], cache.K[h, :length], cache.V[h, :length], scale=scale)
             err = np.abs(got[b, h * G:(h + 1) * G] - want)
             assert (err <= DEC_RTOL * np.abs(want) + DEC_ATOL).all(), (b, h, err.max())
 
