@@ -319,29 +319,13 @@ laser_kv_status_t launch_append(const AppendArgs& a, int n_seg, cudaStream_t st)
 
 // Splits per (sequence, KV head) of a decode call: as many as fill the GPU's resident CTAs once,
 // never more than tiles in the cache.
-struct DecodeGeom { int sets, ctas_per_sm; };
-DecodeGeom decode_geom(int G) { return G <= 4 ? DecodeGeom{1, 2} : DecodeGeom{2, 1}; }
 int decode_splits(const laser_kv_ctx* h, long long len) {
   const laser_kv_config_t& c = h->cfg;
-  const DecodeGeom g = decode_geom(c.n_q_heads / c.n_kv_heads);
-  long long n = (long long)h->num_sms * g.ctas_per_sm / ((long long)c.batch * c.n_kv_heads);
+  long long n = (long long)h->num_sms * kDecCtasPerSm / ((long long)c.batch * c.n_kv_heads);
   const long long tiles = (len + kDecTile - 1) / kDecTile;
   if (n > tiles) n = tiles;
   if (n > kDecMaxSplit) n = kDecMaxSplit;
   return n < 1 ? 1 : (int)n;
-}
-
-template <int GT, int NSET, int NS>
-cudaError_t launch_decode_split(const DecodeArgs& a, dim3 grid, cudaStream_t st) {
-  constexpr uint32_t smem = dec_smem_bytes(GT, NSET, NS);
-  static bool configured = false;       // per instantiation; the attribute is idempotent
-  if (!configured) {
-    const cudaError_t e = cudaFuncSetAttribute(decode_split_kernel<GT, NSET, NS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
-  decode_split_kernel<GT, NSET, NS><<<grid, kDecSetThreads * NSET, smem, st>>>(a);
-  return cudaGetLastError();
 }
 
 }  // namespace
@@ -715,10 +699,17 @@ laser_kv_status_t laser_kv_decode_attention(laser_kv_handle_t h, int32_t layer, 
   if (scratch_bytes < need) return fail(h, LASER_KV_ERR_CAPACITY, "decode_attention: scratch needs %zu bytes, got %zu", need, scratch_bytes);
 
   const size_t layer_off = (size_t)layer * c.batch * c.n_kv_heads * (size_t)d.cap * kHeadDim;
+  // the layer's cache as (d, len, H_kv, batch): rows past len read as zeros
+  CUtensorMap mapK, mapV;
+  {
+    const uint64_t dims[4] = {(uint64_t)kHeadDim, (uint64_t)len, (uint64_t)c.n_kv_heads, (uint64_t)c.batch};
+    const uint64_t strides[3] = {(uint64_t)kHeadDim * 2, (uint64_t)d.cap * kHeadDim * 2,
+                                 (uint64_t)c.n_kv_heads * d.cap * kHeadDim * 2};
+    const uint32_t box[4] = {64, (uint32_t)kDecTile, 1, 1};
+    if (!encode_map(h, &mapK, h->cacheK + layer_off, 4, dims, strides, box)) return LASER_KV_ERR_CUDA;
+    if (!encode_map(h, &mapV, h->cacheV + layer_off, 4, dims, strides, box)) return LASER_KV_ERR_CUDA;
+  }
   DecodeArgs a;
-  a.Kc = h->cacheK + layer_off;
-  a.Vc = h->cacheV + layer_off;
-  a.seg_stride = (long long)d.cap * kHeadDim;
   a.Q = static_cast<const uint16_t*>(Q_dec);
   a.qs_b = q_strides[0];
   a.qs_h = q_strides[1];
@@ -732,12 +723,16 @@ laser_kv_status_t laser_kv_decode_attention(laser_kv_handle_t h, int32_t layer, 
   a.status = reinterpret_cast<int*>(h->ws + h->carve.ctrl);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const dim3 grid((unsigned)n_split, (unsigned)c.n_kv_heads, (unsigned)c.batch);
-  cudaError_t e;
-  if (G == 1) e = launch_decode_split<1, 1, 3>(a, grid, st);
-  else if (G == 2) e = launch_decode_split<2, 1, 3>(a, grid, st);
-  else if (G <= 4) e = launch_decode_split<4, 1, 3>(a, grid, st);
-  else e = launch_decode_split<4, 2, 4>(a, grid, st);
+  static bool configured = false;       // the attribute is idempotent
+  cudaError_t e = cudaSuccess;
+  if (!configured) {
+    e = cudaFuncSetAttribute(decode_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dec_smem_bytes());
+    if (e != cudaSuccess) return fail(h, LASER_KV_ERR_CUDA, "decode_split_kernel attribute: %s", cudaGetErrorString(e));
+    configured = true;
+  }
+  decode_split_kernel<<<grid, kDecThreads, dec_smem_bytes(), st>>>(mapK, mapV, a);
   g_launches.fetch_add(1);
+  e = cudaGetLastError();
   if (e != cudaSuccess) return fail(h, LASER_KV_ERR_CUDA, "decode_split_kernel launch: %s", cudaGetErrorString(e));
   decode_combine_kernel<<<dim3((unsigned)c.n_q_heads, (unsigned)c.batch), 128, 0, st>>>(a);
   g_launches.fetch_add(1);

@@ -2,18 +2,26 @@
 // in the KV cache and are used for the decoding phase): for every sequence and query head,
 //   out = sum_i softmax_i(<q, k_i> * scale) * v_i     over the cache entries i in [0, len)
 // of the query head's KV head. The cache is read once (K and V rows, 256 bytes each): the op is
-// bound by HBM bandwidth, so the arithmetic is plain CUDA-core code fed from shared memory by a
-// ring of bulk copies, and all query heads of a GQA group share every row that is read.
+// bound by HBM bandwidth. All (up to eight) query heads of a GQA group share every row that is
+// read; the two small contractions per row (scores, weighted sum of V) run as warp-level
+// m16n8k16 bf16 MMAs with the heads on the 8-wide dimension, which keeps the instruction count
+// per row far below what the memory pipeline needs (a CUDA-core version of the same loop was
+// bound by instruction issue at half the bandwidth). tcgen05 would need M = 128 per instruction
+// and a round trip through TMEM and shared memory for the numerators; nothing is gained when the
+// tensor pipe is idle 95 % of the time either way.
 //
 //   decode_split_kernel   - one CTA per (split of the cache entries, KV head, sequence); the number
-//                           of splits fills the GPU exactly once. Tiles of 64 K rows and 64 V rows
-//                           arrive through cp.async.bulk into a ring of stages; per tile: scores
-//                           of the G query heads, softmax numerators relative to a running
-//                           reference maximum (raised only when a score exceeds it by 2^20, so the
-//                           common tile needs one barrier), weighted sum of the V rows.
-//                           -> partial (reference max, sum, G x 128 accumulator) per split.
+//                           of splits fills the GPU exactly once. A producer warp brings tiles of
+//                           64 K rows and 64 V rows into a ring of stages with TMA (128-byte
+//                           swizzle, rows past the cache length read as zeros); each of four
+//                           consumer warps owns 16 rows of every tile: scores S^T = K Q^T,
+//                           numerators relative to the warp's running reference maximum (raised
+//                           only when a score exceeds it by 2^20), O^T += V^T P^T with the
+//                           numerators split into two bf16 terms so that the weights keep
+//                           16 mantissa bits. -> partial (max, sum, G x 128 accumulator) per split.
 //   decode_combine_kernel - merges the splits' partials per query head (fixed order).
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -22,18 +30,20 @@
 
 namespace lkv {
 
-constexpr int kDecTile = 64;            // cache rows per stage (16 KB of K and 16 KB of V)
-constexpr int kDecTileBytes = kDecTile * 256;
-constexpr int kDecSetThreads = 256;     // threads that work on one set of up to four query heads
-constexpr int kDecMaxGroup = 8;         // query heads per KV head, at most (two sets of four)
+constexpr int kDecTile = 64;            // cache rows per stage
+constexpr int kDecBoxBytes = kDecTile * 128;   // one TMA box: 64 rows x 64 bf16
+constexpr int kDecStageBytes = 4 * kDecBoxBytes;   // K cols 0-63, K cols 64-127, V cols 0-63, V cols 64-127
+constexpr int kDecStages = 3;
+constexpr int kDecWarps = 4;            // consumer warps, 16 rows of every tile each
+constexpr int kDecThreads = (kDecWarps + 1) * 32;
+constexpr int kDecCtasPerSm = 2;
+constexpr int kDecMaxGroup = 8;         // query heads per KV head, at most (the N of the MMA)
 constexpr int kDecPartFloats = 128 + 2; // per (split, query head): accumulator, reference max, sum
 constexpr int kDecMaxSplit = 512;
 constexpr float kDecRescaleAt = 20.f;   // log2 units a score may exceed the reference maximum by
+constexpr int kDecRedStride = 132;      // floats between heads in the merge buffer (bank spread)
 
 struct DecodeArgs {
-  const uint16_t* Kc;     // cache keys   [batch][H_kv][cap][128]
-  const uint16_t* Vc;     // cache values [batch][H_kv][cap][128]
-  long long seg_stride;   // elements between (sequence, KV head) slabs
   const uint16_t* Q;      // decode queries [batch][H_q][128] via strides
   long long qs_b, qs_h;
   float* part;            // [batch][H_kv][n_split][G][130]
@@ -43,246 +53,212 @@ struct DecodeArgs {
   int* status;
 };
 
-__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
-__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
-__device__ __forceinline__ void unpack8(const uint4& w, float* x) {
-  x[0] = bf16_lo(w.x); x[1] = bf16_hi(w.x); x[2] = bf16_lo(w.y); x[3] = bf16_hi(w.y);
-  x[4] = bf16_lo(w.z); x[5] = bf16_hi(w.z); x[6] = bf16_lo(w.w); x[7] = bf16_hi(w.w);
+__host__ __device__ constexpr uint32_t dec_smem_bytes() {
+  return kDecStages * kDecStageBytes + 2u * kDecStages * 8u + 2u * kDecWarps * 8u * 4u + 1024u;
 }
 
-// Shared memory of one CTA: NS stages of (K tile, V tile), then the small arrays.
-__host__ __device__ constexpr uint32_t dec_smem_bytes(int gt, int nset, int ns) {
-  return (uint32_t)ns * 2u * kDecTileBytes            // stages
-         + 2u * 2u * (gt * nset) * kDecTile * 4u      // scores and numerators, double-buffered
-         + 2u * (gt * nset) * 4u                      // reference maxima, rescale factors
-         + (uint32_t)nset * 8u * gt * 4u              // per-warp sums of numerators
-         + (uint32_t)ns * 8u + 16u;                   // mbarriers, failure flag
+// Byte offset of the 16-byte chunk (0..15 over the 128 dims) of a row inside a K or V tile made
+// of two 128-byte-swizzled boxes.
+__device__ __forceinline__ uint32_t dec_swz(uint32_t row, uint32_t chunk) {
+  return (chunk >> 3) * kDecBoxBytes + row * 128u + (((chunk & 7u) ^ (row & 7u)) << 4);
+}
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t* r) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t addr, uint32_t* r) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr) : "memory");
+}
+// D (16x8, fp32) += A (16x16, bf16, row) * B (16x8, bf16, col)
+__device__ __forceinline__ void mma_bf16(float* d, const uint32_t* a, uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+// Transposes the 8x8 matrix of 16-bit elements that the warp holds one register per lane.
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x) {
+  uint32_t y;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(y) : "r"(x));
+  return y;
+}
+// (lo, hi) -> two bf16 (round to nearest even), lo in the low half
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  uint32_t y;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(y) : "f"(hi), "f"(lo));
+  return y;
 }
 
-// GT = query heads per set (1, 2 or 4; register arrays are sized by it), NSET = sets (1 or 2; a
-// set is 8 warps that walk every tile for their own heads), NS = stages of the ring.
-template <int GT, int NSET, int NS>
-__global__ void __launch_bounds__(kDecSetThreads * NSET, NSET == 1 ? 2 : 1) decode_split_kernel(const DecodeArgs a) {
-  extern __shared__ __align__(128) uint8_t dsm[];
-  constexpr int NH = GT * NSET;
-  constexpr int NT = kDecSetThreads * NSET;
-  uint8_t* tiles = dsm;
-  float* sc_s = reinterpret_cast<float*>(dsm + NS * 2 * kDecTileBytes);   // [2][NH][64] scaled scores
-  float* sc_p = sc_s + 2 * NH * kDecTile;                                  // [2][NH][64] numerators
-  float* m_ref = sc_p + 2 * NH * kDecTile;                                 // [NH]
-  float* fac = m_ref + NH;                                                 // [NH]
-  float* lred = fac + NH;                                                  // [NSET*8][GT]
-  uint64_t* bars = reinterpret_cast<uint64_t*>(lred + NSET * 8 * GT);      // [NS]
-  volatile int* failed = reinterpret_cast<volatile int*>(bars + NS);
+// MMA fragment coordinates of a lane: g = lane / 4 (a row of the 16-row operand, a column of B),
+// c = lane % 4 (the pair of columns 2c, 2c+1). Scores come out as S^T[key g (+8)][heads 2c, 2c+1];
+// the accumulators are O^T[dim 16 mt + g (+8)][heads 2c, 2c+1].
+__global__ void __launch_bounds__(kDecThreads, kDecCtasPerSm)
+decode_split_kernel(const __grid_constant__ CUtensorMap map_k,    // cache K: (d, len, H_kv, batch), box (64, 64, 1, 1)
+                    const __grid_constant__ CUtensorMap map_v,    // cache V, same shape
+                    const DecodeArgs a) {
+  extern __shared__ uint8_t dsm_raw[];
+  const uint32_t base = (smem_u32(dsm_raw) + 1023u) & ~1023u;
+  uint8_t* const gen = dsm_raw + (base - smem_u32(dsm_raw));
+  const uint32_t sm_bars = base + kDecStages * kDecStageBytes;
+  float* wm = reinterpret_cast<float*>(gen + kDecStages * kDecStageBytes + 2 * kDecStages * 8);   // [warps][8] maxima
+  float* wl = wm + kDecWarps * 8;                                                                   // [warps][8] sums
+  float* red = reinterpret_cast<float*>(gen);                     // merge buffer over the stages: [warps][8][132]
+  auto bar_full = [&](int s) { return sm_bars + 8u * s; };
+  auto bar_empty = [&](int s) { return sm_bars + 8u * (kDecStages + s); };
 
   const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int set = warp >> 3, wset = warp & 7;
-  const int l16 = lane & 15, half = lane >> 4;                     // 16 lanes share one cache row
-  const int hw = wset * 2 + half;                                  // half-warp within the set
+  const int g = lane >> 2, c = lane & 3;
   const int e_begin = (int)((long long)split * a.len / a.n_split);
   const int n_rows = (int)((long long)(split + 1) * a.len / a.n_split) - e_begin;
   const int n_tiles = (n_rows + kDecTile - 1) / kDecTile;
-  const uint16_t* Kb = a.Kc + (long long)(b * a.H_kv + h) * a.seg_stride + (long long)e_begin * 128;
-  const uint16_t* Vb = a.Vc + (long long)(b * a.H_kv + h) * a.seg_stride + (long long)e_begin * 128;
 
   if (tid == 0) {
-    for (int s = 0; s < NS; ++s) mbar_init(smem_u32(&bars[s]), 1);
+    for (int s = 0; s < kDecStages; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), kDecWarps); }
     fence_mbar_init();
-    *failed = 0;
   }
-  if (tid < NH) m_ref[tid] = -INFINITY;
   __syncthreads();
-  auto issue = [&](int t) {                                        // one thread: both copies of tile t
-    const int st = t % NS;
-    const uint32_t bytes = (uint32_t)min(kDecTile, n_rows - t * kDecTile) * 256u;
-    const uint32_t bar = smem_u32(&bars[st]);
-    mbar_expect_tx(bar, 2u * bytes);
-    bulk_load(smem_u32(tiles + st * 2 * kDecTileBytes), Kb + (long long)t * kDecTile * 128, bytes, bar);
-    bulk_load(smem_u32(tiles + st * 2 * kDecTileBytes + kDecTileBytes), Vb + (long long)t * kDecTile * 128, bytes, bar);
-  };
-  if (tid == 0)
-    for (int t = 0; t < NS - 1 && t < n_tiles; ++t) issue(t);
 
-  // this lane's 8 dims of every query of the set
-  float q[GT][8];
+  float o[8][4];                 // O^T, eight 16-dim row blocks
+  float m_a = -INFINITY, m_b = -INFINITY, l_a = 0.f, l_b = 0.f;   // heads 2c and 2c+1
 #pragma unroll
-  for (int g = 0; g < GT; ++g) {
-    if (set * GT + g < a.G) {
-      unpack8(*reinterpret_cast<const uint4*>(a.Q + b * a.qs_b + (long long)(h * a.G + set * GT + g) * a.qs_h + l16 * 8), q[g]);
-    } else {
+  for (int mt = 0; mt < 8; ++mt)
 #pragma unroll
-      for (int i = 0; i < 8; ++i) q[g][i] = 0.f;
-    }
-  }
-  float2 acc[GT][4];
-  float lsum[GT];
-#pragma unroll
-  for (int g = 0; g < GT; ++g) {
-    lsum[g] = 0.f;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) acc[g][i] = make_float2(0.f, 0.f);
-  }
+    for (int i = 0; i < 4; ++i) o[mt][i] = 0.f;
 
-  bool alive = true;
-  for (int t = 0; t < n_tiles; ++t) {
-    const int st = t % NS, buf = t & 1;
-    const int rows_here = min(kDecTile, n_rows - t * kDecTile);
-    const uint8_t* kt = tiles + st * 2 * kDecTileBytes + l16 * 16;
-    const uint8_t* vt = kt + kDecTileBytes;
-    float* s_buf = sc_s + buf * NH * kDecTile;
-    float* p_buf = sc_p + buf * NH * kDecTile;
-    bool flag = false;
-    if (!mbar_wait(smem_u32(&bars[st]), (uint32_t)(t / NS) & 1u)) { *failed = 1; flag = true; }
-
-    // ---- scores: a half-warp per row, four rows per half-warp ----------------------------------
-    uint4 w[4];
-#pragma unroll
-    for (int r = 0; r < 4; ++r) w[r] = *reinterpret_cast<const uint4*>(kt + (hw + 16 * r) * 256);
-#pragma unroll
-    for (int r = 0; r < 4; ++r) {
-      const int row = hw + 16 * r;
-      float k[8];
-      unpack8(w[r], k);
-      float s[GT];
-#pragma unroll
-      for (int g = 0; g < GT; ++g) {
-        float2 x = make_float2(0.f, 0.f);
-#pragma unroll
-        for (int i = 0; i < 8; i += 2)
-          x = __ffma2_rn(make_float2(k[i], k[i + 1]), make_float2(q[g][i], q[g][i + 1]), x);
-        s[g] = x.x + x.y;
+  if (warp == kDecWarps) {
+    // ---- producer: one lane keeps the ring full -------------------------------------------------
+    if (lane == 0) {
+      for (int t = 0; t < n_tiles; ++t) {
+        const int st = t % kDecStages;
+        if (t >= kDecStages && !mbar_wait(bar_empty(st), (uint32_t)(t / kDecStages - 1) & 1u)) {
+          record_status(a.status, kStatusTimeout);
+          break;
+        }
+        const uint32_t dst = base + st * kDecStageBytes;
+        const int row0 = e_begin + t * kDecTile;
+        mbar_expect_tx(bar_full(st), kDecStageBytes);
+        tma_load_4d(dst, &map_k, bar_full(st), 0, row0, h, b);
+        tma_load_4d(dst + kDecBoxBytes, &map_k, bar_full(st), 64, row0, h, b);
+        tma_load_4d(dst + 2 * kDecBoxBytes, &map_v, bar_full(st), 0, row0, h, b);
+        tma_load_4d(dst + 3 * kDecBoxBytes, &map_v, bar_full(st), 64, row0, h, b);
       }
-      // sum over the row's 16 lanes; while more than one head is left, each step also halves the
-      // heads a lane keeps, so that the lane ends up with the full sum of one head
-      int mine = 0;
-      int left = GT;
+    }
+  } else {
+    // ---- consumers ------------------------------------------------------------------------------
+    // B fragments of Q^T: head g, dims 16 ks + 2c, +1 and +8, +9 (heads past G are zero rows)
+    uint32_t qb[8][2];
+    {
+      const uint16_t* qrow = a.Q + b * a.qs_b + (long long)(h * a.G + g) * a.qs_h;
 #pragma unroll
-      for (int off = 8; off > 0; off >>= 1) {
-        if (left > 1) {
-          left >>= 1;
-          const bool upper = (lane & off) != 0;
+      for (int ks = 0; ks < 8; ++ks) {
+        qb[ks][0] = g < a.G ? *reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 2 * c) : 0u;
+        qb[ks][1] = g < a.G ? *reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 8 + 2 * c) : 0u;
+      }
+    }
+    for (int t = 0; t < n_tiles; ++t) {
+      const int st = t % kDecStages;
+      if (!__all_sync(0xffffffffu, mbar_wait(bar_full(st), (uint32_t)(t / kDecStages) & 1u))) {   // warp-uniform
+        if (lane == 0) record_status(a.status, kStatusTimeout);
+        break;
+      }
+      const int key0 = t * kDecTile + warp * 16;                   // first of the warp's rows, within the split
+      if (key0 < n_rows) {
+        const uint32_t k_tile = base + st * kDecStageBytes;
+        const uint32_t v_tile = k_tile + 2 * kDecBoxBytes;
+        // scores of 16 keys x 8 heads; two accumulators shorten the dependency chain
+        float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-          for (int j = 0; j < GT / 2; ++j) {
-            if (j < left) {
-              const float send = upper ? s[j] : s[j + left];
-              const float keep = upper ? s[j + left] : s[j];
-              s[j] = keep + __shfl_xor_sync(0xffffffffu, send, off);
-            }
+        for (int ks = 0; ks < 8; ks += 2) {
+          uint32_t k0[4], k1[4];
+          ldsm_x4(k_tile + dec_swz(warp * 16 + (lane & 15), 2 * ks + (lane >> 4)), k0);
+          ldsm_x4(k_tile + dec_swz(warp * 16 + (lane & 15), 2 * ks + 2 + (lane >> 4)), k1);
+          mma_bf16(s0, k0, qb[ks][0], qb[ks][1]);
+          mma_bf16(s1, k1, qb[ks + 1][0], qb[ks + 1][1]);
+        }
+        // rows past the split's end belong to the next split (or read as zeros): weight 0
+        const bool v_lo = key0 + g < n_rows, v_hi = key0 + g + 8 < n_rows;
+        const float x0 = v_lo ? (s0[0] + s1[0]) * a.scale_log2e : -INFINITY;   // key g,   head 2c
+        const float x1 = v_lo ? (s0[1] + s1[1]) * a.scale_log2e : -INFINITY;   // key g,   head 2c+1
+        const float x2 = v_hi ? (s0[2] + s1[2]) * a.scale_log2e : -INFINITY;   // key g+8, head 2c
+        const float x3 = v_hi ? (s0[3] + s1[3]) * a.scale_log2e : -INFINITY;   // key g+8, head 2c+1
+        const float t_a = fmaxf(x0, x2), t_b = fmaxf(x1, x3);
+        if (__any_sync(0xffffffffu, t_a > m_a + kDecRescaleAt || t_b > m_b + kDecRescaleAt)) {
+          // raise the reference maxima to the maxima over the warp's 16 keys (lanes with equal c)
+          float n_a = t_a, n_b = t_b;
+#pragma unroll
+          for (int off = 4; off < 32; off <<= 1) {
+            n_a = fmaxf(n_a, __shfl_xor_sync(0xffffffffu, n_a, off));
+            n_b = fmaxf(n_b, __shfl_xor_sync(0xffffffffu, n_b, off));
           }
-          if (upper) mine += left;
-        } else {
-          s[0] += __shfl_xor_sync(0xffffffffu, s[0], off);
+          n_a = fmaxf(n_a, m_a);                                  // finite: row key0 is valid
+          n_b = fmaxf(n_b, m_b);
+          const float f_a = exp2f(m_a - n_a), f_b = exp2f(m_b - n_b);   // 0 on the first raise
+          m_a = n_a; m_b = n_b;
+          l_a *= f_a; l_b *= f_b;
+#pragma unroll
+          for (int mt = 0; mt < 8; ++mt) { o[mt][0] *= f_a; o[mt][1] *= f_b; o[mt][2] *= f_a; o[mt][3] *= f_b; }
+        }
+        const float p0 = exp2f(x0 - m_a), p1 = exp2f(x1 - m_b), p2 = exp2f(x2 - m_a), p3 = exp2f(x3 - m_b);
+        l_a += p0 + p2;
+        l_b += p1 + p3;
+        // numerators as two bf16 terms each; transposed they are the B fragments of P^T
+        const uint32_t h01 = pack_bf16x2(p0, p1), h23 = pack_bf16x2(p2, p3);
+        const uint32_t r01 = pack_bf16x2(p0 - __uint_as_float(h01 << 16), p1 - __uint_as_float(h01 & 0xFFFF0000u));
+        const uint32_t r23 = pack_bf16x2(p2 - __uint_as_float(h23 << 16), p3 - __uint_as_float(h23 & 0xFFFF0000u));
+        const uint32_t bh0 = movmatrix_trans(h01), bh1 = movmatrix_trans(h23);
+        const uint32_t bl0 = movmatrix_trans(r01), bl1 = movmatrix_trans(r23);
+#pragma unroll
+        for (int mt = 0; mt < 8; ++mt) {
+          uint32_t vt[4];
+          ldsm_x4_trans(v_tile + dec_swz(warp * 16 + (lane & 7) + 8 * (lane >> 4), 2 * mt + ((lane >> 3) & 1)), vt);
+          mma_bf16(o[mt], vt, bh0, bh1);
+          mma_bf16(o[mt], vt, bl0, bl1);
         }
       }
-      // lanes that hold the same head hold the same sum; the lowest of them stores it
-      constexpr int kDup = 16 / GT;
-      const int head = set * GT + mine;
-      if ((l16 & (kDup - 1)) == 0 && head < a.G) {
-        const float sv = row < rows_here ? s[0] * a.scale_log2e : -INFINITY;   // stale rows of a short tile
-        const float m = m_ref[head];
-        s_buf[head * kDecTile + row] = sv;
-        p_buf[head * kDecTile + row] = exp2f(sv - m);
-        flag |= sv > m + kDecRescaleAt;
-      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_empty(st));
     }
-    const int any = __syncthreads_or(flag);
-    // every thread is past the V rows of tile t-1: its stage takes tile t+NS-1
-    if (tid == 0 && t + NS - 1 < n_tiles) issue(t + NS - 1);
-    if (any) {
-      if (*failed) { alive = false; break; }                       // uniform: read after the barrier
-      // raise the reference maxima to the tile's maxima: warp g redoes head g's numerators
-      if (warp < a.G) {
-        const float s0 = s_buf[warp * kDecTile + lane], s1 = s_buf[warp * kDecTile + lane + 32];
-        float tm = fmaxf(s0, s1);
+    // the warp's sums over its keys: lanes with equal c hold different keys
 #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) tm = fmaxf(tm, __shfl_xor_sync(0xffffffffu, tm, off));
-        const float m_old = m_ref[warp];
-        const float m_new = fmaxf(m_old, tm);                      // finite: the tile has a valid row
-        p_buf[warp * kDecTile + lane] = exp2f(s0 - m_new);
-        p_buf[warp * kDecTile + lane + 32] = exp2f(s1 - m_new);
-        __syncwarp();
-        if (lane == 0) { fac[warp] = exp2f(m_old - m_new); m_ref[warp] = m_new; }
-      }
-      __syncthreads();
-#pragma unroll
-      for (int g = 0; g < GT; ++g) {
-        if (set * GT + g < a.G) {
-          const float f = fac[set * GT + g];
-          lsum[g] *= f;
-#pragma unroll
-          for (int i = 0; i < 4; ++i) { acc[g][i].x *= f; acc[g][i].y *= f; }
-        }
-      }
+    for (int off = 4; off < 32; off <<= 1) {
+      l_a += __shfl_xor_sync(0xffffffffu, l_a, off);
+      l_b += __shfl_xor_sync(0xffffffffu, l_b, off);
     }
-
-    // ---- weighted sum of the tile's V rows: the lane keeps 8 dims for each head of the set ------
-#pragma unroll
-    for (int r = 0; r < 4; ++r) w[r] = *reinterpret_cast<const uint4*>(vt + (hw + 16 * r) * 256);
-#pragma unroll
-    for (int r = 0; r < 4; ++r) {
-      const int row = hw + 16 * r;
-      if (row < rows_here) {                                       // stale rows may hold anything
-        float v[8];
-        unpack8(w[r], v);
-#pragma unroll
-        for (int g = 0; g < GT; ++g) {
-          if (set * GT + g < a.G) {
-            const float p = p_buf[(set * GT + g) * kDecTile + row];
-            const float2 pp = make_float2(p, p);
-            lsum[g] += p;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) acc[g][i] = __ffma2_rn(pp, make_float2(v[2 * i], v[2 * i + 1]), acc[g][i]);
-          }
-        }
-      }
-    }
-  }
-  if (!alive) {                                                    // a copy never arrived: report, write nothing
-    if (tid == 0) record_status(a.status, kStatusTimeout);
-    return;
+    if (g == 0) { wm[warp * 8 + 2 * c] = m_a; wm[warp * 8 + 2 * c + 1] = m_b; }
   }
   __syncthreads();                                                 // every tile is consumed: the stages are free
 
-  // the two half-warps of a warp hold different rows of the same dims
+  // ---- merge the consumer warps (a warp that saw no valid row has max -inf and weight 0) ----------
+  if (warp < kDecWarps) {
+    float top_a = -INFINITY, top_b = -INFINITY;
 #pragma unroll
-  for (int g = 0; g < GT; ++g) {
-    lsum[g] += __shfl_xor_sync(0xffffffffu, lsum[g], 16);
+    for (int wi = 0; wi < kDecWarps; ++wi) { top_a = fmaxf(top_a, wm[wi * 8 + 2 * c]); top_b = fmaxf(top_b, wm[wi * 8 + 2 * c + 1]); }
+    const float f_a = m_a == -INFINITY ? 0.f : exp2f(m_a - top_a), f_b = m_b == -INFINITY ? 0.f : exp2f(m_b - top_b);
+    if (g == 0) { wl[warp * 8 + 2 * c] = l_a * f_a; wl[warp * 8 + 2 * c + 1] = l_b * f_b; }
+    float* dst = red + (warp * 8 + 2 * c) * kDecRedStride;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      acc[g][i].x += __shfl_xor_sync(0xffffffffu, acc[g][i].x, 16);
-      acc[g][i].y += __shfl_xor_sync(0xffffffffu, acc[g][i].y, 16);
-    }
-  }
-  float* red = reinterpret_cast<float*>(tiles);                    // [NSET*8 warps][GT][128]
-  if (half == 0) {
-#pragma unroll
-    for (int g = 0; g < GT; ++g) {
-      float4* dst = reinterpret_cast<float4*>(red + (warp * GT + g) * 128 + l16 * 8);
-      dst[0] = make_float4(acc[g][0].x, acc[g][0].y, acc[g][1].x, acc[g][1].y);
-      dst[1] = make_float4(acc[g][2].x, acc[g][2].y, acc[g][3].x, acc[g][3].y);
-    }
-    if (l16 == 0) {
-#pragma unroll
-      for (int g = 0; g < GT; ++g) lred[warp * GT + g] = lsum[g];
+    for (int mt = 0; mt < 8; ++mt) {
+      dst[16 * mt + g] = o[mt][0] * f_a;
+      dst[kDecRedStride + 16 * mt + g] = o[mt][1] * f_b;
+      dst[16 * mt + g + 8] = o[mt][2] * f_a;
+      dst[kDecRedStride + 16 * mt + g + 8] = o[mt][3] * f_b;
     }
   }
   __syncthreads();
   float* part = a.part + (((long long)(b * a.H_kv + h) * a.n_split + split) * a.G) * kDecPartFloats;
-  for (int i = tid; i < a.G * 128; i += NT) {
+  for (int i = tid; i < a.G * 128; i += kDecThreads) {
     const int head = i >> 7, d = i & 127;
-    const float* src = red + ((head / GT) * 8 * GT + head % GT) * 128 + d;   // warp 0 of the head's set
     float sum = 0.f;
 #pragma unroll
-    for (int wi = 0; wi < 8; ++wi) sum += src[wi * GT * 128];
+    for (int wi = 0; wi < kDecWarps; ++wi) sum += red[(wi * 8 + head) * kDecRedStride + d];
     part[head * kDecPartFloats + d] = sum;
   }
   if (tid < a.G) {
-    const float* src = lred + (tid / GT) * 8 * GT + tid % GT;
-    float l = 0.f;
+    float top = -INFINITY, l = 0.f;
 #pragma unroll
-    for (int wi = 0; wi < 8; ++wi) l += src[wi * GT];
-    part[tid * kDecPartFloats + 128] = m_ref[tid];
+    for (int wi = 0; wi < kDecWarps; ++wi) { top = fmaxf(top, wm[wi * 8 + tid]); l += wl[wi * 8 + tid]; }
+    part[tid * kDecPartFloats + 128] = top;
     part[tid * kDecPartFloats + 129] = l;
   }
 }
