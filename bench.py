@@ -551,7 +551,7 @@ def run_decode(args, w, rank, world, local_rank):
                    "context_len": w.context_len, "cache_len_per_head": length, "batch": w.batch,
                    "l2": f"{n_layers} layers' caches cycled ({entries * 512 / 1e6:.0f} MB each)"},
         "clocks": clocks, "e2e": None, "gpu_launches": int(launches),
-        "roofline": {"kernel": "decode_split_kernel + decode_combine_kernel", "bound": "hbm", "achieved": achieved,
+        "roofline": {"kernel": "decode_split_kernel", "bound": "hbm", "achieved": achieved,
                      "peak": peaks["hbm"], "unit": "GB/s", "frac": achieved / peaks["hbm"], "traffic": None,
                      "peak_source": f"hbm_gbs, {peaks['source']}"},
         "cpu_baseline": None,

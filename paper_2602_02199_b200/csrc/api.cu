@@ -52,7 +52,7 @@ struct Derived {
 };
 
 struct Carve {
-  size_t ctrl, hist, qbuckets, lse_part, lse2, s_exact, counts, idx, fix_items, key_buckets, total;
+  size_t ctrl, dec_count, hist, qbuckets, lse_part, lse2, s_exact, counts, idx, fix_items, key_buckets, total;
 };
 
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
@@ -194,6 +194,7 @@ void carve_ws(const laser_kv_config_t* c, const Derived& d, Carve* v) {
   const size_t nseg = d.nseg_max, S = c->block_size;
   const size_t bh = (size_t)c->batch * c->n_kv_heads;
   v->ctrl = take(256);
+  v->dec_count = take(bh * 4);        // finished decode splits per (sequence, KV head)
   v->hist = take(bh * c->lsh_tables * ((size_t)2 << c->lsh_bits));
   v->qbuckets = take(bh * d.GW * c->lsh_tables * 2);
   v->lse_part = take(lse_part_bytes_bound(nseg, d.GW));
@@ -428,7 +429,7 @@ laser_kv_status_t laser_kv_init(const laser_kv_config_t* cfg, const void* hyperp
       return fail(nullptr, LASER_KV_ERR_CUDA, "%s", msg.c_str());
     }
   }
-  if ((e = cudaMemset(h->ws + v.ctrl, 0, 256)) != cudaSuccess) {
+  if ((e = cudaMemset(h->ws + v.ctrl, 0, v.hist - v.ctrl)) != cudaSuccess) {   // status words and decode counters
     delete h;
     return fail(nullptr, LASER_KV_ERR_CUDA, "init: cudaMemset: %s", cudaGetErrorString(e));
   }
@@ -721,6 +722,7 @@ laser_kv_status_t laser_kv_decode_attention(laser_kv_handle_t h, int32_t layer, 
   a.n_split = n_split;
   a.scale_log2e = (softmax_scale == 0.f ? d.scale : softmax_scale) * 1.4426950408889634f;
   a.status = reinterpret_cast<int*>(h->ws + h->carve.ctrl);
+  a.counters = reinterpret_cast<int*>(h->ws + h->carve.dec_count);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const dim3 grid((unsigned)n_split, (unsigned)c.n_kv_heads, (unsigned)c.batch);
   static bool configured = false;       // the attribute is idempotent
@@ -734,10 +736,6 @@ laser_kv_status_t laser_kv_decode_attention(laser_kv_handle_t h, int32_t layer, 
   g_launches.fetch_add(1);
   e = cudaGetLastError();
   if (e != cudaSuccess) return fail(h, LASER_KV_ERR_CUDA, "decode_split_kernel launch: %s", cudaGetErrorString(e));
-  decode_combine_kernel<<<dim3((unsigned)c.n_q_heads, (unsigned)c.batch), 128, 0, st>>>(a);
-  g_launches.fetch_add(1);
-  e = cudaGetLastError();
-  if (e != cudaSuccess) return fail(h, LASER_KV_ERR_CUDA, "decode_combine_kernel launch: %s", cudaGetErrorString(e));
   return LASER_KV_OK;
 }
 
@@ -775,6 +773,7 @@ laser_kv_status_t laser_kv_poll_status(laser_kv_handle_t h, void* stream) {
   h->last_fixups = host[1];
   if (host[0] != 0) {
     cudaMemsetAsync(h->ws + h->carve.ctrl, 0, 4, st);
+    cudaMemsetAsync(h->ws + h->carve.dec_count, 0, h->carve.hist - h->carve.dec_count, st);   // a failed decode call may leave counts
     cudaStreamSynchronize(st);
     if (host[0] == LASER_KV_ERR_TIMEOUT) return fail(h, LASER_KV_ERR_TIMEOUT, "a bounded device-side wait gave up");
     if (host[0] == LASER_KV_ERR_CAPACITY)

@@ -19,7 +19,9 @@
 //                           only when a score exceeds it by 2^20), O^T += V^T P^T with the
 //                           numerators split into two bf16 terms so that the weights keep
 //                           16 mantissa bits. -> partial (max, sum, G x 128 accumulator) per split.
-//   decode_combine_kernel - merges the splits' partials per query head (fixed order).
+//                           The CTA that finishes last for its (sequence, KV head) merges the
+//                           splits' partials in split order and writes the output rows, so the
+//                           whole op is one launch.
 #pragma once
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -38,7 +40,7 @@ constexpr int kDecWarps = 4;            // consumer warps, 16 rows of every tile
 constexpr int kDecThreads = (kDecWarps + 1) * 32;
 constexpr int kDecCtasPerSm = 2;
 constexpr int kDecMaxGroup = 8;         // query heads per KV head, at most (the N of the MMA)
-constexpr int kDecPartFloats = 128 + 2; // per (split, query head): accumulator, reference max, sum
+constexpr int kDecPartFloats = 128 + 4; // per (split, query head): accumulator, reference max, sum, padding to 16 bytes
 constexpr int kDecMaxSplit = 512;
 constexpr float kDecRescaleAt = 20.f;   // log2 units a score may exceed the reference maximum by
 constexpr int kDecRedStride = 132;      // floats between heads in the merge buffer (bank spread)
@@ -46,7 +48,8 @@ constexpr int kDecRedStride = 132;      // floats between heads in the merge buf
 struct DecodeArgs {
   const uint16_t* Q;      // decode queries [batch][H_q][128] via strides
   long long qs_b, qs_h;
-  float* part;            // [batch][H_kv][n_split][G][130]
+  float* part;            // [batch][H_kv][n_split][G][132]
+  int* counters;          // [batch][H_kv] finished splits; zero between calls
   float* out;             // [batch][H_q][128]
   int H_kv, G, len, n_split;
   float scale_log2e;
@@ -117,6 +120,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap map_k,    // cache K: (d
     for (int s = 0; s < kDecStages; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), kDecWarps); }
     fence_mbar_init();
   }
+  if (tid == kDecWarps * 32) { tma_prefetch_desc(&map_k); tma_prefetch_desc(&map_v); }
   __syncthreads();
 
   float o[8][4];                 // O^T, eight 16-dim row blocks
@@ -261,50 +265,76 @@ decode_split_kernel(const __grid_constant__ CUtensorMap map_k,    // cache K: (d
     part[tid * kDecPartFloats + 128] = top;
     part[tid * kDecPartFloats + 129] = l;
   }
-}
 
-// One CTA of 128 threads per (query head, sequence): thread d merges dim d over the splits.
-__global__ void __launch_bounds__(128) decode_combine_kernel(const DecodeArgs a) {
-  __shared__ float wgt[kDecMaxSplit];
-  __shared__ float red_m[4], red_l[4];
-  const int hq = blockIdx.x, b = blockIdx.y;
-  const int h = hq / a.G, g = hq % a.G;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const float* part = a.part + (((long long)(b * a.H_kv + h) * a.n_split) * a.G + g) * kDecPartFloats;
-  const int cstride = a.G * kDecPartFloats;
-
-  float m = -INFINITY;
-  for (int c = threadIdx.x; c < a.n_split; c += 128) m = fmaxf(m, part[c * cstride + 128]);
-#pragma unroll
-  for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
-  if (lane == 0) red_m[warp] = m;
+  // ---- the CTA that finishes last for this (sequence, KV head) merges all splits -----------------
+  __shared__ int s_last;
+  __threadfence();
   __syncthreads();
-  m = fmaxf(fmaxf(red_m[0], red_m[1]), fmaxf(red_m[2], red_m[3]));
-  float l = 0.f;
-  for (int c = threadIdx.x; c < a.n_split; c += 128) {
-    const float wc = exp2f(part[c * cstride + 128] - m);
-    wgt[c] = wc;
-    l += wc * part[c * cstride + 129];
+  if (tid == 0) {
+    int* counter = a.counters + b * a.H_kv + h;
+    s_last = atomicAdd(counter, 1) == a.n_split - 1;
+    if (s_last) *counter = 0;                                      // ready for the next call
   }
-#pragma unroll
-  for (int off = 16; off > 0; off >>= 1) l += __shfl_xor_sync(0xffffffffu, l, off);
-  if (lane == 0) red_l[warp] = l;
   __syncthreads();
-  l = (red_l[0] + red_l[1]) + (red_l[2] + red_l[3]);
-
-  const int d = threadIdx.x;
-  float o[8];
-#pragma unroll
-  for (int j = 0; j < 8; ++j) o[j] = 0.f;
-  for (int c0 = 0; c0 < a.n_split; c0 += 8) {
-    float x[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) x[j] = c0 + j < a.n_split ? part[(c0 + j) * cstride + d] : 0.f;
-#pragma unroll
-    for (int j = 0; j < 8; ++j) o[j] = fmaf(c0 + j < a.n_split ? wgt[c0 + j] : 0.f, x[j], o[j]);
+  if (!s_last) return;
+  __threadfence();
+  const float* seg = a.part + ((long long)(b * a.H_kv + h) * a.n_split) * a.G * kDecPartFloats;
+  const int sstride = a.G * kDecPartFloats;                        // floats between splits
+  float* wgt = reinterpret_cast<float*>(gen + 2 * kDecBoxBytes * 2);   // [G][n_split], past the merge buffer
+  float* msl = wgt + a.G * a.n_split;                              // [G][n_split][2] maxima and sums, read once
+  for (int i = tid; i < a.G * a.n_split; i += kDecThreads) {
+    const int head = i / a.n_split, s = i - head * a.n_split;
+    const float2 v = __ldcg(reinterpret_cast<const float2*>(seg + (long long)s * sstride + head * kDecPartFloats + 128));
+    msl[2 * i] = v.x;
+    msl[2 * i + 1] = v.y;
   }
-  a.out[((long long)b * a.H_kv * a.G + hq) * 128 + d] =
-      (((o[0] + o[1]) + (o[2] + o[3])) + ((o[4] + o[5]) + (o[6] + o[7]))) / l;
+  __syncthreads();
+  for (int head = warp; head < a.G; head += kDecWarps + 1) {
+    const float* ms = msl + 2 * head * a.n_split;
+    float top = -INFINITY;
+    for (int s = lane; s < a.n_split; s += 32) top = fmaxf(top, ms[2 * s]);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) top = fmaxf(top, __shfl_xor_sync(0xffffffffu, top, off));
+    float l = 0.f;
+    for (int s = lane; s < a.n_split; s += 32) {
+      const float ws = exp2f(ms[2 * s] - top);
+      wgt[head * a.n_split + s] = ws;
+      l += ws * ms[2 * s + 1];
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) l += __shfl_xor_sync(0xffffffffu, l, off);
+    if (lane == 0) wl[head] = l;
+  }
+  __syncthreads();
+  for (int i = tid; i < a.G * 32; i += kDecThreads) {
+    const int head = i >> 5, d4 = i & 31;
+    const float* w = wgt + head * a.n_split;
+    const float4* src = reinterpret_cast<const float4*>(seg + head * kDecPartFloats) + d4;
+    float4 acc[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s0 = 0; s0 < a.n_split; s0 += 16) {
+      float4 x[16];
+#pragma unroll
+      for (int j = 0; j < 16; ++j)
+        x[j] = s0 + j < a.n_split ? __ldcg(src + (long long)(s0 + j) * (sstride / 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        const float ws = s0 + j < a.n_split ? w[s0 + j] : 0.f;
+        acc[j & 3].x = fmaf(ws, x[j].x, acc[j & 3].x);
+        acc[j & 3].y = fmaf(ws, x[j].y, acc[j & 3].y);
+        acc[j & 3].z = fmaf(ws, x[j].z, acc[j & 3].z);
+        acc[j & 3].w = fmaf(ws, x[j].w, acc[j & 3].w);
+      }
+    }
+    const float inv = 1.f / wl[head];
+    float4 r;
+    r.x = ((acc[0].x + acc[1].x) + (acc[2].x + acc[3].x)) * inv;
+    r.y = ((acc[0].y + acc[1].y) + (acc[2].y + acc[3].y)) * inv;
+    r.z = ((acc[0].z + acc[1].z) + (acc[2].z + acc[3].z)) * inv;
+    r.w = ((acc[0].w + acc[1].w) + (acc[2].w + acc[3].w)) * inv;
+    reinterpret_cast<float4*>(a.out + ((long long)(b * a.H_kv + h) * a.G + head) * 128)[d4] = r;
+  }
 }
 
 }  // namespace lkv
