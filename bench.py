@@ -187,6 +187,29 @@ def run_reference(args, w, rank, world):
 
 
 # ----------------------------------------------------------------------------------------------
+# multi-rank plumbing (replicas only: no data-path collective)
+# ----------------------------------------------------------------------------------------------
+def rank_layers(rank: int, n_sets: int):
+    """Seeds of the synthetic layers a rank cycles through: disjoint between ranks."""
+    return [rank * n_sets + i for i in range(n_sets)]
+
+
+def max_over_ranks(values, world: int, device):
+    """Element-wise maximum of each rank's device-measured times (ms) over all ranks."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
+def whole_job_value(units_per_rank_step: float, steps: int, world: int, ms: float) -> float:
+    """Units all ranks processed per second, with ms the slowest rank's time for `steps` steps."""
+    return world * units_per_rank_step * steps / (ms * 1e-3)
+
+
+# ----------------------------------------------------------------------------------------------
 # our arm
 # ----------------------------------------------------------------------------------------------
 def run_ours(args, w, rank, world, local_rank):
@@ -205,8 +228,7 @@ def run_ours(args, w, rank, world, local_rank):
     B = Bn.laser_kv_budget(w.context_len, S, w.ratio)
     n_sets = args.input_sets          # distinct layers cycled through so inputs exceed L2
     host = []
-    for i in range(n_sets):
-        layer = rank * n_sets + i
+    for layer in rank_layers(rank, n_sets):
         Ks, Vs, Qs = [], [], []
         for b in range(w.batch):
             k, v = synth.kv_blocks(w, layer, b, 0, nb)
@@ -291,10 +313,7 @@ def run_ours(args, w, rank, world, local_rank):
         eng.laser_kv_poll_status()
         assert int(pos_host[0, 0, 0]) == 0 and int(pos_host[0, 0, -1]) == w.context_len - 1
 
-    t = torch.tensor([ms, e2e_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms, e2e_ms = float(t[0]), float(t[1])
+    ms, e2e_ms = max_over_ranks([ms, e2e_ms], world, dev)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -302,8 +321,8 @@ def run_ours(args, w, rank, world, local_rank):
 
     peaks = load_peaks()
     ms_per_step = ms / args.steps
-    value = world * work["tokens"] * args.steps / (ms * 1e-3)
-    e2e_value = world * work["tokens"] * e2e_steps / (e2e_ms * 1e-3)
+    value = whole_job_value(work["tokens"], args.steps, world, ms)
+    e2e_value = whole_job_value(work["tokens"], e2e_steps, world, e2e_ms)
     h2d = sum(int(x.numel()) * 2 for x in host[0])
     d2h = int(pos_host.numel()) * 4
 
@@ -384,9 +403,9 @@ def run_consensus(args, w, rank, world, local_rank):
     B = Bn.laser_kv_budget(w.context_len, S, w.ratio)
     a, _, k_e, k_l = Bn.laser_kv_partition(B, w.protection_divisor, w.alpha)
     sets = []
-    for i in range(args.input_sets):
-        k, v = synth.kv_blocks(w, rank * args.input_sets + i, 0, 0, nb)
-        q = synth.q_window(w, rank * args.input_sets + i, 0)
+    for layer in rank_layers(rank, args.input_sets):
+        k, v = synth.kv_blocks(w, layer, 0, 0, nb)
+        q = synth.q_window(w, layer, 0)
         sets.append(tuple(torch.from_numpy(x.view(np.int16))[None].to(dev) for x in (k, v, q)))
     P = torch.from_numpy(synth.hyperplanes(w).view(np.int16)).to(dev)
     Kd = torch.zeros((H, nb * B, w.head_dim), dtype=torch.int16, device=dev)
@@ -435,20 +454,18 @@ def run_consensus(args, w, rank, world, local_rank):
     launches = Bn.laser_kv_launch_count() - launches0
     assert int(scr_c[:4].view(torch.int32)[0]) == 0 and int(scr_s[:4].view(torch.int32)[0]) == 0
     clocks = sampler.stop(t0, t1) if rank == 0 else None
-    t = torch.tensor([ms], dtype=torch.float64, device=dev)
+    ms, = max_over_ranks([ms], world, dev)
     if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
         dist.destroy_process_group()
     if rank != 0:
         return
-    ms = float(t[0])
     peaks = load_peaks()
     work = algorithmic_work(w, B)
     ms_per_step = ms / args.steps
     t_tensor = work["flops"] / (peaks["tf"] * 1e12)
     t_hbm = work["bytes"] / (peaks["hbm"] * 1e9)
     line = {
-        "metric": METRIC, "value": world * work["tokens"] * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
+        "metric": METRIC, "value": whole_job_value(work["tokens"], args.steps, world, ms), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": w.name, "policy": "consensus over the KV heads of a layer, one index set per block",
@@ -488,11 +505,11 @@ def run_decode(args, w, rank, world, local_rank):
                          alpha=w.alpha, debug=0, device=local_rank)
     eng = Bn.LaserKV(cfg, P)
     qs = []
-    for layer in range(n_layers):
+    for layer, seed in enumerate(rank_layers(rank, n_layers)):
         ks, vs, qw = [], [], []
         for b in range(w.batch):
-            k, v = synth.kv_blocks(w, rank * n_layers + layer, b, 0, nb)
-            ks.append(k); vs.append(v); qw.append(synth.q_window(w, rank * n_layers + layer, b))
+            k, v = synth.kv_blocks(w, seed, b, 0, nb)
+            ks.append(k); vs.append(v); qw.append(synth.q_window(w, seed, b))
         tk, tv, tq = (torch.from_numpy(np.stack(x).view(np.int16)).to(dev) for x in (ks, vs, qw))
         eng.laser_kv_select_block(layer, tk, tv, tq, nb)
         eng.laser_kv_poll_status()
@@ -530,20 +547,18 @@ def run_decode(args, w, rank, world, local_rank):
     launches = Bn.laser_kv_launch_count() - launches0
     eng.laser_kv_poll_status()
     clocks = sampler.stop(t0, t1) if rank == 0 else None
-    t = torch.tensor([ms], dtype=torch.float64, device=dev)
+    ms, = max_over_ranks([ms], world, dev)
     if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
         dist.destroy_process_group()
     if rank != 0:
         return
-    ms = float(t[0])
     peaks = load_peaks()
     ms_per_step = ms / args.steps
     entries = w.batch * H * length                               # cache entries read per step
     nbytes = entries * 2 * 128 * 2 + w.batch * w.n_q_heads * 128 * (2 + 4)
     achieved = nbytes / (ms_per_step * 1e-3) / 1e9
     line = {
-        "metric": "decode_attention_cache_entries_per_s_per_layer", "value": world * entries * args.steps / (ms * 1e-3),
+        "metric": "decode_attention_cache_entries_per_s_per_layer", "value": whole_job_value(entries, args.steps, world, ms),
         "unit": "cache entries/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
