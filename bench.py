@@ -43,6 +43,7 @@ NCU_TRAFFIC_BYTES = {
     ("llama8b_128k", "stream_kernel<lse>"): 269266944 + 3838720,
     ("llama8b_128k", "stream_kernel<score>"): 270472192 + 7939584,
     ("llama8b_128k", "append_kernel"): 254743808 + 201296896,
+    ("llama8b_128k", "decode_split_kernel"): 261788672 + 3954944,
 }
 
 
@@ -567,8 +568,9 @@ def run_decode(args, w, rank, world, local_rank):
                    "l2": f"{n_layers} layers' caches cycled ({entries * 512 / 1e6:.0f} MB each)"},
         "clocks": clocks, "e2e": None, "gpu_launches": int(launches),
         "roofline": {"kernel": "decode_split_kernel", "bound": "hbm", "achieved": achieved,
-                     "peak": peaks["hbm"], "unit": "GB/s", "frac": achieved / peaks["hbm"], "traffic": None,
-                     "peak_source": f"hbm_gbs, {peaks['source']}"},
+                     "peak": peaks["hbm"], "unit": "GB/s", "frac": achieved / peaks["hbm"],
+                     "traffic": NCU_TRAFFIC_BYTES.get((w.name, "decode_split_kernel")),
+                     "peak_source": f"hbm_gbs, {peaks['source']}", "bytes_per_launch": nbytes},
         "cpu_baseline": None,
     }
     print(json.dumps(line), flush=True)
