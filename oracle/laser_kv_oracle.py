@@ -21,6 +21,9 @@ What each function follows:
                           K-bit SimHash (sign of Gaussian hyperplane projections) per table.
 * ``collision_counts``  - Algorithm 1 line 6: number of (query, table) pairs whose bucket equals
                           the key's bucket (S_lsh is this count divided by R * number of queries).
+* ``collision_probability`` - Section 3.3 "Recall" as worded (tokens ranked by the theoretical hash
+                          collision probability with the query): the expectation of the
+                          collision fraction over the hyperplane draw, (1 - theta/pi)^K per query.
 * ``topk_lower_index``  - the TopK of Algorithm 1 lines 4 and 7, ties to the lower index.
 * ``select_indices``    - Algorithm 1 lines 3-8 on the candidate set left by Section 3.1.
 * ``select_block`` / ``AppendOnlyCache`` - Section 3 (only selected tokens are kept) and the
@@ -299,6 +302,31 @@ class AppendOnlyCache:
             self.V[h, sl] = v_bits[h, idx[h]]
             self.pos[h, sl] = (block_start + idx[h]).astype(np.int32)
         self.length += B
+
+
+# ----------------------------------------------------------------------------------------------
+# recall score in closed form (Section 3.3 "Recall": ranking by the theoretical collision probability)
+# ----------------------------------------------------------------------------------------------
+def collision_probability(q_bits: np.ndarray, k_bits: np.ndarray, n_bits: int) -> np.ndarray:
+    """S_theory[j] = (1/n_queries) * sum_q (1 - theta(q, k_j)/pi)^K.
+
+    A K-bit SimHash table puts q and k in the same bucket exactly when none of K independent
+    Gaussian hyperplanes separates them; one hyperplane separates them with probability
+    theta/pi, theta the angle between them. This is the expectation over the hyperplane draw
+    of Algorithm 1's collision fraction (``collision_counts`` divided by tables * queries).
+    q_bits uint16 [n_queries, d], k_bits uint16 [S, d] -> float64 [S]. A zero vector has no angle:
+    its cosine is taken as 0 (theta = pi/2), the value the hashes give it against any hyperplane
+    draw in expectation.
+    """
+    q = bf16_bits_to_f64(q_bits)
+    k = bf16_bits_to_f64(k_bits)
+    qn = np.sqrt((q * q).sum(axis=1))
+    kn = np.sqrt((k * k).sum(axis=1))
+    dots = q @ k.T                                        # [n_queries, S]
+    denom = qn[:, None] * kn[None, :]
+    cos = np.divide(dots, denom, out=np.zeros_like(dots), where=denom > 0)
+    theta = np.arccos(np.clip(cos, -1.0, 1.0))
+    return ((1.0 - theta / math.pi) ** int(n_bits)).mean(axis=0)
 
 
 # ----------------------------------------------------------------------------------------------
