@@ -271,6 +271,26 @@ laser_kv_status_t laser_kv_collision_counts(const void* K_blk, const void* Q_win
                                             int32_t lsh_bits, int32_t lsh_tables, void* scratch,
                                             size_t scratch_bytes, uint32_t* counts_out, void* stream);
 
+/* Recall score in closed form (Section 3.3 "Recall" as worded: tokens are ranked by their
+ * theoretical hash collision probability with the query; Algorithm 1 line 6 prints the empirical
+ * fraction, whose expectation over the hyperplane draw this is):
+ *   p[b][h][t][j] = (1 / (G*W)) * sum over the window queries q of KV head h's group of
+ *                   (1 - theta(q, k_j) / pi)^lsh_bits,   theta = angle between q and key j of block t
+ * (a zero vector counts as orthogonal to everything). No hyperplanes, no tables. The values are
+ * non-negative floats, so their bit patterns order like unsigned integers: cast p_out to
+ * uint32_t* and pass it as `counts` to laser_kv_two_stage_topk to rank the recall stage by it.
+ *   K_blk, Q_win, kv_strides, q_strides, n_blocks : as for laser_kv_select_block.
+ *   scratch : dev, 16-byte aligned, at least 256 bytes; its first int is a status word (0 or
+ *             LASER_KV_ERR_TIMEOUT), cleared by the call.
+ *   p_out   : dev fp32 [batch][H_kv][n_blocks][S].
+ * head_dim is 128; G*W a multiple of 16, at most 256; lsh_bits in [1, 64]. fp32 arithmetic on exact
+ * bf16 products. */
+laser_kv_status_t laser_kv_collision_probability(const void* K_blk, const void* Q_win, const int64_t kv_strides[3],
+                                                 const int64_t q_strides[3], int32_t batch, int32_t n_q_heads,
+                                                 int32_t n_kv_heads, int32_t block_size, int32_t window,
+                                                 int32_t n_blocks, int32_t lsh_bits, void* scratch,
+                                                 size_t scratch_bytes, float* p_out, void* stream);
+
 /* Consensus aggregation (Section 3.3 "Precision" as printed: a candidate's score is the attention
  * it receives summed over all layers and heads, so that one index set serves every head): adds the
  * per-head outputs of laser_kv_window_scores and laser_kv_collision_counts over the n_heads heads,

@@ -19,7 +19,7 @@ EXPORTS = [
     "laser_kv_profile_read", "laser_kv_window_scores", "laser_kv_window_scores_scratch_bytes",
     "laser_kv_window_scores_static", "laser_kv_window_scores_static_max_bytes",
     "laser_kv_collision_counts", "laser_kv_collision_counts_scratch_bytes", "laser_kv_consensus_accumulate",
-    "laser_kv_decode_attention", "laser_kv_decode_attention_scratch_bytes",
+    "laser_kv_decode_attention", "laser_kv_decode_attention_scratch_bytes", "laser_kv_collision_probability",
 ]
 
 
@@ -131,6 +131,8 @@ def load(build_if_missing: bool = True) -> C.CDLL:
                                               vp, vp]
     lib.laser_kv_consensus_accumulate.restype = i32
     lib.laser_kv_consensus_accumulate.argtypes = [vp, vp, i32, i32, i32, i32, i32, vp, vp, vp]
+    lib.laser_kv_collision_probability.restype = i32
+    lib.laser_kv_collision_probability.argtypes = [vp, vp, p(i64), p(i64), i32, i32, i32, i32, i32, i32, i32, vp, sz, vp, vp]
     lib.laser_kv_decode_attention_scratch_bytes.restype = sz
     lib.laser_kv_decode_attention_scratch_bytes.argtypes = [vp]
     lib.laser_kv_decode_attention.restype = i32
@@ -390,6 +392,24 @@ def laser_kv_collision_counts(K_blk, Q_win, hyperplanes, block_size, n_blocks, l
     _check(load().laser_kv_collision_counts(_ptr(K_blk), _ptr(Q_win), _ptr(hyperplanes), ks, qs, batch, h_q, h_kv,
                                             block_size, window, n_blocks, lsh_bits, lsh_tables, _ptr(scratch),
                                             scratch.numel(), _ptr(out), _stream_ptr(stream)))
+    return out, scratch
+
+
+def laser_kv_collision_probability(K_blk, Q_win, block_size, n_blocks, lsh_bits, scratch=None, stream=None):
+    """K_blk [batch][H_kv][n_blocks*S][128], Q_win [batch][H_q][W][128] (2-byte device tensors) -> the
+    closed-form recall score fp32 [batch][H_kv][n_blocks][S]. Returns (p, scratch); the first int of
+    scratch is the status word. `p.view(torch.int32)` serves as `counts` of laser_kv_two_stage_topk."""
+    import torch
+    batch, h_kv = K_blk.shape[0], K_blk.shape[1]
+    h_q, window = Q_win.shape[1], Q_win.shape[2]
+    if scratch is None:
+        scratch = torch.empty(256, dtype=torch.uint8, device=K_blk.device)
+    out = torch.empty((batch, h_kv, n_blocks, block_size), dtype=torch.float32, device=K_blk.device)
+    ks = (C.c_int64 * 3)(*K_blk.stride()[:3])
+    qs = (C.c_int64 * 3)(*Q_win.stride()[:3])
+    _check(load().laser_kv_collision_probability(_ptr(K_blk), _ptr(Q_win), ks, qs, batch, h_q, h_kv, block_size, window,
+                                                 n_blocks, lsh_bits, _ptr(scratch), scratch.numel(), _ptr(out),
+                                                 _stream_ptr(stream)))
     return out, scratch
 
 

@@ -19,6 +19,7 @@
 #include "stream_gemm.cuh"
 #include "query_proj.cuh"
 #include "decode_attn.cuh"
+#include "theory_score.cuh"
 
 namespace {
 
@@ -1199,6 +1200,82 @@ laser_kv_status_t laser_kv_collision_counts(const void* K_blk, const void* Q_win
     if ((e = cudaGetLastError()) != cudaSuccess)
       return fail(nullptr, LASER_KV_ERR_CUDA, "collision_counts: signfix_kernel: %s", cudaGetErrorString(e));
   }
+  return LASER_KV_OK;
+}
+
+laser_kv_status_t laser_kv_collision_probability(const void* K_blk, const void* Q_win, const int64_t kv_strides[3],
+                                                 const int64_t q_strides[3], int32_t batch, int32_t n_q_heads,
+                                                 int32_t n_kv_heads, int32_t block_size, int32_t window, int32_t n_blocks,
+                                                 int32_t lsh_bits, void* scratch, size_t scratch_bytes, float* p_out,
+                                                 void* stream) {
+  if (!K_blk || !Q_win || !kv_strides || !q_strides || !p_out || !scratch)
+    return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "collision_probability: NULL argument");
+  if (batch < 1 || n_q_heads < 1 || n_kv_heads < 1 || block_size < 1 || window < 1 || n_blocks < 1)
+    return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "collision_probability: sizes must be positive");
+  if (n_q_heads % n_kv_heads) return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "collision_probability: n_q_heads %% n_kv_heads != 0");
+  if (lsh_bits < 1 || lsh_bits > 64) return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "collision_probability: lsh_bits must be in [1, 64]");
+  const int G = n_q_heads / n_kv_heads, GW = G * window;
+  if (GW % 16 || GW > kThMaxQueries || window > 256 || G > 256 || block_size % 8)
+    return fail(nullptr, LASER_KV_ERR_UNSUPPORTED,
+                "collision_probability: G*W must be a multiple of 16, at most 256; block_size a multiple of 8");
+  if ((long long)n_blocks * block_size > 0x7fffffffLL || (long long)n_kv_heads * n_blocks > 65535 || batch > 65535)
+    return fail(nullptr, LASER_KV_ERR_UNSUPPORTED, "collision_probability: too many segments");
+  if (!aligned16(K_blk) || !aligned16(Q_win) || !aligned16(p_out) || !aligned16(scratch))
+    return fail(nullptr, LASER_KV_ERR_ALIGNMENT, "collision_probability: device pointers must be 16-byte aligned");
+  if (scratch_bytes < 256) return fail(nullptr, LASER_KV_ERR_CAPACITY, "collision_probability: scratch needs 256 bytes");
+  for (int i = 0; i < 3; ++i)
+    if (kv_strides[i] < 0 || q_strides[i] < 0 || (kv_strides[i] % 8) || (q_strides[i] % 8))
+      return fail(nullptr, LASER_KV_ERR_ALIGNMENT, "collision_probability: strides must be non-negative multiples of 8 elements");
+  if (kv_strides[2] < kHeadDim || q_strides[2] < kHeadDim || (n_kv_heads > 1 && !kv_strides[1]) || (batch > 1 && !kv_strides[0]) ||
+      (n_q_heads > 1 && !q_strides[1]) || (batch > 1 && !q_strides[0]))
+    return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "collision_probability: bad strides");
+  EncodeTiledFn enc = driver_encode_fn();
+  if (!enc) return fail(nullptr, LASER_KV_ERR_CUDA, "collision_probability: cuTensorMapEncodeTiled not available (no CUDA driver?)");
+  CUtensorMap mapK, mapQ;
+  const cuuint32_t ones[4] = {1, 1, 1, 1};
+  {
+    const cuuint64_t s_tok = (cuuint64_t)kv_strides[2];
+    const cuuint64_t s_head = kv_strides[1] > 0 ? (cuuint64_t)kv_strides[1] : s_tok * (cuuint64_t)n_blocks * block_size;
+    const cuuint64_t s_batch = kv_strides[0] > 0 ? (cuuint64_t)kv_strides[0] : s_head * (cuuint64_t)n_kv_heads;
+    const cuuint64_t dims[4] = {(cuuint64_t)kHeadDim, (cuuint64_t)n_blocks * block_size, (cuuint64_t)n_kv_heads, (cuuint64_t)batch};
+    const cuuint64_t strides[3] = {s_tok * 2, s_head * 2, s_batch * 2};
+    const cuuint32_t box[4] = {64, (cuuint32_t)kThTile, 1, 1};
+    const CUresult r = enc(&mapK, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(K_blk), dims, strides, box, ones,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(nullptr, LASER_KV_ERR_CUDA, "collision_probability: tensor map of K failed (CUresult %d)", (int)r);
+  }
+  {
+    const cuuint64_t s_w = (cuuint64_t)q_strides[2];
+    const cuuint64_t s_head = q_strides[1] > 0 ? (cuuint64_t)q_strides[1] : s_w * (cuuint64_t)window;
+    const cuuint64_t s_batch = q_strides[0] > 0 ? (cuuint64_t)q_strides[0] : s_head * (cuuint64_t)n_q_heads;
+    const cuuint64_t dims[4] = {(cuuint64_t)kHeadDim, (cuuint64_t)window, (cuuint64_t)n_q_heads, (cuuint64_t)batch};
+    const cuuint64_t strides[3] = {s_w * 2, s_head * 2, s_batch * 2};
+    const cuuint32_t box[4] = {64, (cuuint32_t)window, (cuuint32_t)G, 1};
+    const CUresult r = enc(&mapQ, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(Q_win), dims, strides, box, ones,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(nullptr, LASER_KV_ERR_CUDA, "collision_probability: tensor map of Q failed (CUresult %d)", (int)r);
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  cudaError_t e;
+  if ((e = cudaMemsetAsync(scratch, 0, 256, st)) != cudaSuccess)
+    return fail(nullptr, LASER_KV_ERR_CUDA, "collision_probability: memset: %s", cudaGetErrorString(e));
+  TheoryArgs a;
+  a.out = p_out;
+  a.S = block_size; a.nb = n_blocks; a.H_kv = n_kv_heads; a.G = G; a.GW = GW; a.kbits = lsh_bits;
+  a.tiles_in_block = (block_size + kThTile - 1) / kThTile;
+  a.status = static_cast<int*>(scratch);
+  static bool configured = false;       // the attribute is idempotent
+  if (!configured) {
+    e = cudaFuncSetAttribute(theory_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)theory_smem_bytes(kThMaxQueries));
+    if (e != cudaSuccess) return fail(nullptr, LASER_KV_ERR_CUDA, "theory_kernel attribute: %s", cudaGetErrorString(e));
+    configured = true;
+  }
+  const dim3 grid((unsigned)((a.tiles_in_block + kThTilesPerCta - 1) / kThTilesPerCta), (unsigned)(n_kv_heads * n_blocks), (unsigned)batch);
+  theory_kernel<<<grid, kThThreads, theory_smem_bytes(GW), st>>>(mapK, mapQ, a);
+  g_launches.fetch_add(1);
+  if ((e = cudaGetLastError()) != cudaSuccess) return fail(nullptr, LASER_KV_ERR_CUDA, "theory_kernel launch: %s", cudaGetErrorString(e));
   return LASER_KV_OK;
 }
 

@@ -1,0 +1,176 @@
+// Recall score in closed form (Section 3.3 "Recall": tokens are ranked by their theoretical hash
+// collision probability with the query): for every key of a block and KV head,
+//   S_theory[j] = (1 / (G*W)) * sum_q (1 - theta(q, k_j) / pi)^K,
+// theta the angle between window query q and key k_j, K the sign bits per SimHash table. It is the
+// expectation over the hyperplane draw of the collision fraction that the hashing path counts, so
+// it needs no hyperplanes and no tables: one pass over the keys.
+//
+//   theory_kernel - one CTA per (run of eight 64-key tiles of a block, KV head, block, sequence).
+//                   A producer warp brings the head's query group (once) and the key tiles (ring
+//                   of two stages) with TMA, 128-byte swizzle. Each of four consumer warps owns 16
+//                   keys of a tile: key norms from the tile, <q, k> for all G*W queries as
+//                   m16n8k16 bf16 MMAs (keys on M, eight queries per N), then per element
+//                   cos = <q,k> / (|q| |k|), u = acos(-cos) / pi = 1 - theta / pi, u^K, summed
+//                   over the queries. The element-wise chain (acos, log2, exp2; about 35
+//                   instructions) bounds the kernel, not the contraction and not HBM.
+#pragma once
+#include "decode_attn.cuh"
+
+namespace lkv {
+
+constexpr int kThTile = 64;             // keys per stage
+constexpr int kThTileBytes = kThTile * 256;
+constexpr int kThStages = 2;
+constexpr int kThWarps = 4;             // consumer warps, 16 keys of every tile each
+constexpr int kThThreads = (kThWarps + 1) * 32;
+constexpr int kThTilesPerCta = 8;
+constexpr int kThMaxQueries = 256;
+
+struct TheoryArgs {
+  float* out;             // [batch][H_kv][nb][S]
+  int S, nb, H_kv, G, GW, kbits, tiles_in_block;
+  int* status;
+};
+
+__host__ __device__ constexpr uint32_t theory_smem_bytes(int gw) {
+  return 2u * gw * 128u + kThStages * kThTileBytes + kThMaxQueries * 4u + (1u + 2u * kThStages) * 8u + 1024u;
+}
+
+// Byte offset of the 16-byte chunk (0..15) of a row in a tile of two 128-byte-swizzled boxes of
+// `box_bytes` each.
+__device__ __forceinline__ uint32_t swz128(uint32_t row, uint32_t chunk, uint32_t box_bytes) {
+  return (chunk >> 3) * box_bytes + row * 128u + (((chunk & 7u) ^ (row & 7u)) << 4);
+}
+// sum of squares of eight bf16 values
+__device__ __forceinline__ float sum_squares8(const uint4& w) {
+  const uint32_t v[4] = {w.x, w.y, w.z, w.w};
+  float s = 0.f;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float lo = __uint_as_float(v[i] << 16), hi = __uint_as_float(v[i] & 0xFFFF0000u);
+    s = fmaf(lo, lo, s);
+    s = fmaf(hi, hi, s);
+  }
+  return s;
+}
+// (1 - theta/pi)^K from the cosine: acos(-c) = pi - acos(c)
+__device__ __forceinline__ float collide_pow(float c, float kbits) {
+  const float u = acosf(-fminf(fmaxf(c, -1.f), 1.f)) * 0.3183098861837907f;
+  return exp2f(kbits * __log2f(u));                               // u = 0 -> 0
+}
+
+__global__ void __launch_bounds__(kThThreads, 2)
+theory_kernel(const __grid_constant__ CUtensorMap map_k,    // K: (d, nb*S, H_kv, batch), box (64, 64, 1, 1)
+              const __grid_constant__ CUtensorMap map_q,    // Q: (d, W, H_q, batch), box (64, W, G, 1)
+              const TheoryArgs a) {
+  extern __shared__ uint8_t tsm_raw[];
+  const uint32_t base = (smem_u32(tsm_raw) + 1023u) & ~1023u;
+  uint8_t* const gen = tsm_raw + (base - smem_u32(tsm_raw));
+  const uint32_t q_box = (uint32_t)a.GW * 128u;
+  const uint32_t sm_q = base, sm_k = base + 2u * q_box;
+  float* rq = reinterpret_cast<float*>(gen + 2u * q_box + kThStages * kThTileBytes);          // [256] 1/|q|
+  const uint32_t sm_bars = sm_k + kThStages * kThTileBytes + kThMaxQueries * 4u;
+  const uint32_t bar_q = sm_bars;
+  auto bar_full = [&](int s) { return sm_bars + 8u * (1 + s); };
+  auto bar_empty = [&](int s) { return sm_bars + 8u * (1 + kThStages + s); };
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int g = lane >> 2, c = lane & 3;
+  const int h = blockIdx.y / a.nb, t = blockIdx.y % a.nb, b = blockIdx.z;
+  const int tile0 = blockIdx.x * kThTilesPerCta;
+  const int n_tiles = min(kThTilesPerCta, a.tiles_in_block - tile0);
+
+  if (tid == 0) {
+    mbar_init(bar_q, 1);
+    for (int s = 0; s < kThStages; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), kThWarps); }
+    fence_mbar_init();
+  }
+  __syncthreads();
+
+  if (warp == kThWarps) {
+    // ---- producer ---------------------------------------------------------------------------------
+    if (lane == 0) {
+      mbar_expect_tx(bar_q, 2u * q_box);
+      tma_load_4d(sm_q, &map_q, bar_q, 0, 0, h * a.G, b);
+      tma_load_4d(sm_q + q_box, &map_q, bar_q, 64, 0, h * a.G, b);
+      for (int j = 0; j < n_tiles; ++j) {
+        const int st = j % kThStages;
+        if (j >= kThStages && !mbar_wait(bar_empty(st), (uint32_t)(j / kThStages - 1) & 1u)) {
+          record_status(a.status, kStatusTimeout);
+          break;
+        }
+        const uint32_t dst = sm_k + st * kThTileBytes;
+        const int row0 = t * a.S + (tile0 + j) * kThTile;
+        mbar_expect_tx(bar_full(st), kThTileBytes);
+        tma_load_4d(dst, &map_k, bar_full(st), 0, row0, h, b);
+        tma_load_4d(dst + kThTileBytes / 2, &map_k, bar_full(st), 64, row0, h, b);
+      }
+    }
+    return;
+  }
+
+  // ---- consumers ------------------------------------------------------------------------------------
+  bool alive = __all_sync(0xffffffffu, mbar_wait(bar_q, 0));
+  if (alive) {
+    for (int q = tid; q < a.GW; q += kThWarps * 32) {
+      float n2 = 0.f;
+#pragma unroll
+      for (int ch = 0; ch < 16; ++ch) n2 += sum_squares8(*reinterpret_cast<const uint4*>(gen + swz128(q, ch, q_box)));
+      rq[q] = n2 > 0.f ? 1.0f / sqrtf(n2) : 0.f;
+    }
+  }
+  asm volatile("bar.sync 1, %0;" ::"n"(kThWarps * 32) : "memory");     // the consumer warps only
+  const float kbits = (float)a.kbits, inv_gw = 1.0f / (float)a.GW;
+  float* out = a.out + (((long long)(b * a.H_kv + h) * a.nb + t) * a.S);
+
+  for (int j = 0; j < n_tiles && alive; ++j) {
+    const int st = j % kThStages;
+    if (!__all_sync(0xffffffffu, mbar_wait(bar_full(st), (uint32_t)(j / kThStages) & 1u))) {
+      if (lane == 0) record_status(a.status, kStatusTimeout);
+      alive = false;
+      break;
+    }
+    const uint32_t k_tile = sm_k + st * kThTileBytes;
+    const uint8_t* k_gen = gen + 2u * q_box + st * kThTileBytes;
+    // the warp's 16 keys as A fragments for all eight 16-dim steps, and the norms of keys g, g+8
+    uint32_t ak[8][4];
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) ldsm_x4(k_tile + dec_swz(warp * 16 + (lane & 15), 2 * ks + (lane >> 4)), ak[ks]);
+    float n_lo = 0.f, n_hi = 0.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      n_lo += sum_squares8(*reinterpret_cast<const uint4*>(k_gen + dec_swz(warp * 16 + g, c + 4 * i)));
+      n_hi += sum_squares8(*reinterpret_cast<const uint4*>(k_gen + dec_swz(warp * 16 + g + 8, c + 4 * i)));
+    }
+    n_lo += __shfl_xor_sync(0xffffffffu, n_lo, 1); n_lo += __shfl_xor_sync(0xffffffffu, n_lo, 2);
+    n_hi += __shfl_xor_sync(0xffffffffu, n_hi, 1); n_hi += __shfl_xor_sync(0xffffffffu, n_hi, 2);
+    const float rk_lo = n_lo > 0.f ? 1.0f / sqrtf(n_lo) : 0.f, rk_hi = n_hi > 0.f ? 1.0f / sqrtf(n_hi) : 0.f;
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar_empty(st));                     // the tile lives in registers now
+
+    float sum_lo = 0.f, sum_hi = 0.f;
+#pragma unroll 2
+    for (int nt = 0; nt < a.GW / 8; ++nt) {
+      float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int k2 = 0; k2 < 4; ++k2) {
+        uint32_t qf[4];                                             // B fragments of two 16-dim steps
+        ldsm_x4(sm_q + swz128(8 * nt + (lane & 7), 4 * k2 + (lane >> 3), q_box), qf);
+        mma_bf16(acc, ak[2 * k2], qf[0], qf[1]);
+        mma_bf16(acc, ak[2 * k2 + 1], qf[2], qf[3]);
+      }
+      const float2 r = *reinterpret_cast<const float2*>(rq + 8 * nt + 2 * c);
+      sum_lo += collide_pow(acc[0] * rk_lo * r.x, kbits) + collide_pow(acc[1] * rk_lo * r.y, kbits);
+      sum_hi += collide_pow(acc[2] * rk_hi * r.x, kbits) + collide_pow(acc[3] * rk_hi * r.y, kbits);
+    }
+    sum_lo += __shfl_xor_sync(0xffffffffu, sum_lo, 1); sum_lo += __shfl_xor_sync(0xffffffffu, sum_lo, 2);
+    sum_hi += __shfl_xor_sync(0xffffffffu, sum_hi, 1); sum_hi += __shfl_xor_sync(0xffffffffu, sum_hi, 2);
+    if (c == 0) {
+      const int key = (tile0 + j) * kThTile + warp * 16 + g;       // within the block
+      if (key < a.S) out[key] = sum_lo * inv_gw;
+      if (key + 8 < a.S) out[key + 8] = sum_hi * inv_gw;
+    }
+  }
+}
+
+}  // namespace lkv
