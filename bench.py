@@ -576,6 +576,109 @@ def run_decode(args, w, rank, world, local_rank):
     print(json.dumps(line), flush=True)
 
 
+def run_theory(args, w, rank, world, local_rank):
+    """Recall stage ranked by the closed-form collision probability instead of hashed counts: a step
+    is one layer through window scores, the closed-form score, the two-stage top-k and the gather,
+    from step-level entry points. The closed-form kernel is timed by its own CUDA events."""
+    import torch
+    import torch.distributed as dist
+    from paper_2602_02199_b200 import binding as Bn
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    S, nb, H = w.block_size, w.n_blocks, w.n_kv_heads
+    B = Bn.laser_kv_budget(w.context_len, S, w.ratio)
+    a, _, k_e, k_l = Bn.laser_kv_partition(B, w.protection_divisor, w.alpha)
+    sets = []
+    for layer in rank_layers(rank, args.input_sets):
+        ks, vs, qw = [], [], []
+        for b in range(w.batch):
+            k, v = synth.kv_blocks(w, layer, b, 0, nb)
+            ks.append(k); vs.append(v); qw.append(synth.q_window(w, layer, b))
+        sets.append(tuple(torch.from_numpy(np.stack(x).view(np.int16)).to(dev) for x in (ks, vs, qw)))
+    nseg = w.batch * H * nb
+    Kd = torch.zeros((nseg, B, w.head_dim), dtype=torch.int16, device=dev)
+    Vd = torch.zeros_like(Kd)
+    pos = torch.zeros((nseg, B), dtype=torch.int32, device=dev)
+    scr_s = torch.empty(Bn.laser_kv_window_scores_scratch_bytes(w.batch, w.n_q_heads, H, S, w.window, nb),
+                        dtype=torch.uint8, device=dev)
+    scr_p = torch.empty(256, dtype=torch.uint8, device=dev)
+    ev = []
+
+    def step(i, timed=False):
+        tk, tv, tq = sets[i % len(sets)]
+        s = Bn.laser_kv_window_scores(tk, tq, S, nb, scratch=scr_s)
+        if timed:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+        p, _ = Bn.laser_kv_collision_probability(tk, tq, S, nb, w.lsh_bits, scratch=scr_p)
+        if timed:
+            e1.record()
+            ev.append((e0, e1))
+        idx = Bn.laser_kv_two_stage_topk(s.view(nseg, S), p.view(torch.int32).view(nseg, S), a, k_e, k_l)
+        Bn.laser_kv_gather_append(tk.view(nseg, S, 128), tv.view(nseg, S, 128), idx, Kd, Vd, pos, 0, 0)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    launches0 = Bn.laser_kv_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t0 = time.time()
+    e0.record()
+    for i in range(args.steps):
+        step(i, timed=True)
+    e1.record()
+    barrier()
+    t1 = time.time()
+    ms = e0.elapsed_time(e1)
+    kern_ms = sum(x.elapsed_time(y) for x, y in ev) / len(ev)
+    launches = Bn.laser_kv_launch_count() - launches0
+    assert int(scr_p[:4].view(torch.int32)[0]) == 0 and int(scr_s[:4].view(torch.int32)[0]) == 0
+    clocks = sampler.stop(t0, t1) if rank == 0 else None
+    ms, kern_ms = max_over_ranks([ms, kern_ms], world, dev)
+    if world > 1:
+        dist.destroy_process_group()
+    if rank != 0:
+        return
+    work = algorithmic_work(w, B)
+    ms_per_step = ms / args.steps
+    # the closed-form kernel evaluates acos, log2 and exp2 once per (window query, key) pair: at least
+    # three special-function operations per pair, 16 per clock and SM
+    pairs = float(w.batch) * nb * S * w.n_q_heads * w.window
+    sm_mhz = (clocks or {}).get("sm_max_mhz") or 1965.0
+    peak = 16.0 / 3.0 * 148 * sm_mhz * 1e6 / 1e9              # G pairs/s
+    achieved = pairs / (kern_ms * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": whole_job_value(work["tokens"], args.steps, world, ms), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "policy": "recall stage ranked by the closed-form collision probability",
+                   "context_len": w.context_len, "block_size": S, "blocks_per_call": nb, "budget_per_block": B,
+                   "l2": f"inputs larger than L2: {len(sets)} layers of K+V cycled"},
+        "clocks": clocks, "e2e": None, "gpu_launches": int(launches),
+        "roofline": {"kernel": "theory_kernel", "bound": "alu", "achieved": achieved, "peak": peak, "unit": "Gpair/s",
+                     "frac": achieved / peak, "traffic": None, "ms_per_launch": kern_ms,
+                     "peak_source": "3 special-function operations per (query, key) pair at 16 per clock and SM, 148 SMs, "
+                                    "maximum SM clock"},
+        "cpu_baseline": None,
+    }
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -583,9 +686,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama8b_128k", choices=sorted(synth.WORKLOADS))
-    ap.add_argument("--policy", default="per_head", choices=["per_head", "consensus", "decode"],
+    ap.add_argument("--policy", default="per_head", choices=["per_head", "consensus", "decode", "theory"],
                     help="per_head: the hot path (every KV head selects for itself); consensus: one index set per block; "
-                         "decode: attention of one decode step over the compacted cache")
+                         "decode: attention of one decode step over the compacted cache; "
+                         "theory: recall stage ranked by the closed-form collision probability")
     ap.add_argument("--alpha", type=float, default=None,
                     help="exact share of the recall budget (1 = exact attention only, 0 = LSH only; default: the workload's 0.75)")
     ap.add_argument("--divisor", type=int, default=None, help="protection divisor n (default: the workload's)")
@@ -610,6 +714,8 @@ def main():
         run_consensus(args, w, rank, world, local_rank)
     elif args.policy == "decode":
         run_decode(args, w, rank, world, local_rank)
+    elif args.policy == "theory":
+        run_theory(args, w, rank, world, local_rank)
     else:
         run_ours(args, w, rank, world, local_rank)
 

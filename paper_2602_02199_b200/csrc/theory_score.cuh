@@ -7,12 +7,13 @@
 //
 //   theory_kernel - one CTA per (run of eight 64-key tiles of a block, KV head, block, sequence).
 //                   A producer warp brings the head's query group (once) and the key tiles (ring
-//                   of two stages) with TMA, 128-byte swizzle. Each of four consumer warps owns 16
-//                   keys of a tile: key norms from the tile, <q, k> for all G*W queries as
+//                   of two stages) with TMA, 128-byte swizzle. Two groups of four consumer warps
+//                   take alternate tiles, each warp 16 keys of its tile: key norms from the tile, <q, k> for all G*W queries as
 //                   m16n8k16 bf16 MMAs (keys on M, eight queries per N), then per element
 //                   cos = <q,k> / (|q| |k|), u = acos(-cos) / pi = 1 - theta / pi, u^K, summed
-//                   over the queries. The element-wise chain (acos, log2, exp2; about 35
-//                   instructions) bounds the kernel, not the contraction and not HBM.
+//                   over the queries. The element-wise chain (a degree-7 polynomial and a square
+//                   root for acos, log2, exp2; about 20 instructions) bounds the kernel, not the
+//                   contraction and not HBM.
 #pragma once
 #include "decode_attn.cuh"
 
@@ -21,7 +22,7 @@ namespace lkv {
 constexpr int kThTile = 64;             // keys per stage
 constexpr int kThTileBytes = kThTile * 256;
 constexpr int kThStages = 2;
-constexpr int kThWarps = 4;             // consumer warps, 16 keys of every tile each
+constexpr int kThWarps = 8;             // consumer warps: two groups of four take alternate tiles, 16 keys each
 constexpr int kThThreads = (kThWarps + 1) * 32;
 constexpr int kThTilesPerCta = 8;
 constexpr int kThMaxQueries = 256;
@@ -53,10 +54,28 @@ __device__ __forceinline__ float sum_squares8(const uint4& w) {
   }
   return s;
 }
-// (1 - theta/pi)^K from the cosine: acos(-c) = pi - acos(c)
-__device__ __forceinline__ float collide_pow(float c, float kbits) {
-  const float u = acosf(-fminf(fmaxf(c, -1.f), 1.f)) * 0.3183098861837907f;
-  return exp2f(kbits * __log2f(u));                               // u = 0 -> 0
+// acos(x) ~= sqrt(1 - x) * P(x) on [0, 1], |error| < 8e-8 (degree 7, the form of Abramowitz & Stegun
+// 4.4.46; coefficients from the fit in acos_poly.py beside this file)
+#define LKV_ACOS_POLY(STEP) \
+  STEP(-1.2628309199e-03f) STEP(6.6712932680e-03f) STEP(-1.7089810817e-02f) STEP(3.0893053199e-02f) \
+  STEP(-5.0174715211e-02f) STEP(8.8979049893e-02f) STEP(-2.1459880383e-01f) STEP(1.5707963050e+00f)
+__device__ __forceinline__ float sqrt_approx(float x) {
+  float y;
+  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+// (1 - theta/pi)^K for two cosines: u*pi = acos(-c) = pi - acos(c) (c >= 0), acos(|c|) (c < 0);
+// u^K = 2^(K log2(u pi) - K log2(pi)), kbias = -K log2(pi). u = 0 gives 0.
+__device__ __forceinline__ float2 collide_pow2(float2 c, float kbits, float kbias) {
+  const float2 x = make_float2(fminf(fabsf(c.x), 1.f), fminf(fabsf(c.y), 1.f));
+  float2 p = make_float2(0.f, 0.f);                              // Horner, highest coefficient first
+#define LKV_HORNER(A) p = __ffma2_rn(p, x, make_float2(A, A));
+  LKV_ACOS_POLY(LKV_HORNER)
+#undef LKV_HORNER
+  const float2 a = __fmul2_rn(make_float2(sqrt_approx(1.f - x.x), sqrt_approx(1.f - x.y)), p);
+  const float wx = c.x >= 0.f ? 3.14159265358979f - a.x : a.x;
+  const float wy = c.y >= 0.f ? 3.14159265358979f - a.y : a.y;
+  return make_float2(ex2_approx(fmaf(kbits, lg2_approx(wx), kbias)), ex2_approx(fmaf(kbits, lg2_approx(wy), kbias)));
 }
 
 __global__ void __launch_bounds__(kThThreads, 2)
@@ -82,7 +101,7 @@ theory_kernel(const __grid_constant__ CUtensorMap map_k,    // K: (d, nb*S, H_kv
 
   if (tid == 0) {
     mbar_init(bar_q, 1);
-    for (int s = 0; s < kThStages; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), kThWarps); }
+    for (int s = 0; s < kThStages; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 4); }
     fence_mbar_init();
   }
   __syncthreads();
@@ -120,10 +139,11 @@ theory_kernel(const __grid_constant__ CUtensorMap map_k,    // K: (d, nb*S, H_kv
     }
   }
   asm volatile("bar.sync 1, %0;" ::"n"(kThWarps * 32) : "memory");     // the consumer warps only
-  const float kbits = (float)a.kbits, inv_gw = 1.0f / (float)a.GW;
+  const float kbits = (float)a.kbits, kbias = -1.6514961294723187f * (float)a.kbits, inv_gw = 1.0f / (float)a.GW;
   float* out = a.out + (((long long)(b * a.H_kv + h) * a.nb + t) * a.S);
 
-  for (int j = 0; j < n_tiles && alive; ++j) {
+  const int rows = (warp & 3) * 16;                                  // the warp's keys within a tile
+  for (int j = warp >> 2; j < n_tiles && alive; j += 2) {
     const int st = j % kThStages;
     if (!__all_sync(0xffffffffu, mbar_wait(bar_full(st), (uint32_t)(j / kThStages) & 1u))) {
       if (lane == 0) record_status(a.status, kStatusTimeout);
@@ -135,12 +155,12 @@ theory_kernel(const __grid_constant__ CUtensorMap map_k,    // K: (d, nb*S, H_kv
     // the warp's 16 keys as A fragments for all eight 16-dim steps, and the norms of keys g, g+8
     uint32_t ak[8][4];
 #pragma unroll
-    for (int ks = 0; ks < 8; ++ks) ldsm_x4(k_tile + dec_swz(warp * 16 + (lane & 15), 2 * ks + (lane >> 4)), ak[ks]);
+    for (int ks = 0; ks < 8; ++ks) ldsm_x4(k_tile + dec_swz(rows + (lane & 15), 2 * ks + (lane >> 4)), ak[ks]);
     float n_lo = 0.f, n_hi = 0.f;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      n_lo += sum_squares8(*reinterpret_cast<const uint4*>(k_gen + dec_swz(warp * 16 + g, c + 4 * i)));
-      n_hi += sum_squares8(*reinterpret_cast<const uint4*>(k_gen + dec_swz(warp * 16 + g + 8, c + 4 * i)));
+      n_lo += sum_squares8(*reinterpret_cast<const uint4*>(k_gen + dec_swz(rows + g, c + 4 * i)));
+      n_hi += sum_squares8(*reinterpret_cast<const uint4*>(k_gen + dec_swz(rows + g + 8, c + 4 * i)));
     }
     n_lo += __shfl_xor_sync(0xffffffffu, n_lo, 1); n_lo += __shfl_xor_sync(0xffffffffu, n_lo, 2);
     n_hi += __shfl_xor_sync(0xffffffffu, n_hi, 1); n_hi += __shfl_xor_sync(0xffffffffu, n_hi, 2);
@@ -149,7 +169,7 @@ theory_kernel(const __grid_constant__ CUtensorMap map_k,    // K: (d, nb*S, H_kv
     if (lane == 0) mbar_arrive(bar_empty(st));                     // the tile lives in registers now
 
     float sum_lo = 0.f, sum_hi = 0.f;
-#pragma unroll 2
+#pragma unroll 4
     for (int nt = 0; nt < a.GW / 8; ++nt) {
       float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -160,13 +180,15 @@ theory_kernel(const __grid_constant__ CUtensorMap map_k,    // K: (d, nb*S, H_kv
         mma_bf16(acc, ak[2 * k2 + 1], qf[2], qf[3]);
       }
       const float2 r = *reinterpret_cast<const float2*>(rq + 8 * nt + 2 * c);
-      sum_lo += collide_pow(acc[0] * rk_lo * r.x, kbits) + collide_pow(acc[1] * rk_lo * r.y, kbits);
-      sum_hi += collide_pow(acc[2] * rk_hi * r.x, kbits) + collide_pow(acc[3] * rk_hi * r.y, kbits);
+      const float2 p_lo = collide_pow2(__fmul2_rn(make_float2(acc[0], acc[1]), __fmul2_rn(r, make_float2(rk_lo, rk_lo))), kbits, kbias);
+      const float2 p_hi = collide_pow2(__fmul2_rn(make_float2(acc[2], acc[3]), __fmul2_rn(r, make_float2(rk_hi, rk_hi))), kbits, kbias);
+      sum_lo += p_lo.x + p_lo.y;
+      sum_hi += p_hi.x + p_hi.y;
     }
     sum_lo += __shfl_xor_sync(0xffffffffu, sum_lo, 1); sum_lo += __shfl_xor_sync(0xffffffffu, sum_lo, 2);
     sum_hi += __shfl_xor_sync(0xffffffffu, sum_hi, 1); sum_hi += __shfl_xor_sync(0xffffffffu, sum_hi, 2);
     if (c == 0) {
-      const int key = (tile0 + j) * kThTile + warp * 16 + g;       // within the block
+      const int key = (tile0 + j) * kThTile + rows + g;       // within the block
       if (key < a.S) out[key] = sum_lo * inv_gw;
       if (key + 8 < a.S) out[key + 8] = sum_hi * inv_gw;
     }
