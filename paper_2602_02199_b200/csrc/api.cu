@@ -319,6 +319,19 @@ laser_kv_status_t launch_append(const AppendArgs& a, int n_seg, cudaStream_t st)
 }
 
 
+template <int KB>
+cudaError_t launch_theory(const CUtensorMap& mk, const CUtensorMap& mq, const TheoryArgs& a, dim3 grid, cudaStream_t st) {
+  static bool configured = false;       // per instantiation; the attribute is idempotent
+  if (!configured) {
+    const cudaError_t e = cudaFuncSetAttribute(theory_kernel<KB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               (int)theory_smem_bytes(kThMaxQueries));
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  theory_kernel<KB><<<grid, kThThreads, theory_smem_bytes(a.GW), st>>>(mk, mq, a);
+  return cudaGetLastError();
+}
+
 // Splits per (sequence, KV head) of a decode call: as many as fill the GPU's resident CTAs once,
 // never more than tiles in the cache.
 int decode_splits(const laser_kv_ctx* h, long long len) {
@@ -1266,16 +1279,17 @@ laser_kv_status_t laser_kv_collision_probability(const void* K_blk, const void* 
   a.S = block_size; a.nb = n_blocks; a.H_kv = n_kv_heads; a.G = G; a.GW = GW; a.kbits = lsh_bits;
   a.tiles_in_block = (block_size + kThTile - 1) / kThTile;
   a.status = static_cast<int*>(scratch);
-  static bool configured = false;       // the attribute is idempotent
-  if (!configured) {
-    e = cudaFuncSetAttribute(theory_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)theory_smem_bytes(kThMaxQueries));
-    if (e != cudaSuccess) return fail(nullptr, LASER_KV_ERR_CUDA, "theory_kernel attribute: %s", cudaGetErrorString(e));
-    configured = true;
-  }
   const dim3 grid((unsigned)((a.tiles_in_block + kThTilesPerCta - 1) / kThTilesPerCta), (unsigned)(n_kv_heads * n_blocks), (unsigned)batch);
-  theory_kernel<<<grid, kThThreads, theory_smem_bytes(GW), st>>>(mapK, mapQ, a);
+  switch (lsh_bits) {                    // the usual table widths get the multiplication form of u^K
+    case 4: e = launch_theory<4>(mapK, mapQ, a, grid, st); break;
+    case 6: e = launch_theory<6>(mapK, mapQ, a, grid, st); break;
+    case 8: e = launch_theory<8>(mapK, mapQ, a, grid, st); break;
+    case 10: e = launch_theory<10>(mapK, mapQ, a, grid, st); break;
+    case 12: e = launch_theory<12>(mapK, mapQ, a, grid, st); break;
+    default: e = launch_theory<0>(mapK, mapQ, a, grid, st); break;
+  }
   g_launches.fetch_add(1);
-  if ((e = cudaGetLastError()) != cudaSuccess) return fail(nullptr, LASER_KV_ERR_CUDA, "theory_kernel launch: %s", cudaGetErrorString(e));
+  if (e != cudaSuccess) return fail(nullptr, LASER_KV_ERR_CUDA, "theory_kernel launch: %s", cudaGetErrorString(e));
   return LASER_KV_OK;
 }
 

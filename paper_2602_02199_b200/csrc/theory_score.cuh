@@ -12,8 +12,9 @@
 //                   m16n8k16 bf16 MMAs (keys on M, eight queries per N), then per element
 //                   cos = <q,k> / (|q| |k|), u = acos(-cos) / pi = 1 - theta / pi, u^K, summed
 //                   over the queries. The element-wise chain (a degree-7 polynomial and a square
-//                   root for acos, log2, exp2; about 20 instructions) bounds the kernel, not the
-//                   contraction and not HBM.
+//                   root for acos, then u^K by repeated squaring for the usual K, by log2/exp2
+//                   otherwise; under 20 instructions) bounds the kernel, not the contraction and
+//                   not HBM.
 #pragma once
 #include "decode_attn.cuh"
 
@@ -64,8 +65,22 @@ __device__ __forceinline__ float sqrt_approx(float x) {
   asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-// (1 - theta/pi)^K for two cosines: u*pi = acos(-c) = pi - acos(c) (c >= 0), acos(|c|) (c < 0);
-// u^K = 2^(K log2(u pi) - K log2(pi)), kbias = -K log2(pi). u = 0 gives 0.
+// x^KB for two values by repeated squaring (KB a compile-time count of sign bits).
+template <int KB>
+__device__ __forceinline__ float2 pow_int2(float2 x) {
+  float2 r = make_float2(1.f, 1.f), sq = x;
+  bool first = true;
+#pragma unroll
+  for (int b = KB; b > 0; b >>= 1) {
+    if (b & 1) { r = first ? sq : __fmul2_rn(r, sq); first = false; }
+    if (b > 1) sq = __fmul2_rn(sq, sq);
+  }
+  return r;
+}
+// (1 - theta/pi)^K for two cosines: u*pi = acos(-c) = pi - acos(c) (c >= 0), acos(|c|) (c < 0).
+// KB > 0: u^KB by multiplication; KB == 0: any K at run time as 2^(K log2(u pi) - K log2(pi)),
+// kbias = -K log2(pi). u = 0 gives 0 either way.
+template <int KB>
 __device__ __forceinline__ float2 collide_pow2(float2 c, float kbits, float kbias) {
   const float2 x = make_float2(fminf(fabsf(c.x), 1.f), fminf(fabsf(c.y), 1.f));
   float2 p = make_float2(0.f, 0.f);                              // Horner, highest coefficient first
@@ -75,9 +90,11 @@ __device__ __forceinline__ float2 collide_pow2(float2 c, float kbits, float kbia
   const float2 a = __fmul2_rn(make_float2(sqrt_approx(1.f - x.x), sqrt_approx(1.f - x.y)), p);
   const float wx = c.x >= 0.f ? 3.14159265358979f - a.x : a.x;
   const float wy = c.y >= 0.f ? 3.14159265358979f - a.y : a.y;
+  if (KB > 0) return pow_int2<KB>(__fmul2_rn(make_float2(wx, wy), make_float2(0.3183098861837907f, 0.3183098861837907f)));
   return make_float2(ex2_approx(fmaf(kbits, lg2_approx(wx), kbias)), ex2_approx(fmaf(kbits, lg2_approx(wy), kbias)));
 }
 
+template <int KB>
 __global__ void __launch_bounds__(kThThreads, 2)
 theory_kernel(const __grid_constant__ CUtensorMap map_k,    // K: (d, nb*S, H_kv, batch), box (64, 64, 1, 1)
               const __grid_constant__ CUtensorMap map_q,    // Q: (d, W, H_q, batch), box (64, W, G, 1)
@@ -180,8 +197,8 @@ theory_kernel(const __grid_constant__ CUtensorMap map_k,    // K: (d, nb*S, H_kv
         mma_bf16(acc, ak[2 * k2 + 1], qf[2], qf[3]);
       }
       const float2 r = *reinterpret_cast<const float2*>(rq + 8 * nt + 2 * c);
-      const float2 p_lo = collide_pow2(__fmul2_rn(make_float2(acc[0], acc[1]), __fmul2_rn(r, make_float2(rk_lo, rk_lo))), kbits, kbias);
-      const float2 p_hi = collide_pow2(__fmul2_rn(make_float2(acc[2], acc[3]), __fmul2_rn(r, make_float2(rk_hi, rk_hi))), kbits, kbias);
+      const float2 p_lo = collide_pow2<KB>(__fmul2_rn(make_float2(acc[0], acc[1]), __fmul2_rn(r, make_float2(rk_lo, rk_lo))), kbits, kbias);
+      const float2 p_hi = collide_pow2<KB>(__fmul2_rn(make_float2(acc[2], acc[3]), __fmul2_rn(r, make_float2(rk_hi, rk_hi))), kbits, kbias);
       sum_lo += p_lo.x + p_lo.y;
       sum_hi += p_hi.x + p_hi.y;
     }

@@ -57,11 +57,12 @@ def test_collision_probability_against_oracle(name, S, nb, batch):
         assert (idx_np[seg] == own[2]).all(), seg
 
 
-def test_collision_probability_special_vectors():
+@pytest.mark.parametrize("K", [6, 7, 33])      # 6: u^K by multiplication; 7, 33: the run-time form
+def test_collision_probability_special_vectors(K):
     """Keys equal to, orthogonal to and opposite to the only query direction, and a zero key."""
     import torch
     from paper_2602_02199_b200 import binding as Bn
-    S, W, K = 64, 16, 6
+    S, W = 64, 16
     q = np.zeros((1, 1, W, 128), np.float32)
     q[..., 0] = 2.0                                                   # every window query along e0
     k = np.zeros((1, 1, S, 128), np.float32)
@@ -73,5 +74,5 @@ def test_collision_probability_special_vectors():
     tQ = torch.from_numpy(synth.f32_to_bf16_bits(q).view(np.int16)).cuda()
     p, _ = Bn.laser_kv_collision_probability(tK, tQ, S, 1, K)
     got = to_np(p)[0, 0, 0]
-    np.testing.assert_allclose(got[:4], [1.0, 0.5 ** K, 0.0, 0.75 ** K], rtol=1e-5, atol=1e-7)
-    np.testing.assert_allclose(got[4:], 0.5 ** K, rtol=1e-5)         # zero keys count as orthogonal
+    np.testing.assert_allclose(got[:4], [1.0, 0.5 ** K, 0.0, 0.75 ** K], rtol=2e-5, atol=1e-7)
+    np.testing.assert_allclose(got[4:], 0.5 ** K, rtol=2e-5)         # zero keys count as orthogonal
