@@ -68,6 +68,28 @@ def test_decode_attention_against_oracle(name, S, nb, batch, budget, strided, sc
             assert (err <= DEC_RTOL * np.abs(want) + DEC_ATOL).all(), (b, h, err.max())
 
 
+@pytest.mark.parametrize("S,B,nb,G", [(64, 8, 1, 1), (64, 8, 3, 2), (128, 40, 2, 8)])
+def test_decode_attention_on_caches_shorter_than_a_tile(S, B, nb, G):
+    """8, 24 and 80 entries per head (less than, and just over, one 64-row tile); G = 1, 2, 8."""
+    import torch
+    H = 2
+    w = synth.workload("tiny").with_(block_size=S, context_len=nb * S, n_q_heads=H * G, n_kv_heads=H, window=16 // G if G < 8 else 2,
+                                     lsh_tables=8, needles="none")
+    run = run_workload_layer(w, 0, n_blocks=nb, debug=0, budget=B)
+    eng = run["engine"]
+    rng = np.random.default_rng(7)
+    q_bits = synth.f32_to_bf16_bits(rng.standard_normal((1, H * G, 128)).astype(np.float32))
+    out = eng.laser_kv_decode_attention(0, torch.from_numpy(q_bits.view(np.int16)).cuda())
+    eng.laser_kv_poll_status()
+    got = to_np(out)
+    cache = _oracle_cache(w, run, 0)
+    assert cache.length == nb * B
+    for h in range(H):
+        want = O.decode_attention(q_bits[0, h * G:(h + 1) * G], cache.K[h, :cache.length], cache.V[h, :cache.length])
+        err = np.abs(got[0, h * G:(h + 1) * G] - want)
+        assert (err <= DEC_RTOL * np.abs(want) + DEC_ATOL).all(), (h, err.max())
+
+
 def test_decode_attention_reports_an_empty_cache():
     import torch
     from paper_2602_02199_b200 import binding as Bn
