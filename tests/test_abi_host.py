@@ -79,6 +79,18 @@ def test_null_and_misaligned_arguments_are_rejected():
     assert lib.laser_kv_two_stage_topk(None, None, 1, 8, 1, 1, 1, None, None) == B.ERR_INVALID_ARG
     assert lib.laser_kv_gather_append(None, None, 0, 0, None, 1, 1, None, None, 0, None, 0, 0, 0, None) == B.ERR_INVALID_ARG
     assert b"NULL" in lib.laser_kv_last_error(None)
+    # the entry points beside the hot path validate before they touch the device
+    assert lib.laser_kv_decode_attention(None, 0, None, None, 0.0, None, None, 0, None) == B.ERR_INVALID_ARG
+    assert lib.laser_kv_decode_attention_scratch_bytes(None) == 0
+    ks, qs = (C.c_int64 * 3)(0, 1024 * 128, 128), (C.c_int64 * 3)(0, 64 * 128, 128)
+    cp = lib.laser_kv_collision_probability
+    assert cp(None, None, ks, qs, 1, 4, 1, 1024, 64, 1, 10, None, 0, None, None) == B.ERR_INVALID_ARG
+    assert cp(0x1000, 0x2000, ks, qs, 1, 4, 1, 1024, 64, 1, 0, 0x3000, 256, 0x4000, None) == B.ERR_INVALID_ARG    # K = 0
+    assert cp(0x1000, 0x2000, ks, qs, 1, 4, 1, 1024, 72, 1, 10, 0x3000, 256, 0x4000, None) == B.ERR_UNSUPPORTED   # G*W = 288
+    assert cp(0x1008, 0x2000, ks, qs, 1, 4, 1, 1024, 64, 1, 10, 0x3000, 256, 0x4000, None) == B.ERR_ALIGNMENT
+    assert cp(0x1000, 0x2000, ks, qs, 1, 4, 1, 1024, 64, 1, 10, 0x3000, 16, 0x4000, None) == B.ERR_CAPACITY
+    bad = (C.c_int64 * 3)(0, 1024 * 128, 100)
+    assert cp(0x1000, 0x2000, bad, qs, 1, 4, 1, 1024, 64, 1, 10, 0x3000, 256, 0x4000, None) == B.ERR_ALIGNMENT
 
 
 @pytest.mark.skipif(_have_gpu(), reason="checks the no-GPU failure path")
