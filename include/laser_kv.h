@@ -16,6 +16,9 @@
  *     (LASER_KV_ERR_ALIGNMENT otherwise).
  *   - Kernel launches are asynchronous on the caller's stream; nothing is copied back to the
  *     host unless the entry point says so.
+ *   - Kernels launch on the calling thread's current device. laser_kv_init makes the handle's device
+ *     current; a later handle call made while another device is current fails with
+ *     LASER_KV_ERR_STATE. The handle-free step-level entry points run on the current device.
  *   - There is no CPU fallback: without a CUDA device laser_kv_init fails with LASER_KV_ERR_CUDA.
  */
 #ifndef LASER_KV_H_

@@ -101,6 +101,16 @@ laser_kv_status_t fail(laser_kv_ctx* h, laser_kv_status_t s, const char* fmt, ..
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// Kernels launch on the calling thread's current device: it must be the one the handle lives on.
+laser_kv_status_t check_device(laser_kv_ctx* h, const char* who) {
+  int dev = -1;
+  const cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return fail(h, LASER_KV_ERR_CUDA, "%s: cudaGetDevice: %s", who, cudaGetErrorString(e));
+  if (dev != h->cfg.device)
+    return fail(h, LASER_KV_ERR_STATE, "%s: the current device is %d, the handle was created on device %d", who, dev, h->cfg.device);
+  return LASER_KV_OK;
+}
+
 // Persistent grid of a streaming launch: one CTA per SM, never more CTAs than tiles.
 int stream_grid(long long n_tiles, int num_sms) {
   long long g = num_sms < kMaxStreamCtas ? num_sms : kMaxStreamCtas;
@@ -231,16 +241,26 @@ bool encode_map(laser_kv_ctx* h, CUtensorMap* m, const void* ptr, int rank, cons
   return true;
 }
 
+// The dynamic shared-memory limit is an attribute of (kernel, device): set it once per device that
+// the process launches the kernel on. `done` holds one bit per device ordinal below 64.
+template <typename Fn>
+cudaError_t ensure_smem_limit(std::atomic<unsigned long long>& done, Fn* fn, int bytes) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const unsigned long long bit = (dev >= 0 && dev < 64) ? 1ull << dev : 0ull;
+  if (bit && (done.load(std::memory_order_relaxed) & bit)) return cudaSuccess;
+  e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess && bit) done.fetch_or(bit);
+  return e;
+}
+
 template <int MODE, int KB, int TCv>
 cudaError_t launch_stream(const CUtensorMap& mk, const CUtensorMap& ms, const StreamArgs& a, int grid,
                           uint32_t smem, cudaStream_t st) {
-  static bool attr_done = false;   // per instantiation; the attribute is per device function
-  cudaError_t e = cudaSuccess;
-  if (!attr_done) {
-    e = cudaFuncSetAttribute(stream_kernel<MODE, KB, TCv>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
-    if (e != cudaSuccess) return e;
-    attr_done = true;
-  }
+  static std::atomic<unsigned long long> limit_set{0};   // per instantiation
+  const cudaError_t e = ensure_smem_limit(limit_set, stream_kernel<MODE, KB, TCv>, kMaxSmem);
+  if (e != cudaSuccess) return e;
   stream_kernel<MODE, KB, TCv><<<grid, kStreamThreads, smem, st>>>(mk, ms, a);
   g_launches.fetch_add(1);
   return cudaGetLastError();
@@ -261,12 +281,9 @@ cudaError_t launch_proj(int K, int TCv, const CUtensorMap& mk, const CUtensorMap
 template <int KB>
 cudaError_t launch_qsig_t(const CUtensorMap& mq, const CUtensorMap& mp, const QsigArgs& a, dim3 grid, uint32_t smem,
                           cudaStream_t st) {
-  static bool attr_done = false;   // per instantiation; the attribute is per device function
-  if (!attr_done) {
-    const cudaError_t e = cudaFuncSetAttribute(qsig_kernel<KB>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
-    if (e != cudaSuccess) return e;
-    attr_done = true;
-  }
+  static std::atomic<unsigned long long> limit_set{0};   // per instantiation
+  const cudaError_t e = ensure_smem_limit(limit_set, qsig_kernel<KB>, kMaxSmem);
+  if (e != cudaSuccess) return e;
   qsig_kernel<KB><<<grid, kQsigThreads, smem, st>>>(mq, mp, a);
   g_launches.fetch_add(1);
   return cudaGetLastError();
@@ -288,13 +305,10 @@ cudaError_t launch_qsig(int K, const CUtensorMap& mq, const CUtensorMap& mp, con
 // over bytes that are zero everywhere.
 laser_kv_status_t launch_select(const float* s_exact, const uint32_t* counts, int n_seg, int S, int anchors,
                                 int k_exact, int k_lsh, uint32_t count_max, int32_t* idx, cudaStream_t st) {
-  static bool attr_done = false;
+  static std::atomic<unsigned long long> limit_set{0};
   const size_t smem = (size_t)S * 9;
-  if (!attr_done) {
-    if (cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem - 2048) != cudaSuccess)
-      return fail(nullptr, LASER_KV_ERR_CUDA, "cudaFuncSetAttribute(select_kernel) failed");
-    attr_done = true;
-  }
+  if (ensure_smem_limit(limit_set, select_kernel, kMaxSmem - 2048) != cudaSuccess)
+    return fail(nullptr, LASER_KV_ERR_CUDA, "cudaFuncSetAttribute(select_kernel) failed");
   int top_shift = 24;
   if (count_max != 0) {
     top_shift = 0;
@@ -321,13 +335,9 @@ laser_kv_status_t launch_append(const AppendArgs& a, int n_seg, cudaStream_t st)
 
 template <int KB>
 cudaError_t launch_theory(const CUtensorMap& mk, const CUtensorMap& mq, const TheoryArgs& a, dim3 grid, cudaStream_t st) {
-  static bool configured = false;       // per instantiation; the attribute is idempotent
-  if (!configured) {
-    const cudaError_t e = cudaFuncSetAttribute(theory_kernel<KB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                               (int)theory_smem_bytes(kThMaxQueries));
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  static std::atomic<unsigned long long> limit_set{0};   // per instantiation
+  const cudaError_t e = ensure_smem_limit(limit_set, theory_kernel<KB>, (int)theory_smem_bytes(kThMaxQueries));
+  if (e != cudaSuccess) return e;
   theory_kernel<KB><<<grid, kThThreads, theory_smem_bytes(a.GW), st>>>(mk, mq, a);
   return cudaGetLastError();
 }
@@ -455,6 +465,7 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
                                         const void* Q_win, const int64_t kv_strides[3], const int64_t q_strides[3],
                                         int32_t n_blocks, void* stream) {
   if (!h) return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "select_block: NULL handle");
+  if (const laser_kv_status_t ds = check_device(h, "select_block")) return ds;
   const laser_kv_config_t& c = h->cfg;
   const Derived& d = h->d;
   if (layer < 0 || layer >= c.n_layers) return fail(h, LASER_KV_ERR_INVALID_ARG, "select_block: layer %d out of range", layer);
@@ -709,6 +720,7 @@ laser_kv_status_t laser_kv_decode_attention(laser_kv_handle_t h, int32_t layer, 
   const long long len = h->blocks_done[layer] * d.B;
   if (len < 1) return fail(h, LASER_KV_ERR_STATE, "decode_attention: layer %d cache is empty", layer);
   if (len > 0x7fffffffLL) return fail(h, LASER_KV_ERR_UNSUPPORTED, "decode_attention: cache longer than 2^31 entries");
+  if (const laser_kv_status_t ds = check_device(h, "decode_attention")) return ds;
   const int n_split = decode_splits(h, len);
   const size_t need = (size_t)c.batch * c.n_q_heads * n_split * kDecPartFloats * sizeof(float);
   if (scratch_bytes < need) return fail(h, LASER_KV_ERR_CAPACITY, "decode_attention: scratch needs %zu bytes, got %zu", need, scratch_bytes);
@@ -739,13 +751,9 @@ laser_kv_status_t laser_kv_decode_attention(laser_kv_handle_t h, int32_t layer, 
   a.counters = reinterpret_cast<int*>(h->ws + h->carve.dec_count);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const dim3 grid((unsigned)n_split, (unsigned)c.n_kv_heads, (unsigned)c.batch);
-  static bool configured = false;       // the attribute is idempotent
-  cudaError_t e = cudaSuccess;
-  if (!configured) {
-    e = cudaFuncSetAttribute(decode_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dec_smem_bytes());
-    if (e != cudaSuccess) return fail(h, LASER_KV_ERR_CUDA, "decode_split_kernel attribute: %s", cudaGetErrorString(e));
-    configured = true;
-  }
+  static std::atomic<unsigned long long> limit_set{0};
+  cudaError_t e = ensure_smem_limit(limit_set, decode_split_kernel, (int)dec_smem_bytes());
+  if (e != cudaSuccess) return fail(h, LASER_KV_ERR_CUDA, "decode_split_kernel attribute: %s", cudaGetErrorString(e));
   decode_split_kernel<<<grid, kDecThreads, dec_smem_bytes(), st>>>(mapK, mapV, a);
   g_launches.fetch_add(1);
   e = cudaGetLastError();
@@ -779,6 +787,7 @@ laser_kv_status_t laser_kv_debug_view(laser_kv_handle_t h, laser_kv_debug_t* out
 
 laser_kv_status_t laser_kv_poll_status(laser_kv_handle_t h, void* stream) {
   if (!h) return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "poll_status: NULL handle");
+  if (const laser_kv_status_t ds = check_device(h, "poll_status")) return ds;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   int host[4] = {0, 0, 0, 0};
   cudaError_t e = cudaMemcpyAsync(host, h->ws + h->carve.ctrl, sizeof host, cudaMemcpyDeviceToHost, st);
