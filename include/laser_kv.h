@@ -144,9 +144,11 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
 /* Same path driven from HOST memory: copies the (contiguous) host tensors K_host, V_host
  * [batch][H_kv][n_blocks*S][d] and Q_host [batch][H_q][W][d] into the caller's device staging
  * buffers K_stage, V_stage, Q_stage (same shapes), runs laser_kv_select_block on them, and
- * copies the appended positions (int32 [batch][H_kv][n_blocks*B]) to pos_out_host. All copies
- * are asynchronous on `stream` (pin the host buffers for overlap); the call does not
- * synchronise. pos_out_host may be NULL. */
+ * copies the appended positions (int32 [batch][H_kv][n_blocks*B]) to pos_out_host. The blocks
+ * travel in up to four chunks on a copy stream that the handle owns, ordered after the work
+ * already on `stream`; the selection of a chunk runs on `stream` once the chunk has landed, while
+ * the next chunk is copied. Everything the call does is complete when `stream` is (pin the host
+ * buffers, or the copies serialise); the call does not synchronise. pos_out_host may be NULL. */
 laser_kv_status_t laser_kv_select_block_host(laser_kv_handle_t h, int32_t layer,
                                              const void* K_host, const void* V_host,
                                              const void* Q_host, void* K_stage, void* V_stage,

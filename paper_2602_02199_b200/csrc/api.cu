@@ -78,6 +78,10 @@ struct laser_kv_ctx {
   bool have_call = false;
   int last_nb = 0;
   int last_fixups = 0;
+  // host-buffer path: copies run on a stream of their own, chunk by chunk
+  cudaStream_t copy_stream = nullptr;
+  cudaEvent_t ev_join = nullptr;
+  std::vector<cudaEvent_t> ev_chunk;
   // optional per-kernel timing (events only; no device memory)
   bool profiling = false;
   std::vector<cudaEvent_t> ev_pool;
@@ -650,20 +654,46 @@ laser_kv_status_t laser_kv_select_block_host(laser_kv_handle_t h, int32_t layer,
   if (n_blocks < 1 || n_blocks > h->cfg.max_blocks_per_call)
     return fail(h, LASER_KV_ERR_CAPACITY, "select_block_host: n_blocks out of range");
   const laser_kv_config_t& c = h->cfg;
+  if (const laser_kv_status_t ds = check_device(h, "select_block_host")) return ds;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const size_t T = (size_t)n_blocks * c.block_size;
-  const size_t kv_bytes = (size_t)c.batch * c.n_kv_heads * T * kHeadDim * 2;
   const size_t q_bytes = (size_t)c.batch * c.n_q_heads * c.window * kHeadDim * 2;
-  cudaError_t e;
-  if ((e = cudaMemcpyAsync(K_stage, K_host, kv_bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
-      (e = cudaMemcpyAsync(V_stage, V_host, kv_bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
-      (e = cudaMemcpyAsync(Q_stage, Q_host, q_bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess)
+  // The blocks travel in up to four chunks on the handle's copy stream; the selection of a chunk
+  // starts on `stream` as soon as its keys and values have landed, while the next chunk is copied.
+  constexpr int kHostChunks = 4;
+  const int n_chunks = n_blocks < kHostChunks ? n_blocks : kHostChunks;
+  cudaError_t e = cudaSuccess;
+  if (!h->copy_stream) e = cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking);
+  if (e == cudaSuccess && !h->ev_join) e = cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming);
+  while (e == cudaSuccess && (int)h->ev_chunk.size() < kHostChunks) {
+    cudaEvent_t ev;
+    if ((e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming)) == cudaSuccess) h->ev_chunk.push_back(ev);
+  }
+  if (e != cudaSuccess) return fail(h, LASER_KV_ERR_CUDA, "select_block_host: stream or event: %s", cudaGetErrorString(e));
+  // earlier work on `stream` may still read the staging buffers
+  if ((e = cudaEventRecord(h->ev_join, st)) != cudaSuccess || (e = cudaStreamWaitEvent(h->copy_stream, h->ev_join, 0)) != cudaSuccess ||
+      (e = cudaMemcpyAsync(Q_stage, Q_host, q_bytes, cudaMemcpyHostToDevice, h->copy_stream)) != cudaSuccess)
     return fail(h, LASER_KV_ERR_CUDA, "select_block_host: H2D copy: %s", cudaGetErrorString(e));
   const int64_t kvs[3] = {(int64_t)c.n_kv_heads * (int64_t)T * kHeadDim, (int64_t)T * kHeadDim, kHeadDim};
   const int64_t qs[3] = {(int64_t)c.n_q_heads * c.window * kHeadDim, (int64_t)c.window * kHeadDim, kHeadDim};
   const long long before = h->blocks_done[layer];
-  const laser_kv_status_t s = laser_kv_select_block(h, layer, K_stage, V_stage, Q_stage, kvs, qs, n_blocks, stream);
-  if (s != LASER_KV_OK) return s;
+  const size_t pitch = T * kHeadDim * 2, rows = (size_t)c.batch * c.n_kv_heads;
+  for (int ch = 0; ch < n_chunks; ++ch) {
+    const int b0 = (int)((long long)ch * n_blocks / n_chunks), b1 = (int)((long long)(ch + 1) * n_blocks / n_chunks);
+    const size_t off = (size_t)b0 * c.block_size * kHeadDim * 2;           // bytes into every (sequence, head) slab
+    const size_t width = (size_t)(b1 - b0) * c.block_size * kHeadDim * 2;
+    uint8_t* kd = static_cast<uint8_t*>(K_stage) + off;
+    uint8_t* vd = static_cast<uint8_t*>(V_stage) + off;
+    if ((e = cudaMemcpy2DAsync(kd, pitch, static_cast<const uint8_t*>(K_host) + off, pitch, width, rows,
+                               cudaMemcpyHostToDevice, h->copy_stream)) != cudaSuccess ||
+        (e = cudaMemcpy2DAsync(vd, pitch, static_cast<const uint8_t*>(V_host) + off, pitch, width, rows,
+                               cudaMemcpyHostToDevice, h->copy_stream)) != cudaSuccess ||
+        (e = cudaEventRecord(h->ev_chunk[ch], h->copy_stream)) != cudaSuccess ||
+        (e = cudaStreamWaitEvent(st, h->ev_chunk[ch], 0)) != cudaSuccess)
+      return fail(h, LASER_KV_ERR_CUDA, "select_block_host: H2D copy: %s", cudaGetErrorString(e));
+    const laser_kv_status_t s = laser_kv_select_block(h, layer, kd, vd, Q_stage, kvs, qs, b1 - b0, stream);
+    if (s != LASER_KV_OK) return s;
+  }
   if (pos_out_host) {
     const Derived& d = h->d;
     const size_t layer_off = (size_t)layer * c.batch * c.n_kv_heads * (size_t)d.cap;
@@ -818,6 +848,9 @@ void laser_kv_destroy(laser_kv_handle_t h) {
   if (!h) return;
   for (auto& set : h->ev_pending) for (cudaEvent_t ev : set) cudaEventDestroy(ev);
   for (cudaEvent_t ev : h->ev_pool) cudaEventDestroy(ev);
+  for (cudaEvent_t ev : h->ev_chunk) cudaEventDestroy(ev);
+  if (h->ev_join) cudaEventDestroy(h->ev_join);
+  if (h->copy_stream) cudaStreamDestroy(h->copy_stream);
   delete h;
 }
 
