@@ -147,8 +147,12 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
  * copies the appended positions (int32 [batch][H_kv][n_blocks*B]) to pos_out_host. The blocks
  * travel in up to four chunks on a copy stream that the handle owns, ordered after the work
  * already on `stream`; the selection of a chunk runs on `stream` once the chunk has landed, while
- * the next chunk is copied. Everything the call does is complete when `stream` is (pin the host
- * buffers, or the copies serialise); the call does not synchronise. pos_out_host may be NULL. */
+ * the next chunk is copied. Only the kept rows of V are ever read: when V_host is page-locked
+ * memory that the device can address (cudaHostAlloc / cudaHostRegister), the append kernel reads
+ * those rows in place over the bus and V_stage stays untouched; pageable V_host is copied like
+ * K_host. Everything the call does is complete when `stream` is (pin the host buffers, or the
+ * copies serialise); the host buffers must stay valid until then; the call does not synchronise.
+ * pos_out_host may be NULL. */
 laser_kv_status_t laser_kv_select_block_host(laser_kv_handle_t h, int32_t layer,
                                              const void* K_host, const void* V_host,
                                              const void* Q_host, void* K_stage, void* V_stage,

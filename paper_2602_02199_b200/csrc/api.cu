@@ -678,6 +678,18 @@ laser_kv_status_t laser_kv_select_block_host(laser_kv_handle_t h, int32_t layer,
   const int64_t qs[3] = {(int64_t)c.n_q_heads * c.window * kHeadDim, (int64_t)c.window * kHeadDim, kHeadDim};
   const long long before = h->blocks_done[layer];
   const size_t pitch = T * kHeadDim * 2, rows = (size_t)c.batch * c.n_kv_heads;
+  // Only the kept rows of V are ever read (by the append kernel). When the host V buffer is pinned
+  // and mapped into the device's address space the kernel reads those rows in place over the bus
+  // and V is not staged at all; pageable memory takes the copy.
+  const uint8_t* v_mapped = nullptr;
+  {
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, V_host) == cudaSuccess && at.type == cudaMemoryTypeHost && at.devicePointer &&
+        aligned16(at.devicePointer))
+      v_mapped = static_cast<const uint8_t*>(at.devicePointer);
+    else
+      cudaGetLastError();   // an unregistered pointer is not an error here
+  }
   for (int ch = 0; ch < n_chunks; ++ch) {
     const int b0 = (int)((long long)ch * n_blocks / n_chunks), b1 = (int)((long long)(ch + 1) * n_blocks / n_chunks);
     const size_t off = (size_t)b0 * c.block_size * kHeadDim * 2;           // bytes into every (sequence, head) slab
@@ -686,12 +698,13 @@ laser_kv_status_t laser_kv_select_block_host(laser_kv_handle_t h, int32_t layer,
     uint8_t* vd = static_cast<uint8_t*>(V_stage) + off;
     if ((e = cudaMemcpy2DAsync(kd, pitch, static_cast<const uint8_t*>(K_host) + off, pitch, width, rows,
                                cudaMemcpyHostToDevice, h->copy_stream)) != cudaSuccess ||
-        (e = cudaMemcpy2DAsync(vd, pitch, static_cast<const uint8_t*>(V_host) + off, pitch, width, rows,
-                               cudaMemcpyHostToDevice, h->copy_stream)) != cudaSuccess ||
+        (!v_mapped && (e = cudaMemcpy2DAsync(vd, pitch, static_cast<const uint8_t*>(V_host) + off, pitch, width, rows,
+                                             cudaMemcpyHostToDevice, h->copy_stream)) != cudaSuccess) ||
         (e = cudaEventRecord(h->ev_chunk[ch], h->copy_stream)) != cudaSuccess ||
         (e = cudaStreamWaitEvent(st, h->ev_chunk[ch], 0)) != cudaSuccess)
       return fail(h, LASER_KV_ERR_CUDA, "select_block_host: H2D copy: %s", cudaGetErrorString(e));
-    const laser_kv_status_t s = laser_kv_select_block(h, layer, kd, vd, Q_stage, kvs, qs, b1 - b0, stream);
+    const laser_kv_status_t s = laser_kv_select_block(h, layer, kd, v_mapped ? static_cast<const void*>(v_mapped + off) : vd,
+                                                      Q_stage, kvs, qs, b1 - b0, stream);
     if (s != LASER_KV_OK) return s;
   }
   if (pos_out_host) {
