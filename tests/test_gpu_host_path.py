@@ -10,8 +10,9 @@ from parity_util import to_np
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("nb,batch", [(1, 1), (5, 2), (8, 1)])
-def test_host_path_equals_device_path(nb, batch):
+@pytest.mark.parametrize("nb,batch,pin_v", [(1, 1, True), (5, 2, True), (8, 1, True), (5, 2, False)])
+def test_host_path_equals_device_path(nb, batch, pin_v):
+    """pin_v: the kept V rows are read in place from pinned memory; otherwise V is pageable and staged."""
     import torch
     from paper_2602_02199_b200 import binding as Bn
     S = 264
@@ -27,7 +28,9 @@ def test_host_path_equals_device_path(nb, batch):
         k, v = synth.kv_blocks(w, 0, b, 0, nb)
         Ks.append(k); Vs.append(v); Qs.append(synth.q_window(w, 0, b))
     hK = torch.from_numpy(np.stack(Ks).view(np.int16)).pin_memory()
-    hV = torch.from_numpy(np.stack(Vs).view(np.int16)).pin_memory()
+    hV = torch.from_numpy(np.stack(Vs).view(np.int16))
+    if pin_v:
+        hV = hV.pin_memory()
     hQ = torch.from_numpy(np.stack(Qs).view(np.int16)).pin_memory()
     ref = Bn.LaserKV(cfg, P)
     ref.laser_kv_select_block(0, hK.to(dev), hV.to(dev), hQ.to(dev), nb)
