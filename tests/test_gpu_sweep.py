@@ -72,3 +72,11 @@ def test_decode_and_closed_form_score_on_random_geometries(seed):
             want = O.collision_probability(q, run["K"][b, h, t * S:(t + 1) * S], K)
             err = np.abs(p[b, h, t] - want)
             assert (err <= 1e-3 * want + 1e-6).all(), (case, b, h, t, err.max())
+
+
+def test_select_call_at_the_largest_block_size():
+    """block_size 16384 (the limit of the selection kernel's shared memory), two blocks, 12-bit tables."""
+    w = synth.workload("tiny").with_(name="maxblock", n_q_heads=8, n_kv_heads=2, window=64, lsh_bits=12, lsh_tables=8,
+                                     block_size=16384, context_len=2 * 16384, needles="uniform:6", rope_base=500000.0)
+    run = run_workload_layer(w, 0)
+    check_run(w, run, segments=[(0, 0, 0), (0, 1, 1)])
