@@ -171,6 +171,16 @@ laser_kv_status_t laser_kv_debug_view(laser_kv_handle_t h, laser_kv_debug_t* out
  * recompute list overflowed). Clears the word. */
 laser_kv_status_t laser_kv_poll_status(laser_kv_handle_t h, void* stream);
 
+/* Per-layer budgets: an alternative allocation policy on the same kernels (Section 2 discusses
+ * methods that give layers different cache sizes; LASER-KV itself uses one B for every layer,
+ * Appendix B). Sets the number of tokens kept per block in `layer` to budget_per_block, split
+ * by the handle's protection divisor and alpha as in laser_kv_partition. The configured budget
+ * stays the maximum (it sizes the cache and the workspace): 0 <= budget_per_block <= it, else
+ * INVALID_ARG; the layer's cache must be empty (STATE otherwise; laser_kv_reset empties it).
+ * Later calls for the layer keep budget_per_block tokens per block; cache_view's len and decode
+ * attention follow. Host only. */
+laser_kv_status_t laser_kv_set_layer_budget(laser_kv_handle_t h, int32_t layer, int32_t budget_per_block);
+
 /* Forgets the contents of one layer's cache (layer = -1: all layers). Host only. */
 laser_kv_status_t laser_kv_reset(laser_kv_handle_t h, int32_t layer);
 

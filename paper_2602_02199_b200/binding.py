@@ -20,6 +20,7 @@ EXPORTS = [
     "laser_kv_window_scores_static", "laser_kv_window_scores_static_max_bytes",
     "laser_kv_collision_counts", "laser_kv_collision_counts_scratch_bytes", "laser_kv_consensus_accumulate",
     "laser_kv_decode_attention", "laser_kv_decode_attention_scratch_bytes", "laser_kv_collision_probability",
+    "laser_kv_set_layer_budget",
 ]
 
 
@@ -131,6 +132,8 @@ def load(build_if_missing: bool = True) -> C.CDLL:
                                               vp, vp]
     lib.laser_kv_consensus_accumulate.restype = i32
     lib.laser_kv_consensus_accumulate.argtypes = [vp, vp, i32, i32, i32, i32, i32, vp, vp, vp]
+    lib.laser_kv_set_layer_budget.restype = i32
+    lib.laser_kv_set_layer_budget.argtypes = [vp, i32, i32]
     lib.laser_kv_collision_probability.restype = i32
     lib.laser_kv_collision_probability.argtypes = [vp, vp, p(i64), p(i64), i32, i32, i32, i32, i32, i32, i32, vp, sz, vp, vp]
     lib.laser_kv_decode_attention_scratch_bytes.restype = sz
@@ -326,6 +329,9 @@ class LaserKV:
         cnt = (C.c_int32 * 16)()
         _check(self.lib.laser_kv_profile_read(self.handle, C.byref(n), names, ms, cnt), self.handle)
         return {names[i].decode(): (float(ms[i]), int(cnt[i])) for i in range(n.value)}
+
+    def laser_kv_set_layer_budget(self, layer, budget_per_block):
+        _check(self.lib.laser_kv_set_layer_budget(self.handle, layer, budget_per_block), self.handle)
 
     def laser_kv_reset(self, layer=-1):
         _check(self.lib.laser_kv_reset(self.handle, layer), self.handle)

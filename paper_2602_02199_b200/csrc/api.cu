@@ -74,6 +74,9 @@ struct laser_kv_ctx {
   EncodeTiledFn encode = nullptr;
   int num_sms = 1;
   std::vector<long long> blocks_done;   // per layer
+  struct LayerBudget { int B, anchors, k_exact, k_lsh; };
+  std::vector<LayerBudget> budget;      // per layer; the configured budget unless laser_kv_set_layer_budget changed it
+  int last_B = 0;                       // budget of the last select call (debug view)
   std::string last_error;
   bool have_call = false;
   int last_nb = 0;
@@ -446,6 +449,8 @@ laser_kv_status_t laser_kv_init(const laser_kv_config_t* cfg, const void* hyperp
   h->cachePos = reinterpret_cast<int32_t*>(cm + 2 * align_up(per * kHeadDim * 2));
   h->P = static_cast<const uint16_t*>(hyperplanes);
   h->blocks_done.assign(cfg->n_layers, 0);
+  h->budget.assign(cfg->n_layers, laser_kv_ctx::LayerBudget{d.B, d.anchors, d.k_exact, d.k_lsh});
+  h->last_B = d.B;
   {
     const uint64_t dims[2] = {(uint64_t)kHeadDim, (uint64_t)cfg->lsh_tables * cfg->lsh_bits};
     const uint64_t strides[1] = {(uint64_t)kHeadDim * 2};
@@ -492,7 +497,8 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
     return fail(h, LASER_KV_ERR_UNSUPPORTED, "select_block: absolute positions exceed int32");
 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const int S = c.block_size, nb = n_blocks, B = d.B;
+  const laser_kv_ctx::LayerBudget lb = h->budget[layer];
+  const int S = c.block_size, nb = n_blocks, B = lb.B;
   const int nseg = c.batch * c.n_kv_heads * nb;
   uint8_t* ws = h->ws;
   int* ctrl = reinterpret_cast<int*>(ws + h->carve.ctrl);
@@ -549,8 +555,8 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
   // A stage whose share of the recall budget is empty (alpha = 1: no LSH picks; alpha = 0 or n = 2:
   // no exact picks) is not computed, unless the debug view was asked for, which shows every
   // intermediate result.
-  const bool need_lsh = d.k_lsh > 0 || c.debug;
-  const bool need_exact = d.k_exact > 0 || c.debug;
+  const bool need_lsh = lb.k_lsh > 0 || c.debug;
+  const bool need_exact = lb.k_exact > 0 || c.debug;
   // 1. query signatures and bucket histograms; the kernel also clears the counts and restarts the
   //    fix-up counter (ctrl[1]) and the changed counter (ctrl[2]); the status word (ctrl[0]) is kept
   if (need_lsh) {
@@ -618,7 +624,7 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
   mark();
   // 6. two-stage top-k
   {
-    const laser_kv_status_t s = launch_select(s_exact, counts, nseg, S, d.anchors, d.k_exact, d.k_lsh,
+    const laser_kv_status_t s = launch_select(s_exact, counts, nseg, S, lb.anchors, lb.k_exact, lb.k_lsh,
                                                 (uint32_t)d.GW * (uint32_t)c.lsh_tables, idx, st);
     if (s != LASER_KV_OK) { h->last_error = g_last_error; return s; }
   }
@@ -641,6 +647,7 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
   h->blocks_done[layer] += nb;
   h->have_call = true;
   h->last_nb = nb;
+  h->last_B = B;
   return LASER_KV_OK;
 }
 
@@ -710,8 +717,9 @@ laser_kv_status_t laser_kv_select_block_host(laser_kv_handle_t h, int32_t layer,
   if (pos_out_host) {
     const Derived& d = h->d;
     const size_t layer_off = (size_t)layer * c.batch * c.n_kv_heads * (size_t)d.cap;
-    const int32_t* src = h->cachePos + layer_off + before * d.B;
-    e = cudaMemcpy2DAsync(pos_out_host, (size_t)n_blocks * d.B * 4, src, (size_t)d.cap * 4, (size_t)n_blocks * d.B * 4,
+    const size_t Bl = (size_t)h->budget[layer].B;
+    const int32_t* src = h->cachePos + layer_off + before * Bl;
+    e = cudaMemcpy2DAsync(pos_out_host, (size_t)n_blocks * Bl * 4, src, (size_t)d.cap * 4, (size_t)n_blocks * Bl * 4,
                           (size_t)c.batch * c.n_kv_heads, cudaMemcpyDeviceToHost, st);
     if (e != cudaSuccess) return fail(h, LASER_KV_ERR_CUDA, "select_block_host: D2H copy: %s", cudaGetErrorString(e));
   }
@@ -727,7 +735,7 @@ laser_kv_status_t laser_kv_cache_view(laser_kv_handle_t h, int32_t layer, laser_
   out->K = h->cacheK + layer_off * kHeadDim;
   out->V = h->cacheV + layer_off * kHeadDim;
   out->pos = h->cachePos + layer_off;
-  out->len = h->blocks_done[layer] * d.B;
+  out->len = h->blocks_done[layer] * h->budget[layer].B;
   out->cap = d.cap;
   out->kv_strides[0] = (int64_t)c.n_kv_heads * d.cap * kHeadDim;
   out->kv_strides[1] = d.cap * kHeadDim;
@@ -760,7 +768,7 @@ laser_kv_status_t laser_kv_decode_attention(laser_kv_handle_t h, int32_t layer, 
     return fail(h, LASER_KV_ERR_INVALID_ARG, "decode_attention: softmax_scale must be positive (0 selects the configured scale)");
   const int G = c.n_q_heads / c.n_kv_heads;
   if (G > kDecMaxGroup) return fail(h, LASER_KV_ERR_UNSUPPORTED, "decode_attention: more than %d query heads per KV head", kDecMaxGroup);
-  const long long len = h->blocks_done[layer] * d.B;
+  const long long len = h->blocks_done[layer] * h->budget[layer].B;
   if (len < 1) return fail(h, LASER_KV_ERR_STATE, "decode_attention: layer %d cache is empty", layer);
   if (len > 0x7fffffffLL) return fail(h, LASER_KV_ERR_UNSUPPORTED, "decode_attention: cache longer than 2^31 entries");
   if (const laser_kv_status_t ds = check_device(h, "decode_attention")) return ds;
@@ -820,7 +828,7 @@ laser_kv_status_t laser_kv_debug_view(laser_kv_handle_t h, laser_kv_debug_t* out
   out->batch = c.batch;
   out->n_kv_heads = c.n_kv_heads;
   out->block_size = c.block_size;
-  out->budget = h->d.B;
+  out->budget = h->last_B;
   out->gw = h->d.GW;
   out->lsh_tables = c.lsh_tables;
   out->lsh_bits = c.lsh_bits;
@@ -865,6 +873,22 @@ void laser_kv_destroy(laser_kv_handle_t h) {
   if (h->ev_join) cudaEventDestroy(h->ev_join);
   if (h->copy_stream) cudaStreamDestroy(h->copy_stream);
   delete h;
+}
+
+laser_kv_status_t laser_kv_set_layer_budget(laser_kv_handle_t h, int32_t layer, int32_t budget_per_block) {
+  if (!h) return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "set_layer_budget: NULL handle");
+  if (layer < 0 || layer >= h->cfg.n_layers) return fail(h, LASER_KV_ERR_INVALID_ARG, "set_layer_budget: layer out of range");
+  if (budget_per_block < 0 || budget_per_block > h->d.B)
+    return fail(h, LASER_KV_ERR_INVALID_ARG, "set_layer_budget: budget %d outside [0, %d] (the configured budget sizes the cache)",
+                budget_per_block, h->d.B);
+  if (h->blocks_done[layer] != 0)
+    return fail(h, LASER_KV_ERR_STATE, "set_layer_budget: layer %d already holds %lld blocks", layer, h->blocks_done[layer]);
+  laser_kv_ctx::LayerBudget lb;
+  lb.B = budget_per_block;
+  int loc;
+  laser_kv_partition(lb.B, h->cfg.protection_divisor, h->d.alpha, &lb.anchors, &loc, &lb.k_exact, &lb.k_lsh);
+  h->budget[layer] = lb;
+  return LASER_KV_OK;
 }
 
 laser_kv_status_t laser_kv_profile_enable(laser_kv_handle_t h, int32_t on) {
