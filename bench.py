@@ -661,12 +661,12 @@ def run_theory(args, w, rank, world, local_rank):
         return
     work = algorithmic_work(w, B)
     ms_per_step = ms / args.steps
-    # the closed-form kernel is bound by its element-wise chain: per (window query, key) pair 20 fp32
+    # the closed-form kernel is bound by its element-wise chain: per (window query, key) pair 19 fp32
     # operations (cosine 1, clamp 1, 1-x 1, square root 1, degree-7 polynomial 7, product 1, reflection
-    # 2, 1/pi 1, u^10 by squaring 4, sum 1) on 128 fp32 lanes per SM and clock
+    # 2, u^10 by squaring 4, sum 1) on 128 fp32 lanes per SM and clock
     pairs = float(w.batch) * nb * S * w.n_q_heads * w.window
     sm_mhz = (clocks or {}).get("sm_max_mhz") or 1965.0
-    peak = 128.0 / 20.0 * 148 * sm_mhz * 1e6 / 1e9            # G pairs/s
+    peak = 128.0 / 19.0 * 148 * sm_mhz * 1e6 / 1e9            # G pairs/s
     achieved = pairs / (kern_ms * 1e-3) / 1e9
     line = {
         "metric": METRIC, "value": whole_job_value(work["tokens"], args.steps, world, ms), "unit": UNIT, "n_gpus": world,
@@ -678,7 +678,7 @@ def run_theory(args, w, rank, world, local_rank):
         "clocks": clocks, "e2e": None, "gpu_launches": int(launches),
         "roofline": {"kernel": "theory_kernel", "bound": "alu", "achieved": achieved, "peak": peak, "unit": "Gpair/s",
                      "frac": achieved / peak, "traffic": None, "ms_per_launch": kern_ms,
-                     "peak_source": "20 fp32 operations per (query, key) pair on 128 lanes per SM and clock, 148 SMs, "
+                     "peak_source": "19 fp32 operations per (query, key) pair on 128 lanes per SM and clock, 148 SMs, "
                                     "maximum SM clock"},
         "cpu_baseline": None,
     }

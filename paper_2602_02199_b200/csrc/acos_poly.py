@@ -41,7 +41,7 @@ def fit(deg=7, iters=12):
 if __name__ == "__main__":
     coef, e = fit()
     for i, c in enumerate(coef):
-        print(f"a{i} = {c:.10e}")
+        print(f"a{i} = {c:.10e}    a{i} / pi = {c / np.pi:.10e}")
     x = np.linspace(0, 1, 100001)
     approx = np.sqrt(1 - x) * np.polyval(coef[::-1].astype(np.float32).astype(np.float64), x)
     print(f"max |P - f| = {e:.3e}; max |acos error| with float32 coefficients = {np.abs(approx - np.arccos(x)).max():.3e}")

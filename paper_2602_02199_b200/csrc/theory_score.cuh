@@ -55,11 +55,13 @@ __device__ __forceinline__ float sum_squares8(const uint4& w) {
   }
   return s;
 }
-// acos(x) ~= sqrt(1 - x) * P(x) on [0, 1], |error| < 8e-8 (degree 7, the form of Abramowitz & Stegun
-// 4.4.46; coefficients from the fit in acos_poly.py beside this file)
+// acos(x) / pi ~= sqrt(1 - x) * P(x) on [0, 1], |error| < 3e-8 (degree 7, the form of Abramowitz &
+// Stegun 4.4.46; the coefficients are those of the fit in acos_poly.py beside this file, divided by
+// pi). LKV_ACOS_TOP is the leading coefficient, LKV_ACOS_POLY the Horner steps below it.
+#define LKV_ACOS_TOP (-4.0197156638e-04f)
 #define LKV_ACOS_POLY(STEP) \
-  STEP(-1.2628309199e-03f) STEP(6.6712932680e-03f) STEP(-1.7089810817e-02f) STEP(3.0893053199e-02f) \
-  STEP(-5.0174715211e-02f) STEP(8.8979049893e-02f) STEP(-2.1459880383e-01f) STEP(1.5707963050e+00f)
+  STEP(2.1235386008e-03f) STEP(-5.4398557361e-03f) STEP(9.8335642476e-03f) STEP(-1.5971107888e-02f) \
+  STEP(2.8322911244e-02f) STEP(-6.8308920822e-02f) STEP(4.9999999306e-01f)
 __device__ __forceinline__ float sqrt_approx(float x) {
   float y;
   asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -77,21 +79,20 @@ __device__ __forceinline__ float2 pow_int2(float2 x) {
   }
   return r;
 }
-// (1 - theta/pi)^K for two cosines: u*pi = acos(-c) = pi - acos(c) (c >= 0), acos(|c|) (c < 0).
-// KB > 0: u^KB by multiplication; KB == 0: any K at run time as 2^(K log2(u pi) - K log2(pi)),
-// kbias = -K log2(pi). u = 0 gives 0 either way.
+// (1 - theta/pi)^K for two cosines: u = acos(-c) / pi = 1 - acos(c)/pi (c >= 0), acos(|c|)/pi (c < 0).
+// KB > 0: u^KB by multiplication; KB == 0: any K at run time as 2^(K log2 u). u = 0 gives 0 either way.
 template <int KB>
-__device__ __forceinline__ float2 collide_pow2(float2 c, float kbits, float kbias) {
+__device__ __forceinline__ float2 collide_pow2(float2 c, float kbits) {
   const float2 x = make_float2(fminf(fabsf(c.x), 1.f), fminf(fabsf(c.y), 1.f));
-  float2 p = make_float2(0.f, 0.f);                              // Horner, highest coefficient first
+  float2 p = make_float2(LKV_ACOS_TOP, LKV_ACOS_TOP);            // Horner, highest coefficient first
 #define LKV_HORNER(A) p = __ffma2_rn(p, x, make_float2(A, A));
   LKV_ACOS_POLY(LKV_HORNER)
 #undef LKV_HORNER
-  const float2 a = __fmul2_rn(make_float2(sqrt_approx(1.f - x.x), sqrt_approx(1.f - x.y)), p);
-  const float wx = c.x >= 0.f ? 3.14159265358979f - a.x : a.x;
-  const float wy = c.y >= 0.f ? 3.14159265358979f - a.y : a.y;
-  if (KB > 0) return pow_int2<KB>(__fmul2_rn(make_float2(wx, wy), make_float2(0.3183098861837907f, 0.3183098861837907f)));
-  return make_float2(ex2_approx(fmaf(kbits, lg2_approx(wx), kbias)), ex2_approx(fmaf(kbits, lg2_approx(wy), kbias)));
+  const float2 om = __ffma2_rn(x, make_float2(-1.f, -1.f), make_float2(1.f, 1.f));   // 1 - x
+  const float2 a = __fmul2_rn(make_float2(sqrt_approx(om.x), sqrt_approx(om.y)), p);
+  const float2 u = make_float2(c.x >= 0.f ? 1.f - a.x : a.x, c.y >= 0.f ? 1.f - a.y : a.y);
+  if (KB > 0) return pow_int2<KB>(u);
+  return make_float2(ex2_approx(kbits * lg2_approx(u.x)), ex2_approx(kbits * lg2_approx(u.y)));
 }
 
 template <int KB>
@@ -156,7 +157,7 @@ theory_kernel(const __grid_constant__ CUtensorMap map_k,    // K: (d, nb*S, H_kv
     }
   }
   asm volatile("bar.sync 1, %0;" ::"n"(kThWarps * 32) : "memory");     // the consumer warps only
-  const float kbits = (float)a.kbits, kbias = -1.6514961294723187f * (float)a.kbits, inv_gw = 1.0f / (float)a.GW;
+  const float kbits = (float)a.kbits, inv_gw = 1.0f / (float)a.GW;
   float* out = a.out + (((long long)(b * a.H_kv + h) * a.nb + t) * a.S);
 
   const int rows = (warp & 3) * 16;                                  // the warp's keys within a tile
@@ -197,8 +198,8 @@ theory_kernel(const __grid_constant__ CUtensorMap map_k,    // K: (d, nb*S, H_kv
         mma_bf16(acc, ak[2 * k2 + 1], qf[2], qf[3]);
       }
       const float2 r = *reinterpret_cast<const float2*>(rq + 8 * nt + 2 * c);
-      const float2 p_lo = collide_pow2<KB>(__fmul2_rn(make_float2(acc[0], acc[1]), __fmul2_rn(r, make_float2(rk_lo, rk_lo))), kbits, kbias);
-      const float2 p_hi = collide_pow2<KB>(__fmul2_rn(make_float2(acc[2], acc[3]), __fmul2_rn(r, make_float2(rk_hi, rk_hi))), kbits, kbias);
+      const float2 p_lo = collide_pow2<KB>(__fmul2_rn(make_float2(acc[0], acc[1]), __fmul2_rn(r, make_float2(rk_lo, rk_lo))), kbits);
+      const float2 p_hi = collide_pow2<KB>(__fmul2_rn(make_float2(acc[2], acc[3]), __fmul2_rn(r, make_float2(rk_hi, rk_hi))), kbits);
       sum_lo += p_lo.x + p_lo.y;
       sum_hi += p_hi.x + p_hi.y;
     }
