@@ -80,3 +80,19 @@ def test_select_call_at_the_largest_block_size():
                                      block_size=16384, context_len=2 * 16384, needles="uniform:6", rope_base=500000.0)
     run = run_workload_layer(w, 0)
     check_run(w, run, segments=[(0, 0, 0), (0, 1, 1)])
+
+
+@pytest.mark.parametrize("name,alpha", [("tiny", 0.75), ("tiny", 1.0), ("llama8b_32k", 0.75), ("qwen7b_128k", 0.75)])
+def test_planted_needles_stay_in_every_heads_cache(name, alpha):
+    """The synthetic contexts plant keys with cosine 0.9 to a window query of each KV head's group:
+    the exact stage must keep all of them, whatever else it keeps (a functional check of the selection
+    on needle-like structure, not an accuracy figure)."""
+    w = synth.workload(name).with_(alpha=alpha)
+    run = run_workload_layer(w, 0, debug=0, alpha=alpha)
+    _, _, pos, n = run["engine"].laser_kv_cache_view(0)
+    pos = to_np(pos)[:, :, :n]
+    for b in range(w.batch):
+        needles = synth.needle_positions(w, 0, b)
+        assert len(needles) > 0
+        for h in range(w.n_kv_heads):
+            assert np.isin(needles, pos[b, h]).all(), (b, h)
