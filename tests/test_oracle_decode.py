@@ -88,3 +88,18 @@ def test_large_logits_concentrate_on_the_aligned_entry_without_overflow():
     got = O.decode_attention(q, _bf16(base), v)
     assert np.isfinite(got).all()
     np.testing.assert_allclose(got[0], O.bf16_bits_to_f64(v[2]), rtol=1e-12, atol=1e-100)
+
+
+def test_matches_the_library_attention_routine():
+    """Plain softmax attention is a library routine: torch's scaled_dot_product_attention in float64."""
+    import torch
+    rng = np.random.default_rng(9)
+    G, n, d = 4, 300, 128
+    q = _bf16(rng.standard_normal((G, d)))
+    k = _bf16(rng.standard_normal((n, d)) * 2)
+    v = _bf16(rng.standard_normal((n, d)))
+    tq, tk, tv = (torch.from_numpy(O.bf16_bits_to_f64(x)) for x in (q, k, v))
+    want = torch.nn.functional.scaled_dot_product_attention(tq[None], tk[None], tv[None])[0].numpy()
+    np.testing.assert_allclose(O.decode_attention(q, k, v), want, rtol=1e-11, atol=1e-13)
+    want2 = torch.nn.functional.scaled_dot_product_attention(tq[None], tk[None], tv[None], scale=0.3)[0].numpy()
+    np.testing.assert_allclose(O.decode_attention(q, k, v, scale=0.3), want2, rtol=1e-11, atol=1e-13)

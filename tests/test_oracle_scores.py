@@ -109,3 +109,14 @@ def test_aligned_key_ranks_first():
     if here.size:
         rank = (s > s[here[0]]).sum()
         assert rank < 32
+
+
+def test_matches_the_library_softmax_routine():
+    """Column sums of scipy's softmax over the keys (a library routine) are the window scores."""
+    from scipy.special import softmax
+    rng = np.random.default_rng(21)
+    q = _bf16(rng.standard_normal((24, 128)))
+    k = _bf16(rng.standard_normal((200, 128)) * 1.5)
+    logits = (O.bf16_bits_to_f64(q) @ O.bf16_bits_to_f64(k).T) / math.sqrt(128)
+    want = softmax(logits, axis=1).sum(axis=0)
+    np.testing.assert_allclose(O.window_scores(q, k), want, rtol=1e-12)
