@@ -553,7 +553,25 @@ def run_decode(args, w, rank, world, local_rank):
     launches = Bn.laser_kv_launch_count() - launches0
     eng.laser_kv_poll_status()
     clocks = sampler.stop(t0, t1) if rank == 0 else None
-    ms, = max_over_ranks([ms], world, dev)
+    # end to end: the step's queries come from pinned host memory, its output goes back to the host
+    e2e_steps, e2e_ms = 0, 0.0
+    if not args.skip_e2e:
+        q_host = [q.cpu().pin_memory() for q in qs]
+        q_dev = torch.empty_like(qs[0])
+        out_host = torch.empty(out.shape, dtype=out.dtype).pin_memory()
+        e2e_steps = max(args.e2e_steps, 20)
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        f0.record()
+        for i in range(e2e_steps):
+            q_dev.copy_(q_host[i % n_layers], non_blocking=True)
+            eng.laser_kv_decode_attention(i % n_layers, q_dev, out=out)
+            out_host.copy_(out, non_blocking=True)
+            torch.cuda.current_stream().synchronize()          # the host reads the result of every step
+        f1.record()
+        barrier()
+        e2e_ms = f0.elapsed_time(f1)
+    ms, e2e_ms = max_over_ranks([ms, e2e_ms], world, dev)
     if world > 1:
         dist.destroy_process_group()
     if rank != 0:
@@ -563,6 +581,27 @@ def run_decode(args, w, rank, world, local_rank):
     entries = w.batch * H * length                               # cache entries read per step
     nbytes = entries * 2 * 128 * 2 + w.batch * w.n_q_heads * 128 * (2 + 4)
     achieved = nbytes / (ms_per_step * 1e-3) / 1e9
+    e2e = None
+    if e2e_steps:
+        e2e = {"value": whole_job_value(entries, e2e_steps, world, e2e_ms), "unit": "cache entries/s",
+               "h2d_bytes_per_step": int(qs[0].numel()) * 2, "d2h_bytes_per_step": int(out.numel()) * 4,
+               "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps}
+    cpu = None
+    if not args.skip_cpu:
+        # the oracle on a bounded sample: one KV head's group over the first entries of that head's cache
+        from oracle import laser_kv_oracle as O
+        Kc, Vc, _, n = eng.laser_kv_cache_view(0)
+        n_s = min(n, 16384)
+        kb = Kc[0, 0, :n_s].cpu().numpy().view(np.uint16)
+        vb = Vc[0, 0, :n_s].cpu().numpy().view(np.uint16)
+        qb = qs[0][0, :w.group].cpu().numpy().view(np.uint16)
+        O.decode_attention(qb, kb, vb)
+        reps, c0 = 0, time.time()
+        while time.time() - c0 < 5.0:
+            O.decode_attention(qb, kb, vb)
+            reps += 1
+        cpu = {"value": reps * n_s / (time.time() - c0), "unit": "cache entries/s", "cores": os.cpu_count(), "kind": "oracle",
+               "sample": f"one KV head's group over the first {n_s} cache entries of that head, repeated for 5 s"}
     line = {
         "metric": "decode_attention_cache_entries_per_s_per_layer", "value": whole_job_value(entries, args.steps, world, ms),
         "unit": "cache entries/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -571,12 +610,12 @@ def run_decode(args, w, rank, world, local_rank):
         "config": {"workload": w.name, "policy": "decode attention over the compacted cache of one layer",
                    "context_len": w.context_len, "cache_len_per_head": length, "batch": w.batch,
                    "l2": f"{n_layers} layers' caches cycled ({entries * 512 / 1e6:.0f} MB each)"},
-        "clocks": clocks, "e2e": None, "gpu_launches": int(launches),
+        "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         "roofline": {"kernel": "decode_split_kernel", "bound": "hbm", "achieved": achieved,
                      "peak": peaks["hbm"], "unit": "GB/s", "frac": achieved / peaks["hbm"],
                      "traffic": NCU_TRAFFIC_BYTES.get((w.name, "decode_split_kernel")),
                      "peak_source": f"hbm_gbs, {peaks['source']}", "bytes_per_launch": nbytes},
-        "cpu_baseline": None,
+        "cpu_baseline": cpu,
     }
     print(json.dumps(line), flush=True)
 
