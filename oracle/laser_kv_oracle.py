@@ -36,7 +36,7 @@ softmax over the block's own keys, bit = [projection >= 0], tie rule) are listed
 notes of the repository and restated at each function.
 
 Parity status: every function is pinned in the CPU test suite by something other than itself:
-budget and partition by the values the paper prints and hand-evaluated tables; the softmax
+budget and partition by tables evaluated by hand as exact fractions at the paper's settings; the softmax
 scores and the decode attention by library routines (scipy's softmax, torch's
 scaled_dot_product_attention in float64), hand cases and scalar loops; SimHash bits by hand
 cases and the (1 - theta/pi)^K collision rate; collision counts by a scalar triple loop; the
