@@ -293,13 +293,13 @@ def run_ours(args, w, rank, world, local_rank):
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
     e2e_ms = float("nan")
     pos_host = torch.empty((w.batch, w.n_kv_heads, nb * B), dtype=torch.int32).pin_memory()
-    stage = None if args.skip_e2e else tuple(torch.empty_like(t) for t in devs[0])
+    stages = None if args.skip_e2e else [tuple(torch.empty_like(t) for t in devs[0]) for _ in range(2)]
 
     def e2e_step(i):
         s = i % n_sets
         eng.laser_kv_reset(s)
-        eng.laser_kv_select_block_host(s, host[s][0], host[s][1], host[s][2], stage[0], stage[1], stage[2], nb,
-                                       pos_host)
+        st = stages[i % 2]                 # two sets of staging buffers: the next step's copies start under this step's tail
+        eng.laser_kv_select_block_host(s, host[s][0], host[s][1], host[s][2], st[0], st[1], st[2], nb, pos_host)
 
     if not args.skip_e2e:
         e2e_step(0)

@@ -152,7 +152,11 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
  * those rows in place over the bus and V_stage stays untouched; pageable V_host is copied like
  * K_host. Everything the call does is complete when `stream` is (pin the host buffers, or the
  * copies serialise); the host buffers must stay valid until then; the call does not synchronise.
- * pos_out_host may be NULL. */
+ * The copies of a call wait for the previous host-path call of this handle that used the same
+ * staging buffers (and, for buffers the handle has not seen, for everything already on `stream`):
+ * a caller who alternates between two sets of staging buffers gets the next call's copies running
+ * under the tail of the previous call. The staging buffers belong to the call until `stream` has
+ * passed it. pos_out_host may be NULL. */
 laser_kv_status_t laser_kv_select_block_host(laser_kv_handle_t h, int32_t layer,
                                              const void* K_host, const void* V_host,
                                              const void* Q_host, void* K_stage, void* V_stage,

@@ -85,6 +85,9 @@ struct laser_kv_ctx {
   cudaStream_t copy_stream = nullptr;
   cudaEvent_t ev_join = nullptr;
   std::vector<cudaEvent_t> ev_chunk;
+  // staging buffers of recent host-path calls with the event that marks the end of their last use
+  struct StageUse { const void* k; const void* v; const void* q; cudaEvent_t done; };
+  std::vector<StageUse> stage_use;
   // optional per-kernel timing (events only; no device memory)
   bool profiling = false;
   std::vector<cudaEvent_t> ev_pool;
@@ -677,9 +680,23 @@ laser_kv_status_t laser_kv_select_block_host(laser_kv_handle_t h, int32_t layer,
     if ((e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming)) == cudaSuccess) h->ev_chunk.push_back(ev);
   }
   if (e != cudaSuccess) return fail(h, LASER_KV_ERR_CUDA, "select_block_host: stream or event: %s", cudaGetErrorString(e));
-  // earlier work on `stream` may still read the staging buffers
-  if ((e = cudaEventRecord(h->ev_join, st)) != cudaSuccess || (e = cudaStreamWaitEvent(h->copy_stream, h->ev_join, 0)) != cudaSuccess ||
-      (e = cudaMemcpyAsync(Q_stage, Q_host, q_bytes, cudaMemcpyHostToDevice, h->copy_stream)) != cudaSuccess)
+  // The copies must not overtake earlier readers of the staging buffers. Buffers that an earlier
+  // host-path call of this handle used are released by that call's own event, so that a caller who
+  // alternates between two sets of staging buffers gets the next call's copies running under the
+  // tail of the previous call; buffers not seen before wait for everything already on `stream`.
+  constexpr size_t kStageSlots = 4;
+  bool known = false;
+  for (auto& u : h->stage_use) {
+    if (u.k == K_stage || u.v == V_stage || u.q == Q_stage) {
+      known = true;
+      if ((e = cudaStreamWaitEvent(h->copy_stream, u.done, 0)) != cudaSuccess)
+        return fail(h, LASER_KV_ERR_CUDA, "select_block_host: wait: %s", cudaGetErrorString(e));
+    }
+  }
+  if (!known && ((e = cudaEventRecord(h->ev_join, st)) != cudaSuccess ||
+                 (e = cudaStreamWaitEvent(h->copy_stream, h->ev_join, 0)) != cudaSuccess))
+    return fail(h, LASER_KV_ERR_CUDA, "select_block_host: wait: %s", cudaGetErrorString(e));
+  if ((e = cudaMemcpyAsync(Q_stage, Q_host, q_bytes, cudaMemcpyHostToDevice, h->copy_stream)) != cudaSuccess)
     return fail(h, LASER_KV_ERR_CUDA, "select_block_host: H2D copy: %s", cudaGetErrorString(e));
   const int64_t kvs[3] = {(int64_t)c.n_kv_heads * (int64_t)T * kHeadDim, (int64_t)T * kHeadDim, kHeadDim};
   const int64_t qs[3] = {(int64_t)c.n_q_heads * c.window * kHeadDim, (int64_t)c.window * kHeadDim, kHeadDim};
@@ -722,6 +739,28 @@ laser_kv_status_t laser_kv_select_block_host(laser_kv_handle_t h, int32_t layer,
     e = cudaMemcpy2DAsync(pos_out_host, (size_t)n_blocks * Bl * 4, src, (size_t)d.cap * 4, (size_t)n_blocks * Bl * 4,
                           (size_t)c.batch * c.n_kv_heads, cudaMemcpyDeviceToHost, st);
     if (e != cudaSuccess) return fail(h, LASER_KV_ERR_CUDA, "select_block_host: D2H copy: %s", cudaGetErrorString(e));
+  }
+  // remember when this call's last reader of the staging buffers is done
+  {
+    laser_kv_ctx::StageUse* slot = nullptr;
+    for (auto& u : h->stage_use)
+      if (u.k == K_stage && u.v == V_stage && u.q == Q_stage) slot = &u;
+    if (!slot) {
+      // drop every entry that shares a buffer with this call, then take a free or the oldest slot
+      for (size_t i = 0; i < h->stage_use.size();) {
+        auto& u = h->stage_use[i];
+        if (u.k == K_stage || u.v == V_stage || u.q == Q_stage) { cudaEventDestroy(u.done); h->stage_use.erase(h->stage_use.begin() + i); }
+        else ++i;
+      }
+      if (h->stage_use.size() >= kStageSlots) { cudaEventDestroy(h->stage_use.front().done); h->stage_use.erase(h->stage_use.begin()); }
+      cudaEvent_t ev;
+      if ((e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming)) != cudaSuccess)
+        return fail(h, LASER_KV_ERR_CUDA, "select_block_host: event: %s", cudaGetErrorString(e));
+      h->stage_use.push_back(laser_kv_ctx::StageUse{K_stage, V_stage, Q_stage, ev});
+      slot = &h->stage_use.back();
+    }
+    if ((e = cudaEventRecord(slot->done, st)) != cudaSuccess)
+      return fail(h, LASER_KV_ERR_CUDA, "select_block_host: event: %s", cudaGetErrorString(e));
   }
   return LASER_KV_OK;
 }
@@ -870,6 +909,7 @@ void laser_kv_destroy(laser_kv_handle_t h) {
   for (auto& set : h->ev_pending) for (cudaEvent_t ev : set) cudaEventDestroy(ev);
   for (cudaEvent_t ev : h->ev_pool) cudaEventDestroy(ev);
   for (cudaEvent_t ev : h->ev_chunk) cudaEventDestroy(ev);
+  for (auto& u : h->stage_use) cudaEventDestroy(u.done);
   if (h->ev_join) cudaEventDestroy(h->ev_join);
   if (h->copy_stream) cudaStreamDestroy(h->copy_stream);
   delete h;
