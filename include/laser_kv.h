@@ -156,7 +156,8 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
  * staging buffers (and, for buffers the handle has not seen, for everything already on `stream`):
  * a caller who alternates between two sets of staging buffers gets the next call's copies running
  * under the tail of the previous call. The staging buffers belong to the call until `stream` has
- * passed it. pos_out_host may be NULL. */
+ * passed it; any other work of the caller that touches them must be ordered against the host-path
+ * calls by the caller. pos_out_host may be NULL. */
 laser_kv_status_t laser_kv_select_block_host(laser_kv_handle_t h, int32_t layer,
                                              const void* K_host, const void* V_host,
                                              const void* Q_host, void* K_stage, void* V_stage,
