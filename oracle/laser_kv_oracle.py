@@ -55,7 +55,7 @@ import numpy as np
 __all__ = [
     "bf16_bits_to_f64", "budget", "partition", "window_scores", "simhash_projections",
     "simhash_buckets", "collision_counts", "topk_lower_index", "select_indices",
-    "select_block", "AppendOnlyCache", "BlockResult",
+    "group_queries", "select_block", "AppendOnlyCache", "BlockResult",
 ]
 
 
@@ -206,6 +206,21 @@ def select_indices(s_exact: np.ndarray, counts: np.ndarray, S: int, anchors: int
 # ----------------------------------------------------------------------------------------------
 # the whole per-block path for one (layer, sequence)
 # ----------------------------------------------------------------------------------------------
+def group_queries(q_bits: np.ndarray, n_kv_heads: int, h: int) -> np.ndarray:
+    """The window queries that score KV head h's keys: query heads h*G, h*G+1, ..., h*G+G-1
+    (G = H_q / H_kv consecutive query heads share one KV head - grouped-query attention), each
+    with its W window queries, as rows [G*W, d] in (head, window position) order.
+
+    q_bits uint16 [H_q, W, d].
+    """
+    h_q, W, d = q_bits.shape
+    if h_q % n_kv_heads:
+        raise ValueError("n_q_heads must be a multiple of n_kv_heads")
+    G = h_q // n_kv_heads
+    heads = [h * G + g for g in range(G)]
+    return np.concatenate([q_bits[i] for i in heads], axis=0)
+
+
 @dataclass
 class BlockResult:
     s_exact: np.ndarray          # float64 [H_kv, S]
@@ -240,7 +255,7 @@ def select_block(k_bits: np.ndarray, q_bits: np.ndarray, p_bits: np.ndarray, *, 
                       np.zeros((h_kv, G * W, n_tables), np.int64),
                       np.zeros((h_kv, G * W, n_tables)), [], [], np.zeros((h_kv, B), np.int64))
     for h in range(h_kv):
-        qg = q_bits[h * G:(h + 1) * G].reshape(G * W, d)
+        qg = group_queries(q_bits, h_kv, h)
         out.s_exact[h] = window_scores(qg, k_bits[h], scale)
         out.key_buckets[h], out.key_min_abs[h] = simhash_buckets(k_bits[h], p_bits, n_bits, n_tables)
         out.query_buckets[h], out.query_min_abs[h] = simhash_buckets(qg, p_bits, n_bits, n_tables)

@@ -69,11 +69,7 @@ def load(build_if_missing: bool = True) -> C.CDLL:
     if _lib is not None:
         return _lib
     if build_if_missing:
-        try:
-            _build.build()
-        except Exception:
-            if not os.path.exists(_build.LIB):
-                raise
+        _build.build()      # a no-op when the library is newer than its sources; a failed rebuild raises
     if not os.path.exists(_build.LIB):
         raise RuntimeError(f"{_build.LIB} is missing: build it with python -m paper_2602_02199_b200.build")
     lib = C.CDLL(_build.LIB)

@@ -180,7 +180,7 @@ def test_window_scores_entry_point_against_oracle():
             G = w.group
             for h in (0, w.n_kv_heads - 1):
                 for t in range(nb):
-                    want = O.window_scores(Q[h * G:(h + 1) * G].reshape(-1, 128), K[h, t * S:(t + 1) * S],
+                    want = O.window_scores(O.group_queries(Q, w.n_kv_heads, h), K[h, t * S:(t + 1) * S],
                                            None if scale == 0.0 else scale)
                     err = np.abs(out[0, h, t] - want)
                     assert (err <= SCORE_RTOL * np.abs(want) + SCORE_ATOL).all(), (name, h, t, err.max())
@@ -212,12 +212,21 @@ def test_gather_append_entry_point_bit_exact():
 
 
 def test_headline_config_full_size_sampled_segments():
+    import torch
     # 128k context, 16 blocks of 8192 in one call (the launch shape the benchmark times); the
     # oracle checks sampled (head, block) segments in full and the cache of every segment.
     w = synth.workload("llama8b_128k")
     run = run_workload_layer(w, 3, debug=1)
     segs = [(0, 0, 0), (0, 3, 1), (0, 5, 7), (0, 7, 15), (0, 2, 11)]   # blocks holding needles included
     check_run(w, run, segments=segs)
+    # the benchmarked path keeps no per-key bucket ids (debug = 0), which is another branch of the
+    # projection epilogue: its cache must equal, bit for bit, the one the oracle has just checked
+    lean = run_workload_layer(w, 3, debug=0, inputs_of=run)
+    n = run["n_blocks"] * run["B"]
+    for x, y in zip(run["engine"].laser_kv_cache_view(0)[:3], lean["engine"].laser_kv_cache_view(0)[:3]):
+        assert torch.equal(x[:, :, :n], y[:, :, :n])
+    d1, d0 = run["engine"].laser_kv_debug_view(), lean["engine"].laser_kv_debug_view()
+    assert torch.equal(d1.counts, d0.counts) and torch.equal(d1.s_exact, d0.s_exact) and torch.equal(d1.idx, d0.idx)
 
 
 @pytest.mark.parametrize("name,n_blocks,segs", [

@@ -68,7 +68,7 @@ def test_decode_and_closed_form_score_on_random_geometries(seed):
         p = to_np(p)
         for _ in range(3):
             b, h, t = int(rng.integers(batch)), int(rng.integers(hkv)), int(rng.integers(nb))
-            q = run["Q"][b, h * G:(h + 1) * G].reshape(G * W, 128)
+            q = O.group_queries(run["Q"][b], hkv, h)
             want = O.collision_probability(q, run["K"][b, h, t * S:(t + 1) * S], K)
             err = np.abs(p[b, h, t] - want)
             assert (err <= 1e-3 * want + 1e-6).all(), (case, b, h, t, err.max())

@@ -39,7 +39,7 @@ def test_collision_probability_against_oracle(name, S, nb, batch):
     G = w.group
     for b in range(batch):
         for h in range(w.n_kv_heads):
-            q = Q[b, h * G:(h + 1) * G].reshape(G * w.window, w.head_dim)
+            q = O.group_queries(Q[b], w.n_kv_heads, h)
             for t in range(nb):
                 want = O.collision_probability(q, K[b, h, t * S:(t + 1) * S], w.lsh_bits)
                 err = np.abs(got[b, h, t] - want)
