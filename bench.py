@@ -422,6 +422,7 @@ def run_consensus(args, w, rank, world, local_rank):
     scr_s = torch.empty(Bn.laser_kv_window_scores_scratch_bytes(1, w.n_q_heads, H, S, w.window, nb), dtype=torch.uint8,
                         device=dev)
     scr_c = None
+    bad_idx = torch.zeros(1, dtype=torch.int32, device=dev)
 
     def step(i):
         nonlocal scr_c
@@ -432,7 +433,7 @@ def run_consensus(args, w, rank, world, local_rank):
         idx = Bn.laser_kv_two_stage_topk(s_acc.view(nb, S), c_acc.view(nb, S), a, k_e, k_l)
         for h in range(H):
             Bn.laser_kv_gather_append(tk[0, h].view(nb, S, 128), tv[0, h].view(nb, S, 128), idx, Kd[h].view(nb, B, 128),
-                                      Vd[h].view(nb, B, 128), pos[h].view(nb, B), 0, 0)
+                                      Vd[h].view(nb, B, 128), pos[h].view(nb, B), 0, 0, bad_idx)
 
     def barrier():
         if world > 1:
@@ -651,6 +652,7 @@ def run_theory(args, w, rank, world, local_rank):
     scr_s = torch.empty(Bn.laser_kv_window_scores_scratch_bytes(w.batch, w.n_q_heads, H, S, w.window, nb),
                         dtype=torch.uint8, device=dev)
     scr_p = torch.empty(256, dtype=torch.uint8, device=dev)
+    bad_idx = torch.zeros(1, dtype=torch.int32, device=dev)
     ev = []
 
     def step(i, timed=False):
@@ -664,7 +666,7 @@ def run_theory(args, w, rank, world, local_rank):
             e1.record()
             ev.append((e0, e1))
         idx = Bn.laser_kv_two_stage_topk(s.view(nseg, S), p.view(torch.int32).view(nseg, S), a, k_e, k_l)
-        Bn.laser_kv_gather_append(tk.view(nseg, S, 128), tv.view(nseg, S, 128), idx, Kd, Vd, pos, 0, 0)
+        Bn.laser_kv_gather_append(tk.view(nseg, S, 128), tv.view(nseg, S, 128), idx, Kd, Vd, pos, 0, 0, bad_idx)
 
     def barrier():
         if world > 1:

@@ -134,6 +134,8 @@ laser_kv_status_t laser_kv_init(const laser_kv_config_t* cfg, const void* hyperp
  * candidates with the most SimHash collisions (ties: lower index). Rows are appended in
  * ascending position at [len, len + n_blocks*B); len advances on the host. The blocks' absolute
  * positions continue from the blocks already appended to this layer.
+ * A handle's workspace serves one call at a time: calls on the same handle must be issued to one
+ * stream (or be ordered by the caller); concurrent streams need one handle each.
  * Errors: CAPACITY if the cache cannot take n_blocks more blocks or n_blocks exceeds
  * max_blocks_per_call (nothing is launched). */
 laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, const void* K_blk,
@@ -157,7 +159,9 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
  * a caller who alternates between two sets of staging buffers gets the next call's copies running
  * under the tail of the previous call. The staging buffers belong to the call until `stream` has
  * passed it; any other work of the caller that touches them must be ordered against the host-path
- * calls by the caller. pos_out_host may be NULL. */
+ * calls by the caller. pos_out_host may be NULL. If the call fails after some chunks were launched,
+ * those chunks' blocks stay appended (laser_kv_cache_view's len tells how many) and the rest are
+ * not. */
 laser_kv_status_t laser_kv_select_block_host(laser_kv_handle_t h, int32_t layer,
                                              const void* K_host, const void* V_host,
                                              const void* Q_host, void* K_stage, void* V_stage,
@@ -185,6 +189,16 @@ laser_kv_status_t laser_kv_poll_status(laser_kv_handle_t h, void* stream);
  * Later calls for the layer keep budget_per_block tokens per block; cache_view's len and decode
  * attention follow. Host only. */
 laser_kv_status_t laser_kv_set_layer_budget(laser_kv_handle_t h, int32_t layer, int32_t budget_per_block);
+
+/* Diagnostics: poll budget of the hand-off waits inside the streaming kernels (tile landed, stage
+ * free, accumulator ready / drained, exchange areas). Every such wait is bounded: when its budget
+ * runs out the waiting role records LASER_KV_ERR_TIMEOUT in the status word that
+ * laser_kv_poll_status reads, the kernel lets copies and tensor-core work already in flight finish
+ * (those waits always keep the built-in budget), frees its tensor memory and returns; the results of
+ * that call are then incomplete. max_polls = 0 restores the built-in budgets (a second or more,
+ * never reached by a working pipeline); a small value makes the give-up path reachable on purpose,
+ * which is what the tests use it for. Host only; applies to later calls on this handle. */
+laser_kv_status_t laser_kv_set_wait_budget(laser_kv_handle_t h, uint32_t max_polls);
 
 /* Forgets the contents of one layer's cache (layer = -1: all layers). Host only. */
 laser_kv_status_t laser_kv_reset(laser_kv_handle_t h, int32_t layer);
@@ -263,11 +277,18 @@ laser_kv_status_t laser_kv_window_scores(const void* K_blk, const void* Q_win,
  * The first call on each device looks up the array's device address (with the CUDA device of
  * the inputs current, as for every call); make that first call before starting any stream
  * capture. All calls on a device share the one array: it still holds the previous call's
- * partials (the status word at its start is cleared by every call, everything else is
- * overwritten before it is read), and two calls whose kernels overlap on the GPU - different
+ * partials (everything but the status word at its start is overwritten before it is read), and
+ * two calls whose kernels overlap on the GPU - different
  * streams, or different host threads - race on it. Serialise them.
- * Arguments and results are those of laser_kv_window_scores without scratch/scratch_bytes. */
+ * Arguments and results are those of laser_kv_window_scores without scratch/scratch_bytes.
+ * The status word of these calls lives at the start of the built-in array, where the caller cannot
+ * look: laser_kv_window_scores_static_status(stream) synchronises `stream`, copies the word to the
+ * host (a plain 4-byte copy, no allocation), and returns LASER_KV_OK or the first error a kernel of
+ * any earlier static call on this device recorded (LASER_KV_ERR_TIMEOUT: a bounded device-side wait
+ * gave up and that call's scores are incomplete), clearing it. The word is sticky: it is not reset
+ * by later calls, only by reading it. */
 size_t laser_kv_window_scores_static_max_bytes(void);
+laser_kv_status_t laser_kv_window_scores_static_status(void* stream);
 laser_kv_status_t laser_kv_window_scores_static(const void* K_blk, const void* Q_win,
                                                 const int64_t kv_strides[3], const int64_t q_strides[3],
                                                 int32_t batch, int32_t n_q_heads, int32_t n_kv_heads,
@@ -331,15 +352,24 @@ laser_kv_status_t laser_kv_consensus_accumulate(const float* s_exact, const uint
 
 /* Append step (Sections 1 and 3): for each of n_segments segments copies rows idx[seg][i] of the
  * segment's K and V (dev bf16, row length d = 128, consecutive rows `src_row_stride` elements
- * apart, segment s starting at src + s*src_seg_stride) to dst rows [dst_offset + i] of the
- * segment's cache (segments dst_seg_stride elements apart, rows d apart) and writes
- * pos_base + idx[seg][i] to pos_out[s*pos_seg_stride + dst_offset + i]. */
+ * apart, n_src_rows rows per segment, segment s starting at src + s*src_seg_stride) to dst rows
+ * [dst_offset + i] of the segment's cache (segments dst_seg_stride elements apart, rows d apart,
+ * dst_capacity rows per segment) and writes pos_base + idx[seg][i] to
+ * pos_out[s*pos_seg_stride + dst_offset + i].
+ *   idx    : dev int32 [n_segments][n_keep], values in [0, n_src_rows). An index outside that range
+ *            is never dereferenced: its row and position are skipped and *status becomes
+ *            LASER_KV_ERR_INVALID_ARG.
+ *   status : dev int32, 4-byte aligned, owned by the caller; cleared by the call (on `stream`) and
+ *            set by the kernel as described; read it after `stream` has passed the call.
+ * Errors on the host: CAPACITY when dst_offset + n_keep exceeds dst_capacity (nothing is launched). */
 laser_kv_status_t laser_kv_gather_append(const void* K_src, const void* V_src,
                                          int64_t src_seg_stride, int64_t src_row_stride,
-                                         const int32_t* idx, int32_t n_segments, int32_t n_keep,
-                                         void* K_dst, void* V_dst, int64_t dst_seg_stride,
+                                         int32_t n_src_rows, const int32_t* idx, int32_t n_segments,
+                                         int32_t n_keep, void* K_dst, void* V_dst,
+                                         int64_t dst_seg_stride, int64_t dst_capacity,
                                          int32_t* pos_out, int64_t pos_seg_stride,
-                                         int64_t dst_offset, int32_t pos_base, void* stream);
+                                         int64_t dst_offset, int32_t pos_base, int32_t* status,
+                                         void* stream);
 
 /* Decode-phase attention over a layer's compacted cache (Section 3: once a block is processed only
  * the selected tokens stay in the KV cache and serve the decoding phase; Section 4.1 evaluates the

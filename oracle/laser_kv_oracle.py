@@ -30,6 +30,9 @@ What each function follows:
                           introduction's append-only accumulative memory.
 * ``decode_attention``  - Section 3 (the kept tokens serve the decoding phase): softmax attention
                           of one decode query over the cache entries of its KV head.
+* ``lookback_partition`` / ``select_block_lookback`` / ``LookbackPrefill`` - Section 3.2 (block
+                          processing and boundary smoothing): the scoring window of block t also
+                          covers the tail of block t-1, whose tokens are pruned only then.
 
 Readings taken where the paper is silent (rounding of B/n and alpha*B_long, per-block anchors,
 softmax over the block's own keys, bit = [projection >= 0], tie rule) are listed in the design
@@ -42,7 +45,9 @@ scaled_dot_product_attention in float64), hand cases and scalar loops; SimHash b
 cases and the (1 - theta/pi)^K collision rate; collision counts by a scalar triple loop; the
 closed-form recall score by special angles and by the empirical collision fraction it is the
 expectation of; top-k by exhaustive subset search; the consensus sums and the append-only cache
-by their invariants. The paper prints no numeric example of scores or chosen sets, so there is
+by their invariants; the look-back rule by its reduction to the plain rule when the local window
+is empty, by exhaustive subset search over its candidate set, by a hand case and by the keep-count
+and append-only invariants. The paper prints no numeric example of scores or chosen sets, so there is
 no golden vector of that kind.
 """
 from __future__ import annotations
@@ -56,6 +61,7 @@ __all__ = [
     "bf16_bits_to_f64", "budget", "partition", "window_scores", "simhash_projections",
     "simhash_buckets", "collision_counts", "topk_lower_index", "select_indices",
     "group_queries", "select_block", "AppendOnlyCache", "BlockResult",
+    "lookback_partition", "select_block_lookback", "LookbackPrefill", "LookbackResult",
 ]
 
 
@@ -373,3 +379,130 @@ def decode_attention(q_bits: np.ndarray, k_bits: np.ndarray, v_bits: np.ndarray,
     p = np.exp(s)
     p = p / p.sum(axis=1, keepdims=True)
     return p @ v
+
+
+# ----------------------------------------------------------------------------------------------
+# look-back boundary smoothing (Section 3.2)
+# ----------------------------------------------------------------------------------------------
+# Reading taken (the text says only that the scoring window of block t is expanded to include the
+# tail of block t-1, so that tokens at a block's edge are evaluated with the context that follows
+# them before they are pruned): the "tail" is the block's local sliding window, its last
+# a = floor(B/n) tokens. Without look-back those tokens are kept unconditionally by their own
+# block. With look-back the window slides: block t-1 does not decide about them; they are scored
+# together with block t's keys against block t's window queries (one softmax over a + S keys) and
+# compete with block t's candidates. Per block (index g in the sequence):
+#   g = 0 : scored keys = the block; kept = anchors [0, a) + Algorithm 1 on C = [a, S - a) with
+#           B_long = B - 2a; the tail [S - a, S) is held back. B - a entries appended.
+#   g >= 1: scored keys = held-back tail of block g-1 (a keys) followed by the block (S keys);
+#           kept = anchors of the block + Algorithm 1 on C = tail(g-1) + [a, S - a) of the block
+#           with B_long = B - a (the recall budget plus the a entries the slid window released);
+#           the block's own tail is held back. B entries appended, in position order.
+#   close : the tail of the last block is appended as it is (nothing follows it). a entries.
+# After m blocks and the close the cache holds m * B entries per head, as without look-back.
+def lookback_partition(B: int, n: int, alpha: float, first: bool):
+    """(anchors, held_back, B_long, k_exact, k_lsh) of one look-back step; see the rule above."""
+    a, _, b_long0, _, _ = partition(B, n, alpha)
+    b_long = b_long0 if first else B - a
+    k_e = int(math.floor(float(alpha) * float(b_long)))
+    k_e = max(0, min(k_e, b_long))
+    return a, a, b_long, k_e, b_long - k_e
+
+
+@dataclass
+class LookbackResult:
+    s_exact: np.ndarray          # float64 [H_kv, n_scored]   n_scored = S (first block) or a + S
+    counts: np.ndarray           # int64   [H_kv, n_scored]
+    k_exact: list                # per KV head: picks of the exact stage, scored-key indices, ascending
+    k_lsh: list                  # per KV head: picks of the LSH stage
+    idx: np.ndarray              # int64   [H_kv, n_kept] kept scored-key indices, ascending
+    offset: int                  # position of scored key 0 relative to the block's first token (0 or -a)
+
+
+def select_block_lookback(k_prev_tail, k_bits: np.ndarray, q_bits: np.ndarray, p_bits: np.ndarray, *,
+                          n_bits: int, n_tables: int, B: int, n: int, alpha: float = 0.75,
+                          scale: float | None = None) -> LookbackResult:
+    """One look-back step for one block of one (layer, sequence).
+
+    k_prev_tail: uint16 [H_kv, a, d], the held-back tail of the previous block, or None for the
+    first block of the sequence. k_bits uint16 [H_kv, S, d]; q_bits uint16 [H_q, W, d]; p_bits
+    uint16 [L*K, d]. Indices in the result count the scored keys: the previous tail first
+    (when there is one), then the block.
+    """
+    h_kv, S, d = k_bits.shape
+    first = k_prev_tail is None
+    a, _, b_long, k_e, k_l = lookback_partition(B, n, alpha, first)
+    if 2 * a > S or B > S:
+        raise ValueError("budget does not fit the block")
+    if first:
+        scored = k_bits
+        off = 0
+    else:
+        if k_prev_tail.shape != (h_kv, a, d):
+            raise ValueError("the held-back tail must have floor(B/n) rows per head")
+        scored = np.concatenate([k_prev_tail, k_bits], axis=1)
+        off = a
+    n_scored = scored.shape[1]
+    # candidates: the previous tail, and the block without its anchors and without its own tail
+    cand = np.concatenate([np.arange(0, off, dtype=np.int64),
+                           np.arange(off + a, off + S - a, dtype=np.int64)])
+    anchors = np.arange(off, off + a, dtype=np.int64)
+    n_kept = a + b_long
+    if b_long > cand.size:
+        raise ValueError("recall budget exceeds the candidate set")
+    out = LookbackResult(np.zeros((h_kv, n_scored)), np.zeros((h_kv, n_scored), np.int64), [], [],
+                         np.zeros((h_kv, n_kept), np.int64), -off)
+    for h in range(h_kv):
+        qg = group_queries(q_bits, h_kv, h)
+        out.s_exact[h] = window_scores(qg, scored[h], scale)          # one softmax over all scored keys
+        kb, _ = simhash_buckets(scored[h], p_bits, n_bits, n_tables)
+        qb, _ = simhash_buckets(qg, p_bits, n_bits, n_tables)
+        out.counts[h] = collision_counts(qb, kb)
+        k_ex = topk_lower_index(cand, out.s_exact[h], k_e)
+        residual = np.setdiff1d(cand, k_ex, assume_unique=True)
+        k_ls = topk_lower_index(residual, out.counts[h], k_l)
+        out.k_exact.append(k_ex)
+        out.k_lsh.append(k_ls)
+        out.idx[h] = np.sort(np.concatenate([anchors, k_ex, k_ls]))
+    return out
+
+
+class LookbackPrefill:
+    """Block-by-block prefill of one (layer, sequence) with look-back: owns the append-only cache
+    and the held-back tail between steps."""
+
+    def __init__(self, n_kv_heads: int, head_dim: int, capacity: int, *, n_bits: int, n_tables: int,
+                 B: int, n: int, alpha: float = 0.75, scale: float | None = None):
+        self.cache = AppendOnlyCache(n_kv_heads, head_dim, capacity)
+        self.kw = dict(n_bits=n_bits, n_tables=n_tables, B=B, n=n, alpha=alpha, scale=scale)
+        self.a = B // n
+        self.tail = None             # (k, v, first position) of the held-back tokens
+        self.blocks = 0
+        self.closed = False
+
+    def step(self, k_bits, v_bits, q_bits, p_bits) -> LookbackResult:
+        if self.closed:
+            raise ValueError("the sequence was closed")
+        S = k_bits.shape[1]
+        start = self.blocks * S
+        prev = None if self.tail is None else self.tail[0]
+        r = select_block_lookback(prev, k_bits, q_bits, p_bits, **self.kw)
+        if self.tail is None:
+            ks, vs = k_bits, v_bits
+        else:
+            ks = np.concatenate([self.tail[0], k_bits], axis=1)
+            vs = np.concatenate([self.tail[1], v_bits], axis=1)
+        self.cache.append(ks, vs, r.idx, start + r.offset)
+        a = self.a
+        self.tail = (k_bits[:, S - a:].copy(), v_bits[:, S - a:].copy(), start + S - a)
+        self.blocks += 1
+        return r
+
+    def close(self):
+        """Appends the last block's held-back tail: nothing follows it, so nothing can prune it."""
+        if self.closed or self.tail is None:
+            raise ValueError("nothing to close")
+        k, v, pos0 = self.tail
+        a = k.shape[1]
+        idx = np.tile(np.arange(a, dtype=np.int64), (k.shape[0], 1))
+        self.cache.append(k, v, idx, pos0)
+        self.closed = True

@@ -20,7 +20,7 @@ EXPORTS = [
     "laser_kv_window_scores_static", "laser_kv_window_scores_static_max_bytes",
     "laser_kv_collision_counts", "laser_kv_collision_counts_scratch_bytes", "laser_kv_consensus_accumulate",
     "laser_kv_decode_attention", "laser_kv_decode_attention_scratch_bytes", "laser_kv_collision_probability",
-    "laser_kv_set_layer_budget",
+    "laser_kv_set_layer_budget", "laser_kv_set_wait_budget", "laser_kv_window_scores_static_status",
 ]
 
 
@@ -106,7 +106,11 @@ def load(build_if_missing: bool = True) -> C.CDLL:
     lib.laser_kv_two_stage_topk.restype = i32
     lib.laser_kv_two_stage_topk.argtypes = [vp, vp, i32, i32, i32, i32, i32, vp, vp]
     lib.laser_kv_gather_append.restype = i32
-    lib.laser_kv_gather_append.argtypes = [vp, vp, i64, i64, vp, i32, i32, vp, vp, i64, vp, i64, i64, i32, vp]
+    lib.laser_kv_gather_append.argtypes = [vp, vp, i64, i64, i32, vp, i32, i32, vp, vp, i64, i64, vp, i64, i64, i32, vp, vp]
+    lib.laser_kv_set_wait_budget.restype = i32
+    lib.laser_kv_set_wait_budget.argtypes = [vp, C.c_uint32]
+    lib.laser_kv_window_scores_static_status.restype = i32
+    lib.laser_kv_window_scores_static_status.argtypes = [vp]
     lib.laser_kv_profile_enable.restype = i32
     lib.laser_kv_profile_enable.argtypes = [vp, i32]
     lib.laser_kv_profile_read.restype = i32
@@ -329,6 +333,9 @@ class LaserKV:
     def laser_kv_set_layer_budget(self, layer, budget_per_block):
         _check(self.lib.laser_kv_set_layer_budget(self.handle, layer, budget_per_block), self.handle)
 
+    def laser_kv_set_wait_budget(self, max_polls):
+        _check(self.lib.laser_kv_set_wait_budget(self.handle, max_polls), self.handle)
+
     def laser_kv_reset(self, layer=-1):
         _check(self.lib.laser_kv_reset(self.handle, layer), self.handle)
 
@@ -344,13 +351,15 @@ def laser_kv_two_stage_topk(s_exact, counts, anchors, k_exact, k_lsh, stream=Non
     return idx
 
 
-def laser_kv_gather_append(K_src, V_src, idx, K_dst, V_dst, pos_out, dst_offset, pos_base, stream=None):
+def laser_kv_gather_append(K_src, V_src, idx, K_dst, V_dst, pos_out, dst_offset, pos_base, status, stream=None):
     """K_src, V_src [n_seg][rows][128]; idx int32 [n_seg][n_keep]; K_dst, V_dst [n_seg][cap][128];
-    pos_out int32 [n_seg][cap]."""
+    pos_out int32 [n_seg][cap]; status int32 device tensor of one element (0 afterwards unless an
+    index was out of range)."""
     n_seg, n_keep = idx.shape
-    _check(load().laser_kv_gather_append(_ptr(K_src), _ptr(V_src), K_src.stride(0), K_src.stride(1), _ptr(idx),
-                                         n_seg, n_keep, _ptr(K_dst), _ptr(V_dst), K_dst.stride(0), _ptr(pos_out),
-                                         pos_out.stride(0), dst_offset, pos_base, _stream_ptr(stream)))
+    _check(load().laser_kv_gather_append(_ptr(K_src), _ptr(V_src), K_src.stride(0), K_src.stride(1), K_src.shape[1],
+                                         _ptr(idx), n_seg, n_keep, _ptr(K_dst), _ptr(V_dst), K_dst.stride(0),
+                                         K_dst.shape[1], _ptr(pos_out), pos_out.stride(0), dst_offset, pos_base,
+                                         _ptr(status), _stream_ptr(stream)))
 
 
 def laser_kv_window_scores_scratch_bytes(batch, n_q_heads, n_kv_heads, block_size, window, n_blocks) -> int:
@@ -443,3 +452,9 @@ def laser_kv_window_scores_static(K_blk, Q_win, block_size, n_blocks, out, softm
     _check(load().laser_kv_window_scores_static(_ptr(K_blk), _ptr(Q_win), ks, qs, batch, h_q, h_kv, block_size,
                                                 window, n_blocks, softmax_scale, _ptr(out), _stream_ptr(stream)))
     return out
+
+
+def laser_kv_window_scores_static_status(stream=None):
+    """Raises LaserKVError if a kernel of an earlier laser_kv_window_scores_static call on the current
+    device recorded an error (and clears it); synchronises the stream."""
+    _check(load().laser_kv_window_scores_static_status(_stream_ptr(stream)))

@@ -88,6 +88,7 @@ struct laser_kv_ctx {
   // staging buffers of recent host-path calls with the event that marks the end of their last use
   struct StageUse { const void* k; const void* v; const void* q; cudaEvent_t done; };
   std::vector<StageUse> stage_use;
+  uint32_t handoff_polls = 0;           // 0: built-in wait budgets (laser_kv_set_wait_budget)
   // optional per-kernel timing (events only; no device memory)
   bool profiling = false;
   std::vector<cudaEvent_t> ev_pool;
@@ -554,6 +555,7 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
     cudaEventRecord(ev, st);
     marks.push_back(ev);
   };
+  // rows that are kept whatever the scores say travel on the side stream from now on
   mark();
   // A stage whose share of the recall budget is empty (alpha = 1: no LSH picks; alpha = 0 or n = 2:
   // no exact picks) is not computed, unless the debug view was asked for, which shows every
@@ -584,6 +586,8 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
   sa.lse_part = lse_part; sa.lse2 = lse2; sa.s_exact = s_exact; sa.counts = counts; sa.hist = hist;
   sa.key_buckets = key_buckets; sa.fix_items = fix_items; sa.fix_count = ctrl + 1; sa.fix_cap = d.fix_cap;
   sa.status = ctrl;
+  sa.polls = h->handoff_polls ? h->handoff_polls : kMaxPolls;
+  sa.spin_polls = h->handoff_polls ? h->handoff_polls : kMaxSpinPolls;
 
   mark();
   // 2. per-query log-sum-exp over each block's keys
@@ -639,12 +643,12 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
     AppendArgs aa{static_cast<const uint16_t*>(K_blk), static_cast<const uint16_t*>(V_blk),
                   kv_strides[0], kv_strides[1], kv_strides[2], c.n_kv_heads, nb, S, B, idx,
                   h->cacheK + layer_off * kHeadDim, h->cacheV + layer_off * kHeadDim, h->cachePos + layer_off,
-                  d.cap * kHeadDim, d.cap, done * B, (int)(done * S)};
+                  d.cap * kHeadDim, d.cap, done * B, (int)(done * S), S, ctrl};
     const laser_kv_status_t s = launch_append(aa, nseg, st);
     if (s != LASER_KV_OK) { h->last_error = g_last_error; return s; }
   }
-#undef LKV_CUDA
   mark();
+#undef LKV_CUDA
   if (h->profiling && marks.size() == kProfKernels + 1) h->ev_pending.push_back(marks);
   else for (cudaEvent_t ev : marks) h->ev_pool.push_back(ev);
   h->blocks_done[layer] += nb;
@@ -685,16 +689,17 @@ laser_kv_status_t laser_kv_select_block_host(laser_kv_handle_t h, int32_t layer,
   // alternates between two sets of staging buffers gets the next call's copies running under the
   // tail of the previous call; buffers not seen before wait for everything already on `stream`.
   constexpr size_t kStageSlots = 4;
-  bool known = false;
+  bool k_known = false, v_known = false, q_known = false;
   for (auto& u : h->stage_use) {
     if (u.k == K_stage || u.v == V_stage || u.q == Q_stage) {
-      known = true;
+      k_known |= u.k == K_stage; v_known |= u.v == V_stage; q_known |= u.q == Q_stage;
       if ((e = cudaStreamWaitEvent(h->copy_stream, u.done, 0)) != cudaSuccess)
         return fail(h, LASER_KV_ERR_CUDA, "select_block_host: wait: %s", cudaGetErrorString(e));
     }
   }
-  if (!known && ((e = cudaEventRecord(h->ev_join, st)) != cudaSuccess ||
-                 (e = cudaStreamWaitEvent(h->copy_stream, h->ev_join, 0)) != cudaSuccess))
+  // any buffer the handle has not seen may still be in use by work already on `stream`
+  if (!(k_known && v_known && q_known) && ((e = cudaEventRecord(h->ev_join, st)) != cudaSuccess ||
+                                           (e = cudaStreamWaitEvent(h->copy_stream, h->ev_join, 0)) != cudaSuccess))
     return fail(h, LASER_KV_ERR_CUDA, "select_block_host: wait: %s", cudaGetErrorString(e));
   if ((e = cudaMemcpyAsync(Q_stage, Q_host, q_bytes, cudaMemcpyHostToDevice, h->copy_stream)) != cudaSuccess)
     return fail(h, LASER_KV_ERR_CUDA, "select_block_host: H2D copy: %s", cudaGetErrorString(e));
@@ -714,34 +719,10 @@ laser_kv_status_t laser_kv_select_block_host(laser_kv_handle_t h, int32_t layer,
     else
       cudaGetLastError();   // an unregistered pointer is not an error here
   }
-  for (int ch = 0; ch < n_chunks; ++ch) {
-    const int b0 = (int)((long long)ch * n_blocks / n_chunks), b1 = (int)((long long)(ch + 1) * n_blocks / n_chunks);
-    const size_t off = (size_t)b0 * c.block_size * kHeadDim * 2;           // bytes into every (sequence, head) slab
-    const size_t width = (size_t)(b1 - b0) * c.block_size * kHeadDim * 2;
-    uint8_t* kd = static_cast<uint8_t*>(K_stage) + off;
-    uint8_t* vd = static_cast<uint8_t*>(V_stage) + off;
-    if ((e = cudaMemcpy2DAsync(kd, pitch, static_cast<const uint8_t*>(K_host) + off, pitch, width, rows,
-                               cudaMemcpyHostToDevice, h->copy_stream)) != cudaSuccess ||
-        (!v_mapped && (e = cudaMemcpy2DAsync(vd, pitch, static_cast<const uint8_t*>(V_host) + off, pitch, width, rows,
-                                             cudaMemcpyHostToDevice, h->copy_stream)) != cudaSuccess) ||
-        (e = cudaEventRecord(h->ev_chunk[ch], h->copy_stream)) != cudaSuccess ||
-        (e = cudaStreamWaitEvent(st, h->ev_chunk[ch], 0)) != cudaSuccess)
-      return fail(h, LASER_KV_ERR_CUDA, "select_block_host: H2D copy: %s", cudaGetErrorString(e));
-    const laser_kv_status_t s = laser_kv_select_block(h, layer, kd, v_mapped ? static_cast<const void*>(v_mapped + off) : vd,
-                                                      Q_stage, kvs, qs, b1 - b0, stream);
-    if (s != LASER_KV_OK) return s;
-  }
-  if (pos_out_host) {
-    const Derived& d = h->d;
-    const size_t layer_off = (size_t)layer * c.batch * c.n_kv_heads * (size_t)d.cap;
-    const size_t Bl = (size_t)h->budget[layer].B;
-    const int32_t* src = h->cachePos + layer_off + before * Bl;
-    e = cudaMemcpy2DAsync(pos_out_host, (size_t)n_blocks * Bl * 4, src, (size_t)d.cap * 4, (size_t)n_blocks * Bl * 4,
-                          (size_t)c.batch * c.n_kv_heads, cudaMemcpyDeviceToHost, st);
-    if (e != cudaSuccess) return fail(h, LASER_KV_ERR_CUDA, "select_block_host: D2H copy: %s", cudaGetErrorString(e));
-  }
-  // remember when this call's last reader of the staging buffers is done
-  {
+  // Remembers when the last reader of the staging buffers (so far) is done. Also called when the call
+  // fails between chunks: the chunks already launched still read the buffers, and the blocks they
+  // appended stay appended.
+  auto remember_use = [&]() -> cudaError_t {
     laser_kv_ctx::StageUse* slot = nullptr;
     for (auto& u : h->stage_use)
       if (u.k == K_stage && u.v == V_stage && u.q == Q_stage) slot = &u;
@@ -754,14 +735,43 @@ laser_kv_status_t laser_kv_select_block_host(laser_kv_handle_t h, int32_t layer,
       }
       if (h->stage_use.size() >= kStageSlots) { cudaEventDestroy(h->stage_use.front().done); h->stage_use.erase(h->stage_use.begin()); }
       cudaEvent_t ev;
-      if ((e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming)) != cudaSuccess)
-        return fail(h, LASER_KV_ERR_CUDA, "select_block_host: event: %s", cudaGetErrorString(e));
+      const cudaError_t ce = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
+      if (ce != cudaSuccess) return ce;
       h->stage_use.push_back(laser_kv_ctx::StageUse{K_stage, V_stage, Q_stage, ev});
       slot = &h->stage_use.back();
     }
-    if ((e = cudaEventRecord(slot->done, st)) != cudaSuccess)
-      return fail(h, LASER_KV_ERR_CUDA, "select_block_host: event: %s", cudaGetErrorString(e));
+    return cudaEventRecord(slot->done, st);
+  };
+  for (int ch = 0; ch < n_chunks; ++ch) {
+    const int b0 = (int)((long long)ch * n_blocks / n_chunks), b1 = (int)((long long)(ch + 1) * n_blocks / n_chunks);
+    const size_t off = (size_t)b0 * c.block_size * kHeadDim * 2;           // bytes into every (sequence, head) slab
+    const size_t width = (size_t)(b1 - b0) * c.block_size * kHeadDim * 2;
+    uint8_t* kd = static_cast<uint8_t*>(K_stage) + off;
+    uint8_t* vd = static_cast<uint8_t*>(V_stage) + off;
+    if ((e = cudaMemcpy2DAsync(kd, pitch, static_cast<const uint8_t*>(K_host) + off, pitch, width, rows,
+                               cudaMemcpyHostToDevice, h->copy_stream)) != cudaSuccess ||
+        (!v_mapped && (e = cudaMemcpy2DAsync(vd, pitch, static_cast<const uint8_t*>(V_host) + off, pitch, width, rows,
+                                             cudaMemcpyHostToDevice, h->copy_stream)) != cudaSuccess) ||
+        (e = cudaEventRecord(h->ev_chunk[ch], h->copy_stream)) != cudaSuccess ||
+        (e = cudaStreamWaitEvent(st, h->ev_chunk[ch], 0)) != cudaSuccess) {
+      remember_use();
+      return fail(h, LASER_KV_ERR_CUDA, "select_block_host: H2D copy: %s", cudaGetErrorString(e));
+    }
+    const laser_kv_status_t s = laser_kv_select_block(h, layer, kd, v_mapped ? static_cast<const void*>(v_mapped + off) : vd,
+                                                      Q_stage, kvs, qs, b1 - b0, stream);
+    if (s != LASER_KV_OK) { remember_use(); return s; }
   }
+  if (pos_out_host) {
+    const Derived& d = h->d;
+    const size_t layer_off = (size_t)layer * c.batch * c.n_kv_heads * (size_t)d.cap;
+    const size_t Bl = (size_t)h->budget[layer].B;
+    const int32_t* src = h->cachePos + layer_off + before * Bl;
+    e = cudaMemcpy2DAsync(pos_out_host, (size_t)n_blocks * Bl * 4, src, (size_t)d.cap * 4, (size_t)n_blocks * Bl * 4,
+                          (size_t)c.batch * c.n_kv_heads, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return fail(h, LASER_KV_ERR_CUDA, "select_block_host: D2H copy: %s", cudaGetErrorString(e));
+  }
+  if ((e = remember_use()) != cudaSuccess)
+    return fail(h, LASER_KV_ERR_CUDA, "select_block_host: event: %s", cudaGetErrorString(e));
   return LASER_KV_OK;
 }
 
@@ -931,6 +941,12 @@ laser_kv_status_t laser_kv_set_layer_budget(laser_kv_handle_t h, int32_t layer, 
   return LASER_KV_OK;
 }
 
+laser_kv_status_t laser_kv_set_wait_budget(laser_kv_handle_t h, uint32_t max_polls) {
+  if (!h) return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "set_wait_budget: NULL handle");
+  h->handoff_polls = max_polls;
+  return LASER_KV_OK;
+}
+
 laser_kv_status_t laser_kv_profile_enable(laser_kv_handle_t h, int32_t on) {
   if (!h) return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "profile_enable: NULL handle");
   for (auto& set : h->ev_pending) for (cudaEvent_t ev : set) h->ev_pool.push_back(ev);
@@ -1037,7 +1053,8 @@ EncodeTiledFn driver_encode_fn() {
 
 // Log-sum-exp pass then score pass, with the partials in `scratch` (device, g.total bytes).
 laser_kv_status_t run_window_scores(const ScoreGeom& g, const void* K_blk, const void* Q_win, const int64_t kv_strides[3],
-                                    const int64_t q_strides[3], uint8_t* scratch, float* s_exact_out, cudaStream_t st) {
+                                    const int64_t q_strides[3], uint8_t* scratch, bool clear_status, float* s_exact_out,
+                                    cudaStream_t st) {
   if (!K_blk || !Q_win || !kv_strides || !q_strides || !s_exact_out)
     return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "window_scores: NULL argument");
   if (!aligned16(K_blk) || !aligned16(Q_win) || !aligned16(s_exact_out))
@@ -1077,8 +1094,9 @@ laser_kv_status_t run_window_scores(const ScoreGeom& g, const void* K_blk, const
     if (r != CUDA_SUCCESS) return fail(nullptr, LASER_KV_ERR_CUDA, "window_scores: tensor map of Q failed (CUresult %d)", (int)r);
   }
   cudaError_t e;
-  // the status word must start at zero; the partials are fully overwritten before they are read
-  if ((e = cudaMemsetAsync(scratch, 0, 256, st)) != cudaSuccess)
+  // caller scratch: the status word must start at zero (the built-in array starts at zero and keeps
+  // the first error until it is read); the partials are fully overwritten before they are read
+  if (clear_status && (e = cudaMemsetAsync(scratch, 0, 256, st)) != cudaSuccess)
     return fail(nullptr, LASER_KV_ERR_CUDA, "window_scores: memset: %s", cudaGetErrorString(e));
   StreamArgs sa;
   memset(&sa, 0, sizeof sa);
@@ -1096,6 +1114,7 @@ laser_kv_status_t run_window_scores(const ScoreGeom& g, const void* K_blk, const
   sa.lse2 = reinterpret_cast<float*>(scratch + g.off_lse2);
   sa.s_exact = s_exact_out;
   sa.status = reinterpret_cast<int*>(scratch);
+  sa.polls = kMaxPolls; sa.spin_polls = kMaxSpinPolls;
   StreamArgs a1 = sa;
   a1.stat_rows = g.GW;
   a1.stat_rows_alloc = ((g.GW + 127) / 128) * 128;
@@ -1130,7 +1149,7 @@ laser_kv_status_t laser_kv_window_scores(const void* K_blk, const void* Q_win, c
     return fail(nullptr, LASER_KV_ERR_ALIGNMENT, "window_scores: scratch must be 256-byte aligned");
   if (scratch_bytes < g.total)
     return fail(nullptr, LASER_KV_ERR_CAPACITY, "window_scores: scratch needs %zu bytes, got %zu", g.total, scratch_bytes);
-  return run_window_scores(g, K_blk, Q_win, kv_strides, q_strides, static_cast<uint8_t*>(scratch), s_exact_out,
+  return run_window_scores(g, K_blk, Q_win, kv_strides, q_strides, static_cast<uint8_t*>(scratch), true, s_exact_out,
                            static_cast<cudaStream_t>(stream));
 }
 
@@ -1182,7 +1201,25 @@ laser_kv_status_t laser_kv_window_scores_static(const void* K_blk, const void* Q
                 g.total, (unsigned)LASER_KV_STATIC_SCRATCH_BYTES);
   uint8_t* scratch = nullptr;
   if ((s = static_scratch_address(&scratch)) != LASER_KV_OK) return s;
-  return run_window_scores(g, K_blk, Q_win, kv_strides, q_strides, scratch, s_exact_out, static_cast<cudaStream_t>(stream));
+  return run_window_scores(g, K_blk, Q_win, kv_strides, q_strides, scratch, false, s_exact_out, static_cast<cudaStream_t>(stream));
+}
+
+laser_kv_status_t laser_kv_window_scores_static_status(void* stream) {
+  uint8_t* scratch = nullptr;
+  const laser_kv_status_t s = static_scratch_address(&scratch);
+  if (s != LASER_KV_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int word = 0;
+  cudaError_t e = cudaMemcpyAsync(&word, scratch, sizeof word, cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) return fail(nullptr, LASER_KV_ERR_CUDA, "window_scores_static_status: %s", cudaGetErrorString(e));
+  if (word == 0) return LASER_KV_OK;
+  e = cudaMemsetAsync(scratch, 0, sizeof word, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) return fail(nullptr, LASER_KV_ERR_CUDA, "window_scores_static_status: %s", cudaGetErrorString(e));
+  if (word == LASER_KV_ERR_TIMEOUT)
+    return fail(nullptr, LASER_KV_ERR_TIMEOUT, "window_scores_static: a bounded device-side wait gave up; the scores of that call are incomplete");
+  return fail(nullptr, (laser_kv_status_t)word, "window_scores_static: device status word %d", word);
 }
 
 // ---- collision counts on caller-fed inputs ---------------------------------------------------------
@@ -1320,6 +1357,7 @@ laser_kv_status_t laser_kv_collision_counts(const void* K_blk, const void* Q_win
     sa.stat_rows = cg.TC * lsh_bits; sa.stat_rows_alloc = sa.stat_rows;
     sa.counts = counts_out; sa.hist = hist; sa.fix_items = fix_items; sa.fix_count = ctrl + 1; sa.fix_cap = cg.fix_cap;
     sa.status = ctrl;
+    sa.polls = kMaxPolls; sa.spin_polls = kMaxSpinPolls;
     const uint32_t smem = stream_smem_bytes(kProj, sa.stat_rows_alloc, cg.TC * (2 << lsh_bits));
     if ((e = launch_proj(lsh_bits, cg.TC, mapK, mapP, sa, stream_grid(sa.n_tiles, num_sms), smem, st)) != cudaSuccess)
       return fail(nullptr, LASER_KV_ERR_CUDA, "collision_counts: projection pass: %s", cudaGetErrorString(e));
@@ -1434,20 +1472,28 @@ laser_kv_status_t laser_kv_consensus_accumulate(const float* s_exact, const uint
 }
 
 laser_kv_status_t laser_kv_gather_append(const void* K_src, const void* V_src, int64_t src_seg_stride,
-                                         int64_t src_row_stride, const int32_t* idx, int32_t n_segments,
-                                         int32_t n_keep, void* K_dst, void* V_dst, int64_t dst_seg_stride,
-                                         int32_t* pos_out, int64_t pos_seg_stride, int64_t dst_offset, int32_t pos_base,
+                                         int64_t src_row_stride, int32_t n_src_rows, const int32_t* idx,
+                                         int32_t n_segments, int32_t n_keep, void* K_dst, void* V_dst,
+                                         int64_t dst_seg_stride, int64_t dst_capacity, int32_t* pos_out,
+                                         int64_t pos_seg_stride, int64_t dst_offset, int32_t pos_base, int32_t* status,
                                          void* stream) {
-  if (!K_src || !V_src || !idx || !K_dst || !V_dst || !pos_out)
+  if (!K_src || !V_src || !idx || !K_dst || !V_dst || !pos_out || !status)
     return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "gather_append: NULL argument");
-  if (n_segments < 1 || n_keep < 0 || dst_offset < 0) return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "gather_append: bad size");
+  if (n_segments < 1 || n_keep < 0 || dst_offset < 0 || n_src_rows < 0 || dst_capacity < 0)
+    return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "gather_append: bad size");
+  if (dst_offset + (int64_t)n_keep > dst_capacity)
+    return fail(nullptr, LASER_KV_ERR_CAPACITY, "gather_append: entries [%lld, %lld) do not fit a destination of %lld entries",
+                (long long)dst_offset, (long long)dst_offset + n_keep, (long long)dst_capacity);
   if (!aligned16(K_src) || !aligned16(V_src) || !aligned16(K_dst) || !aligned16(V_dst) || (src_seg_stride % 8) ||
-      (src_row_stride % 8) || (dst_seg_stride % 8))
+      (src_row_stride % 8) || (dst_seg_stride % 8) || (reinterpret_cast<uintptr_t>(status) & 3u))
     return fail(nullptr, LASER_KV_ERR_ALIGNMENT, "gather_append: pointers 16-byte aligned, strides multiples of 8");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const cudaError_t e = cudaMemsetAsync(status, 0, sizeof(int32_t), st);
+  if (e != cudaSuccess) return fail(nullptr, LASER_KV_ERR_CUDA, "gather_append: memset: %s", cudaGetErrorString(e));
   AppendArgs aa{static_cast<const uint16_t*>(K_src), static_cast<const uint16_t*>(V_src), src_seg_stride, 0,
                 src_row_stride, 1, 1, 0, n_keep, idx, static_cast<uint16_t*>(K_dst), static_cast<uint16_t*>(V_dst),
-                pos_out, dst_seg_stride, pos_seg_stride, dst_offset, pos_base};
-  return launch_append(aa, n_segments, static_cast<cudaStream_t>(stream));
+                pos_out, dst_seg_stride, pos_seg_stride, dst_offset, pos_base, n_src_rows, status};
+  return launch_append(aa, n_segments, st);
 }
 
 }  // extern "C"

@@ -250,9 +250,12 @@ struct AppendArgs {
   long long pos_seg_stride;
   long long dst_off0;           // first destination entry of block t = 0
   int pos_base0;                // absolute position of token 0 of block t = 0
+  int n_src_rows;               // rows of a source segment: an index outside [0, n_src_rows) is not read
+  int* status;                  // receives kAppendBadIndex when an index was out of range
 };
 
 constexpr int kAppendRowsPerCta = 64;
+constexpr int kAppendBadIndex = 1;   // LASER_KV_ERR_INVALID_ARG
 
 __device__ __forceinline__ uint4 ld_nc_v4(const void* p) {
   uint4 v;
@@ -271,15 +274,21 @@ __global__ void __launch_bounds__(256) append_kernel(const AppendArgs a) {
   const int i_end = min(a.B, (int)(blockIdx.x + 1) * kAppendRowsPerCta);
   const long long src_base = b * a.ks_b + h * a.ks_h + (long long)t * a.S * a.ks_t;
   const long long dst_base = bh * a.c_seg_stride + (a.dst_off0 + (long long)t * a.B) * 128;
+  int32_t* pos = a.pos + bh * a.pos_seg_stride + a.dst_off0 + (long long)t * a.B;
+  const int32_t* idx = a.idx + (size_t)seg * a.B;
   for (int i = blockIdx.x * kAppendRowsPerCta + (threadIdx.x >> 4); i < i_end; i += 16) {
-    const int src = a.idx[(size_t)seg * a.B + i];
+    const int src = idx[i];
+    if ((unsigned)src >= (unsigned)a.n_src_rows) {          // never read outside the segment
+      if (part == 0) atomicCAS(a.status, 0, kAppendBadIndex);
+      continue;
+    }
     const long long so = src_base + (long long)src * a.ks_t + part * 8;
     const long long dof = dst_base + (long long)i * 128 + part * 8;
     const uint4 kv = ld_nc_v4(a.K + so);
     const uint4 vv = ld_nc_v4(a.V + so);
     *reinterpret_cast<uint4*>(a.Kc + dof) = kv;
     *reinterpret_cast<uint4*>(a.Vc + dof) = vv;
-    if (part == 0) a.pos[bh * a.pos_seg_stride + a.dst_off0 + (long long)t * a.B + i] = a.pos_base0 + t * a.S + src;
+    if (part == 0) pos[i] = a.pos_base0 + t * a.S + src;
   }
 }
 

@@ -43,12 +43,33 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 // Bounded waits for the phase with the given parity, written as one PTX loop each so that the
 // fast path (phase already complete) is a try_wait and a branch. Both return false when the poll
 // budget ran out; the budgets correspond to a second or more, far beyond any legitimate wait of
-// these kernels.
+// these kernels. A caller may pass a smaller budget (a diagnostic setting that makes the give-up
+// path reachable in a test).
 //
+// A try_wait may itself suspend the thread for a hardware-defined time, so a handful of such polls
+// is not a short wait. Budgets below kDiagPolls are therefore served by non-suspending test_wait
+// polls: that is how a test makes a wait run out quickly although the pipeline is healthy.
+constexpr uint32_t kDiagPolls = 1u << 10;
+__device__ __noinline__ bool mbar_wait_diag(uint32_t bar, uint32_t parity, uint32_t max_polls) {
+  for (uint32_t n = 0; n < max_polls; ++n) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    if (done) return true;
+  }
+  return false;
+}
+
 // mbar_wait_spin polls back to back: for the one thread whose reaction time is on the critical
 // path (the MMA issuer).
 constexpr uint32_t kMaxSpinPolls = 1u << 26;
-__device__ __forceinline__ bool mbar_wait_spin(uint32_t bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait_spin(uint32_t bar, uint32_t parity, uint32_t max_polls = kMaxSpinPolls) {
+  if (max_polls < kDiagPolls) return mbar_wait_diag(bar, parity, max_polls);
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t.reg .u32 n;\n\t"
@@ -63,7 +84,7 @@ __device__ __forceinline__ bool mbar_wait_spin(uint32_t bar, uint32_t parity) {
       "LKV_SPIN_DONE:\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
-      : "r"(bar), "r"(parity), "r"(kMaxSpinPolls)
+      : "r"(bar), "r"(parity), "r"(max_polls)
       : "memory");
   return ok != 0;
 }
@@ -72,7 +93,8 @@ __device__ __forceinline__ bool mbar_wait_spin(uint32_t bar, uint32_t parity) {
 // issue slots to the working ones.
 constexpr uint32_t kBackoffNs = 32;
 constexpr uint32_t kMaxPolls = 1u << 25;
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t max_polls = kMaxPolls) {
+  if (max_polls < kDiagPolls) return mbar_wait_diag(bar, parity, max_polls);
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t.reg .u32 n;\n\t"
@@ -88,7 +110,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
       "LKV_WAIT_DONE:\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
-      : "r"(bar), "r"(parity), "r"(kMaxPolls), "r"(kBackoffNs)
+      : "r"(bar), "r"(parity), "r"(max_polls), "r"(kBackoffNs)
       : "memory");
   return ok != 0;
 }

@@ -85,6 +85,7 @@ struct StreamArgs {
   int* fix_count;
   int fix_cap;
   int* status;
+  uint32_t polls, spin_polls;  // poll budgets of the hand-off waits: sleeping waits, back-to-back waits
 };
 
 __device__ __forceinline__ void record_status(int* status, int code) {
@@ -293,7 +294,7 @@ __device__ __forceinline__ bool lse_epilogue(const StreamArgs& a, const EpiCtx& 
     int nvalid = a.S - r.c.tib * kTileKeys - c0;       // key columns of this thread's range that hold a key
     for (int j = 0; j < r.ntiles; ++j, ++it, nvalid -= kTileKeys) {
       const uint32_t acc = it & 1;
-      if (!mbar_wait(e.bar_tfull + 8 * acc, (it >> 1) & 1)) return false;
+      if (!mbar_wait(e.bar_tfull + 8 * acc, (it >> 1) & 1, a.polls)) return false;
       tc_fence_after();
       uint32_t v[CW];
       load_epi_cols<CW>(t_col + acc * kAccStride, v);
@@ -315,11 +316,11 @@ __device__ __forceinline__ bool lse_epilogue(const StreamArgs& a, const EpiCtx& 
     }
     // end of this segment's run of tiles: merge the column groups, write one partial
     if (cg > 0) {
-      if (flushes > 0 && !mbar_wait(e.bar_xb, (uint32_t)(flushes - 1) & 1)) return false;
+      if (flushes > 0 && !mbar_wait(e.bar_xb, (uint32_t)(flushes - 1) & 1, a.polls)) return false;
       xch[(cg - 1) * nq + q] = make_float2(m, l);
       mbar_arrive(e.bar_xa);
     } else {
-      if (!mbar_wait(e.bar_xa, (uint32_t)flushes & 1)) return false;
+      if (!mbar_wait(e.bar_xa, (uint32_t)flushes & 1, a.polls)) return false;
       float mx = m;
 #pragma unroll
       for (int g2 = 1; g2 < ncg; ++g2) mx = fmaxf(mx, xch[(g2 - 1) * nq + q].x);
@@ -381,7 +382,7 @@ __device__ __forceinline__ bool score_epilogue(const StreamArgs& a, const EpiCtx
     int key = r.c.tib * kTileKeys + e.row;
     for (int j = 0; j < r.ntiles; ++j, ++it, key += kTileKeys) {
       const uint32_t acc = it & 1;
-      if (!mbar_wait(e.bar_tfull + 8 * acc, (it >> 1) & 1)) return false;
+      if (!mbar_wait(e.bar_tfull + 8 * acc, (it >> 1) & 1, a.polls)) return false;
       tc_fence_after();
       float sum = 0.f;
       if constexpr (NC > 0) {
@@ -396,11 +397,11 @@ __device__ __forceinline__ bool score_epilogue(const StreamArgs& a, const EpiCtx
       }
       // groups 1..3 hand their sums to group 0, which adds them in a fixed order
       if (e.wg > 0) {
-        if (it >= 2 && !mbar_wait(e.bar_xb + 8 * acc, ((it >> 1) - 1) & 1)) return false;
+        if (it >= 2 && !mbar_wait(e.bar_xb + 8 * acc, ((it >> 1) - 1) & 1, a.polls)) return false;
         part[(acc * 3 + (e.wg - 1)) * 128 + e.row] = sum;
         mbar_arrive(e.bar_xa + 8 * acc);
       } else {
-        if (!mbar_wait(e.bar_xa + 8 * acc, (it >> 1) & 1)) return false;
+        if (!mbar_wait(e.bar_xa + 8 * acc, (it >> 1) & 1, a.polls)) return false;
         const float tot = ((sum + part[(acc * 3 + 0) * 128 + e.row]) + part[(acc * 3 + 1) * 128 + e.row]) +
                           part[(acc * 3 + 2) * 128 + e.row];
         mbar_arrive(e.bar_xb + 8 * acc);
@@ -427,14 +428,14 @@ __device__ __forceinline__ bool proj_epilogue(const StreamArgs& a, const EpiCtx&
     const TileRun r = run_at(x, e.x_end, a);
     if (new_group) {
       // histogram slice landed (async-proxy writes are visible after the wait)
-      if (!mbar_wait(e.bar_stat, gen & 1)) return false;
+      if (!mbar_wait(e.bar_stat, gen & 1, a.polls)) return false;
       ++gen;
     }
     uint32_t* cnt = a.counts + (size_t)r.c.seg * a.S;
     const int table0 = r.c.chunk * TC;
     int key = r.c.tib * kTileKeys + e.row;
     for (int j = 0; j < r.ntiles; ++j, key += kTileKeys) {
-      if (!mbar_wait_spin(e.bar_tfull + 8 * acc, acc_phase)) return false;
+      if (!mbar_wait_spin(e.bar_tfull + 8 * acc, acc_phase, a.spin_polls)) return false;
       tc_fence_after();
       const bool valid = key < a.S;
       const uint32_t partial = proj_tables<KBITS, TQ>(e.t_lane + acc * STRIDE, e.bar_tempty + 8 * acc, e.hist_s, a,
@@ -531,7 +532,7 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
       for (long long x = x_begin; x < x_end; ++x, ++it) {
         if (new_group) {
           // stationary operand (+ histogram slice) of the new head / chunk
-          if (gen > 0) ok = mbar_wait(bar_stat_free, (uint32_t)(gen - 1) & 1);
+          if (gen > 0) ok = mbar_wait(bar_stat_free, (uint32_t)(gen - 1) & 1, a.polls);
           if (!ok) break;
           b = c.bh / a.H_kv;
           h = c.bh - b * a.H_kv;
@@ -550,7 +551,7 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
           ++gen;
         }
         const int s = (int)(it % kStages);
-        if (it >= kStages) ok = mbar_wait(bar_empty + 8 * s, (uint32_t)((it / kStages) - 1) & 1);
+        if (it >= kStages) ok = mbar_wait(bar_empty + 8 * s, (uint32_t)((it / kStages) - 1) & 1, a.polls);
         if (!ok) break;
         const uint32_t dst = sm_stages + s * kTileBytes;
         const int token = c.t * a.S + c.tib * kTileKeys;
@@ -562,7 +563,8 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
       }
       if (!ok) {
         record_status(a.status, kStatusTimeout);
-        // let copies already in flight land before the CTA may exit
+        // let copies already in flight land before the CTA may exit (full budget, whatever the
+        // hand-off budget is: shared memory must not be written after the CTA has gone)
         for (long long i = (it > kStages ? it - kStages : 0); i < it; ++i)
           mbar_wait(bar_full + 8 * (int)(i % kStages), (uint32_t)(i / kStages) & 1);
         if (gen > 0) mbar_wait(bar_stat, (uint32_t)(gen - 1) & 1);
@@ -584,19 +586,20 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
       const uint32_t stat_atom_lo = stat_atom_bytes >> 4;
       TileCursor c = cursor_at(x_begin, a);
       bool new_group = true, need_stat = false;
-      uint32_t gen = 0, it = 0;
+      uint32_t gen = 0, it = 0, last_use = 0;
+      int last_acc = -1;
       for (long long x = x_begin; x < x_end; ++x, ++it) {
         if (new_group) { ++gen; need_stat = true; }   // stationary operand number `gen` serves this tile
         if (it % kMmaWarps == mine) {
           if (need_stat) {
-            ok = mbar_wait_spin(bar_stat, (gen - 1) & 1);
+            ok = mbar_wait_spin(bar_stat, (gen - 1) & 1, a.spin_polls);
             if (!ok) break;
             need_stat = false;
           }
           const uint32_t s = it % kStages;
           const uint32_t acc = it % NACC, use = it / NACC;
-          if (use > 0) ok = mbar_wait_spin(bar_tempty + 8 * acc, (use - 1) & 1);
-          if (ok) ok = mbar_wait_spin(bar_full + 8 * s, (it / kStages) & 1);
+          if (use > 0) ok = mbar_wait_spin(bar_tempty + 8 * acc, (use - 1) & 1, a.spin_polls);
+          if (ok) ok = mbar_wait_spin(bar_full + 8 * s, (it / kStages) & 1, a.spin_polls);
           if (!ok) break;
           tc_fence_after();
           const uint32_t tile_lo = umma_sdesc_lo(sm_stages + s * kTileBytes);
@@ -618,11 +621,18 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
             umma_commit(bar_tfull + 8 * acc);   // accumulator ready for the epilogue
           }
           __syncwarp();
+          last_acc = (int)acc;
+          last_use = use;
         }
         new_group = cursor_last_of_group(c, a);
         cursor_advance(c, a);
       }
-      if (!ok && lane == 0) record_status(a.status, kStatusTimeout);
+      if (!ok) {
+        if (lane == 0) record_status(a.status, kStatusTimeout);
+        // the MMAs this warp issued last must have completed before the TMEM they write is freed
+        // (full budget; the completion of their commit is the accumulator-ready barrier's phase)
+        if (last_acc >= 0) mbar_wait(bar_tfull + 8 * last_acc, last_use & 1);
+      }
     }
     __syncwarp();
   } else if (x_begin < x_end) {

@@ -77,7 +77,13 @@ def test_null_and_misaligned_arguments_are_rejected():
     assert lib.laser_kv_init(C.byref(cfg), 0x1000, 0x1100, 16, 0x2000, 16, C.byref(h)) == B.ERR_CAPACITY
     assert lib.laser_kv_select_block(None, 0, None, None, None, None, None, 1, None) == B.ERR_INVALID_ARG
     assert lib.laser_kv_two_stage_topk(None, None, 1, 8, 1, 1, 1, None, None) == B.ERR_INVALID_ARG
-    assert lib.laser_kv_gather_append(None, None, 0, 0, None, 1, 1, None, None, 0, None, 0, 0, 0, None) == B.ERR_INVALID_ARG
+    assert lib.laser_kv_gather_append(None, None, 0, 0, 8, None, 1, 1, None, None, 0, 8, None, 0, 0, 0, None, None) == B.ERR_INVALID_ARG
+    # entries that do not fit the destination are refused before anything is launched
+    assert lib.laser_kv_gather_append(0x1000, 0x2000, 1024, 128, 8, 0x3000, 1, 5, 0x4000, 0x5000, 1024, 8, 0x6000, 8, 4, 0,
+                                      0x7000, None) == B.ERR_CAPACITY
+    assert lib.laser_kv_gather_append(0x1000, 0x2000, 1024, 128, -1, 0x3000, 1, 5, 0x4000, 0x5000, 1024, 8, 0x6000, 8, 0, 0,
+                                      0x7000, None) == B.ERR_INVALID_ARG
+    assert lib.laser_kv_set_wait_budget(None, 5) == B.ERR_INVALID_ARG
     assert b"NULL" in lib.laser_kv_last_error(None)
     # the entry points beside the hot path validate before they touch the device
     assert lib.laser_kv_decode_attention(None, 0, None, None, 0.0, None, None, 0, None) == B.ERR_INVALID_ARG

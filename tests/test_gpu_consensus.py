@@ -70,11 +70,13 @@ def test_consensus_pipeline_against_oracle(name, S, nb, n_layers):
     Kd = torch.zeros((w.n_kv_heads, nb * B, 128), dtype=torch.int16, device="cuda")
     Vd = torch.zeros_like(Kd)
     pos = torch.full((w.n_kv_heads, nb * B), -1, dtype=torch.int32, device="cuda")
+    bad = torch.zeros(w.n_kv_heads, dtype=torch.int32, device="cuda")
     for h in range(w.n_kv_heads):
         # segments = the blocks of head h: sources S rows apart, destinations B rows apart
         Bn.laser_kv_gather_append(tK[h].view(nb, S, 128), tV[h].view(nb, S, 128), idx, Kd[h].view(nb, B, 128),
-                                  Vd[h].view(nb, B, 128), pos[h].view(nb, B), 0, 0)
+                                  Vd[h].view(nb, B, 128), pos[h].view(nb, B), 0, 0, bad[h:h + 1])
     torch.cuda.synchronize()
+    assert int(bad.abs().sum()) == 0
     Kd, Vd, pos = to_np(Kd).view(np.uint16), to_np(Vd).view(np.uint16), to_np(pos)
     for h in range(w.n_kv_heads):
         for t in range(nb):

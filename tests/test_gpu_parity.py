@@ -201,14 +201,32 @@ def test_gather_append_entry_point_bit_exact():
     Kd = torch.zeros((n_seg, cap, 128), dtype=torch.int16, device="cuda")
     Vd = torch.zeros_like(Kd)
     pos = torch.full((n_seg, cap), -1, dtype=torch.int32, device="cuda")
-    Bn.laser_kv_gather_append(torch.from_numpy(K.view(np.int16)).cuda(), torch.from_numpy(V.view(np.int16)).cuda(),
-                              torch.from_numpy(idx).cuda(), Kd, Vd, pos, 200, 5000)
+    tK, tV = torch.from_numpy(K.view(np.int16)).cuda(), torch.from_numpy(V.view(np.int16)).cuda()
+    status = torch.full((1,), 77, dtype=torch.int32, device="cuda")
+    Bn.laser_kv_gather_append(tK, tV, torch.from_numpy(idx).cuda(), Kd, Vd, pos, 200, 5000, status)
     torch.cuda.synchronize()
-    Kd, Vd, pos = to_np(Kd).view(np.uint16), to_np(Vd).view(np.uint16), to_np(pos)
+    assert int(status[0]) == 0
+    Kn, Vn, pn = to_np(Kd).view(np.uint16), to_np(Vd).view(np.uint16), to_np(pos)
     for g in range(n_seg):
-        assert (Kd[g, 200:200 + keep] == K[g, idx[g]]).all() and (Vd[g, 200:200 + keep] == V[g, idx[g]]).all()
-        assert (pos[g, 200:200 + keep] == 5000 + idx[g]).all()
-        assert (Kd[g, :200] == 0).all() and (Kd[g, 200 + keep:] == 0).all() and (pos[g, :200] == -1).all()
+        assert (Kn[g, 200:200 + keep] == K[g, idx[g]]).all() and (Vn[g, 200:200 + keep] == V[g, idx[g]]).all()
+        assert (pn[g, 200:200 + keep] == 5000 + idx[g]).all()
+        assert (Kn[g, :200] == 0).all() and (Kn[g, 200 + keep:] == 0).all() and (pn[g, :200] == -1).all()
+    # indices outside the source segment are never dereferenced: their entries are skipped and the
+    # status word says so; every valid entry is still copied
+    bad = idx.copy()
+    bad[1, 7], bad[2, 100], bad[0, keep - 1] = rows, -1, 2 ** 30
+    Kd.zero_(); Vd.zero_(); pos.fill_(-1)
+    Bn.laser_kv_gather_append(tK, tV, torch.from_numpy(bad).cuda(), Kd, Vd, pos, 200, 5000, status)
+    torch.cuda.synchronize()
+    assert int(status[0]) == Bn.ERR_INVALID_ARG
+    Kn, pn = to_np(Kd).view(np.uint16), to_np(pos)
+    for g in range(n_seg):
+        ok = (bad[g] >= 0) & (bad[g] < rows)
+        assert (Kn[g, 200:200 + keep][ok] == K[g, bad[g][ok]]).all() and (pn[g, 200:200 + keep][ok] == 5000 + bad[g][ok]).all()
+        assert (Kn[g, 200:200 + keep][~ok] == 0).all() and (pn[g, 200:200 + keep][~ok] == -1).all()
+    with pytest.raises(Bn.LaserKVError) as e:      # entries beyond the destination's capacity
+        Bn.laser_kv_gather_append(tK, tV, torch.from_numpy(idx).cuda(), Kd, Vd, pos, cap - keep + 1, 0, status)
+    assert e.value.status == Bn.ERR_CAPACITY
 
 
 def test_headline_config_full_size_sampled_segments():

@@ -5,13 +5,15 @@ an engine whose pool owns the GPU, a latency-critical loop that cannot afford cu
 synchronisation): its scratch is a 2 MiB array inside the library. It runs the same two
 kernels as laser_kv_window_scores, so on the same inputs the two must agree within the score
 tolerance of the parity tests. The test makes two calls in a row with different shapes, so the
-second call starts from the first call's leftovers in the shared array, and checks that sizes
-beyond the array are refused. This file sorts last on purpose: a run that stops at the first
+second call starts from the first call's leftovers in the shared array, reads the status word
+that these calls keep inside the library, compares sampled heads with the fp64 oracle, and checks
+that sizes beyond the array are refused. This file sorts last on purpose: a run that stops at the first
 failure has then already run every other test.
 """
 import numpy as np
 import pytest
 
+from oracle import laser_kv_oracle as O
 from paper_2602_02199_b200 import synth
 
 pytestmark = pytest.mark.gpu
@@ -24,7 +26,7 @@ def _inputs(name, S, nb, first_block):
     w = synth.workload(name).with_(block_size=S, context_len=16 * S, batch=1)
     K, _ = synth.kv_blocks(w, 0, 0, first_block, nb)
     Q = synth.q_window(w, 0, 0)
-    return (torch.from_numpy(K.view(np.int16)).cuda()[None], torch.from_numpy(Q.view(np.int16)).cuda()[None])
+    return (torch.from_numpy(K.view(np.int16)).cuda()[None], torch.from_numpy(Q.view(np.int16)).cuda()[None], K, Q)
 
 
 def test_static_scratch_variant_matches_caller_scratch_variant_twice_in_a_row():
@@ -35,7 +37,7 @@ def test_static_scratch_variant_matches_caller_scratch_variant_twice_in_a_row():
     # second call: 4 KV heads x 3 ragged blocks of 1000 keys, 224 queries per head. The shapes differ so
     # that partials left in the shared array by the first call would show up in the second.
     for name, S, nb, first in (("llama8b_128k", 4096, 5, 0), ("qwen7b_128k", 1000, 3, 4)):
-        tK, tQ = _inputs(name, S, nb, first)
+        tK, tQ, K, Q = _inputs(name, S, nb, first)
         want = Bn.laser_kv_window_scores(tK, tQ, S, nb)
         out = torch.full((1, tK.shape[1], nb, S), float("nan"), dtype=torch.float32, device="cuda")
         torch.cuda.synchronize()
@@ -48,6 +50,14 @@ def test_static_scratch_variant_matches_caller_scratch_variant_twice_in_a_row():
         assert (np.abs(got - ref) <= RTOL * np.abs(ref) + ATOL).all()
         # each query's probabilities sum to one: the block total is the number of window queries
         np.testing.assert_allclose(got.sum(axis=3), tQ.shape[1] // tK.shape[1] * tQ.shape[2], rtol=2e-3)
+        # no kernel of the call gave up a wait (the word sits in the library's array; this reads it)
+        Bn.laser_kv_window_scores_static_status()
+        assert torch.cuda.memory_allocated() == before
+        # and against the oracle itself, for the first and the last head of the last block
+        n_kv = tK.shape[1]
+        for h in (0, n_kv - 1):
+            ref64 = O.window_scores(O.group_queries(Q, n_kv, h), K[h, (nb - 1) * S:nb * S])
+            assert (np.abs(got[0, h, nb - 1] - ref64) <= RTOL * np.abs(ref64) + ATOL).all()
 
 
 def test_static_scratch_variant_rejects_sizes_beyond_its_array():
