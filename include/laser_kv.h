@@ -68,6 +68,9 @@ typedef struct {
   double  alpha;               /* exact share of the recall budget; negative => 0.75             */
   float   softmax_scale;       /* 0 => 1/sqrt(head_dim)                                          */
   int32_t device;              /* CUDA device ordinal                                            */
+  int32_t lookback;            /* 0: every block keeps its own local window (Section 3.1 alone);
+                                  1: look-back boundary smoothing (Section 3.2), see
+                                  laser_kv_select_block                                           */
 } laser_kv_config_t;
 
 /* Views returned by laser_kv_cache_view: entries [0, len) of every (sequence, KV head) are
@@ -96,6 +99,10 @@ typedef struct {
   const int32_t*  idx;           /* dev int32 [batch][H_kv][nb][B]   kept block-local indices    */
   int32_t n_blocks, batch, n_kv_heads, block_size, budget, gw, lsh_tables, lsh_bits;
   int32_t n_sign_fixups;         /* host: near-zero projections recomputed exactly (last poll)   */
+  int32_t segment_keys;          /* scored keys per segment: the "S" of the arrays above; block_size,
+                                    or block_size + floor(B/n) for the later blocks under look-back */
+  int32_t segment_shift;         /* scored key 0 is this many tokens before the block's first token
+                                    (0, or floor(B/n) for the later blocks under look-back)        */
 } laser_kv_debug_t;
 
 /* Appendix B, Eq. 1: B = floor(2 r S_block L / (S_block + L)) evaluated in IEEE double.
@@ -134,6 +141,23 @@ laser_kv_status_t laser_kv_init(const laser_kv_config_t* cfg, const void* hyperp
  * candidates with the most SimHash collisions (ties: lower index). Rows are appended in
  * ascending position at [len, len + n_blocks*B); len advances on the host. The blocks' absolute
  * positions continue from the blocks already appended to this layer.
+ * With config.lookback = 1 (Section 3.2: the scoring window of block t is expanded to include the
+ * tail of block t-1, so that tokens at a block's edge are judged with the context that follows them)
+ * the local window slides instead of being kept block by block. With a = floor(B/n):
+ *   - the first block of a sequence keeps its a anchors and Algorithm 1's picks from [a, S - a) with
+ *     the recall budget B - 2a; its last a tokens are held back (B - a entries appended);
+ *   - every later block scores the held-back a tokens of the previous block together with its own S
+ *     keys (one softmax over a + S keys, one collision count each), keeps its a anchors, and runs
+ *     Algorithm 1 on the held-back tokens plus [a, S - a) of the block with recall budget B - a
+ *     (k_exact = floor(alpha * (B - a))); its own last a tokens are held back in turn (B entries
+ *     appended, ascending positions);
+ *   - laser_kv_lookback_close appends the tail of the last block. The cache then holds B entries per
+ *     block, as without look-back.
+ * The held-back tokens are not stored by the library: for every block but the first of the sequence
+ * the a rows before K_blk / V_blk (same strides) must be the previous block's last a tokens, i.e. the
+ * pointers must point into a buffer that holds the context contiguously. laser_kv_select_block_host
+ * does not support look-back. laser_kv_debug_view then describes the last pass only (the first block
+ * of a sequence is a pass of its own).
  * A handle's workspace serves one call at a time: calls on the same handle must be issued to one
  * stream (or be ordered by the caller); concurrent streams need one handle each.
  * Errors: CAPACITY if the cache cannot take n_blocks more blocks or n_blocks exceeds
@@ -142,6 +166,14 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
                                         const void* V_blk, const void* Q_win,
                                         const int64_t kv_strides[3], const int64_t q_strides[3],
                                         int32_t n_blocks, void* stream);
+
+/* Closes a look-back sequence (config.lookback = 1): appends the a = floor(B/n) tokens that the last
+ * block held back - nothing follows them, so nothing can prune them. K_tail / V_tail: dev bf16
+ * [batch][H_kv][a][d] through kv_strides, the last a rows of the last block (K_blk + (S - a) rows of
+ * that block, same strides). Afterwards the layer accepts no block until laser_kv_reset. STATE if the
+ * handle has no look-back, the layer holds no block or is closed already. */
+laser_kv_status_t laser_kv_lookback_close(laser_kv_handle_t h, int32_t layer, const void* K_tail,
+                                          const void* V_tail, const int64_t kv_strides[3], void* stream);
 
 /* Same path driven from HOST memory: copies the (contiguous) host tensors K_host, V_host
  * [batch][H_kv][n_blocks*S][d] and Q_host [batch][H_q][W][d] into the caller's device staging

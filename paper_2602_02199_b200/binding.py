@@ -21,6 +21,7 @@ EXPORTS = [
     "laser_kv_collision_counts", "laser_kv_collision_counts_scratch_bytes", "laser_kv_consensus_accumulate",
     "laser_kv_decode_attention", "laser_kv_decode_attention_scratch_bytes", "laser_kv_collision_probability",
     "laser_kv_set_layer_budget", "laser_kv_set_wait_budget", "laser_kv_window_scores_static_status",
+    "laser_kv_lookback_close",
 ]
 
 
@@ -32,7 +33,7 @@ class Config(C.Structure):
         ("lsh_bits", C.c_int32), ("lsh_tables", C.c_int32), ("protection_divisor", C.c_int32),
         ("budget_per_block", C.c_int32), ("debug", C.c_int32), ("context_len", C.c_int64),
         ("ratio", C.c_double), ("alpha", C.c_double), ("softmax_scale", C.c_float),
-        ("device", C.c_int32),
+        ("device", C.c_int32), ("lookback", C.c_int32),
     ]
 
 
@@ -47,7 +48,7 @@ class Debug(C.Structure):
                 ("idx", C.c_void_p), ("n_blocks", C.c_int32), ("batch", C.c_int32),
                 ("n_kv_heads", C.c_int32), ("block_size", C.c_int32), ("budget", C.c_int32),
                 ("gw", C.c_int32), ("lsh_tables", C.c_int32), ("lsh_bits", C.c_int32),
-                ("n_sign_fixups", C.c_int32)]
+                ("n_sign_fixups", C.c_int32), ("segment_keys", C.c_int32), ("segment_shift", C.c_int32)]
 
 
 class LaserKVError(RuntimeError):
@@ -107,6 +108,8 @@ def load(build_if_missing: bool = True) -> C.CDLL:
     lib.laser_kv_two_stage_topk.argtypes = [vp, vp, i32, i32, i32, i32, i32, vp, vp]
     lib.laser_kv_gather_append.restype = i32
     lib.laser_kv_gather_append.argtypes = [vp, vp, i64, i64, i32, vp, i32, i32, vp, vp, i64, i64, vp, i64, i64, i32, vp, vp]
+    lib.laser_kv_lookback_close.restype = i32
+    lib.laser_kv_lookback_close.argtypes = [vp, i32, vp, vp, p(i64), vp]
     lib.laser_kv_set_wait_budget.restype = i32
     lib.laser_kv_set_wait_budget.argtypes = [vp, C.c_uint32]
     lib.laser_kv_window_scores_static_status.restype = i32
@@ -174,10 +177,10 @@ def laser_kv_launch_count() -> int:
 def make_config(*, n_layers, batch, n_q_heads, n_kv_heads, block_size, window, max_blocks,
                 max_blocks_per_call, lsh_bits, lsh_tables, protection_divisor, budget_per_block=0,
                 context_len=0, ratio=0.25, alpha=0.75, softmax_scale=0.0, debug=0, device=0,
-                head_dim=128) -> Config:
+                head_dim=128, lookback=0) -> Config:
     return Config(n_layers, batch, n_q_heads, n_kv_heads, head_dim, block_size, window, max_blocks,
                   max_blocks_per_call, lsh_bits, lsh_tables, protection_divisor, budget_per_block,
-                  debug, context_len, ratio, alpha, softmax_scale, device)
+                  debug, context_len, ratio, alpha, softmax_scale, device, lookback)
 
 
 def _ptr(t) -> int:
@@ -201,6 +204,8 @@ class DebugTensors:
     hist: object
     idx: object
     n_sign_fixups: int
+    segment_keys: int = 0
+    segment_shift: int = 0
 
 
 class LaserKV:
@@ -260,6 +265,13 @@ class LaserKV:
                                                    _ptr(Q_stage), n_blocks, _ptr(pos_out_host),
                                                    _stream_ptr(stream)), self.handle)
 
+    def laser_kv_lookback_close(self, layer, K_tail, V_tail, stream=None):
+        """K_tail, V_tail: [batch][H_kv][a][d] views of the last block's last a = floor(B/n) rows."""
+        ks = (C.c_int64 * 3)(*K_tail.stride()[:3])
+        assert tuple(V_tail.stride()) == tuple(K_tail.stride())
+        _check(self.lib.laser_kv_lookback_close(self.handle, layer, _ptr(K_tail), _ptr(V_tail), ks,
+                                                _stream_ptr(stream)), self.handle)
+
     def laser_kv_cache_view(self, layer):
         """Returns (K, V, pos, len) as torch views [batch][H_kv][cap][d] / [batch][H_kv][cap]."""
         torch = self._torch
@@ -279,7 +291,7 @@ class LaserKV:
         _check(self.lib.laser_kv_debug_view(self.handle, C.byref(d)), self.handle)
         base = self.workspace.data_ptr()
         nseg = d.batch * d.n_kv_heads * d.n_blocks
-        S, L = d.block_size, d.lsh_tables
+        S, L = d.segment_keys, d.lsh_tables
 
         def view(ptr, nbytes, dtype, shape):
             if not ptr:
@@ -297,7 +309,7 @@ class LaserKV:
             hist=view(d.hist, d.batch * d.n_kv_heads * L * (2 << d.lsh_bits), torch.int16,
                       (d.batch, d.n_kv_heads, L, 1 << d.lsh_bits)),
             idx=view(d.idx, nseg * max(d.budget, 1) * 4, torch.int32, shp + (max(d.budget, 1),)),
-            n_sign_fixups=int(d.n_sign_fixups))
+            n_sign_fixups=int(d.n_sign_fixups), segment_keys=int(d.segment_keys), segment_shift=int(d.segment_shift))
 
     def laser_kv_decode_attention(self, layer, Q_dec, softmax_scale=0.0, out=None, stream=None):
         """Q_dec: [batch][H_q][d] 2-byte tensor (contiguous last dim) -> fp32 [batch][H_q][d]."""

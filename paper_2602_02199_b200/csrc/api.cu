@@ -48,6 +48,7 @@ struct Derived {
   double alpha, ratio;
   float scale;
   int fix_cap;
+  int S_ws;            // largest number of scored keys per segment (sizes the workspace)
   long long cap;       // cache entries per (sequence, KV head)
   int nseg_max;
 };
@@ -73,13 +74,16 @@ struct laser_kv_ctx {
   CUtensorMap mapPq;   // hyperplanes, box = the eight tables of one query-signature CTA
   EncodeTiledFn encode = nullptr;
   int num_sms = 1;
-  std::vector<long long> blocks_done;   // per layer
+  std::vector<long long> blocks_done;   // per layer: blocks processed
+  std::vector<long long> entries_done;  // per layer: cache entries final per (sequence, KV head)
+  std::vector<char> lookback_closed;    // per layer: the held-back tail of the last block was appended
   struct LayerBudget { int B, anchors, k_exact, k_lsh; };
   std::vector<LayerBudget> budget;      // per layer; the configured budget unless laser_kv_set_layer_budget changed it
   int last_B = 0;                       // budget of the last select call (debug view)
   std::string last_error;
   bool have_call = false;
   int last_nb = 0;
+  int last_S_len = 0, last_shift = 0;   // scored keys per segment of the last pass, rows of them before the block
   int last_fixups = 0;
   // host-buffer path: copies run on a stream of their own, chunk by chunk
   cudaStream_t copy_stream = nullptr;
@@ -203,7 +207,11 @@ laser_kv_status_t derive(const laser_kv_config_t* c, Derived* d) {
   const long long nseg = (long long)c->batch * c->n_kv_heads * c->max_blocks_per_call;
   if (nseg > (1 << 22)) return fail(nullptr, LASER_KV_ERR_UNSUPPORTED, "config: too many segments per call");
   d->nseg_max = (int)nseg;
-  long long fc = nseg * c->block_size * (long long)c->lsh_tables / 256;
+  if (c->lookback != 0 && c->lookback != 1)
+    return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "config: lookback must be 0 or 1");
+  // with look-back a segment is the previous block's held-back tail followed by the block
+  d->S_ws = c->block_size + (c->lookback ? d->anchors : 0);
+  long long fc = nseg * d->S_ws * (long long)c->lsh_tables / 256;
   if (fc < 4096) fc = 4096;
   if (fc > (1 << 26)) fc = 1 << 26;
   d->fix_cap = (int)fc;
@@ -213,7 +221,7 @@ laser_kv_status_t derive(const laser_kv_config_t* c, Derived* d) {
 void carve_ws(const laser_kv_config_t* c, const Derived& d, Carve* v) {
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
-  const size_t nseg = d.nseg_max, S = c->block_size;
+  const size_t nseg = d.nseg_max, S = d.S_ws;
   const size_t bh = (size_t)c->batch * c->n_kv_heads;
   v->ctrl = take(256);
   v->dec_count = take(bh * 4);        // finished decode splits per (sequence, KV head)
@@ -222,7 +230,7 @@ void carve_ws(const laser_kv_config_t* c, const Derived& d, Carve* v) {
   v->lse_part = take(lse_part_bytes_bound(nseg, d.GW));
   v->lse2 = take(nseg * d.GW * 4);
   v->s_exact = take(nseg * S * 4);
-  v->counts = take(nseg * S * 4);
+  v->counts = take(nseg * S * 4 + 16);     // cleared in 16-byte units
   v->idx = take(nseg * (size_t)(d.B > 0 ? d.B : 1) * 4);
   v->fix_items = take((size_t)d.fix_cap * sizeof(int4));
   v->key_buckets = take(c->debug ? nseg * S * c->lsh_tables * 2 : 0);
@@ -314,10 +322,9 @@ cudaError_t launch_qsig(int K, const CUtensorMap& mq, const CUtensorMap& mp, con
 
 // `count_max` bounds every count (0 = no bound known): it lets the count stage skip radix passes
 // over bytes that are zero everywhere.
-laser_kv_status_t launch_select(const float* s_exact, const uint32_t* counts, int n_seg, int S, int anchors,
-                                int k_exact, int k_lsh, uint32_t count_max, int32_t* idx, cudaStream_t st) {
+laser_kv_status_t launch_select(SelectArgs a, int n_seg, uint32_t count_max, cudaStream_t st) {
   static std::atomic<unsigned long long> limit_set{0};
-  const size_t smem = (size_t)S * 9;
+  const size_t smem = (size_t)a.S * 9;
   if (ensure_smem_limit(limit_set, select_kernel, kMaxSmem - 2048) != cudaSuccess)
     return fail(nullptr, LASER_KV_ERR_CUDA, "cudaFuncSetAttribute(select_kernel) failed");
   int top_shift = 24;
@@ -325,7 +332,7 @@ laser_kv_status_t launch_select(const float* s_exact, const uint32_t* counts, in
     top_shift = 0;
     while (top_shift < 24 && (count_max >> (top_shift + 8)) != 0) top_shift += 8;
   }
-  SelectArgs a{s_exact, counts, idx, S, anchors, k_exact, k_lsh, top_shift};
+  a.count_top_shift = top_shift;
   select_kernel<<<n_seg, kSelThreads, smem, st>>>(a);
   g_launches.fetch_add(1);
   const cudaError_t e = cudaGetLastError();
@@ -453,6 +460,8 @@ laser_kv_status_t laser_kv_init(const laser_kv_config_t* cfg, const void* hyperp
   h->cachePos = reinterpret_cast<int32_t*>(cm + 2 * align_up(per * kHeadDim * 2));
   h->P = static_cast<const uint16_t*>(hyperplanes);
   h->blocks_done.assign(cfg->n_layers, 0);
+  h->entries_done.assign(cfg->n_layers, 0);
+  h->lookback_closed.assign(cfg->n_layers, 0);
   h->budget.assign(cfg->n_layers, laser_kv_ctx::LayerBudget{d.B, d.anchors, d.k_exact, d.k_lsh});
   h->last_B = d.B;
   {
@@ -474,36 +483,75 @@ laser_kv_status_t laser_kv_init(const laser_kv_config_t* cfg, const void* hyperp
   return LASER_KV_OK;
 }
 
-laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, const void* K_blk, const void* V_blk,
-                                        const void* Q_win, const int64_t kv_strides[3], const int64_t q_strides[3],
-                                        int32_t n_blocks, void* stream) {
-  if (!h) return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "select_block: NULL handle");
-  if (const laser_kv_status_t ds = check_device(h, "select_block")) return ds;
+}  // extern "C"
+
+namespace {
+
+// Geometry of one group of launches of the select path: which keys a segment scores and what
+// becomes of them (Section 3.1's partition; Section 3.2's look-back shifts it by one local window).
+struct CallGeom {
+  int S_len;                 // scored keys per segment
+  int shift;                 // rows before the block's first token that belong to the segment (0 or anchors)
+  int keep_a_lo, keep_a_hi, keep_b_lo, keep_b_hi, excl_lo, excl_hi, cand_lo, cand_hi;   // scored-key index ranges
+  int k_exact, k_lsh;
+  int B_out;                 // cache entries per block and head
+};
+
+// The plain rule: anchors and local window kept, Algorithm 1 on what lies between.
+CallGeom plain_geom(int S, const laser_kv_ctx::LayerBudget& lb) {
+  CallGeom g;
+  g.S_len = S; g.shift = 0;
+  g.keep_a_lo = 0; g.keep_a_hi = lb.anchors; g.keep_b_lo = S - lb.anchors; g.keep_b_hi = S;
+  g.excl_lo = g.excl_hi = 0;
+  g.cand_lo = lb.anchors; g.cand_hi = S - lb.anchors;
+  g.k_exact = lb.k_exact; g.k_lsh = lb.k_lsh;
+  g.B_out = lb.B;
+  return g;
+}
+
+// Look-back (Section 3.2): a block's local window [S - a, S) is held back and scored again with the
+// next block. First block of a sequence: anchors + Algorithm 1 on [a, S - a) with the plain recall
+// budget. Later blocks: the segment is the previous block's tail followed by the block; the block's
+// anchors are kept, the tail of the previous block and the block's middle are the candidates with
+// recall budget B - a, the block's own tail is held back.
+CallGeom lookback_geom(int S, const laser_kv_ctx::LayerBudget& lb, double alpha, bool first) {
+  const int a = lb.anchors;
+  CallGeom g;
+  g.keep_b_lo = g.keep_b_hi = 0;
+  if (first) {
+    g.S_len = S; g.shift = 0;
+    g.keep_a_lo = 0; g.keep_a_hi = a;
+    g.excl_lo = S - a; g.excl_hi = S;
+    g.cand_lo = a; g.cand_hi = S - a;
+    g.k_exact = lb.k_exact; g.k_lsh = lb.k_lsh;
+    g.B_out = lb.B - a;
+  } else {
+    g.S_len = S + a; g.shift = a;
+    g.keep_a_lo = a; g.keep_a_hi = 2 * a;
+    g.excl_lo = S; g.excl_hi = S + a;
+    g.cand_lo = 0; g.cand_hi = S;
+    const int b_long = lb.B - a;
+    int ke = (int)std::floor(alpha * (double)b_long);
+    if (ke < 0) ke = 0;
+    if (ke > b_long) ke = b_long;
+    g.k_exact = ke; g.k_lsh = b_long - ke;
+    g.B_out = lb.B;
+  }
+  return g;
+}
+
+// One pass of the path over nb consecutive blocks with the same geometry. K_blk / V_blk point at
+// the first token of the first block; with g.shift > 0 the g.shift rows before it (the tail of the
+// previous block) are read as well. `first_block` is the index of the first block in the sequence,
+// `entries_done` the cache entries already final per head.
+laser_kv_status_t run_select(laser_kv_ctx* h, int layer, const void* K_blk, const void* V_blk, const void* Q_win,
+                             const int64_t kv_strides[3], const int64_t q_strides[3], int nb, const CallGeom& g,
+                             long long first_block, long long entries_done, cudaStream_t st) {
   const laser_kv_config_t& c = h->cfg;
   const Derived& d = h->d;
-  if (layer < 0 || layer >= c.n_layers) return fail(h, LASER_KV_ERR_INVALID_ARG, "select_block: layer %d out of range", layer);
-  if (!K_blk || !V_blk || !Q_win || !kv_strides || !q_strides)
-    return fail(h, LASER_KV_ERR_INVALID_ARG, "select_block: NULL argument");
-  if (n_blocks < 1) return fail(h, LASER_KV_ERR_INVALID_ARG, "select_block: n_blocks must be >= 1");
-  if (n_blocks > c.max_blocks_per_call)
-    return fail(h, LASER_KV_ERR_CAPACITY, "select_block: n_blocks %d exceeds max_blocks_per_call %d", n_blocks, c.max_blocks_per_call);
-  if (h->blocks_done[layer] + n_blocks > c.max_blocks)
-    return fail(h, LASER_KV_ERR_CAPACITY, "select_block: layer %d cache holds %lld of %d blocks; cannot append %d",
-                layer, h->blocks_done[layer], c.max_blocks, n_blocks);
-  if (!aligned16(K_blk) || !aligned16(V_blk) || !aligned16(Q_win))
-    return fail(h, LASER_KV_ERR_ALIGNMENT, "select_block: device pointers must be 16-byte aligned");
-  for (int i = 0; i < 3; ++i)
-    if (kv_strides[i] < 0 || q_strides[i] < 0 || (kv_strides[i] % 8) || (q_strides[i] % 8))
-      return fail(h, LASER_KV_ERR_ALIGNMENT, "select_block: strides must be non-negative multiples of 8 elements");
-  if (kv_strides[2] < kHeadDim || q_strides[2] < kHeadDim)
-    return fail(h, LASER_KV_ERR_INVALID_ARG, "select_block: row stride smaller than head_dim");
-  if ((long long)(h->blocks_done[layer] + n_blocks) * c.block_size > 0x7fffffffLL)
-    return fail(h, LASER_KV_ERR_UNSUPPORTED, "select_block: absolute positions exceed int32");
-
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const laser_kv_ctx::LayerBudget lb = h->budget[layer];
-  const int S = c.block_size, nb = n_blocks, B = lb.B;
+  const int S = c.block_size, S_len = g.S_len, B = g.B_out;
   const int nseg = c.batch * c.n_kv_heads * nb;
+  const int tiles_in_block = (S_len + kTileKeys - 1) / kTileKeys;
   uint8_t* ws = h->ws;
   int* ctrl = reinterpret_cast<int*>(ws + h->carve.ctrl);
   uint16_t* hist = reinterpret_cast<uint16_t*>(ws + h->carve.hist);
@@ -515,20 +563,24 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
   int32_t* idx = reinterpret_cast<int32_t*>(ws + h->carve.idx);
   int4* fix_items = reinterpret_cast<int4*>(ws + h->carve.fix_items);
   uint16_t* key_buckets = c.debug ? reinterpret_cast<uint16_t*>(ws + h->carve.key_buckets) : nullptr;
+  // the segment's first key: g.shift rows before the block
+  const uint16_t* K0 = static_cast<const uint16_t*>(K_blk) - (long long)g.shift * kv_strides[2];
+  const uint16_t* V0 = static_cast<const uint16_t*>(V_blk) - (long long)g.shift * kv_strides[2];
 
   // TMA descriptors for this call's K and Q_win
   CUtensorMap mapK, mapQ;
   {
-    const uint64_t dims[4] = {(uint64_t)kHeadDim, (uint64_t)nb * S, (uint64_t)c.n_kv_heads, (uint64_t)c.batch};
+    const uint64_t tokens = (uint64_t)nb * S + g.shift;
+    const uint64_t dims[4] = {(uint64_t)kHeadDim, tokens, (uint64_t)c.n_kv_heads, (uint64_t)c.batch};
     // a dimension of extent 1 never advances; give it a dense stride if the caller passed 0
     const uint64_t s_tok = (uint64_t)kv_strides[2];
-    const uint64_t s_head = kv_strides[1] > 0 ? (uint64_t)kv_strides[1] : s_tok * (uint64_t)nb * S;
+    const uint64_t s_head = kv_strides[1] > 0 ? (uint64_t)kv_strides[1] : s_tok * tokens;
     const uint64_t s_batch = kv_strides[0] > 0 ? (uint64_t)kv_strides[0] : s_head * (uint64_t)c.n_kv_heads;
     if ((c.n_kv_heads > 1 && kv_strides[1] == 0) || (c.batch > 1 && kv_strides[0] == 0))
       return fail(h, LASER_KV_ERR_INVALID_ARG, "select_block: zero stride on a dimension of extent > 1");
     const uint64_t strides[3] = {s_tok * 2, s_head * 2, s_batch * 2};
     const uint32_t box[4] = {(uint32_t)kAtomCols, (uint32_t)kTileKeys, 1, 1};
-    if (!encode_map(h, &mapK, K_blk, 4, dims, strides, box)) return LASER_KV_ERR_CUDA;
+    if (!encode_map(h, &mapK, K0, 4, dims, strides, box)) return LASER_KV_ERR_CUDA;
   }
   {
     const uint64_t dims[4] = {(uint64_t)kHeadDim, (uint64_t)c.window, (uint64_t)c.n_q_heads, (uint64_t)c.batch};
@@ -555,30 +607,29 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
     cudaEventRecord(ev, st);
     marks.push_back(ev);
   };
-  // rows that are kept whatever the scores say travel on the side stream from now on
   mark();
   // A stage whose share of the recall budget is empty (alpha = 1: no LSH picks; alpha = 0 or n = 2:
   // no exact picks) is not computed, unless the debug view was asked for, which shows every
   // intermediate result.
-  const bool need_lsh = lb.k_lsh > 0 || c.debug;
-  const bool need_exact = lb.k_exact > 0 || c.debug;
+  const bool need_lsh = g.k_lsh > 0 || c.debug;
+  const bool need_exact = g.k_exact > 0 || c.debug;
   // 1. query signatures and bucket histograms; the kernel also clears the counts and restarts the
   //    fix-up counter (ctrl[1]) and the changed counter (ctrl[2]); the status word (ctrl[0]) is kept
   if (need_lsh) {
     const int q_alloc = ((d.GW + 127) / 128) * 128;
     QsigArgs qa{static_cast<const uint16_t*>(Q_win), q_strides[0], q_strides[1], q_strides[2], h->P, hist, qb,
                 c.n_kv_heads, d.G, c.window, d.GW, q_alloc, c.lsh_tables,
-                reinterpret_cast<uint4*>(counts), (long long)nseg * S / 4, ctrl + 1, ctrl};
+                reinterpret_cast<uint4*>(counts), ((long long)nseg * S_len + 3) / 4, ctrl + 1, ctrl};
     dim3 grid(c.lsh_tables / kQsigTables, c.n_kv_heads, c.batch);
     LKV_CUDA(launch_qsig(c.lsh_bits, mapQ, h->mapPq, qa, grid, qsig_smem_bytes(q_alloc, c.lsh_bits), st), "qsig_kernel");
   }
 
   StreamArgs sa;
   memset(&sa, 0, sizeof sa);
-  sa.S = S; sa.nb = nb; sa.H_kv = c.n_kv_heads; sa.batch = c.batch;
+  sa.S = S_len; sa.S_stride = S; sa.nb = nb; sa.H_kv = c.n_kv_heads; sa.batch = c.batch;
   sa.G = d.G; sa.W = c.window; sa.GW = d.GW;
-  sa.tiles_in_block = d.tiles_in_block; sa.nseg = nseg;
-  const long long seg_tiles = (long long)nseg * d.tiles_in_block;
+  sa.tiles_in_block = tiles_in_block; sa.nseg = nseg;
+  const long long seg_tiles = (long long)nseg * tiles_in_block;
   const int base_ctas = stream_grid(seg_tiles, h->num_sms);
   sa.n_tiles = seg_tiles; sa.lse_ctas = base_ctas; sa.n_slot = lse_slots(base_ctas, nseg);
   sa.n_chunks = d.n_chunks; sa.tables_per_chunk = d.TC; sa.lsh_bits = c.lsh_bits; sa.lsh_tables = c.lsh_tables;
@@ -587,10 +638,10 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
   sa.key_buckets = key_buckets; sa.fix_items = fix_items; sa.fix_count = ctrl + 1; sa.fix_cap = d.fix_cap;
   sa.status = ctrl;
   sa.polls = h->handoff_polls ? h->handoff_polls : kMaxPolls;
-  sa.spin_polls = h->handoff_polls ? h->handoff_polls : kMaxSpinPolls;
+  sa.poll_ns = h->handoff_polls ? 0u : kPollHintNs;
 
   mark();
-  // 2. per-query log-sum-exp over each block's keys
+  // 2. per-query log-sum-exp over each segment's keys
   if (need_exact) {
     StreamArgs a1 = sa;
     a1.stat_rows = d.GW;
@@ -621,9 +672,9 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
   mark();
   // 5. exact signs where the tensor-core projection was too close to zero
   if (need_lsh) {
-    SignfixArgs fa{static_cast<const uint16_t*>(K_blk), kv_strides[0], kv_strides[1], kv_strides[2], h->P, hist,
-                   counts, key_buckets, fix_items, ctrl + 1, d.fix_cap, c.n_kv_heads, nb, S, c.lsh_bits,
-                   c.lsh_tables, ctrl + 2};
+    SignfixArgs fa{K0, kv_strides[0], kv_strides[1], kv_strides[2], h->P, hist,
+                   counts, key_buckets, fix_items, ctrl + 1, d.fix_cap, c.n_kv_heads, nb, S_len, c.lsh_bits,
+                   c.lsh_tables, ctrl + 2, S};
     signfix_kernel<<<kSignfixCtas, 256, 0, st>>>(fa);
     g_launches.fetch_add(1);
     LKV_CUDA(cudaGetLastError(), "signfix_kernel");
@@ -631,19 +682,18 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
   mark();
   // 6. two-stage top-k
   {
-    const laser_kv_status_t s = launch_select(s_exact, counts, nseg, S, lb.anchors, lb.k_exact, lb.k_lsh,
-                                                (uint32_t)d.GW * (uint32_t)c.lsh_tables, idx, st);
+    SelectArgs sel{s_exact, counts, idx, S_len, g.k_exact, g.k_lsh, g.keep_a_lo, g.keep_a_hi, g.keep_b_lo, g.keep_b_hi,
+                   g.excl_lo, g.excl_hi, g.cand_lo, g.cand_hi, 0};
+    const laser_kv_status_t s = launch_select(sel, nseg, (uint32_t)d.GW * (uint32_t)c.lsh_tables, st);
     if (s != LASER_KV_OK) { h->last_error = g_last_error; return s; }
   }
   mark();
   // 7. gather + append
   {
-    const long long done = h->blocks_done[layer];
     const size_t layer_off = (size_t)layer * c.batch * c.n_kv_heads * (size_t)d.cap;
-    AppendArgs aa{static_cast<const uint16_t*>(K_blk), static_cast<const uint16_t*>(V_blk),
-                  kv_strides[0], kv_strides[1], kv_strides[2], c.n_kv_heads, nb, S, B, idx,
+    AppendArgs aa{K0, V0, kv_strides[0], kv_strides[1], kv_strides[2], c.n_kv_heads, nb, S, B, idx,
                   h->cacheK + layer_off * kHeadDim, h->cacheV + layer_off * kHeadDim, h->cachePos + layer_off,
-                  d.cap * kHeadDim, d.cap, done * B, (int)(done * S), S, ctrl};
+                  d.cap * kHeadDim, d.cap, entries_done, (int)(first_block * S) - g.shift, S_len, ctrl};
     const laser_kv_status_t s = launch_append(aa, nseg, st);
     if (s != LASER_KV_OK) { h->last_error = g_last_error; return s; }
   }
@@ -651,10 +701,110 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
 #undef LKV_CUDA
   if (h->profiling && marks.size() == kProfKernels + 1) h->ev_pending.push_back(marks);
   else for (cudaEvent_t ev : marks) h->ev_pool.push_back(ev);
-  h->blocks_done[layer] += nb;
   h->have_call = true;
   h->last_nb = nb;
   h->last_B = B;
+  h->last_S_len = S_len;
+  h->last_shift = g.shift;
+  return LASER_KV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, const void* K_blk, const void* V_blk,
+                                        const void* Q_win, const int64_t kv_strides[3], const int64_t q_strides[3],
+                                        int32_t n_blocks, void* stream) {
+  if (!h) return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "select_block: NULL handle");
+  if (const laser_kv_status_t ds = check_device(h, "select_block")) return ds;
+  const laser_kv_config_t& c = h->cfg;
+  if (layer < 0 || layer >= c.n_layers) return fail(h, LASER_KV_ERR_INVALID_ARG, "select_block: layer %d out of range", layer);
+  if (!K_blk || !V_blk || !Q_win || !kv_strides || !q_strides)
+    return fail(h, LASER_KV_ERR_INVALID_ARG, "select_block: NULL argument");
+  if (n_blocks < 1) return fail(h, LASER_KV_ERR_INVALID_ARG, "select_block: n_blocks must be >= 1");
+  if (n_blocks > c.max_blocks_per_call)
+    return fail(h, LASER_KV_ERR_CAPACITY, "select_block: n_blocks %d exceeds max_blocks_per_call %d", n_blocks, c.max_blocks_per_call);
+  if (h->lookback_closed[layer])
+    return fail(h, LASER_KV_ERR_STATE, "select_block: layer %d was closed by laser_kv_lookback_close; reset it first", layer);
+  if (h->blocks_done[layer] + n_blocks > c.max_blocks)
+    return fail(h, LASER_KV_ERR_CAPACITY, "select_block: layer %d cache holds %lld of %d blocks; cannot append %d",
+                layer, h->blocks_done[layer], c.max_blocks, n_blocks);
+  if (!aligned16(K_blk) || !aligned16(V_blk) || !aligned16(Q_win))
+    return fail(h, LASER_KV_ERR_ALIGNMENT, "select_block: device pointers must be 16-byte aligned");
+  for (int i = 0; i < 3; ++i)
+    if (kv_strides[i] < 0 || q_strides[i] < 0 || (kv_strides[i] % 8) || (q_strides[i] % 8))
+      return fail(h, LASER_KV_ERR_ALIGNMENT, "select_block: strides must be non-negative multiples of 8 elements");
+  if (kv_strides[2] < kHeadDim || q_strides[2] < kHeadDim)
+    return fail(h, LASER_KV_ERR_INVALID_ARG, "select_block: row stride smaller than head_dim");
+  if ((long long)(h->blocks_done[layer] + n_blocks) * c.block_size > 0x7fffffffLL)
+    return fail(h, LASER_KV_ERR_UNSUPPORTED, "select_block: absolute positions exceed int32");
+
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const laser_kv_ctx::LayerBudget lb = h->budget[layer];
+  const int S = c.block_size;
+  const long long done = h->blocks_done[layer];
+  laser_kv_status_t s = LASER_KV_OK;
+  if (!c.lookback || lb.anchors == 0) {
+    s = run_select(h, layer, K_blk, V_blk, Q_win, kv_strides, q_strides, n_blocks, plain_geom(S, lb), done,
+                   h->entries_done[layer], st);
+    if (s != LASER_KV_OK) return s;
+    h->entries_done[layer] += (long long)n_blocks * lb.B;
+  } else {
+    // the first block of a sequence has no tail before it: it goes alone, the others follow in one pass
+    int first_n = 0;
+    if (done == 0) {
+      const CallGeom g0 = lookback_geom(S, lb, h->d.alpha, true);
+      s = run_select(h, layer, K_blk, V_blk, Q_win, kv_strides, q_strides, 1, g0, 0, 0, st);
+      if (s != LASER_KV_OK) return s;
+      h->entries_done[layer] = g0.B_out;
+      first_n = 1;
+    }
+    if (n_blocks > first_n) {
+      const CallGeom g1 = lookback_geom(S, lb, h->d.alpha, false);
+      const long long off = (long long)first_n * S * kv_strides[2];
+      s = run_select(h, layer, static_cast<const uint16_t*>(K_blk) + off, static_cast<const uint16_t*>(V_blk) + off, Q_win,
+                     kv_strides, q_strides, n_blocks - first_n, g1, done + first_n, h->entries_done[layer], st);
+      if (s != LASER_KV_OK) return s;
+      h->entries_done[layer] += (long long)(n_blocks - first_n) * g1.B_out;
+    }
+  }
+  h->blocks_done[layer] += n_blocks;
+  return LASER_KV_OK;
+}
+
+laser_kv_status_t laser_kv_lookback_close(laser_kv_handle_t h, int32_t layer, const void* K_tail, const void* V_tail,
+                                          const int64_t kv_strides[3], void* stream) {
+  if (!h) return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "lookback_close: NULL handle");
+  if (const laser_kv_status_t ds = check_device(h, "lookback_close")) return ds;
+  const laser_kv_config_t& c = h->cfg;
+  const Derived& d = h->d;
+  if (layer < 0 || layer >= c.n_layers) return fail(h, LASER_KV_ERR_INVALID_ARG, "lookback_close: layer %d out of range", layer);
+  if (!c.lookback) return fail(h, LASER_KV_ERR_STATE, "lookback_close: the handle was created without look-back");
+  if (h->lookback_closed[layer]) return fail(h, LASER_KV_ERR_STATE, "lookback_close: layer %d is already closed", layer);
+  if (h->blocks_done[layer] == 0) return fail(h, LASER_KV_ERR_STATE, "lookback_close: layer %d holds no block", layer);
+  const laser_kv_ctx::LayerBudget lb = h->budget[layer];
+  if (lb.anchors == 0) { h->lookback_closed[layer] = 1; return LASER_KV_OK; }     // nothing was held back
+  if (!K_tail || !V_tail || !kv_strides) return fail(h, LASER_KV_ERR_INVALID_ARG, "lookback_close: NULL argument");
+  if (!aligned16(K_tail) || !aligned16(V_tail))
+    return fail(h, LASER_KV_ERR_ALIGNMENT, "lookback_close: device pointers must be 16-byte aligned");
+  for (int i = 0; i < 3; ++i)
+    if (kv_strides[i] < 0 || (kv_strides[i] % 8))
+      return fail(h, LASER_KV_ERR_ALIGNMENT, "lookback_close: strides must be non-negative multiples of 8 elements");
+  if (kv_strides[2] < kHeadDim || (c.n_kv_heads > 1 && !kv_strides[1]) || (c.batch > 1 && !kv_strides[0]))
+    return fail(h, LASER_KV_ERR_INVALID_ARG, "lookback_close: bad strides");
+  const int a = lb.anchors;
+  const size_t layer_off = (size_t)layer * c.batch * c.n_kv_heads * (size_t)d.cap;
+  int* ctrl = reinterpret_cast<int*>(h->ws + h->carve.ctrl);
+  const long long first_pos = h->blocks_done[layer] * c.block_size - a;
+  AppendArgs aa{static_cast<const uint16_t*>(K_tail), static_cast<const uint16_t*>(V_tail), kv_strides[0], kv_strides[1],
+                kv_strides[2], c.n_kv_heads, 1, 0, a, nullptr, h->cacheK + layer_off * kHeadDim,
+                h->cacheV + layer_off * kHeadDim, h->cachePos + layer_off, d.cap * kHeadDim, d.cap,
+                h->entries_done[layer], (int)first_pos, a, ctrl};
+  const laser_kv_status_t s = launch_append(aa, c.batch * c.n_kv_heads, static_cast<cudaStream_t>(stream));
+  if (s != LASER_KV_OK) { h->last_error = g_last_error; return s; }
+  h->entries_done[layer] += a;
+  h->lookback_closed[layer] = 1;
   return LASER_KV_OK;
 }
 
@@ -668,6 +818,9 @@ laser_kv_status_t laser_kv_select_block_host(laser_kv_handle_t h, int32_t layer,
   if (n_blocks < 1 || n_blocks > h->cfg.max_blocks_per_call)
     return fail(h, LASER_KV_ERR_CAPACITY, "select_block_host: n_blocks out of range");
   const laser_kv_config_t& c = h->cfg;
+  if (c.lookback)
+    return fail(h, LASER_KV_ERR_UNSUPPORTED, "select_block_host: look-back needs the previous block's tail in device memory; "
+                                             "use laser_kv_select_block on a contiguous device copy of the context");
   if (const laser_kv_status_t ds = check_device(h, "select_block_host")) return ds;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const size_t T = (size_t)n_blocks * c.block_size;
@@ -784,7 +937,7 @@ laser_kv_status_t laser_kv_cache_view(laser_kv_handle_t h, int32_t layer, laser_
   out->K = h->cacheK + layer_off * kHeadDim;
   out->V = h->cacheV + layer_off * kHeadDim;
   out->pos = h->cachePos + layer_off;
-  out->len = h->blocks_done[layer] * h->budget[layer].B;
+  out->len = h->entries_done[layer];
   out->cap = d.cap;
   out->kv_strides[0] = (int64_t)c.n_kv_heads * d.cap * kHeadDim;
   out->kv_strides[1] = d.cap * kHeadDim;
@@ -817,7 +970,7 @@ laser_kv_status_t laser_kv_decode_attention(laser_kv_handle_t h, int32_t layer, 
     return fail(h, LASER_KV_ERR_INVALID_ARG, "decode_attention: softmax_scale must be positive (0 selects the configured scale)");
   const int G = c.n_q_heads / c.n_kv_heads;
   if (G > kDecMaxGroup) return fail(h, LASER_KV_ERR_UNSUPPORTED, "decode_attention: more than %d query heads per KV head", kDecMaxGroup);
-  const long long len = h->blocks_done[layer] * h->budget[layer].B;
+  const long long len = h->entries_done[layer];
   if (len < 1) return fail(h, LASER_KV_ERR_STATE, "decode_attention: layer %d cache is empty", layer);
   if (len > 0x7fffffffLL) return fail(h, LASER_KV_ERR_UNSUPPORTED, "decode_attention: cache longer than 2^31 entries");
   if (const laser_kv_status_t ds = check_device(h, "decode_attention")) return ds;
@@ -877,6 +1030,8 @@ laser_kv_status_t laser_kv_debug_view(laser_kv_handle_t h, laser_kv_debug_t* out
   out->batch = c.batch;
   out->n_kv_heads = c.n_kv_heads;
   out->block_size = c.block_size;
+  out->segment_keys = h->last_S_len;
+  out->segment_shift = h->last_shift;
   out->budget = h->last_B;
   out->gw = h->d.GW;
   out->lsh_tables = c.lsh_tables;
@@ -909,8 +1064,12 @@ laser_kv_status_t laser_kv_poll_status(laser_kv_handle_t h, void* stream) {
 laser_kv_status_t laser_kv_reset(laser_kv_handle_t h, int32_t layer) {
   if (!h) return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "reset: NULL handle");
   if (layer < -1 || layer >= h->cfg.n_layers) return fail(h, LASER_KV_ERR_INVALID_ARG, "reset: layer out of range");
-  if (layer == -1) std::fill(h->blocks_done.begin(), h->blocks_done.end(), 0);
-  else h->blocks_done[layer] = 0;
+  for (int l = 0; l < h->cfg.n_layers; ++l) {
+    if (layer != -1 && l != layer) continue;
+    h->blocks_done[l] = 0;
+    h->entries_done[l] = 0;
+    h->lookback_closed[l] = 0;
+  }
   return LASER_KV_OK;
 }
 
@@ -1003,7 +1162,8 @@ laser_kv_status_t laser_kv_two_stage_topk(const float* s_exact, const uint32_t* 
     return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "two_stage_topk: keep count exceeds the segment");
   if (S > 16384) return fail(nullptr, LASER_KV_ERR_UNSUPPORTED, "two_stage_topk: S > 16384");
   if (2 * anchors + k_exact + k_lsh == 0) return LASER_KV_OK;
-  return launch_select(s_exact, counts, n_segments, S, anchors, k_exact, k_lsh, 0u, idx_out, static_cast<cudaStream_t>(stream));
+  const SelectArgs sel{s_exact, counts, idx_out, S, k_exact, k_lsh, 0, anchors, S - anchors, S, 0, 0, anchors, S - anchors, 0};
+  return launch_select(sel, n_segments, 0u, static_cast<cudaStream_t>(stream));
 }
 
 // ---- window scores on caller-fed inputs ----------------------------------------------------------
@@ -1104,7 +1264,7 @@ laser_kv_status_t run_window_scores(const ScoreGeom& g, const void* K_blk, const
   if ((e = cudaGetDevice(&dev)) != cudaSuccess ||
       (e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess)
     return fail(nullptr, LASER_KV_ERR_CUDA, "window_scores: device query: %s", cudaGetErrorString(e));
-  sa.S = g.S; sa.nb = g.nb; sa.H_kv = g.H_kv; sa.batch = g.batch;
+  sa.S = g.S; sa.S_stride = g.S; sa.nb = g.nb; sa.H_kv = g.H_kv; sa.batch = g.batch;
   sa.G = g.G; sa.W = g.W; sa.GW = g.GW; sa.tiles_in_block = g.tiles_in_block; sa.nseg = g.nseg;
   sa.n_tiles = (long long)g.nseg * g.tiles_in_block;
   const int ctas = stream_grid(sa.n_tiles, num_sms);
@@ -1114,7 +1274,7 @@ laser_kv_status_t run_window_scores(const ScoreGeom& g, const void* K_blk, const
   sa.lse2 = reinterpret_cast<float*>(scratch + g.off_lse2);
   sa.s_exact = s_exact_out;
   sa.status = reinterpret_cast<int*>(scratch);
-  sa.polls = kMaxPolls; sa.spin_polls = kMaxSpinPolls;
+  sa.polls = kMaxPolls; sa.poll_ns = kPollHintNs;
   StreamArgs a1 = sa;
   a1.stat_rows = g.GW;
   a1.stat_rows_alloc = ((g.GW + 127) / 128) * 128;
@@ -1350,21 +1510,21 @@ laser_kv_status_t laser_kv_collision_counts(const void* K_blk, const void* Q_win
   {
     StreamArgs sa;
     memset(&sa, 0, sizeof sa);
-    sa.S = g.S; sa.nb = g.nb; sa.H_kv = g.H_kv; sa.batch = g.batch;
+    sa.S = g.S; sa.S_stride = g.S; sa.nb = g.nb; sa.H_kv = g.H_kv; sa.batch = g.batch;
     sa.G = g.G; sa.W = g.W; sa.GW = g.GW; sa.tiles_in_block = g.tiles_in_block; sa.nseg = g.nseg;
     sa.n_chunks = cg.n_chunks; sa.tables_per_chunk = cg.TC; sa.lsh_bits = lsh_bits; sa.lsh_tables = lsh_tables;
     sa.n_tiles = (long long)g.nseg * g.tiles_in_block * cg.n_chunks;
     sa.stat_rows = cg.TC * lsh_bits; sa.stat_rows_alloc = sa.stat_rows;
     sa.counts = counts_out; sa.hist = hist; sa.fix_items = fix_items; sa.fix_count = ctrl + 1; sa.fix_cap = cg.fix_cap;
     sa.status = ctrl;
-    sa.polls = kMaxPolls; sa.spin_polls = kMaxSpinPolls;
+    sa.polls = kMaxPolls; sa.poll_ns = kPollHintNs;
     const uint32_t smem = stream_smem_bytes(kProj, sa.stat_rows_alloc, cg.TC * (2 << lsh_bits));
     if ((e = launch_proj(lsh_bits, cg.TC, mapK, mapP, sa, stream_grid(sa.n_tiles, num_sms), smem, st)) != cudaSuccess)
       return fail(nullptr, LASER_KV_ERR_CUDA, "collision_counts: projection pass: %s", cudaGetErrorString(e));
   }
   {
     SignfixArgs fa{static_cast<const uint16_t*>(K_blk), kv_strides[0], kv_strides[1], kv_strides[2], P, hist, counts_out,
-                   nullptr, fix_items, ctrl + 1, cg.fix_cap, g.H_kv, g.nb, g.S, lsh_bits, lsh_tables, ctrl + 2};
+                   nullptr, fix_items, ctrl + 1, cg.fix_cap, g.H_kv, g.nb, g.S, lsh_bits, lsh_tables, ctrl + 2, g.S};
     signfix_kernel<<<kSignfixCtas, 256, 0, st>>>(fa);
     g_launches.fetch_add(1);
     if ((e = cudaGetLastError()) != cudaSuccess)

@@ -33,6 +33,7 @@ struct SignfixArgs {
   int cap;
   int H_kv, nb, S, K, L;
   int* n_changed;
+  int S_stride;           // tokens between the first keys of consecutive segments
 };
 
 constexpr int kSignfixCtas = 1184;   // 8 CTAs of 256 threads per SM: all resident, about one item per lane group
@@ -53,7 +54,7 @@ __global__ void __launch_bounds__(256) signfix_kernel(const SignfixArgs a) {
     const int h = (seg / a.nb) % a.H_kv;
     const int b = seg / (a.nb * a.H_kv);
     // sixteen key elements per lane
-    const uint16_t* krow = a.Kp + b * a.ks_b + h * a.ks_h + ((long long)t * a.S + key) * a.ks_t + sl * 16;
+    const uint16_t* krow = a.Kp + b * a.ks_b + h * a.ks_h + ((long long)t * a.S_stride + key) * a.ks_t + sl * 16;
     const uint4 ka = *reinterpret_cast<const uint4*>(krow), kb = *reinterpret_cast<const uint4*>(krow + 8);
     const uint32_t kw[8] = {ka.x, ka.y, ka.z, ka.w, kb.x, kb.y, kb.z, kb.w};
     uint32_t code = old_code;
@@ -196,11 +197,17 @@ __device__ void mark_topk(const uint32_t* vals, uint8_t* flag, int lo, int hi, i
   __syncthreads();
 }
 
+// The S scored keys of a segment fall into three classes: kept whatever their scores (two index
+// ranges: Section 3.1's anchors and local window), excluded (one range: a tail that is held back
+// for the next block under look-back, Section 3.2), and candidates (everything else).
 struct SelectArgs {
   const float* s_exact;     // [n_seg][S]
   const uint32_t* counts;   // [n_seg][S]
-  int32_t* idx;             // [n_seg][B]
-  int S, anchors, k_exact, k_lsh;
+  int32_t* idx;             // [n_seg][B], B = kept + k_exact + k_lsh
+  int S, k_exact, k_lsh;
+  int keep_a_lo, keep_a_hi, keep_b_lo, keep_b_hi;   // kept ranges [lo, hi); empty when lo >= hi
+  int excl_lo, excl_hi;                             // excluded range
+  int cand_lo, cand_hi;                             // a range that contains every candidate
   int count_top_shift;      // highest byte position (0, 8, 16 or 24) in which two counts can differ
 };
 
@@ -213,12 +220,14 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectArgs
   __shared__ int misc[2];
   __shared__ int warp_sums[33];
   const int seg = blockIdx.x;
-  const int S = a.S, lo = a.anchors, hi = a.S - a.anchors;
-  const int B = 2 * a.anchors + a.k_exact + a.k_lsh;
+  const int S = a.S, lo = a.cand_lo, hi = a.cand_hi;
+  const int B = max(0, a.keep_a_hi - a.keep_a_lo) + max(0, a.keep_b_hi - a.keep_b_lo) + a.k_exact + a.k_lsh;
+  // flag: 0 candidate, 1 kept, 2 excluded
   for (int j = threadIdx.x; j < S; j += kSelThreads) {
     ukey[j] = orderable_f32(a.s_exact[(size_t)seg * S + j]);
     ucnt[j] = a.counts[(size_t)seg * S + j];
-    flag[j] = (j < lo || j >= hi) ? 1 : 0;
+    const bool kept = (j >= a.keep_a_lo && j < a.keep_a_hi) || (j >= a.keep_b_lo && j < a.keep_b_hi);
+    flag[j] = kept ? 1 : ((j >= a.excl_lo && j < a.excl_hi) ? 2 : 0);
   }
   __syncthreads();
   mark_topk(ukey, flag, lo, hi, a.k_exact, 24, hist, misc, warp_sums);            // K_exact
@@ -227,11 +236,11 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectArgs
   const int per = (S + kSelThreads - 1) / kSelThreads;
   const int j0 = threadIdx.x * per, j1 = min(S, j0 + per);
   int cnt = 0;
-  for (int j = j0; j < j1; ++j) cnt += flag[j];
+  for (int j = j0; j < j1; ++j) cnt += flag[j] == 1;
   int total;
   int out = block_exclusive_scan(cnt, warp_sums, total);
   for (int j = j0; j < j1; ++j)
-    if (flag[j]) { if (out < B) a.idx[(size_t)seg * B + out] = j; ++out; }
+    if (flag[j] == 1) { if (out < B) a.idx[(size_t)seg * B + out] = j; ++out; }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -241,8 +250,10 @@ struct AppendArgs {
   const uint16_t* K;
   const uint16_t* V;
   long long ks_b, ks_h, ks_t;   // source strides (elements): batch, head, token
-  int H_kv, nb, S, B;
-  const int32_t* idx;           // [batch][H_kv][nb][B]
+  int H_kv, nb;
+  int S_stride;                 // source rows between the first rows of consecutive blocks
+  int B;                        // entries per segment
+  const int32_t* idx;           // [batch][H_kv][nb][B]; NULL: entry i is source row i
   uint16_t* Kc;
   uint16_t* Vc;
   int32_t* pos;
@@ -272,12 +283,12 @@ __global__ void __launch_bounds__(256) append_kernel(const AppendArgs a) {
   const int h = bh % a.H_kv, b = bh / a.H_kv;
   const int part = threadIdx.x & 15;
   const int i_end = min(a.B, (int)(blockIdx.x + 1) * kAppendRowsPerCta);
-  const long long src_base = b * a.ks_b + h * a.ks_h + (long long)t * a.S * a.ks_t;
+  const long long src_base = b * a.ks_b + h * a.ks_h + (long long)t * a.S_stride * a.ks_t;
   const long long dst_base = bh * a.c_seg_stride + (a.dst_off0 + (long long)t * a.B) * 128;
   int32_t* pos = a.pos + bh * a.pos_seg_stride + a.dst_off0 + (long long)t * a.B;
-  const int32_t* idx = a.idx + (size_t)seg * a.B;
+  const int32_t* idx = a.idx ? a.idx + (size_t)seg * a.B : nullptr;
   for (int i = blockIdx.x * kAppendRowsPerCta + (threadIdx.x >> 4); i < i_end; i += 16) {
-    const int src = idx[i];
+    const int src = idx ? idx[i] : i;
     if ((unsigned)src >= (unsigned)a.n_src_rows) {          // never read outside the segment
       if (part == 0) atomicCAS(a.status, 0, kAppendBadIndex);
       continue;
@@ -288,7 +299,7 @@ __global__ void __launch_bounds__(256) append_kernel(const AppendArgs a) {
     const uint4 vv = ld_nc_v4(a.V + so);
     *reinterpret_cast<uint4*>(a.Kc + dof) = kv;
     *reinterpret_cast<uint4*>(a.Vc + dof) = vv;
-    if (part == 0) pos[i] = a.pos_base0 + t * a.S + src;
+    if (part == 0) pos[i] = a.pos_base0 + t * a.S_stride + src;
   }
 }
 

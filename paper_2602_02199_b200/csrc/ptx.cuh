@@ -1,6 +1,6 @@
 // Thin inline-PTX wrappers for the sm_100a features the kernels use: mbarriers, TMA tiled and
 // bulk copies, tcgen05 (5th-generation tensor core) MMA with TMEM accumulators.
-// Every wait is bounded by a cycle budget; a wait that gives up returns false and the caller
+// Every wait is bounded by a poll budget; a wait that gives up returns false and the caller
 // records LASER_KV_ERR_TIMEOUT in the status word and unwinds (no trap, no endless loop).
 #pragma once
 #include <cuda.h>
@@ -40,69 +40,28 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-// Bounded waits for the phase with the given parity, written as one PTX loop each so that the
-// fast path (phase already complete) is a try_wait and a branch. Both return false when the poll
-// budget ran out; the budgets correspond to a second or more, far beyond any legitimate wait of
-// these kernels. A caller may pass a smaller budget (a diagnostic setting that makes the give-up
-// path reachable in a test).
-//
-// A try_wait may itself suspend the thread for a hardware-defined time, so a handful of such polls
-// is not a short wait. Budgets below kDiagPolls are therefore served by non-suspending test_wait
-// polls: that is how a test makes a wait run out quickly although the pipeline is healthy.
-constexpr uint32_t kDiagPolls = 1u << 10;
-__device__ __noinline__ bool mbar_wait_diag(uint32_t bar, uint32_t parity, uint32_t max_polls) {
-  for (uint32_t n = 0; n < max_polls; ++n) {
-    uint32_t done;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(done)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    if (done) return true;
-  }
-  return false;
-}
-
-// mbar_wait_spin polls back to back: for the one thread whose reaction time is on the critical
-// path (the MMA issuer).
-constexpr uint32_t kMaxSpinPolls = 1u << 26;
-__device__ __forceinline__ bool mbar_wait_spin(uint32_t bar, uint32_t parity, uint32_t max_polls = kMaxSpinPolls) {
-  if (max_polls < kDiagPolls) return mbar_wait_diag(bar, parity, max_polls);
+// Bounded waits for the phase with the given parity. One poll is a try_wait that may suspend the
+// thread for up to `hint_ns` nanoseconds (the hardware may cut that short; it returns as soon as
+// the phase completes), so the longest wait is max_polls * hint_ns: the built-in budgets give about
+// two seconds, far beyond any legitimate wait of these kernels. A wait that runs out returns false;
+// the caller records LASER_KV_ERR_TIMEOUT and unwinds. hint_ns = 0 is the diagnostic form: every
+// poll is a non-suspending test_wait, so that a handful of polls really is a short time and a test
+// can make a healthy pipeline's waits run out.
+constexpr uint32_t kMaxPolls = 200;
+constexpr uint32_t kPollHintNs = 10u * 1000u * 1000u;
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t max_polls = kMaxPolls,
+                                          uint32_t hint_ns = kPollHintNs) {
   uint32_t ok;
   asm volatile(
-      "{\n\t.reg .pred p;\n\t.reg .u32 n;\n\t"
-      "mov.u32 n, 0;\n"
-      "LKV_SPIN_TRY:\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "@p bra LKV_SPIN_DONE;\n\t"
-      "add.u32 n, n, 1;\n\t"
-      "setp.lt.u32 p, n, %3;\n\t"
-      "@p bra LKV_SPIN_TRY;\n\t"
-      "setp.ne.u32 p, n, n;\n"
-      "LKV_SPIN_DONE:\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity), "r"(max_polls)
-      : "memory");
-  return ok != 0;
-}
-
-// mbar_wait sleeps a few tens of nanoseconds between polls, so that many waiting warps leave the
-// issue slots to the working ones.
-constexpr uint32_t kBackoffNs = 32;
-constexpr uint32_t kMaxPolls = 1u << 25;
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t max_polls = kMaxPolls) {
-  if (max_polls < kDiagPolls) return mbar_wait_diag(bar, parity, max_polls);
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t.reg .u32 n;\n\t"
-      "mov.u32 n, 0;\n"
-      "LKV_WAIT_TRY:\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "{\n\t.reg .pred p, q;\n\t.reg .u32 n;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"      // fast path: already complete
       "@p bra LKV_WAIT_DONE;\n\t"
-      "nanosleep.u32 %4;\n\t"
+      "mov.u32 n, 0;\n\t"
+      "setp.eq.u32 q, %4, 0;\n"
+      "LKV_WAIT_TRY:\n\t"
+      "@!q mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %4;\n\t"
+      "@q mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "@p bra LKV_WAIT_DONE;\n\t"
       "add.u32 n, n, 1;\n\t"
       "setp.lt.u32 p, n, %3;\n\t"
       "@p bra LKV_WAIT_TRY;\n\t"
@@ -110,9 +69,15 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_
       "LKV_WAIT_DONE:\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
-      : "r"(bar), "r"(parity), "r"(max_polls), "r"(kBackoffNs)
+      : "r"(bar), "r"(parity), "r"(max_polls), "r"(hint_ns)
       : "memory");
   return ok != 0;
+}
+// The same wait under the name the critical-path roles (MMA issuer, projection epilogue) use.
+constexpr uint32_t kMaxSpinPolls = kMaxPolls;
+__device__ __forceinline__ bool mbar_wait_spin(uint32_t bar, uint32_t parity, uint32_t max_polls = kMaxPolls,
+                                               uint32_t hint_ns = kPollHintNs) {
+  return mbar_wait(bar, parity, max_polls, hint_ns);
 }
 
 // ---- TMA -------------------------------------------------------------------------------------

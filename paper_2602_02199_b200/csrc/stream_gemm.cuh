@@ -61,7 +61,8 @@ enum : int { kStatusOk = 0, kStatusCapacity = 3, kStatusTimeout = 6 };
 
 struct StreamArgs {
   // problem geometry
-  int S;               // keys per block
+  int S;               // keys per segment (a block; with look-back, the held-back tail of the previous block + the block)
+  int S_stride;        // tokens between the first keys of consecutive segments (the block size)
   int nb;              // blocks in this call
   int H_kv, batch;
   int G, W, GW;        // GQA group size, window, G*W
@@ -85,7 +86,7 @@ struct StreamArgs {
   int* fix_count;
   int fix_cap;
   int* status;
-  uint32_t polls, spin_polls;  // poll budgets of the hand-off waits: sleeping waits, back-to-back waits
+  uint32_t polls, poll_ns;     // budget of the hand-off waits: polls, and nanoseconds a poll may suspend
 };
 
 __device__ __forceinline__ void record_status(int* status, int code) {
@@ -294,7 +295,7 @@ __device__ __forceinline__ bool lse_epilogue(const StreamArgs& a, const EpiCtx& 
     int nvalid = a.S - r.c.tib * kTileKeys - c0;       // key columns of this thread's range that hold a key
     for (int j = 0; j < r.ntiles; ++j, ++it, nvalid -= kTileKeys) {
       const uint32_t acc = it & 1;
-      if (!mbar_wait(e.bar_tfull + 8 * acc, (it >> 1) & 1, a.polls)) return false;
+      if (!mbar_wait(e.bar_tfull + 8 * acc, (it >> 1) & 1, a.polls, a.poll_ns)) return false;
       tc_fence_after();
       uint32_t v[CW];
       load_epi_cols<CW>(t_col + acc * kAccStride, v);
@@ -316,11 +317,11 @@ __device__ __forceinline__ bool lse_epilogue(const StreamArgs& a, const EpiCtx& 
     }
     // end of this segment's run of tiles: merge the column groups, write one partial
     if (cg > 0) {
-      if (flushes > 0 && !mbar_wait(e.bar_xb, (uint32_t)(flushes - 1) & 1, a.polls)) return false;
+      if (flushes > 0 && !mbar_wait(e.bar_xb, (uint32_t)(flushes - 1) & 1, a.polls, a.poll_ns)) return false;
       xch[(cg - 1) * nq + q] = make_float2(m, l);
       mbar_arrive(e.bar_xa);
     } else {
-      if (!mbar_wait(e.bar_xa, (uint32_t)flushes & 1, a.polls)) return false;
+      if (!mbar_wait(e.bar_xa, (uint32_t)flushes & 1, a.polls, a.poll_ns)) return false;
       float mx = m;
 #pragma unroll
       for (int g2 = 1; g2 < ncg; ++g2) mx = fmaxf(mx, xch[(g2 - 1) * nq + q].x);
@@ -382,7 +383,7 @@ __device__ __forceinline__ bool score_epilogue(const StreamArgs& a, const EpiCtx
     int key = r.c.tib * kTileKeys + e.row;
     for (int j = 0; j < r.ntiles; ++j, ++it, key += kTileKeys) {
       const uint32_t acc = it & 1;
-      if (!mbar_wait(e.bar_tfull + 8 * acc, (it >> 1) & 1, a.polls)) return false;
+      if (!mbar_wait(e.bar_tfull + 8 * acc, (it >> 1) & 1, a.polls, a.poll_ns)) return false;
       tc_fence_after();
       float sum = 0.f;
       if constexpr (NC > 0) {
@@ -397,11 +398,11 @@ __device__ __forceinline__ bool score_epilogue(const StreamArgs& a, const EpiCtx
       }
       // groups 1..3 hand their sums to group 0, which adds them in a fixed order
       if (e.wg > 0) {
-        if (it >= 2 && !mbar_wait(e.bar_xb + 8 * acc, ((it >> 1) - 1) & 1, a.polls)) return false;
+        if (it >= 2 && !mbar_wait(e.bar_xb + 8 * acc, ((it >> 1) - 1) & 1, a.polls, a.poll_ns)) return false;
         part[(acc * 3 + (e.wg - 1)) * 128 + e.row] = sum;
         mbar_arrive(e.bar_xa + 8 * acc);
       } else {
-        if (!mbar_wait(e.bar_xa + 8 * acc, (it >> 1) & 1, a.polls)) return false;
+        if (!mbar_wait(e.bar_xa + 8 * acc, (it >> 1) & 1, a.polls, a.poll_ns)) return false;
         const float tot = ((sum + part[(acc * 3 + 0) * 128 + e.row]) + part[(acc * 3 + 1) * 128 + e.row]) +
                           part[(acc * 3 + 2) * 128 + e.row];
         mbar_arrive(e.bar_xb + 8 * acc);
@@ -428,14 +429,14 @@ __device__ __forceinline__ bool proj_epilogue(const StreamArgs& a, const EpiCtx&
     const TileRun r = run_at(x, e.x_end, a);
     if (new_group) {
       // histogram slice landed (async-proxy writes are visible after the wait)
-      if (!mbar_wait(e.bar_stat, gen & 1, a.polls)) return false;
+      if (!mbar_wait(e.bar_stat, gen & 1, a.polls, a.poll_ns)) return false;
       ++gen;
     }
     uint32_t* cnt = a.counts + (size_t)r.c.seg * a.S;
     const int table0 = r.c.chunk * TC;
     int key = r.c.tib * kTileKeys + e.row;
     for (int j = 0; j < r.ntiles; ++j, key += kTileKeys) {
-      if (!mbar_wait_spin(e.bar_tfull + 8 * acc, acc_phase, a.spin_polls)) return false;
+      if (!mbar_wait_spin(e.bar_tfull + 8 * acc, acc_phase, a.polls, a.poll_ns)) return false;
       tc_fence_after();
       const bool valid = key < a.S;
       const uint32_t partial = proj_tables<KBITS, TQ>(e.t_lane + acc * STRIDE, e.bar_tempty + 8 * acc, e.hist_s, a,
@@ -532,7 +533,7 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
       for (long long x = x_begin; x < x_end; ++x, ++it) {
         if (new_group) {
           // stationary operand (+ histogram slice) of the new head / chunk
-          if (gen > 0) ok = mbar_wait(bar_stat_free, (uint32_t)(gen - 1) & 1, a.polls);
+          if (gen > 0) ok = mbar_wait(bar_stat_free, (uint32_t)(gen - 1) & 1, a.polls, a.poll_ns);
           if (!ok) break;
           b = c.bh / a.H_kv;
           h = c.bh - b * a.H_kv;
@@ -551,10 +552,10 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
           ++gen;
         }
         const int s = (int)(it % kStages);
-        if (it >= kStages) ok = mbar_wait(bar_empty + 8 * s, (uint32_t)((it / kStages) - 1) & 1, a.polls);
+        if (it >= kStages) ok = mbar_wait(bar_empty + 8 * s, (uint32_t)((it / kStages) - 1) & 1, a.polls, a.poll_ns);
         if (!ok) break;
         const uint32_t dst = sm_stages + s * kTileBytes;
-        const int token = c.t * a.S + c.tib * kTileKeys;
+        const int token = c.t * a.S_stride + c.tib * kTileKeys;
         mbar_expect_tx(bar_full + 8 * s, kTileBytes);
         tma_load_4d(dst, &map_keys, bar_full + 8 * s, 0, token, h, b);
         tma_load_4d(dst + kTileAtomBytes, &map_keys, bar_full + 8 * s, kAtomCols, token, h, b);
@@ -592,14 +593,14 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
         if (new_group) { ++gen; need_stat = true; }   // stationary operand number `gen` serves this tile
         if (it % kMmaWarps == mine) {
           if (need_stat) {
-            ok = mbar_wait_spin(bar_stat, (gen - 1) & 1, a.spin_polls);
+            ok = mbar_wait_spin(bar_stat, (gen - 1) & 1, a.polls, a.poll_ns);
             if (!ok) break;
             need_stat = false;
           }
           const uint32_t s = it % kStages;
           const uint32_t acc = it % NACC, use = it / NACC;
-          if (use > 0) ok = mbar_wait_spin(bar_tempty + 8 * acc, (use - 1) & 1, a.spin_polls);
-          if (ok) ok = mbar_wait_spin(bar_full + 8 * s, (it / kStages) & 1, a.spin_polls);
+          if (use > 0) ok = mbar_wait_spin(bar_tempty + 8 * acc, (use - 1) & 1, a.polls, a.poll_ns);
+          if (ok) ok = mbar_wait_spin(bar_full + 8 * s, (it / kStages) & 1, a.polls, a.poll_ns);
           if (!ok) break;
           tc_fence_after();
           const uint32_t tile_lo = umma_sdesc_lo(sm_stages + s * kTileBytes);

@@ -52,9 +52,11 @@ def check_signatures(codes_gpu: np.ndarray, x_bits: np.ndarray, p_bits: np.ndarr
 
 def check_segment(*, k_bits, q_bits_group, p_bits, n_bits, n_tables, S, anchors, k_exact, k_lsh,
                   scale, s_gpu, counts_gpu, idx_gpu, qcodes_gpu, kcodes_gpu=None, lse2_gpu=None,
-                  what="segment"):
-    """One (sequence, KV head, block): k_bits [S, d], q_bits_group [G*W, d]; GPU arrays already on
-    the host. Returns a small dict of statistics."""
+                  what="segment", cand=None, kept=None):
+    """One (sequence, KV head, block): k_bits [S, d] (the scored keys), q_bits_group [G*W, d]; GPU
+    arrays already on the host. By default the candidates are [anchors, S - anchors) and the rest is
+    kept (Section 3.1); `cand` and `kept` (ascending index arrays) override that (look-back).
+    Returns a small dict of statistics."""
     stats = {}
     # --- scores ---
     s_or = O.window_scores(q_bits_group, k_bits, scale)
@@ -89,16 +91,18 @@ def check_segment(*, k_bits, q_bits_group, p_bits, n_bits, n_tables, S, anchors,
             _, mabs = O.simhash_buckets(k_bits[bad], p_bits, n_bits, n_tables)
             assert (mabs.min(axis=1) < SIGN_EXEMPT).all(), f"{what}: collision counts differ"
     # --- selection ---
-    B = 2 * anchors + k_exact + k_lsh
+    if cand is None:
+        cand = np.arange(anchors, S - anchors)
+        kept = np.concatenate([np.arange(anchors), np.arange(S - anchors, S)])
+    B = len(kept) + k_exact + k_lsh
     assert idx_gpu.shape == (B,)
     if B > 1:
         assert (np.diff(idx_gpu) > 0).all(), f"{what}: kept indices not strictly ascending"
-    cand = np.arange(anchors, S - anchors)
     # what the selector must produce from the GPU's own scores and counts (bit-exact)
     ke_g = O.topk_lower_index(cand, s_gpu.astype(np.float64), k_exact)
     resid = np.setdiff1d(cand, ke_g, assume_unique=True)
     kl_g = O.topk_lower_index(resid, counts_gpu.astype(np.int64), k_lsh)
-    want_idx = np.sort(np.concatenate([np.arange(anchors), ke_g, kl_g, np.arange(S - anchors, S)]))
+    want_idx = np.sort(np.concatenate([kept, ke_g, kl_g]))
     assert (idx_gpu.astype(np.int64) == want_idx).all(), f"{what}: kept index list differs from the two-stage rule"
     # the GPU's exact picks against the oracle's: only boundary tokens may differ
     ke_o = O.topk_lower_index(cand, s_or, k_exact)
