@@ -35,9 +35,9 @@ from paper_2602_02199_b200 import synth  # noqa: E402
 METRIC = "kv_tokens_scored_and_compacted_per_s_per_layer"
 UNIT = "tokens/s"
 
-# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch, from the ncu capture
-# summarised in profiles/select_call_llama8b_128k.md, keyed by (workload, kernel). A missing key
-# means: not captured for this workload, or the kernel has changed since the capture.
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch, from the committed ncu
+# summary of the select call, keyed by (workload, kernel). A missing key means: not captured for
+# this workload, or the kernel has changed since the capture.
 NCU_TRAFFIC_BYTES = {
     ("llama8b_128k", "stream_kernel<proj>"): 274789120 + 7261184,
     ("llama8b_128k", "stream_kernel<lse>"): 269266944 + 3838720,
@@ -91,7 +91,7 @@ class ClockSampler:
             self.proc.wait(timeout=2)
         except Exception:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
+        sm, mx, pw, reasons = [], [], [], set()
         rows = [l for (t, l) in self.lines if t0 - 0.05 <= t <= t1 + 0.15] or [l for (_, l) in self.lines]
         for l in rows:
             f = [x.strip() for x in l.split(",")]
@@ -101,11 +101,15 @@ class ClockSampler:
                 sm.append(float(f[0])); mx.append(float(f[1]))
             except ValueError:
                 continue
+            try:
+                pw.append(float(f[2]))
+            except ValueError:
+                pass
             for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[4:8]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                "reasons": sorted(reasons), "samples": len(sm), "power_w": statistics.median(pw) if pw else None}
 
 
 def algorithmic_work(w: synth.Workload, B: int):
@@ -138,42 +142,58 @@ def oracle_sample_step(w, k_blk, q, P, heads, B):
                           alpha=w.alpha)
 
 
-def time_oracle(w, steps, warmup, target_s=1.5):
-    """Times the oracle on `heads_per_step` KV heads of one block per step; returns tokens/s where a
-    block counts as S tokens only when all H_kv heads were processed."""
-    from oracle import laser_kv_oracle as O
-    B = O.budget(w.context_len, w.block_size, w.ratio)
-    k_blk, v_blk = synth.kv_block(w, 0, 0, 1)
-    q, P = synth.q_window(w, 0, 0), synth.hyperplanes(w)
-    t0 = time.perf_counter()
-    oracle_sample_step(w, k_blk, q, P, [0], B)
-    one = time.perf_counter() - t0
-    heads_per_step = int(max(1, min(w.n_kv_heads, round(target_s / max(one, 1e-3)))))
-    heads = list(range(heads_per_step))
-    for _ in range(warmup):
-        oracle_sample_step(w, k_blk, q, P, heads, B)
-    t0 = time.perf_counter()
-    for _ in range(steps):
-        r = oracle_sample_step(w, k_blk, q, P, heads, B)
-        cache = O.AppendOnlyCache(len(heads), w.head_dim, B)
-        cache.append(k_blk[heads], v_blk[heads], r.idx, w.block_size)
-    dt = (time.perf_counter() - t0) / steps
-    tokens_per_step = w.block_size * heads_per_step / w.n_kv_heads
+def numpy_threads() -> int:
+    """Threads the BLAS behind numpy uses for the oracle's matrix products."""
     try:
         from threadpoolctl import threadpool_info
-        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+        return max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
     except Exception:
-        cores = os.cpu_count() or 1
-    sample = (f"{heads_per_step} of {w.n_kv_heads} KV heads of one {w.block_size}-token block per step "
-              f"(block 1 of {w.n_blocks}, layer 0); a block counts as {w.block_size} tokens when all heads are done")
-    return tokens_per_step / dt, dt, cores, sample
+        return os.cpu_count() or 1
+
+
+def time_oracle(w, steps, warmup, budget_s=20.0):
+    """Times the oracle, as it stands, on whole units of the workload: every KV head of a block
+    (selection and append), block after block. One step = one block of one layer (the tiny workload:
+    the whole layer, all of its blocks). Returns tokens/s; `steps` is cut so that the timed part stays
+    near `budget_s` seconds."""
+    from oracle import laser_kv_oracle as O
+    B = O.budget(w.context_len, w.block_size, w.ratio)
+    q, P = synth.q_window(w, 0, 0), synth.hyperplanes(w)
+    blocks = list(range(w.n_blocks)) if w.n_blocks * w.block_size <= 8192 else [1]
+    data = [synth.kv_block(w, 0, 0, t) for t in blocks]
+    heads = list(range(w.n_kv_heads))
+
+    def one_step():
+        for t, (k_blk, v_blk) in zip(blocks, data):
+            r = oracle_sample_step(w, k_blk, q, P, heads, B)
+            cache = O.AppendOnlyCache(len(heads), w.head_dim, B)
+            cache.append(k_blk, v_blk, r.idx, t * w.block_size)
+
+    t0 = time.perf_counter()
+    one_step()                                   # also the warm-up
+    one = time.perf_counter() - t0
+    for _ in range(max(0, warmup - 1)):
+        one_step()
+    steps = int(max(1, min(steps, budget_s // max(one, 1e-3))))
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        one_step()
+    dt = (time.perf_counter() - t0) / steps
+    tokens_per_step = w.block_size * len(blocks)
+    if len(blocks) > 1:
+        sample = (f"the whole layer per step: all {w.n_kv_heads} KV heads of all {len(blocks)} blocks of {w.block_size} "
+                  f"tokens (layer 0, sequence 0)")
+    else:
+        sample = (f"one whole block per step: all {w.n_kv_heads} KV heads of block 1 of {w.n_blocks} ({w.block_size} tokens, "
+                  f"layer 0, sequence 0), selection and append; a layer is {w.n_blocks} such blocks"
+                  + (f" x {w.batch} sequences" if w.batch > 1 else "") + ", nothing else is extrapolated")
+    return tokens_per_step / dt, dt, numpy_threads(), sample, steps
 
 
 def run_reference(args, w, rank, world):
     if rank != 0:
         return
-    steps = max(1, min(args.steps, 40))
-    value, dt, cores, sample = time_oracle(w, steps, min(args.warmup, 3))
+    value, dt, cores, sample, steps = time_oracle(w, max(1, min(args.steps, 40)), min(args.warmup, 3), budget_s=120.0)
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
         "warmup": min(args.warmup, 3), "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
@@ -270,7 +290,7 @@ def run_ours(args, w, rank, world, local_rank):
     if rank == 0:
         sampler.start()
         time.sleep(0.25)
-    eng.laser_kv_profile_enable(True)
+    # ---- the headline: K steps, nothing recorded between the kernels ----
     launches0 = Bn.laser_kv_launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
@@ -283,11 +303,42 @@ def run_ours(args, w, rank, world, local_rank):
     t_wall1 = time.time()
     ms = e0.elapsed_time(e1)
     launches = Bn.laser_kv_launch_count() - launches0
-    prof = eng.laser_kv_profile_read()
-    eng.laser_kv_profile_enable(False)
     eng.laser_kv_poll_status()
     sign_fixups = int(eng.laser_kv_debug_view().n_sign_fixups)
     clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
+
+    # ---- per-kernel breakdown: a separate loop with CUDA events between the kernels ----
+    prof_steps = max(1, min(args.steps, 50))
+    eng.laser_kv_profile_enable(True)
+    for i in range(prof_steps):
+        step(i)
+    prof = eng.laser_kv_profile_read()
+    eng.laser_kv_profile_enable(False)
+
+    # ---- sustained: the same step back to back for about 1.5 s, long enough for the power cap to
+    #      settle the SM clock; reported beside the headline, with the clock it ran at ----
+    sustained = None
+    if not args.skip_sustained:
+        sus_steps = int(max(args.steps, min(20000, 1500.0 / max(ms / args.steps, 1e-3))))
+        sus_sampler = ClockSampler(local_rank)
+        if rank == 0:
+            sus_sampler.start()
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        tw0 = time.time()
+        s0.record()
+        for i in range(sus_steps):
+            step(i)
+        s1.record()
+        barrier()
+        tw1 = time.time()
+        sus_ms, = max_over_ranks([s0.elapsed_time(s1)], world, dev)
+        if rank == 0:
+            sc = sus_sampler.stop(tw0 + 0.3, tw1)         # the first 0.3 s: the clock is still settling
+            sustained = {"steps": sus_steps, "ms_per_step": sus_ms / sus_steps, "sm_mhz": sc["sm_mhz"],
+                         "power_w": sc.get("power_w"), "reasons": sc["reasons"], "samples": sc.get("samples"),
+                         "ms_per_step_x_ghz": (sus_ms / sus_steps) * (sc["sm_mhz"] or 0.0) / 1000.0}
+        eng.laser_kv_poll_status()
 
     # ---- end to end: pinned host inputs -> device, select, appended positions -> host ----
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
@@ -352,6 +403,8 @@ def run_ours(args, w, rank, world, local_rank):
     t_tensor = work["flops"] / (peaks["tf"] * 1e12)
     path = {
         "hbm_frac": t_hbm / (ms_per_step * 1e-3), "tensor_frac": t_tensor / (ms_per_step * 1e-3),
+        "hbm_frac_of_8tbs_nominal": work["bytes"] / 8e12 / (ms_per_step * 1e-3),
+        "tensor_frac_of_sustained": work["flops"] / (peaks["tf_sustained"] * 1e12) / (ms_per_step * 1e-3),
         "binding_frac": max(t_hbm, t_tensor) / (ms_per_step * 1e-3),
         "bytes_alg_per_step": work["bytes"], "flops_alg_per_step": work["flops"],
         "kernels_ms_per_step": {k: v[0] / v[1] for k, v in kern.items()},
@@ -362,7 +415,7 @@ def run_ours(args, w, rank, world, local_rank):
     if args.skip_cpu:
         cpu_value, cores, sample = None, 0, "skipped (--skip-cpu)"
     else:
-        cpu_value, _, cores, sample = time_oracle(w, steps=max(1, args.cpu_steps), warmup=1)
+        cpu_value, _, cores, sample, _ = time_oracle(w, steps=max(1, args.cpu_steps), warmup=1)
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -375,6 +428,7 @@ def run_ours(args, w, rank, world, local_rank):
                    "l2": f"inputs larger than L2: {n_sets} layers of K+V ({2 * host[0][0].numel() * 2 >> 20} MiB each) cycled",
                    "parallelism": "replicas" if world > 1 else "single"},
         "clocks": clocks,
+        "sustained": sustained,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps,
                 "note": "pinned host K and Q copied in four chunks, kept V rows read in place from pinned host "
@@ -745,6 +799,7 @@ def main():
     ap.add_argument("--cpu-steps", type=int, default=6)
     ap.add_argument("--skip-cpu", action="store_true", help="omit the oracle timing (profiling runs)")
     ap.add_argument("--skip-e2e", action="store_true", help="omit the host-buffer timing (profiling runs)")
+    ap.add_argument("--skip-sustained", action="store_true", help="omit the 1.5 s sustained loop (profiling runs)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     rank = int(os.environ.get("RANK", "0"))

@@ -167,10 +167,24 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
                                         const int64_t kv_strides[3], const int64_t q_strides[3],
                                         int32_t n_blocks, void* stream);
 
+/* A last block that has fewer tokens than block_size (the paper's contexts are whole numbers of
+ * blocks; reading taken here: the same rule on the tokens there are). n_tokens in [1, block_size)
+ * tokens at K_blk / V_blk (same layout and strides as laser_kv_select_block, one block) are scored
+ * against Q_win and selected with the budget B_t = min(B, n_tokens): anchors and local window
+ * floor(B_t/n) each, recall budget B_t - 2*floor(B_t/n) split by alpha; a block with no more tokens
+ * than B keeps all of them. B_t entries are appended (under look-back the block's last floor(B_t/n)
+ * tokens are held back for laser_kv_lookback_close like any block's, and the previous block's
+ * held-back tokens are decided here). Afterwards the layer accepts no further block until
+ * laser_kv_reset (positions would no longer be those of whole blocks). */
+laser_kv_status_t laser_kv_select_tail(laser_kv_handle_t h, int32_t layer, const void* K_blk,
+                                       const void* V_blk, const void* Q_win,
+                                       const int64_t kv_strides[3], const int64_t q_strides[3],
+                                       int32_t n_tokens, void* stream);
+
 /* Closes a look-back sequence (config.lookback = 1): appends the a = floor(B/n) tokens that the last
  * block held back - nothing follows them, so nothing can prune them. K_tail / V_tail: dev bf16
- * [batch][H_kv][a][d] through kv_strides, the last a rows of the last block (K_blk + (S - a) rows of
- * that block, same strides). Afterwards the layer accepts no block until laser_kv_reset. STATE if the
+ * [batch][H_kv][a][d] through kv_strides, the last a rows of the last block (same strides as the
+ * block; a = floor(B_t/n) of that block's own budget when it was a short one). Afterwards the layer accepts no block until laser_kv_reset. STATE if the
  * handle has no look-back, the layer holds no block or is closed already. */
 laser_kv_status_t laser_kv_lookback_close(laser_kv_handle_t h, int32_t layer, const void* K_tail,
                                           const void* V_tail, const int64_t kv_strides[3], void* stream);

@@ -30,6 +30,9 @@ What each function follows:
                           introduction's append-only accumulative memory.
 * ``decode_attention``  - Section 3 (the kept tokens serve the decoding phase): softmax attention
                           of one decode query over the cache entries of its KV head.
+* ``tail_budget``       - a last block with fewer tokens than a block (not covered by the paper,
+                          whose contexts are whole numbers of blocks): the same rule with
+                          B_t = min(B, tokens).
 * ``lookback_partition`` / ``select_block_lookback`` / ``LookbackPrefill`` - Section 3.2 (block
                           processing and boundary smoothing): the scoring window of block t also
                           covers the tail of block t-1, whose tokens are pruned only then.
@@ -61,7 +64,7 @@ __all__ = [
     "bf16_bits_to_f64", "budget", "partition", "window_scores", "simhash_projections",
     "simhash_buckets", "collision_counts", "topk_lower_index", "select_indices",
     "group_queries", "select_block", "AppendOnlyCache", "BlockResult",
-    "lookback_partition", "select_block_lookback", "LookbackPrefill", "LookbackResult",
+    "lookback_partition", "select_block_lookback", "LookbackPrefill", "LookbackResult", "tail_budget",
 ]
 
 
@@ -395,17 +398,30 @@ def decode_attention(q_bits: np.ndarray, k_bits: np.ndarray, v_bits: np.ndarray,
 #           B_long = B - 2a; the tail [S - a, S) is held back. B - a entries appended.
 #   g >= 1: scored keys = held-back tail of block g-1 (a keys) followed by the block (S keys);
 #           kept = anchors of the block + Algorithm 1 on C = tail(g-1) + [a, S - a) of the block
-#           with B_long = B - a (the recall budget plus the a entries the slid window released);
+#           with B_long = (B - 2a) + a = B - a (the recall budget plus the a entries the slid window released);
 #           the block's own tail is held back. B entries appended, in position order.
 #   close : the tail of the last block is appended as it is (nothing follows it). a entries.
 # After m blocks and the close the cache holds m * B entries per head, as without look-back.
-def lookback_partition(B: int, n: int, alpha: float, first: bool):
-    """(anchors, held_back, B_long, k_exact, k_lsh) of one look-back step; see the rule above."""
+def lookback_partition(B: int, n: int, alpha: float, released: int):
+    """(anchors, held_back, B_long, k_exact, k_lsh) of one look-back step; see the rule above.
+    `released` is the number of held-back tokens of the previous block that this step decides about
+    (0 for the first block of a sequence): the recall budget is the block's own B - 2a plus those
+    entries, which the previous block's local window no longer occupies."""
     a, _, b_long0, _, _ = partition(B, n, alpha)
-    b_long = b_long0 if first else B - a
+    b_long = b_long0 + released
     k_e = int(math.floor(float(alpha) * float(b_long)))
     k_e = max(0, min(k_e, b_long))
     return a, a, b_long, k_e, b_long - k_e
+
+
+def tail_budget(B: int, n_tokens: int) -> int:
+    """Budget of a last block that has fewer tokens than a block (the paper's contexts are whole
+    numbers of blocks; reading taken: the same rule on the tokens there are): B_t = min(B, S_t).
+    The partition of B_t by the protection divisor and alpha is the usual one, so a tail block with
+    at least B tokens keeps B of them and a shorter one keeps all of its tokens."""
+    if n_tokens < 1:
+        raise ValueError("a block has at least one token")
+    return min(B, n_tokens)
 
 
 @dataclass
@@ -430,17 +446,19 @@ def select_block_lookback(k_prev_tail, k_bits: np.ndarray, q_bits: np.ndarray, p
     """
     h_kv, S, d = k_bits.shape
     first = k_prev_tail is None
-    a, _, b_long, k_e, k_l = lookback_partition(B, n, alpha, first)
+    a, _, b_long, k_e, k_l = lookback_partition(B, n, alpha, 0 if first else k_prev_tail.shape[1])
     if 2 * a > S or B > S:
         raise ValueError("budget does not fit the block")
     if first:
         scored = k_bits
         off = 0
     else:
-        if k_prev_tail.shape != (h_kv, a, d):
-            raise ValueError("the held-back tail must have floor(B/n) rows per head")
+        # the previous block's tail has that block's own floor(B/n) rows (a shorter last block, see
+        # tail_budget, has a smaller budget than the blocks before it)
+        if k_prev_tail.shape[0] != h_kv or k_prev_tail.shape[2] != d:
+            raise ValueError("the held-back tail must be [H_kv, rows, d]")
         scored = np.concatenate([k_prev_tail, k_bits], axis=1)
-        off = a
+        off = k_prev_tail.shape[1]
     n_scored = scored.shape[1]
     # candidates: the previous tail, and the block without its anchors and without its own tail
     cand = np.concatenate([np.arange(0, off, dtype=np.int64),
@@ -477,24 +495,38 @@ class LookbackPrefill:
         self.a = B // n
         self.tail = None             # (k, v, first position) of the held-back tokens
         self.blocks = 0
+        self.tokens = 0
+        self.block_size = None
+        self.short = False
         self.closed = False
 
     def step(self, k_bits, v_bits, q_bits, p_bits) -> LookbackResult:
-        if self.closed:
-            raise ValueError("the sequence was closed")
+        """One block. A block with fewer tokens than the ones before it (the last one) runs with
+        tail_budget(B, tokens); nothing may follow it but close()."""
+        if self.closed or self.short:
+            raise ValueError("the sequence was closed or has had its short last block")
         S = k_bits.shape[1]
-        start = self.blocks * S
+        if self.block_size is None:
+            self.block_size = S
+        start = self.tokens
+        kw = dict(self.kw)
+        if S < self.block_size:
+            kw["B"] = tail_budget(kw["B"], S)
+            self.short = True
+        elif S != self.block_size:
+            raise ValueError("only the last block may differ in length, and only by being shorter")
         prev = None if self.tail is None else self.tail[0]
-        r = select_block_lookback(prev, k_bits, q_bits, p_bits, **self.kw)
+        r = select_block_lookback(prev, k_bits, q_bits, p_bits, **kw)
         if self.tail is None:
             ks, vs = k_bits, v_bits
         else:
             ks = np.concatenate([self.tail[0], k_bits], axis=1)
             vs = np.concatenate([self.tail[1], v_bits], axis=1)
         self.cache.append(ks, vs, r.idx, start + r.offset)
-        a = self.a
+        a = kw["B"] // kw["n"]
         self.tail = (k_bits[:, S - a:].copy(), v_bits[:, S - a:].copy(), start + S - a)
         self.blocks += 1
+        self.tokens += S
         return r
 
     def close(self):

@@ -21,7 +21,7 @@ EXPORTS = [
     "laser_kv_collision_counts", "laser_kv_collision_counts_scratch_bytes", "laser_kv_consensus_accumulate",
     "laser_kv_decode_attention", "laser_kv_decode_attention_scratch_bytes", "laser_kv_collision_probability",
     "laser_kv_set_layer_budget", "laser_kv_set_wait_budget", "laser_kv_window_scores_static_status",
-    "laser_kv_lookback_close",
+    "laser_kv_lookback_close", "laser_kv_select_tail",
 ]
 
 
@@ -108,6 +108,8 @@ def load(build_if_missing: bool = True) -> C.CDLL:
     lib.laser_kv_two_stage_topk.argtypes = [vp, vp, i32, i32, i32, i32, i32, vp, vp]
     lib.laser_kv_gather_append.restype = i32
     lib.laser_kv_gather_append.argtypes = [vp, vp, i64, i64, i32, vp, i32, i32, vp, vp, i64, i64, vp, i64, i64, i32, vp, vp]
+    lib.laser_kv_select_tail.restype = i32
+    lib.laser_kv_select_tail.argtypes = [vp, i32, vp, vp, vp, p(i64), p(i64), i32, vp]
     lib.laser_kv_lookback_close.restype = i32
     lib.laser_kv_lookback_close.argtypes = [vp, i32, vp, vp, p(i64), vp]
     lib.laser_kv_set_wait_budget.restype = i32
@@ -264,6 +266,14 @@ class LaserKV:
                                                    _ptr(Q_host), _ptr(K_stage), _ptr(V_stage),
                                                    _ptr(Q_stage), n_blocks, _ptr(pos_out_host),
                                                    _stream_ptr(stream)), self.handle)
+
+    def laser_kv_select_tail(self, layer, K_blk, V_blk, Q_win, n_tokens, stream=None):
+        """A last block of n_tokens < block_size tokens: K_blk, V_blk [batch][H_kv][n_tokens][d]."""
+        ks = (C.c_int64 * 3)(*K_blk.stride()[:3])
+        assert tuple(V_blk.stride()) == tuple(K_blk.stride()) and K_blk.stride(3) == 1
+        qs = (C.c_int64 * 3)(*Q_win.stride()[:3])
+        _check(self.lib.laser_kv_select_tail(self.handle, layer, _ptr(K_blk), _ptr(V_blk), _ptr(Q_win),
+                                             ks, qs, n_tokens, _stream_ptr(stream)), self.handle)
 
     def laser_kv_lookback_close(self, layer, K_tail, V_tail, stream=None):
         """K_tail, V_tail: [batch][H_kv][a][d] views of the last block's last a = floor(B/n) rows."""

@@ -76,7 +76,10 @@ struct laser_kv_ctx {
   int num_sms = 1;
   std::vector<long long> blocks_done;   // per layer: blocks processed
   std::vector<long long> entries_done;  // per layer: cache entries final per (sequence, KV head)
-  std::vector<char> lookback_closed;    // per layer: the held-back tail of the last block was appended
+  std::vector<long long> tokens_done;   // per layer: tokens of the blocks processed
+  std::vector<int> held_back;           // per layer: tokens the last block holds back (look-back), 0 once appended
+  std::vector<char> sealed;             // per layer: a short last block or the look-back close ended the sequence
+  std::vector<char> lookback_done;      // per layer: laser_kv_lookback_close has run
   struct LayerBudget { int B, anchors, k_exact, k_lsh; };
   std::vector<LayerBudget> budget;      // per layer; the configured budget unless laser_kv_set_layer_budget changed it
   int last_B = 0;                       // budget of the last select call (debug view)
@@ -461,7 +464,10 @@ laser_kv_status_t laser_kv_init(const laser_kv_config_t* cfg, const void* hyperp
   h->P = static_cast<const uint16_t*>(hyperplanes);
   h->blocks_done.assign(cfg->n_layers, 0);
   h->entries_done.assign(cfg->n_layers, 0);
-  h->lookback_closed.assign(cfg->n_layers, 0);
+  h->tokens_done.assign(cfg->n_layers, 0);
+  h->held_back.assign(cfg->n_layers, 0);
+  h->sealed.assign(cfg->n_layers, 0);
+  h->lookback_done.assign(cfg->n_layers, 0);
   h->budget.assign(cfg->n_layers, laser_kv_ctx::LayerBudget{d.B, d.anchors, d.k_exact, d.k_lsh});
   h->last_B = d.B;
   {
@@ -495,61 +501,54 @@ struct CallGeom {
   int keep_a_lo, keep_a_hi, keep_b_lo, keep_b_hi, excl_lo, excl_hi, cand_lo, cand_hi;   // scored-key index ranges
   int k_exact, k_lsh;
   int B_out;                 // cache entries per block and head
+  int S_tok;                 // tokens per block of this pass (the block size; fewer for a short last block)
+  int held_back;             // tokens of each block that stay undecided after the pass (look-back)
 };
 
-// The plain rule: anchors and local window kept, Algorithm 1 on what lies between.
-CallGeom plain_geom(int S, const laser_kv_ctx::LayerBudget& lb) {
+// Geometry of a pass over blocks of `S_tok` tokens with budget `B` per block (Section 3.1: anchors
+// and local window a = floor(B/n) each, recall budget B - 2a split by alpha, Algorithm 1 lines 4/7).
+// Plain rule: anchors and local window kept, Algorithm 1 on what lies between.
+// Look-back (Section 3.2): the block's local window is held back instead and the `released`
+// held-back tokens of the previous block (0 for the first block of a sequence) are scored with it:
+// the segment is those tokens followed by the block, the block's anchors are kept, the released
+// tokens and the block's middle are the candidates, and the recall budget grows by the entries the
+// previous window no longer occupies.
+CallGeom make_geom(int S_tok, int B, int n, double alpha, bool lookback, int released) {
+  const int a = B / n;
   CallGeom g;
-  g.S_len = S; g.shift = 0;
-  g.keep_a_lo = 0; g.keep_a_hi = lb.anchors; g.keep_b_lo = S - lb.anchors; g.keep_b_hi = S;
-  g.excl_lo = g.excl_hi = 0;
-  g.cand_lo = lb.anchors; g.cand_hi = S - lb.anchors;
-  g.k_exact = lb.k_exact; g.k_lsh = lb.k_lsh;
-  g.B_out = lb.B;
-  return g;
-}
-
-// Look-back (Section 3.2): a block's local window [S - a, S) is held back and scored again with the
-// next block. First block of a sequence: anchors + Algorithm 1 on [a, S - a) with the plain recall
-// budget. Later blocks: the segment is the previous block's tail followed by the block; the block's
-// anchors are kept, the tail of the previous block and the block's middle are the candidates with
-// recall budget B - a, the block's own tail is held back.
-CallGeom lookback_geom(int S, const laser_kv_ctx::LayerBudget& lb, double alpha, bool first) {
-  const int a = lb.anchors;
-  CallGeom g;
-  g.keep_b_lo = g.keep_b_hi = 0;
-  if (first) {
-    g.S_len = S; g.shift = 0;
-    g.keep_a_lo = 0; g.keep_a_hi = a;
-    g.excl_lo = S - a; g.excl_hi = S;
-    g.cand_lo = a; g.cand_hi = S - a;
-    g.k_exact = lb.k_exact; g.k_lsh = lb.k_lsh;
-    g.B_out = lb.B - a;
+  g.S_tok = S_tok;
+  const int b_long = B - 2 * a + (lookback ? released : 0);
+  int ke = (int)std::floor(alpha * (double)b_long);
+  if (ke < 0) ke = 0;
+  if (ke > b_long) ke = b_long;
+  g.k_exact = ke; g.k_lsh = b_long - ke;
+  g.held_back = lookback ? a : 0;
+  if (!lookback) {
+    g.S_len = S_tok; g.shift = 0;
+    g.keep_a_lo = 0; g.keep_a_hi = a; g.keep_b_lo = S_tok - a; g.keep_b_hi = S_tok;
+    g.excl_lo = g.excl_hi = 0;
+    g.cand_lo = a; g.cand_hi = S_tok - a;
+    g.B_out = B;
   } else {
-    g.S_len = S + a; g.shift = a;
-    g.keep_a_lo = a; g.keep_a_hi = 2 * a;
-    g.excl_lo = S; g.excl_hi = S + a;
-    g.cand_lo = 0; g.cand_hi = S;
-    const int b_long = lb.B - a;
-    int ke = (int)std::floor(alpha * (double)b_long);
-    if (ke < 0) ke = 0;
-    if (ke > b_long) ke = b_long;
-    g.k_exact = ke; g.k_lsh = b_long - ke;
-    g.B_out = lb.B;
+    g.S_len = S_tok + released; g.shift = released;
+    g.keep_a_lo = released; g.keep_a_hi = released + a; g.keep_b_lo = g.keep_b_hi = 0;
+    g.excl_lo = released + S_tok - a; g.excl_hi = released + S_tok;
+    g.cand_lo = 0; g.cand_hi = released + S_tok - a;
+    g.B_out = a + b_long;
   }
   return g;
 }
 
 // One pass of the path over nb consecutive blocks with the same geometry. K_blk / V_blk point at
 // the first token of the first block; with g.shift > 0 the g.shift rows before it (the tail of the
-// previous block) are read as well. `first_block` is the index of the first block in the sequence,
+// previous block) are read as well. `first_token` is the position of the first block's first token,
 // `entries_done` the cache entries already final per head.
 laser_kv_status_t run_select(laser_kv_ctx* h, int layer, const void* K_blk, const void* V_blk, const void* Q_win,
                              const int64_t kv_strides[3], const int64_t q_strides[3], int nb, const CallGeom& g,
-                             long long first_block, long long entries_done, cudaStream_t st) {
+                             long long first_token, long long entries_done, cudaStream_t st) {
   const laser_kv_config_t& c = h->cfg;
   const Derived& d = h->d;
-  const int S = c.block_size, S_len = g.S_len, B = g.B_out;
+  const int S = g.S_tok, S_len = g.S_len, B = g.B_out;
   const int nseg = c.batch * c.n_kv_heads * nb;
   const int tiles_in_block = (S_len + kTileKeys - 1) / kTileKeys;
   uint8_t* ws = h->ws;
@@ -693,7 +692,7 @@ laser_kv_status_t run_select(laser_kv_ctx* h, int layer, const void* K_blk, cons
     const size_t layer_off = (size_t)layer * c.batch * c.n_kv_heads * (size_t)d.cap;
     AppendArgs aa{K0, V0, kv_strides[0], kv_strides[1], kv_strides[2], c.n_kv_heads, nb, S, B, idx,
                   h->cacheK + layer_off * kHeadDim, h->cacheV + layer_off * kHeadDim, h->cachePos + layer_off,
-                  d.cap * kHeadDim, d.cap, entries_done, (int)(first_block * S) - g.shift, S_len, ctrl};
+                  d.cap * kHeadDim, d.cap, entries_done, (int)first_token - g.shift, S_len, ctrl};
     const laser_kv_status_t s = launch_append(aa, nseg, st);
     if (s != LASER_KV_OK) { h->last_error = g_last_error; return s; }
   }
@@ -713,63 +712,99 @@ laser_kv_status_t run_select(laser_kv_ctx* h, int layer, const void* K_blk, cons
 
 extern "C" {
 
+// Argument checks shared by the block and the short-block entry points.
+static laser_kv_status_t check_select_args(laser_kv_ctx* h, int layer, const void* K_blk, const void* V_blk, const void* Q_win,
+                                           const int64_t kv_strides[3], const int64_t q_strides[3], const char* who) {
+  const laser_kv_config_t& c = h->cfg;
+  if (layer < 0 || layer >= c.n_layers) return fail(h, LASER_KV_ERR_INVALID_ARG, "%s: layer %d out of range", who, layer);
+  if (!K_blk || !V_blk || !Q_win || !kv_strides || !q_strides) return fail(h, LASER_KV_ERR_INVALID_ARG, "%s: NULL argument", who);
+  if (h->sealed[layer])
+    return fail(h, LASER_KV_ERR_STATE, "%s: layer %d has had its last block (a short block or laser_kv_lookback_close); reset it first", who, layer);
+  if (!aligned16(K_blk) || !aligned16(V_blk) || !aligned16(Q_win))
+    return fail(h, LASER_KV_ERR_ALIGNMENT, "%s: device pointers must be 16-byte aligned", who);
+  for (int i = 0; i < 3; ++i)
+    if (kv_strides[i] < 0 || q_strides[i] < 0 || (kv_strides[i] % 8) || (q_strides[i] % 8))
+      return fail(h, LASER_KV_ERR_ALIGNMENT, "%s: strides must be non-negative multiples of 8 elements", who);
+  if (kv_strides[2] < kHeadDim || q_strides[2] < kHeadDim)
+    return fail(h, LASER_KV_ERR_INVALID_ARG, "%s: row stride smaller than head_dim", who);
+  return LASER_KV_OK;
+}
+
 laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, const void* K_blk, const void* V_blk,
                                         const void* Q_win, const int64_t kv_strides[3], const int64_t q_strides[3],
                                         int32_t n_blocks, void* stream) {
   if (!h) return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "select_block: NULL handle");
   if (const laser_kv_status_t ds = check_device(h, "select_block")) return ds;
   const laser_kv_config_t& c = h->cfg;
-  if (layer < 0 || layer >= c.n_layers) return fail(h, LASER_KV_ERR_INVALID_ARG, "select_block: layer %d out of range", layer);
-  if (!K_blk || !V_blk || !Q_win || !kv_strides || !q_strides)
-    return fail(h, LASER_KV_ERR_INVALID_ARG, "select_block: NULL argument");
+  if (const laser_kv_status_t as = check_select_args(h, layer, K_blk, V_blk, Q_win, kv_strides, q_strides, "select_block")) return as;
   if (n_blocks < 1) return fail(h, LASER_KV_ERR_INVALID_ARG, "select_block: n_blocks must be >= 1");
   if (n_blocks > c.max_blocks_per_call)
     return fail(h, LASER_KV_ERR_CAPACITY, "select_block: n_blocks %d exceeds max_blocks_per_call %d", n_blocks, c.max_blocks_per_call);
-  if (h->lookback_closed[layer])
-    return fail(h, LASER_KV_ERR_STATE, "select_block: layer %d was closed by laser_kv_lookback_close; reset it first", layer);
   if (h->blocks_done[layer] + n_blocks > c.max_blocks)
     return fail(h, LASER_KV_ERR_CAPACITY, "select_block: layer %d cache holds %lld of %d blocks; cannot append %d",
                 layer, h->blocks_done[layer], c.max_blocks, n_blocks);
-  if (!aligned16(K_blk) || !aligned16(V_blk) || !aligned16(Q_win))
-    return fail(h, LASER_KV_ERR_ALIGNMENT, "select_block: device pointers must be 16-byte aligned");
-  for (int i = 0; i < 3; ++i)
-    if (kv_strides[i] < 0 || q_strides[i] < 0 || (kv_strides[i] % 8) || (q_strides[i] % 8))
-      return fail(h, LASER_KV_ERR_ALIGNMENT, "select_block: strides must be non-negative multiples of 8 elements");
-  if (kv_strides[2] < kHeadDim || q_strides[2] < kHeadDim)
-    return fail(h, LASER_KV_ERR_INVALID_ARG, "select_block: row stride smaller than head_dim");
-  if ((long long)(h->blocks_done[layer] + n_blocks) * c.block_size > 0x7fffffffLL)
+  if (h->tokens_done[layer] + (long long)n_blocks * c.block_size > 0x7fffffffLL)
     return fail(h, LASER_KV_ERR_UNSUPPORTED, "select_block: absolute positions exceed int32");
 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const laser_kv_ctx::LayerBudget lb = h->budget[layer];
-  const int S = c.block_size;
-  const long long done = h->blocks_done[layer];
+  const int S = c.block_size, n = c.protection_divisor;
+  const bool lookback = c.lookback && lb.anchors > 0;
   laser_kv_status_t s = LASER_KV_OK;
-  if (!c.lookback || lb.anchors == 0) {
-    s = run_select(h, layer, K_blk, V_blk, Q_win, kv_strides, q_strides, n_blocks, plain_geom(S, lb), done,
-                   h->entries_done[layer], st);
+  int first_n = 0;
+  if (lookback && h->blocks_done[layer] == 0) {
+    // the first block of a sequence has no held-back tokens before it: it goes alone
+    const CallGeom g0 = make_geom(S, lb.B, n, h->d.alpha, true, 0);
+    s = run_select(h, layer, K_blk, V_blk, Q_win, kv_strides, q_strides, 1, g0, 0, 0, st);
     if (s != LASER_KV_OK) return s;
-    h->entries_done[layer] += (long long)n_blocks * lb.B;
-  } else {
-    // the first block of a sequence has no tail before it: it goes alone, the others follow in one pass
-    int first_n = 0;
-    if (done == 0) {
-      const CallGeom g0 = lookback_geom(S, lb, h->d.alpha, true);
-      s = run_select(h, layer, K_blk, V_blk, Q_win, kv_strides, q_strides, 1, g0, 0, 0, st);
-      if (s != LASER_KV_OK) return s;
-      h->entries_done[layer] = g0.B_out;
-      first_n = 1;
-    }
-    if (n_blocks > first_n) {
-      const CallGeom g1 = lookback_geom(S, lb, h->d.alpha, false);
-      const long long off = (long long)first_n * S * kv_strides[2];
-      s = run_select(h, layer, static_cast<const uint16_t*>(K_blk) + off, static_cast<const uint16_t*>(V_blk) + off, Q_win,
-                     kv_strides, q_strides, n_blocks - first_n, g1, done + first_n, h->entries_done[layer], st);
-      if (s != LASER_KV_OK) return s;
-      h->entries_done[layer] += (long long)(n_blocks - first_n) * g1.B_out;
-    }
+    h->entries_done[layer] = g0.B_out;
+    h->blocks_done[layer] = 1;
+    h->tokens_done[layer] = S;
+    h->held_back[layer] = g0.held_back;
+    first_n = 1;
   }
-  h->blocks_done[layer] += n_blocks;
+  if (n_blocks > first_n) {
+    const CallGeom g1 = make_geom(S, lb.B, n, h->d.alpha, lookback, lookback ? h->held_back[layer] : 0);
+    const long long off = (long long)first_n * S * kv_strides[2];
+    const int nb = n_blocks - first_n;
+    s = run_select(h, layer, static_cast<const uint16_t*>(K_blk) + off, static_cast<const uint16_t*>(V_blk) + off, Q_win,
+                   kv_strides, q_strides, nb, g1, h->tokens_done[layer], h->entries_done[layer], st);
+    if (s != LASER_KV_OK) return s;
+    h->entries_done[layer] += (long long)nb * g1.B_out;
+    h->blocks_done[layer] += nb;
+    h->tokens_done[layer] += (long long)nb * S;
+    h->held_back[layer] = g1.held_back;
+  }
+  return LASER_KV_OK;
+}
+
+laser_kv_status_t laser_kv_select_tail(laser_kv_handle_t h, int32_t layer, const void* K_blk, const void* V_blk,
+                                       const void* Q_win, const int64_t kv_strides[3], const int64_t q_strides[3],
+                                       int32_t n_tokens, void* stream) {
+  if (!h) return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "select_tail: NULL handle");
+  if (const laser_kv_status_t ds = check_device(h, "select_tail")) return ds;
+  const laser_kv_config_t& c = h->cfg;
+  if (const laser_kv_status_t as = check_select_args(h, layer, K_blk, V_blk, Q_win, kv_strides, q_strides, "select_tail")) return as;
+  if (n_tokens < 1 || n_tokens >= c.block_size)
+    return fail(h, LASER_KV_ERR_INVALID_ARG, "select_tail: n_tokens must be in [1, block_size); whole blocks go through laser_kv_select_block");
+  if (h->blocks_done[layer] + 1 > c.max_blocks)
+    return fail(h, LASER_KV_ERR_CAPACITY, "select_tail: layer %d cache holds %lld of %d blocks", layer, h->blocks_done[layer], c.max_blocks);
+  if (h->tokens_done[layer] + n_tokens > 0x7fffffffLL)
+    return fail(h, LASER_KV_ERR_UNSUPPORTED, "select_tail: absolute positions exceed int32");
+  const laser_kv_ctx::LayerBudget lb = h->budget[layer];
+  const int B_t = lb.B < n_tokens ? lb.B : n_tokens;           // the same rule on the tokens there are
+  const bool lookback = c.lookback != 0;
+  const CallGeom g = make_geom(n_tokens, B_t, c.protection_divisor, h->d.alpha, lookback, lookback ? h->held_back[layer] : 0);
+  if (g.B_out > 0) {
+    const laser_kv_status_t s = run_select(h, layer, K_blk, V_blk, Q_win, kv_strides, q_strides, 1, g, h->tokens_done[layer],
+                                           h->entries_done[layer], static_cast<cudaStream_t>(stream));
+    if (s != LASER_KV_OK) return s;
+  }
+  h->entries_done[layer] += g.B_out;
+  h->blocks_done[layer] += 1;
+  h->tokens_done[layer] += n_tokens;
+  h->held_back[layer] = g.held_back;
+  h->sealed[layer] = 1;
   return LASER_KV_OK;
 }
 
@@ -781,30 +816,32 @@ laser_kv_status_t laser_kv_lookback_close(laser_kv_handle_t h, int32_t layer, co
   const Derived& d = h->d;
   if (layer < 0 || layer >= c.n_layers) return fail(h, LASER_KV_ERR_INVALID_ARG, "lookback_close: layer %d out of range", layer);
   if (!c.lookback) return fail(h, LASER_KV_ERR_STATE, "lookback_close: the handle was created without look-back");
-  if (h->lookback_closed[layer]) return fail(h, LASER_KV_ERR_STATE, "lookback_close: layer %d is already closed", layer);
   if (h->blocks_done[layer] == 0) return fail(h, LASER_KV_ERR_STATE, "lookback_close: layer %d holds no block", layer);
-  const laser_kv_ctx::LayerBudget lb = h->budget[layer];
-  if (lb.anchors == 0) { h->lookback_closed[layer] = 1; return LASER_KV_OK; }     // nothing was held back
-  if (!K_tail || !V_tail || !kv_strides) return fail(h, LASER_KV_ERR_INVALID_ARG, "lookback_close: NULL argument");
-  if (!aligned16(K_tail) || !aligned16(V_tail))
-    return fail(h, LASER_KV_ERR_ALIGNMENT, "lookback_close: device pointers must be 16-byte aligned");
-  for (int i = 0; i < 3; ++i)
-    if (kv_strides[i] < 0 || (kv_strides[i] % 8))
-      return fail(h, LASER_KV_ERR_ALIGNMENT, "lookback_close: strides must be non-negative multiples of 8 elements");
-  if (kv_strides[2] < kHeadDim || (c.n_kv_heads > 1 && !kv_strides[1]) || (c.batch > 1 && !kv_strides[0]))
-    return fail(h, LASER_KV_ERR_INVALID_ARG, "lookback_close: bad strides");
-  const int a = lb.anchors;
-  const size_t layer_off = (size_t)layer * c.batch * c.n_kv_heads * (size_t)d.cap;
-  int* ctrl = reinterpret_cast<int*>(h->ws + h->carve.ctrl);
-  const long long first_pos = h->blocks_done[layer] * c.block_size - a;
-  AppendArgs aa{static_cast<const uint16_t*>(K_tail), static_cast<const uint16_t*>(V_tail), kv_strides[0], kv_strides[1],
-                kv_strides[2], c.n_kv_heads, 1, 0, a, nullptr, h->cacheK + layer_off * kHeadDim,
-                h->cacheV + layer_off * kHeadDim, h->cachePos + layer_off, d.cap * kHeadDim, d.cap,
-                h->entries_done[layer], (int)first_pos, a, ctrl};
-  const laser_kv_status_t s = launch_append(aa, c.batch * c.n_kv_heads, static_cast<cudaStream_t>(stream));
-  if (s != LASER_KV_OK) { h->last_error = g_last_error; return s; }
-  h->entries_done[layer] += a;
-  h->lookback_closed[layer] = 1;
+  if (h->lookback_done[layer]) return fail(h, LASER_KV_ERR_STATE, "lookback_close: layer %d is already closed", layer);
+  const int a = h->held_back[layer];
+  if (a > 0) {
+    if (!K_tail || !V_tail || !kv_strides) return fail(h, LASER_KV_ERR_INVALID_ARG, "lookback_close: NULL argument");
+    if (!aligned16(K_tail) || !aligned16(V_tail))
+      return fail(h, LASER_KV_ERR_ALIGNMENT, "lookback_close: device pointers must be 16-byte aligned");
+    for (int i = 0; i < 3; ++i)
+      if (kv_strides[i] < 0 || (kv_strides[i] % 8))
+        return fail(h, LASER_KV_ERR_ALIGNMENT, "lookback_close: strides must be non-negative multiples of 8 elements");
+    if (kv_strides[2] < kHeadDim || (c.n_kv_heads > 1 && !kv_strides[1]) || (c.batch > 1 && !kv_strides[0]))
+      return fail(h, LASER_KV_ERR_INVALID_ARG, "lookback_close: bad strides");
+    const size_t layer_off = (size_t)layer * c.batch * c.n_kv_heads * (size_t)d.cap;
+    int* ctrl = reinterpret_cast<int*>(h->ws + h->carve.ctrl);
+    const long long first_pos = h->tokens_done[layer] - a;
+    AppendArgs aa{static_cast<const uint16_t*>(K_tail), static_cast<const uint16_t*>(V_tail), kv_strides[0], kv_strides[1],
+                  kv_strides[2], c.n_kv_heads, 1, 0, a, nullptr, h->cacheK + layer_off * kHeadDim,
+                  h->cacheV + layer_off * kHeadDim, h->cachePos + layer_off, d.cap * kHeadDim, d.cap,
+                  h->entries_done[layer], (int)first_pos, a, ctrl};
+    const laser_kv_status_t s = launch_append(aa, c.batch * c.n_kv_heads, static_cast<cudaStream_t>(stream));
+    if (s != LASER_KV_OK) { h->last_error = g_last_error; return s; }
+    h->entries_done[layer] += a;
+    h->held_back[layer] = 0;
+  }
+  h->lookback_done[layer] = 1;
+  h->sealed[layer] = 1;
   return LASER_KV_OK;
 }
 
@@ -858,7 +895,7 @@ laser_kv_status_t laser_kv_select_block_host(laser_kv_handle_t h, int32_t layer,
     return fail(h, LASER_KV_ERR_CUDA, "select_block_host: H2D copy: %s", cudaGetErrorString(e));
   const int64_t kvs[3] = {(int64_t)c.n_kv_heads * (int64_t)T * kHeadDim, (int64_t)T * kHeadDim, kHeadDim};
   const int64_t qs[3] = {(int64_t)c.n_q_heads * c.window * kHeadDim, (int64_t)c.window * kHeadDim, kHeadDim};
-  const long long before = h->blocks_done[layer];
+  const long long before = h->entries_done[layer];
   const size_t pitch = T * kHeadDim * 2, rows = (size_t)c.batch * c.n_kv_heads;
   // Only the kept rows of V are ever read (by the append kernel). When the host V buffer is pinned
   // and mapped into the device's address space the kernel reads those rows in place over the bus
@@ -917,9 +954,9 @@ laser_kv_status_t laser_kv_select_block_host(laser_kv_handle_t h, int32_t layer,
   if (pos_out_host) {
     const Derived& d = h->d;
     const size_t layer_off = (size_t)layer * c.batch * c.n_kv_heads * (size_t)d.cap;
-    const size_t Bl = (size_t)h->budget[layer].B;
-    const int32_t* src = h->cachePos + layer_off + before * Bl;
-    e = cudaMemcpy2DAsync(pos_out_host, (size_t)n_blocks * Bl * 4, src, (size_t)d.cap * 4, (size_t)n_blocks * Bl * 4,
+    const size_t n_new = (size_t)(h->entries_done[layer] - before);
+    const int32_t* src = h->cachePos + layer_off + before;
+    e = cudaMemcpy2DAsync(pos_out_host, n_new * 4, src, (size_t)d.cap * 4, n_new * 4,
                           (size_t)c.batch * c.n_kv_heads, cudaMemcpyDeviceToHost, st);
     if (e != cudaSuccess) return fail(h, LASER_KV_ERR_CUDA, "select_block_host: D2H copy: %s", cudaGetErrorString(e));
   }
@@ -1068,7 +1105,10 @@ laser_kv_status_t laser_kv_reset(laser_kv_handle_t h, int32_t layer) {
     if (layer != -1 && l != layer) continue;
     h->blocks_done[l] = 0;
     h->entries_done[l] = 0;
-    h->lookback_closed[l] = 0;
+    h->tokens_done[l] = 0;
+    h->held_back[l] = 0;
+    h->sealed[l] = 0;
+    h->lookback_done[l] = 0;
   }
   return LASER_KV_OK;
 }

@@ -42,7 +42,7 @@ def _check_pass(w, eng, K, Q, P, B, first_block, n_blocks):
     """The debug view of the last pass (blocks first_block .. first_block + n_blocks - 1) against the oracle."""
     S, n = w.block_size, w.protection_divisor
     first = first_block == 0
-    a, _, b_long, k_e, k_l = O.lookback_partition(B, n, w.alpha, first)
+    a, _, b_long, k_e, k_l = O.lookback_partition(B, n, w.alpha, 0 if first else B // n)
     dbg = eng.laser_kv_debug_view()
     off = 0 if first else a
     assert dbg.segment_keys == S + off and dbg.segment_shift == off
@@ -142,4 +142,62 @@ def test_lookback_state_errors_and_reset():
     e0.laser_kv_select_block(0, t2["K"], t2["V"], t2["Q"], 2)
     with pytest.raises(Bn.LaserKVError) as err:
         e0.laser_kv_lookback_close(0, *tail)
+    assert err.value.status == Bn.ERR_STATE
+
+
+@pytest.mark.parametrize("lookback,S_t", [(0, 200), (0, 72), (0, 8), (1, 200), (1, 72), (1, 1)])
+def test_short_last_block(lookback, S_t):
+    """Two whole blocks and a last one of S_t < S tokens (S_t above and below the budget, and tiny):
+    the short block runs with B_t = min(B, S_t); under look-back it also decides about the held-back
+    tokens of the block before it."""
+    import torch
+    from paper_2602_02199_b200 import binding as Bn
+    S, B, nb = 256, 96, 3
+    w = synth.workload("tiny").with_(name=f"tail{lookback}_{S_t}", block_size=S, context_len=nb * S, n_layers=1,
+                                     needles="uniform:3", lsh_bits=8, lsh_tables=16)
+    K, V, Q, P, t, engine = _setup(w, nb, B, lookback=lookback)
+    n, a = w.protection_divisor, B // w.protection_divisor
+    T = 2 * S + S_t
+    e = engine()
+    e.laser_kv_select_block(0, t["K"][:, :, :2 * S], t["V"][:, :, :2 * S], t["Q"], 2)
+    e.laser_kv_select_tail(0, t["K"][:, :, 2 * S:T], t["V"][:, :, 2 * S:T], t["Q"], S_t)
+    e.laser_kv_poll_status()
+    B_t = O.tail_budget(B, S_t)
+    a_t = B_t // n
+    released = a if lookback else 0
+    _, _, b_long, k_e, k_l = O.lookback_partition(B_t, n, w.alpha, released) if lookback else (0, 0) + O.partition(B_t, n, w.alpha)[2:]
+    dbg = e.laser_kv_debug_view()
+    assert dbg.segment_keys == S_t + released and dbg.segment_shift == released
+    s_all, c_all, idx_all = to_np(dbg.s_exact), to_np(dbg.counts), to_np(dbg.idx)
+    qc_all, kc_all, lse_all = to_np(dbg.query_buckets), to_np(dbg.key_buckets), to_np(dbg.lse2)
+    if lookback:
+        cand = np.concatenate([np.arange(0, released), np.arange(released + a_t, released + S_t - a_t)])
+        kept = np.arange(released, released + a_t)
+    else:
+        cand = np.arange(a_t, S_t - a_t)
+        kept = np.concatenate([np.arange(a_t), np.arange(S_t - a_t, S_t)])
+    n_out = len(kept) + k_e + k_l
+    assert n_out == (B_t - a_t + released if lookback else B_t)
+    for h in range(w.n_kv_heads):
+        scored = K[0, h, 2 * S - released:T]
+        if n_out:
+            check_segment(k_bits=scored, q_bits_group=O.group_queries(Q[0], w.n_kv_heads, h), p_bits=P, n_bits=w.lsh_bits,
+                          n_tables=w.lsh_tables, S=S_t + released, anchors=a_t, k_exact=k_e, k_lsh=k_l, scale=None,
+                          s_gpu=s_all[0, h, 0], counts_gpu=c_all[0, h, 0], idx_gpu=idx_all[0, h, 0][:n_out],
+                          qcodes_gpu=qc_all[0, h], kcodes_gpu=kc_all[0, h, 0], lse2_gpu=lse_all[0, h, 0],
+                          what=f"tail h{h}", cand=cand, kept=kept)
+    if lookback:
+        e.laser_kv_lookback_close(0, t["K"][:, :, T - a_t:T], t["V"][:, :, T - a_t:T])
+        e.laser_kv_poll_status()
+    Kc, Vc, pos, length = e.laser_kv_cache_view(0)
+    assert length == 2 * B + B_t
+    Kc, Vc, pos = to_np(Kc).view(np.uint16), to_np(Vc).view(np.uint16), to_np(pos)
+    for h in range(w.n_kv_heads):
+        p = pos[0, h, :length].astype(np.int64)
+        assert (np.diff(p) > 0).all() and p[-1] == T - 1 and (p < T).all()
+        assert (Kc[0, h, :length] == K[0, h, p]).all() and (Vc[0, h, :length] == V[0, h, p]).all()
+        if S_t <= B:                                            # a short block no larger than the budget is kept whole
+            assert set(range(2 * S, T)) <= set(p.tolist())
+    with pytest.raises(Bn.LaserKVError) as err:                # nothing follows a short block
+        e.laser_kv_select_block(0, t["K"][:, :, :S], t["V"][:, :, :S], t["Q"], 1)
     assert err.value.status == Bn.ERR_STATE

@@ -24,10 +24,12 @@ def _small(S=64, seed=11, **kw):
 
 def test_partition_of_a_lookback_step():
     # first block: the plain recall budget; later blocks: the window's released entries join it
-    assert O.lookback_partition(3855, 4, 0.75, True) == (963, 963, 1929, 1446, 483)
-    assert O.lookback_partition(3855, 4, 0.75, False) == (963, 963, 3855 - 963, math.floor(0.75 * 2892), 2892 - 2169)
-    assert O.lookback_partition(40, 2, 0.75, False) == (20, 20, 20, 15, 5)          # n = 2: only released entries
-    assert O.lookback_partition(6, 8, 0.5, False) == (0, 0, 6, 3, 3)               # empty window: plain rule
+    assert O.lookback_partition(3855, 4, 0.75, 0) == (963, 963, 1929, 1446, 483)
+    assert O.lookback_partition(3855, 4, 0.75, 963) == (963, 963, 3855 - 963, math.floor(0.75 * 2892), 2892 - 2169)
+    assert O.lookback_partition(40, 2, 0.75, 20) == (20, 20, 20, 15, 5)            # n = 2: only released entries
+    assert O.lookback_partition(6, 8, 0.5, 0) == (0, 0, 6, 3, 3)                   # empty window: plain rule
+    # a short last block (budget 100, a = 25) after full blocks that held 963 tokens back
+    assert O.lookback_partition(100, 4, 0.5, 963) == (25, 25, 50 + 963, 506, 507)
 
 
 def test_empty_local_window_reduces_to_the_plain_rule():
@@ -153,3 +155,35 @@ def test_prefill_keep_counts_order_and_append_only():
         assert set(range(4 * 64 - a, 4 * 64)) <= set(p.tolist())
     with pytest.raises(ValueError):
         run.step(*synth.kv_block(w, 0, 0, 0), synth.q_window(w, 0, 0), P)
+
+
+def test_short_last_block_plain_rule_and_lookback_totals():
+    # plain rule: a last block of S_t tokens runs with B_t = min(B, S_t)
+    assert O.tail_budget(24, 40) == 24 and O.tail_budget(24, 10) == 10 and O.tail_budget(24, 24) == 24
+    w, P = _small(S=64, seed=9)
+    q = synth.q_window(w, 0, 0)
+    k, v = synth.kv_block(w, 0, 0, 2)
+    for S_t in (40, 10, 1):
+        Bt = O.tail_budget(24, S_t)
+        r = O.select_block(k[:, :S_t], q, P, n_bits=4, n_tables=8, B=Bt, n=4)
+        assert r.idx.shape == (2, Bt) and (r.idx < S_t).all()
+        if S_t <= 24:                                       # fewer tokens than the budget: all of them are kept
+            assert r.idx[0].tolist() == list(range(S_t))
+    # look-back with a short last block: the cache ends with (full blocks) * B + B_t entries
+    B, n = 24, 4
+    for S_t in (40, 10):
+        run = O.LookbackPrefill(2, 128, capacity=4 * B, n_bits=4, n_tables=8, B=B, n=n)
+        for t in range(2):
+            kk, vv = synth.kv_block(w, 0, 0, t)
+            run.step(kk, vv, q, P)
+        run.step(k[:, :S_t], v[:, :S_t], q, P)
+        with pytest.raises(ValueError):
+            run.step(k, v, q, P)                            # nothing follows a short block
+        run.close()
+        Bt = O.tail_budget(B, S_t)
+        assert run.cache.length == 2 * B + Bt
+        for h in range(2):
+            p = run.cache.pos[h, :run.cache.length]
+            assert (np.diff(p) > 0).all() and p[-1] == 2 * 64 + S_t - 1
+            if S_t <= B:                                    # every token of the short block is there
+                assert set(range(128, 128 + S_t)) <= set(p.tolist())
