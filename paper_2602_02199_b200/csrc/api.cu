@@ -29,9 +29,9 @@ constexpr int kHeadDim = 128;
 constexpr size_t kAlign = 256;
 constexpr int kMaxSmem = 227 * 1024;
 
-constexpr int kProfKernels = 7;
+constexpr int kProfKernels = 6;
 const char* const kProfNames[kProfKernels] = {"qsig_kernel", "stream_kernel<lse>", "stream_kernel<score>",
-                                              "stream_kernel<proj>", "signfix_kernel", "select_kernel", "append_kernel"};
+                                              "stream_kernel<proj>", "select_kernel", "append_kernel"};
 
 std::atomic<long long> g_launches{0};
 thread_local std::string g_last_error;
@@ -54,7 +54,7 @@ struct Derived {
 };
 
 struct Carve {
-  size_t ctrl, dec_count, hist, qbuckets, lse_part, lse2, s_exact, counts, idx, fix_items, key_buckets, total;
+  size_t ctrl, dec_count, hist, qbuckets, lse_part, lse2, s_exact, counts, idx, fix_counts, fix_items, key_buckets, total;
 };
 
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
@@ -214,9 +214,10 @@ laser_kv_status_t derive(const laser_kv_config_t* c, Derived* d) {
     return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "config: lookback must be 0 or 1");
   // with look-back a segment is the previous block's held-back tail followed by the block
   d->S_ws = c->block_size + (c->lookback ? d->anchors : 0);
-  long long fc = nseg * d->S_ws * (long long)c->lsh_tables / 256;
-  if (fc < 4096) fc = 4096;
-  if (fc > (1 << 26)) fc = 1 << 26;
+  // exact-sign work list of a segment: about 5e-4 of its (key, table) pairs are expected
+  long long fc = d->S_ws * (long long)c->lsh_tables / 256;
+  if (fc < 256) fc = 256;
+  if (fc > (1 << 22)) fc = 1 << 22;
   d->fix_cap = (int)fc;
   return LASER_KV_OK;
 }
@@ -235,7 +236,8 @@ void carve_ws(const laser_kv_config_t* c, const Derived& d, Carve* v) {
   v->s_exact = take(nseg * S * 4);
   v->counts = take(nseg * S * 4 + 16);     // cleared in 16-byte units
   v->idx = take(nseg * (size_t)(d.B > 0 ? d.B : 1) * 4);
-  v->fix_items = take((size_t)d.fix_cap * sizeof(int4));
+  v->fix_counts = take(nseg * sizeof(int));
+  v->fix_items = take(nseg * (size_t)d.fix_cap * sizeof(int4));
   v->key_buckets = take(c->debug ? nseg * S * c->lsh_tables * 2 : 0);
   v->total = off;
 }
@@ -561,6 +563,7 @@ laser_kv_status_t run_select(laser_kv_ctx* h, int layer, const void* K_blk, cons
   uint32_t* counts = reinterpret_cast<uint32_t*>(ws + h->carve.counts);
   int32_t* idx = reinterpret_cast<int32_t*>(ws + h->carve.idx);
   int4* fix_items = reinterpret_cast<int4*>(ws + h->carve.fix_items);
+  int* fix_counts = reinterpret_cast<int*>(ws + h->carve.fix_counts);
   uint16_t* key_buckets = c.debug ? reinterpret_cast<uint16_t*>(ws + h->carve.key_buckets) : nullptr;
   // the segment's first key: g.shift rows before the block
   const uint16_t* K0 = static_cast<const uint16_t*>(K_blk) - (long long)g.shift * kv_strides[2];
@@ -618,7 +621,7 @@ laser_kv_status_t run_select(laser_kv_ctx* h, int layer, const void* K_blk, cons
     const int q_alloc = ((d.GW + 127) / 128) * 128;
     QsigArgs qa{static_cast<const uint16_t*>(Q_win), q_strides[0], q_strides[1], q_strides[2], h->P, hist, qb,
                 c.n_kv_heads, d.G, c.window, d.GW, q_alloc, c.lsh_tables,
-                reinterpret_cast<uint4*>(counts), ((long long)nseg * S_len + 3) / 4, ctrl + 1, ctrl};
+                reinterpret_cast<uint4*>(counts), ((long long)nseg * S_len + 3) / 4, ctrl + 1, fix_counts, nseg, ctrl};
     dim3 grid(c.lsh_tables / kQsigTables, c.n_kv_heads, c.batch);
     LKV_CUDA(launch_qsig(c.lsh_bits, mapQ, h->mapPq, qa, grid, qsig_smem_bytes(q_alloc, c.lsh_bits), st), "qsig_kernel");
   }
@@ -634,7 +637,7 @@ laser_kv_status_t run_select(laser_kv_ctx* h, int layer, const void* K_blk, cons
   sa.n_chunks = d.n_chunks; sa.tables_per_chunk = d.TC; sa.lsh_bits = c.lsh_bits; sa.lsh_tables = c.lsh_tables;
   sa.scale_log2e = d.scale * 1.4426950408889634f;
   sa.lse_part = lse_part; sa.lse2 = lse2; sa.s_exact = s_exact; sa.counts = counts; sa.hist = hist;
-  sa.key_buckets = key_buckets; sa.fix_items = fix_items; sa.fix_count = ctrl + 1; sa.fix_cap = d.fix_cap;
+  sa.key_buckets = key_buckets; sa.fix_items = fix_items; sa.fix_count = fix_counts; sa.fix_cap = d.fix_cap;
   sa.status = ctrl;
   sa.polls = h->handoff_polls ? h->handoff_polls : kMaxPolls;
   sa.poll_ns = h->handoff_polls ? 0u : kPollHintNs;
@@ -669,25 +672,18 @@ laser_kv_status_t run_select(laser_kv_ctx* h, int layer, const void* K_blk, cons
              "projection pass");
   }
   mark();
-  // 5. exact signs where the tensor-core projection was too close to zero
-  if (need_lsh) {
-    SignfixArgs fa{K0, kv_strides[0], kv_strides[1], kv_strides[2], h->P, hist,
-                   counts, key_buckets, fix_items, ctrl + 1, d.fix_cap, c.n_kv_heads, nb, S_len, c.lsh_bits,
-                   c.lsh_tables, ctrl + 2, S};
-    signfix_kernel<<<kSignfixCtas, 256, 0, st>>>(fa);
-    g_launches.fetch_add(1);
-    LKV_CUDA(cudaGetLastError(), "signfix_kernel");
-  }
-  mark();
-  // 6. two-stage top-k
+  // 5. exact signs where the tensor-core projection was too close to zero (every segment's CTA
+  //    settles its own list first), then the two-stage top-k
   {
     SelectArgs sel{s_exact, counts, idx, S_len, g.k_exact, g.k_lsh, g.keep_a_lo, g.keep_a_hi, g.keep_b_lo, g.keep_b_hi,
-                   g.excl_lo, g.excl_hi, g.cand_lo, g.cand_hi, 0};
+                   g.excl_lo, g.excl_hi, g.cand_lo, g.cand_hi, 0, need_lsh ? 1 : 0,
+                   SignfixArgs{K0, kv_strides[0], kv_strides[1], kv_strides[2], h->P, hist, counts, key_buckets, fix_items,
+                               fix_counts, d.fix_cap, c.n_kv_heads, nb, S_len, c.lsh_bits, c.lsh_tables, ctrl + 2, S, ctrl + 1}};
     const laser_kv_status_t s = launch_select(sel, nseg, (uint32_t)d.GW * (uint32_t)c.lsh_tables, st);
     if (s != LASER_KV_OK) { h->last_error = g_last_error; return s; }
   }
   mark();
-  // 7. gather + append
+  // 6. gather + append
   {
     const size_t layer_off = (size_t)layer * c.batch * c.n_kv_heads * (size_t)d.cap;
     AppendArgs aa{K0, V0, kv_strides[0], kv_strides[1], kv_strides[2], c.n_kv_heads, nb, S, B, idx,
@@ -1092,7 +1088,7 @@ laser_kv_status_t laser_kv_poll_status(laser_kv_handle_t h, void* stream) {
     cudaStreamSynchronize(st);
     if (host[0] == LASER_KV_ERR_TIMEOUT) return fail(h, LASER_KV_ERR_TIMEOUT, "a bounded device-side wait gave up");
     if (host[0] == LASER_KV_ERR_CAPACITY)
-      return fail(h, LASER_KV_ERR_CAPACITY, "exact-sign recompute list overflowed (%d items, capacity %d)", host[1], h->d.fix_cap);
+      return fail(h, LASER_KV_ERR_CAPACITY, "an exact-sign recompute list overflowed (%d items in all, capacity %d per segment)", host[1], h->d.fix_cap);
     return fail(h, (laser_kv_status_t)host[0], "device status word %d", host[0]);
   }
   return LASER_KV_OK;
@@ -1428,7 +1424,7 @@ namespace {
 struct CountGeom {
   ScoreGeom g;
   int K, L, TC, n_chunks, fix_cap;
-  size_t off_hist, off_qb, off_fix, total;   // scratch layout after the 256-byte control block
+  size_t off_hist, off_qb, off_fixcnt, off_fix, total;   // scratch layout after the 256-byte control block
 };
 
 laser_kv_status_t count_geometry(int32_t batch, int32_t n_q_heads, int32_t n_kv_heads, int32_t block_size, int32_t window,
@@ -1444,15 +1440,16 @@ laser_kv_status_t count_geometry(int32_t batch, int32_t n_q_heads, int32_t n_kv_
   if ((long long)cg->g.GW * lsh_tables > 0x7fffffffLL)
     return fail(nullptr, LASER_KV_ERR_UNSUPPORTED, "collision_counts: G*W*lsh_tables too large");
   cg->n_chunks = lsh_tables / cg->TC;
-  long long fc = (long long)cg->g.nseg * block_size * lsh_tables / 256;
-  if (fc < 4096) fc = 4096;
-  if (fc > (1 << 26)) fc = 1 << 26;
+  long long fc = (long long)block_size * lsh_tables / 256;
+  if (fc < 256) fc = 256;
+  if (fc > (1 << 22)) fc = 1 << 22;
   cg->fix_cap = (int)fc;
   const size_t bh = (size_t)batch * n_kv_heads;
   size_t off = 256;
   cg->off_hist = off; off = align_up(off + bh * lsh_tables * ((size_t)2 << lsh_bits));
   cg->off_qb = off;   off = align_up(off + bh * cg->g.GW * lsh_tables * 2);
-  cg->off_fix = off;  off = align_up(off + (size_t)cg->fix_cap * sizeof(int4));
+  cg->off_fixcnt = off; off = align_up(off + (size_t)cg->g.nseg * sizeof(int));
+  cg->off_fix = off;  off = align_up(off + (size_t)cg->g.nseg * cg->fix_cap * sizeof(int4));
   cg->total = off;
   return LASER_KV_OK;
 }
@@ -1534,6 +1531,7 @@ laser_kv_status_t laser_kv_collision_counts(const void* K_blk, const void* Q_win
   uint16_t* hist = reinterpret_cast<uint16_t*>(sc + cg.off_hist);
   uint16_t* qb = reinterpret_cast<uint16_t*>(sc + cg.off_qb);
   int4* fix_items = reinterpret_cast<int4*>(sc + cg.off_fix);
+  int* fix_counts = reinterpret_cast<int*>(sc + cg.off_fixcnt);
   // the status word must start at zero; the query-signature kernel restarts the other counters
   if ((e = cudaMemsetAsync(sc, 0, 256, st)) != cudaSuccess)
     return fail(nullptr, LASER_KV_ERR_CUDA, "collision_counts: memset: %s", cudaGetErrorString(e));
@@ -1542,7 +1540,7 @@ laser_kv_status_t laser_kv_collision_counts(const void* K_blk, const void* Q_win
     const int q_alloc = ((g.GW + 127) / 128) * 128;
     QsigArgs qa{static_cast<const uint16_t*>(Q_win), q_strides[0], q_strides[1], q_strides[2], P, hist, qb,
                 g.H_kv, g.G, g.W, g.GW, q_alloc, lsh_tables,
-                reinterpret_cast<uint4*>(counts_out), (long long)g.nseg * g.S / 4, ctrl + 1, ctrl};
+                reinterpret_cast<uint4*>(counts_out), (long long)g.nseg * g.S / 4, ctrl + 1, fix_counts, g.nseg, ctrl};
     dim3 grid(lsh_tables / kQsigTables, g.H_kv, g.batch);
     if ((e = launch_qsig(lsh_bits, mapQ, mapPq, qa, grid, qsig_smem_bytes(q_alloc, lsh_bits), st)) != cudaSuccess)
       return fail(nullptr, LASER_KV_ERR_CUDA, "collision_counts: qsig_kernel: %s", cudaGetErrorString(e));
@@ -1555,7 +1553,7 @@ laser_kv_status_t laser_kv_collision_counts(const void* K_blk, const void* Q_win
     sa.n_chunks = cg.n_chunks; sa.tables_per_chunk = cg.TC; sa.lsh_bits = lsh_bits; sa.lsh_tables = lsh_tables;
     sa.n_tiles = (long long)g.nseg * g.tiles_in_block * cg.n_chunks;
     sa.stat_rows = cg.TC * lsh_bits; sa.stat_rows_alloc = sa.stat_rows;
-    sa.counts = counts_out; sa.hist = hist; sa.fix_items = fix_items; sa.fix_count = ctrl + 1; sa.fix_cap = cg.fix_cap;
+    sa.counts = counts_out; sa.hist = hist; sa.fix_items = fix_items; sa.fix_count = fix_counts; sa.fix_cap = cg.fix_cap;
     sa.status = ctrl;
     sa.polls = kMaxPolls; sa.poll_ns = kPollHintNs;
     const uint32_t smem = stream_smem_bytes(kProj, sa.stat_rows_alloc, cg.TC * (2 << lsh_bits));
@@ -1564,8 +1562,8 @@ laser_kv_status_t laser_kv_collision_counts(const void* K_blk, const void* Q_win
   }
   {
     SignfixArgs fa{static_cast<const uint16_t*>(K_blk), kv_strides[0], kv_strides[1], kv_strides[2], P, hist, counts_out,
-                   nullptr, fix_items, ctrl + 1, cg.fix_cap, g.H_kv, g.nb, g.S, lsh_bits, lsh_tables, ctrl + 2, g.S};
-    signfix_kernel<<<kSignfixCtas, 256, 0, st>>>(fa);
+                   nullptr, fix_items, fix_counts, cg.fix_cap, g.H_kv, g.nb, g.S, lsh_bits, lsh_tables, ctrl + 2, g.S, ctrl + 1};
+    signfix_kernel<<<dim3(kSignfixCtasPerSeg, g.nseg), 256, 0, st>>>(fa);
     g_launches.fetch_add(1);
     if ((e = cudaGetLastError()) != cudaSuccess)
       return fail(nullptr, LASER_KV_ERR_CUDA, "collision_counts: signfix_kernel: %s", cudaGetErrorString(e));

@@ -16,10 +16,12 @@ __device__ __forceinline__ double bf16_to_f64(uint16_t b) {
 
 // ------------------------------------------------------------------------------------------------
 // Exact recomputation of flagged key signs. An item names a key, a table, the provisional bucket
-// code and a mask of the code bits whose projection was too small to trust. Eight lanes per item:
-// for every masked bit the 128-term dot product is formed in fp64 (exact bf16 products, sixteen
-// terms per lane, reduction over the eight lanes) and the bit is replaced by its exact sign. If the bucket code
-// changes, the key's count is corrected by hist[new] - hist[old].
+// code and a mask of the code bits whose projection was too small to trust. Every segment has its
+// own list. Eight lanes per item: for every masked bit the 128-term dot product is formed in fp64
+// (exact bf16 products, sixteen terms per lane, reduction over the eight lanes) and the bit is
+// replaced by its exact sign. If the bucket code changes, the key's count is corrected by
+// hist[new] - hist[old]. The selection kernel runs this for its own segment before it reads the
+// counts; the kernel below serves callers that want the counts alone.
 // ------------------------------------------------------------------------------------------------
 struct SignfixArgs {
   const uint16_t* Kp;     // keys via strides
@@ -28,31 +30,32 @@ struct SignfixArgs {
   const uint16_t* hist;
   uint32_t* counts;
   uint16_t* key_buckets;  // or nullptr
-  const int4* items;      // (segment, key, table, code | mask << 16)
-  const int* n_items;
+  const int4* items;      // [seg][cap]: (segment, key, table, code | mask << 16)
+  const int* n_items;     // [seg]
   int cap;
   int H_kv, nb, S, K, L;
   int* n_changed;
   int S_stride;           // tokens between the first keys of consecutive segments
+  int* n_total;           // sum of the list lengths (reporting)
 };
 
-constexpr int kSignfixCtas = 1184;   // 8 CTAs of 256 threads per SM: all resident, about one item per lane group
-
-__global__ void __launch_bounds__(256) signfix_kernel(const SignfixArgs a) {
+// The items of segment `seg`, taken by lane group `gid` of `ngroups` (a group = eight consecutive
+// lanes of a warp; all 32 lanes of the warp must call). `smem_counts`, when given, is the calling
+// CTA's copy of the segment's counts and receives the corrections as well.
+__device__ __forceinline__ void signfix_segment(const SignfixArgs& a, int seg, int gid, int ngroups, uint32_t* smem_counts) {
   const int lane = threadIdx.x & 31;
   const int sl = lane & 7;                              // lane within the group of eight that shares an item
   const uint32_t gmask = 0xFFu << (lane & 24);          // the group's lanes
-  const int gid = (blockIdx.x * blockDim.x + threadIdx.x) >> 3;
-  const int ngroups = (gridDim.x * blockDim.x) >> 3;
-  const int n = min(*a.n_items, a.cap);
+  const int n = min(a.n_items[seg], a.cap);
+  const int4* items = a.items + (size_t)seg * a.cap;
+  const int t = seg % a.nb;
+  const int h = (seg / a.nb) % a.H_kv;
+  const int b = seg / (a.nb * a.H_kv);
   for (int it = gid; it < n; it += ngroups) {
-    const int4 item = a.items[it];
-    const int seg = item.x, key = item.y, r = item.z;
+    const int4 item = items[it];
+    const int key = item.y, r = item.z;
     const uint32_t old_code = (uint32_t)item.w & 0xFFFFu;
     uint32_t mask = (uint32_t)item.w >> 16;
-    const int t = seg % a.nb;
-    const int h = (seg / a.nb) % a.H_kv;
-    const int b = seg / (a.nb * a.H_kv);
     // sixteen key elements per lane
     const uint16_t* krow = a.Kp + b * a.ks_b + h * a.ks_h + ((long long)t * a.S_stride + key) * a.ks_t + sl * 16;
     const uint4 ka = *reinterpret_cast<const uint4*>(krow), kb = *reinterpret_cast<const uint4*>(krow + 8);
@@ -79,10 +82,18 @@ __global__ void __launch_bounds__(256) signfix_kernel(const SignfixArgs a) {
       const uint16_t* hr = a.hist + ((size_t)(b * a.H_kv + h) * a.L + r) * ((size_t)1 << a.K);
       const uint32_t delta = (uint32_t)hr[code] - (uint32_t)hr[old_code];
       atomicAdd(a.counts + (size_t)seg * a.S + key, delta);
+      if (smem_counts) atomicAdd(smem_counts + key, delta);
       if (a.key_buckets) a.key_buckets[((size_t)seg * a.S + key) * a.L + r] = (uint16_t)code;
       atomicAdd(a.n_changed, 1);
     }
   }
+  if (gid == 0 && sl == 0) atomicAdd(a.n_total, a.n_items[seg]);
+}
+
+constexpr int kSignfixCtasPerSeg = 2;   // CTAs of 256 threads (32 lane groups each) per segment
+
+__global__ void __launch_bounds__(256) signfix_kernel(const SignfixArgs a) {
+  signfix_segment(a, blockIdx.y, (int)((blockIdx.x * blockDim.x + threadIdx.x) >> 3), (int)((gridDim.x * blockDim.x) >> 3), nullptr);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -209,6 +220,8 @@ struct SelectArgs {
   int excl_lo, excl_hi;                             // excluded range
   int cand_lo, cand_hi;                             // a range that contains every candidate
   int count_top_shift;      // highest byte position (0, 8, 16 or 24) in which two counts can differ
+  int has_fix;              // nonzero: `fix` names the segment lists of doubtful key signs to settle first
+  SignfixArgs fix;
 };
 
 __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectArgs a) {
@@ -230,6 +243,10 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_kernel(const SelectArgs
     flag[j] = kept ? 1 : ((j >= a.excl_lo && j < a.excl_hi) ? 2 : 0);
   }
   __syncthreads();
+  if (a.has_fix) {          // exact signs first: the corrections reach the shared-memory counts as well
+    signfix_segment(a.fix, seg, (int)(threadIdx.x >> 3), kSelThreads >> 3, ucnt);
+    __syncthreads();
+  }
   mark_topk(ukey, flag, lo, hi, a.k_exact, 24, hist, misc, warp_sums);            // K_exact
   mark_topk(ucnt, flag, lo, hi, a.k_lsh, a.count_top_shift, hist, misc, warp_sums);  // K_lsh from the residual
   // ordered compaction of all kept indices

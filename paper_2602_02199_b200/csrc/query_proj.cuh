@@ -33,6 +33,8 @@ struct QsigArgs {
   uint4* zero_begin;       // the call's collision counts, cleared here (16-byte units)
   long long zero_n;
   int* counters;           // fix-up and changed counters, restarted here
+  int* seg_counters;       // per-segment fix-up list lengths, restarted here
+  int n_seg_counters;
   int* status;
 };
 
@@ -118,6 +120,8 @@ qsig_kernel(const __grid_constant__ CUtensorMap map_q,    // Q: (d, W, H_q, batc
     const long long z0 = cta * per, z1 = min(a.zero_n, z0 + per);
     for (long long i = z0 + threadIdx.x; i < z1; i += kQsigThreads) a.zero_begin[i] = make_uint4(0u, 0u, 0u, 0u);
     if (cta == 0 && threadIdx.x < 2) a.counters[threadIdx.x] = 0;
+    if (cta == nctas - 1)
+      for (int i = threadIdx.x; i < a.n_seg_counters; i += kQsigThreads) a.seg_counters[i] = 0;
     for (uint32_t i = threadIdx.x; i < kQsigTables * nbins; i += kQsigThreads) bins[i] = 0;
   }
   __syncthreads();

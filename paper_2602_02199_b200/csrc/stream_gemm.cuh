@@ -82,9 +82,9 @@ struct StreamArgs {
   uint32_t* counts;        // [seg][S]
   const uint16_t* hist;    // [batch][H_kv][L][2^K]
   uint16_t* key_buckets;   // [seg][S][L] or nullptr
-  int4* fix_items;         // (seg, key, table, provisional bucket | doubtful bits << 16)
-  int* fix_count;
-  int fix_cap;
+  int4* fix_items;         // [seg][fix_cap]: (seg, key, table, provisional bucket | doubtful bits << 16)
+  int* fix_count;          // [seg]: items queued for the segment
+  int fix_cap;             // items a segment's list can hold
   int* status;
   uint32_t polls, poll_ns;     // budget of the hand-off waits: polls, and nanoseconds a poll may suspend
 };
@@ -238,8 +238,8 @@ __device__ __forceinline__ uint32_t proj_tables(uint32_t t_acc, uint32_t bar_rel
 #pragma unroll
         for (int k = 0; k < KBITS; ++k)
           if (!(fabsf(__uint_as_float(v[t * KBITS + k])) >= tau)) doubt |= 1u << (KBITS - 1 - k);
-        const int slot = atomicAdd(a.fix_count, 1);
-        if (slot < a.fix_cap) a.fix_items[slot] = make_int4(seg, key, r, (int)(code[t] | (doubt << 16)));
+        const int slot = atomicAdd(a.fix_count + seg, 1);
+        if (slot < a.fix_cap) a.fix_items[(size_t)seg * a.fix_cap + slot] = make_int4(seg, key, r, (int)(code[t] | (doubt << 16)));
         else record_status(a.status, kStatusCapacity);
       }
     }
