@@ -293,7 +293,7 @@ __device__ __forceinline__ uint4 ld_nc_v4(const void* p) {
   return v;
 }
 
-__global__ void __launch_bounds__(256) append_kernel(const AppendArgs a) {
+__global__ void __launch_bounds__(256, 8) append_kernel(const AppendArgs a) {
   const int seg = blockIdx.y;                      // (b*H_kv + h)*nb + t
   const int t = seg % a.nb;
   const int bh = seg / a.nb;
