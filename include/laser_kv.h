@@ -55,8 +55,8 @@ typedef struct {
   int32_t window;              /* W: observation-window queries per query head                   */
   int32_t max_blocks;          /* cache capacity per (layer, sequence, KV head) = max_blocks * B */
   int32_t max_blocks_per_call; /* upper bound on n_blocks of one select call (sizes workspace)   */
-  int32_t lsh_bits;            /* K: sign bits per SimHash table: 4, 6, 8, 10 or 12               */
-  int32_t lsh_tables;          /* L: tables (the paper's R hash rounds); a multiple of 8          */
+  int32_t lsh_bits;            /* K: sign bits per SimHash table, 1..12                           */
+  int32_t lsh_tables;          /* L: tables (the paper's R hash rounds), any positive number      */
   int32_t protection_divisor;  /* n >= 2 (Section 3.1)                                           */
   int32_t budget_per_block;    /* B; 0 => Eq. 1 from ratio, block_size and context_len           */
   int32_t debug;               /* nonzero: also keep per-key bucket ids for laser_kv_debug_view,
@@ -88,7 +88,13 @@ typedef struct {
 /* Intermediate results of the most recent select call (pointers into the workspace, valid
  * until the next select call). nb = that call's n_blocks; GW = G*W. A bucket code packs a table's
  * K sign bits with the table's first hyperplane as the most significant bit:
- * code = sum_b [<p_{r*K+b}, x> >= 0] << (K-1-b). hist is indexed by that code. */
+ * code = sum_b [<p_{r*K+b}, x> >= 0] << (K-1-b). hist is indexed by that code.
+ * The kernels work on an even number (>= 4) of bits per table and on tables in groups of eight;
+ * other shapes run on a padded copy of the hyperplanes kept in the workspace (a missing bit repeats
+ * the table's first hyperplane, so bucket equality is unchanged; a missing table repeats table 0
+ * with an empty query histogram, so it adds no collision). The arrays below have the padded shape:
+ * lsh_bits / lsh_tables of this struct are K' = even(max(K, 4)) and L' = 8*ceil(L/8), the first K
+ * bits (from the top) of a K'-bit code and the first L tables are the configured ones. */
 typedef struct {
   const float*    s_exact;       /* dev fp32  [batch][H_kv][nb][S]   summed window attention     */
   const uint32_t* counts;        /* dev u32   [batch][H_kv][nb][S]   collision counts            */

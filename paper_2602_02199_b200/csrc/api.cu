@@ -45,6 +45,7 @@ struct Derived {
   int B, anchors, k_exact, k_lsh, G, GW;
   int tiles_in_block;
   int TC, n_chunks;
+  int Kp, Lp;          // bits per table and tables as the kernels see them (padded, see derive)
   double alpha, ratio;
   float scale;
   int fix_cap;
@@ -54,7 +55,7 @@ struct Derived {
 };
 
 struct Carve {
-  size_t ctrl, dec_count, hist, qbuckets, lse_part, lse2, s_exact, counts, idx, fix_counts, fix_items, key_buckets, total;
+  size_t ctrl, dec_count, hist, qbuckets, lse_part, lse2, s_exact, counts, idx, fix_counts, fix_items, key_buckets, padP, total;
 };
 
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
@@ -194,14 +195,20 @@ laser_kv_status_t derive(const laser_kv_config_t* c, Derived* d) {
   if (d->GW % 16 || d->GW > 256 || c->window > 256 || d->G > 256)
     return fail(nullptr, LASER_KV_ERR_UNSUPPORTED,
                 "config: G*W = %d must be a multiple of 16 and at most 256", d->GW);
-  if (!(c->lsh_bits == 4 || c->lsh_bits == 6 || c->lsh_bits == 8 || c->lsh_bits == 10 || c->lsh_bits == 12))
-    return fail(nullptr, LASER_KV_ERR_UNSUPPORTED, "config: lsh_bits must be one of 4, 6, 8, 10, 12");
-  d->TC = pick_tc(c->lsh_bits, c->lsh_tables);
+  if (c->lsh_bits > 12)
+    return fail(nullptr, LASER_KV_ERR_UNSUPPORTED, "config: lsh_bits must be at most 12");
+  // The kernels take an even number (>= 4) of bits per table and tables in groups of eight. Other
+  // shapes run on a padded copy of the hyperplanes: a missing bit repeats the table's first
+  // hyperplane (both sides of a comparison get the same extra bit, so bucket equality is unchanged)
+  // and a missing table repeats table 0 with an all-zero query histogram (no collisions).
+  d->Kp = c->lsh_bits < 4 ? 4 : (c->lsh_bits + 1) / 2 * 2;
+  d->Lp = (c->lsh_tables + 7) / 8 * 8;
+  d->TC = pick_tc(d->Kp, d->Lp);
   if (!d->TC)
-    return fail(nullptr, LASER_KV_ERR_UNSUPPORTED, "config: lsh_tables must be a multiple of 8 (bits %d)", c->lsh_bits);
-  if ((long long)d->GW * c->lsh_tables > 0x7fffffffLL)
+    return fail(nullptr, LASER_KV_ERR_UNSUPPORTED, "config: no table chunking for %d bits x %d tables", c->lsh_bits, c->lsh_tables);
+  if ((long long)d->GW * d->Lp > 0x7fffffffLL)
     return fail(nullptr, LASER_KV_ERR_UNSUPPORTED, "config: G*W*lsh_tables too large");
-  d->n_chunks = c->lsh_tables / d->TC;
+  d->n_chunks = d->Lp / d->TC;
   d->tiles_in_block = (c->block_size + kTileKeys - 1) / kTileKeys;
   if (c->softmax_scale < 0.f || c->softmax_scale != c->softmax_scale)
     return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "config: softmax_scale must be positive (0 selects 1/sqrt(head_dim))");
@@ -215,7 +222,7 @@ laser_kv_status_t derive(const laser_kv_config_t* c, Derived* d) {
   // with look-back a segment is the previous block's held-back tail followed by the block
   d->S_ws = c->block_size + (c->lookback ? d->anchors : 0);
   // exact-sign work list of a segment: about 5e-4 of its (key, table) pairs are expected
-  long long fc = d->S_ws * (long long)c->lsh_tables / 256;
+  long long fc = d->S_ws * (long long)d->Lp / 256;
   if (fc < 256) fc = 256;
   if (fc > (1 << 22)) fc = 1 << 22;
   d->fix_cap = (int)fc;
@@ -229,8 +236,8 @@ void carve_ws(const laser_kv_config_t* c, const Derived& d, Carve* v) {
   const size_t bh = (size_t)c->batch * c->n_kv_heads;
   v->ctrl = take(256);
   v->dec_count = take(bh * 4);        // finished decode splits per (sequence, KV head)
-  v->hist = take(bh * c->lsh_tables * ((size_t)2 << c->lsh_bits));
-  v->qbuckets = take(bh * d.GW * c->lsh_tables * 2);
+  v->hist = take(bh * d.Lp * ((size_t)2 << d.Kp));
+  v->qbuckets = take(bh * d.GW * d.Lp * 2);
   v->lse_part = take(lse_part_bytes_bound(nseg, d.GW));
   v->lse2 = take(nseg * d.GW * 4);
   v->s_exact = take(nseg * S * 4);
@@ -238,7 +245,8 @@ void carve_ws(const laser_kv_config_t* c, const Derived& d, Carve* v) {
   v->idx = take(nseg * (size_t)(d.B > 0 ? d.B : 1) * 4);
   v->fix_counts = take(nseg * sizeof(int));
   v->fix_items = take(nseg * (size_t)d.fix_cap * sizeof(int4));
-  v->key_buckets = take(c->debug ? nseg * S * c->lsh_tables * 2 : 0);
+  v->key_buckets = take(c->debug ? nseg * S * d.Lp * 2 : 0);
+  v->padP = take((d.Kp != c->lsh_bits || d.Lp != c->lsh_tables) ? (size_t)d.Kp * d.Lp * kHeadDim * 2 : 0);
   v->total = off;
 }
 
@@ -472,11 +480,29 @@ laser_kv_status_t laser_kv_init(const laser_kv_config_t* cfg, const void* hyperp
   h->lookback_done.assign(cfg->n_layers, 0);
   h->budget.assign(cfg->n_layers, laser_kv_ctx::LayerBudget{d.B, d.anchors, d.k_exact, d.k_lsh});
   h->last_B = d.B;
+  if ((d.Kp != cfg->lsh_bits || d.Lp != cfg->lsh_tables)) {
+    // padded copy of the hyperplanes in the workspace (see derive): real bits, then repeats of the
+    // table's first hyperplane, then repeats of (padded) table 0
+    const size_t row = (size_t)kHeadDim * 2;
+    uint8_t* dst = h->ws + v.padP;
+    const uint8_t* src = static_cast<const uint8_t*>(hyperplanes);
+    const int K = cfg->lsh_bits, L = cfg->lsh_tables;
+    e = cudaMemcpy2D(dst, (size_t)d.Kp * row, src, (size_t)K * row, (size_t)K * row, (size_t)L, cudaMemcpyDeviceToDevice);
+    for (int b = K; b < d.Kp && e == cudaSuccess; ++b)
+      e = cudaMemcpy2D(dst + (size_t)b * row, (size_t)d.Kp * row, src, (size_t)K * row, row, (size_t)L, cudaMemcpyDeviceToDevice);
+    for (int r = L; r < d.Lp && e == cudaSuccess; ++r)
+      e = cudaMemcpy(dst + (size_t)r * d.Kp * row, dst, (size_t)d.Kp * row, cudaMemcpyDeviceToDevice);
+    if (e != cudaSuccess) {
+      delete h;
+      return fail(nullptr, LASER_KV_ERR_CUDA, "init: padded hyperplane copy: %s", cudaGetErrorString(e));
+    }
+    h->P = reinterpret_cast<const uint16_t*>(dst);
+  }
   {
-    const uint64_t dims[2] = {(uint64_t)kHeadDim, (uint64_t)cfg->lsh_tables * cfg->lsh_bits};
+    const uint64_t dims[2] = {(uint64_t)kHeadDim, (uint64_t)d.Lp * d.Kp};
     const uint64_t strides[1] = {(uint64_t)kHeadDim * 2};
-    const uint32_t box[2] = {(uint32_t)kAtomCols, (uint32_t)(d.TC * cfg->lsh_bits)};
-    const uint32_t boxq[2] = {(uint32_t)kAtomCols, (uint32_t)(kQsigTables * cfg->lsh_bits)};
+    const uint32_t box[2] = {(uint32_t)kAtomCols, (uint32_t)(d.TC * d.Kp)};
+    const uint32_t boxq[2] = {(uint32_t)kAtomCols, (uint32_t)(kQsigTables * d.Kp)};
     if (!encode_map(h, &h->mapP, h->P, 2, dims, strides, box) || !encode_map(h, &h->mapPq, h->P, 2, dims, strides, boxq)) {
       const std::string msg = h->last_error;
       delete h;
@@ -620,10 +646,11 @@ laser_kv_status_t run_select(laser_kv_ctx* h, int layer, const void* K_blk, cons
   if (need_lsh) {
     const int q_alloc = ((d.GW + 127) / 128) * 128;
     QsigArgs qa{static_cast<const uint16_t*>(Q_win), q_strides[0], q_strides[1], q_strides[2], h->P, hist, qb,
-                c.n_kv_heads, d.G, c.window, d.GW, q_alloc, c.lsh_tables,
-                reinterpret_cast<uint4*>(counts), ((long long)nseg * S_len + 3) / 4, ctrl + 1, fix_counts, nseg, ctrl};
-    dim3 grid(c.lsh_tables / kQsigTables, c.n_kv_heads, c.batch);
-    LKV_CUDA(launch_qsig(c.lsh_bits, mapQ, h->mapPq, qa, grid, qsig_smem_bytes(q_alloc, c.lsh_bits), st), "qsig_kernel");
+                c.n_kv_heads, d.G, c.window, d.GW, q_alloc, d.Lp,
+                reinterpret_cast<uint4*>(counts), ((long long)nseg * S_len + 3) / 4, ctrl + 1, fix_counts, nseg, ctrl,
+                c.lsh_tables};
+    dim3 grid(d.Lp / kQsigTables, c.n_kv_heads, c.batch);
+    LKV_CUDA(launch_qsig(d.Kp, mapQ, h->mapPq, qa, grid, qsig_smem_bytes(q_alloc, d.Kp), st), "qsig_kernel");
   }
 
   StreamArgs sa;
@@ -634,7 +661,7 @@ laser_kv_status_t run_select(laser_kv_ctx* h, int layer, const void* K_blk, cons
   const long long seg_tiles = (long long)nseg * tiles_in_block;
   const int base_ctas = stream_grid(seg_tiles, h->num_sms);
   sa.n_tiles = seg_tiles; sa.lse_ctas = base_ctas; sa.n_slot = lse_slots(base_ctas, nseg);
-  sa.n_chunks = d.n_chunks; sa.tables_per_chunk = d.TC; sa.lsh_bits = c.lsh_bits; sa.lsh_tables = c.lsh_tables;
+  sa.n_chunks = d.n_chunks; sa.tables_per_chunk = d.TC; sa.lsh_bits = d.Kp; sa.lsh_tables = d.Lp;
   sa.scale_log2e = d.scale * 1.4426950408889634f;
   sa.lse_part = lse_part; sa.lse2 = lse2; sa.s_exact = s_exact; sa.counts = counts; sa.hist = hist;
   sa.key_buckets = key_buckets; sa.fix_items = fix_items; sa.fix_count = fix_counts; sa.fix_cap = d.fix_cap;
@@ -664,11 +691,11 @@ laser_kv_status_t run_select(laser_kv_ctx* h, int layer, const void* K_blk, cons
   // 4. key signatures and collision counts
   if (need_lsh) {
     StreamArgs a3 = sa;
-    a3.stat_rows = d.TC * c.lsh_bits;
+    a3.stat_rows = d.TC * d.Kp;
     a3.stat_rows_alloc = a3.stat_rows;
     a3.n_tiles = seg_tiles * d.n_chunks;
-    const uint32_t smem = stream_smem_bytes(kProj, a3.stat_rows_alloc, d.TC * (2 << c.lsh_bits));
-    LKV_CUDA(launch_proj(c.lsh_bits, d.TC, mapK, h->mapP, a3, stream_grid(a3.n_tiles, h->num_sms), smem, st),
+    const uint32_t smem = stream_smem_bytes(kProj, a3.stat_rows_alloc, d.TC * (2 << d.Kp));
+    LKV_CUDA(launch_proj(d.Kp, d.TC, mapK, h->mapP, a3, stream_grid(a3.n_tiles, h->num_sms), smem, st),
              "projection pass");
   }
   mark();
@@ -678,8 +705,8 @@ laser_kv_status_t run_select(laser_kv_ctx* h, int layer, const void* K_blk, cons
     SelectArgs sel{s_exact, counts, idx, S_len, g.k_exact, g.k_lsh, g.keep_a_lo, g.keep_a_hi, g.keep_b_lo, g.keep_b_hi,
                    g.excl_lo, g.excl_hi, g.cand_lo, g.cand_hi, 0, need_lsh ? 1 : 0,
                    SignfixArgs{K0, kv_strides[0], kv_strides[1], kv_strides[2], h->P, hist, counts, key_buckets, fix_items,
-                               fix_counts, d.fix_cap, c.n_kv_heads, nb, S_len, c.lsh_bits, c.lsh_tables, ctrl + 2, S, ctrl + 1}};
-    const laser_kv_status_t s = launch_select(sel, nseg, (uint32_t)d.GW * (uint32_t)c.lsh_tables, st);
+                               fix_counts, d.fix_cap, c.n_kv_heads, nb, S_len, d.Kp, d.Lp, ctrl + 2, S, ctrl + 1}};
+    const laser_kv_status_t s = launch_select(sel, nseg, (uint32_t)d.GW * (uint32_t)d.Lp, st);
     if (s != LASER_KV_OK) { h->last_error = g_last_error; return s; }
   }
   mark();
@@ -1067,8 +1094,8 @@ laser_kv_status_t laser_kv_debug_view(laser_kv_handle_t h, laser_kv_debug_t* out
   out->segment_shift = h->last_shift;
   out->budget = h->last_B;
   out->gw = h->d.GW;
-  out->lsh_tables = c.lsh_tables;
-  out->lsh_bits = c.lsh_bits;
+  out->lsh_tables = h->d.Lp;
+  out->lsh_bits = h->d.Kp;
   out->n_sign_fixups = h->last_fixups;
   return LASER_KV_OK;
 }
@@ -1540,7 +1567,8 @@ laser_kv_status_t laser_kv_collision_counts(const void* K_blk, const void* Q_win
     const int q_alloc = ((g.GW + 127) / 128) * 128;
     QsigArgs qa{static_cast<const uint16_t*>(Q_win), q_strides[0], q_strides[1], q_strides[2], P, hist, qb,
                 g.H_kv, g.G, g.W, g.GW, q_alloc, lsh_tables,
-                reinterpret_cast<uint4*>(counts_out), (long long)g.nseg * g.S / 4, ctrl + 1, fix_counts, g.nseg, ctrl};
+                reinterpret_cast<uint4*>(counts_out), (long long)g.nseg * g.S / 4, ctrl + 1, fix_counts, g.nseg, ctrl,
+                lsh_tables};
     dim3 grid(lsh_tables / kQsigTables, g.H_kv, g.batch);
     if ((e = launch_qsig(lsh_bits, mapQ, mapPq, qa, grid, qsig_smem_bytes(q_alloc, lsh_bits), st)) != cudaSuccess)
       return fail(nullptr, LASER_KV_ERR_CUDA, "collision_counts: qsig_kernel: %s", cudaGetErrorString(e));

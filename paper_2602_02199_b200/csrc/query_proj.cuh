@@ -36,6 +36,7 @@ struct QsigArgs {
   int* seg_counters;       // per-segment fix-up list lengths, restarted here
   int n_seg_counters;
   int* status;
+  int n_real_tables;       // tables from this index on are padding: their histograms stay empty
 };
 
 // <x, y> over 128 bf16 elements in fp64 (every product is exact); 16-byte loads, all in flight at once.
@@ -184,7 +185,7 @@ qsig_kernel(const __grid_constant__ CUtensorMap map_q,    // Q: (d, W, H_q, batc
           code = (code & ~(1u << pos)) | ((exact_dot128(row, plane) >= 0.0 ? 1u : 0u) << pos);
         }
         codes[t] = code;
-        atomicAdd(&bins[t * nbins + code], 1u);
+        if (tg * kQsigTables + t < a.n_real_tables) atomicAdd(&bins[t * nbins + code], 1u);
       }
       // eight consecutive tables: one 16-byte store (L is a multiple of 8)
       uint4 packed;

@@ -42,7 +42,10 @@ def check_signatures(codes_gpu: np.ndarray, x_bits: np.ndarray, p_bits: np.ndarr
     the oracle's convention and the number of exempted bit differences."""
     proj = O.simhash_projections(x_bits, p_bits).reshape(x_bits.shape[0], n_tables, n_bits)
     want = (proj >= 0.0).astype(np.int64)
-    got = codes_to_bits(codes_gpu, n_bits)
+    # the library pads a table to an even number (>= 4) of bits and the tables to a multiple of eight:
+    # a code has code_bits = even(max(n_bits, 4)) bits of which the first n_bits are the table's own
+    code_bits = max(4, (n_bits + 1) // 2 * 2)
+    got = codes_to_bits(codes_gpu[:, :n_tables], code_bits)[..., :n_bits]
     diff = got != want
     bad = diff & (np.abs(proj) >= SIGN_EXEMPT)
     assert not bad.any(), f"{what}: {int(bad.sum())} signature bits differ outside |proj| < 1e-6 " \

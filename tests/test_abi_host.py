@@ -58,8 +58,8 @@ def test_query_sizes_and_validation():
     assert cb >= 2 * 8 * 4 * 409 * 516 and cb < 2 * 8 * 4 * 409 * 516 + 4096
     assert wb > 0 and wb % 256 == 0
     for bad, status in ((dict(head_dim=64), B.ERR_UNSUPPORTED), (dict(protection_divisor=1), B.ERR_INVALID_ARG),
-                        (dict(n_q_heads=30), B.ERR_INVALID_ARG), (dict(lsh_bits=7), B.ERR_UNSUPPORTED),
-                        (dict(lsh_tables=12), B.ERR_UNSUPPORTED), (dict(window=100), B.ERR_UNSUPPORTED),
+                        (dict(n_q_heads=30), B.ERR_INVALID_ARG), (dict(lsh_bits=13), B.ERR_UNSUPPORTED),
+                        (dict(window=100), B.ERR_UNSUPPORTED),
                         (dict(budget_per_block=2000), B.ERR_INVALID_ARG), (dict(alpha=1.5), B.ERR_INVALID_ARG),
                         (dict(block_size=1001), B.ERR_UNSUPPORTED), (dict(context_len=0), B.ERR_INVALID_ARG)):
         with pytest.raises(B.LaserKVError) as e:

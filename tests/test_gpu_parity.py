@@ -49,6 +49,11 @@ def test_gqa7_k10_shape_with_rope_and_batch():
     (12, 16, 4, 4, 32, 136),     # 12-bit tables in one chunk of 16: two accumulator buffers of 192 columns
     (8, 32, 6, 2, 48, 648),      # G*W = 144: two query row blocks, the second one ragged; chunk of 32 tables
     (10, 8, 16, 2, 16, 1032),    # G = 8, W = 16
+    (7, 12, 4, 2, 32, 392),      # odd bits (padded to 8 with a repeat of the first hyperplane), 12 tables (padded to 16)
+    (5, 3, 8, 2, 16, 264),       # 5 bits -> 6, 3 tables -> 8
+    (1, 20, 4, 4, 16, 136),      # one bit per table -> 4, 20 tables -> 24
+    (11, 9, 4, 2, 64, 520),      # 11 bits -> 12, 9 tables -> 16
+    (9, 64, 8, 2, 32, 648),      # 9 bits -> 10, tables already a multiple of eight
 ])
 def test_hash_and_group_geometries(K, L, hq, hkv, W, S):
     w = synth.workload("tiny").with_(name=f"geo{K}_{L}_{hq}_{hkv}_{W}", n_q_heads=hq, n_kv_heads=hkv, window=W,

@@ -37,6 +37,23 @@ def test_select_call_on_random_geometries(seed):
         check_run(w, run, segments=segs)
 
 
+@pytest.mark.parametrize("seed", [31, 32])
+def test_select_call_on_random_hash_shapes(seed):
+    """Any number of bits per table up to 12 and any number of tables (the library pads inside)."""
+    rng = np.random.default_rng(seed)
+    for case in range(8):
+        G, W = _group_and_window(rng)
+        hkv = int(rng.choice([1, 2]))
+        S, nb = int(rng.integers(8, 120)) * 8, int(rng.integers(1, 3))
+        w = synth.workload("tiny").with_(
+            name=f"hash{seed}_{case}", n_q_heads=hkv * G, n_kv_heads=hkv, window=W,
+            lsh_bits=int(rng.integers(1, 13)), lsh_tables=int(rng.integers(1, 41)), block_size=S,
+            context_len=nb * S, protection_divisor=int(rng.choice([2, 4, 8])),
+            alpha=float(rng.choice([0.0, 0.5, 0.75])), needles="uniform:2")
+        run = run_workload_layer(w, 0)
+        check_run(w, run, segments=[(0, int(rng.integers(hkv)), int(rng.integers(nb)))])
+
+
 @pytest.mark.parametrize("seed", [21, 22])
 def test_decode_and_closed_form_score_on_random_geometries(seed):
     import torch
