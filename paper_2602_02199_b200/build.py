@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "liblaserkv.so")
 SOURCES = ["api.cu"]
-HEADERS = ["ptx.cuh", "stream_gemm.cuh", "aux_kernels.cuh", "query_proj.cuh", "decode_attn.cuh", "theory_score.cuh"]
+HEADERS = ["ptx.cuh", "theory_math.cuh", "stream_gemm.cuh", "aux_kernels.cuh", "query_proj.cuh", "decode_attn.cuh"]
 
 
 def _nvcc() -> str:

@@ -1,4 +1,4 @@
-"""Prints the coefficients used by theory_score.cuh: a degree-7 polynomial P with
+"""Prints the coefficients used by theory_math.cuh: a degree-7 polynomial P with
 acos(x) ~= sqrt(1 - x) * P(x) on [0, 1] (the form of Abramowitz & Stegun 4.4.46), fitted here by
 interpolation at Chebyshev nodes followed by a few Remez-style exchange steps, in float64.
 

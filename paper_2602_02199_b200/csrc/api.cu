@@ -19,7 +19,6 @@
 #include "stream_gemm.cuh"
 #include "query_proj.cuh"
 #include "decode_attn.cuh"
-#include "theory_score.cuh"
 
 namespace {
 
@@ -363,15 +362,6 @@ laser_kv_status_t launch_append(const AppendArgs& a, int n_seg, cudaStream_t st)
   return LASER_KV_OK;
 }
 
-
-template <int KB>
-cudaError_t launch_theory(const CUtensorMap& mk, const CUtensorMap& mq, const TheoryArgs& a, dim3 grid, cudaStream_t st) {
-  static std::atomic<unsigned long long> limit_set{0};   // per instantiation
-  const cudaError_t e = ensure_smem_limit(limit_set, theory_kernel<KB>, (int)theory_smem_bytes(kThMaxQueries));
-  if (e != cudaSuccess) return e;
-  theory_kernel<KB><<<grid, kThThreads, theory_smem_bytes(a.GW), st>>>(mk, mq, a);
-  return cudaGetLastError();
-}
 
 // Splits per (sequence, KV head) of a decode call: as many as fill the GPU's resident CTAs once,
 // never more than tiles in the cache.
@@ -1611,7 +1601,7 @@ laser_kv_status_t laser_kv_collision_probability(const void* K_blk, const void* 
   if (n_q_heads % n_kv_heads) return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "collision_probability: n_q_heads %% n_kv_heads != 0");
   if (lsh_bits < 1 || lsh_bits > 64) return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "collision_probability: lsh_bits must be in [1, 64]");
   const int G = n_q_heads / n_kv_heads, GW = G * window;
-  if (GW % 16 || GW > kThMaxQueries || window > 256 || G > 256 || block_size % 8)
+  if (GW % 16 || GW > 256 || window > 256 || G > 256 || block_size % 8)
     return fail(nullptr, LASER_KV_ERR_UNSUPPORTED,
                 "collision_probability: G*W must be a multiple of 16, at most 256; block_size a multiple of 8");
   if ((long long)n_blocks * block_size > 0x7fffffffLL || (long long)n_kv_heads * n_blocks > 65535 || batch > 65535)
@@ -1628,51 +1618,53 @@ laser_kv_status_t laser_kv_collision_probability(const void* K_blk, const void* 
   EncodeTiledFn enc = driver_encode_fn();
   if (!enc) return fail(nullptr, LASER_KV_ERR_CUDA, "collision_probability: cuTensorMapEncodeTiled not available (no CUDA driver?)");
   CUtensorMap mapK, mapQ;
-  const cuuint32_t ones[4] = {1, 1, 1, 1};
   {
     const cuuint64_t s_tok = (cuuint64_t)kv_strides[2];
     const cuuint64_t s_head = kv_strides[1] > 0 ? (cuuint64_t)kv_strides[1] : s_tok * (cuuint64_t)n_blocks * block_size;
     const cuuint64_t s_batch = kv_strides[0] > 0 ? (cuuint64_t)kv_strides[0] : s_head * (cuuint64_t)n_kv_heads;
     const cuuint64_t dims[4] = {(cuuint64_t)kHeadDim, (cuuint64_t)n_blocks * block_size, (cuuint64_t)n_kv_heads, (cuuint64_t)batch};
     const cuuint64_t strides[3] = {s_tok * 2, s_head * 2, s_batch * 2};
-    const cuuint32_t box[4] = {64, (cuuint32_t)kThTile, 1, 1};
-    const CUresult r = enc(&mapK, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(K_blk), dims, strides, box, ones,
-                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return fail(nullptr, LASER_KV_ERR_CUDA, "collision_probability: tensor map of K failed (CUresult %d)", (int)r);
-  }
-  {
+    const cuuint32_t box[4] = {(cuuint32_t)kAtomCols, (cuuint32_t)kTileKeys, 1, 1};
     const cuuint64_t s_w = (cuuint64_t)q_strides[2];
-    const cuuint64_t s_head = q_strides[1] > 0 ? (cuuint64_t)q_strides[1] : s_w * (cuuint64_t)window;
-    const cuuint64_t s_batch = q_strides[0] > 0 ? (cuuint64_t)q_strides[0] : s_head * (cuuint64_t)n_q_heads;
-    const cuuint64_t dims[4] = {(cuuint64_t)kHeadDim, (cuuint64_t)window, (cuuint64_t)n_q_heads, (cuuint64_t)batch};
-    const cuuint64_t strides[3] = {s_w * 2, s_head * 2, s_batch * 2};
-    const cuuint32_t box[4] = {64, (cuuint32_t)window, (cuuint32_t)G, 1};
-    const CUresult r = enc(&mapQ, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(Q_win), dims, strides, box, ones,
-                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return fail(nullptr, LASER_KV_ERR_CUDA, "collision_probability: tensor map of Q failed (CUresult %d)", (int)r);
+    const cuuint64_t q_head = q_strides[1] > 0 ? (cuuint64_t)q_strides[1] : s_w * (cuuint64_t)window;
+    const cuuint64_t q_batch = q_strides[0] > 0 ? (cuuint64_t)q_strides[0] : q_head * (cuuint64_t)n_q_heads;
+    const cuuint64_t qdims[4] = {(cuuint64_t)kHeadDim, (cuuint64_t)window, (cuuint64_t)n_q_heads, (cuuint64_t)batch};
+    const cuuint64_t qstrides[3] = {s_w * 2, q_head * 2, q_batch * 2};
+    const cuuint32_t qbox[4] = {(cuuint32_t)kAtomCols, (cuuint32_t)window, (cuuint32_t)G, 1};
+    if (!encode_bf16_map(enc, &mapK, K_blk, 4, dims, strides, box) || !encode_bf16_map(enc, &mapQ, Q_win, 4, qdims, qstrides, qbox))
+      return fail(nullptr, LASER_KV_ERR_CUDA, "collision_probability: cuTensorMapEncodeTiled failed");
   }
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   cudaError_t e;
   if ((e = cudaMemsetAsync(scratch, 0, 256, st)) != cudaSuccess)
     return fail(nullptr, LASER_KV_ERR_CUDA, "collision_probability: memset: %s", cudaGetErrorString(e));
-  TheoryArgs a;
-  a.out = p_out;
-  a.S = block_size; a.nb = n_blocks; a.H_kv = n_kv_heads; a.G = G; a.GW = GW; a.kbits = lsh_bits;
-  a.tiles_in_block = (block_size + kThTile - 1) / kThTile;
-  a.status = static_cast<int*>(scratch);
-  const dim3 grid((unsigned)((a.tiles_in_block + kThTilesPerCta - 1) / kThTilesPerCta), (unsigned)(n_kv_heads * n_blocks), (unsigned)batch);
+  int dev = 0, num_sms = 0;
+  if ((e = cudaGetDevice(&dev)) != cudaSuccess ||
+      (e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess)
+    return fail(nullptr, LASER_KV_ERR_CUDA, "collision_probability: device query: %s", cudaGetErrorString(e));
+  StreamArgs sa;
+  memset(&sa, 0, sizeof sa);
+  sa.S = block_size; sa.S_stride = block_size; sa.nb = n_blocks; sa.H_kv = n_kv_heads; sa.batch = batch;
+  sa.G = G; sa.W = window; sa.GW = GW;
+  sa.tiles_in_block = (block_size + kTileKeys - 1) / kTileKeys;
+  sa.nseg = batch * n_kv_heads * n_blocks;
+  sa.n_tiles = (long long)sa.nseg * sa.tiles_in_block;
+  sa.stat_rows = GW; sa.stat_rows_alloc = GW;
+  sa.lsh_bits = lsh_bits;
+  sa.s_exact = p_out;
+  sa.status = static_cast<int*>(scratch);
+  sa.polls = kMaxPolls; sa.poll_ns = kPollHintNs;
+  const int ctas = stream_grid(sa.n_tiles, num_sms);
+  const uint32_t smem = stream_smem_bytes(kTheory, sa.stat_rows_alloc, 0);
   switch (lsh_bits) {                    // the usual table widths get the multiplication form of u^K
-    case 4: e = launch_theory<4>(mapK, mapQ, a, grid, st); break;
-    case 6: e = launch_theory<6>(mapK, mapQ, a, grid, st); break;
-    case 8: e = launch_theory<8>(mapK, mapQ, a, grid, st); break;
-    case 10: e = launch_theory<10>(mapK, mapQ, a, grid, st); break;
-    case 12: e = launch_theory<12>(mapK, mapQ, a, grid, st); break;
-    default: e = launch_theory<0>(mapK, mapQ, a, grid, st); break;
+    case 4: e = launch_stream<kTheory, 4, 0>(mapK, mapQ, sa, ctas, smem, st); break;
+    case 6: e = launch_stream<kTheory, 6, 0>(mapK, mapQ, sa, ctas, smem, st); break;
+    case 8: e = launch_stream<kTheory, 8, 0>(mapK, mapQ, sa, ctas, smem, st); break;
+    case 10: e = launch_stream<kTheory, 10, 0>(mapK, mapQ, sa, ctas, smem, st); break;
+    case 12: e = launch_stream<kTheory, 12, 0>(mapK, mapQ, sa, ctas, smem, st); break;
+    default: e = launch_stream<kTheory, 0, 0>(mapK, mapQ, sa, ctas, smem, st); break;
   }
-  g_launches.fetch_add(1);
-  if (e != cudaSuccess) return fail(nullptr, LASER_KV_ERR_CUDA, "theory_kernel launch: %s", cudaGetErrorString(e));
+  if (e != cudaSuccess) return fail(nullptr, LASER_KV_ERR_CUDA, "collision_probability: launch: %s", cudaGetErrorString(e));
   return LASER_KV_OK;
 }
 

@@ -18,6 +18,10 @@
 //            window queries per bucket) and adds the collisions to count[key]. Signs decided by
 //            a projection that is tiny relative to the key's other projections are queued for
 //            an exact recomputation.
+//   kTheory: D[key][query] as kScore; instead of softmax weights the epilogue turns every inner
+//            product into the cosine of the angle between query and key (key norms from the tile
+//            in shared memory, query norms from the stationary operand) and sums the closed-form
+//            collision probability (1 - theta/pi)^K over the queries.
 //
 // Warp roles (608 threads): warp 0 = TMA producer, warps 1 and 2 = MMA issuers (warp 1 also owns
 // the TMEM allocation), warps 3..18 = four epilogue groups of four warps (TMEM lane quarter =
@@ -29,6 +33,7 @@
 // inside the tile loop.
 #pragma once
 #include "ptx.cuh"
+#include "theory_math.cuh"
 
 namespace lkv {
 
@@ -43,6 +48,7 @@ constexpr int kMmaWarps = 2;
 constexpr int kStreamThreads = 32 * (1 + kMmaWarps) + kEpilogueThreads;
 constexpr int kEpiCols = 64;                   // accumulator columns an epilogue thread holds at most
 constexpr int kXchBytes = 8192;                // exchange area between epilogue warps
+constexpr int kXchTheoryBytes = 12288;         // kTheory adds the key-norm partials [2][4 groups][128 keys]
 constexpr int kTmemCols = 512;
 constexpr int kAccStride = 256;                // TMEM columns per accumulator buffer (kLse, kScore: two buffers)
 constexpr int kMaxAcc = 4;                     // most accumulator buffers of any mode
@@ -55,7 +61,7 @@ __host__ __device__ constexpr int proj_num_acc(int kbits, int tc) {
 constexpr int kMaxStreamCtas = 256;            // upper bound of the persistent grid (slot arithmetic)
 constexpr int kPolyPairsOf32 = 10;             // of every 32 column pairs, this many take 2^x on the FMA pipe
 
-enum StreamMode { kLse = 0, kScore = 1, kProj = 2 };
+enum StreamMode { kLse = 0, kScore = 1, kProj = 2, kTheory = 3 };
 
 enum : int { kStatusOk = 0, kStatusCapacity = 3, kStatusTimeout = 6 };
 
@@ -256,6 +262,10 @@ struct EpiCtx {
   uint32_t bar_tfull, bar_tempty, bar_stat, bar_stat_free, bar_xa, bar_xb;
   uint8_t* xch_s;              // exchange area
   const uint16_t* hist_s;      // histogram slice (kProj)
+  uint32_t bar_full, bar_empty, bar_kn;   // kTheory: the epilogue reads the key tile itself
+  const uint8_t* stat_s;       // stationary operand, generic pointer (kTheory: query norms)
+  const uint8_t* stages_s;     // key-tile ring, generic pointer
+  uint32_t stat_atom_bytes;
 };
 
 // A run: the tiles of one block segment that fall inside the CTA's slice. The epilogue loops walk
@@ -451,11 +461,122 @@ __device__ __forceinline__ bool proj_epilogue(const StreamArgs& a, const EpiCtx&
   return true;
 }
 
+// Sum of squares of the bf16 elements of 16-byte chunks [c_begin, c_begin + n) of row `row` of an
+// operand stored as two 64-column halves (`half_bytes` apart) of 128-byte rows with the 128-byte
+// swizzle (8-row groups 1024 bytes apart).
+__device__ __forceinline__ float row_sum_squares(const uint8_t* op, uint32_t half_bytes, int row, int c_begin, int n) {
+  float s2 = 0.f;
+  const uint8_t* r = op + (uint32_t)(row >> 3) * 1024u + (uint32_t)(row & 7) * 128u;
+  for (int c16 = c_begin; c16 < c_begin + n; ++c16) {
+    const uint4 w = *reinterpret_cast<const uint4*>(r + (uint32_t)(c16 >> 3) * half_bytes + (uint32_t)(((c16 & 7) ^ (row & 7)) << 4));
+    const uint32_t v[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float lo = __uint_as_float(v[i] << 16), hi = __uint_as_float(v[i] & 0xFFFF0000u);
+      s2 = fmaf(lo, lo, s2);
+      s2 = fmaf(hi, hi, s2);
+    }
+  }
+  return s2;
+}
+
+// kTheory: NC query columns [c0, c0 + NC) per thread; KB sign bits per table (0: any number, taken
+// from the arguments at run time). The four groups each square-sum a quarter of every key row of
+// the tile (the stage is released by the MMAs' commit and by the sixteen epilogue warps), the
+// groups' sums of the collision probabilities meet in group 0 as in the score pass.
+template <int NC, int KB>
+__device__ __forceinline__ bool theory_epilogue(const StreamArgs& a, const EpiCtx& e, int c0) {
+  float* rqw = reinterpret_cast<float*>(e.xch_s) + e.ewarp * kEpiCols;       // this warp's 1/|q| values
+  float* part = reinterpret_cast<float*>(e.xch_s + 16 * kEpiCols * 4);       // [2 acc][3 groups][128 keys]
+  float* kn = reinterpret_cast<float*>(e.xch_s + 16 * kEpiCols * 4 + 2 * 3 * 128 * 4);   // [2][4 groups][128 keys]
+  const float kbits = (float)a.lsh_bits, inv_gw = 1.0f / (float)a.GW;
+  bool new_group = true;
+  uint32_t gen = 0, it = 0;
+  for (long long x = e.x_begin; x < e.x_end;) {
+    const TileRun r = run_at(x, e.x_end, a);
+    if (new_group) {
+      // the head's window queries landed: 1 / |q| of this warp's columns
+      if (!mbar_wait(e.bar_stat, gen & 1, a.polls, a.poll_ns)) return false;
+      ++gen;
+      __syncwarp();
+      if constexpr (NC > 0) {
+#pragma unroll
+        for (int half = 0; half < (NC + 31) / 32; ++half) {
+          const int j = e.lane + 32 * half;
+          if (j < NC) {
+            const float n2 = row_sum_squares(e.stat_s, e.stat_atom_bytes, c0 + j, 0, 16);
+            rqw[j] = n2 > 0.f ? 1.0f / sqrtf(n2) : 0.f;      // correctly rounded: acos is ill-conditioned at |cos| = 1
+          }
+        }
+      }
+      __syncwarp();
+    }
+    float* out = a.s_exact + (size_t)r.c.seg * a.S;
+    int key = r.c.tib * kTileKeys + e.row;
+    for (int j = 0; j < r.ntiles; ++j, ++it, key += kTileKeys) {
+      // this group's quarter of the key norms, straight from the tile in shared memory
+      const uint32_t st = it % kStages;
+      if (!mbar_wait(e.bar_full + 8 * st, (it / kStages) & 1, a.polls, a.poll_ns)) return false;
+      const float q2 = row_sum_squares(e.stages_s + st * kTileBytes, kTileAtomBytes, e.row, 4 * e.wg, 4);
+      float* knb = kn + (it & 1) * (kEpiGroups * 128);
+      knb[e.wg * 128 + e.row] = q2;
+      __syncwarp();
+      if (e.lane == 0) { mbar_arrive(e.bar_empty + 8 * st); mbar_arrive(e.bar_kn + 8 * (it & 1)); }
+      if (!mbar_wait(e.bar_kn + 8 * (it & 1), (it >> 1) & 1, a.polls, a.poll_ns)) return false;
+      const float n2 = (knb[e.row] + knb[128 + e.row]) + (knb[256 + e.row] + knb[384 + e.row]);
+      const float rk = n2 > 0.f ? 1.0f / sqrtf(n2) : 0.f;
+
+      const uint32_t acc = it & 1;
+      if (!mbar_wait(e.bar_tfull + 8 * acc, (it >> 1) & 1, a.polls, a.poll_ns)) return false;
+      tc_fence_after();
+      float sum = 0.f;
+      if constexpr (NC > 0) {
+        uint32_t v[NC];
+        load_epi_cols<NC>(e.t_lane + acc * kAccStride + c0, v);
+        tc_fence_before();
+        mbar_arrive(e.bar_tempty + 8 * acc);
+        const float2 rk2 = make_float2(rk, rk);
+        float2 s0 = make_float2(0.f, 0.f), s1 = make_float2(0.f, 0.f);
+#pragma unroll
+        for (int k = 0; k < NC; k += 4) {
+          const float4 rq = *reinterpret_cast<const float4*>(rqw + k);
+          const float2 c0v = __fmul2_rn(make_float2(__uint_as_float(v[k]), __uint_as_float(v[k + 1])),
+                                        __fmul2_rn(make_float2(rq.x, rq.y), rk2));
+          const float2 c1v = __fmul2_rn(make_float2(__uint_as_float(v[k + 2]), __uint_as_float(v[k + 3])),
+                                        __fmul2_rn(make_float2(rq.z, rq.w), rk2));
+          s0 = add2(s0, collide_pow2<KB>(c0v, kbits));
+          s1 = add2(s1, collide_pow2<KB>(c1v, kbits));
+        }
+        sum = (s0.x + s0.y) + (s1.x + s1.y);
+      } else {
+        tc_fence_before();
+        mbar_arrive(e.bar_tempty + 8 * acc);
+      }
+      // groups 1..3 hand their sums to group 0, which adds them in a fixed order
+      if (e.wg > 0) {
+        if (it >= 2 && !mbar_wait(e.bar_xb + 8 * acc, ((it >> 1) - 1) & 1, a.polls, a.poll_ns)) return false;
+        part[(acc * 3 + (e.wg - 1)) * 128 + e.row] = sum;
+        mbar_arrive(e.bar_xa + 8 * acc);
+      } else {
+        if (!mbar_wait(e.bar_xa + 8 * acc, (it >> 1) & 1, a.polls, a.poll_ns)) return false;
+        const float tot = ((sum + part[(acc * 3 + 0) * 128 + e.row]) + part[(acc * 3 + 1) * 128 + e.row]) +
+                          part[(acc * 3 + 2) * 128 + e.row];
+        mbar_arrive(e.bar_xb + 8 * acc);
+        if (key < a.S) out[key] = tot * inv_gw;
+      }
+    }
+    x += r.ntiles;
+    new_group = r.ends_group;
+    if (new_group && x < e.x_end) mbar_arrive(e.bar_stat_free);
+  }
+  return true;
+}
+
 // Shared memory carve-up, identical on host (sizes) and device (addresses).
 __host__ __device__ inline uint32_t stream_smem_bytes(int mode, int stat_rows_alloc, int hist_bytes) {
   uint32_t b = 2u * stat_rows_alloc * 128u + kStages * kTileBytes;
   if (mode == kProj) b += (hist_bytes + 127u) & ~127u;
-  b += kXchBytes;    // exchange area: per-warp log-sum-exp values, cross-group partials
+  b += (mode == kTheory) ? kXchTheoryBytes : kXchBytes;    // exchange area: per-warp values, cross-group partials
   b += 256;          // barriers + TMEM slot
   return b + 1024;   // slack for 1024-byte alignment of the base
 }
@@ -483,7 +604,7 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
   const uint32_t sm_hist = cur;
   if (MODE == kProj) cur += (hist_bytes + 127u) & ~127u;
   const uint32_t sm_xch = cur;
-  cur += kXchBytes;
+  cur += (MODE == kTheory) ? kXchTheoryBytes : kXchBytes;
   const uint32_t sm_bars = cur;
   const uint32_t sm_tmem_slot = cur + 192;
   const uint32_t bar_full = sm_bars;                   // kStages barriers: tile landed
@@ -494,6 +615,7 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
   const uint32_t bar_stat_free = bar_stat + 8;         // stationary operand no longer in use
   const uint32_t bar_xa = bar_stat_free + 8;           // 2: mode-specific hand-off, "data written"
   const uint32_t bar_xb = bar_xa + 16;                 // 2: mode-specific hand-off, "data consumed"
+  const uint32_t bar_kn = bar_xb + 16;                 // 2: kTheory, key-norm partials of a tile written
   uint8_t* const gen_base = smem_raw + (base - smem_u32(smem_raw));
   const uint16_t* hist_s = reinterpret_cast<const uint16_t*>(gen_base + (sm_hist - base));
   uint8_t* const xch_s = gen_base + (sm_xch - base);
@@ -502,7 +624,12 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
   const int nmb = (MODE == kLse) ? (a.GW + 127) / 128 : 1;   // query row blocks of 128
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+    // a stage is free once the MMAs have read it; under kTheory the epilogue warps read it too
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(bar_full + 8 * s, 1);
+      mbar_init(bar_empty + 8 * s, MODE == kTheory ? 1 + kEpilogueThreads / 32 : 1);
+    }
+    if (MODE == kTheory) { mbar_init(bar_kn, kEpilogueThreads / 32); mbar_init(bar_kn + 8, kEpilogueThreads / 32); }
     for (int s = 0; s < kMaxAcc; ++s) { mbar_init(bar_tfull + 8 * s, 1); mbar_init(bar_tempty + 8 * s, kEpilogueThreads); }
     mbar_init(bar_stat, 1);
     mbar_init(bar_stat_free, kEpilogueThreads);
@@ -653,6 +780,10 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
     e.bar_xa = bar_xa; e.bar_xb = bar_xb;
     e.xch_s = xch_s;
     e.hist_s = hist_s;
+    e.bar_full = bar_full; e.bar_empty = bar_empty; e.bar_kn = bar_kn;
+    e.stat_s = gen_base + (sm_stat - base);
+    e.stages_s = gen_base + (sm_stages - base);
+    e.stat_atom_bytes = stat_atom_bytes;
     bool ok;
     if constexpr (MODE == kLse) {
       ok = (nmb == 2) ? lse_epilogue<64>(a, e, nmb) : lse_epilogue<32>(a, e, nmb);
@@ -667,6 +798,17 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
         case 32: ok = score_epilogue<32>(a, e, c0); break;
         case 16: ok = score_epilogue<16>(a, e, c0); break;
         default: ok = score_epilogue<0>(a, e, c0); break;
+      }
+    } else if constexpr (MODE == kTheory) {
+      const int cw = ((a.GW + kEpiGroups - 1) / kEpiGroups + 15) & ~15;
+      const int c0 = e.wg * cw;
+      const int ncols = max(0, min(a.GW, c0 + cw) - c0);
+      switch (ncols) {
+        case 64: ok = theory_epilogue<64, KBITS>(a, e, c0); break;
+        case 48: ok = theory_epilogue<48, KBITS>(a, e, c0); break;
+        case 32: ok = theory_epilogue<32, KBITS>(a, e, c0); break;
+        case 16: ok = theory_epilogue<16, KBITS>(a, e, c0); break;
+        default: ok = theory_epilogue<0, KBITS>(a, e, c0); break;
       }
     } else {
       ok = proj_epilogue<KBITS, TC>(a, e);
