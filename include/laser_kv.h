@@ -52,7 +52,10 @@ typedef struct {
   int32_t n_kv_heads;          /* H_kv; H_q % H_kv == 0; G = H_q / H_kv (GQA group)              */
   int32_t head_dim;            /* d; must be 128                                                 */
   int32_t block_size;          /* S: tokens per block (Section 3.2); multiple of 8               */
-  int32_t window;              /* W: observation-window queries per query head                   */
+  int32_t window;              /* W: observation-window queries per query head; G*W a multiple of
+                                  16; above 256 the group's queries are scored in 2..4 equal parts of
+                                  window positions (W divisible by the number of parts, every part a
+                                  multiple of 16 queries), up to G*W = 1024                       */
   int32_t max_blocks;          /* cache capacity per (layer, sequence, KV head) = max_blocks * B */
   int32_t max_blocks_per_call; /* upper bound on n_blocks of one select call (sizes workspace)   */
   int32_t lsh_bits;            /* K: sign bits per SimHash table, 1..12                           */
@@ -109,6 +112,10 @@ typedef struct {
                                     or block_size + floor(B/n) for the later blocks under look-back */
   int32_t segment_shift;         /* scored key 0 is this many tokens before the block's first token
                                     (0, or floor(B/n) for the later blocks under look-back)        */
+  int32_t window_part;           /* W' = W / parts: a group of more than 256 window queries is scored
+                                    in up to four parts of W' window positions each; the GW rows of
+                                    lse2 and query_buckets are ordered (part, head of the group,
+                                    position within the part), which is (head, position) when W' = W */
 } laser_kv_debug_t;
 
 /* Appendix B, Eq. 1: B = floor(2 r S_block L / (S_block + L)) evaluated in IEEE double.

@@ -48,7 +48,8 @@ class Debug(C.Structure):
                 ("idx", C.c_void_p), ("n_blocks", C.c_int32), ("batch", C.c_int32),
                 ("n_kv_heads", C.c_int32), ("block_size", C.c_int32), ("budget", C.c_int32),
                 ("gw", C.c_int32), ("lsh_tables", C.c_int32), ("lsh_bits", C.c_int32),
-                ("n_sign_fixups", C.c_int32), ("segment_keys", C.c_int32), ("segment_shift", C.c_int32)]
+                ("n_sign_fixups", C.c_int32), ("segment_keys", C.c_int32), ("segment_shift", C.c_int32),
+                ("window_part", C.c_int32)]
 
 
 class LaserKVError(RuntimeError):
@@ -208,6 +209,7 @@ class DebugTensors:
     n_sign_fixups: int
     segment_keys: int = 0
     segment_shift: int = 0
+    window_part: int = 0
 
 
 class LaserKV:
@@ -319,7 +321,8 @@ class LaserKV:
             hist=view(d.hist, d.batch * d.n_kv_heads * L * (2 << d.lsh_bits), torch.int16,
                       (d.batch, d.n_kv_heads, L, 1 << d.lsh_bits)),
             idx=view(d.idx, nseg * max(d.budget, 1) * 4, torch.int32, shp + (max(d.budget, 1),)),
-            n_sign_fixups=int(d.n_sign_fixups), segment_keys=int(d.segment_keys), segment_shift=int(d.segment_shift))
+            n_sign_fixups=int(d.n_sign_fixups), segment_keys=int(d.segment_keys), segment_shift=int(d.segment_shift),
+            window_part=int(d.window_part))
 
     def laser_kv_decode_attention(self, layer, Q_dec, softmax_scale=0.0, out=None, stream=None):
         """Q_dec: [batch][H_q][d] 2-byte tensor (contiguous last dim) -> fp32 [batch][H_q][d]."""

@@ -42,6 +42,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 
 struct Derived {
   int B, anchors, k_exact, k_lsh, G, GW;
+  int n_qparts, Wp, GWp;   // parts a wide window is scored in; window positions and queries per part
   int tiles_in_block;
   int TC, n_chunks;
   int Kp, Lp;          // bits per table and tables as the kernels see them (padded, see derive)
@@ -191,9 +192,16 @@ laser_kv_status_t derive(const laser_kv_config_t* c, Derived* d) {
   laser_kv_partition(d->B, c->protection_divisor, d->alpha, &d->anchors, &loc, &d->k_exact, &d->k_lsh);
   d->G = c->n_q_heads / c->n_kv_heads;
   d->GW = d->G * c->window;
-  if (d->GW % 16 || d->GW > 256 || c->window > 256 || d->G > 256)
+  // A pass of the scoring kernels holds at most 256 window queries of a KV head's group; a wider
+  // window is scored in parts (equal ranges of window positions, all heads of the group each):
+  // the probabilities and the collision histograms of the parts simply add up.
+  d->n_qparts = (d->GW + 255) / 256;
+  if (d->G > 256 || d->n_qparts > 4 || c->window % d->n_qparts || (d->GW / d->n_qparts) % 16)
     return fail(nullptr, LASER_KV_ERR_UNSUPPORTED,
-                "config: G*W = %d must be a multiple of 16 and at most 256", d->GW);
+                "config: G*W = %d must split into at most 4 equal parts of window positions, each a multiple of 16 "
+                "queries and at most 256", d->GW);
+  d->Wp = c->window / d->n_qparts;
+  d->GWp = d->G * d->Wp;
   if (c->lsh_bits > 12)
     return fail(nullptr, LASER_KV_ERR_UNSUPPORTED, "config: lsh_bits must be at most 12");
   // The kernels take an even number (>= 4) of bits per table and tables in groups of eight. Other
@@ -237,7 +245,7 @@ void carve_ws(const laser_kv_config_t* c, const Derived& d, Carve* v) {
   v->dec_count = take(bh * 4);        // finished decode splits per (sequence, KV head)
   v->hist = take(bh * d.Lp * ((size_t)2 << d.Kp));
   v->qbuckets = take(bh * d.GW * d.Lp * 2);
-  v->lse_part = take(lse_part_bytes_bound(nseg, d.GW));
+  v->lse_part = take(lse_part_bytes_bound(nseg, d.GWp));
   v->lse2 = take(nseg * d.GW * 4);
   v->s_exact = take(nseg * S * 4);
   v->counts = take(nseg * S * 4 + 16);     // cleared in 16-byte units
@@ -608,7 +616,7 @@ laser_kv_status_t run_select(laser_kv_ctx* h, int layer, const void* K_blk, cons
     if ((c.n_q_heads > 1 && q_strides[1] == 0) || (c.batch > 1 && q_strides[0] == 0))
       return fail(h, LASER_KV_ERR_INVALID_ARG, "select_block: zero stride on a dimension of extent > 1");
     const uint64_t strides[3] = {s_w * 2, s_head * 2, s_batch * 2};
-    const uint32_t box[4] = {(uint32_t)kAtomCols, (uint32_t)c.window, (uint32_t)d.G, 1};
+    const uint32_t box[4] = {(uint32_t)kAtomCols, (uint32_t)d.Wp, (uint32_t)d.G, 1};
     if (!encode_map(h, &mapQ, Q_win, 4, dims, strides, box)) return LASER_KV_ERR_CUDA;
   }
 
@@ -634,19 +642,21 @@ laser_kv_status_t run_select(laser_kv_ctx* h, int layer, const void* K_blk, cons
   // 1. query signatures and bucket histograms; the kernel also clears the counts and restarts the
   //    fix-up counter (ctrl[1]) and the changed counter (ctrl[2]); the status word (ctrl[0]) is kept
   if (need_lsh) {
-    const int q_alloc = ((d.GW + 127) / 128) * 128;
-    QsigArgs qa{static_cast<const uint16_t*>(Q_win), q_strides[0], q_strides[1], q_strides[2], h->P, hist, qb,
-                c.n_kv_heads, d.G, c.window, d.GW, q_alloc, d.Lp,
-                reinterpret_cast<uint4*>(counts), ((long long)nseg * S_len + 3) / 4, ctrl + 1, fix_counts, nseg, ctrl,
-                c.lsh_tables};
-    dim3 grid(d.Lp / kQsigTables, c.n_kv_heads, c.batch);
-    LKV_CUDA(launch_qsig(d.Kp, mapQ, h->mapPq, qa, grid, qsig_smem_bytes(q_alloc, d.Kp), st), "qsig_kernel");
+    const int q_alloc = ((d.GWp + 127) / 128) * 128;
+    for (int part = 0; part < d.n_qparts; ++part) {      // a window wider than a pass: its parts add up in the histogram
+      QsigArgs qa{static_cast<const uint16_t*>(Q_win), q_strides[0], q_strides[1], q_strides[2], h->P, hist, qb,
+                  c.n_kv_heads, d.G, d.Wp, d.GWp, q_alloc, d.Lp,
+                  reinterpret_cast<uint4*>(counts), ((long long)nseg * S_len + 3) / 4, ctrl + 1, fix_counts, nseg, ctrl,
+                  c.lsh_tables, part * d.Wp, part * d.GWp, d.GW, part == 0 ? 1 : 0};
+      dim3 grid(d.Lp / kQsigTables, c.n_kv_heads, c.batch);
+      LKV_CUDA(launch_qsig(d.Kp, mapQ, h->mapPq, qa, grid, qsig_smem_bytes(q_alloc, d.Kp), st), "qsig_kernel");
+    }
   }
 
   StreamArgs sa;
   memset(&sa, 0, sizeof sa);
   sa.S = S_len; sa.S_stride = S; sa.nb = nb; sa.H_kv = c.n_kv_heads; sa.batch = c.batch;
-  sa.G = d.G; sa.W = c.window; sa.GW = d.GW;
+  sa.G = d.G; sa.W = d.Wp; sa.GW = d.GWp; sa.lse2_stride = d.GW;
   sa.tiles_in_block = tiles_in_block; sa.nseg = nseg;
   const long long seg_tiles = (long long)nseg * tiles_in_block;
   const int base_ctas = stream_grid(seg_tiles, h->num_sms);
@@ -663,8 +673,8 @@ laser_kv_status_t run_select(laser_kv_ctx* h, int layer, const void* K_blk, cons
   // 2. per-query log-sum-exp over each segment's keys
   if (need_exact) {
     StreamArgs a1 = sa;
-    a1.stat_rows = d.GW;
-    a1.stat_rows_alloc = ((d.GW + 127) / 128) * 128;
+    a1.stat_rows = d.GWp;
+    a1.stat_rows_alloc = ((d.GWp + 127) / 128) * 128;
     const uint32_t smem = stream_smem_bytes(kLse, a1.stat_rows_alloc, 0);
     LKV_CUDA((launch_stream<kLse, 0, 0>(mapK, mapQ, a1, base_ctas, smem, st)), "lse pass");
   }
@@ -672,10 +682,22 @@ laser_kv_status_t run_select(laser_kv_ctx* h, int layer, const void* K_blk, cons
   // 3. summed attention probabilities per key
   if (need_exact) {
     StreamArgs a2 = sa;
-    a2.stat_rows = d.GW;
-    a2.stat_rows_alloc = d.GW;
+    a2.stat_rows = d.GWp;
+    a2.stat_rows_alloc = d.GWp;
     const uint32_t smem = stream_smem_bytes(kScore, a2.stat_rows_alloc, 0);
     LKV_CUDA((launch_stream<kScore, 0, 0>(mapK, mapQ, a2, base_ctas, smem, st)), "score pass");
+    // the remaining parts of a window wider than a pass: their probabilities add to the first part's
+    for (int part = 1; part < d.n_qparts; ++part) {
+      StreamArgs b1 = sa, b2 = sa;
+      b1.q_w0 = b2.q_w0 = part * d.Wp;
+      b1.lse2_off = b2.lse2_off = part * d.GWp;
+      b1.stat_rows = b2.stat_rows = d.GWp;
+      b1.stat_rows_alloc = ((d.GWp + 127) / 128) * 128;
+      b2.stat_rows_alloc = d.GWp;
+      b2.accumulate = 1;
+      LKV_CUDA((launch_stream<kLse, 0, 0>(mapK, mapQ, b1, base_ctas, stream_smem_bytes(kLse, b1.stat_rows_alloc, 0), st)), "lse pass");
+      LKV_CUDA((launch_stream<kScore, 0, 0>(mapK, mapQ, b2, base_ctas, smem, st)), "score pass");
+    }
   }
   mark();
   // 4. key signatures and collision counts
@@ -1084,6 +1106,7 @@ laser_kv_status_t laser_kv_debug_view(laser_kv_handle_t h, laser_kv_debug_t* out
   out->segment_shift = h->last_shift;
   out->budget = h->last_B;
   out->gw = h->d.GW;
+  out->window_part = h->d.Wp;
   out->lsh_tables = h->d.Lp;
   out->lsh_bits = h->d.Kp;
   out->n_sign_fixups = h->last_fixups;
@@ -1318,7 +1341,7 @@ laser_kv_status_t run_window_scores(const ScoreGeom& g, const void* K_blk, const
       (e = cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess)
     return fail(nullptr, LASER_KV_ERR_CUDA, "window_scores: device query: %s", cudaGetErrorString(e));
   sa.S = g.S; sa.S_stride = g.S; sa.nb = g.nb; sa.H_kv = g.H_kv; sa.batch = g.batch;
-  sa.G = g.G; sa.W = g.W; sa.GW = g.GW; sa.tiles_in_block = g.tiles_in_block; sa.nseg = g.nseg;
+  sa.G = g.G; sa.W = g.W; sa.GW = g.GW; sa.lse2_stride = g.GW; sa.tiles_in_block = g.tiles_in_block; sa.nseg = g.nseg;
   sa.n_tiles = (long long)g.nseg * g.tiles_in_block;
   const int ctas = stream_grid(sa.n_tiles, num_sms);
   sa.lse_ctas = ctas; sa.n_slot = lse_slots(ctas, g.nseg);
@@ -1558,7 +1581,7 @@ laser_kv_status_t laser_kv_collision_counts(const void* K_blk, const void* Q_win
     QsigArgs qa{static_cast<const uint16_t*>(Q_win), q_strides[0], q_strides[1], q_strides[2], P, hist, qb,
                 g.H_kv, g.G, g.W, g.GW, q_alloc, lsh_tables,
                 reinterpret_cast<uint4*>(counts_out), (long long)g.nseg * g.S / 4, ctrl + 1, fix_counts, g.nseg, ctrl,
-                lsh_tables};
+                lsh_tables, 0, 0, g.GW, 1};
     dim3 grid(lsh_tables / kQsigTables, g.H_kv, g.batch);
     if ((e = launch_qsig(lsh_bits, mapQ, mapPq, qa, grid, qsig_smem_bytes(q_alloc, lsh_bits), st)) != cudaSuccess)
       return fail(nullptr, LASER_KV_ERR_CUDA, "collision_counts: qsig_kernel: %s", cudaGetErrorString(e));

@@ -37,6 +37,10 @@ struct QsigArgs {
   int n_seg_counters;
   int* status;
   int n_real_tables;       // tables from this index on are padding: their histograms stay empty
+  int q_w0;                // first window position of this pass; W and GW describe the pass
+  int q_row0, q_rows_total;   // qbuckets rows: [bh][q_rows_total][L], this pass starts at row q_row0
+  int first_part;          // nonzero: clear the counts, restart the counters, store the histogram;
+                           // zero: a later part of a wide window: add to the histogram
 };
 
 // <x, y> over 128 bf16 elements in fp64 (every product is exact); 16-byte loads, all in flight at once.
@@ -108,8 +112,8 @@ qsig_kernel(const __grid_constant__ CUtensorMap map_q,    // Q: (d, W, H_q, batc
 
   if (warp == 0 && lane == 0) {
     mbar_expect_tx(bar_load, 2u * a.GW * 128u + 2u * N * 128u);
-    tma_load_4d(sm_q, &map_q, bar_load, 0, 0, h * a.G, b);
-    tma_load_4d(sm_q + q_atom, &map_q, bar_load, kAtomCols, 0, h * a.G, b);
+    tma_load_4d(sm_q, &map_q, bar_load, 0, a.q_w0, h * a.G, b);
+    tma_load_4d(sm_q + q_atom, &map_q, bar_load, kAtomCols, a.q_w0, h * a.G, b);
     tma_load_2d(sm_p, &map_p, bar_load, 0, tg * N);
     tma_load_2d(sm_p + N * 128u, &map_p, bar_load, kAtomCols, tg * N);
   }
@@ -119,10 +123,12 @@ qsig_kernel(const __grid_constant__ CUtensorMap map_q,    // Q: (d, W, H_q, batc
     const long long nctas = (long long)gridDim.x * gridDim.y * gridDim.z;
     const long long per = (a.zero_n + nctas - 1) / nctas;
     const long long z0 = cta * per, z1 = min(a.zero_n, z0 + per);
-    for (long long i = z0 + threadIdx.x; i < z1; i += kQsigThreads) a.zero_begin[i] = make_uint4(0u, 0u, 0u, 0u);
-    if (cta == 0 && threadIdx.x < 2) a.counters[threadIdx.x] = 0;
-    if (cta == nctas - 1)
-      for (int i = threadIdx.x; i < a.n_seg_counters; i += kQsigThreads) a.seg_counters[i] = 0;
+    if (a.first_part) {
+      for (long long i = z0 + threadIdx.x; i < z1; i += kQsigThreads) a.zero_begin[i] = make_uint4(0u, 0u, 0u, 0u);
+      if (cta == 0 && threadIdx.x < 2) a.counters[threadIdx.x] = 0;
+      if (cta == nctas - 1)
+        for (int i = threadIdx.x; i < a.n_seg_counters; i += kQsigThreads) a.seg_counters[i] = 0;
+    }
     for (uint32_t i = threadIdx.x; i < kQsigTables * nbins; i += kQsigThreads) bins[i] = 0;
   }
   __syncthreads();
@@ -166,7 +172,7 @@ qsig_kernel(const __grid_constant__ CUtensorMap map_q,    // Q: (d, W, H_q, batc
 #pragma unroll
       for (int k = 0; k < 16; k += 2) amax = max3_abs(__uint_as_float(v[k]), __uint_as_float(v[k + 1]), amax);
       const float tau = amax * (1.0f / 32768.0f);
-      const uint16_t* row = a.Q + b * a.qs_b + (long long)(h * a.G + q / a.W) * a.qs_h + (q % a.W) * a.qs_w;
+      const uint16_t* row = a.Q + b * a.qs_b + (long long)(h * a.G + q / a.W) * a.qs_h + (a.q_w0 + q % a.W) * a.qs_w;
       uint32_t codes[kQsigTables];
 #pragma unroll
       for (int t = 0; t < kQsigTables; ++t) {
@@ -193,7 +199,7 @@ qsig_kernel(const __grid_constant__ CUtensorMap map_q,    // Q: (d, W, H_q, batc
       packed.y = codes[2] | (codes[3] << 16);
       packed.z = codes[4] | (codes[5] << 16);
       packed.w = codes[6] | (codes[7] << 16);
-      *reinterpret_cast<uint4*>(a.qbuckets + (bh * a.GW + q) * a.lsh_tables + tg * kQsigTables) = packed;
+      *reinterpret_cast<uint4*>(a.qbuckets + (bh * a.q_rows_total + a.q_row0 + q) * a.lsh_tables + tg * kQsigTables) = packed;
     }
   }
   if (!ok) record_status(a.status, kStatusTimeout);
@@ -201,7 +207,8 @@ qsig_kernel(const __grid_constant__ CUtensorMap map_q,    // Q: (d, W, H_q, batc
   __syncthreads();
   if (ok) {
     uint16_t* out = a.hist + (bh * a.lsh_tables + (size_t)tg * kQsigTables) * nbins;
-    for (uint32_t i = threadIdx.x; i < kQsigTables * nbins; i += kQsigThreads) out[i] = (uint16_t)bins[i];
+    for (uint32_t i = threadIdx.x; i < kQsigTables * nbins; i += kQsigThreads)
+      out[i] = (uint16_t)(a.first_part ? bins[i] : bins[i] + out[i]);
   }
   if (warp == 0) {
     tc_fence_after();

@@ -71,7 +71,10 @@ struct StreamArgs {
   int S_stride;        // tokens between the first keys of consecutive segments (the block size)
   int nb;              // blocks in this call
   int H_kv, batch;
-  int G, W, GW;        // GQA group size, window, G*W
+  int G, W, GW;        // GQA group size, window queries per head in this pass, G*W
+  int q_w0;            // first window position of this pass (a window wider than 256/G queries is scored in parts)
+  int accumulate;      // kScore: add to s_exact instead of storing (second and later parts)
+  int lse2_stride, lse2_off;   // lse2[seg * lse2_stride + lse2_off + query of this pass]
   int tiles_in_block;  // ceil(S / 128)
   int nseg;            // batch * H_kv * nb
   long long n_tiles;   // tiles of this launch: nseg * tiles_in_block (* n_chunks for kProj)
@@ -383,7 +386,7 @@ __device__ __forceinline__ bool score_epilogue(const StreamArgs& a, const EpiCtx
             if (pe.x != -INFINITY) sum += pe.y * exp2f(pe.x - mx);
           }
           const float lse = mx + log2f(sum);
-          if (r.c.tib == 0 && e.quarter == 0) a.lse2[(size_t)r.c.seg * a.GW + qq] = lse;
+          if (r.c.tib == 0 && e.quarter == 0) a.lse2[(size_t)r.c.seg * a.lse2_stride + a.lse2_off + qq] = lse;
           lw[j] = -lse;
         }
       }
@@ -416,7 +419,7 @@ __device__ __forceinline__ bool score_epilogue(const StreamArgs& a, const EpiCtx
         const float tot = ((sum + part[(acc * 3 + 0) * 128 + e.row]) + part[(acc * 3 + 1) * 128 + e.row]) +
                           part[(acc * 3 + 2) * 128 + e.row];
         mbar_arrive(e.bar_xb + 8 * acc);
-        if (key < a.S) out[key] = tot;
+        if (key < a.S) out[key] = a.accumulate ? out[key] + tot : tot;
       }
     }
     x += r.ntiles;
@@ -673,8 +676,8 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
             const uint16_t* hsrc = a.hist + ((size_t)c.bh * a.lsh_tables + (size_t)c.chunk * TC) * ((size_t)1 << KBITS);
             bulk_load(sm_hist, hsrc, hist_bytes, bar_stat);
           } else {
-            tma_load_4d(sm_stat, &map_stat, bar_stat, 0, 0, h * a.G, b);
-            tma_load_4d(sm_stat + stat_atom_bytes, &map_stat, bar_stat, kAtomCols, 0, h * a.G, b);
+            tma_load_4d(sm_stat, &map_stat, bar_stat, 0, a.q_w0, h * a.G, b);
+            tma_load_4d(sm_stat + stat_atom_bytes, &map_stat, bar_stat, kAtomCols, a.q_w0, h * a.G, b);
           }
           ++gen;
         }

@@ -174,6 +174,13 @@ def check_run(w: synth.Workload, run, segments=None, alpha=None):
     qc_all = to_np(dbg.query_buckets)
     kc_all = to_np(dbg.key_buckets) if dbg.key_buckets is not None else None
     lse_all = to_np(dbg.lse2)
+    if dbg.window_part != W:
+        # a wide window is scored in parts: the library orders the group's queries (part, head, position
+        # in the part); bring its per-query arrays into the oracle's (head, position) order
+        Wp = dbg.window_part
+        order = np.array([(r // (G * Wp)) * Wp + ((r % (G * Wp)) // Wp) * W + (r % Wp) for r in range(G * W)])
+        inv = np.argsort(order)
+        qc_all, lse_all = qc_all[:, :, inv], lse_all[..., inv]
     if segments is None:
         segments = [(b, h, t) for b in range(w.batch) for h in range(w.n_kv_heads) for t in range(nb)]
     stats = []

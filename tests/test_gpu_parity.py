@@ -54,6 +54,9 @@ def test_gqa7_k10_shape_with_rope_and_batch():
     (1, 20, 4, 4, 16, 136),      # one bit per table -> 4, 20 tables -> 24
     (11, 9, 4, 2, 64, 520),      # 11 bits -> 12, 9 tables -> 16
     (9, 64, 8, 2, 32, 648),      # 9 bits -> 10, tables already a multiple of eight
+    (8, 16, 8, 2, 128, 520),     # G*W = 512: the window is scored in two parts of 64 positions
+    (10, 8, 6, 2, 96, 392),      # G*W = 288: two parts of 48 positions (144 queries each)
+    (8, 8, 8, 1, 128, 264),      # G*W = 1024: four parts of 32 positions
 ])
 def test_hash_and_group_geometries(K, L, hq, hkv, W, S):
     w = synth.workload("tiny").with_(name=f"geo{K}_{L}_{hq}_{hkv}_{W}", n_q_heads=hq, n_kv_heads=hkv, window=W,
