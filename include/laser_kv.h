@@ -270,6 +270,18 @@ const char* laser_kv_status_string(laser_kv_status_t s);
  * error of a call that had no handle (init, query_sizes, step entry points). */
 const char* laser_kv_last_error(laser_kv_handle_t h);
 
+/* Per-handle counters since laser_kv_init (host only, no synchronisation): calls of the select
+ * entry points, blocks and tokens they covered (tokens per sequence, summed over the batch), cache
+ * entries appended per (sequence, KV head) summed over sequences and heads, and the bytes the method
+ * itself has to move for that work (keys read once, window queries and hyperplanes per call, every
+ * kept K and V row read once and written once, positions). With the environment variable
+ * LASER_KV_LOG set to a non-empty value other than 0 when the handle is created, every select call,
+ * reset and destroy also writes one line to stderr (host side only; nothing changes on the device). */
+typedef struct {
+  int64_t select_calls, blocks, tokens, entries_appended, algorithmic_bytes;
+} laser_kv_counters_t;
+laser_kv_status_t laser_kv_get_counters(laser_kv_handle_t h, laser_kv_counters_t* out);
+
 /* Number of this library's kernels launched by the calling process so far (all handles). */
 int64_t laser_kv_launch_count(void);
 

@@ -21,7 +21,7 @@ EXPORTS = [
     "laser_kv_collision_counts", "laser_kv_collision_counts_scratch_bytes", "laser_kv_consensus_accumulate",
     "laser_kv_decode_attention", "laser_kv_decode_attention_scratch_bytes", "laser_kv_collision_probability",
     "laser_kv_set_layer_budget", "laser_kv_set_wait_budget", "laser_kv_window_scores_static_status",
-    "laser_kv_lookback_close", "laser_kv_select_tail",
+    "laser_kv_lookback_close", "laser_kv_select_tail", "laser_kv_get_counters",
 ]
 
 
@@ -50,6 +50,11 @@ class Debug(C.Structure):
                 ("gw", C.c_int32), ("lsh_tables", C.c_int32), ("lsh_bits", C.c_int32),
                 ("n_sign_fixups", C.c_int32), ("segment_keys", C.c_int32), ("segment_shift", C.c_int32),
                 ("window_part", C.c_int32)]
+
+
+class Counters(C.Structure):
+    _fields_ = [("select_calls", C.c_int64), ("blocks", C.c_int64), ("tokens", C.c_int64),
+                ("entries_appended", C.c_int64), ("algorithmic_bytes", C.c_int64)]
 
 
 class LaserKVError(RuntimeError):
@@ -109,6 +114,8 @@ def load(build_if_missing: bool = True) -> C.CDLL:
     lib.laser_kv_two_stage_topk.argtypes = [vp, vp, i32, i32, i32, i32, i32, vp, vp]
     lib.laser_kv_gather_append.restype = i32
     lib.laser_kv_gather_append.argtypes = [vp, vp, i64, i64, i32, vp, i32, i32, vp, vp, i64, i64, vp, i64, i64, i32, vp, vp]
+    lib.laser_kv_get_counters.restype = i32
+    lib.laser_kv_get_counters.argtypes = [vp, p(Counters)]
     lib.laser_kv_select_tail.restype = i32
     lib.laser_kv_select_tail.argtypes = [vp, i32, vp, vp, vp, p(i64), p(i64), i32, vp]
     lib.laser_kv_lookback_close.restype = i32
@@ -357,6 +364,11 @@ class LaserKV:
 
     def laser_kv_set_layer_budget(self, layer, budget_per_block):
         _check(self.lib.laser_kv_set_layer_budget(self.handle, layer, budget_per_block), self.handle)
+
+    def laser_kv_get_counters(self):
+        c = Counters()
+        _check(self.lib.laser_kv_get_counters(self.handle, C.byref(c)), self.handle)
+        return {k: int(getattr(c, k)) for k, _ in Counters._fields_}
 
     def laser_kv_set_wait_budget(self, max_polls):
         _check(self.lib.laser_kv_set_wait_budget(self.handle, max_polls), self.handle)

@@ -9,6 +9,7 @@
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <string>
@@ -97,6 +98,8 @@ struct laser_kv_ctx {
   struct StageUse { const void* k; const void* v; const void* q; cudaEvent_t done; };
   std::vector<StageUse> stage_use;
   uint32_t handoff_polls = 0;           // 0: built-in wait budgets (laser_kv_set_wait_budget)
+  laser_kv_counters_t counters = {0, 0, 0, 0, 0};
+  bool log = false;                     // LASER_KV_LOG: one stderr line per call
   // optional per-kernel timing (events only; no device memory)
   bool profiling = false;
   std::vector<cudaEvent_t> ev_pool;
@@ -470,6 +473,10 @@ laser_kv_status_t laser_kv_init(const laser_kv_config_t* cfg, const void* hyperp
   h->cacheV = reinterpret_cast<uint16_t*>(cm + align_up(per * kHeadDim * 2));
   h->cachePos = reinterpret_cast<int32_t*>(cm + 2 * align_up(per * kHeadDim * 2));
   h->P = static_cast<const uint16_t*>(hyperplanes);
+  {
+    const char* lg = getenv("LASER_KV_LOG");
+    h->log = lg && lg[0] && strcmp(lg, "0") != 0;
+  }
   h->blocks_done.assign(cfg->n_layers, 0);
   h->entries_done.assign(cfg->n_layers, 0);
   h->tokens_done.assign(cfg->n_layers, 0);
@@ -740,6 +747,21 @@ laser_kv_status_t run_select(laser_kv_ctx* h, int layer, const void* K_blk, cons
   h->last_B = B;
   h->last_S_len = S_len;
   h->last_shift = g.shift;
+  {
+    laser_kv_counters_t& k = h->counters;
+    const long long rows = (long long)c.batch * c.n_kv_heads * nb;
+    k.blocks += nb;
+    k.tokens += (long long)c.batch * nb * S;
+    k.entries_appended += rows * B;
+    k.algorithmic_bytes += rows * S * kHeadDim * 2                               // keys, once
+                           + (long long)c.batch * c.n_q_heads * c.window * kHeadDim * 2
+                           + (long long)c.lsh_tables * c.lsh_bits * kHeadDim * 2
+                           + rows * B * (4LL * kHeadDim * 2 + 4);                   // kept K and V rows in and out, positions
+    if (h->log)
+      fprintf(stderr, "[laser_kv] layer %d: %d block(s) of %d tokens (segment %d keys, %d before the block), "
+                      "%d entries per block and head, k_exact %d, k_lsh %d, first token %lld\n",
+              layer, nb, S, S_len, g.shift, B, g.k_exact, g.k_lsh, first_token);
+  }
   return LASER_KV_OK;
 }
 
@@ -782,6 +804,7 @@ laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, cons
     return fail(h, LASER_KV_ERR_UNSUPPORTED, "select_block: absolute positions exceed int32");
 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  h->counters.select_calls += 1;
   const laser_kv_ctx::LayerBudget lb = h->budget[layer];
   const int S = c.block_size, n = c.protection_divisor;
   const bool lookback = c.lookback && lb.anchors > 0;
@@ -826,6 +849,7 @@ laser_kv_status_t laser_kv_select_tail(laser_kv_handle_t h, int32_t layer, const
     return fail(h, LASER_KV_ERR_CAPACITY, "select_tail: layer %d cache holds %lld of %d blocks", layer, h->blocks_done[layer], c.max_blocks);
   if (h->tokens_done[layer] + n_tokens > 0x7fffffffLL)
     return fail(h, LASER_KV_ERR_UNSUPPORTED, "select_tail: absolute positions exceed int32");
+  h->counters.select_calls += 1;
   const laser_kv_ctx::LayerBudget lb = h->budget[layer];
   const int B_t = lb.B < n_tokens ? lb.B : n_tokens;           // the same rule on the tokens there are
   const bool lookback = c.lookback != 0;
@@ -1137,6 +1161,7 @@ laser_kv_status_t laser_kv_poll_status(laser_kv_handle_t h, void* stream) {
 laser_kv_status_t laser_kv_reset(laser_kv_handle_t h, int32_t layer) {
   if (!h) return fail(nullptr, LASER_KV_ERR_INVALID_ARG, "reset: NULL handle");
   if (layer < -1 || layer >= h->cfg.n_layers) return fail(h, LASER_KV_ERR_INVALID_ARG, "reset: layer out of range");
+  if (h->log) fprintf(stderr, "[laser_kv] reset layer %d\n", layer);
   for (int l = 0; l < h->cfg.n_layers; ++l) {
     if (layer != -1 && l != layer) continue;
     h->blocks_done[l] = 0;
@@ -1151,6 +1176,10 @@ laser_kv_status_t laser_kv_reset(laser_kv_handle_t h, int32_t layer) {
 
 void laser_kv_destroy(laser_kv_handle_t h) {
   if (!h) return;
+  if (h->log)
+    fprintf(stderr, "[laser_kv] destroy: %lld select call(s), %lld block(s), %lld tokens, %lld entries appended\n",
+            (long long)h->counters.select_calls, (long long)h->counters.blocks, (long long)h->counters.tokens,
+            (long long)h->counters.entries_appended);
   for (auto& set : h->ev_pending) for (cudaEvent_t ev : set) cudaEventDestroy(ev);
   for (cudaEvent_t ev : h->ev_pool) cudaEventDestroy(ev);
   for (cudaEvent_t ev : h->ev_chunk) cudaEventDestroy(ev);
@@ -1173,6 +1202,12 @@ laser_kv_status_t laser_kv_set_layer_budget(laser_kv_handle_t h, int32_t layer, 
   int loc;
   laser_kv_partition(lb.B, h->cfg.protection_divisor, h->d.alpha, &lb.anchors, &loc, &lb.k_exact, &lb.k_lsh);
   h->budget[layer] = lb;
+  return LASER_KV_OK;
+}
+
+laser_kv_status_t laser_kv_get_counters(laser_kv_handle_t h, laser_kv_counters_t* out) {
+  if (!h || !out) return fail(h, LASER_KV_ERR_INVALID_ARG, "get_counters: NULL argument");
+  *out = h->counters;
   return LASER_KV_OK;
 }
 

@@ -84,6 +84,7 @@ def test_null_and_misaligned_arguments_are_rejected():
     assert lib.laser_kv_gather_append(0x1000, 0x2000, 1024, 128, -1, 0x3000, 1, 5, 0x4000, 0x5000, 1024, 8, 0x6000, 8, 0, 0,
                                       0x7000, None) == B.ERR_INVALID_ARG
     assert lib.laser_kv_set_wait_budget(None, 5) == B.ERR_INVALID_ARG
+    assert lib.laser_kv_get_counters(None, None) == B.ERR_INVALID_ARG
     assert b"NULL" in lib.laser_kv_last_error(None)
     # the entry points beside the hot path validate before they touch the device
     assert lib.laser_kv_decode_attention(None, 0, None, None, 0.0, None, None, 0, None) == B.ERR_INVALID_ARG

@@ -129,6 +129,17 @@ def test_append_only_across_calls_and_capacity():
     assert inc.laser_kv_cache_view(1)[3] == 0
 
 
+def test_counters_follow_the_calls():
+    w = synth.workload("tiny").with_(block_size=256, context_len=1024)
+    run = run_workload_layer(w, 0, debug=0)
+    c = run["engine"].laser_kv_get_counters()
+    B, S, nb, hk = run["B"], 256, 4, w.n_kv_heads
+    assert c["select_calls"] == 1 and c["blocks"] == nb and c["tokens"] == nb * S
+    assert c["entries_appended"] == hk * nb * B
+    want = hk * nb * S * 256 + w.n_q_heads * w.window * 256 + w.lsh_tables * w.lsh_bits * 256 + hk * nb * B * (4 * 256 + 4)
+    assert c["algorithmic_bytes"] == want
+
+
 def test_same_inputs_twice_give_identical_bytes():
     w = synth.workload("tiny").with_(block_size=512, context_len=1024)
     r1 = run_workload_layer(w, 0)
