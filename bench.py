@@ -39,11 +39,11 @@ UNIT = "tokens/s"
 # summary of the select call, keyed by (workload, kernel). A missing key means: not captured for
 # this workload, or the kernel has changed since the capture.
 NCU_TRAFFIC_BYTES = {
-    ("llama8b_128k", "stream_kernel<proj>"): 274824192 + 7053824,
-    ("llama8b_128k", "stream_kernel<lse>"): 269270016 + 3895808,
-    ("llama8b_128k", "stream_kernel<score>"): 270836736 + 8108288,
-    ("llama8b_128k", "append_kernel"): 254742272 + 203583744,
-    ("llama8b_128k", "select_kernel"): 17702656,
+    ("llama8b_128k", "stream_kernel<proj>"): 274882816 + 7054848,
+    ("llama8b_128k", "stream_kernel<lse>"): 269269248 + 4089600,
+    ("llama8b_128k", "stream_kernel<score>"): 270997248 + 8295936,
+    ("llama8b_128k", "append_kernel"): 254738688 + 203578368,
+    ("llama8b_128k", "select_kernel"): 17701632,
     ("llama8b_128k", "decode_split_kernel"): 261788672 + 3954944,
 }
 
