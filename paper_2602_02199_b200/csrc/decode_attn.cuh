@@ -57,7 +57,7 @@ struct DecodeArgs {
 };
 
 __host__ __device__ constexpr uint32_t dec_smem_bytes() {
-  return kDecStages * kDecStageBytes + 2u * kDecStages * 8u + 2u * kDecWarps * 8u * 4u + 1024u;
+  return kDecStages * kDecStageBytes + (2u * kDecStages + 1u) * 8u + 2u * kDecWarps * 8u * 4u + 1024u;
 }
 
 // Byte offset of the 16-byte chunk (0..15 over the 128 dims) of a row inside a K or V tile made
@@ -103,7 +103,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap map_k,    // cache K: (d
   const uint32_t base = (smem_u32(dsm_raw) + 1023u) & ~1023u;
   uint8_t* const gen = dsm_raw + (base - smem_u32(dsm_raw));
   const uint32_t sm_bars = base + kDecStages * kDecStageBytes;
-  float* wm = reinterpret_cast<float*>(gen + kDecStages * kDecStageBytes + 2 * kDecStages * 8);   // [warps][8] maxima
+  float* wm = reinterpret_cast<float*>(gen + kDecStages * kDecStageBytes + (2 * kDecStages + 1) * 8);   // [warps][8] maxima
   float* wl = wm + kDecWarps * 8;                                                                   // [warps][8] sums
   float* red = reinterpret_cast<float*>(gen);                     // merge buffer over the stages: [warps][8][132]
   auto bar_full = [&](int s) { return sm_bars + 8u * s; };
@@ -118,6 +118,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap map_k,    // cache K: (d
 
   if (tid == 0) {
     for (int s = 0; s < kDecStages; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), kDecWarps); }
+    mbar_init(sm_bars + 8u * (2 * kDecStages), 1);                 // the merge's bulk copies
     fence_mbar_init();
   }
   if (tid == kDecWarps * 32) { tma_prefetch_desc(&map_k); tma_prefetch_desc(&map_v); }
@@ -267,22 +268,40 @@ decode_split_kernel(const __grid_constant__ CUtensorMap map_k,    // cache K: (d
   }
 
   // ---- the CTA that finishes last for this (sequence, KV head) merges all splits -----------------
+  // The partials of this (sequence, KV head) are contiguous, split-major. The last CTA brings them
+  // into the free stage ring with one bulk copy per round (a ring too small for all splits of many
+  // heads takes several rounds) while the splits' maxima and sums are read and turned into weights.
   __shared__ int s_last;
-  __threadfence();
-  __syncthreads();
+  const float* seg = a.part + ((long long)(b * a.H_kv + h) * a.n_split) * a.G * kDecPartFloats;
+  const int sstride = a.G * kDecPartFloats;                        // floats between splits
+  const int gn = a.G * a.n_split;
+  float* wgt = reinterpret_cast<float*>(gen);                      // [G][n_split]
+  float* msl = wgt + gn;                                           // [G][n_split][2] maxima and sums
+  const uint32_t data_off = ((uint32_t)gn * 12u + 15u) & ~15u;
+  const float4* data = reinterpret_cast<const float4*>(gen + data_off);
+  // splits per round: a multiple of four (the accumulator of a split is its index modulo four), >= 8
+  const int per_round = (int)((kDecStages * kDecStageBytes - data_off) / ((uint32_t)sstride * 4u)) & ~3;
+  const uint32_t bar_merge = sm_bars + 8u * (2 * kDecStages);
+  auto fetch = [&](int s0, int ns) {                               // one thread
+    fence_proxy_async_smem();                                      // the ring was last touched by ordinary accesses
+    mbar_expect_tx(bar_merge, (uint32_t)ns * (uint32_t)sstride * 4u);
+    bulk_load(base + data_off, seg + (long long)s0 * sstride, (uint32_t)ns * (uint32_t)sstride * 4u, bar_merge);
+  };
+  __syncthreads();                                                 // the CTA's partial is written ...
   if (tid == 0) {
+    __threadfence();                                               // ... and visible before the count goes up
     int* counter = a.counters + b * a.H_kv + h;
     s_last = atomicAdd(counter, 1) == a.n_split - 1;
-    if (s_last) *counter = 0;                                      // ready for the next call
+    if (s_last) {
+      *counter = 0;                                                // ready for the next call
+      __threadfence();                                             // the other CTAs' partials are visible from here on
+      fence_proxy_async_global();                                  // also to the copy engine
+      fetch(0, min(per_round, a.n_split));
+    }
   }
   __syncthreads();
   if (!s_last) return;
-  __threadfence();
-  const float* seg = a.part + ((long long)(b * a.H_kv + h) * a.n_split) * a.G * kDecPartFloats;
-  const int sstride = a.G * kDecPartFloats;                        // floats between splits
-  float* wgt = reinterpret_cast<float*>(gen + 2 * kDecBoxBytes * 2);   // [G][n_split], past the merge buffer
-  float* msl = wgt + a.G * a.n_split;                              // [G][n_split][2] maxima and sums, read once
-  for (int i = tid; i < a.G * a.n_split; i += kDecThreads) {
+  for (int i = tid; i < gn; i += kDecThreads) {
     const int head = i / a.n_split, s = i - head * a.n_split;
     const float2 v = __ldcg(reinterpret_cast<const float2*>(seg + (long long)s * sstride + head * kDecPartFloats + 128));
     msl[2 * i] = v.x;
@@ -305,35 +324,67 @@ decode_split_kernel(const __grid_constant__ CUtensorMap map_k,    // cache K: (d
     for (int off = 16; off > 0; off >>= 1) l += __shfl_xor_sync(0xffffffffu, l, off);
     if (lane == 0) wl[head] = l;
   }
-  __syncthreads();
-  for (int i = tid; i < a.G * 32; i += kDecThreads) {
-    const int head = i >> 5, d4 = i & 31;
-    const float* w = wgt + head * a.n_split;
-    const float4* src = reinterpret_cast<const float4*>(seg + head * kDecPartFloats) + d4;
-    float4 acc[4];
+  // thread -> up to two (head, four dims) items; four accumulators per item, split s adds to s % 4
+  constexpr int kItems = (kDecMaxGroup * 32 + kDecThreads - 1) / kDecThreads;
+  float4 acc[kItems][4];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int s0 = 0; s0 < a.n_split; s0 += 16) {
-      float4 x[16];
+  for (int it = 0; it < kItems; ++it)
 #pragma unroll
-      for (int j = 0; j < 16; ++j)
-        x[j] = s0 + j < a.n_split ? __ldcg(src + (long long)(s0 + j) * (sstride / 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int j = 0; j < 4; ++j) acc[it][j] = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int s0 = 0; s0 < a.n_split; s0 += per_round) {
+    const int ns = min(per_round, a.n_split - s0);
+    if (s0 > 0) {
+      __syncthreads();                                             // the previous round's rows are read
+      if (tid == 0) fetch(s0, ns);
+    }
+    const bool landed = mbar_wait(bar_merge, (uint32_t)(s0 / per_round) & 1u);
+    if (!__syncthreads_and(landed)) {                              // also: the weights are written
+      if (tid == 0) record_status(a.status, kStatusTimeout);
+      return;
+    }
 #pragma unroll
-      for (int j = 0; j < 16; ++j) {
-        const float ws = s0 + j < a.n_split ? w[s0 + j] : 0.f;
-        acc[j & 3].x = fmaf(ws, x[j].x, acc[j & 3].x);
-        acc[j & 3].y = fmaf(ws, x[j].y, acc[j & 3].y);
-        acc[j & 3].z = fmaf(ws, x[j].z, acc[j & 3].z);
-        acc[j & 3].w = fmaf(ws, x[j].w, acc[j & 3].w);
+    for (int it = 0; it < kItems; ++it) {
+      const int i = tid + it * kDecThreads;
+      if (i < a.G * 32) {
+        const int head = i >> 5, d4 = i & 31;
+        const float* w = wgt + head * a.n_split + s0;
+        const float4* x = data + head * (kDecPartFloats / 4) + d4;
+        const int ns4 = ns & ~3;
+        for (int s = 0; s < ns4; s += 4) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const float ws = w[s + j];
+            const float4 v = x[(s + j) * (sstride / 4)];
+            float4& c4 = acc[it][j];
+            c4.x = fmaf(ws, v.x, c4.x); c4.y = fmaf(ws, v.y, c4.y); c4.z = fmaf(ws, v.z, c4.z); c4.w = fmaf(ws, v.w, c4.w);
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < 3; ++j) {
+          if (ns4 + j < ns) {
+            const float ws = w[ns4 + j];
+            const float4 v = x[(ns4 + j) * (sstride / 4)];
+            float4& c4 = acc[it][j];
+            c4.x = fmaf(ws, v.x, c4.x); c4.y = fmaf(ws, v.y, c4.y); c4.z = fmaf(ws, v.z, c4.z); c4.w = fmaf(ws, v.w, c4.w);
+          }
+        }
       }
     }
-    const float inv = 1.f / wl[head];
-    float4 r;
-    r.x = ((acc[0].x + acc[1].x) + (acc[2].x + acc[3].x)) * inv;
-    r.y = ((acc[0].y + acc[1].y) + (acc[2].y + acc[3].y)) * inv;
-    r.z = ((acc[0].z + acc[1].z) + (acc[2].z + acc[3].z)) * inv;
-    r.w = ((acc[0].w + acc[1].w) + (acc[2].w + acc[3].w)) * inv;
-    reinterpret_cast<float4*>(a.out + ((long long)(b * a.H_kv + h) * a.G + head) * 128)[d4] = r;
+  }
+#pragma unroll
+  for (int it = 0; it < kItems; ++it) {
+    const int i = tid + it * kDecThreads;
+    if (i < a.G * 32) {
+      const int head = i >> 5, d4 = i & 31;
+      const float inv = 1.f / wl[head];
+      const float4* c4 = acc[it];
+      float4 r;
+      r.x = ((c4[0].x + c4[1].x) + (c4[2].x + c4[3].x)) * inv;
+      r.y = ((c4[0].y + c4[1].y) + (c4[2].y + c4[3].y)) * inv;
+      r.z = ((c4[0].z + c4[1].z) + (c4[2].z + c4[3].z)) * inv;
+      r.w = ((c4[0].w + c4[1].w) + (c4[2].w + c4[3].w)) * inv;
+      reinterpret_cast<float4*>(a.out + ((long long)(b * a.H_kv + h) * a.G + head) * 128)[d4] = r;
+    }
   }
 }
 
