@@ -44,7 +44,7 @@ NCU_TRAFFIC_BYTES = {
     ("llama8b_128k", "stream_kernel<score>"): 270997248 + 8295936,
     ("llama8b_128k", "append_kernel"): 254738688 + 203578368,
     ("llama8b_128k", "select_kernel"): 17701632,
-    ("llama8b_128k", "decode_split_kernel"): 261801472 + 3964160,
+    ("llama8b_128k", "decode_split_kernel"): 252766464 + 4244480,
 }
 
 

@@ -112,17 +112,13 @@ decode_split_kernel(const __grid_constant__ CUtensorMap map_k,    // cache K: (d
   const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, c = lane & 3;
-  const int e_begin = (int)((long long)split * a.len / a.n_split);
-  const int n_rows = (int)((long long)(split + 1) * a.len / a.n_split) - e_begin;
-  const int n_tiles = (n_rows + kDecTile - 1) / kDecTile;
-
-  if (tid == 0) {
-    for (int s = 0; s < kDecStages; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), kDecWarps); }
-    mbar_init(sm_bars + 8u * (2 * kDecStages), 1);                 // the merge's bulk copies
-    fence_mbar_init();
-  }
-  if (tid == kDecWarps * 32) { tma_prefetch_desc(&map_k); tma_prefetch_desc(&map_v); }
-  __syncthreads();
+  // splits are whole tiles (the host launches at most one split per tile): no CTA reads rows of
+  // its neighbour, and only the cache's last tile is partial
+  const int tiles_total = (a.len + kDecTile - 1) / kDecTile;
+  const int tile_begin = (int)((long long)split * tiles_total / a.n_split);
+  const int n_tiles = (int)((long long)(split + 1) * tiles_total / a.n_split) - tile_begin;
+  const int e_begin = tile_begin * kDecTile;
+  const int n_rows = min(a.len - e_begin, n_tiles * kDecTile);
 
   float o[8][4];                 // O^T, eight 16-dim row blocks
   float m_a = -INFINITY, m_b = -INFINITY, l_a = 0.f, l_b = 0.f;   // heads 2c and 2c+1
@@ -132,21 +128,33 @@ decode_split_kernel(const __grid_constant__ CUtensorMap map_k,    // cache K: (d
     for (int i = 0; i < 4; ++i) o[mt][i] = 0.f;
 
   if (warp == kDecWarps) {
-    // ---- producer: one lane keeps the ring full -------------------------------------------------
+    // ---- producer: one lane sets the barriers up and keeps the ring full --------------------------
+    auto issue = [&](int t) {
+      const int st = t % kDecStages;
+      const uint32_t dst = base + st * kDecStageBytes;
+      const int row0 = e_begin + t * kDecTile;
+      mbar_expect_tx(bar_full(st), kDecStageBytes);
+      tma_load_4d(dst, &map_k, bar_full(st), 0, row0, h, b);
+      tma_load_4d(dst + kDecBoxBytes, &map_k, bar_full(st), 64, row0, h, b);
+      tma_load_4d(dst + 2 * kDecBoxBytes, &map_v, bar_full(st), 0, row0, h, b);
+      tma_load_4d(dst + 3 * kDecBoxBytes, &map_v, bar_full(st), 64, row0, h, b);
+    };
     if (lane == 0) {
-      for (int t = 0; t < n_tiles; ++t) {
-        const int st = t % kDecStages;
-        if (t >= kDecStages && !mbar_wait(bar_empty(st), (uint32_t)(t / kDecStages - 1) & 1u)) {
+      for (int s = 0; s < kDecStages; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), kDecWarps); }
+      mbar_init(sm_bars + 8u * (2 * kDecStages), 1);               // the merge's bulk copies
+      fence_mbar_init();
+      // the first tiles are on their way before the other warps have seen the barriers
+      for (int t = 0; t < min(n_tiles, kDecStages); ++t) issue(t);
+    }
+    __syncwarp();
+    __syncthreads();                                               // the barriers are set up
+    if (lane == 0) {
+      for (int t = kDecStages; t < n_tiles; ++t) {
+        if (!mbar_wait(bar_empty(t % kDecStages), (uint32_t)(t / kDecStages - 1) & 1u)) {
           record_status(a.status, kStatusTimeout);
           break;
         }
-        const uint32_t dst = base + st * kDecStageBytes;
-        const int row0 = e_begin + t * kDecTile;
-        mbar_expect_tx(bar_full(st), kDecStageBytes);
-        tma_load_4d(dst, &map_k, bar_full(st), 0, row0, h, b);
-        tma_load_4d(dst + kDecBoxBytes, &map_k, bar_full(st), 64, row0, h, b);
-        tma_load_4d(dst + 2 * kDecBoxBytes, &map_v, bar_full(st), 0, row0, h, b);
-        tma_load_4d(dst + 3 * kDecBoxBytes, &map_v, bar_full(st), 64, row0, h, b);
+        issue(t);
       }
     }
   } else {
@@ -161,6 +169,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap map_k,    // cache K: (d
         qb[ks][1] = g < a.G ? *reinterpret_cast<const uint32_t*>(qrow + 16 * ks + 8 + 2 * c) : 0u;
       }
     }
+    __syncthreads();                                               // the barriers are set up
     for (int t = 0; t < n_tiles; ++t) {
       const int st = t % kDecStages;
       if (!__all_sync(0xffffffffu, mbar_wait(bar_full(st), (uint32_t)(t / kDecStages) & 1u))) {   // warp-uniform
@@ -181,7 +190,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap map_k,    // cache K: (d
           mma_bf16(s0, k0, qb[ks][0], qb[ks][1]);
           mma_bf16(s1, k1, qb[ks + 1][0], qb[ks + 1][1]);
         }
-        // rows past the split's end belong to the next split (or read as zeros): weight 0
+        // rows past the cache's end read as zeros: weight 0
         const bool v_lo = key0 + g < n_rows, v_hi = key0 + g + 8 < n_rows;
         const float x0 = v_lo ? (s0[0] + s1[0]) * a.scale_log2e : -INFINITY;   // key g,   head 2c
         const float x1 = v_lo ? (s0[1] + s1[1]) * a.scale_log2e : -INFINITY;   // key g,   head 2c+1
