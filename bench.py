@@ -194,12 +194,18 @@ def time_oracle(w, steps, warmup, budget_s=20.0):
 def run_reference(args, w, rank, world):
     if rank != 0:
         return
+    from oracle import laser_kv_oracle as O
     value, dt, cores, sample, steps = time_oracle(w, max(1, min(args.steps, 40)), min(args.warmup, 3), budget_s=120.0)
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
         "warmup": min(args.warmup, 3), "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": w.name, "context_len": w.context_len, "block_size": w.block_size,
+                   "blocks_per_call": w.n_blocks, "batch": w.batch, "n_q_heads": w.n_q_heads,
+                   "n_kv_heads": w.n_kv_heads, "window": w.window, "lsh_bits": w.lsh_bits,
+                   "lsh_tables": w.lsh_tables, "protection_divisor": w.protection_divisor,
+                   "budget_per_block": O.budget(w.context_len, w.block_size, w.ratio), "alpha": w.alpha,
+                   "lookback": False,
                    "note": "CPU oracle (numpy fp64) timed on the host cores; bounded sample per step"},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
