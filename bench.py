@@ -39,11 +39,11 @@ UNIT = "tokens/s"
 # summary of the select call, keyed by (workload, kernel). A missing key means: not captured for
 # this workload, or the kernel has changed since the capture.
 NCU_TRAFFIC_BYTES = {
-    ("llama8b_128k", "stream_kernel<proj>"): 274882816 + 7054848,
-    ("llama8b_128k", "stream_kernel<lse>"): 269269248 + 4089600,
-    ("llama8b_128k", "stream_kernel<score>"): 270997248 + 8295936,
-    ("llama8b_128k", "append_kernel"): 254738688 + 203578368,
-    ("llama8b_128k", "select_kernel"): 17701632,
+    ("llama8b_128k", "stream_kernel<proj>"): 274973952 + 7255808,
+    ("llama8b_128k", "stream_kernel<lse>"): 269278464 + 4002816,
+    ("llama8b_128k", "stream_kernel<score>"): 270919424 + 8417280,
+    ("llama8b_128k", "append_kernel"): 254745600 + 203824640,
+    ("llama8b_128k", "select_kernel"): 17701376,
     ("llama8b_128k", "decode_split_kernel"): 252766464 + 4244480,
 }
 

@@ -196,13 +196,13 @@ __device__ __forceinline__ uint32_t proj_tables(uint32_t t_acc, uint32_t bar_rel
                                                 const StreamArgs& a, int seg, int key, int table0, int t_begin,
                                                 bool valid) {
   constexpr int NC = NT * KBITS;                               // columns of this thread
-  constexpr int LD = (NC & -NC) < 32 ? (NC & -NC) : 32;        // load width: a power of two that divides NC
   constexpr uint32_t bucket_mask = (1u << KBITS) - 1u;
   uint32_t v[NC];
   uint32_t v16[16];
   const uint32_t t_col = t_acc + t_begin * KBITS;
 #pragma unroll
-  for (int j = 0; j < NC / LD; ++j) tmem_ld_cols<LD>(t_col + j * LD, v + j * LD);
+  for (int j = 0; j < NC / 32; ++j) tmem_ld_x32(t_col + 32 * j, v + 32 * j);
+  if constexpr (NC % 32 != 0) tmem_ld_cols<NC % 32>(t_col + (NC / 32) * 32, v + (NC / 32) * 32);
   tmem_ld_x16(t_acc, v16);
   tmem_wait_ld();
   reg_fence<NC>(v);
