@@ -303,6 +303,22 @@ cudaError_t launch_stream(const CUtensorMap& mk, const CUtensorMap& ms, const St
   static std::atomic<unsigned long long> limit_set{0};   // per instantiation
   const cudaError_t e = ensure_smem_limit(limit_set, stream_kernel<MODE, KB, TCv>, kMaxSmem);
   if (e != cudaSuccess) return e;
+  if (a.overlap_prev) {
+    // may start while the kernel before it in the stream, whose results it does not read, still runs
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kStreamThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t le = cudaLaunchKernelEx(&cfg, stream_kernel<MODE, KB, TCv>, mk, ms, a);
+    g_launches.fetch_add(1);
+    return le != cudaSuccess ? le : cudaGetLastError();
+  }
   stream_kernel<MODE, KB, TCv><<<grid, kStreamThreads, smem, st>>>(mk, ms, a);
   g_launches.fetch_add(1);
   return cudaGetLastError();
@@ -654,7 +670,8 @@ laser_kv_status_t run_select(laser_kv_ctx* h, int layer, const void* K_blk, cons
       QsigArgs qa{static_cast<const uint16_t*>(Q_win), q_strides[0], q_strides[1], q_strides[2], h->P, hist, qb,
                   c.n_kv_heads, d.G, d.Wp, d.GWp, q_alloc, d.Lp,
                   reinterpret_cast<uint4*>(counts), ((long long)nseg * S_len + 3) / 4, ctrl + 1, fix_counts, nseg, ctrl,
-                  c.lsh_tables, part * d.Wp, part * d.GWp, d.GW, part == 0 ? 1 : 0};
+                  c.lsh_tables, part * d.Wp, part * d.GWp, d.GW, part == 0 ? 1 : 0,
+                  (need_exact && !h->profiling) ? 1 : 0};
       dim3 grid(d.Lp / kQsigTables, c.n_kv_heads, c.batch);
       LKV_CUDA(launch_qsig(d.Kp, mapQ, h->mapPq, qa, grid, qsig_smem_bytes(q_alloc, d.Kp), st), "qsig_kernel");
     }
@@ -683,6 +700,8 @@ laser_kv_status_t run_select(laser_kv_ctx* h, int layer, const void* K_blk, cons
     a1.stat_rows = d.GWp;
     a1.stat_rows_alloc = ((d.GWp + 127) / 128) * 128;
     const uint32_t smem = stream_smem_bytes(kLse, a1.stat_rows_alloc, 0);
+    a1.overlap_prev = (need_lsh && !h->profiling) ? 1 : 0;      // beside the query-signature kernel
+    a1.release_next = h->profiling ? 0 : 1;                       // the score pass sets itself up meanwhile
     LKV_CUDA((launch_stream<kLse, 0, 0>(mapK, mapQ, a1, base_ctas, smem, st)), "lse pass");
   }
   mark();
@@ -692,6 +711,10 @@ laser_kv_status_t run_select(laser_kv_ctx* h, int layer, const void* K_blk, cons
     a2.stat_rows = d.GWp;
     a2.stat_rows_alloc = d.GWp;
     const uint32_t smem = stream_smem_bytes(kScore, a2.stat_rows_alloc, 0);
+    // the projection pass reads nothing the score pass writes: it takes each SM as the score pass leaves it
+    const bool proj_beside = need_lsh && !h->profiling;
+    a2.release_next = (proj_beside && d.n_qparts == 1) ? 1 : 0;
+    a2.overlap_prev = h->profiling ? 0 : 1;
     LKV_CUDA((launch_stream<kScore, 0, 0>(mapK, mapQ, a2, base_ctas, smem, st)), "score pass");
     // the remaining parts of a window wider than a pass: their probabilities add to the first part's
     for (int part = 1; part < d.n_qparts; ++part) {
@@ -702,6 +725,10 @@ laser_kv_status_t run_select(laser_kv_ctx* h, int layer, const void* K_blk, cons
       b1.stat_rows_alloc = ((d.GWp + 127) / 128) * 128;
       b2.stat_rows_alloc = d.GWp;
       b2.accumulate = 1;
+      b2.release_next = (proj_beside && part == d.n_qparts - 1) ? 1 : 0;
+      b1.overlap_prev = 0;                                        // follows a score pass: launched the ordinary way
+      b1.release_next = h->profiling ? 0 : 1;
+      b2.overlap_prev = h->profiling ? 0 : 1;
       LKV_CUDA((launch_stream<kLse, 0, 0>(mapK, mapQ, b1, base_ctas, stream_smem_bytes(kLse, b1.stat_rows_alloc, 0), st)), "lse pass");
       LKV_CUDA((launch_stream<kScore, 0, 0>(mapK, mapQ, b2, base_ctas, smem, st)), "score pass");
     }
@@ -714,6 +741,7 @@ laser_kv_status_t run_select(laser_kv_ctx* h, int layer, const void* K_blk, cons
     a3.stat_rows_alloc = a3.stat_rows;
     a3.n_tiles = seg_tiles * d.n_chunks;
     const uint32_t smem = stream_smem_bytes(kProj, a3.stat_rows_alloc, d.TC * (2 << d.Kp));
+    a3.overlap_prev = (need_exact && !h->profiling) ? 1 : 0;     // beside the tail of the score pass
     LKV_CUDA(launch_proj(d.Kp, d.TC, mapK, h->mapP, a3, stream_grid(a3.n_tiles, h->num_sms), smem, st),
              "projection pass");
   }

@@ -23,6 +23,14 @@ __device__ __forceinline__ bool elect_one() {
   return pred != 0;
 }
 
+// ---- programmatic dependent launch ----------------------------------------------------------
+// A kernel launched with the programmatic-serialization attribute may start as soon as every CTA of
+// the kernel before it in the stream has called allow_dependents() (or has exited); it must not
+// rely on that kernel's results before grid_dependency_wait() has returned, which waits for that
+// kernel's completion and the visibility of its writes. Without the attribute both are no-ops.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void allow_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---- mbarrier -------------------------------------------------------------------------------
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));

@@ -41,6 +41,7 @@ struct QsigArgs {
   int q_row0, q_rows_total;   // qbuckets rows: [bh][q_rows_total][L], this pass starts at row q_row0
   int first_part;          // nonzero: clear the counts, restart the counters, store the histogram;
                            // zero: a later part of a wide window: add to the histogram
+  int release_next;        // nonzero: the next kernel in the stream was launched to start beside this one
 };
 
 // <x, y> over 128 bf16 elements in fp64 (every product is exact); 16-byte loads, all in flight at once.
@@ -84,6 +85,9 @@ qsig_kernel(const __grid_constant__ CUtensorMap map_q,    // Q: (d, W, H_q, batc
   constexpr uint32_t bucket_mask = nbins - 1u;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tg = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  // the log-sum-exp pass that follows needs nothing from this kernel: it may take the SMs this
+  // small grid leaves free (it waits for this kernel only before it ends)
+  if (a.release_next) allow_dependents();
   const int nmb = (a.GW + 127) / 128;
   const size_t bh = (size_t)b * a.H_kv + h;
 

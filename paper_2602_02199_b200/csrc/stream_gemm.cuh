@@ -96,6 +96,10 @@ struct StreamArgs {
   int fix_cap;             // items a segment's list can hold
   int* status;
   uint32_t polls, poll_ns;     // budget of the hand-off waits: polls, and nanoseconds a poll may suspend
+  int overlap_prev;    // launched to start beside the kernel before it: it waits for that kernel before it
+                       // ends, so that what follows in the stream follows both (kLse, kProj: they use none of
+                       // its results), and before its epilogue reads the normalisers (kScore after kLse)
+  int release_next;    // the kernel after this one was launched that way: let it take the SMs as they fall free
 };
 
 __device__ __forceinline__ void record_status(int* status, int code) {
@@ -649,6 +653,8 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // (a score pass that itself started early releases its successor only once it has waited: see below)
+  if (a.release_next && !(MODE == kScore && a.overlap_prev)) allow_dependents();
 
   if (warp == 0) {
     // ================= TMA producer =================
@@ -791,6 +797,14 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
     if constexpr (MODE == kLse) {
       ok = (nmb == 2) ? lse_epilogue<64>(a, e, nmb) : lse_epilogue<32>(a, e, nmb);
     } else if constexpr (MODE == kScore) {
+      // started beside the log-sum-exp pass: tiles are loaded and multiplied meanwhile, but the
+      // normalisers are read (and scores written) only once that pass has completed
+      // The projection pass that may follow beside this one needs the query histograms and the cleared
+      // counts of the kernel before the log-sum-exp pass, so it is released only after this wait.
+      if (a.overlap_prev) {
+        grid_dependency_wait();
+        if (a.release_next) allow_dependents();
+      }
       // group g sums the query columns [c0, c1); widths are multiples of 16, at most 64
       const int cw = ((a.GW + kEpiGroups - 1) / kEpiGroups + 15) & ~15;
       const int c0 = e.wg * cw;
@@ -822,6 +836,7 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
   // ---- teardown ----------------------------------------------------------------------------
   tc_fence_before();
   __syncthreads();
+  if (a.overlap_prev) grid_dependency_wait();
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, kTmemCols);
