@@ -149,6 +149,39 @@ def test_same_inputs_twice_give_identical_bytes():
         assert (to_np(a[:, :, :n]) == to_np(b[:, :, :n])).all()
 
 
+@pytest.mark.parametrize("debug", [0, 1])
+def test_back_to_back_calls_on_small_grids_repeat_bit_for_bit(debug):
+    """The log-sum-exp, score and projection kernels of a call start before the kernel ahead of them
+    has finished. On grids this small (a few CTAs per kernel) all of them are on the GPU at once, so
+    a kernel that read something too early would see it half written. Forty calls are queued without
+    a host synchronisation between them, alternating between two inputs; every call's appended rows
+    and positions must equal those of the same input run alone on a fresh handle."""
+    import torch
+    from paper_2602_02199_b200 import binding as Bn
+    for S, nb, hkv, G, W, K, L in ((264, 1, 2, 4, 32, 8, 16), (136, 3, 1, 7, 16, 10, 8), (1024, 2, 4, 2, 64, 6, 24)):
+        w = synth.workload("tiny").with_(name=f"b2b{S}", block_size=S, context_len=nb * S, n_q_heads=hkv * G, n_kv_heads=hkv,
+                                         window=W, lsh_bits=K, lsh_tables=L, needles="uniform:2")
+        ref = [run_workload_layer(w, layer, debug=debug) for layer in (0, 1)]
+        B, n = ref[0]["B"], nb * ref[0]["B"]
+        want = [[to_np(x[:, :, :n]).copy() for x in r["engine"].laser_kv_cache_view(0)[:3]] for r in ref]
+        cfg = Bn.make_config(n_layers=1, batch=w.batch, n_q_heads=w.n_q_heads, n_kv_heads=hkv, block_size=S, window=W,
+                             max_blocks=40 * nb, max_blocks_per_call=nb, lsh_bits=K, lsh_tables=L,
+                             protection_divisor=w.protection_divisor, budget_per_block=B, alpha=w.alpha, debug=debug)
+        eng = Bn.LaserKV(cfg, ref[0]["tP"])
+        for call in range(40):                               # queued back to back, no synchronisation
+            r = ref[call % 2]
+            eng.laser_kv_select_block(0, r["tK"], r["tV"], r["tQ"], nb)
+        eng.laser_kv_poll_status()
+        Kc, Vc, pc, m = eng.laser_kv_cache_view(0)
+        assert m == 40 * n
+        Kc, Vc, pc = to_np(Kc), to_np(Vc), to_np(pc)
+        for call in range(40):
+            sl = slice(call * n, (call + 1) * n)
+            wk, wv, wp = want[call % 2]
+            assert (Kc[:, :, sl] == wk).all() and (Vc[:, :, sl] == wv).all(), (S, call)
+            assert (pc[:, :, sl] - call * nb * S == wp).all(), (S, call)
+
+
 @pytest.mark.parametrize("alpha", [1.0, 0.0])
 def test_single_stage_policies_skip_the_unused_stage_and_keep_the_cache(alpha):
     # alpha = 1 (exact attention only) and alpha = 0 (LSH only): without the debug view the unused
