@@ -173,6 +173,10 @@ laser_kv_status_t laser_kv_init(const laser_kv_config_t* cfg, const void* hyperp
  * of a sequence is a pass of its own).
  * A handle's workspace serves one call at a time: calls on the same handle must be issued to one
  * stream (or be ordered by the caller); concurrent streams need one handle each.
+ * Inside a call some kernels are launched so that they may start before the kernel ahead of them
+ * has drained (programmatic stream serialization, where a kernel does not read that kernel's
+ * results). Towards everything else on the stream the call behaves as ordinary launches do: its
+ * first kernel starts after all earlier work, and work queued after the call starts after all of it.
  * Errors: CAPACITY if the cache cannot take n_blocks more blocks or n_blocks exceeds
  * max_blocks_per_call (nothing is launched). */
 laser_kv_status_t laser_kv_select_block(laser_kv_handle_t h, int32_t layer, const void* K_blk,
