@@ -56,7 +56,7 @@ struct Derived {
 };
 
 struct Carve {
-  size_t ctrl, dec_count, hist, qbuckets, lse_part, lse2, s_exact, counts, idx, fix_counts, fix_items, key_buckets, padP, total;
+  size_t ctrl, dec_count, hist, qbuckets, lse_part, lse_flags, lse2, s_exact, counts, idx, fix_counts, fix_items, key_buckets, padP, total;
 };
 
 size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
@@ -102,6 +102,10 @@ struct laser_kv_ctx {
   bool log = false;                     // LASER_KV_LOG: one stderr line per call
   // optional per-kernel timing (events only; no device memory)
   bool profiling = false;
+  // ordering words of kernels that run beside each other: how far the query-signature kernel's
+  // completion counter (ctrl word 8, only grows) will have got once everything launched so far has
+  // run, and the value the next log-sum-exp pass writes into its flags (never 0, the flags' initial state)
+  uint32_t qsig_done_total = 0, lse_epoch = 0;
   std::vector<cudaEvent_t> ev_pool;
   std::vector<std::vector<cudaEvent_t>> ev_pending;
   float prof_ms[kProfKernels] = {0};
@@ -249,6 +253,7 @@ void carve_ws(const laser_kv_config_t* c, const Derived& d, Carve* v) {
   v->hist = take(bh * d.Lp * ((size_t)2 << d.Kp));
   v->qbuckets = take(bh * d.GW * d.Lp * 2);
   v->lse_part = take(lse_part_bytes_bound(nseg, d.GWp));
+  v->lse_flags = take(lse_part_bytes_bound(nseg, 1) / sizeof(float2) * sizeof(int));   // one word per (segment, slot)
   v->lse2 = take(nseg * d.GW * 4);
   v->s_exact = take(nseg * S * 4);
   v->counts = take(nseg * S * 4 + 16);     // cleared in 16-byte units
@@ -530,7 +535,8 @@ laser_kv_status_t laser_kv_init(const laser_kv_config_t* cfg, const void* hyperp
       return fail(nullptr, LASER_KV_ERR_CUDA, "%s", msg.c_str());
     }
   }
-  if ((e = cudaMemset(h->ws + v.ctrl, 0, v.hist - v.ctrl)) != cudaSuccess) {   // status words and decode counters
+  if ((e = cudaMemset(h->ws + v.ctrl, 0, v.hist - v.ctrl)) != cudaSuccess ||   // status words and decode counters
+      (e = cudaMemset(h->ws + v.lse_flags, 0, v.lse2 - v.lse_flags)) != cudaSuccess) {   // no partial is flagged yet
     delete h;
     return fail(nullptr, LASER_KV_ERR_CUDA, "init: cudaMemset: %s", cudaGetErrorString(e));
   }
@@ -605,6 +611,7 @@ laser_kv_status_t run_select(laser_kv_ctx* h, int layer, const void* K_blk, cons
   uint16_t* hist = reinterpret_cast<uint16_t*>(ws + h->carve.hist);
   uint16_t* qb = reinterpret_cast<uint16_t*>(ws + h->carve.qbuckets);
   float2* lse_part = reinterpret_cast<float2*>(ws + h->carve.lse_part);
+  int* lse_flags = reinterpret_cast<int*>(ws + h->carve.lse_flags);
   float* lse2 = reinterpret_cast<float*>(ws + h->carve.lse2);
   float* s_exact = reinterpret_cast<float*>(ws + h->carve.s_exact);
   uint32_t* counts = reinterpret_cast<uint32_t*>(ws + h->carve.counts);
@@ -671,9 +678,10 @@ laser_kv_status_t run_select(laser_kv_ctx* h, int layer, const void* K_blk, cons
                   c.n_kv_heads, d.G, d.Wp, d.GWp, q_alloc, d.Lp,
                   reinterpret_cast<uint4*>(counts), ((long long)nseg * S_len + 3) / 4, ctrl + 1, fix_counts, nseg, ctrl,
                   c.lsh_tables, part * d.Wp, part * d.GWp, d.GW, part == 0 ? 1 : 0,
-                  (need_exact && !h->profiling) ? 1 : 0};
+                  (need_exact && !h->profiling) ? 1 : 0, ctrl + 8};
       dim3 grid(d.Lp / kQsigTables, c.n_kv_heads, c.batch);
       LKV_CUDA(launch_qsig(d.Kp, mapQ, h->mapPq, qa, grid, qsig_smem_bytes(q_alloc, d.Kp), st), "qsig_kernel");
+      h->qsig_done_total += grid.x * grid.y * grid.z;
     }
   }
 
@@ -701,7 +709,12 @@ laser_kv_status_t run_select(laser_kv_ctx* h, int layer, const void* K_blk, cons
     a1.stat_rows_alloc = ((d.GWp + 127) / 128) * 128;
     const uint32_t smem = stream_smem_bytes(kLse, a1.stat_rows_alloc, 0);
     a1.overlap_prev = (need_lsh && !h->profiling) ? 1 : 0;      // beside the query-signature kernel
-    a1.release_next = h->profiling ? 0 : 1;                       // the score pass sets itself up meanwhile
+    a1.release_next = h->profiling ? 0 : 1;                       // the score pass starts as SMs fall free
+    if (!h->profiling) {
+      if (++h->lse_epoch == 0) h->lse_epoch = 1;
+      a1.lse_flags = lse_flags;
+      a1.lse_epoch = (int)h->lse_epoch;
+    }
     LKV_CUDA((launch_stream<kLse, 0, 0>(mapK, mapQ, a1, base_ctas, smem, st)), "lse pass");
   }
   mark();
@@ -715,6 +728,8 @@ laser_kv_status_t run_select(laser_kv_ctx* h, int layer, const void* K_blk, cons
     const bool proj_beside = need_lsh && !h->profiling;
     a2.release_next = (proj_beside && d.n_qparts == 1) ? 1 : 0;
     a2.overlap_prev = h->profiling ? 0 : 1;
+    if (!h->profiling) { a2.lse_flags = lse_flags; a2.lse_epoch = (int)h->lse_epoch; }
+    if (a2.release_next) { a2.gate_counter = ctrl + 8; a2.gate_target = (int)h->qsig_done_total; }
     LKV_CUDA((launch_stream<kScore, 0, 0>(mapK, mapQ, a2, base_ctas, smem, st)), "score pass");
     // the remaining parts of a window wider than a pass: their probabilities add to the first part's
     for (int part = 1; part < d.n_qparts; ++part) {
@@ -729,6 +744,12 @@ laser_kv_status_t run_select(laser_kv_ctx* h, int layer, const void* K_blk, cons
       b1.overlap_prev = 0;                                        // follows a score pass: launched the ordinary way
       b1.release_next = h->profiling ? 0 : 1;
       b2.overlap_prev = h->profiling ? 0 : 1;
+      if (!h->profiling) {
+        if (++h->lse_epoch == 0) h->lse_epoch = 1;
+        b1.lse_flags = b2.lse_flags = lse_flags;
+        b1.lse_epoch = b2.lse_epoch = (int)h->lse_epoch;
+      }
+      if (b2.release_next) { b2.gate_counter = ctrl + 8; b2.gate_target = (int)h->qsig_done_total; }
       LKV_CUDA((launch_stream<kLse, 0, 0>(mapK, mapQ, b1, base_ctas, stream_smem_bytes(kLse, b1.stat_rows_alloc, 0), st)), "lse pass");
       LKV_CUDA((launch_stream<kScore, 0, 0>(mapK, mapQ, b2, base_ctas, smem, st)), "score pass");
     }
@@ -742,6 +763,7 @@ laser_kv_status_t run_select(laser_kv_ctx* h, int layer, const void* K_blk, cons
     a3.n_tiles = seg_tiles * d.n_chunks;
     const uint32_t smem = stream_smem_bytes(kProj, a3.stat_rows_alloc, d.TC * (2 << d.Kp));
     a3.overlap_prev = (need_exact && !h->profiling) ? 1 : 0;     // beside the tail of the score pass
+    a3.end_wait = a3.overlap_prev;                                // the selection kernel follows both
     LKV_CUDA(launch_proj(d.Kp, d.TC, mapK, h->mapP, a3, stream_grid(a3.n_tiles, h->num_sms), smem, st),
              "projection pass");
   }

@@ -31,6 +31,35 @@ __device__ __forceinline__ bool elect_one() {
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void allow_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// Bounded waits on words in global memory that another kernel of the same stream writes: a counter
+// that only grows has reached `target` (signed difference, so it may wrap), or a flag equals `value`.
+// They order kernels that run beside each other. The kernel that writes has always started, and
+// never waits for the reader, before the reader is launched, so the waits end; the poll limit is a
+// backstop after which the caller records a timeout.
+__device__ __forceinline__ int ld_acquire_gpu(const int* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release_gpu(int* p, int v) {
+  asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ bool wait_counter_reached(const int* counter, int target, uint32_t max_polls) {
+  for (uint32_t n = 0; n < max_polls; ++n) {
+    if (ld_acquire_gpu(counter) - target >= 0) return true;
+    __nanosleep(100);
+  }
+  return false;
+}
+__device__ __forceinline__ bool wait_flag_equals(const int* flag, int value, uint32_t max_polls) {
+  for (uint32_t n = 0; n < max_polls; ++n) {
+    if (ld_acquire_gpu(flag) == value) return true;
+    __nanosleep(100);
+  }
+  return false;
+}
+constexpr uint32_t kMaxFlagPolls = 1u << 23;     // x 100 ns and more: about a second
+
 // ---- mbarrier -------------------------------------------------------------------------------
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));

@@ -42,6 +42,8 @@ struct QsigArgs {
   int first_part;          // nonzero: clear the counts, restart the counters, store the histogram;
                            // zero: a later part of a wide window: add to the histogram
   int release_next;        // nonzero: the next kernel in the stream was launched to start beside this one
+  int* done_counter;       // every CTA adds one when its results are written: the projection pass, which may
+                           // start while later kernels still run, is held back until all of them have
 };
 
 // <x, y> over 128 bf16 elements in fp64 (every product is exact); 16-byte loads, all in flight at once.
@@ -217,6 +219,13 @@ qsig_kernel(const __grid_constant__ CUtensorMap map_q,    // Q: (d, W, H_q, batc
   if (warp == 0) {
     tc_fence_after();
     tmem_dealloc(tmem_base, tmem_cols);
+  }
+  if (a.done_counter) {
+    __syncthreads();                                   // the CTA's histograms, codes and zeros are written ...
+    if (threadIdx.x == 0) {
+      __threadfence();                                 // ... and visible before the count goes up
+      atomicAdd(a.done_counter, 1);
+    }
   }
 }
 

@@ -96,10 +96,16 @@ struct StreamArgs {
   int fix_cap;             // items a segment's list can hold
   int* status;
   uint32_t polls, poll_ns;     // budget of the hand-off waits: polls, and nanoseconds a poll may suspend
-  int overlap_prev;    // launched to start beside the kernel before it: it waits for that kernel before it
-                       // ends, so that what follows in the stream follows both (kLse, kProj: they use none of
-                       // its results), and before its epilogue reads the normalisers (kScore after kLse)
+  int overlap_prev;    // launched (with the programmatic-serialization attribute) to start beside the kernel ahead
   int release_next;    // the kernel after this one was launched that way: let it take the SMs as they fall free
+  int end_wait;        // wait for the grid ahead before this kernel ends, so that what follows in the stream follows both
+  // Words in global memory that order kernels running beside each other without waiting for a whole
+  // grid (which, besides coupling every CTA to the slowest one, takes microseconds after the grid's
+  // last CTA has gone):
+  int* lse_flags;             // [seg][n_slot]: kLse writes lse_epoch when a segment's partial of a CTA is in place,
+  int lse_epoch;              //   kScore waits for the flags of the partials it is about to read (null: ordinary order)
+  const int* gate_counter;    // kScore: the count the query-signature kernel's CTAs add to (or null) ...
+  int gate_target;            // ... and its value when all are done: only then is the projection pass released
 };
 
 __device__ __forceinline__ void record_status(int* status, int code) {
@@ -349,9 +355,18 @@ __device__ __forceinline__ bool lse_epilogue(const StreamArgs& a, const EpiCtx& 
         if (o.x != -INFINITY) lt += o.y * ex2_approx(o.x - mx);
       }
       mbar_arrive(e.bar_xb);
-      if (q < a.GW) {
-        const int slot = (int)blockIdx.x - cta_of_tile((long long)r.c.seg * a.tiles_in_block, a.n_tiles, gridDim.x);
-        a.lse_part[((size_t)r.c.seg * a.n_slot + slot) * a.GW + q] = make_float2(mx, lt);
+      const int slot = (int)blockIdx.x - cta_of_tile((long long)r.c.seg * a.tiles_in_block, a.n_tiles, gridDim.x);
+      if (q < a.GW) a.lse_part[((size_t)r.c.seg * a.n_slot + slot) * a.GW + q] = make_float2(mx, lt);
+      if (a.lse_flags) {
+        // the score pass may be reading already: the partial's flag goes up once every thread of this
+        // column group has stored (and fenced) its entry
+        __threadfence();
+        mbar_arrive(e.bar_kn);
+        if (q == 0) {
+          if (!mbar_wait(e.bar_kn, (uint32_t)flushes & 1, a.polls, a.poll_ns)) return false;
+          __threadfence();
+          st_release_gpu(a.lse_flags + (size_t)r.c.seg * a.n_slot + slot, a.lse_epoch);
+        }
       }
     }
     ++flushes;
@@ -375,6 +390,14 @@ __device__ __forceinline__ bool score_epilogue(const StreamArgs& a, const EpiCtx
       const long long first = (long long)r.c.seg * a.tiles_in_block;
       const int cf = cta_of_tile(first, a.n_tiles, a.lse_ctas);
       const int n_used = cta_of_tile(first + a.tiles_in_block - 1, a.n_tiles, a.lse_ctas) - cf + 1;
+      if (a.lse_flags) {
+        // the log-sum-exp pass may still be running: wait for the flags of this segment's partials
+        bool ready = true;
+        if (e.lane < n_used)
+          ready = wait_flag_equals(a.lse_flags + (size_t)r.c.seg * a.n_slot + e.lane, a.lse_epoch,
+                                   a.poll_ns == 0 ? a.polls : kMaxFlagPolls);
+        if (!__all_sync(0xffffffffu, ready)) return false;
+      }
       __syncwarp();
 #pragma unroll
       for (int half = 0; half < (NC + 31) / 32; ++half) {
@@ -383,10 +406,10 @@ __device__ __forceinline__ bool score_epilogue(const StreamArgs& a, const EpiCtx
           const int qq = c0 + j;
           const float2* p = a.lse_part + (size_t)r.c.seg * a.n_slot * a.GW + qq;
           float mx = -INFINITY;
-          for (int s2 = 0; s2 < n_used; ++s2) mx = fmaxf(mx, p[(size_t)s2 * a.GW].x);
+          for (int s2 = 0; s2 < n_used; ++s2) mx = fmaxf(mx, __ldcg(p + (size_t)s2 * a.GW).x);
           float sum = 0.f;
           for (int s2 = 0; s2 < n_used; ++s2) {
-            const float2 pe = p[(size_t)s2 * a.GW];
+            const float2 pe = __ldcg(p + (size_t)s2 * a.GW);
             if (pe.x != -INFINITY) sum += pe.y * exp2f(pe.x - mx);
           }
           const float lse = mx + log2f(sum);
@@ -641,6 +664,7 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
     mbar_init(bar_stat, 1);
     mbar_init(bar_stat_free, kEpilogueThreads);
     if (MODE == kLse) {
+      mbar_init(bar_kn, nmb * 128);                      // column group 0 stored a segment's partial (flag hand-off)
       mbar_init(bar_xa, kEpilogueThreads - nmb * 128);   // column groups 1.. wrote their (max, sum)
       mbar_init(bar_xb, nmb * 128);                      // column group 0 merged them
     } else {
@@ -654,7 +678,16 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   // (a score pass that itself started early releases its successor only once it has waited: see below)
-  if (a.release_next && !(MODE == kScore && a.overlap_prev)) allow_dependents();
+  if (a.release_next) {
+    if (a.gate_counter == nullptr) {
+      allow_dependents();
+    } else if (threadIdx.x == 0) {
+      // the kernel to be released needs what the query-signature kernel wrote: its CTAs count themselves done
+      if (!wait_counter_reached(a.gate_counter, a.gate_target, a.poll_ns == 0 ? a.polls : kMaxFlagPolls))
+        record_status(a.status, kStatusTimeout);
+      allow_dependents();
+    }
+  }
 
   if (warp == 0) {
     // ================= TMA producer =================
@@ -797,14 +830,9 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
     if constexpr (MODE == kLse) {
       ok = (nmb == 2) ? lse_epilogue<64>(a, e, nmb) : lse_epilogue<32>(a, e, nmb);
     } else if constexpr (MODE == kScore) {
-      // started beside the log-sum-exp pass: tiles are loaded and multiplied meanwhile, but the
-      // normalisers are read (and scores written) only once that pass has completed
-      // The projection pass that may follow beside this one needs the query histograms and the cleared
-      // counts of the kernel before the log-sum-exp pass, so it is released only after this wait.
-      if (a.overlap_prev) {
-        grid_dependency_wait();
-        if (a.release_next) allow_dependents();
-      }
+      // started beside the log-sum-exp pass: tiles are loaded and multiplied meanwhile; the normalisers
+      // of a segment are read once their flags are up (or, without flags, once that grid has completed)
+      if (a.overlap_prev && a.lse_flags == nullptr) grid_dependency_wait();
       // group g sums the query columns [c0, c1); widths are multiples of 16, at most 64
       const int cw = ((a.GW + kEpiGroups - 1) / kEpiGroups + 15) & ~15;
       const int c0 = e.wg * cw;
@@ -836,7 +864,7 @@ stream_kernel(const __grid_constant__ CUtensorMap map_keys,   // K: (d, token, h
   // ---- teardown ----------------------------------------------------------------------------
   tc_fence_before();
   __syncthreads();
-  if (a.overlap_prev) grid_dependency_wait();
+  if (a.end_wait) grid_dependency_wait();
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, kTmemCols);
