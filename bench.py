@@ -39,11 +39,11 @@ UNIT = "tokens/s"
 # summary of the select call, keyed by (workload, kernel). A missing key means: not captured for
 # this workload, or the kernel has changed since the capture.
 NCU_TRAFFIC_BYTES = {
-    ("llama8b_128k", "stream_kernel<proj>"): 274761728 + 7632896,
-    ("llama8b_128k", "stream_kernel<lse>"): 269270784 + 4050432,
-    ("llama8b_128k", "stream_kernel<score>"): 271289600 + 10112512,
-    ("llama8b_128k", "append_kernel"): 254782976 + 203437824,
-    ("llama8b_128k", "select_kernel"): 17701376,
+    ("llama8b_128k", "stream_kernel<proj>"): 274964480 + 7900416,
+    ("llama8b_128k", "stream_kernel<lse>"): 269273344 + 4132096,
+    ("llama8b_128k", "stream_kernel<score>"): 270247936 + 6919168,
+    ("llama8b_128k", "append_kernel"): 254738688 + 203495168,
+    ("llama8b_128k", "select_kernel"): 17701888,
     ("llama8b_128k", "decode_split_kernel"): 252766464 + 4244480,
 }
 
